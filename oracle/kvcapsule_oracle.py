@@ -1,0 +1,213 @@
+"""KVCapsule CPU oracle -- TEST INFRASTRUCTURE, NOT THE PRODUCT PATH.
+
+A plain, slow, fp64 numpy statement of what the KVCapsule decode-time hot path
+computes, written from the paper (arxiv 2605.16439).  Only tests, the smoke
+check and the benchmark's CPU-baseline leg may import it.  It shares no code
+with the CUDA library and imports nothing from it.
+
+Two forms of the decode step are given:
+
+* Form 1 (`decode_attend_definition`) is the definition: reconstruct full-length
+  vision keys and values from the capsules (Sec. 3.1 "Selective Retention and
+  Reconstruction for Keys", "Sequence-Level Low-Rank Compression for Values"),
+  concatenate with the untouched text K/V (Sec. 3.2 "Decoding Stage") and run
+  the standard attention of Sec. 3.1's first equation.
+* Form 2 (`decode_attend_fused`) takes Algorithm 1's steps in the paper's order
+  and notation (scores in compressed space, expansion by theta, softmax,
+  re-projection by U^T, product with the compressed values plus the mu term).
+
+Readings of the paper taken here (each also listed in the design document):
+  - f_theta acts linearly along the token axis: K_hat = theta^T K_tilde with one
+    dense m x n matrix per KV head (Alg. 1 "MatMul(S_full, theta)" and App. D's
+    theta in R^{H_kv x m x n} are only consistent with that).
+  - the softmax runs jointly over all R*n reconstructed vision positions and
+    the T text positions of a query head (Sec. 3.2 "Decoding Stage").
+  - "rank R" of Alg. 1 = number of n-token vision blocks per sequence; theta, U,
+    mu and the retained index set are shared by all blocks and sequences.
+  - mu is a fixed per-(layer, KV head) vector (Sec. 3.2 first paragraph).
+  - "P mu" in Alg. 1 step 4 = (sum_i P_i) mu^T.
+  - compression ratio rho = 1 - l_r;  m = ceil(l_r n) in integer arithmetic on
+    rho expressed in permille.
+  - rho = 0 is a pass-through: capsules hold K and V verbatim.
+
+Parity pins: every function below is pinned by tests/test_oracle_pins.py
+(library attention, lossless constructions, Eckart-Young, closed forms, brute
+force, form 1 == form 2).  What is NOT pinned: behaviour with trained
+parameters (no trained parameters exist here) -- "parity unpinned" for that.
+
+Shapes (paper notation): q [B,H_q,d]; K_vis,V_vis [B,H_kv,R*n,d];
+idx [m] or [H_kv,m]; theta,U [H_kv,m,n]; mu [H_kv,d];
+K_tilde,V_tilde [B,H_kv,R,m,d]; K_txt,V_txt [B,H_kv,T,d]; out [B,H_q,d].
+"""
+from __future__ import annotations
+
+import numpy as np
+
+F64 = np.float64
+
+
+# --------------------------------------------------------------------------
+# integer maps (Sec. 3.1: |M_l| = ceil(l_r n);  Alg. 1: Reshape to [B,H_kv,G,R,m])
+# --------------------------------------------------------------------------
+def retained_len(n: int, ratio_permille: int) -> int:
+    """m = ceil(l_r * n) with l_r = 1 - rho, rho = ratio_permille / 1000, in integers."""
+    if n <= 0 or not (0 <= ratio_permille < 1000):
+        raise ValueError("need n > 0 and 0 <= ratio_permille < 1000")
+    return (n * (1000 - ratio_permille) + 999) // 1000
+
+
+def grouping_map(N_v: int, n: int) -> np.ndarray:
+    """Vision token t (cache order) -> (block r, offset i): t = r*n + i.  int32 [N_v,2]."""
+    if n <= 0 or N_v % n != 0:
+        raise ValueError("N_v must be a whole number of n-token blocks")
+    t = np.arange(N_v, dtype=np.int64)
+    return np.stack([t // n, t % n], axis=1).astype(np.int32)
+
+
+def _idx_for_head(idx: np.ndarray, h: int) -> np.ndarray:
+    idx = np.asarray(idx)
+    return idx[h] if idx.ndim == 2 else idx
+
+
+# --------------------------------------------------------------------------
+# standard attention (Sec. 3.1, first equation), single decode query, GQA
+# --------------------------------------------------------------------------
+def softmax(x: np.ndarray) -> np.ndarray:
+    x = np.asarray(x, F64)
+    e = np.exp(x - np.max(x))
+    return e / np.sum(e)
+
+
+def attention(q, K, V) -> np.ndarray:
+    """softmax(q K^T / sqrt(d)) V per query head; query head hq reads KV head hq // G."""
+    q, K, V = (np.asarray(a, F64) for a in (q, K, V))
+    B, H_q, d = q.shape
+    H_kv = K.shape[1]
+    G = H_q // H_kv
+    out = np.zeros((B, H_q, d), F64)
+    for b in range(B):
+        for hq in range(H_q):
+            h = hq // G
+            s = (K[b, h] @ q[b, hq]) / np.sqrt(F64(d))
+            out[b, hq] = softmax(s) @ V[b, h]
+    return out
+
+
+# --------------------------------------------------------------------------
+# prefill-stage compression (Sec. 3.2 "Prefilling Stage")
+# --------------------------------------------------------------------------
+def compress(K_vis, V_vis, idx, U, mu, n: int, passthrough: bool = False):
+    """K_tilde = rows idx of each block's keys; V_tilde = U (V - 1 mu^T) per block."""
+    K_vis, V_vis = np.asarray(K_vis, F64), np.asarray(V_vis, F64)
+    B, H_kv, N_v, d = K_vis.shape
+    if N_v % n != 0:
+        raise ValueError("N_v must be a whole number of n-token blocks")
+    R = N_v // n
+    if passthrough:
+        return (K_vis.reshape(B, H_kv, R, n, d).copy(), V_vis.reshape(B, H_kv, R, n, d).copy())
+    U, mu = np.asarray(U, F64), np.asarray(mu, F64)
+    m = U.shape[1]
+    K_t = np.zeros((B, H_kv, R, m, d), F64)
+    V_t = np.zeros((B, H_kv, R, m, d), F64)
+    for b in range(B):
+        for h in range(H_kv):
+            sel = _idx_for_head(idx, h)
+            for r in range(R):
+                K_blk = K_vis[b, h, r * n:(r + 1) * n]
+                V_blk = V_vis[b, h, r * n:(r + 1) * n]
+                K_t[b, h, r] = K_blk[sel]                       # row selection by M_l
+                V_center = V_blk - np.ones((n, 1), F64) * mu[h][None, :]
+                V_t[b, h, r] = U[h] @ V_center                  # sequence-level PCA projection
+    return K_t, V_t
+
+
+# --------------------------------------------------------------------------
+# decode-stage reconstruction (Sec. 3.2 "Decoding Stage")
+# --------------------------------------------------------------------------
+def reconstruct(K_t, V_t, theta, U, mu, passthrough: bool = False):
+    """K_hat = theta^T K_tilde,  V_hat = U^T V_tilde + 1 mu^T;  returns [B,H_kv,R*n,d] each."""
+    K_t, V_t = np.asarray(K_t, F64), np.asarray(V_t, F64)
+    B, H_kv, R, m, d = K_t.shape
+    if passthrough:
+        return K_t.reshape(B, H_kv, R * m, d).copy(), V_t.reshape(B, H_kv, R * m, d).copy()
+    theta, U, mu = np.asarray(theta, F64), np.asarray(U, F64), np.asarray(mu, F64)
+    n = theta.shape[2]
+    K_hat = np.zeros((B, H_kv, R * n, d), F64)
+    V_hat = np.zeros((B, H_kv, R * n, d), F64)
+    for b in range(B):
+        for h in range(H_kv):
+            for r in range(R):
+                K_hat[b, h, r * n:(r + 1) * n] = theta[h].T @ K_t[b, h, r]
+                V_hat[b, h, r * n:(r + 1) * n] = U[h].T @ V_t[b, h, r] + np.ones((n, 1), F64) * mu[h][None, :]
+    return K_hat, V_hat
+
+
+def decode_attend_definition(q, K_t, V_t, theta, U, mu, K_txt, V_txt, passthrough: bool = False):
+    """Form 1: reconstruct, concatenate with text K/V, run the original attention."""
+    K_hat, V_hat = reconstruct(K_t, V_t, theta, U, mu, passthrough)
+    K_all = np.concatenate([K_hat, np.asarray(K_txt, F64)], axis=2)
+    V_all = np.concatenate([V_hat, np.asarray(V_txt, F64)], axis=2)
+    return attention(q, K_all, V_all)
+
+
+# --------------------------------------------------------------------------
+# Algorithm 1 (fused KVCapsule), with the text tail in the same softmax
+# --------------------------------------------------------------------------
+def decode_attend_fused(q, K_t, V_t, theta, U, mu, K_txt, V_txt, passthrough: bool = False):
+    """Form 2: Alg. 1's four steps, text logits joined before the softmax."""
+    q, K_t, V_t = np.asarray(q, F64), np.asarray(K_t, F64), np.asarray(V_t, F64)
+    K_txt, V_txt = np.asarray(K_txt, F64), np.asarray(V_txt, F64)
+    B, H_q, d = q.shape
+    _, H_kv, R, m, _ = K_t.shape
+    G = H_q // H_kv
+    T = K_txt.shape[2]
+    sigma = 1.0 / np.sqrt(F64(d))
+    if passthrough:
+        n = m
+        theta = np.broadcast_to(np.eye(m, dtype=F64), (H_kv, m, m))
+        U = theta
+        mu = np.zeros((H_kv, d), F64)
+    else:
+        theta, U, mu = np.asarray(theta, F64), np.asarray(U, F64), np.asarray(mu, F64)
+        n = theta.shape[2]
+    Y = np.zeros((B, H_q, d), F64)
+    for b in range(B):
+        for h in range(H_kv):
+            Q_bh = q[b, h * G:(h + 1) * G]                                  # [G,d]
+            # Step 1: scores in compressed sequence space, shaped [G,R,m]
+            S_full = np.stack([Q_bh @ K_t[b, h, r].T for r in range(R)], axis=1) * sigma if R else np.zeros((G, 0, m))
+            # Step 2: expand to spatial resolution, softmax (jointly with the text logits)
+            L_img = S_full @ theta[h]                                       # [G,R,n]
+            L_txt = (Q_bh @ K_txt[b, h].T) * sigma                          # [G,T]
+            L_all = np.concatenate([L_img.reshape(G, R * n), L_txt], axis=1)
+            P_all = np.stack([softmax(L_all[g]) for g in range(G)], axis=0)
+            P = P_all[:, :R * n].reshape(G, R, n)
+            P_txt = P_all[:, R * n:]
+            # Step 3: associative re-projection with transposed U
+            W = P @ U[h].T                                                  # [G,R,m]
+            # Step 4: multiply with compressed values, add the P mu term and the text values
+            y = np.zeros((G, d), F64)
+            for r in range(R):
+                y += W[:, r, :] @ V_t[b, h, r]
+            y += P.sum(axis=(1, 2))[:, None] * mu[h][None, :]
+            y += P_txt @ V_txt[b, h]
+            Y[b, h * G:(h + 1) * G] = y
+    return Y
+
+
+# --------------------------------------------------------------------------
+# persistent-memory footprint of one layer (App. D, Eqs. 1-2)
+# --------------------------------------------------------------------------
+def footprint_base(B, H_kv, c, n_vis, t, d, b_kv) -> int:
+    """Eq. 1: 2 B H_kv (c + n + t) d b_kv."""
+    return 2 * B * H_kv * (c + n_vis + t) * d * b_kv
+
+
+def footprint_kvcapsule(B, H_kv, c, n, R, t, d, b_kv, ratio_permille, b_param=None) -> int:
+    """Eq. 2 with R blocks of n tokens: compressed cache + S_recon(theta) + S_PCA(U, mu)."""
+    b_param = b_kv if b_param is None else b_param
+    m = retained_len(n, ratio_permille)
+    cache = 2 * B * H_kv * (c + R * m + t) * d * b_kv
+    s_recon = H_kv * m * n * b_param
+    s_pca = H_kv * m * n * b_param + H_kv * d * b_param
+    return cache + s_recon + s_pca

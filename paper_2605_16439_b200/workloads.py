@@ -1,0 +1,173 @@
+"""Seeded synthetic inputs for the KVCapsule decode path.
+
+This module only draws random tensors; it holds none of the method's arithmetic
+(the retained length m is passed in by the caller).  The same generated buffers
+are handed to the CPU oracle and to the CUDA library, so neither depends on the
+other.  Everything is produced with torch ops so that the benchmark can draw
+full-size workloads directly in device memory; parity tests draw on the CPU.
+
+Recipe (stands in for the vision/text activations of LLaVA-NeXT / Qwen2-VL /
+InternVL3-shaped models, which are not available offline):
+  * vision K and V, independently per (sequence, KV head, block, channel):
+    N(0,1) field on the block's g x g patch grid, 3x3 box filter over the grid
+    (mean over the in-grid neighbours at the border), plus 0.1 * N(0,1) noise;
+    tokens in row-major grid order.
+  * video: consecutive blocks are frames of an AR(1) process with coefficient
+    rho_t: x_0 = e_0, x_f = rho_t x_{f-1} + sqrt(1 - rho_t^2) e_f, each e_f a
+    smoothed field as above.
+  * text K/V and the decode query: N(0,1).
+  * parameters theta, U [H_kv,m,n] and mu [H_kv,d]: N(0, 1/d).
+  * retained indices: evenly spaced, idx[j] = floor(j n / m); or a sorted seeded
+    random subset (irregular gathers).
+bf16 workloads are rounded to bf16 once, here, and both sides start from the
+rounded values.
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+
+import torch
+
+
+@dataclasses.dataclass(frozen=True)
+class Shape:
+    """One workload shape (paper notation)."""
+    name: str
+    layers: int
+    B: int
+    H_q: int
+    H_kv: int
+    d: int
+    grid: int          # g: block = g x g patch grid, n = g*g
+    R: int             # vision blocks per sequence
+    T0: int            # text tokens at the first decode step
+    steps: int         # decode steps
+    dtype: str         # "f32" | "bf16"
+    ratio_permille: int = 600
+    ar1: float = 0.0   # temporal AR(1) coefficient across blocks (video)
+
+    @property
+    def n(self) -> int:
+        return self.grid * self.grid
+
+    @property
+    def G(self) -> int:
+        return self.H_q // self.H_kv
+
+    @property
+    def N_v(self) -> int:
+        return self.R * self.n
+
+
+# The five configurations of the benchmark spec (index = config number).
+CONFIGS = (
+    Shape("config0-single-layer-fp32", 1, 1, 8, 2, 128, 24, 1, 32, 1, "f32"),
+    Shape("config1-llava-next-7b", 32, 8, 32, 32, 128, 24, 5, 128, 256, "bf16"),
+    Shape("config2-qwen2-vl-7b", 28, 16, 28, 4, 128, 32, 8, 256, 512, "bf16"),
+    Shape("config3-internvl3-8b-video", 28, 4, 28, 4, 128, 16, 32, 512, 1024, "bf16", ar1=0.9),
+)
+
+
+def torch_dtype(name: str) -> torch.dtype:
+    return {"f32": torch.float32, "bf16": torch.bfloat16}[name]
+
+
+def _gen(seed: int, device) -> torch.Generator:
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed))
+    return g
+
+
+def smoothed_field(lead: tuple, grid: int, d: int, gen: torch.Generator, device) -> torch.Tensor:
+    """[*lead, grid*grid, d] fp32: box-filtered Gaussian field per channel plus 0.1 noise."""
+    n = grid * grid
+    numel_lead = int(math.prod(lead)) if lead else 1
+    base = torch.randn((numel_lead * d, 1, grid, grid), generator=gen, device=device, dtype=torch.float32)
+    sm = torch.nn.functional.avg_pool2d(base, 3, stride=1, padding=1, count_include_pad=False)
+    del base
+    sm = sm.reshape(numel_lead, d, n).transpose(1, 2)          # token-major, channel-minor
+    noise = torch.randn((numel_lead, n, d), generator=gen, device=device, dtype=torch.float32)
+    out = sm + 0.1 * noise
+    return out.reshape(*lead, n, d).contiguous()
+
+
+def vision_kv(B: int, H_kv: int, R: int, grid: int, d: int, seed: int, device="cpu",
+              dtype=torch.float32, ar1: float = 0.0) -> torch.Tensor:
+    """One of K_vis / V_vis: [B, H_kv, R*n, d]."""
+    gen = _gen(seed, device)
+    n = grid * grid
+    if ar1 == 0.0:
+        x = smoothed_field((B, H_kv, R), grid, d, gen, device)
+    else:
+        x = torch.empty((B, H_kv, R, n, d), device=device, dtype=torch.float32)
+        prev = None
+        for f in range(R):
+            e = smoothed_field((B, H_kv), grid, d, gen, device)
+            prev = e if prev is None else ar1 * prev + math.sqrt(1.0 - ar1 * ar1) * e
+            x[:, :, f] = prev
+    return x.reshape(B, H_kv, R * n, d).to(dtype).contiguous()
+
+
+def gaussian(shape: tuple, seed: int, device="cpu", dtype=torch.float32, std: float = 1.0) -> torch.Tensor:
+    gen = _gen(seed, device)
+    return (torch.randn(shape, generator=gen, device=device, dtype=torch.float32) * std).to(dtype).contiguous()
+
+
+def params(H_kv: int, m: int, n: int, d: int, seed: int, device="cpu", dtype=torch.float32):
+    """(theta, U, mu) ~ N(0, 1/d) in the shapes of App. D."""
+    std = 1.0 / math.sqrt(d)
+    theta = gaussian((H_kv, m, n), seed * 7 + 1, device, dtype, std)
+    U = gaussian((H_kv, m, n), seed * 7 + 2, device, dtype, std)
+    mu = gaussian((H_kv, d), seed * 7 + 3, device, dtype, std)
+    return theta, U, mu
+
+
+def evenly_spaced_idx(n: int, m: int) -> torch.Tensor:
+    """idx[j] = floor(j n / m), strictly increasing for m <= n; int32 [m]."""
+    j = torch.arange(m, dtype=torch.int64)
+    return ((j * n) // m).to(torch.int32)
+
+
+def random_sorted_idx(n: int, m: int, seed: int, H_kv: int = 0) -> torch.Tensor:
+    """Sorted random m-subset of 0..n-1; [m] if H_kv == 0 else one subset per KV head [H_kv, m]."""
+    gen = _gen(seed, "cpu")
+    rows = max(H_kv, 1)
+    out = torch.stack([torch.sort(torch.randperm(n, generator=gen)[:m]).values for _ in range(rows)])
+    out = out.to(torch.int32)
+    return out if H_kv else out[0]
+
+
+def layer_seed(config_index: int, layer: int) -> int:
+    return 1000 * config_index + layer
+
+
+def decode_inputs(shape: Shape, m: int, seed: int, device="cpu", T: int | None = None,
+                  T_cap: int | None = None):
+    """All tensors of one layer's decode problem, in the storage dtype of `shape`.
+
+    Returns a dict: K_vis, V_vis [B,H_kv,N_v,d]; K_txt, V_txt [B,H_kv,T_cap,d] (rows >= T are
+    filled too, they must not influence the result); q [B,H_q,d]; theta, U, mu; idx [m].
+    """
+    dt = torch_dtype(shape.dtype)
+    T = shape.T0 if T is None else T
+    T_cap = T if T_cap is None else T_cap
+    s = seed * 16
+    theta, U, mu = params(shape.H_kv, m, shape.n, shape.d, s + 5, device, dt)
+    return dict(
+        K_vis=vision_kv(shape.B, shape.H_kv, shape.R, shape.grid, shape.d, s + 0, device, dt, shape.ar1),
+        V_vis=vision_kv(shape.B, shape.H_kv, shape.R, shape.grid, shape.d, s + 1, device, dt, shape.ar1),
+        K_txt=gaussian((shape.B, shape.H_kv, T_cap, shape.d), s + 2, device, dt),
+        V_txt=gaussian((shape.B, shape.H_kv, T_cap, shape.d), s + 3, device, dt),
+        q=gaussian((shape.B, shape.H_q, shape.d), s + 4, device, dt),
+        theta=theta, U=U, mu=mu,
+        idx=evenly_spaced_idx(shape.n, m),
+        T=T, T_cap=T_cap,
+    )
+
+
+def shard_batch(B_total: int, rank: int, world: int) -> tuple[int, int]:
+    """Contiguous slice [lo, hi) of the sequences owned by `rank` (no data-path exchange)."""
+    base, rem = divmod(B_total, world)
+    lo = rank * base + min(rank, rem)
+    return lo, lo + base + (1 if rank < rem else 0)

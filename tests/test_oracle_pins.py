@@ -1,0 +1,319 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+None of these tests touches the CUDA library.  Each pin is chosen so that a
+plausible slip in the oracle (dropped mu term, wrong sign, wrong index set,
+transposed operand, wrong GQA head map, missing 1/sqrt(d), separate instead of
+joint softmax, wrong block order) fails at least one of them.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import kvcapsule_oracle as orc
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rng(seed):
+    return np.random.default_rng(seed)
+
+
+def _library_attention(q, K, V):
+    """torch's fp64 scaled-dot-product attention as an independent library routine."""
+    B, H_q, d = q.shape
+    G = H_q // K.shape[1]
+    qt = torch.from_numpy(np.ascontiguousarray(q)).reshape(B, H_q, 1, d)
+    Kt = torch.from_numpy(np.ascontiguousarray(K)).repeat_interleave(G, dim=1)
+    Vt = torch.from_numpy(np.ascontiguousarray(V)).repeat_interleave(G, dim=1)
+    out = torch.nn.functional.scaled_dot_product_attention(qt, Kt, Vt)
+    return out.reshape(B, H_q, d).numpy()
+
+
+def _problem(seed, B=2, H_q=6, H_kv=2, d=8, n=12, m=5, R=3, T=4):
+    r = _rng(seed)
+    return dict(
+        q=r.standard_normal((B, H_q, d)),
+        K_vis=r.standard_normal((B, H_kv, R * n, d)),
+        V_vis=r.standard_normal((B, H_kv, R * n, d)),
+        K_txt=r.standard_normal((B, H_kv, T, d)),
+        V_txt=r.standard_normal((B, H_kv, T, d)),
+        theta=r.standard_normal((H_kv, m, n)) / math.sqrt(d),
+        U=r.standard_normal((H_kv, m, n)) / math.sqrt(d),
+        mu=r.standard_normal((H_kv, d)),
+        idx=np.sort(r.permutation(n)[:m]).astype(np.int32),
+        n=n, m=m, R=R, T=T,
+    )
+
+
+# ---------------------------------------------------------------- integer maps
+def test_retained_len_table():
+    # m = ceil((1 - rho) n), Sec. 3.1; the values used by every configuration
+    assert orc.retained_len(576, 600) == 231
+    assert orc.retained_len(1024, 600) == 410
+    assert orc.retained_len(256, 600) == 103
+    assert [orc.retained_len(1024, r) for r in (0, 200, 400, 600, 800)] == [1024, 820, 615, 410, 205]
+    for n in (1, 7, 576, 1000, 1024):
+        for r in (0, 1, 333, 500, 950, 999):
+            m = orc.retained_len(n, r)
+            assert m == math.ceil(n * (1000 - r) / 1000)          # exact rational ceil
+            assert 1 <= m <= n
+    with pytest.raises(ValueError):
+        orc.retained_len(16, 1000)
+
+
+def test_grouping_map_is_block_decomposition():
+    g = orc.grouping_map(3 * 7, 7)
+    assert g.dtype == np.int32 and g.shape == (21, 2)
+    for t in range(21):
+        assert g[t, 0] * 7 + g[t, 1] == t and 0 <= g[t, 1] < 7
+    with pytest.raises(ValueError):
+        orc.grouping_map(20, 7)
+
+
+# ---------------------------------------------------------------- attention vs a library
+@pytest.mark.parametrize("seed", [0, 1])
+def test_attention_matches_library_routine(seed):
+    r = _rng(seed)
+    q = r.standard_normal((2, 6, 16))
+    K = r.standard_normal((2, 3, 37, 16))
+    V = r.standard_normal((2, 3, 37, 16))
+    np.testing.assert_allclose(orc.attention(q, K, V), _library_attention(q, K, V), atol=1e-13)
+
+
+def test_softmax_invariants():
+    r = _rng(3)
+    x = r.standard_normal(50) * 5
+    p = orc.softmax(x)
+    assert abs(p.sum() - 1.0) < 1e-12 and (p >= 0).all()
+    np.testing.assert_allclose(orc.softmax(x + 123.456), p, atol=1e-13)
+    # closed form on two logits: logistic function
+    a, b = 0.3, -1.1
+    np.testing.assert_allclose(orc.softmax(np.array([a, b]))[0], 1 / (1 + math.exp(b - a)), atol=1e-15)
+
+
+def test_output_lies_in_value_hull():
+    p = _problem(4)
+    K_t, V_t = orc.compress(p["K_vis"], p["V_vis"], p["idx"], p["U"], p["mu"], p["n"])
+    K_hat, V_hat = orc.reconstruct(K_t, V_t, p["theta"], p["U"], p["mu"])
+    out = orc.decode_attend_definition(p["q"], K_t, V_t, p["theta"], p["U"], p["mu"], p["K_txt"], p["V_txt"])
+    V_all = np.concatenate([V_hat, p["V_txt"]], axis=2)
+    G = p["q"].shape[1] // V_all.shape[1]
+    for hq in range(p["q"].shape[1]):
+        lo, hi = V_all[:, hq // G].min(axis=1), V_all[:, hq // G].max(axis=1)
+        assert (out[:, hq] >= lo - 1e-12).all() and (out[:, hq] <= hi + 1e-12).all()
+
+
+# ---------------------------------------------------------------- limit cases of the whole path
+def test_ratio_zero_is_uncompressed_attention_exactly():
+    p = _problem(5)
+    K_t, V_t = orc.compress(p["K_vis"], p["V_vis"], None, None, None, p["n"], passthrough=True)
+    assert K_t.shape == (2, 2, p["R"], p["n"], 8)
+    out = orc.decode_attend_definition(p["q"], K_t, V_t, None, None, None, p["K_txt"], p["V_txt"], passthrough=True)
+    K_all = np.concatenate([p["K_vis"], p["K_txt"]], axis=2)
+    V_all = np.concatenate([p["V_vis"], p["V_txt"]], axis=2)
+    assert np.array_equal(out, orc.attention(p["q"], K_all, V_all))          # bit for bit
+    np.testing.assert_allclose(out, _library_attention(p["q"], K_all, V_all), atol=1e-13)
+    fused = orc.decode_attend_fused(p["q"], K_t, V_t, None, None, None, p["K_txt"], p["V_txt"], passthrough=True)
+    np.testing.assert_allclose(fused, out, atol=1e-13)
+
+
+def test_no_vision_blocks_is_text_attention():
+    p = _problem(6, R=0)
+    K_t = np.zeros((2, 2, 0, p["m"], 8))
+    for f in (orc.decode_attend_definition, orc.decode_attend_fused):
+        out = f(p["q"], K_t, K_t, p["theta"], p["U"], p["mu"], p["K_txt"], p["V_txt"])
+        np.testing.assert_allclose(out, _library_attention(p["q"], p["K_txt"], p["V_txt"]), atol=1e-13)
+
+
+# ---------------------------------------------------------------- lossless constructions
+def _lossless_key_side(p, r):
+    """theta with theta[:, idx] = I_m and K = theta^T C  =>  K_hat == K."""
+    H_kv, m, n = p["theta"].shape
+    theta = p["theta"].copy()
+    for h in range(H_kv):
+        theta[h][:, p["idx"]] = np.eye(m)
+    B, _, N_v, d = p["K_vis"].shape
+    C = r.standard_normal((B, H_kv, p["R"], m, d))
+    K_vis = np.einsum("hmn,bhrmd->bhrnd", theta, C).reshape(B, H_kv, N_v, d)
+    return theta, K_vis
+
+
+def _lossless_value_side(p, r):
+    """U with orthonormal rows and V = U^T C + 1 mu^T  =>  V_hat == V."""
+    H_kv, m, n = p["U"].shape
+    U = np.stack([np.linalg.qr(r.standard_normal((n, m)))[0].T for _ in range(H_kv)])
+    B, _, N_v, d = p["V_vis"].shape
+    C = r.standard_normal((B, H_kv, p["R"], m, d))
+    V_vis = np.einsum("hmn,bhrmd->bhrnd", U, C) + p["mu"][None, :, None, None, :]
+    return U, V_vis.reshape(B, H_kv, N_v, d)
+
+
+def test_lossless_parameters_reproduce_full_attention():
+    p = _problem(7)
+    r = _rng(70)
+    theta, K_vis = _lossless_key_side(p, r)
+    U, V_vis = _lossless_value_side(p, r)
+    K_t, V_t = orc.compress(K_vis, V_vis, p["idx"], U, p["mu"], p["n"])
+    K_hat, V_hat = orc.reconstruct(K_t, V_t, theta, U, p["mu"])
+    np.testing.assert_allclose(K_hat, K_vis, atol=1e-12)
+    np.testing.assert_allclose(V_hat, V_vis, atol=1e-12)
+    K_all = np.concatenate([K_vis, p["K_txt"]], axis=2)
+    V_all = np.concatenate([V_vis, p["V_txt"]], axis=2)
+    want = _library_attention(p["q"], K_all, V_all)
+    for f in (orc.decode_attend_definition, orc.decode_attend_fused):
+        got = f(p["q"], K_t, V_t, theta, U, p["mu"], p["K_txt"], p["V_txt"])
+        np.testing.assert_allclose(got, want, atol=1e-11)
+
+
+def test_per_head_index_sets():
+    p = _problem(8)
+    r = _rng(80)
+    idx2 = np.stack([np.sort(r.permutation(p["n"])[:p["m"]]) for _ in range(2)]).astype(np.int32)
+    assert not np.array_equal(idx2[0], idx2[1])
+    K_t, _ = orc.compress(p["K_vis"], p["V_vis"], idx2, p["U"], p["mu"], p["n"])
+    for h in range(2):
+        for blk in range(p["R"]):
+            for j in range(p["m"]):
+                assert np.array_equal(K_t[1, h, blk, j], p["K_vis"][1, h, blk * p["n"] + idx2[h, j]])
+
+
+def test_value_pca_is_eckart_young_optimal():
+    # U = top-m left singular vectors of the centred block (Sec. 3.1): the residual
+    # energy of the re-projection equals the discarded singular values' energy.
+    r = _rng(9)
+    n, m, d = 24, 7, 10
+    V = r.standard_normal((1, 1, n, d)) @ np.diag(np.linspace(2, 0.1, d))
+    mu = V.mean(axis=2)[0]                                  # [1,d]
+    Uf, s, _ = np.linalg.svd(V[0, 0] - mu, full_matrices=False)
+    U = Uf[:, :m].T[None]                                   # [1,m,n]
+    _, V_t = orc.compress(V, V, np.arange(m), U, mu, n)
+    _, V_hat = orc.reconstruct(V_t, V_t, U, U, mu)
+    resid = np.sum((V - V_hat) ** 2)
+    np.testing.assert_allclose(resid, np.sum(s[m:] ** 2), rtol=1e-10)
+
+
+# ---------------------------------------------------------------- fused algebra
+@pytest.mark.parametrize("seed,kw", [(10, {}), (11, dict(B=1, H_q=4, H_kv=4, R=1, T=0)),
+                                     (12, dict(H_q=8, H_kv=1, n=9, m=9, R=2, T=1))])
+def test_definition_equals_algorithm_1(seed, kw):
+    p = _problem(seed, **kw)
+    K_t, V_t = orc.compress(p["K_vis"], p["V_vis"], p["idx"], p["U"], p["mu"], p["n"])
+    a = orc.decode_attend_definition(p["q"], K_t, V_t, p["theta"], p["U"], p["mu"], p["K_txt"], p["V_txt"])
+    b = orc.decode_attend_fused(p["q"], K_t, V_t, p["theta"], p["U"], p["mu"], p["K_txt"], p["V_txt"])
+    np.testing.assert_allclose(a, b, atol=1e-10)
+
+
+def test_block_order_and_split_merge_invariance():
+    # Softmax attention is invariant to permuting KV positions; permuting whole vision
+    # blocks must therefore leave the result unchanged, and a log-sum-exp merge of the
+    # per-block partial results must reproduce it.
+    p = _problem(13)
+    K_t, V_t = orc.compress(p["K_vis"], p["V_vis"], p["idx"], p["U"], p["mu"], p["n"])
+    ref = orc.decode_attend_definition(p["q"], K_t, V_t, p["theta"], p["U"], p["mu"], p["K_txt"], p["V_txt"])
+    perm = [2, 0, 1]
+    out = orc.decode_attend_definition(p["q"], K_t[:, :, perm], V_t[:, :, perm], p["theta"], p["U"], p["mu"],
+                                       p["K_txt"], p["V_txt"])
+    np.testing.assert_allclose(out, ref, atol=1e-12)
+    K_hat, V_hat = orc.reconstruct(K_t, V_t, p["theta"], p["U"], p["mu"])
+    n, d = p["n"], 8
+    parts = [(K_hat[:, :, r * n:(r + 1) * n], V_hat[:, :, r * n:(r + 1) * n]) for r in range(p["R"])]
+    parts.append((p["K_txt"], p["V_txt"]))
+    B, H_q = p["q"].shape[:2]
+    G = H_q // 2
+    for b in range(B):
+        for hq in range(H_q):
+            ms, ls, ys = [], [], []
+            for Kp, Vp in parts:
+                s = Kp[b, hq // G] @ p["q"][b, hq] / math.sqrt(d)
+                ms.append(s.max()); e = np.exp(s - s.max()); ls.append(e.sum()); ys.append(e @ Vp[b, hq // G])
+            M = max(ms)
+            num = sum(math.exp(mi - M) * yi for mi, yi in zip(ms, ys))
+            den = sum(math.exp(mi - M) * li for mi, li in zip(ms, ls))
+            np.testing.assert_allclose(num / den, ref[b, hq], atol=1e-12)
+
+
+# ---------------------------------------------------------------- brute force, tiny grid
+def test_tiny_grid_brute_force():
+    """n = 4 (2x2 grid), m = 2, d = 2, G = 1, T = 1: every step with scalar loops."""
+    r = _rng(14)
+    n, m, d, T = 4, 2, 2, 1
+    K = r.standard_normal((n, d)); V = r.standard_normal((n, d))
+    kt = r.standard_normal((T, d)); vt = r.standard_normal((T, d))
+    q = r.standard_normal(d)
+    th = r.standard_normal((m, n)); U = r.standard_normal((m, n)); mu = r.standard_normal(d)
+    idx = [1, 3]
+    # compress
+    Kc = [[K[idx[j]][c] for c in range(d)] for j in range(m)]
+    Vc = [[sum(U[j][i] * (V[i][c] - mu[c]) for i in range(n)) for c in range(d)] for j in range(m)]
+    # reconstruct
+    Kh = [[sum(th[j][i] * Kc[j][c] for j in range(m)) for c in range(d)] for i in range(n)]
+    Vh = [[sum(U[j][i] * Vc[j][c] for j in range(m)) + mu[c] for c in range(d)] for i in range(n)]
+    rowsK = Kh + [list(kt[0])]
+    rowsV = Vh + [list(vt[0])]
+    logits = [sum(q[c] * rk[c] for c in range(d)) / math.sqrt(d) for rk in rowsK]
+    mx = max(logits)
+    ex = [math.exp(l - mx) for l in logits]
+    Z = sum(ex)
+    want = [sum(ex[i] / Z * rowsV[i][c] for i in range(n + T)) for c in range(d)]
+
+    K_t, V_t = orc.compress(K[None, None], V[None, None], np.array(idx), U[None], mu[None], n)
+    np.testing.assert_allclose(K_t[0, 0, 0], np.array(Kc), atol=0)
+    np.testing.assert_allclose(V_t[0, 0, 0], np.array(Vc), atol=1e-14)
+    for f in (orc.decode_attend_definition, orc.decode_attend_fused):
+        got = f(q[None, None], K_t, V_t, th[None], U[None], mu[None], kt[None, None], vt[None, None])
+        np.testing.assert_allclose(got[0, 0], want, atol=1e-13)
+
+
+def test_scalar_closed_form():
+    """n = 2, m = 1, d = 1: the whole path is a three-way logistic mixture in closed form."""
+    k0, k1, v0, v1 = 0.7, -0.4, 1.5, -2.0
+    a, b, u0, u1, mu, q, kt, vt = 0.9, -0.3, 0.6, 0.8, 0.25, 1.3, 0.2, 3.0
+    K = np.array([k0, k1]).reshape(1, 1, 2, 1); V = np.array([v0, v1]).reshape(1, 1, 2, 1)
+    K_t, V_t = orc.compress(K, V, np.array([0]), np.array([[[u0, u1]]]), np.array([[mu]]), 2)
+    vtil = u0 * (v0 - mu) + u1 * (v1 - mu)
+    assert K_t[0, 0, 0, 0, 0] == k0 and abs(V_t[0, 0, 0, 0, 0] - vtil) < 1e-15
+    l = [q * a * k0, q * b * k0, q * kt]                     # sigma = 1/sqrt(1)
+    w = [math.exp(x) for x in l]
+    want = (w[0] * (u0 * vtil + mu) + w[1] * (u1 * vtil + mu) + w[2] * vt) / sum(w)
+    for f in (orc.decode_attend_definition, orc.decode_attend_fused):
+        got = f(np.array([[[q]]]), K_t, V_t, np.array([[[a, b]]]), np.array([[[u0, u1]]]), np.array([[mu]]),
+                np.array([[[[kt]]]]), np.array([[[[vt]]]]))
+        assert abs(got[0, 0, 0] - want) < 1e-14
+
+
+# ---------------------------------------------------------------- sizes (App. D)
+def _golden(name):
+    vals = {}
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                k, v = line.split()
+                vals[k] = float(v)
+    return vals
+
+
+def test_memory_footprint_closed_forms_and_paper_ratio():
+    g = _golden("paper_constants.txt")
+    B, H_kv, d, b = 16, 4, 128, 2
+    n, R, c, t = 1024, 8, 256, 0
+    m = orc.retained_len(n, 600)
+    base = orc.footprint_base(B, H_kv, c, R * n, t, d, b)
+    ours = orc.footprint_kvcapsule(B, H_kv, c, n, R, t, d, b, 600)
+    assert base == 2 * 16 * 4 * (256 + 8192) * 128 * 2
+    cache = 2 * B * H_kv * (c + R * m + t) * d * b
+    assert ours == cache + 2 * H_kv * m * n * b + H_kv * d * b
+    # the paper's headline persistent-memory reduction at 60 % compression
+    assert round(base / cache, 1) == g["memory_reduction_at_60pct"]
+    # with the batch-independent parameter overhead included the reduction is a little lower
+    assert 2.2 < base / ours < base / cache
+    # vision-only reduction is 1 / l_r up to the ceiling
+    for nn in (576, 1024, 256):
+        assert abs(nn / orc.retained_len(nn, 600) - 2.5) < 0.02
+    # parameter overhead is independent of batch size and generated length (Sec. 4.3)
+    o1 = orc.footprint_kvcapsule(1, H_kv, c, n, R, 0, d, b, 600) - 2 * 1 * H_kv * (c + R * m) * d * b
+    o2 = orc.footprint_kvcapsule(64, H_kv, c, n, R, 99, d, b, 600) - 2 * 64 * H_kv * (c + R * m + 99) * d * b
+    assert o1 == o2
