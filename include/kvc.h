@@ -1,0 +1,134 @@
+/*
+ * kvc.h -- C ABI of the KVCapsule decode-time hot path for NVIDIA B200 (sm_100a).
+ *
+ * KVCapsule (arxiv 2605.16439) keeps a VLM backbone unchanged and stores, per layer, the
+ * vision-token K/V of each n-token image block in compressed form ("capsules"):
+ *   keys   : the m = ceil(l_r n) rows picked by a fixed index set M_l          (Sec. 3.1, keys)
+ *   values : V_tilde = U_l (V - 1 mu_l^T), a projection along the token axis  (Sec. 3.1, values)
+ * and, at every decode step, attends over the reconstructed vision K/V together with the
+ * untouched text K/V (Sec. 3.2).  The library never writes full-size vision K/V: it follows
+ * the associative order of Algorithm 1 (scores in compressed space, expansion by theta,
+ * softmax, re-projection by U^T, product with V_tilde plus the mu term).
+ *
+ * Conventions
+ *   - Every tensor pointer is a DEVICE pointer to caller-owned, contiguous memory unless a
+ *     comment says "host".  The library owns only the opaque kvc_layer (a host struct plus a
+ *     small device copy of the index set).
+ *   - Calls are asynchronous on the given CUDA stream (a cudaStream_t passed as void*; NULL is
+ *     the legacy default stream).  They never synchronise and, except kvc_layer_create /
+ *     kvc_layer_destroy, never allocate or free device memory.
+ *   - All functions returning int return a kvc_status.  Argument and shape errors are found on
+ *     the host before anything is launched.  No exception crosses this boundary.
+ *   - Layouts are row-major with the last index fastest; d (head dimension) must be 128.
+ *   - dtype is the storage type of q, K, V, capsules, theta, U, mu and out; all arithmetic
+ *     accumulates in fp32.
+ */
+#ifndef KVC_H_
+#define KVC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(KVC_BUILD) && defined(__GNUC__)
+#define KVC_API __attribute__((visibility("default")))
+#else
+#define KVC_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  KVC_OK = 0,
+  KVC_ERR_ARG = -1,        /* null pointer, negative size                               */
+  KVC_ERR_SHAPE = -2,      /* unsupported or inconsistent shape                         */
+  KVC_ERR_DTYPE = -3,      /* unknown dtype                                             */
+  KVC_ERR_NO_PARAMS = -4,  /* theta / U / mu / idx missing for a ratio > 0              */
+  KVC_ERR_WORKSPACE = -5,  /* workspace pointer null or misaligned                      */
+  KVC_ERR_CUDA = -6,       /* a CUDA runtime call failed (launch, copy, allocation)     */
+  KVC_ERR_TIMEOUT = -7,    /* a bounded device-side wait gave up                        */
+  KVC_ERR_BOUNDS = -8      /* an index set entry is out of range or not increasing      */
+} kvc_status;
+
+typedef enum { KVC_F32 = 0, KVC_BF16 = 1 } kvc_dtype;
+
+/* One parameter set = one (layer, compression ratio); the paper trains M_l, theta_l, U_l, mu_l
+ * per layer for a given retention ratio (App. C, Algorithm 2) and fixes them at inference
+ * (Sec. 3.2).  Shapes follow App. D: theta, U in R^{H_kv x m x n}, mu in R^{H_kv x d}. */
+typedef struct {
+  int layer;              /* informational                                                    */
+  int H_q, H_kv;          /* query heads, KV heads; G = H_q / H_kv must be an integer <= 16    */
+  int d;                  /* head dimension, must be 128                                       */
+  int n;                  /* tokens per vision block ("an image with size n", Sec. 3.1)        */
+  int ratio_permille;     /* compression ratio rho * 1000 in [0, 1000); l_r = 1 - rho          */
+  int dtype;              /* kvc_dtype                                                         */
+  const int32_t* idx;     /* HOST pointer: retained-key indices, 0-based, strictly increasing; */
+  int idx_per_head;       /*   [m] if 0, [H_kv][m] if 1.  Ignored when ratio_permille == 0.    */
+  const void* theta;      /* [H_kv][m][n]  key / score reconstruction matrix (borrowed)        */
+  const void* U;          /* [H_kv][m][n]  value PCA basis (borrowed); rows need not be orthonormal */
+  const void* mu;         /* [H_kv][d]     value centering vector (borrowed)                   */
+} kvc_layer_desc;
+
+typedef struct kvc_layer kvc_layer;
+
+/* m = ceil((1 - rho) n) (Sec. 3.1), computed as (n*(1000-ratio_permille)+999)/1000 in integers.
+ * Returns -1 for n <= 0 or a ratio outside [0, 1000). */
+KVC_API int kvc_retained_len(int n, int ratio_permille);
+
+/* Validates the descriptor (KVC_ERR_SHAPE / _DTYPE / _NO_PARAMS / _BOUNDS), copies the index set
+ * to device memory and returns a handle.  theta, U and mu are borrowed: they must stay valid and
+ * unchanged while the handle is in use.  ratio_permille == 0 is the pass-through limit: m = n,
+ * capsules hold K and V verbatim, idx / theta / U / mu are ignored.
+ * The device that is current at this call must be current for every later call with the handle. */
+KVC_API int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out);
+KVC_API int kvc_layer_destroy(kvc_layer* layer);
+
+/* Bytes of the capsule store for B sequences of R blocks:  K_tilde [B][H_kv][R][m][d] followed
+ * by V_tilde [B][H_kv][R][m][d] (the compressed-cache term of App. D, Eq. 2, vision part). */
+KVC_API size_t kvc_capsule_bytes(const kvc_layer* layer, int B, int R);
+
+/* Bytes of scratch kvc_decode_attend needs for up to B sequences, R blocks and T_cap text rows.
+ * The scratch holds only temporaries of one call (compressed scores, expanded-probability
+ * projections, split partials); it needs no initialisation and must be 256-byte aligned. */
+KVC_API size_t kvc_workspace_bytes(const kvc_layer* layer, int B, int R, int T_cap);
+
+/* Prefill-stage compression (Sec. 3.2 "Prefilling Stage").  For every sequence b, KV head h and
+ * block r:  K_tilde[b,h,r,j,:] = K_vis[b,h,r*n + idx[j],:],
+ *           V_tilde[b,h,r]     = U[h] (V_vis[b,h,r*n:(r+1)*n] - 1 mu[h]^T).
+ * K_vis, V_vis: [B][H_kv][R*n][d].  capsules: out, kvc_capsule_bytes(layer,B,R) bytes.
+ * B == 0 or R == 0 is a no-op. */
+KVC_API int kvc_compress(const kvc_layer* layer, const void* K_vis, const void* V_vis, int B, int R,
+                 void* capsules, void* stream);
+
+/* Decode-stage attention over reconstructed vision K/V plus text K/V (Sec. 3.2 "Decoding Stage",
+ * Algorithm 1).  out[b,hq,:] = softmax_over(R*n + T)( sigma q . [theta^T K_tilde ; K_txt] ) .
+ * [U^T V_tilde + 1 mu^T ; V_txt],  sigma = 1/sqrt(d), query head hq reading KV head hq / G.
+ * q, out: [B][H_q][d].  K_txt, V_txt: [B][H_kv][T_cap][d] of which the first T rows are valid
+ * (may be NULL when T == 0).  R == 0 attends over text only; R == 0 and T == 0 is KVC_ERR_SHAPE.
+ * workspace: kvc_workspace_bytes(layer, B, R, >= T) bytes; calls sharing a workspace must be
+ * stream-ordered. */
+KVC_API int kvc_decode_attend(const kvc_layer* layer, const void* q, const void* capsules, int B, int R,
+                      const void* K_txt, const void* V_txt, int T, int T_cap, void* out,
+                      void* workspace, void* stream);
+
+/* Uncompressed decode attention over K, V [B][H_kv][S_cap][d] (first S rows valid), the standard
+ * attention of Sec. 3.1; the comparator the compressed path is measured against.  Uses the same
+ * workspace rule with R = 0, T_cap = S_cap. */
+KVC_API int kvc_attend_full(const kvc_layer* layer, const void* q, const void* K, const void* V, int B,
+                    int S, int S_cap, void* out, void* workspace, void* stream);
+
+/* Integer maps as the device path uses them (read back from the device copy):
+ * idx_out: HOST [H_kv][m] retained indices per KV head; group_out: HOST [R*n][2] = (block r,
+ * offset i) of vision token t = r*n + i (the Reshape of Alg. 1 step 1).  Either may be NULL. */
+KVC_API int kvc_export_maps(const kvc_layer* layer, int R, int32_t* idx_out, int32_t* group_out);
+
+/* Retained length m and the row stride (in elements) of internal score buffers. */
+KVC_API int kvc_layer_m(const kvc_layer* layer);
+
+KVC_API const char* kvc_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVC_H_ */

@@ -1,0 +1,163 @@
+"""Thin ctypes binding of libkvc.so: argument marshalling only, every step runs in the CUDA kernels.
+
+Function names mirror the C ABI declared in include/kvc.h.  torch is used for device memory and
+the current stream; there is no CPU fallback: a missing library or a failing call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libkvc.so")
+
+KVC_F32, KVC_BF16 = 0, 1
+_DTYPES = {torch.float32: KVC_F32, torch.bfloat16: KVC_BF16}
+
+
+class KvcError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = _lib().kvc_strerror(status).decode() if _LIB is not None else "?"
+        super().__init__(f"{where}: {msg} (status {status})")
+
+
+class kvc_layer_desc(C.Structure):
+    _fields_ = [("layer", C.c_int), ("H_q", C.c_int), ("H_kv", C.c_int), ("d", C.c_int), ("n", C.c_int),
+                ("ratio_permille", C.c_int), ("dtype", C.c_int), ("idx", C.POINTER(C.c_int32)),
+                ("idx_per_head", C.c_int), ("theta", C.c_void_p), ("U", C.c_void_p), ("mu", C.c_void_p)]
+
+
+_LIB = None
+
+
+def _lib() -> C.CDLL:
+    """Loads libkvc.so once; raises if it has not been built (python -m paper_2605_16439_b200.build)."""
+    global _LIB
+    if _LIB is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2605_16439_b200.build`")
+        lib = C.CDLL(LIB_PATH)
+        vp, i = C.c_void_p, C.c_int
+        lib.kvc_retained_len.argtypes = [i, i]; lib.kvc_retained_len.restype = i
+        lib.kvc_layer_create.argtypes = [C.POINTER(kvc_layer_desc), C.POINTER(vp)]; lib.kvc_layer_create.restype = i
+        lib.kvc_layer_destroy.argtypes = [vp]; lib.kvc_layer_destroy.restype = i
+        lib.kvc_layer_m.argtypes = [vp]; lib.kvc_layer_m.restype = i
+        lib.kvc_capsule_bytes.argtypes = [vp, i, i]; lib.kvc_capsule_bytes.restype = C.c_size_t
+        lib.kvc_workspace_bytes.argtypes = [vp, i, i, i]; lib.kvc_workspace_bytes.restype = C.c_size_t
+        lib.kvc_compress.argtypes = [vp, vp, vp, i, i, vp, vp]; lib.kvc_compress.restype = i
+        lib.kvc_decode_attend.argtypes = [vp, vp, vp, i, i, vp, vp, i, i, vp, vp, vp]
+        lib.kvc_decode_attend.restype = i
+        lib.kvc_attend_full.argtypes = [vp, vp, vp, vp, i, i, i, vp, vp, vp]; lib.kvc_attend_full.restype = i
+        lib.kvc_export_maps.argtypes = [vp, i, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+        lib.kvc_export_maps.restype = i
+        lib.kvc_strerror.argtypes = [i]; lib.kvc_strerror.restype = C.c_char_p
+        _LIB = lib
+    return _LIB
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise KvcError(status, where)
+
+
+def _ptr(t) -> int | None:
+    if t is None:
+        return None
+    if not t.is_contiguous():
+        raise ValueError("tensors passed to the kvc library must be contiguous")
+    return t.data_ptr()
+
+
+def _stream(stream=None) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def kvc_retained_len(n: int, ratio_permille: int) -> int:
+    return _lib().kvc_retained_len(n, ratio_permille)
+
+
+class Layer:
+    """Owns one kvc_layer handle and keeps the borrowed parameter tensors alive."""
+
+    def __init__(self, H_q: int, H_kv: int, d: int, n: int, ratio_permille: int, dtype: torch.dtype,
+                 idx=None, theta=None, U=None, mu=None, layer: int = 0):
+        if dtype not in _DTYPES:
+            raise KvcError(-3, "kvc_layer_create") if _LIB else ValueError("unsupported dtype")
+        self.H_q, self.H_kv, self.d, self.n, self.dtype = H_q, H_kv, d, n, dtype
+        self.ratio_permille = ratio_permille
+        self._keep = (theta, U, mu)
+        desc = kvc_layer_desc()
+        desc.layer, desc.H_q, desc.H_kv, desc.d, desc.n = layer, H_q, H_kv, d, n
+        desc.ratio_permille, desc.dtype = ratio_permille, _DTYPES[dtype]
+        idx_host = None
+        if idx is not None:
+            idx_host = idx.detach().to("cpu", torch.int32).contiguous()
+            desc.idx = C.cast(idx_host.data_ptr(), C.POINTER(C.c_int32))
+            desc.idx_per_head = 1 if idx_host.dim() == 2 else 0
+        for name, t in (("theta", theta), ("U", U), ("mu", mu)):
+            if t is not None and t.dtype != dtype:
+                raise ValueError(f"{name} must have the layer's storage dtype")
+            setattr(desc, name, _ptr(t))
+        h = C.c_void_p()
+        _check(_lib().kvc_layer_create(C.byref(desc), C.byref(h)), "kvc_layer_create")
+        self.handle = h
+        self.m = _lib().kvc_layer_m(h)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            _lib().kvc_layer_destroy(self.handle)
+            self.handle = None
+
+    __del__ = close
+
+
+def kvc_capsule_bytes(layer: Layer, B: int, R: int) -> int:
+    return _lib().kvc_capsule_bytes(layer.handle, B, R)
+
+
+def kvc_workspace_bytes(layer: Layer, B: int, R: int, T_cap: int) -> int:
+    return _lib().kvc_workspace_bytes(layer.handle, B, R, T_cap)
+
+
+def alloc_capsules(layer: Layer, B: int, R: int, device="cuda") -> torch.Tensor:
+    return torch.empty(max(kvc_capsule_bytes(layer, B, R), 1), dtype=torch.uint8, device=device)
+
+
+def alloc_workspace(layer: Layer, B: int, R: int, T_cap: int, device="cuda") -> torch.Tensor:
+    return torch.empty(kvc_workspace_bytes(layer, B, R, T_cap), dtype=torch.uint8, device=device)
+
+
+def kvc_compress(layer: Layer, K_vis, V_vis, B: int, R: int, capsules, stream=None) -> None:
+    _check(_lib().kvc_compress(layer.handle, _ptr(K_vis), _ptr(V_vis), B, R, _ptr(capsules), _stream(stream)),
+           "kvc_compress")
+
+
+def kvc_decode_attend(layer: Layer, q, capsules, B: int, R: int, K_txt, V_txt, T: int, T_cap: int, out,
+                      workspace, stream=None) -> None:
+    _check(_lib().kvc_decode_attend(layer.handle, _ptr(q), _ptr(capsules), B, R, _ptr(K_txt), _ptr(V_txt), T,
+                                    T_cap, _ptr(out), _ptr(workspace), _stream(stream)), "kvc_decode_attend")
+
+
+def kvc_attend_full(layer: Layer, q, K, V, B: int, S: int, S_cap: int, out, workspace, stream=None) -> None:
+    _check(_lib().kvc_attend_full(layer.handle, _ptr(q), _ptr(K), _ptr(V), B, S, S_cap, _ptr(out),
+                                  _ptr(workspace), _stream(stream)), "kvc_attend_full")
+
+
+def kvc_export_maps(layer: Layer, R: int):
+    """(idx [H_kv, m] int32, group [R*n, 2] int32) as the device path holds them."""
+    idx = torch.empty((layer.H_kv, layer.m), dtype=torch.int32)
+    grp = torch.empty((R * layer.n, 2), dtype=torch.int32)
+    _check(_lib().kvc_export_maps(layer.handle, R, C.cast(idx.data_ptr(), C.POINTER(C.c_int32)),
+                                  C.cast(grp.data_ptr(), C.POINTER(C.c_int32))), "kvc_export_maps")
+    return idx, grp
+
+
+def capsule_views(layer: Layer, capsules, B: int, R: int):
+    """(K_tilde, V_tilde) [B,H_kv,R,m,d] typed views of a capsule store (no copy)."""
+    half = kvc_capsule_bytes(layer, B, R) // 2
+    shape = (B, layer.H_kv, R, layer.m, layer.d)
+    return (capsules[:half].view(layer.dtype).view(shape), capsules[half:2 * half].view(layer.dtype).view(shape))

@@ -1,0 +1,213 @@
+// Host side of the C ABI: validation, layer handles, workspace layout, kernel sequencing.
+#include <new>
+#include <vector>
+
+#include "kvc_internal.cuh"
+
+namespace kvc {
+
+static size_t elem_bytes(int dtype) { return dtype == KVC_BF16 ? 2 : 4; }
+
+WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap) {
+  WsLayout w{};
+  const int H_kv = L->desc.H_kv, G = L->G, n = L->desc.n, ms = L->ms;
+  const int rows_h = B * G * R;
+  const int row_tiles = ceil_div(rows_h, EXP_ROWS) * H_kv;
+  if (L->passthrough || rows_h == 0) {
+    w.NS = 1;
+    w.IR = align_up(n, EXP_IC);
+  } else {
+    int ns = ceil_div(EXP_TARGET_CTAS, row_tiles);
+    ns = ns < 1 ? 1 : ns;
+    const int max_ns = ceil_div(n, EXP_IC);
+    ns = ns > max_ns ? max_ns : ns;
+    w.IR = (int)align_up((size_t)ceil_div(n, ns), EXP_IC);
+    w.NS = ceil_div(n, w.IR);
+  }
+  w.NTC = ceil_div(T_cap, TXT_CHUNK);
+  w.nsplit = R + w.NTC;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  w.off_S = take(sizeof(float) * (size_t)H_kv * rows_h * ms);
+  w.off_stxt = take(sizeof(float) * (size_t)B * H_kv * G * (T_cap > 0 ? T_cap : 1));
+  // sized so that the bytes never shrink when B or R grow (NS falls as the row count rises)
+  const size_t w_rows = (size_t)(EXP_TARGET_CTAS + row_tiles) * EXP_ROWS;
+  w.off_W = take(sizeof(float) * w_rows * ms);
+  w.off_wstat = take(sizeof(float2) * w_rows);
+  w.off_ypart = take(sizeof(float) * (size_t)B * H_kv * G * w.nsplit * D);
+  w.off_ystat = take(sizeof(float2) * (size_t)B * H_kv * G * w.nsplit);
+  w.off_cnt = take(sizeof(int) * (size_t)B * H_kv);
+  w.total = off;
+  return w;
+}
+
+}  // namespace kvc
+
+using namespace kvc;
+
+extern "C" {
+
+int kvc_retained_len(int n, int ratio_permille) {
+  if (n <= 0 || ratio_permille < 0 || ratio_permille >= 1000) return -1;
+  return (int)(((long long)n * (1000 - ratio_permille) + 999) / 1000);
+}
+
+const char* kvc_strerror(int s) {
+  switch (s) {
+    case KVC_OK: return "ok";
+    case KVC_ERR_ARG: return "invalid argument (null pointer or negative size)";
+    case KVC_ERR_SHAPE: return "unsupported or inconsistent shape";
+    case KVC_ERR_DTYPE: return "unknown dtype";
+    case KVC_ERR_NO_PARAMS: return "theta / U / mu / idx missing for a compression ratio > 0";
+    case KVC_ERR_WORKSPACE: return "workspace null or not 256-byte aligned";
+    case KVC_ERR_CUDA: return "CUDA runtime error";
+    case KVC_ERR_TIMEOUT: return "bounded device-side wait gave up";
+    case KVC_ERR_BOUNDS: return "index set entry out of range or not strictly increasing";
+    default: return "unknown status";
+  }
+}
+
+int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out) {
+  if (!desc || !out) return KVC_ERR_ARG;
+  *out = nullptr;
+  if (desc->dtype != KVC_F32 && desc->dtype != KVC_BF16) return KVC_ERR_DTYPE;
+  if (desc->d != D || desc->H_q <= 0 || desc->H_kv <= 0 || desc->H_q % desc->H_kv != 0 ||
+      desc->H_q / desc->H_kv > MAX_G || desc->n <= 0)
+    return KVC_ERR_SHAPE;
+  const int m = kvc_retained_len(desc->n, desc->ratio_permille);
+  if (m < 1) return KVC_ERR_SHAPE;
+  const bool pass = desc->ratio_permille == 0;
+  if (!pass && (!desc->idx || !desc->theta || !desc->U || !desc->mu)) return KVC_ERR_NO_PARAMS;
+
+  std::vector<int32_t> idx((size_t)desc->H_kv * m);
+  for (int h = 0; h < desc->H_kv; ++h)
+    for (int j = 0; j < m; ++j) {
+      const int32_t v = pass ? j : desc->idx[(desc->idx_per_head ? (size_t)h * m : 0) + j];
+      if (v < 0 || v >= desc->n || (j > 0 && v <= idx[(size_t)h * m + j - 1])) return KVC_ERR_BOUNDS;
+      idx[(size_t)h * m + j] = v;
+    }
+
+  kvc_layer* L = new (std::nothrow) kvc_layer();
+  if (!L) return KVC_ERR_ARG;
+  L->desc = *desc;
+  L->desc.idx = nullptr;
+  L->m = m;
+  L->ms = (m + 15) / 16 * 16;
+  L->G = desc->H_q / desc->H_kv;
+  L->passthrough = pass ? 1 : 0;
+  L->d_idx = nullptr;
+  if (cudaGetDevice(&L->device) != cudaSuccess ||
+      cudaMalloc(&L->d_idx, idx.size() * sizeof(int32_t)) != cudaSuccess ||
+      cudaMemcpy(L->d_idx, idx.data(), idx.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess) {
+    if (L->d_idx) cudaFree(L->d_idx);
+    delete L;
+    cudaGetLastError();
+    return KVC_ERR_CUDA;
+  }
+  *out = L;
+  return KVC_OK;
+}
+
+int kvc_layer_destroy(kvc_layer* L) {
+  if (!L) return KVC_OK;
+  if (L->d_idx) cudaFree(L->d_idx);
+  delete L;
+  return KVC_OK;
+}
+
+int kvc_layer_m(const kvc_layer* L) { return L ? L->m : -1; }
+
+size_t kvc_capsule_bytes(const kvc_layer* L, int B, int R) {
+  if (!L || B < 0 || R < 0) return 0;
+  return (size_t)2 * B * L->desc.H_kv * R * L->m * D * elem_bytes(L->desc.dtype);
+}
+
+size_t kvc_workspace_bytes(const kvc_layer* L, int B, int R, int T_cap) {
+  if (!L || B < 0 || R < 0 || T_cap < 0) return 0;
+  return ws_layout(L, B, R, T_cap).total;
+}
+
+int kvc_compress(const kvc_layer* L, const void* K_vis, const void* V_vis, int B, int R, void* capsules,
+                 void* stream) {
+  if (!L || B < 0 || R < 0) return KVC_ERR_ARG;
+  if (B == 0 || R == 0) return KVC_OK;
+  if (!K_vis || !V_vis || !capsules) return KVC_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t half = kvc_capsule_bytes(L, B, R) / 2;
+  void* Kc = capsules;
+  void* Vc = static_cast<char*>(capsules) + half;
+  cudaError_t e;
+  if (L->passthrough) {
+    e = cudaMemcpyAsync(Kc, K_vis, half, cudaMemcpyDeviceToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(Vc, V_vis, half, cudaMemcpyDeviceToDevice, st);
+  } else {
+    e = launch_compress(L, K_vis, V_vis, B, R, Kc, Vc, st);
+  }
+  return e == cudaSuccess ? KVC_OK : KVC_ERR_CUDA;
+}
+
+static int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B, int R,
+                         const void* K_txt, const void* V_txt, int T, int T_cap, void* out, void* workspace,
+                         cudaStream_t st) {
+  if (!L || B < 0 || R < 0 || T < 0 || T_cap < T) return KVC_ERR_ARG;
+  if (B == 0) return KVC_OK;
+  if (R == 0 && T == 0) return KVC_ERR_SHAPE;
+  if (!q || !out || (R > 0 && !capsules) || (T > 0 && (!K_txt || !V_txt))) return KVC_ERR_ARG;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255)) return KVC_ERR_WORKSPACE;
+
+  DecodeArgs a{};
+  a.ws = ws_layout(L, B, R, T);
+  char* ws = static_cast<char*>(workspace);
+  const size_t half = kvc_capsule_bytes(L, B, R) / 2;
+  a.q = q;
+  a.Kc = capsules;
+  a.Vc = capsules ? static_cast<const char*>(capsules) + half : nullptr;
+  a.K_txt = K_txt; a.V_txt = V_txt;
+  a.theta = L->desc.theta; a.U = L->desc.U; a.mu = L->desc.mu;
+  a.out = out;
+  a.B = B; a.H_kv = L->desc.H_kv; a.G = L->G; a.R = R; a.m = L->m; a.ms = L->ms; a.n = L->desc.n;
+  a.T = T; a.T_cap = T_cap > 0 ? T_cap : 1; a.Ts = T > 0 ? T : 1;
+  a.passthrough = L->passthrough;
+  a.S = reinterpret_cast<float*>(ws + a.ws.off_S);
+  a.s_txt = reinterpret_cast<float*>(ws + a.ws.off_stxt);
+  a.W = reinterpret_cast<float*>(ws + a.ws.off_W);
+  a.wstat = reinterpret_cast<float2*>(ws + a.ws.off_wstat);
+  a.ypart = reinterpret_cast<float*>(ws + a.ws.off_ypart);
+  a.ystat = reinterpret_cast<float2*>(ws + a.ws.off_ystat);
+  a.cnt = reinterpret_cast<int*>(ws + a.ws.off_cnt);
+
+  cudaError_t e = launch_scores(a, L->desc.dtype, st);
+  if (e == cudaSuccess) e = launch_expand(a, L->desc.dtype, st);
+  if (e == cudaSuccess) e = launch_output(a, L->desc.dtype, st);
+  return e == cudaSuccess ? KVC_OK : KVC_ERR_CUDA;
+}
+
+int kvc_decode_attend(const kvc_layer* L, const void* q, const void* capsules, int B, int R, const void* K_txt,
+                      const void* V_txt, int T, int T_cap, void* out, void* workspace, void* stream) {
+  return decode_common(L, q, capsules, B, R, K_txt, V_txt, T, T_cap, out, workspace,
+                       static_cast<cudaStream_t>(stream));
+}
+
+int kvc_attend_full(const kvc_layer* L, const void* q, const void* K, const void* V, int B, int S, int S_cap,
+                    void* out, void* workspace, void* stream) {
+  return decode_common(L, q, nullptr, B, 0, K, V, S, S_cap, out, workspace, static_cast<cudaStream_t>(stream));
+}
+
+int kvc_export_maps(const kvc_layer* L, int R, int32_t* idx_out, int32_t* group_out) {
+  if (!L || R < 0) return KVC_ERR_ARG;
+  if (idx_out) {
+    if (cudaMemcpy(idx_out, L->d_idx, (size_t)L->desc.H_kv * L->m * sizeof(int32_t), cudaMemcpyDeviceToHost) !=
+        cudaSuccess)
+      return KVC_ERR_CUDA;
+  }
+  if (group_out) {
+    const int n = L->desc.n;
+    for (long long t = 0; t < (long long)R * n; ++t) {
+      group_out[2 * t] = (int32_t)(t / n);
+      group_out[2 * t + 1] = (int32_t)(t % n);
+    }
+  }
+  return KVC_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,112 @@
+// Internal declarations shared by the KVCapsule CUDA translation units (not part of the ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kvc.h"
+
+namespace kvc {
+
+constexpr int D = 128;              // head dimension (all supported models)
+constexpr int MAX_G = 16;           // query heads per KV head
+constexpr int SCORE_TILE_ROWS = 64; // K rows per CTA in the score kernel
+constexpr int TXT_CHUNK = 256;      // text rows per split in the output kernel
+constexpr int EXP_ROWS = 16;        // rows per CTA in the generic expansion kernel
+constexpr int EXP_IC = 64;          // vision positions per inner chunk of the expansion
+constexpr int EXP_TARGET_CTAS = 296;
+
+inline __host__ __device__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
+inline __host__ __device__ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---- 16-byte vector access, converted to fp32 -----------------------------------------------
+template <typename T> struct Elems16;
+template <> struct Elems16<float> { static constexpr int N = 4; };
+template <> struct Elems16<__nv_bfloat16> { static constexpr int N = 8; };
+
+__device__ __forceinline__ void unpack16(const uint4& v, float (&f)[4], float*) {
+  f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+  f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+}
+__device__ __forceinline__ void unpack16(const uint4& v, float (&f)[8], __nv_bfloat16*) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    f[2 * i] = __uint_as_float(w[i] << 16);
+    f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+template <typename T>
+__device__ __forceinline__ void load16(const T* p, float (&f)[Elems16<T>::N]) {
+  uint4 v = __ldg(reinterpret_cast<const uint4*>(p));
+  unpack16(v, f, (T*)nullptr);
+}
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+__device__ __forceinline__ void store_elem(float* p, float x) { *p = x; }
+__device__ __forceinline__ void store_elem(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
+
+// ---- workspace layout of one decode call -----------------------------------------------------
+struct WsLayout {
+  int NS;          // splits of the n axis in the expansion kernel
+  int IR;          // vision positions per split (multiple of EXP_IC)
+  int NTC;         // text chunks
+  int nsplit;      // R + NTC output splits per (sequence, KV head)
+  size_t off_S;    // fp32 [H_kv][B][G][R][ms]   compressed scores, sigma applied
+  size_t off_stxt; // fp32 [B][H_kv][G][T]       text logits
+  size_t off_W;    // fp32 [NS][H_kv][B*G*R][ms] unnormalised P U^T per split
+  size_t off_wstat;// float2 [NS][H_kv][B*G*R]   (max, sum) per row and split
+  size_t off_ypart;// fp32 [B][H_kv][G][nsplit][D]
+  size_t off_ystat;// float2 [B][H_kv][G][nsplit]
+  size_t off_cnt;  // int [B*H_kv]
+  size_t total;
+};
+
+}  // namespace kvc
+
+struct kvc_layer {
+  kvc_layer_desc desc;   // idx pointer cleared after the copy
+  int m;                 // retained length
+  int ms;                // row stride of score buffers (m rounded up to 16)
+  int G;
+  int passthrough;       // ratio_permille == 0
+  int device;
+  int32_t* d_idx;        // device [H_kv][m]
+};
+
+namespace kvc {
+
+WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap);
+
+struct DecodeArgs {
+  const void* q;
+  const void* Kc;      // K_tilde  [B][H_kv][R][m][D]
+  const void* Vc;      // V_tilde
+  const void* K_txt;
+  const void* V_txt;
+  const void* theta;
+  const void* U;
+  const void* mu;
+  void* out;
+  int B, H_kv, G, R, m, ms, n, T, T_cap;
+  int Ts;              // row stride of s_txt
+  int passthrough;
+  float* S;
+  float* s_txt;
+  float* W;
+  float2* wstat;
+  float* ypart;
+  float2* ystat;
+  int* cnt;
+  WsLayout ws;
+};
+
+// launchers (each returns a cudaError_t from the launch)
+cudaError_t launch_scores(const DecodeArgs& a, int dtype, cudaStream_t st);
+cudaError_t launch_expand(const DecodeArgs& a, int dtype, cudaStream_t st);
+cudaError_t launch_output(const DecodeArgs& a, int dtype, cudaStream_t st);
+cudaError_t launch_compress(const kvc_layer* L, const void* K_vis, const void* V_vis, int B, int R,
+                            void* Kc, void* Vc, cudaStream_t st);
+
+}  // namespace kvc

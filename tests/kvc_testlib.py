@@ -1,0 +1,66 @@
+"""Shared helpers of the parity tests: run the CUDA path and the CPU oracle on the same buffers."""
+from __future__ import annotations
+
+import dataclasses
+
+import numpy as np
+import torch
+
+from oracle import kvcapsule_oracle as orc
+from paper_2605_16439_b200 import binding as kvc
+from paper_2605_16439_b200 import workloads as wl
+
+TOL = {"f32": 1e-4, "bf16": 2e-2}       # max-abs bounds of the benchmark spec
+
+
+def np64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to("cpu", torch.float32).numpy().astype(np.float64)
+
+
+def make_problem(shape: wl.Shape, seed: int, T=None, T_cap=None, idx=None):
+    m = orc.retained_len(shape.n, shape.ratio_permille)
+    p = wl.decode_inputs(shape, m, seed, "cpu", T, T_cap)
+    if idx is not None:
+        p["idx"] = idx
+    p["m"] = m
+    return p
+
+
+def oracle_run(shape: wl.Shape, p, form: str = "fused"):
+    """(K_tilde, V_tilde, out) in fp64 from the (already rounded) storage-dtype inputs."""
+    passthrough = shape.ratio_permille == 0
+    T = p["T"]
+    args = [np64(p[k]) for k in ("K_vis", "V_vis")]
+    K_t, V_t = orc.compress(args[0], args[1], p["idx"].numpy(), np64(p["U"]), np64(p["mu"]), shape.n, passthrough)
+    f = orc.decode_attend_fused if form == "fused" else orc.decode_attend_definition
+    out = f(np64(p["q"]), K_t, V_t, np64(p["theta"]), np64(p["U"]), np64(p["mu"]),
+            np64(p["K_txt"])[:, :, :T], np64(p["V_txt"])[:, :, :T], passthrough)
+    return K_t, V_t, out
+
+
+def gpu_layer(shape: wl.Shape, p, dev="cuda"):
+    dt = wl.torch_dtype(shape.dtype)
+    if shape.ratio_permille == 0:
+        return kvc.Layer(shape.H_q, shape.H_kv, shape.d, shape.n, 0, dt)
+    return kvc.Layer(shape.H_q, shape.H_kv, shape.d, shape.n, shape.ratio_permille, dt, idx=p["idx"],
+                     theta=p["theta"].to(dev), U=p["U"].to(dev), mu=p["mu"].to(dev))
+
+
+def gpu_run(shape: wl.Shape, p, dev="cuda"):
+    """(K_tilde, V_tilde, out) from the CUDA library through the C ABI."""
+    layer = gpu_layer(shape, p, dev)
+    B, R, T, T_cap = shape.B, shape.R, p["T"], p["T_cap"]
+    caps = kvc.alloc_capsules(layer, B, R, dev)
+    kvc.kvc_compress(layer, p["K_vis"].to(dev), p["V_vis"].to(dev), B, R, caps)
+    ws = kvc.alloc_workspace(layer, B, R, T_cap, dev)
+    out = torch.full((B, shape.H_q, shape.d), float("nan"), dtype=wl.torch_dtype(shape.dtype), device=dev)
+    K_txt = p["K_txt"].to(dev) if T_cap > 0 else None
+    V_txt = p["V_txt"].to(dev) if T_cap > 0 else None
+    kvc.kvc_decode_attend(layer, p["q"].to(dev), caps if R > 0 else None, B, R, K_txt, V_txt, T, T_cap, out, ws)
+    torch.cuda.synchronize()
+    K_t, V_t = kvc.capsule_views(layer, caps, B, R) if R > 0 else (None, None)
+    return layer, K_t, V_t, out
+
+
+def small(shape: wl.Shape, **kw) -> wl.Shape:
+    return dataclasses.replace(shape, **kw)

@@ -1,0 +1,224 @@
+"""CUDA path vs CPU oracle, element by element, on the same seeded inputs (through the C ABI).
+
+Bounds (task statement): max-abs 1e-4 for fp32 storage, 2e-2 for bf16 storage with fp32
+accumulation (end to end: compress + decode, oracle in fp64 on the bf16-rounded inputs); the
+selected key rows and the integer maps bit-exact.
+"""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import kvcapsule_oracle as orc
+from paper_2605_16439_b200 import binding as kvc
+from paper_2605_16439_b200 import build as kvc_build
+from paper_2605_16439_b200 import workloads as wl
+
+import kvc_testlib as tl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    kvc_build.build()
+
+
+def _check(shape, p, form="fused"):
+    tol = tl.TOL[shape.dtype]
+    K_o, V_o, out_o = tl.oracle_run(shape, p, form)
+    layer, K_g, V_g, out_g = tl.gpu_run(shape, p)
+    if shape.R > 0:
+        # key capsules are copies of input rows: bit-exact
+        assert np.array_equal(tl.np64(K_g), K_o)
+        # value capsules: fp32 accumulation, then one rounding to the storage type
+        v_tol = 1e-4 if shape.dtype == "f32" else 2e-2 * max(1.0, float(np.abs(V_o).max()))
+        assert np.abs(tl.np64(V_g) - V_o).max() <= v_tol
+    got = tl.np64(out_g)
+    assert np.isfinite(got).all()
+    err = np.abs(got - out_o).max()
+    assert err <= tol, f"max-abs error {err} > {tol}"
+    return err
+
+
+# ------------------------------------------------------------------ the task's configurations
+def test_config0_fp32_exact_shape():
+    shape = wl.CONFIGS[0]
+    p = tl.make_problem(shape, wl.layer_seed(0, 0))
+    _check(shape, p, "fused")
+    _check(shape, p, "definition")
+
+
+@pytest.mark.parametrize("ci,kw", [
+    (1, dict(B=2, H_q=4, H_kv=4)),              # LLaVA-NeXT shape: MHA, n=576, m=231, R=5
+    (2, dict(B=2, H_q=14, H_kv=2, R=3)),        # Qwen2-VL shape: G=7, n=1024, m=410
+    (3, dict(B=1, H_q=7, H_kv=1, R=6)),         # InternVL3 video shape: n=256, m=103, AR(1) frames
+])
+def test_reduced_7b_shapes_bf16(ci, kw):
+    shape = tl.small(wl.CONFIGS[ci], **kw)
+    p = tl.make_problem(shape, wl.layer_seed(ci, 3), T=shape.T0 + 5, T_cap=shape.T0 + 64)
+    _check(shape, p)
+
+
+@pytest.mark.parametrize("ratio", [0, 200, 400, 600, 800, 950])
+def test_ratio_sweep_bf16(ratio):
+    shape = tl.small(wl.CONFIGS[2], B=1, H_q=7, H_kv=1, R=2, grid=16, ratio_permille=ratio)
+    p = tl.make_problem(shape, 40 + ratio, T=33)
+    _check(shape, p)
+
+
+@pytest.mark.parametrize("ratio", [0, 600])
+def test_ratio_fp32(ratio):
+    shape = tl.small(wl.CONFIGS[0], B=2, R=3, grid=12, ratio_permille=ratio)
+    p = tl.make_problem(shape, 50 + ratio, T=31)
+    _check(shape, p)
+
+
+# ------------------------------------------------------------------ head grouping
+@pytest.mark.parametrize("H_q,H_kv", [(3, 3), (4, 2), (6, 2), (5, 1), (8, 1), (12, 1), (16, 1)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_gqa_group_sizes(H_q, H_kv, dtype):
+    shape = wl.Shape("gqa", 1, 2, H_q, H_kv, 128, 8, 3, 40, 1, dtype)
+    p = tl.make_problem(shape, 60 + H_q)
+    _check(shape, p)
+
+
+# ------------------------------------------------------------------ degenerate and ragged cases
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("R,T", [(0, 1), (0, 300), (1, 0), (3, 0), (2, 1), (2, 255), (2, 256), (2, 257), (1, 700)])
+def test_empty_and_ragged_sides(dtype, R, T):
+    shape = wl.Shape("edge", 1, 2, 4, 2, 128, 7, R, T, 1, dtype)          # n = 49, m = 20
+    p = tl.make_problem(shape, 70 + R * 1000 + T, T=T, T_cap=T + 3)
+    _check(shape, p)
+
+
+def test_rows_beyond_T_do_not_leak():
+    shape = wl.Shape("tcap", 1, 1, 4, 2, 128, 6, 2, 17, 1, "f32")
+    p = tl.make_problem(shape, 81, T=17, T_cap=64)
+    p["K_txt"][:, :, 17:] = 1e4
+    p["V_txt"][:, :, 17:] = float("nan")
+    _check(shape, p)
+
+
+def test_tiny_block_and_m_equal_one():
+    shape = wl.Shape("tiny", 1, 1, 2, 1, 128, 2, 3, 2, 1, "f32", ratio_permille=900)   # n = 4, m = 1
+    p = tl.make_problem(shape, 82)
+    assert p["m"] == 1
+    _check(shape, p)
+
+
+def test_large_logits_are_stable():
+    shape = wl.Shape("big", 1, 1, 4, 2, 128, 8, 2, 9, 1, "f32")
+    p = tl.make_problem(shape, 83)
+    p["q"] *= 30.0                                   # logits of a few hundred
+    _check(shape, p)
+
+
+# ------------------------------------------------------------------ index sets and integer maps
+def test_irregular_and_per_head_index_sets():
+    shape = wl.Shape("idx", 1, 2, 6, 3, 128, 9, 2, 12, 1, "bf16")
+    m = orc.retained_len(shape.n, 600)
+    for idx in (wl.random_sorted_idx(shape.n, m, 5), wl.random_sorted_idx(shape.n, m, 6, H_kv=3)):
+        p = tl.make_problem(shape, 90, idx=idx)
+        _check(shape, p)
+
+
+def test_exported_maps_are_bit_exact():
+    shape = wl.Shape("maps", 1, 1, 6, 3, 128, 10, 4, 1, 1, "f32")
+    m = orc.retained_len(shape.n, 600)
+    idx = wl.random_sorted_idx(shape.n, m, 7, H_kv=3)
+    p = tl.make_problem(shape, 91, idx=idx)
+    layer = tl.gpu_layer(shape, p)
+    assert layer.m == m == kvc.kvc_retained_len(shape.n, 600)
+    idx_out, grp = kvc.kvc_export_maps(layer, shape.R)
+    assert torch.equal(idx_out, idx)
+    assert np.array_equal(grp.numpy(), orc.grouping_map(shape.N_v, shape.n))
+    # a shared index set is broadcast to every KV head
+    p2 = tl.make_problem(shape, 91)
+    idx_out2, _ = kvc.kvc_export_maps(tl.gpu_layer(shape, p2), 0)
+    assert torch.equal(idx_out2, p2["idx"][None].expand(3, m))
+    assert kvc.kvc_capsule_bytes(layer, 5, 4) == 2 * 5 * 3 * 4 * m * 128 * 4
+
+
+# ------------------------------------------------------------------ comparator and ABI behaviour on device
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_uncompressed_comparator_matches_plain_attention(dtype):
+    dt = wl.torch_dtype(dtype)
+    B, H_q, H_kv, S, S_cap = 2, 8, 2, 1000, 1024
+    q = wl.gaussian((B, H_q, 128), 1, "cpu", dt)
+    K = wl.gaussian((B, H_kv, S_cap, 128), 2, "cpu", dt)
+    V = wl.gaussian((B, H_kv, S_cap, 128), 3, "cpu", dt)
+    layer = kvc.Layer(H_q, H_kv, 128, 64, 0, dt)
+    ws = kvc.alloc_workspace(layer, B, 0, S_cap)
+    out = torch.empty((B, H_q, 128), dtype=dt, device="cuda")
+    kvc.kvc_attend_full(layer, q.cuda(), K.cuda(), V.cuda(), B, S, S_cap, out, ws)
+    torch.cuda.synchronize()
+    want = orc.attention(tl.np64(q), tl.np64(K)[:, :, :S], tl.np64(V)[:, :, :S])
+    assert np.abs(tl.np64(out) - want).max() <= tl.TOL[dtype]
+
+
+def test_device_side_argument_errors_and_noops():
+    shape = wl.Shape("err", 1, 1, 4, 2, 128, 4, 1, 4, 1, "f32")
+    p = tl.make_problem(shape, 95)
+    layer = tl.gpu_layer(shape, p)
+    caps = kvc.alloc_capsules(layer, 1, 1)
+    ws = kvc.alloc_workspace(layer, 1, 1, 4)
+    out = torch.zeros((1, 4, 128), device="cuda")
+    q = p["q"].cuda()
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_decode_attend(layer, q, caps, 1, 0, None, None, 0, 0, out, ws)
+    assert e.value.status == -2                                            # nothing to attend over
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_decode_attend(layer, q, caps, 1, 1, None, None, 0, 0, out, None)
+    assert e.value.status == -5
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_decode_attend(layer, q, caps, 1, 1, None, None, 3, 4, out, ws)
+    assert e.value.status == -1                                            # T > 0 but no text K/V
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_decode_attend(layer, q, caps, 1, 1, q, q, 5, 4, out, ws)
+    assert e.value.status == -1                                            # T > T_cap
+    kvc.kvc_decode_attend(layer, q, caps, 0, 1, None, None, 0, 0, out, ws)   # B == 0: no-op
+    kvc.kvc_compress(layer, None, None, 0, 1, None)                          # no-op
+    torch.cuda.synchronize()
+    assert float(out.abs().sum()) == 0.0
+
+
+def test_repeat_calls_are_bitwise_deterministic_and_workspace_needs_no_init():
+    shape = tl.small(wl.CONFIGS[2], B=2, H_q=14, H_kv=2, R=2, grid=16)
+    p = tl.make_problem(shape, 96, T=70)
+    layer = tl.gpu_layer(shape, p)
+    B, R = shape.B, shape.R
+    caps = kvc.alloc_capsules(layer, B, R)
+    kvc.kvc_compress(layer, p["K_vis"].cuda(), p["V_vis"].cuda(), B, R, caps)
+    ws = kvc.alloc_workspace(layer, B, R, 70)
+    q, Kt, Vt = p["q"].cuda(), p["K_txt"].cuda(), p["V_txt"].cuda()
+    outs = []
+    for fill in (0x00, 0xFF, 0x7F):
+        ws.fill_(fill)                               # poison: the call may not depend on old contents
+        out = torch.empty((B, shape.H_q, 128), dtype=torch.bfloat16, device="cuda")
+        kvc.kvc_decode_attend(layer, q, caps, B, R, Kt, Vt, 70, 70, out, ws)
+        outs.append(out.clone())
+    torch.cuda.synchronize()
+    assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16))
+    assert torch.equal(outs[0].view(torch.int16), outs[2].view(torch.int16))
+
+
+def test_decode_steps_with_growing_text_tail():
+    """A few decode steps: the text tail grows by one row per step inside a fixed-capacity buffer."""
+    shape = tl.small(wl.CONFIGS[1], B=1, H_q=2, H_kv=2, R=2, grid=8)
+    T0, steps = 30, 4
+    p = tl.make_problem(shape, 97, T=T0 + steps, T_cap=T0 + steps)
+    layer = tl.gpu_layer(shape, p)
+    caps = kvc.alloc_capsules(layer, 1, 2)
+    kvc.kvc_compress(layer, p["K_vis"].cuda(), p["V_vis"].cuda(), 1, 2, caps)
+    ws = kvc.alloc_workspace(layer, 1, 2, T0 + steps)
+    Kt, Vt, q = p["K_txt"].cuda(), p["V_txt"].cuda(), p["q"].cuda()
+    for s in range(steps):
+        T = T0 + s
+        out = torch.empty((1, 2, 128), dtype=torch.bfloat16, device="cuda")
+        kvc.kvc_decode_attend(layer, q, caps, 1, 2, Kt, Vt, T, T0 + steps, out, ws)
+        torch.cuda.synchronize()
+        ps = dict(p); ps["T"] = T
+        _, _, want = tl.oracle_run(shape, ps)
+        assert np.abs(tl.np64(out) - want).max() <= tl.TOL["bf16"]
