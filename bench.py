@@ -1,0 +1,457 @@
+"""Benchmark of the KVCapsule decode hot path on B200: capsule compress + fused reconstruct/decode attention.
+
+One bench "step" is one pass of the whole hot path over one batch of synthetic sequences: every
+layer's vision K/V is compressed once (prefill stage), then `decode_steps` decode steps run, each
+calling the fused decode attention of every layer with the text tail one row longer than the step
+before.  `value` is decode tokens/s of the whole job: sequences x decode steps / time.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 1]
+
+Under torchrun (N > 1) every rank runs the same per-GPU batch on its own GPU (weak scaling, no
+data-path collective: sequences are independent); time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch
+
+from paper_2605_16439_b200 import workloads as wl
+
+FALLBACK_HBM_GBS = 6650.0       # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
+NOMINAL_HBM_GBS = 8000.0        # the figure the task's metric quotes its percentage against
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
+# the ncu capture summarised under profiles/, keyed by (kernel, workload name); None = not captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--config", type=int, default=1, help="index into the task's configurations (1 = LLaVA-NeXT-7B shape)")
+    ap.add_argument("--decode-steps", type=int, default=None, help="override the configuration's decode steps")
+    ap.add_argument("--layers", type=int, default=None)
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--ratio", type=int, default=None, help="compression ratio in permille")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-comparator", action="store_true")
+    ap.add_argument("--no-profile", action="store_true", help="do not bracket kernels with events in the timed region")
+    ap.add_argument("--oracle-decode-steps", type=int, default=8)
+    return ap.parse_args()
+
+
+def pick_shape(a) -> wl.Shape:
+    s = wl.CONFIGS[a.config]
+    kw = {}
+    if a.decode_steps is not None: kw["steps"] = a.decode_steps
+    if a.layers is not None: kw["layers"] = a.layers
+    if a.batch is not None: kw["B"] = a.batch
+    if a.ratio is not None: kw["ratio_permille"] = a.ratio
+    return dataclasses.replace(s, **kw)
+
+
+def elem_bytes(shape) -> int:
+    return 2 if shape.dtype == "bf16" else 4
+
+
+def contract_bytes_per_layer_call(shape, m, T) -> int:
+    """Capsule bytes + text-KV bytes + Q/O bytes of one kvc_decode_attend call."""
+    b = elem_bytes(shape)
+    return (2 * shape.B * shape.H_kv * shape.R * m * shape.d * b + 2 * shape.B * shape.H_kv * T * shape.d * b
+            + 2 * shape.B * shape.H_q * shape.d * b)
+
+
+def stream_kernel_bytes(shape, m, T) -> int:
+    """Algorithmic bytes of ONE launch of the scores (or output) kernel: one of K_tilde/V_tilde, one of the
+    text K/V, and q (or out)."""
+    b = elem_bytes(shape)
+    return (shape.B * shape.H_kv * (shape.R * m + T) * shape.d * b + shape.B * shape.H_q * shape.d * b)
+
+
+# --------------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu, self.proc, self.path = gpu_index, None, None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)], stdout=f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                c = [x.strip() for x in line.split(",")]
+                if len(c) < 9:
+                    continue
+                try:
+                    sm.append(float(c[1])); mx.append(float(c[2]))
+                except ValueError:
+                    continue
+                for nm, v in zip(names, c[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(nm)
+        os.unlink(self.path)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------- GPU arm
+class Job:
+    """All device state of one rank's batch: per-layer inputs, parameters, capsule stores, text tails."""
+
+    def __init__(self, shape: wl.Shape, config_index: int, dev, rank: int):
+        from paper_2605_16439_b200 import binding as kvc
+        self.kvc, self.shape, self.dev = kvc, shape, dev
+        dt = wl.torch_dtype(shape.dtype)
+        self.m = kvc.kvc_retained_len(shape.n, shape.ratio_permille)
+        self.T_cap = shape.T0 + shape.steps
+        self.layers = []
+        for l in range(shape.layers):
+            seed = wl.layer_seed(config_index, l) + 100000 * rank
+            p = wl.decode_inputs(shape, self.m, seed, dev, T=shape.T0, T_cap=self.T_cap)
+            if shape.ratio_permille == 0:
+                layer = kvc.Layer(shape.H_q, shape.H_kv, shape.d, shape.n, 0, dt, layer=l)
+            else:
+                layer = kvc.Layer(shape.H_q, shape.H_kv, shape.d, shape.n, shape.ratio_permille, dt, idx=p["idx"],
+                                  theta=p["theta"], U=p["U"], mu=p["mu"], layer=l)
+            p["layer"] = layer
+            p["caps"] = kvc.alloc_capsules(layer, shape.B, shape.R, dev)
+            p["out"] = torch.zeros((shape.B, shape.H_q, shape.d), dtype=dt, device=dev)
+            self.layers.append(p)
+        self.ws = kvc.alloc_workspace(self.layers[0]["layer"], shape.B, shape.R, self.T_cap, dev)
+        self.launches = 0
+
+    def compress_all(self):
+        s = self.shape
+        for p in self.layers:
+            self.kvc.kvc_compress(p["layer"], p["K_vis"], p["V_vis"], s.B, s.R, p["caps"])
+        self.launches += (0 if s.ratio_permille == 0 else 2) * len(self.layers)
+
+    def decode_step(self, t: int):
+        s = self.shape
+        T = s.T0 + t
+        for p in self.layers:
+            self.kvc.kvc_decode_attend(p["layer"], p["q"], p["caps"], s.B, s.R, p["K_txt"], p["V_txt"], T,
+                                       self.T_cap, p["out"], self.ws)
+        self.launches += 3 * len(self.layers)
+
+    def step(self):
+        self.compress_all()
+        for t in range(self.shape.steps):
+            self.decode_step(t)
+
+
+def timed(fn, reps: int, dev) -> float:
+    """Milliseconds of `reps` calls of fn on the current stream, device-timed."""
+    st, en = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    st.record()
+    for _ in range(reps):
+        fn()
+    en.record()
+    torch.cuda.synchronize(dev)
+    return st.elapsed_time(en)
+
+
+def run_e2e(job: Job, dev) -> dict:
+    """The same job driven from HOST buffers: per step the vision K/V of every layer, and per decode step
+    and layer the query and the new text K/V row, are copied from pinned host memory, and the attention
+    output is copied back, all inside the timed region."""
+    s, kvc = job.shape, job.kvc
+    dt = wl.torch_dtype(s.dtype)
+    host = []
+    for p in job.layers:
+        host.append(dict(K_vis=p["K_vis"].to("cpu").pin_memory(), V_vis=p["V_vis"].to("cpu").pin_memory(),
+                         q=p["q"].to("cpu").pin_memory(),
+                         k_row=p["K_txt"][:, :, 0].contiguous().to("cpu").pin_memory(),
+                         v_row=p["V_txt"][:, :, 0].contiguous().to("cpu").pin_memory(),
+                         out=torch.empty((s.B, s.H_q, s.d), dtype=dt).pin_memory()))
+    h2d = d2h = 0
+
+    def one_step():
+        nonlocal h2d, d2h
+        h2d = d2h = 0
+        for p, h in zip(job.layers, host):
+            p["K_vis"].copy_(h["K_vis"], non_blocking=True)
+            p["V_vis"].copy_(h["V_vis"], non_blocking=True)
+            h2d += h["K_vis"].numel() * h["K_vis"].element_size() * 2
+            kvc.kvc_compress(p["layer"], p["K_vis"], p["V_vis"], s.B, s.R, p["caps"])
+        for t in range(s.steps):
+            T = s.T0 + t
+            for p, h in zip(job.layers, host):
+                p["q"].copy_(h["q"], non_blocking=True)
+                p["K_txt"][:, :, T - 1].copy_(h["k_row"], non_blocking=True)
+                p["V_txt"][:, :, T - 1].copy_(h["v_row"], non_blocking=True)
+                kvc.kvc_decode_attend(p["layer"], p["q"], p["caps"], s.B, s.R, p["K_txt"], p["V_txt"], T, job.T_cap,
+                                      p["out"], job.ws)
+                h["out"].copy_(p["out"], non_blocking=True)
+                h2d += (h["q"].numel() + 2 * h["k_row"].numel()) * h["q"].element_size()
+                d2h += h["out"].numel() * h["out"].element_size()
+
+    one_step()                                   # warm-up (also pages the pinned buffers in)
+    torch.cuda.synchronize(dev)
+    t0 = time.perf_counter()
+    ms = timed(one_step, 1, dev)
+    wall = (time.perf_counter() - t0) * 1e3
+    ms = max(ms, wall)                           # host-side copies and launches count end to end
+    return {"ms": ms, "h2d": h2d, "d2h": d2h}
+
+
+def run_comparator(shape: wl.Shape, dev, reps_layers: int = 8, steps: int = 16) -> dict:
+    """Our own uncompressed decode attention (kvc_attend_full) over full vision + text K/V of the same shape."""
+    from paper_2605_16439_b200 import binding as kvc
+    dt = wl.torch_dtype(shape.dtype)
+    S_cap = shape.N_v + shape.T0 + shape.steps
+    nl = min(reps_layers, shape.layers)
+    layer = kvc.Layer(shape.H_q, shape.H_kv, shape.d, shape.n, 0, dt)
+    bufs = []
+    for l in range(nl):
+        bufs.append((wl.gaussian((shape.B, shape.H_kv, S_cap, shape.d), 900 + l, dev, dt),
+                     wl.gaussian((shape.B, shape.H_kv, S_cap, shape.d), 950 + l, dev, dt),
+                     wl.gaussian((shape.B, shape.H_q, shape.d), 990 + l, dev, dt)))
+    ws = kvc.alloc_workspace(layer, shape.B, 0, S_cap, dev)
+    out = torch.empty((shape.B, shape.H_q, shape.d), dtype=dt, device=dev)
+    S_mid = shape.N_v + shape.T0 + shape.steps // 2
+
+    def run():
+        for _ in range(steps):
+            for K, V, q in bufs:
+                kvc.kvc_attend_full(layer, q, K, V, shape.B, S_mid, S_cap, out, ws)
+    run()
+    ms = timed(run, 1, dev)
+    per_layer_ms = ms / (steps * nl)
+    step_ms = per_layer_ms * shape.layers
+    bytes_call = 2 * shape.B * shape.H_kv * S_mid * shape.d * elem_bytes(shape)
+    return {"kernel": "kvc_attend_full (uncompressed, our own)", "ms_per_layer_call": per_layer_ms,
+            "tokens_per_s": shape.B / (step_ms * 1e-3), "hbm_gbs": bytes_call / (per_layer_ms * 1e-3) / 1e9,
+            "kv_len": S_mid, "sample": f"{nl} distinct layers x {steps} calls at the mid-run text length"}
+
+
+# --------------------------------------------------------------------------------------------- CPU oracle arm
+def oracle_sample(shape: wl.Shape, config_index: int, decode_steps: int) -> dict:
+    """Times the CPU oracle, as it stands, on ONE layer: one compress plus `decode_steps` decode steps of
+    Algorithm 1's order, and scales to the full job (layers x steps) by the per-call averages."""
+    import numpy as np
+    from oracle import kvcapsule_oracle as orc
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    m = orc.retained_len(shape.n, shape.ratio_permille)
+    T_cap = shape.T0 + shape.steps
+    p = wl.decode_inputs(shape, m, wl.layer_seed(config_index, 0), "cpu", T=shape.T0, T_cap=T_cap)
+    f64 = lambda t: t.float().numpy().astype(np.float64)
+    a = {k: f64(p[k]) for k in ("K_vis", "V_vis", "K_txt", "V_txt", "q", "theta", "U", "mu")}
+    passthrough = shape.ratio_permille == 0
+    t0 = time.perf_counter()
+    K_t, V_t = orc.compress(a["K_vis"], a["V_vis"], p["idx"].numpy(), a["U"], a["mu"], shape.n, passthrough)
+    t_comp = time.perf_counter() - t0
+    ts = []
+    stride = max(1, shape.steps // decode_steps)
+    for t in list(range(0, shape.steps, stride))[:decode_steps]:
+        T = shape.T0 + t
+        t0 = time.perf_counter()
+        orc.decode_attend_fused(a["q"], K_t, V_t, a["theta"], a["U"], a["mu"], a["K_txt"][:, :, :T],
+                                a["V_txt"][:, :, :T], passthrough)
+        ts.append(time.perf_counter() - t0)
+    t_dec = sum(ts) / len(ts)
+    total = shape.layers * (t_comp + shape.steps * t_dec)
+    return {"value": shape.B * shape.steps / total, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+            "sample": (f"1 of {shape.layers} layers, full batch: 1 compress ({t_comp:.2f} s) + {len(ts)} of "
+                       f"{shape.steps} decode steps spread over the run ({t_dec * 1e3:.0f} ms each); scaled to "
+                       f"layers x steps"),
+            "cpu_seconds": t_comp + sum(ts)}
+
+
+def config_dict(shape: wl.Shape, m: int, extra=None) -> dict:
+    c = {"workload": shape.name, "layers": shape.layers, "batch_per_gpu": shape.B, "H_q": shape.H_q,
+         "H_kv": shape.H_kv, "d": shape.d, "n": shape.n, "R": shape.R, "m": m,
+         "ratio": shape.ratio_permille / 1000.0, "text_tokens": f"{shape.T0}->{shape.T0 + shape.steps}",
+         "decode_steps": shape.steps,
+         "l2": "inputs larger than L2: every layer call streams its own >126 MB of capsules and text K/V"}
+    if extra:
+        c.update(extra)
+    return c
+
+
+def run_reference(a, shape, rank):
+    if rank != 0:
+        return
+    from oracle import kvcapsule_oracle as orc
+    m = orc.retained_len(shape.n, shape.ratio_permille)
+    nd = max(2, a.oracle_decode_steps // 2)
+    for _ in range(a.warmup if a.warmup < 2 else 1):
+        oracle_sample(shape, a.config, 1)
+    vals = [oracle_sample(shape, a.config, nd) for _ in range(a.steps)]
+    v = statistics.mean(x["value"] for x in vals)
+    line = {"impl": "reference", "metric": "decode tokens/s", "value": v, "unit": "tokens/s", "n_gpus": a.gpus,
+            "steps": a.steps, "warmup": a.warmup, "ms_per_step": shape.B * shape.steps / v * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_dict(shape, m),
+            "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": vals[0]["cores"], "kind": "oracle",
+                             "sample": vals[0]["sample"]},
+            "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    a = parse_args()
+    shape = pick_shape(a)
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if a.impl == "reference":
+        run_reference(a, shape, rank)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    from paper_2605_16439_b200 import build as kvc_build
+    if rank == 0 or not os.path.exists(kvc_build.LIB):
+        kvc_build.build()
+    import torch.distributed as dist
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    from paper_2605_16439_b200 import binding as kvc
+
+    job = Job(shape, a.config, dev, rank)
+    m = job.m
+    for _ in range(max(a.warmup, 3)):
+        job.step()
+    torch.cuda.synchronize(dev)
+
+    calls = shape.layers * shape.steps
+    if not a.no_profile:
+        kvc.kvc_profile_start(a.steps * (3 * calls + 2 * shape.layers))
+    job.launches = 0
+    sampler = ClockSampler(local)
+    if world > 1:
+        dist.barrier()
+    sampler.start()
+    ms = timed(job.step, a.steps, dev)
+    clocks = sampler.stop()
+    if world > 1:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.barrier()
+        ms = float(t.item())
+    prof = {}
+    if not a.no_profile:
+        kvc.kvc_profile_stop()
+        prof = kvc.kvc_profile_read()
+        kvc.kvc_profile_start(0)
+        kvc.kvc_profile_stop()
+    launches = job.launches
+
+    ms_step = ms / a.steps
+    tokens_per_s = world * shape.B * shape.steps / (ms_step * 1e-3)
+
+    # decode-only and compress-only figures (context for the whole-step value)
+    ms_compress = timed(job.compress_all, 1, dev)
+    ms_decode = timed(lambda: [job.decode_step(t) for t in range(shape.steps)], 1, dev)
+    T_mid = shape.T0 + (shape.steps - 1) / 2.0
+    contract = contract_bytes_per_layer_call(shape, m, T_mid)
+    decode_gbs = contract * calls / (ms_decode * 1e-3) / 1e9
+
+    # roofline of the dominant kernel, from the event brackets recorded inside the timed region
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    else:
+        peak, peak_src = FALLBACK_HBM_GBS, "fallback"
+    roofline = None
+    kernels = {}
+    if prof:
+        tot = sum(v[0] for v in prof.values()) or 1.0
+        for k, (t, n) in prof.items():
+            if n:
+                kernels[k] = {"launches": n, "total_ms": round(t, 3), "avg_us": round(t / n * 1e3, 3),
+                              "share": round(t / tot, 4)}
+        dom = max(("scores", "output"), key=lambda k: prof[k][0])
+        t_dom, n_dom = prof[dom]
+        alg = stream_kernel_bytes(shape, m, T_mid)
+        achieved = alg / (t_dom / n_dom * 1e-3) / 1e9
+        traffic = NCU_TRAFFIC_BYTES.get((dom, shape.name))
+        roofline = {"kernel": dom, "bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                    "frac": round(achieved / peak, 4), "traffic": traffic, "peak_source": peak_src,
+                    "algorithmic_bytes_per_launch": int(alg), "avg_launch_us": round(t_dom / n_dom * 1e3, 3)}
+
+    line = {"metric": "decode tokens/s", "value": round(tokens_per_s, 2), "unit": "tokens/s", "n_gpus": world,
+            "steps": a.steps, "warmup": max(a.warmup, 3), "ms_per_step": round(ms_step, 3),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": shape.dtype,
+            "data": "synthetic", "config": config_dict(shape, m, {"global_batch": world * shape.B,
+                                                                   "parallelism": f"batch-sharded x{world}"}),
+            "clocks": clocks, "gpu_launches": launches,
+            "ms_per_decode_step": round(ms_decode / shape.steps, 4),
+            "ms_per_layer_call": round(ms_decode / calls, 5),
+            "ms_compress_all_layers": round(ms_compress, 3),
+            "decode_contract_gbs": round(decode_gbs, 1),
+            "decode_frac_of_8tbs": round(decode_gbs / NOMINAL_HBM_GBS, 4),
+            "decode_frac_of_measured_peak": round(decode_gbs / peak, 4),
+            "kernels": kernels, "roofline": roofline}
+
+    if rank == 0 and world == 1:
+        if not a.no_comparator:
+            line["comparator"] = run_comparator(shape, dev)
+        if not a.no_e2e:
+            e = run_e2e(job, dev)
+            line["e2e"] = {"value": round(shape.B * shape.steps / (e["ms"] * 1e-3), 2), "unit": "tokens/s",
+                           "h2d_bytes_per_step": e["h2d"], "d2h_bytes_per_step": e["d2h"],
+                           "ms_per_step": round(e["ms"], 3)}
+        if not a.no_cpu_baseline:
+            line["cpu_baseline"] = oracle_sample(shape, a.config, a.oracle_decode_steps)
+    elif world > 1 and not a.no_e2e:
+        e = run_e2e(job, dev)
+        t = torch.tensor([e["ms"]], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        line["e2e"] = {"value": round(world * shape.B * shape.steps / (float(t.item()) * 1e-3), 2),
+                       "unit": "tokens/s", "h2d_bytes_per_step": e["h2d"], "d2h_bytes_per_step": e["d2h"]}
+    line["paper_context"] = "paper: up to 2x decode TPS and 2.4x KV memory at 60% (AMD MI250X, Torch-level); context only"
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

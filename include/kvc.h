@@ -128,6 +128,26 @@ KVC_API int kvc_layer_m(const kvc_layer* layer);
 
 KVC_API const char* kvc_strerror(int status);
 
+/* ---- optional instrumentation (measurement only; the paper has no counterpart) -------------
+ * While profiling is on, every kernel the library launches is bracketed by two CUDA events
+ * recorded on the launching stream, until max_launches brackets have been used.  Global,
+ * not thread-safe, and meant for benchmarks: the events serialise nothing but add a little
+ * launch work.  kvc_profile_read sums, for one kernel id, the elapsed time of its brackets;
+ * call it after the stream has been synchronised.  kvc_profile_start allocates host-side
+ * event objects only. */
+typedef enum {
+  KVC_KERNEL_SCORES = 0,          /* Alg. 1 step 1 + text logits  */
+  KVC_KERNEL_EXPAND = 1,          /* Alg. 1 steps 2-3             */
+  KVC_KERNEL_OUTPUT = 2,          /* Alg. 1 step 4 + text + merge */
+  KVC_KERNEL_GATHER_KEYS = 3,     /* key row selection            */
+  KVC_KERNEL_PROJECT_VALUES = 4,  /* value centre + project       */
+  KVC_KERNEL_COUNT = 5
+} kvc_kernel_id;
+KVC_API int kvc_profile_start(int max_launches);
+KVC_API int kvc_profile_stop(void);
+KVC_API int kvc_profile_read(int kernel_id, double* total_ms, long long* launches);
+KVC_API const char* kvc_kernel_name(int kernel_id);
+
 #ifdef __cplusplus
 }
 #endif

@@ -54,6 +54,11 @@ def _lib() -> C.CDLL:
         lib.kvc_export_maps.argtypes = [vp, i, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         lib.kvc_export_maps.restype = i
         lib.kvc_strerror.argtypes = [i]; lib.kvc_strerror.restype = C.c_char_p
+        lib.kvc_profile_start.argtypes = [i]; lib.kvc_profile_start.restype = i
+        lib.kvc_profile_stop.argtypes = []; lib.kvc_profile_stop.restype = i
+        lib.kvc_profile_read.argtypes = [i, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
+        lib.kvc_profile_read.restype = i
+        lib.kvc_kernel_name.argtypes = [i]; lib.kvc_kernel_name.restype = C.c_char_p
         _LIB = lib
     return _LIB
 
@@ -161,3 +166,24 @@ def capsule_views(layer: Layer, capsules, B: int, R: int):
     half = kvc_capsule_bytes(layer, B, R) // 2
     shape = (B, layer.H_kv, R, layer.m, layer.d)
     return (capsules[:half].view(layer.dtype).view(shape), capsules[half:2 * half].view(layer.dtype).view(shape))
+
+
+KVC_KERNEL_COUNT = 5
+
+
+def kvc_profile_start(max_launches: int) -> None:
+    _check(_lib().kvc_profile_start(max_launches), "kvc_profile_start")
+
+
+def kvc_profile_stop() -> None:
+    _check(_lib().kvc_profile_stop(), "kvc_profile_stop")
+
+
+def kvc_profile_read() -> dict:
+    """{kernel name: (total_ms, launches)} of the bracketed launches; synchronise the stream first."""
+    out = {}
+    for k in range(KVC_KERNEL_COUNT):
+        ms, n = C.c_double(), C.c_longlong()
+        _check(_lib().kvc_profile_read(k, C.byref(ms), C.byref(n)), "kvc_profile_read")
+        out[_lib().kvc_kernel_name(k).decode()] = (ms.value, n.value)
+    return out

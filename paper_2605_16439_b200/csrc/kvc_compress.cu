@@ -74,10 +74,15 @@ static cudaError_t launch_compress_t(const kvc_layer* L, const void* K_vis, cons
   const int H_kv = L->desc.H_kv, n = L->desc.n, m = L->m;
   const long long total_rows = (long long)B * H_kv * R * m;
   const long long warps = (total_rows + RPI - 1) / RPI;
-  gather_keys_kernel<T><<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(
-      static_cast<const T*>(K_vis), static_cast<T*>(Kc), L->d_idx, H_kv, R, n, m, total_rows);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e;
+  {
+    ProfScope prof(KVC_KERNEL_GATHER_KEYS, st);
+    gather_keys_kernel<T><<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(
+        static_cast<const T*>(K_vis), static_cast<T*>(Kc), L->d_idx, H_kv, R, n, m, total_rows);
+    e = cudaGetLastError();
+  }
   if (e != cudaSuccess) return e;
+  ProfScope prof(KVC_KERNEL_PROJECT_VALUES, st);
   dim3 grid((unsigned)(B * H_kv * R), (unsigned)ceil_div(m, 32));
   project_values_kernel<T><<<grid, 256, 0, st>>>(static_cast<const T*>(V_vis), static_cast<T*>(Vc),
                                                  static_cast<const T*>(L->desc.U),

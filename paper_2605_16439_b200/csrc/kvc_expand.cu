@@ -155,6 +155,7 @@ static cudaError_t launch_expand_t(const DecodeArgs& a, cudaStream_t st) {
 
 cudaError_t launch_expand(const DecodeArgs& a, int dtype, cudaStream_t st) {
   if (a.R == 0) return cudaSuccess;
+  ProfScope prof(KVC_KERNEL_EXPAND, st);
   if (a.passthrough) {
     const int nrows = a.H_kv * a.B * a.G * a.R;
     passthrough_softmax_kernel<<<ceil_div(nrows, 8), 256, 0, st>>>(a);

@@ -102,6 +102,15 @@ struct DecodeArgs {
   WsLayout ws;
 };
 
+// optional event brackets around a launch (kvc_profile_*)
+bool prof_begin(int kernel_id, cudaStream_t st);
+void prof_end(cudaStream_t st);
+struct ProfScope {
+  cudaStream_t st; bool on;
+  ProfScope(int kernel_id, cudaStream_t s) : st(s), on(prof_begin(kernel_id, s)) {}
+  ~ProfScope() { if (on) prof_end(st); }
+};
+
 // launchers (each returns a cudaError_t from the launch)
 cudaError_t launch_scores(const DecodeArgs& a, int dtype, cudaStream_t st);
 cudaError_t launch_expand(const DecodeArgs& a, int dtype, cudaStream_t st);

@@ -190,6 +190,7 @@ static cudaError_t launch_output_t(const DecodeArgs& a, cudaStream_t st) {
 }
 
 cudaError_t launch_output(const DecodeArgs& a, int dtype, cudaStream_t st) {
+  ProfScope prof(KVC_KERNEL_OUTPUT, st);
   return dtype == KVC_BF16 ? launch_output_t<__nv_bfloat16>(a, st) : launch_output_t<float>(a, st);
 }
 

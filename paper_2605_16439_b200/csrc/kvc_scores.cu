@@ -91,6 +91,7 @@ static cudaError_t launch_scores_t(const DecodeArgs& a, cudaStream_t st) {
   const int tiles_txt = ceil_div(a.T, SCORE_TILE_ROWS);
   const unsigned grid = (unsigned)(a.B * a.H_kv * (tiles_vis + tiles_txt));
   if (grid == 0) return cudaSuccess;
+  ProfScope prof(KVC_KERNEL_SCORES, st);
   if (a.G == 1) scores_kernel<T, 1><<<grid, 256, 0, st>>>(a, tiles_vis, tiles_txt);
   else if (a.G == 2) scores_kernel<T, 2><<<grid, 256, 0, st>>>(a, tiles_vis, tiles_txt);
   else if (a.G <= 4) scores_kernel<T, 4><<<grid, 256, 0, st>>>(a, tiles_vis, tiles_txt);
