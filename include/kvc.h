@@ -118,6 +118,30 @@ KVC_API int kvc_decode_attend(const kvc_layer* layer, const void* q, const void*
 KVC_API int kvc_attend_full(const kvc_layer* layer, const void* q, const void* K, const void* V, int B,
                     int S, int S_cap, void* out, void* workspace, void* stream);
 
+/* Decode attention without a caller-provided scratch buffer (an addition of this library; the
+ * paper has no counterpart).  Same arguments, result and errors as kvc_decode_attend, minus the
+ * workspace: the temporaries go to a fixed KVC_STATIC_SCRATCH_BYTES array inside the library's
+ * device image, so the call performs no device allocation of any kind.  It is meant for callers
+ * that cannot allocate where they decode: an engine whose memory pool is fully committed to KV
+ * blocks, code running under an allocator it does not own, or a loop in which an allocation's
+ * implicit device synchronisation is unacceptable.
+ *   - Limit: the shape must need at most KVC_STATIC_SCRATCH_BYTES of scratch (what
+ *     kvc_workspace_bytes(layer, B, R, T) reports); larger shapes return KVC_ERR_WORKSPACE
+ *     ("workspace ...: static scratch too small") and nothing is launched.
+ *   - The array costs KVC_STATIC_SCRATCH_BYTES of device memory on every GPU that loads the
+ *     library, for the life of the process.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps the previous call's contents.  The
+ *     kernels clear the few words that must start at zero themselves, so no reset is needed,
+ *     but two calls whose kernels overlap on the GPU (different streams, no ordering) race on it:
+ *     order them on one stream or with events. */
+#define KVC_STATIC_SCRATCH_BYTES (16u << 20)
+KVC_API size_t kvc_static_scratch_bytes(void);
+KVC_API int kvc_decode_attend_static(const kvc_layer* layer, const void* q, const void* capsules, int B,
+                                     int R, const void* K_txt, const void* V_txt, int T, int T_cap,
+                                     void* out, void* stream);
+
 /* Integer maps as the device path uses them (read back from the device copy):
  * idx_out: HOST [H_kv][m] retained indices per KV head; group_out: HOST [R*n][2] = (block r,
  * offset i) of vision token t = r*n + i (the Reshape of Alg. 1 step 1).  Either may be NULL. */

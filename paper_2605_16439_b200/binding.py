@@ -51,6 +51,9 @@ def _lib() -> C.CDLL:
         lib.kvc_decode_attend.argtypes = [vp, vp, vp, i, i, vp, vp, i, i, vp, vp, vp]
         lib.kvc_decode_attend.restype = i
         lib.kvc_attend_full.argtypes = [vp, vp, vp, vp, i, i, i, vp, vp, vp]; lib.kvc_attend_full.restype = i
+        lib.kvc_decode_attend_static.argtypes = [vp, vp, vp, i, i, vp, vp, i, i, vp, vp]
+        lib.kvc_decode_attend_static.restype = i
+        lib.kvc_static_scratch_bytes.argtypes = []; lib.kvc_static_scratch_bytes.restype = C.c_size_t
         lib.kvc_export_maps.argtypes = [vp, i, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         lib.kvc_export_maps.restype = i
         lib.kvc_strerror.argtypes = [i]; lib.kvc_strerror.restype = C.c_char_p
@@ -145,6 +148,19 @@ def kvc_decode_attend(layer: Layer, q, capsules, B: int, R: int, K_txt, V_txt, T
                       workspace, stream=None) -> None:
     _check(_lib().kvc_decode_attend(layer.handle, _ptr(q), _ptr(capsules), B, R, _ptr(K_txt), _ptr(V_txt), T,
                                     T_cap, _ptr(out), _ptr(workspace), _stream(stream)), "kvc_decode_attend")
+
+
+def kvc_decode_attend_static(layer: Layer, q, capsules, B: int, R: int, K_txt, V_txt, T: int, T_cap: int, out,
+                             stream=None) -> None:
+    """kvc_decode_attend for callers that cannot allocate a workspace: the scratch is a fixed array inside the
+    library (kvc_static_scratch_bytes() bytes); larger shapes raise KvcError(-5).  Calls on one device share
+    that array, so keep them stream-ordered."""
+    _check(_lib().kvc_decode_attend_static(layer.handle, _ptr(q), _ptr(capsules), B, R, _ptr(K_txt), _ptr(V_txt),
+                                           T, T_cap, _ptr(out), _stream(stream)), "kvc_decode_attend_static")
+
+
+def kvc_static_scratch_bytes() -> int:
+    return _lib().kvc_static_scratch_bytes()
 
 
 def kvc_attend_full(layer: Layer, q, K, V, B: int, S: int, S_cap: int, out, workspace, stream=None) -> None:

@@ -59,7 +59,7 @@ const char* kvc_strerror(int s) {
     case KVC_ERR_SHAPE: return "unsupported or inconsistent shape";
     case KVC_ERR_DTYPE: return "unknown dtype";
     case KVC_ERR_NO_PARAMS: return "theta / U / mu / idx missing for a compression ratio > 0";
-    case KVC_ERR_WORKSPACE: return "workspace null or not 256-byte aligned";
+    case KVC_ERR_WORKSPACE: return "workspace null, not 256-byte aligned, or static scratch too small for this shape";
     case KVC_ERR_CUDA: return "CUDA runtime error";
     case KVC_ERR_TIMEOUT: return "bounded device-side wait gave up";
     case KVC_ERR_BOUNDS: return "index set entry out of range or not strictly increasing";
@@ -146,9 +146,11 @@ int kvc_compress(const kvc_layer* L, const void* K_vis, const void* V_vis, int B
   return e == cudaSuccess ? KVC_OK : KVC_ERR_CUDA;
 }
 
-static int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B, int R,
-                         const void* K_txt, const void* V_txt, int T, int T_cap, void* out, void* workspace,
-                         cudaStream_t st) {
+}  // extern "C"
+
+namespace kvc {
+int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B, int R, const void* K_txt,
+                  const void* V_txt, int T, int T_cap, void* out, void* workspace, cudaStream_t st) {
   if (!L || B < 0 || R < 0 || T < 0 || T_cap < T) return KVC_ERR_ARG;
   if (B == 0) return KVC_OK;
   if (R == 0 && T == 0) return KVC_ERR_SHAPE;
@@ -181,6 +183,9 @@ static int decode_common(const kvc_layer* L, const void* q, const void* capsules
   if (e == cudaSuccess) e = launch_output(a, L->desc.dtype, st);
   return e == cudaSuccess ? KVC_OK : KVC_ERR_CUDA;
 }
+}  // namespace kvc
+
+extern "C" {
 
 int kvc_decode_attend(const kvc_layer* L, const void* q, const void* capsules, int B, int R, const void* K_txt,
                       const void* V_txt, int T, int T_cap, void* out, void* workspace, void* stream) {

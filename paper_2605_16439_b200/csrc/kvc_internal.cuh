@@ -102,6 +102,11 @@ struct DecodeArgs {
   WsLayout ws;
 };
 
+// validation + the three launches of one decode call; `workspace` is any 256-byte aligned device
+// scratch of ws_layout(L, B, R, T).total bytes
+int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B, int R, const void* K_txt,
+                  const void* V_txt, int T, int T_cap, void* out, void* workspace, cudaStream_t st);
+
 // optional event brackets around a launch (kvc_profile_*)
 bool prof_begin(int kernel_id, cudaStream_t st);
 void prof_end(cudaStream_t st);
