@@ -88,8 +88,9 @@ KVC_API int kvc_layer_destroy(kvc_layer* layer);
  * by V_tilde [B][H_kv][R][m][d] (the compressed-cache term of App. D, Eq. 2, vision part). */
 KVC_API size_t kvc_capsule_bytes(const kvc_layer* layer, int B, int R);
 
-/* Bytes of scratch kvc_decode_attend needs for up to B sequences, R blocks and T_cap text rows.
- * The scratch holds only temporaries of one call (compressed scores, expanded-probability
+/* Bytes of scratch kvc_decode_attend needs for B sequences of R blocks and up to T_cap text rows
+ * (the figure grows with T_cap but is not monotone in B and R: size it for the B and R you call
+ * with).  The scratch holds only temporaries of one call (compressed scores, expanded-probability
  * projections, split partials); it needs no initialisation and must be 256-byte aligned. */
 KVC_API size_t kvc_workspace_bytes(const kvc_layer* layer, int B, int R, int T_cap);
 
@@ -106,8 +107,8 @@ KVC_API int kvc_compress(const kvc_layer* layer, const void* K_vis, const void* 
  * [U^T V_tilde + 1 mu^T ; V_txt],  sigma = 1/sqrt(d), query head hq reading KV head hq / G.
  * q, out: [B][H_q][d].  K_txt, V_txt: [B][H_kv][T_cap][d] of which the first T rows are valid
  * (may be NULL when T == 0).  R == 0 attends over text only; R == 0 and T == 0 is KVC_ERR_SHAPE.
- * workspace: kvc_workspace_bytes(layer, B, R, >= T) bytes; calls sharing a workspace must be
- * stream-ordered. */
+ * workspace: kvc_workspace_bytes(layer, B, R, T_max) bytes for the same B and R and any
+ * T_max >= T; calls sharing a workspace must be stream-ordered. */
 KVC_API int kvc_decode_attend(const kvc_layer* layer, const void* q, const void* capsules, int B, int R,
                       const void* K_txt, const void* V_txt, int T, int T_cap, void* out,
                       void* workspace, void* stream);
@@ -142,6 +143,13 @@ KVC_API int kvc_decode_attend_static(const kvc_layer* layer, const void* q, cons
                                      int R, const void* K_txt, const void* V_txt, int T, int T_cap,
                                      void* out, void* stream);
 
+/* Device status word of the last kvc_decode_attend call that used `workspace` with these B, R, T:
+ * 0, or KVC_ERR_TIMEOUT if a bounded device-side wait (bulk-copy completion) gave up, in which case
+ * that call's output is invalid.  Synchronous (copies one int to the host); the kernels never trap
+ * or spin without limit. */
+KVC_API int kvc_read_device_status(const kvc_layer* layer, int B, int R, int T, const void* workspace,
+                                   int* status_out);
+
 /* Integer maps as the device path uses them (read back from the device copy):
  * idx_out: HOST [H_kv][m] retained indices per KV head; group_out: HOST [R*n][2] = (block r,
  * offset i) of vision token t = r*n + i (the Reshape of Alg. 1 step 1).  Either may be NULL. */
@@ -162,10 +170,11 @@ KVC_API const char* kvc_strerror(int status);
 typedef enum {
   KVC_KERNEL_SCORES = 0,          /* Alg. 1 step 1 + text logits  */
   KVC_KERNEL_EXPAND = 1,          /* Alg. 1 steps 2-3             */
-  KVC_KERNEL_OUTPUT = 2,          /* Alg. 1 step 4 + text + merge */
+  KVC_KERNEL_OUTPUT = 2,          /* Alg. 1 step 4 + text values  */
   KVC_KERNEL_GATHER_KEYS = 3,     /* key row selection            */
   KVC_KERNEL_PROJECT_VALUES = 4,  /* value centre + project       */
-  KVC_KERNEL_COUNT = 5
+  KVC_KERNEL_MERGE = 5,           /* log-sum-exp merge of partials */
+  KVC_KERNEL_COUNT = 6
 } kvc_kernel_id;
 KVC_API int kvc_profile_start(int max_launches);
 KVC_API int kvc_profile_stop(void);

@@ -54,6 +54,8 @@ def _lib() -> C.CDLL:
         lib.kvc_decode_attend_static.argtypes = [vp, vp, vp, i, i, vp, vp, i, i, vp, vp]
         lib.kvc_decode_attend_static.restype = i
         lib.kvc_static_scratch_bytes.argtypes = []; lib.kvc_static_scratch_bytes.restype = C.c_size_t
+        lib.kvc_read_device_status.argtypes = [vp, i, i, i, vp, C.POINTER(i)]
+        lib.kvc_read_device_status.restype = i
         lib.kvc_export_maps.argtypes = [vp, i, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         lib.kvc_export_maps.restype = i
         lib.kvc_strerror.argtypes = [i]; lib.kvc_strerror.restype = C.c_char_p
@@ -168,6 +170,13 @@ def kvc_attend_full(layer: Layer, q, K, V, B: int, S: int, S_cap: int, out, work
                                   _ptr(workspace), _stream(stream)), "kvc_attend_full")
 
 
+def kvc_read_device_status(layer: Layer, B: int, R: int, T: int, workspace) -> int:
+    out = C.c_int(-99)
+    _check(_lib().kvc_read_device_status(layer.handle, B, R, T, _ptr(workspace), C.byref(out)),
+           "kvc_read_device_status")
+    return out.value
+
+
 def kvc_export_maps(layer: Layer, R: int):
     """(idx [H_kv, m] int32, group [R*n, 2] int32) as the device path holds them."""
     idx = torch.empty((layer.H_kv, layer.m), dtype=torch.int32)
@@ -184,7 +193,7 @@ def capsule_views(layer: Layer, capsules, B: int, R: int):
     return (capsules[:half].view(layer.dtype).view(shape), capsules[half:2 * half].view(layer.dtype).view(shape))
 
 
-KVC_KERNEL_COUNT = 5
+KVC_KERNEL_COUNT = 6
 
 
 def kvc_profile_start(max_launches: int) -> None:

@@ -12,31 +12,44 @@ WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap) {
   WsLayout w{};
   const int H_kv = L->desc.H_kv, G = L->G, n = L->desc.n, ms = L->ms;
   const int rows_h = B * G * R;
-  const int row_tiles = ceil_div(rows_h, EXP_ROWS) * H_kv;
+  // tensor-core expansion: bf16 storage and 16-byte aligned rows of theta / U
+  w.use_mma = (!L->passthrough && L->desc.dtype == KVC_BF16 && n % 8 == 0) ? 1 : 0;
+  w.CG = 1;
+  w.cgw = ms;
+  int row_tiles;
+  if (w.use_mma) {
+    w.CG = ceil_div(ms, 256);
+    w.cgw = (int)align_up((size_t)ceil_div(ms, w.CG), 16);
+    row_tiles = ceil_div(rows_h, 64) * H_kv * w.CG;
+  } else {
+    row_tiles = ceil_div(rows_h, EXP_ROWS) * H_kv;
+  }
   if (L->passthrough || rows_h == 0) {
     w.NS = 1;
-    w.IR = align_up(n, EXP_IC);
+    w.IR = (int)align_up(n, EXP_IC);
   } else {
     int ns = ceil_div(EXP_TARGET_CTAS, row_tiles);
     ns = ns < 1 ? 1 : ns;
-    const int max_ns = ceil_div(n, EXP_IC);
+    int max_ns = ceil_div(n, EXP_IC);
+    max_ns = max_ns > MAX_NS ? MAX_NS : max_ns;
     ns = ns > max_ns ? max_ns : ns;
     w.IR = (int)align_up((size_t)ceil_div(n, ns), EXP_IC);
     w.NS = ceil_div(n, w.IR);
   }
-  w.NTC = ceil_div(T_cap, TXT_CHUNK);
-  w.nsplit = R + w.NTC;
+  const int VR = R * L->m;
+  w.Pv = ceil_div(VR, OUT_PART_ROWS);
+  w.pr = w.Pv > 0 ? ceil_div(VR, w.Pv) : 0;
+  w.NTC = ceil_div(T_cap, OUT_PART_ROWS);
+  w.nsplit = w.Pv + w.NTC;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
-  w.off_S = take(sizeof(float) * (size_t)H_kv * rows_h * ms);
+  w.off_cnt = take(sizeof(int) * ((size_t)B * H_kv + 1));
+  w.off_S = take((w.use_mma ? sizeof(__nv_bfloat16) : sizeof(float)) * (size_t)H_kv * rows_h * ms);
   w.off_stxt = take(sizeof(float) * (size_t)B * H_kv * G * (T_cap > 0 ? T_cap : 1));
-  // sized so that the bytes never shrink when B or R grow (NS falls as the row count rises)
-  const size_t w_rows = (size_t)(EXP_TARGET_CTAS + row_tiles) * EXP_ROWS;
-  w.off_W = take(sizeof(float) * w_rows * ms);
-  w.off_wstat = take(sizeof(float2) * w_rows);
+  w.off_W = take(sizeof(float) * (size_t)w.NS * H_kv * rows_h * ms);
+  w.off_wstat = take(sizeof(float2) * (size_t)w.NS * H_kv * rows_h);
   w.off_ypart = take(sizeof(float) * (size_t)B * H_kv * G * w.nsplit * D);
   w.off_ystat = take(sizeof(float2) * (size_t)B * H_kv * G * w.nsplit);
-  w.off_cnt = take(sizeof(int) * (size_t)B * H_kv);
   w.total = off;
   return w;
 }
@@ -171,12 +184,14 @@ int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B
   a.T = T; a.T_cap = T_cap > 0 ? T_cap : 1; a.Ts = T > 0 ? T : 1;
   a.passthrough = L->passthrough;
   a.S = reinterpret_cast<float*>(ws + a.ws.off_S);
+  a.Sb = reinterpret_cast<__nv_bfloat16*>(ws + a.ws.off_S);
   a.s_txt = reinterpret_cast<float*>(ws + a.ws.off_stxt);
   a.W = reinterpret_cast<float*>(ws + a.ws.off_W);
   a.wstat = reinterpret_cast<float2*>(ws + a.ws.off_wstat);
   a.ypart = reinterpret_cast<float*>(ws + a.ws.off_ypart);
   a.ystat = reinterpret_cast<float2*>(ws + a.ws.off_ystat);
   a.cnt = reinterpret_cast<int*>(ws + a.ws.off_cnt);
+  a.status = a.cnt + (size_t)B * L->desc.H_kv;
 
   cudaError_t e = launch_scores(a, L->desc.dtype, st);
   if (e == cudaSuccess) e = launch_expand(a, L->desc.dtype, st);
@@ -196,6 +211,13 @@ int kvc_decode_attend(const kvc_layer* L, const void* q, const void* capsules, i
 int kvc_attend_full(const kvc_layer* L, const void* q, const void* K, const void* V, int B, int S, int S_cap,
                     void* out, void* workspace, void* stream) {
   return decode_common(L, q, nullptr, B, 0, K, V, S, S_cap, out, workspace, static_cast<cudaStream_t>(stream));
+}
+
+int kvc_read_device_status(const kvc_layer* L, int B, int R, int T, const void* workspace, int* status_out) {
+  if (!L || !workspace || !status_out || B < 0 || R < 0 || T < 0) return KVC_ERR_ARG;
+  const WsLayout w = ws_layout(L, B, R, T);
+  const char* p = static_cast<const char*>(workspace) + w.off_cnt + sizeof(int) * (size_t)B * L->desc.H_kv;
+  return cudaMemcpy(status_out, p, sizeof(int), cudaMemcpyDeviceToHost) == cudaSuccess ? KVC_OK : KVC_ERR_CUDA;
 }
 
 int kvc_export_maps(const kvc_layer* L, int R, int32_t* idx_out, int32_t* group_out) {

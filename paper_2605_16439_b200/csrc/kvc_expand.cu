@@ -161,6 +161,7 @@ cudaError_t launch_expand(const DecodeArgs& a, int dtype, cudaStream_t st) {
     passthrough_softmax_kernel<<<ceil_div(nrows, 8), 256, 0, st>>>(a);
     return cudaGetLastError();
   }
+  if (a.ws.use_mma) return launch_expand_mma(a, st);
   return dtype == KVC_BF16 ? launch_expand_t<__nv_bfloat16>(a, st) : launch_expand_t<float>(a, st);
 }
 

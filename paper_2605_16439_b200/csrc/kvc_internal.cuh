@@ -12,10 +12,11 @@ namespace kvc {
 constexpr int D = 128;              // head dimension (all supported models)
 constexpr int MAX_G = 16;           // query heads per KV head
 constexpr int SCORE_TILE_ROWS = 64; // K rows per CTA in the score kernel
-constexpr int TXT_CHUNK = 256;      // text rows per split in the output kernel
+constexpr int OUT_PART_ROWS = 256;  // value rows per CTA of the output kernel (vision or text run)
 constexpr int EXP_ROWS = 16;        // rows per CTA in the generic expansion kernel
 constexpr int EXP_IC = 64;          // vision positions per inner chunk of the expansion
 constexpr int EXP_TARGET_CTAS = 296;
+constexpr int MAX_NS = 16;          // upper bound of the n-axis splits of the expansion
 
 inline __host__ __device__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline __host__ __device__ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -49,17 +50,20 @@ __device__ __forceinline__ void store_elem(__nv_bfloat16* p, float x) { *p = __f
 
 // ---- workspace layout of one decode call -----------------------------------------------------
 struct WsLayout {
+  int use_mma;     // 1: tensor-core expansion (bf16 S), 0: CUDA-core fp32 expansion
   int NS;          // splits of the n axis in the expansion kernel
   int IR;          // vision positions per split (multiple of EXP_IC)
-  int NTC;         // text chunks
-  int nsplit;      // R + NTC output splits per (sequence, KV head)
-  size_t off_S;    // fp32 [H_kv][B][G][R][ms]   compressed scores, sigma applied
+  int CG, cgw;     // tensor-core expansion: column groups of W and their width (multiple of 16)
+  int Pv, pr;      // output kernel: parts of the R*m vision rows per (sequence, KV head), rows per part
+  int NTC;         // output kernel: parts of the T text rows
+  int nsplit;      // Pv + NTC partials per (sequence, KV head)
+  size_t off_S;    // fp32 or bf16 [H_kv][B][G][R][ms]   compressed scores, sigma applied
   size_t off_stxt; // fp32 [B][H_kv][G][T]       text logits
   size_t off_W;    // fp32 [NS][H_kv][B*G*R][ms] unnormalised P U^T per split
   size_t off_wstat;// float2 [NS][H_kv][B*G*R]   (max, sum) per row and split
   size_t off_ypart;// fp32 [B][H_kv][G][nsplit][D]
   size_t off_ystat;// float2 [B][H_kv][G][nsplit]
-  size_t off_cnt;  // int [B*H_kv]
+  size_t off_cnt;  // int [B*H_kv] arrival counters, then one int device status word
   size_t total;
 };
 
@@ -92,13 +96,15 @@ struct DecodeArgs {
   int B, H_kv, G, R, m, ms, n, T, T_cap;
   int Ts;              // row stride of s_txt
   int passthrough;
-  float* S;
+  float* S;            // fp32 scores (CUDA-core expansion)
+  __nv_bfloat16* Sb;   // bf16 scores (tensor-core expansion); exactly one of S / Sb is used
   float* s_txt;
   float* W;
   float2* wstat;
   float* ypart;
   float2* ystat;
   int* cnt;
+  int* status;         // device status word (0 = ok, else a kvc_status), cleared by the score kernel
   WsLayout ws;
 };
 
@@ -116,9 +122,29 @@ struct ProfScope {
   ~ProfScope() { if (on) prof_end(st); }
 };
 
+// Launch with programmatic stream serialisation: the kernel may begin while the preceding kernel of
+// the stream is still running, and must execute griddepcontrol.wait before touching anything that
+// kernel (or anything before it) writes.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // launchers (each returns a cudaError_t from the launch)
 cudaError_t launch_scores(const DecodeArgs& a, int dtype, cudaStream_t st);
 cudaError_t launch_expand(const DecodeArgs& a, int dtype, cudaStream_t st);
+cudaError_t launch_expand_mma(const DecodeArgs& a, cudaStream_t st);
 cudaError_t launch_output(const DecodeArgs& a, int dtype, cudaStream_t st);
 cudaError_t launch_compress(const kvc_layer* L, const void* K_vis, const void* V_vis, int B, int R,
                             void* Kc, void* Vc, cudaStream_t st);

@@ -76,6 +76,7 @@ const char* kvc_kernel_name(int kernel_id) {
     case KVC_KERNEL_OUTPUT: return "output";
     case KVC_KERNEL_GATHER_KEYS: return "gather_keys";
     case KVC_KERNEL_PROJECT_VALUES: return "project_values";
+    case KVC_KERNEL_MERGE: return "merge";
     default: return "?";
   }
 }
