@@ -168,7 +168,7 @@ class Job:
         for p in self.layers:
             self.kvc.kvc_decode_attend(p["layer"], p["q"], p["caps"], s.B, s.R, p["K_txt"], p["V_txt"], T,
                                        self.T_cap, p["out"], self.ws)
-        self.launches += 4 * len(self.layers)
+        self.launches += 5 * len(self.layers)
 
     def step(self):
         self.compress_all()
@@ -378,7 +378,7 @@ def main():
     prof = {}
     ms_bracketed = None
     if not a.no_profile:
-        kvc.kvc_profile_start(a.steps * (4 * calls + 2 * shape.layers))
+        kvc.kvc_profile_start(a.steps * (5 * calls + 2 * shape.layers))
         ms_bracketed = timed(job.step, a.steps, dev) / a.steps
         kvc.kvc_profile_stop()
         prof = kvc.kvc_profile_read()

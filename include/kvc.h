@@ -174,7 +174,8 @@ typedef enum {
   KVC_KERNEL_GATHER_KEYS = 3,     /* key row selection            */
   KVC_KERNEL_PROJECT_VALUES = 4,  /* value centre + project       */
   KVC_KERNEL_MERGE = 5,           /* log-sum-exp merge of partials */
-  KVC_KERNEL_COUNT = 6
+  KVC_KERNEL_COMBINE = 6,         /* n-split partials of Alg. 1 step 3 combined per row */
+  KVC_KERNEL_COUNT = 7
 } kvc_kernel_id;
 KVC_API int kvc_profile_start(int max_launches);
 KVC_API int kvc_profile_stop(void);

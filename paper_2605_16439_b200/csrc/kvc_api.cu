@@ -36,18 +36,37 @@ WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap) {
     w.IR = (int)align_up((size_t)ceil_div(n, ns), EXP_IC);
     w.NS = ceil_div(n, w.IR);
   }
-  const int VR = R * L->m;
-  w.Pv = ceil_div(VR, OUT_PART_ROWS);
-  w.pr = w.Pv > 0 ? ceil_div(VR, w.Pv) : 0;
-  w.NTC = ceil_div(T_cap, OUT_PART_ROWS);
-  w.nsplit = w.Pv + w.NTC;
+  w.cpb = ceil_div(L->m, OUT_CHUNK);
+  w.ct = ceil_div(T_cap, OUT_CHUNK);
+  w.chunks_per_bh = R * w.cpb + w.ct;
+  w.GT = G == 1 ? 1 : (G == 2 ? 2 : (G <= 4 ? 4 : 8));
+  {
+    const long long total = (long long)B * H_kv * w.chunks_per_bh;
+    const int per_sm = w.GT <= 2 ? 3 : 2;
+    long long ctas = (long long)(L->num_sms > 0 ? L->num_sms : 148) * per_sm;
+    if (ctas > total) ctas = total;
+    if (ctas < 1) ctas = 1;
+    w.cpc = (int)((total + ctas - 1) / ctas);
+    if (w.cpc < 1) w.cpc = 1;
+    w.out_ctas = (int)((total + w.cpc - 1) / w.cpc);
+  }
+  {
+    // a (sequence, KV head) spans chunks_per_bh <= cpc * ctas / (B*H_kv) chunks, hence at most that many + 1 CTAs;
+    // the bound does not depend on T, so a workspace sized for T_cap fits every T <= T_cap
+    const long long ctas_max = (long long)(L->num_sms > 0 ? L->num_sms : 148) * (w.GT <= 2 ? 3 : 2);
+    const long long bh = (long long)B * H_kv;
+    w.nsplit = (int)((ctas_max + (bh > 0 ? bh : 1) - 1) / (bh > 0 ? bh : 1)) + 2;
+  }
+  w.Ts = (int)align_up((size_t)(T_cap > 0 ? T_cap : 1), 4);
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   w.off_cnt = take(sizeof(int) * ((size_t)B * H_kv + 1));
   w.off_S = take((w.use_mma ? sizeof(__nv_bfloat16) : sizeof(float)) * (size_t)H_kv * rows_h * ms);
-  w.off_stxt = take(sizeof(float) * (size_t)B * H_kv * G * (T_cap > 0 ? T_cap : 1));
+  w.off_stxt = take(sizeof(float) * (size_t)B * H_kv * G * w.Ts);
   w.off_W = take(sizeof(float) * (size_t)w.NS * H_kv * rows_h * ms);
   w.off_wstat = take(sizeof(float2) * (size_t)w.NS * H_kv * rows_h);
+  w.off_Wc = take(sizeof(float) * (size_t)H_kv * rows_h * ms);
+  w.off_statc = take(sizeof(float4) * (size_t)H_kv * rows_h);
   w.off_ypart = take(sizeof(float) * (size_t)B * H_kv * G * w.nsplit * D);
   w.off_ystat = take(sizeof(float2) * (size_t)B * H_kv * G * w.nsplit);
   w.total = off;
@@ -109,7 +128,9 @@ int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out) {
   L->G = desc->H_q / desc->H_kv;
   L->passthrough = pass ? 1 : 0;
   L->d_idx = nullptr;
+  L->num_sms = 0;
   if (cudaGetDevice(&L->device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&L->num_sms, cudaDevAttrMultiProcessorCount, L->device) != cudaSuccess ||
       cudaMalloc(&L->d_idx, idx.size() * sizeof(int32_t)) != cudaSuccess ||
       cudaMemcpy(L->d_idx, idx.data(), idx.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess) {
     if (L->d_idx) cudaFree(L->d_idx);
@@ -181,13 +202,15 @@ int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B
   a.theta = L->desc.theta; a.U = L->desc.U; a.mu = L->desc.mu;
   a.out = out;
   a.B = B; a.H_kv = L->desc.H_kv; a.G = L->G; a.R = R; a.m = L->m; a.ms = L->ms; a.n = L->desc.n;
-  a.T = T; a.T_cap = T_cap > 0 ? T_cap : 1; a.Ts = T > 0 ? T : 1;
+  a.T = T; a.T_cap = T_cap > 0 ? T_cap : 1; a.Ts = a.ws.Ts;
   a.passthrough = L->passthrough;
   a.S = reinterpret_cast<float*>(ws + a.ws.off_S);
   a.Sb = reinterpret_cast<__nv_bfloat16*>(ws + a.ws.off_S);
   a.s_txt = reinterpret_cast<float*>(ws + a.ws.off_stxt);
   a.W = reinterpret_cast<float*>(ws + a.ws.off_W);
   a.wstat = reinterpret_cast<float2*>(ws + a.ws.off_wstat);
+  a.Wcomb = reinterpret_cast<float*>(ws + a.ws.off_Wc);
+  a.statc = reinterpret_cast<float4*>(ws + a.ws.off_statc);
   a.ypart = reinterpret_cast<float*>(ws + a.ws.off_ypart);
   a.ystat = reinterpret_cast<float2*>(ws + a.ws.off_ystat);
   a.cnt = reinterpret_cast<int*>(ws + a.ws.off_cnt);

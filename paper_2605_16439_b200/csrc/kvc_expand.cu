@@ -6,6 +6,7 @@
 //
 // This translation unit holds the CUDA-core fp32 version, used for fp32 storage (1e-4 parity) and
 // as the fallback shape-agnostic path.
+#include "kvc_async.cuh"
 #include "kvc_internal.cuh"
 
 namespace kvc {
@@ -117,13 +118,15 @@ __global__ void __launch_bounds__(256) expand_kernel(DecodeArgs a) {
     a.wstat[((size_t)split * a.H_kv + h) * nrows_h + row0 + tid] = make_float2(rowmax[tid], rowsum[tid]);
 }
 
-// rho = 0: theta = U = I, so L_img = S_comp and W = P.  One warp per row.
+// rho = 0: theta = U = I, so L_img = S_comp and W = P.  One warp per row; writes the combined format.
 __global__ void __launch_bounds__(256) passthrough_softmax_kernel(DecodeArgs a) {
+  grid_dep_wait();
+  grid_dep_launch();
   const int nrows = a.H_kv * a.B * a.G * a.R;
   const int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (row >= nrows) return;
   const float* s = a.S + (size_t)row * a.ms;
-  float* w = a.W + (size_t)row * a.ms;
+  float* w = a.Wcomb + (size_t)row * a.ms;
   float mx = -INFINITY;
   for (int j = lane; j < a.m; j += 32) mx = fmaxf(mx, s[j]);
 #pragma unroll
@@ -136,7 +139,44 @@ __global__ void __launch_bounds__(256) passthrough_softmax_kernel(DecodeArgs a) 
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-  if (lane == 0) a.wstat[row] = make_float2(mx, sum);
+  if (lane == 0) a.statc[row] = make_float4(mx, sum, 0.f, 0.f);
+}
+
+// The n-split partials of one row combined relative to the row's overall maximum:
+//   Wcomb[row][:] = sum_s e^{max_s - max} W_s[row][:],   statc[row] = (max, sum_s e^{max_s - max} sum_s).
+// One warp per row (KV head, sequence, head in group, block).
+__global__ void __launch_bounds__(256) combine_kernel(DecodeArgs a) {
+  grid_dep_wait();
+  grid_dep_launch();
+  const int nrows = a.H_kv * a.B * a.G * a.R;
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= nrows) return;
+  const int NS = a.ws.NS;
+  float2 st = make_float2(-INFINITY, 0.f);
+  if (lane < NS) st = a.wstat[(size_t)lane * nrows + row];
+  float mx = st.x;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  const float my_sc = lane < NS ? __expf(st.x - mx) : 0.f;
+  float sum = my_sc * st.y;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  float sc[MAX_NS];
+#pragma unroll
+  for (int s = 0; s < MAX_NS; ++s) sc[s] = __shfl_sync(0xffffffffu, my_sc, s);
+  const size_t sstride = (size_t)nrows * a.ms;
+  const float* wp = a.W + (size_t)row * a.ms;
+  float* wo = a.Wcomb + (size_t)row * a.ms;
+  for (int j = lane; j < a.ms; j += 32) {
+    float v[MAX_NS];
+#pragma unroll
+    for (int s = 0; s < MAX_NS; ++s) v[s] = s < NS ? __ldcg(wp + s * sstride + j) : 0.f;
+    float w = 0.f;
+#pragma unroll
+    for (int s = 0; s < MAX_NS; ++s) w = fmaf(sc[s], v[s], w);
+    wo[j] = w;
+  }
+  if (lane == 0) a.statc[row] = make_float4(mx, sum, 0.f, 0.f);
 }
 
 static size_t expand_smem_bytes(int ms) {
@@ -155,14 +195,20 @@ static cudaError_t launch_expand_t(const DecodeArgs& a, cudaStream_t st) {
 
 cudaError_t launch_expand(const DecodeArgs& a, int dtype, cudaStream_t st) {
   if (a.R == 0) return cudaSuccess;
-  ProfScope prof(KVC_KERNEL_EXPAND, st);
+  const int nrows = a.H_kv * a.B * a.G * a.R;
   if (a.passthrough) {
-    const int nrows = a.H_kv * a.B * a.G * a.R;
-    passthrough_softmax_kernel<<<ceil_div(nrows, 8), 256, 0, st>>>(a);
-    return cudaGetLastError();
+    ProfScope prof(KVC_KERNEL_EXPAND, st);
+    return launch_dependent(passthrough_softmax_kernel, dim3(ceil_div(nrows, 8)), dim3(256), 0, st, a);
   }
-  if (a.ws.use_mma) return launch_expand_mma(a, st);
-  return dtype == KVC_BF16 ? launch_expand_t<__nv_bfloat16>(a, st) : launch_expand_t<float>(a, st);
+  cudaError_t e;
+  {
+    ProfScope prof(KVC_KERNEL_EXPAND, st);
+    if (a.ws.use_mma) e = launch_expand_mma(a, st);
+    else e = dtype == KVC_BF16 ? launch_expand_t<__nv_bfloat16>(a, st) : launch_expand_t<float>(a, st);
+  }
+  if (e != cudaSuccess) return e;
+  ProfScope prof(KVC_KERNEL_COMBINE, st);
+  return launch_dependent(combine_kernel, dim3(ceil_div(nrows, 8)), dim3(256), 0, st, a);
 }
 
 }  // namespace kvc

@@ -12,7 +12,7 @@ namespace kvc {
 constexpr int D = 128;              // head dimension (all supported models)
 constexpr int MAX_G = 16;           // query heads per KV head
 constexpr int SCORE_TILE_ROWS = 64; // K rows per CTA in the score kernel
-constexpr int OUT_PART_ROWS = 256;  // value rows per CTA of the output kernel (vision or text run)
+constexpr int OUT_CHUNK = 64;       // value rows per ring stage of the output kernel
 constexpr int EXP_ROWS = 16;        // rows per CTA in the generic expansion kernel
 constexpr int EXP_IC = 64;          // vision positions per inner chunk of the expansion
 constexpr int EXP_TARGET_CTAS = 296;
@@ -54,13 +54,17 @@ struct WsLayout {
   int NS;          // splits of the n axis in the expansion kernel
   int IR;          // vision positions per split (multiple of EXP_IC)
   int CG, cgw;     // tensor-core expansion: column groups of W and their width (multiple of 16)
-  int Pv, pr;      // output kernel: parts of the R*m vision rows per (sequence, KV head), rows per part
-  int NTC;         // output kernel: parts of the T text rows
-  int nsplit;      // Pv + NTC partials per (sequence, KV head)
+  // output kernel: the value rows of a (sequence, KV head) are cut into chunks of <= OUT_CHUNK rows
+  // (cpb per vision block, ct for the text run); CTA c streams chunks [c*cpc, (c+1)*cpc) of the flat list
+  int cpb, ct, chunks_per_bh, cpc, out_ctas, GT;
+  int nsplit;      // partial slots per (sequence, KV head): CTAs that can touch its chunk range
+  int Ts;          // row stride of the text logits (T rounded up to a multiple of 4)
   size_t off_S;    // fp32 or bf16 [H_kv][B][G][R][ms]   compressed scores, sigma applied
   size_t off_stxt; // fp32 [B][H_kv][G][T]       text logits
   size_t off_W;    // fp32 [NS][H_kv][B*G*R][ms] unnormalised P U^T per split
   size_t off_wstat;// float2 [NS][H_kv][B*G*R]   (max, sum) per row and split
+  size_t off_Wc;   // fp32 [H_kv][B*G*R][ms]     the splits combined, relative to one maximum per row
+  size_t off_statc;// float4 [H_kv][B*G*R]       (max, sum, 0, 0) of the combined row
   size_t off_ypart;// fp32 [B][H_kv][G][nsplit][D]
   size_t off_ystat;// float2 [B][H_kv][G][nsplit]
   size_t off_cnt;  // int [B*H_kv] arrival counters, then one int device status word
@@ -76,6 +80,7 @@ struct kvc_layer {
   int G;
   int passthrough;       // ratio_permille == 0
   int device;
+  int num_sms;
   int32_t* d_idx;        // device [H_kv][m]
 };
 
@@ -101,6 +106,8 @@ struct DecodeArgs {
   float* s_txt;
   float* W;
   float2* wstat;
+  float* Wcomb;
+  float4* statc;
   float* ypart;
   float2* ystat;
   int* cnt;

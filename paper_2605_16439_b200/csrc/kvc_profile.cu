@@ -77,6 +77,7 @@ const char* kvc_kernel_name(int kernel_id) {
     case KVC_KERNEL_GATHER_KEYS: return "gather_keys";
     case KVC_KERNEL_PROJECT_VALUES: return "project_values";
     case KVC_KERNEL_MERGE: return "merge";
+    case KVC_KERNEL_COMBINE: return "combine";
     default: return "?";
   }
 }
