@@ -175,7 +175,8 @@ typedef enum {
   KVC_KERNEL_PROJECT_VALUES = 4,  /* value centre + project       */
   KVC_KERNEL_MERGE = 5,           /* log-sum-exp merge of partials */
   KVC_KERNEL_COMBINE = 6,         /* n-split partials of Alg. 1 step 3 combined per row */
-  KVC_KERNEL_COUNT = 7
+  KVC_KERNEL_FUSED = 7,           /* Alg. 1 steps 1-4 + text + normalisation in one kernel (bf16) */
+  KVC_KERNEL_COUNT = 8
 } kvc_kernel_id;
 KVC_API int kvc_profile_start(int max_launches);
 KVC_API int kvc_profile_stop(void);

@@ -69,6 +69,12 @@ WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap) {
   w.off_statc = take(sizeof(float4) * (size_t)H_kv * rows_h);
   w.off_ypart = take(sizeof(float) * (size_t)B * H_kv * G * w.nsplit * D);
   w.off_ystat = take(sizeof(float2) * (size_t)B * H_kv * G * w.nsplit);
+  {
+    const FusedPlan fp = (B > 0 && R > 0) ? plan_fused(L, B, R) : FusedPlan{};
+    const size_t np = (fp.ok && fp.nrg > 1) ? (size_t)B * H_kv * fp.nrg * G : 0;
+    w.off_fpy = take(sizeof(float) * np * D);
+    w.off_fpml = take(sizeof(float2) * np);
+  }
   w.total = off;
   return w;
 }
@@ -128,12 +134,16 @@ int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out) {
   L->G = desc->H_q / desc->H_kv;
   L->passthrough = pass ? 1 : 0;
   L->d_idx = nullptr;
+  L->d_cnt = nullptr;
   L->num_sms = 0;
   if (cudaGetDevice(&L->device) != cudaSuccess ||
       cudaDeviceGetAttribute(&L->num_sms, cudaDevAttrMultiProcessorCount, L->device) != cudaSuccess ||
       cudaMalloc(&L->d_idx, idx.size() * sizeof(int32_t)) != cudaSuccess ||
-      cudaMemcpy(L->d_idx, idx.data(), idx.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess) {
+      cudaMemcpy(L->d_idx, idx.data(), idx.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMalloc(&L->d_cnt, KVC_MAX_COUNTERS * sizeof(int)) != cudaSuccess ||
+      cudaMemset(L->d_cnt, 0, KVC_MAX_COUNTERS * sizeof(int)) != cudaSuccess) {
     if (L->d_idx) cudaFree(L->d_idx);
+    if (L->d_cnt) cudaFree(L->d_cnt);
     delete L;
     cudaGetLastError();
     return KVC_ERR_CUDA;
@@ -145,6 +155,7 @@ int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out) {
 int kvc_layer_destroy(kvc_layer* L) {
   if (!L) return KVC_OK;
   if (L->d_idx) cudaFree(L->d_idx);
+  if (L->d_cnt) cudaFree(L->d_cnt);
   delete L;
   return KVC_OK;
 }
@@ -215,6 +226,21 @@ int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B
   a.ystat = reinterpret_cast<float2*>(ws + a.ws.off_ystat);
   a.cnt = reinterpret_cast<int*>(ws + a.ws.off_cnt);
   a.status = a.cnt + (size_t)B * L->desc.H_kv;
+  a.fpart_y = reinterpret_cast<float*>(ws + a.ws.off_fpy);
+  a.fpart_ml = reinterpret_cast<float2*>(ws + a.ws.off_fpml);
+
+  // bf16 storage with TMA-compatible shapes and pointers: the whole of Algorithm 1 in one kernel
+  if (R > 0) {
+    const FusedPlan fp = plan_fused(L, B, R);
+    const uintptr_t align = reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(capsules) |
+                            reinterpret_cast<uintptr_t>(out) | (T > 0 ? reinterpret_cast<uintptr_t>(K_txt) |
+                            reinterpret_cast<uintptr_t>(V_txt) : 0) | reinterpret_cast<uintptr_t>(L->desc.mu);
+    if (fp.ok && (align & 15) == 0) {
+      bool encoded = false;
+      const cudaError_t fe = launch_fused(L, a, fp, st, &encoded);
+      if (encoded) return fe == cudaSuccess ? KVC_OK : KVC_ERR_CUDA;
+    }
+  }
 
   cudaError_t e = launch_scores(a, L->desc.dtype, st);
   if (e == cudaSuccess) e = launch_expand(a, L->desc.dtype, st);

@@ -17,6 +17,7 @@ constexpr int EXP_ROWS = 16;        // rows per CTA in the generic expansion ker
 constexpr int EXP_IC = 64;          // vision positions per inner chunk of the expansion
 constexpr int EXP_TARGET_CTAS = 296;
 constexpr int MAX_NS = 16;          // upper bound of the n-axis splits of the expansion
+constexpr int KVC_MAX_COUNTERS = 8192;  // (sequence, KV head) arrival counters owned by a layer handle
 
 inline __host__ __device__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline __host__ __device__ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -68,7 +69,26 @@ struct WsLayout {
   size_t off_ypart;// fp32 [B][H_kv][G][nsplit][D]
   size_t off_ystat;// float2 [B][H_kv][G][nsplit]
   size_t off_cnt;  // int [B*H_kv] arrival counters, then one int device status word
+  size_t off_fpy;  // fp32 [B*H_kv][nrg][G][D]  partial outputs of the one-kernel path (units that split the block axis)
+  size_t off_fpml; // float2 [B*H_kv][nrg][G]   their (max, sum)
   size_t total;
+};
+
+// Launch plan of the one-kernel bf16 decode path (kvc_fused.cu); ok == 0 when the shape is served by the
+// three-phase path instead.
+struct FusedPlan {
+  int ok;
+  int MT;            // 16-row tiles of expansion rows per unit
+  int NB, RB;        // sequences and vision blocks per unit
+  int nbg, nrg;      // unit groups along the batch and the block axis
+  int units;         // H_kv * nbg * nrg
+  int JC, NJ;        // 16-row sub-chunks of the m axis per stage; stages per pass over the m axis
+  int TCH;           // text rows per stage and sequence
+  int ncg;           // n / 64
+  int stages, grid;
+  uint32_t par_bytes, k_half_bytes, txt_half_bytes, stage_bytes, misc_bytes;
+  uint32_t off_q, off_S, off_W, off_wred, off_rstat, off_tstat, off_hstat, off_yred;   // relative to the end of the ring
+  size_t smem_bytes;
 };
 
 }  // namespace kvc
@@ -82,11 +102,13 @@ struct kvc_layer {
   int device;
   int num_sms;
   int32_t* d_idx;        // device [H_kv][m]
+  int* d_cnt;            // device [KVC_MAX_COUNTERS] arrival counters of the one-kernel decode path; zero between calls
 };
 
 namespace kvc {
 
 WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap);
+FusedPlan plan_fused(const kvc_layer* L, int B, int R);
 
 struct DecodeArgs {
   const void* q;
@@ -111,7 +133,9 @@ struct DecodeArgs {
   float* ypart;
   float2* ystat;
   int* cnt;
-  int* status;         // device status word (0 = ok, else a kvc_status), cleared by the score kernel
+  int* status;         // device status word (0 = ok, else a kvc_status), cleared by the first kernel of the call
+  float* fpart_y;      // partials of the one-kernel path
+  float2* fpart_ml;
   WsLayout ws;
 };
 
@@ -153,6 +177,8 @@ cudaError_t launch_scores(const DecodeArgs& a, int dtype, cudaStream_t st);
 cudaError_t launch_expand(const DecodeArgs& a, int dtype, cudaStream_t st);
 cudaError_t launch_expand_mma(const DecodeArgs& a, cudaStream_t st);
 cudaError_t launch_output(const DecodeArgs& a, int dtype, cudaStream_t st);
+// one-kernel path; *encoded == false (and nothing launched) if the tensor maps could not be built
+cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPlan& p, cudaStream_t st, bool* encoded);
 cudaError_t launch_compress(const kvc_layer* L, const void* K_vis, const void* V_vis, int B, int R,
                             void* Kc, void* Vc, cudaStream_t st);
 

@@ -78,6 +78,7 @@ const char* kvc_kernel_name(int kernel_id) {
     case KVC_KERNEL_PROJECT_VALUES: return "project_values";
     case KVC_KERNEL_MERGE: return "merge";
     case KVC_KERNEL_COMBINE: return "combine";
+    case KVC_KERNEL_FUSED: return "fused";
     default: return "?";
   }
 }
