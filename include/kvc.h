@@ -160,6 +160,9 @@ KVC_API int kvc_layer_m(const kvc_layer* layer);
 
 KVC_API const char* kvc_strerror(int status);
 
+/* Text of the CUDA runtime error behind the calling thread's most recent KVC_ERR_CUDA ("no error" if none). */
+KVC_API const char* kvc_last_cuda_error(void);
+
 /* ---- optional instrumentation (measurement only; the paper has no counterpart) -------------
  * While profiling is on, every kernel the library launches is bracketed by two CUDA events
  * recorded on the launching stream, until max_launches brackets have been used.  Global,

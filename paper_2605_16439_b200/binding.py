@@ -21,6 +21,8 @@ class KvcError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
         msg = _lib().kvc_strerror(status).decode() if _LIB is not None else "?"
+        if status == -6 and _LIB is not None:
+            msg += ": " + _lib().kvc_last_cuda_error().decode()
         super().__init__(f"{where}: {msg} (status {status})")
 
 
@@ -59,6 +61,7 @@ def _lib() -> C.CDLL:
         lib.kvc_export_maps.argtypes = [vp, i, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         lib.kvc_export_maps.restype = i
         lib.kvc_strerror.argtypes = [i]; lib.kvc_strerror.restype = C.c_char_p
+        lib.kvc_last_cuda_error.argtypes = []; lib.kvc_last_cuda_error.restype = C.c_char_p
         lib.kvc_profile_start.argtypes = [i]; lib.kvc_profile_start.restype = i
         lib.kvc_profile_stop.argtypes = []; lib.kvc_profile_stop.restype = i
         lib.kvc_profile_read.argtypes = [i, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
@@ -118,8 +121,11 @@ class Layer:
         self.m = _lib().kvc_layer_m(h)
 
     def close(self):
-        if getattr(self, "handle", None):
-            _lib().kvc_layer_destroy(self.handle)
+        if getattr(self, "handle", None) and _LIB is not None:      # at interpreter exit the library may be gone already
+            try:
+                _LIB.kvc_layer_destroy(self.handle)
+            except Exception:
+                pass
             self.handle = None
 
     __del__ = close

@@ -83,7 +83,20 @@ WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap) {
 
 using namespace kvc;
 
+namespace kvc {
+static thread_local cudaError_t g_last_cuda = cudaSuccess;
+// KVC_OK, or KVC_ERR_CUDA after remembering the error for kvc_last_cuda_error (the runtime's own slot is cleared)
+int cuda_status(cudaError_t e) {
+  if (e == cudaSuccess) return KVC_OK;
+  g_last_cuda = e;
+  cudaGetLastError();
+  return KVC_ERR_CUDA;
+}
+}  // namespace kvc
+
 extern "C" {
+
+const char* kvc_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda); }
 
 int kvc_retained_len(int n, int ratio_permille) {
   if (n <= 0 || ratio_permille < 0 || ratio_permille >= 1000) return -1;
@@ -188,7 +201,7 @@ int kvc_compress(const kvc_layer* L, const void* K_vis, const void* V_vis, int B
   } else {
     e = launch_compress(L, K_vis, V_vis, B, R, Kc, Vc, st);
   }
-  return e == cudaSuccess ? KVC_OK : KVC_ERR_CUDA;
+  return cuda_status(e);
 }
 
 }  // extern "C"
@@ -238,14 +251,14 @@ int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B
     if (fp.ok && (align & 15) == 0) {
       bool encoded = false;
       const cudaError_t fe = launch_fused(L, a, fp, st, &encoded);
-      if (encoded) return fe == cudaSuccess ? KVC_OK : KVC_ERR_CUDA;
+      if (encoded) return cuda_status(fe);
     }
   }
 
   cudaError_t e = launch_scores(a, L->desc.dtype, st);
   if (e == cudaSuccess) e = launch_expand(a, L->desc.dtype, st);
   if (e == cudaSuccess) e = launch_output(a, L->desc.dtype, st);
-  return e == cudaSuccess ? KVC_OK : KVC_ERR_CUDA;
+  return cuda_status(e);
 }
 }  // namespace kvc
 

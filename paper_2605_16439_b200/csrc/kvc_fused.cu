@@ -6,27 +6,29 @@
 // shared-memory stages filled by the TMA engine (tiled tensor maps, 128-byte swizzle):
 //   pass A   stage c = rows [16 JC c, 16 JC (c+1)) of K_tilde of every block of the unit  +  the same rows
 //            of theta[h] (all n columns).  Scores S_c = sigma q K_c^T go through shared memory as bf16 and
-//            are multiplied into the logits L += S_c theta_c, which stay in registers (rows x n, fp32).
+//            are multiplied into the logits L += S_c theta_c, which stay in registers (rows x n, fp32,
+//            every warp owning a range of 16-column groups).
 //   text     stage = TCH rows of K_txt and V_txt per sequence; every warp runs an online-softmax
 //            attention over its own 16-row tiles.
 //   softmax  one maximum per (sequence, head) over all blocks of the unit and its text rows; P = 2^(L - max).
 //   pass C   stage c = rows of V_tilde + the same rows of U[h]:  W_c = P U_c^T (split over the warps' column
-//            ranges, reduced through shared memory), then y += W_c V_c.
+//            ranges, reduced through shared memory), then y^T += V_c^T W_c^T.
 // theta/U rows (L2-resident, shared by all sequences) and capsule rows (HBM) arrive interleaved in the same
-// stages, so both streams stay busy for the whole unit.  All matrix products run on mma.sync m16n8k16.
-// A unit that holds every block of its sequences writes `out` directly; otherwise the units of a
-// (sequence, KV head) leave (max, sum, y) partials and the last one to arrive merges them.
+// stages, so both streams stay busy for the whole unit.  All matrix products run on mma.sync m16n8k16; the
+// products with value rows are taken transposed (head dimension as M, heads as N) so that a group of up to
+// 8 heads costs one 8-wide tile.  A unit that holds every block of its sequences writes `out` directly;
+// otherwise the units of a (sequence, KV head) leave (max, sum, y) partials and the last one to arrive
+// merges them.
 #include "kvc_tma.cuh"
 #include "kvc_internal.cuh"
 
 namespace kvc {
 
-constexpr int FW = 8;                        // consumer warps
-constexpr int FTHREADS = (FW + 1) * 32;      // + one producer warp
-constexpr int FCONS = FW * 32;
 constexpr int FMAX_STAGES = 8;
 constexpr int QLD = 136;                     // row stride of the query tile in elements (272 B: conflict-free ldmatrix)
-constexpr int SLD = 24;                      // row stride of the 16-column score / weight tiles (48 B)
+constexpr int SLD = 24;                      // row stride of the 16-column weight tile (48 B)
+constexpr int ROWS = 16;                     // expansion rows per unit (one MMA row tile)
+constexpr int YHG = 2;                       // heads per round of the final cross-warp reduction
 constexpr uint32_t SMEM_LIMIT = 232448;      // 227 KB per CTA on sm_100
 
 struct FusedArgs {
@@ -35,6 +37,9 @@ struct FusedArgs {
   __nv_bfloat16* out;
   int B, H_kv, G, R, m, n, T;
   int NB, RB, nbg, nrg, units, JC, NJ, TCH, Tper, ncg, stages;
+  int ktw;            // 16-column groups of L per warp
+  int msplit, mshift; // the 8 row tiles of a value block go to msplit = 8 >> mshift tasks
+  int sld;            // row stride of the score tile in elements (16 JC + 8)
   uint32_t par_bytes, k_half_bytes, txt_half_bytes, stage_bytes;
   uint32_t off_q, off_S, off_W, off_wred, off_rstat, off_tstat, off_hstat, off_yred;
   float* part_y;      // [B*H_kv][nrg][G][D]  partial outputs (only when nrg > 1)
@@ -43,16 +48,16 @@ struct FusedArgs {
   int* status;        // device status word
 };
 
-__device__ __forceinline__ void consumer_sync() { named_barrier_sync(1, FCONS); }
-
-template <int MT, int NTW, int NH>
-__global__ void __launch_bounds__(FTHREADS, 1)
+// FWT consumer warps + one producer warp.  Every consumer warp owns up to KTW 16-column groups of the logits;
+// NH = 8-head tiles of the group (1: G <= 8, 2: G <= 16)
+template <int FWT, int KTW, int NH>
+__global__ void __launch_bounds__((FWT + 1) * 32, 1)
 fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                     const __grid_constant__ CUtensorMap tmKt, const __grid_constant__ CUtensorMap tmVt,
                     const __grid_constant__ CUtensorMap tmTh, const __grid_constant__ CUtensorMap tmU,
                     const FusedArgs a) {
-  constexpr int ROWS = 16 * MT;
-  constexpr int KK = (NTW + 1) / 2;
+  constexpr int FCONS = FWT * 32;
+  constexpr int FTHREADS = FCONS + 32;
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* sm = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
   __shared__ __align__(8) uint64_t full_bar[FMAX_STAGES], empty_bar[FMAX_STAGES];
@@ -60,73 +65,73 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
-    for (int s = 0; s < a.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], FW); }
+    for (int s = 0; s < a.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], FWT); }
     fence_mbar_init();
   }
   // score and weight tiles start as zeros: their padding rows and columns are read by the MMAs
   {
     uint32_t* z = reinterpret_cast<uint32_t*>(sm + a.off_S);
-    const int words = (2 * ROWS * SLD + (ROWS + 16) * SLD) / 2;
+    const int words = (2 * ROWS * a.sld + (ROWS + 16) * SLD) / 2;
     for (int i = tid; i < words; i += FTHREADS) z[i] = 0u;
   }
   __syncthreads();
 
   const int per_h = a.nbg * a.nrg;
 
-  if (warp == FW) {
+  if (warp == FWT) {
     // ================= producer: one thread feeds the ring =================
+    // It walks the stage sequence of this CTA's units: per unit NJ stages of pass A, the text stages, NJ stages
+    // of pass C.  A slot is refilled as soon as every consumer warp has released it.
     if (lane != 0) return;
     tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmTh); tma_prefetch_desc(&tmU);
     if (a.T > 0) { tma_prefetch_desc(&tmKt); tma_prefetch_desc(&tmVt); }
-    bool dead = false, first = true;
-    uint32_t it = 0;
-    for (int u = blockIdx.x; u < a.units && !dead; u += gridDim.x) {
+    bool first = true;
+    uint32_t slot = 0, phase = 1;              // parity to wait for on the empty barrier: 1 passes on a fresh barrier
+    for (int u = blockIdx.x; u < a.units; u += gridDim.x) {
       const int h = u / per_h, rem = u - h * per_h;
       const int bg = rem / a.nrg, rg = rem - bg * a.nrg;
       const int b0 = bg * a.NB, r0 = rg * a.RB;
       const int ts0 = rg * a.Tper;
       const int ts1 = min(a.T, ts0 + a.Tper);
       const int nts = ts1 > ts0 ? (ts1 - ts0 + a.TCH - 1) / a.TCH : 0;
-      for (int pass = 0; pass < 2 && !dead; ++pass) {
-        const CUtensorMap* tp = pass == 0 ? &tmTh : &tmU;
-        const CUtensorMap* tk = pass == 0 ? &tmK : &tmV;
-        for (int c = 0; c < a.NJ; ++c, ++it) {
-          const uint32_t slot = it % a.stages, use = it / a.stages;
-          if (use > 0 && !mbar_wait_bounded(&empty_bar[slot], (use - 1) & 1u)) { dead = true; break; }
+      for (int part = 0; part < 3; ++part) {
+        const int count = part == 1 ? nts : a.NJ;
+        for (int c = 0; c < count; ++c) {
+          if (!mbar_wait_bounded(&empty_bar[slot], phase)) { atomicExch(a.status, (int)KVC_ERR_TIMEOUT); return; }
           unsigned char* dst = sm + slot * a.stage_bytes;
-          const int j0 = c * 16 * a.JC;
-          mbar_expect_tx(&full_bar[slot], a.par_bytes + 2 * a.k_half_bytes);
-          tma_load_4d(dst, tp, 0, j0, 0, h, &full_bar[slot]);                 // parameters: never written by this library
-          if (first) { grid_dep_wait(); first = false; }                       // everything else may come from the stream's previous kernel
-          tma_load_5d(dst + a.par_bytes, tk, 0, j0, r0, h, b0, &full_bar[slot]);
-          tma_load_5d(dst + a.par_bytes + a.k_half_bytes, tk, 64, j0, r0, h, b0, &full_bar[slot]);
-        }
-        if (pass == 0) {
-          for (int ts = 0; ts < nts && !dead; ++ts, ++it) {
-            const uint32_t slot = it % a.stages, use = it / a.stages;
-            if (use > 0 && !mbar_wait_bounded(&empty_bar[slot], (use - 1) & 1u)) { dead = true; break; }
-            unsigned char* dst = sm + slot * a.stage_bytes;
-            const int y = ts0 + ts * a.TCH;
-            mbar_expect_tx(&full_bar[slot], 4 * a.txt_half_bytes);
-            tma_load_4d(dst, &tmKt, 0, y, h, b0, &full_bar[slot]);
-            tma_load_4d(dst + a.txt_half_bytes, &tmKt, 64, y, h, b0, &full_bar[slot]);
-            tma_load_4d(dst + 2 * a.txt_half_bytes, &tmVt, 0, y, h, b0, &full_bar[slot]);
-            tma_load_4d(dst + 3 * a.txt_half_bytes, &tmVt, 64, y, h, b0, &full_bar[slot]);
+          uint64_t* bar = &full_bar[slot];
+          if (part == 1) {
+            const int y = ts0 + c * a.TCH;
+            mbar_expect_tx(bar, 4 * a.txt_half_bytes);
+            if (first) { grid_dep_wait(); first = false; }
+            tma_load_4d(dst, &tmKt, 0, y, h, b0, bar);
+            tma_load_4d(dst + a.txt_half_bytes, &tmKt, 64, y, h, b0, bar);
+            tma_load_4d(dst + 2 * a.txt_half_bytes, &tmVt, 0, y, h, b0, bar);
+            tma_load_4d(dst + 3 * a.txt_half_bytes, &tmVt, 64, y, h, b0, bar);
+          } else {
+            const CUtensorMap* tp = part == 0 ? &tmTh : &tmU;
+            const CUtensorMap* tk = part == 0 ? &tmK : &tmV;
+            const int j0 = c * 16 * a.JC;
+            mbar_expect_tx(bar, a.par_bytes + 2 * a.k_half_bytes);
+            tma_load_4d(dst, tp, 0, j0, 0, h, bar);                  // parameters: never written by this library
+            if (first) { grid_dep_wait(); first = false; }            // everything else may come from the stream's previous kernel
+            tma_load_5d(dst + a.par_bytes, tk, 0, j0, r0, h, b0, bar);
+            tma_load_5d(dst + a.par_bytes + a.k_half_bytes, tk, 64, j0, r0, h, b0, bar);
           }
+          if (++slot == (uint32_t)a.stages) { slot = 0; phase ^= 1u; }
         }
       }
     }
-    if (dead) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
     return;
   }
 
   // ================= consumers =================
   const int gid = lane >> 2, t4 = lane & 3;
-  const int G = a.G, RB = a.RB, JC = a.JC, ncg = a.ncg;
-  const int WPG = FW / a.NB;                       // warps per sequence of the unit
+  const int G = a.G, RB = a.RB, JC = a.JC;
+  const int WPG = FWT / a.NB;                      // warps per sequence of the unit
   const int bl = warp / WPG, wig = warp - bl * WPG;
-  const int c0 = warp * ncg * 8;                   // first column of L owned by this warp
   const int rows16 = 16 * JC;                      // rows of one block inside a stage
+  const int sld = a.sld;
   const uint32_t sm_u = smem_addr(sm);
   const uint32_t q_u = sm_u + a.off_q, S_u = sm_u + a.off_S, W_u = sm_u + a.off_W;
   __nv_bfloat16* q_sm = reinterpret_cast<__nv_bfloat16*>(sm + a.off_q);
@@ -134,29 +139,52 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   __nv_bfloat16* W_sm = reinterpret_cast<__nv_bfloat16*>(sm + a.off_W);
   float* wred = reinterpret_cast<float*>(sm + a.off_wred);
   float* rmax = reinterpret_cast<float*>(sm + a.off_rstat);
-  float* rsum = rmax + FW * ROWS;
+  float* rsum = rmax + FWT * ROWS;
   float* tmax = reinterpret_cast<float*>(sm + a.off_tstat);
-  float* tsum = tmax + FW * 16;
+  float* tsum = tmax + FWT * 16;
   float* hmax = reinterpret_cast<float*>(sm + a.off_hstat);
   float* hsum = hmax + a.NB * 16;
   float* vsum = hsum + a.NB * 16;
   float* yred = reinterpret_cast<float*>(sm + a.off_yred);
   const float qscale = 0.08838834764831845f * 1.4426950408889634f;   // sigma = 1/sqrt(128), logits kept in log2 units
-  const int lrow = (lane & 7) + ((lane >> 3) & 1) * 8;              // ldmatrix row pattern: rows 0-15 in lanes 0-15, repeated
+  const int l7 = lane & 7;
+  const int lrow = l7 + ((lane >> 3) & 1) * 8;     // ldmatrix address pattern A: rows 0-15 by lanes 0-15, twice
   const int lhi = lane >> 4;
+  const int lrowB = l7 + lhi * 8;                  // address pattern B: rows 0-7 | 0-7 | 8-15 | 8-15
+  const int lmid = (lane >> 3) & 1;
+
+  // this warp's 16-column groups of the logits, and the byte offsets of its fragments inside a parameter tile
+  const int KT = a.n >> 4;
+  const int kt0 = warp * a.ktw;
+  const int my_kt = max(0, min(a.ktw, KT - kt0));
+  uint32_t th_off[KTW], u_off[KTW];                // theta: [k = row][n = col] read transposed;  U: [n = row][k = col]
+#pragma unroll
+  for (int kt = 0; kt < KTW; ++kt) {
+    const int ktc = kt < my_kt ? kt0 + kt : 0;
+    const int col_t = ktc * 16 + lhi * 8, col_u = ktc * 16 + lmid * 8;
+    th_off[kt] = (uint32_t)(((col_t >> 6) * rows16 + lrow) * 128 + ((((col_t & 63) >> 3) ^ l7) << 4));
+    u_off[kt] = (uint32_t)(((col_u >> 6) * rows16 + lrowB) * 128 + ((((col_u & 63) >> 3) ^ l7) << 4));
+  }
 
   grid_dep_wait();
   grid_dep_launch();
   if (blockIdx.x == 0 && tid == 0) *a.status = 0;
 
-  uint32_t it = 0;
+  uint32_t slot = 0, phase = 0;
   bool dead = false;
+  // the stage in `slot` has been consumed by this warp
+  auto release = [&]() {
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&empty_bar[slot]);
+    if (++slot == (uint32_t)a.stages) { slot = 0; phase ^= 1u; }
+  };
 
   for (int u = blockIdx.x; u < a.units; u += gridDim.x) {
     const int h = u / per_h, rem = u - h * per_h;
     const int bg = rem / a.nrg, rg = rem - bg * a.nrg;
     const int b0 = bg * a.NB, r0 = rg * a.RB;
     const int nbv = min(a.NB, a.B - b0);
+    const int rbv = min(RB, a.R - r0);
     const int ts0 = rg * a.Tper;
     const int ts1 = min(a.T, ts0 + a.Tper);
     const int nts = ts1 > ts0 ? (ts1 - ts0 + a.TCH - 1) / a.TCH : 0;
@@ -169,129 +197,127 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         v = *reinterpret_cast<const uint4*>(a.q + ((size_t)(b0 + tb) * a.H_kv * G + (size_t)h * G + g) * D + piece * 8);
       *reinterpret_cast<uint4*>(q_sm + (tb * 16 + g) * QLD + piece * 8) = v;
     }
-    consumer_sync();
+    named_barrier_sync(1, FCONS);
     uint32_t qf[NH][8][2];                          // B operand of the score MMA: heads of sequence bl
 #pragma unroll
     for (int nh = 0; nh < NH; ++nh)
 #pragma unroll
       for (int k2 = 0; k2 < 4; ++k2) {
         uint32_t r[4];
-        ldsm_x4(r, q_u + (uint32_t)(((bl * 16 + nh * 8 + (lane & 7)) * QLD + k2 * 32 + (lane >> 3) * 8) * 2));
+        ldsm_x4(r, q_u + (uint32_t)(((bl * 16 + nh * 8 + l7) * QLD + k2 * 32 + (lane >> 3) * 8) * 2));
         qf[nh][2 * k2][0] = r[0]; qf[nh][2 * k2][1] = r[1];
         qf[nh][2 * k2 + 1][0] = r[2]; qf[nh][2 * k2 + 1][1] = r[3];
       }
 
-    // expansion rows held by this lane: rho = mt*16 + gid + 8*hr  <->  (sequence, block, head)
-    bool rvalid[MT][2];
-    int rhead[MT][2];
+    // expansion rows held by this lane: rho = gid + 8*hr  <->  (sequence, block, head)
+    bool rvalid[2];
+    int rhead[2];
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-      for (int hr = 0; hr < 2; ++hr) {
-        const int rho = mt * 16 + gid + 8 * hr;
-        const int bi = rho / G, g = rho - bi * G;
-        const int rbl = bi / RB, rrl = bi - rbl * RB;
-        rvalid[mt][hr] = rho < a.NB * RB * G && rbl < nbv && r0 + rrl < a.R;
-        rhead[mt][hr] = rvalid[mt][hr] ? rbl * 16 + g : 0;
-      }
+    for (int hr = 0; hr < 2; ++hr) {
+      const int rho = gid + 8 * hr;
+      const int bi = rho / G, g = rho - bi * G;
+      const int rbl = bi / RB, rrl = bi - rbl * RB;
+      rvalid[hr] = rho < a.NB * RB * G && rbl < nbv && rrl < rbv;
+      rhead[hr] = rvalid[hr] ? rbl * 16 + g : 0;
+    }
 
-    float accL[MT][NTW][4];
+    float accL[2 * KTW][4];
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
+    for (int nt = 0; nt < 2 * KTW; ++nt)
 #pragma unroll
-      for (int nt = 0; nt < NTW; ++nt)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) accL[mt][nt][e] = 0.f;
+      for (int e = 0; e < 4; ++e) accL[nt][e] = 0.f;
 
     // =============================== pass A: scores and expansion by theta ===============================
     int buf = 0;
-    for (int c = 0; c < a.NJ; ++c, ++it) {
-      const uint32_t slot = it % a.stages, use = it / a.stages;
-      if (!dead && !mbar_wait_bounded(&full_bar[slot], use & 1u)) dead = true;
+    for (int c = 0; c < a.NJ; ++c) {
+      if (!dead && !mbar_wait_bounded(&full_bar[slot], phase)) dead = true;
       const uint32_t par_u = sm_u + slot * a.stage_bytes, k_u = par_u + a.par_bytes;
-      for (int s = 0; s < JC; ++s) {
-        if ((c * JC + s) * 16 >= a.m) break;
-        // S_c[rows of my blocks][16] = sigma q K_c^T
-        for (int rl = wig; rl < RB; rl += WPG) {
-          const int bi = bl * RB + rl;
-          const int row = bi * rows16 + s * 16 + lrow;
-          float sc[NH][4];
+      const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);          // 16-row sub-chunks with rows below m
+      __nv_bfloat16* Sb = S_sm + buf * (ROWS * sld);
+      // S[rows of block][16] = sigma q K^T for my (block, sub-chunk) tasks
+      for (int task = wig; task < RB * nsub; task += WPG) {
+        const int rl = task / nsub, s = task - rl * nsub;
+        const int bi = bl * RB + rl;
+        const uint32_t rowoff = k_u + (uint32_t)((bi * rows16 + s * 16 + lrow) * 128);
+        uint32_t af[8][4];
 #pragma unroll
-          for (int nh = 0; nh < NH; ++nh)
+        for (int ks = 0; ks < 8; ++ks)
+          ldsm_x4(af[ks], rowoff + (ks >> 2) * a.k_half_bytes + (uint32_t)(((((ks & 3) * 2 + lhi)) ^ l7) << 4));
+        float sc[NH][2][4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) sc[nh][e] = 0.f;
+        for (int nh = 0; nh < NH; ++nh)
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            uint32_t af[4];
-            ldsm_x4(af, k_u + (ks >> 2) * a.k_half_bytes + swz(row, (ks & 3) * 2 + lhi));
+          for (int x = 0; x < 2; ++x)
 #pragma unroll
-            for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(sc[nh], af, qf[nh][ks][0], qf[nh][ks][1]);
+            for (int e = 0; e < 4; ++e) sc[nh][x][e] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+#pragma unroll
+          for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(sc[nh][ks & 1], af[ks], qf[nh][ks][0], qf[nh][ks][1]);
+#pragma unroll
+        for (int nh = 0; nh < NH; ++nh)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int head = nh * 8 + 2 * t4 + (e & 1), j = gid + (e >> 1) * 8;
+            if (head < G) Sb[(bi * G + head) * sld + s * 16 + j] = __float2bfloat16_rn((sc[nh][0][e] + sc[nh][1][e]) * qscale);
           }
-          __nv_bfloat16* Sb = S_sm + buf * (ROWS * SLD);
-#pragma unroll
-          for (int nh = 0; nh < NH; ++nh)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int head = nh * 8 + 2 * t4 + (e & 1), j = gid + (e >> 1) * 8;
-              if (head < G) Sb[(bi * G + head) * SLD + j] = __float2bfloat16_rn(sc[nh][e] * qscale);
-            }
-        }
-        consumer_sync();
-        // L[:, my columns] += S_c theta_c
-        uint32_t af[MT][4];
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt)
-          ldsm_x4(af[mt], S_u + (uint32_t)((buf * (ROWS * SLD) + (mt * 16 + lrow) * SLD + lhi * 8) * 2));
-#pragma unroll
-        for (int np = 0; np < KK; ++np) {
-          if (2 * np < ncg) {
-            int col = c0 + np * 16 + lhi * 8;
-            if (col >= a.n) col = c0;
-            const int row = (col >> 6) * rows16 + s * 16 + lrow;
-            uint32_t bf[4];
-            ldsm_x4_t(bf, par_u + swz(row, (col & 63) >> 3));
-            const int n1 = 2 * np + 1 < NTW ? 2 * np + 1 : NTW - 1;
-#pragma unroll
-            for (int mt = 0; mt < MT; ++mt) {
-              mma_bf16_16816(accL[mt][2 * np], af[mt], bf[0], bf[1]);
-              if (2 * np + 1 < NTW && 2 * np + 1 < ncg) mma_bf16_16816(accL[mt][n1], af[mt], bf[2], bf[3]);
-            }
-          }
-        }
-        buf ^= 1;
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&empty_bar[slot]);
+      named_barrier_sync(1, FCONS);
+      // L[:, my column groups] += S theta
+      for (int s = 0; s < nsub; ++s) {
+        uint32_t as[4];
+        ldsm_x4(as, S_u + (uint32_t)((buf * (ROWS * sld) + lrow * sld + s * 16 + lhi * 8) * 2));
+        uint32_t bf[KTW][4];
+#pragma unroll
+        for (int kt = 0; kt < KTW; ++kt)
+          if (kt < my_kt) ldsm_x4_t(bf[kt], par_u + th_off[kt] + (uint32_t)(s * 2048));
+#pragma unroll
+        for (int kt = 0; kt < KTW; ++kt)
+          if (kt < my_kt) {
+            mma_bf16_16816(accL[2 * kt], as, bf[kt][0], bf[kt][1]);
+            mma_bf16_16816(accL[2 * kt + 1], as, bf[kt][2], bf[kt][3]);
+          }
+      }
+      buf ^= 1;
+      release();
     }
 
     // =============================== text rows: online-softmax attention per warp ===============================
-    float yacc[16][4];
+    // yacc[mt][nh]: y^T tile, rows = head-dimension mt*16 + gid (+8), columns = heads nh*8 + 2*t4 (+1) of sequence bl
+    float yacc[8][NH][4];
 #pragma unroll
-    for (int nt = 0; nt < 16; ++nt)
+    for (int mt = 0; mt < 8; ++mt)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) yacc[nt][e] = 0.f;
-    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-    for (int ts = 0; ts < nts; ++ts, ++it) {
-      const uint32_t slot = it % a.stages, use = it / a.stages;
-      if (!dead && !mbar_wait_bounded(&full_bar[slot], use & 1u)) dead = true;
+      for (int nh = 0; nh < NH; ++nh)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) yacc[mt][nh][e] = 0.f;
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // heads gid and gid + 8
+    for (int ts = 0; ts < nts; ++ts) {
+      if (!dead && !mbar_wait_bounded(&full_bar[slot], phase)) dead = true;
       const uint32_t kt_u = sm_u + slot * a.stage_bytes, vt_u = kt_u + 2 * a.txt_half_bytes;
       for (int tile = wig; tile * 16 < a.TCH; tile += WPG) {
         const int t_first = ts0 + ts * a.TCH + tile * 16;
         if (t_first >= ts1) break;
         const int row0 = bl * a.TCH + tile * 16;
+        const uint32_t rowB = (uint32_t)((row0 + lrowB) * 128);
+        // logits [16 heads][16 text rows] = q K_txt^T
         float cc[2][4];
 #pragma unroll
         for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
           for (int e = 0; e < 4; ++e) cc[nt][e] = 0.f;
+        {
+          uint32_t bk[8][4];
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          uint32_t aq[4], bk[4];
-          ldsm_x4(aq, q_u + (uint32_t)(((bl * 16 + lrow) * QLD + ks * 16 + lhi * 8) * 2));
-          ldsm_x4(bk, kt_u + (ks >> 2) * a.txt_half_bytes +
-                          swz(row0 + (lane & 7) + lhi * 8, (ks & 3) * 2 + ((lane >> 3) & 1)));
-          mma_bf16_16816(cc[0], aq, bk[0], bk[1]);
-          mma_bf16_16816(cc[1], aq, bk[2], bk[3]);
+          for (int ks = 0; ks < 8; ++ks)
+            ldsm_x4(bk[ks], kt_u + (ks >> 2) * a.txt_half_bytes + rowB + (uint32_t)(((((ks & 3) * 2 + lmid)) ^ l7) << 4));
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            uint32_t aq[4];
+            ldsm_x4(aq, q_u + (uint32_t)(((bl * 16 + lrow) * QLD + ks * 16 + lhi * 8) * 2));
+            mma_bf16_16816(cc[0], aq, bk[ks][0], bk[ks][1]);
+            mma_bf16_16816(cc[1], aq, bk[ks][2], bk[ks][3]);
+          }
         }
         // cc[nt][e]: head gid + 8*(e>>1), text row t_first + nt*8 + 2*t4 + (e&1)
 #pragma unroll
@@ -301,13 +327,14 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             const int t = t_first + nt * 8 + 2 * t4 + (e & 1);
             cc[nt][e] = t < ts1 ? cc[nt][e] * qscale : -INFINITY;
           }
+        float scl[2];
 #pragma unroll
         for (int hr = 0; hr < 2; ++hr) {
           float mx = fmaxf(fmaxf(cc[0][2 * hr], cc[0][2 * hr + 1]), fmaxf(cc[1][2 * hr], cc[1][2 * hr + 1]));
           mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
           mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
           const float m_new = fmaxf(m_run[hr], mx);              // finite: the tile has at least one valid row
-          const float scl = fast_exp2(m_run[hr] - m_new);        // 0 on the first tile
+          scl[hr] = fast_exp2(m_run[hr] - m_new);                // 0 on the first tile
           m_run[hr] = m_new;
           float ps = 0.f;
 #pragma unroll
@@ -318,224 +345,248 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
               cc[nt][2 * hr + k] = p;
               ps += p;
             }
-          l_run[hr] = l_run[hr] * scl + ps;
-          if (scl != 1.f) {
+          l_run[hr] = l_run[hr] * scl[hr] + ps;
+        }
+        // the accumulator's columns are heads: fetch their factors from the lanes that own those heads as rows
 #pragma unroll
-            for (int nt = 0; nt < 16; ++nt) { yacc[nt][2 * hr] *= scl; yacc[nt][2 * hr + 1] *= scl; }
+        for (int nh = 0; nh < NH; ++nh) {
+          const float c0s = __shfl_sync(0xffffffffu, scl[nh], (2 * t4) * 4);
+          const float c1s = __shfl_sync(0xffffffffu, scl[nh], (2 * t4 + 1) * 4);
+          if (c0s != 1.f || c1s != 1.f) {
+#pragma unroll
+            for (int mt = 0; mt < 8; ++mt) {
+              yacc[mt][nh][0] *= c0s; yacc[mt][nh][1] *= c1s;
+              yacc[mt][nh][2] *= c0s; yacc[mt][nh][3] *= c1s;
+            }
           }
         }
-        uint32_t pa[4];
-        pa[0] = pack2_bf16(cc[0][0], cc[0][1]); pa[1] = pack2_bf16(cc[0][2], cc[0][3]);
-        pa[2] = pack2_bf16(cc[1][0], cc[1][1]); pa[3] = pack2_bf16(cc[1][2], cc[1][3]);
+        // y^T[128][heads] += V_txt^T[128][16 rows] P^T[16 rows][heads]
+        uint32_t pb[2][2];
+        pb[0][0] = pack2_bf16(cc[0][0], cc[0][1]); pb[0][1] = pack2_bf16(cc[1][0], cc[1][1]);
+        pb[1][0] = pack2_bf16(cc[0][2], cc[0][3]); pb[1][1] = pack2_bf16(cc[1][2], cc[1][3]);
+        uint32_t av[8][4];
 #pragma unroll
-        for (int np = 0; np < 8; ++np) {
-          const int col = np * 16 + lhi * 8;
-          uint32_t bv[4];
-          ldsm_x4_t(bv, vt_u + (col >> 6) * a.txt_half_bytes + swz(row0 + lrow, (col & 63) >> 3));
-          mma_bf16_16816(yacc[2 * np], pa, bv[0], bv[1]);
-          mma_bf16_16816(yacc[2 * np + 1], pa, bv[2], bv[3]);
-        }
+        for (int mt = 0; mt < 8; ++mt)
+          ldsm_x4_t(av[mt], vt_u + (mt >> 2) * a.txt_half_bytes + rowB + (uint32_t)(((((mt & 3) * 2 + lmid)) ^ l7) << 4));
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+          for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(yacc[mt][nh], av[mt], pb[nh][0], pb[nh][1]);
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&empty_bar[slot]);
+      release();
     }
 
     // =============================== joint softmax over the unit's blocks and text rows ===============================
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
+    for (int hr = 0; hr < 2; ++hr) {
+      float mx = -INFINITY;
 #pragma unroll
-      for (int hr = 0; hr < 2; ++hr) {
+      for (int nt = 0; nt < 2 * KTW; ++nt)
+        if (nt < 2 * my_kt) mx = fmaxf(mx, fmaxf(accL[nt][2 * hr], accL[nt][2 * hr + 1]));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      if (t4 == 0) rmax[warp * ROWS + gid + 8 * hr] = rvalid[hr] ? mx : -INFINITY;
+    }
+    if (t4 == 0) { tmax[warp * 16 + gid] = m_run[0]; tmax[warp * 16 + gid + 8] = m_run[1]; }
+    named_barrier_sync(1, FCONS);
+    if (warp == 0) {
+      // maximum of every expansion row over the warps, then of every (sequence, head) over its blocks and text rows
+      if (lane < ROWS) {
         float mx = -INFINITY;
 #pragma unroll
-        for (int nt = 0; nt < NTW; ++nt)
-          if (nt < ncg) mx = fmaxf(mx, fmaxf(accL[mt][nt][2 * hr], accL[mt][nt][2 * hr + 1]));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-        if (t4 == 0) rmax[warp * ROWS + mt * 16 + gid + 8 * hr] = rvalid[mt][hr] ? mx : -INFINITY;
+        for (int w = 0; w < FWT; ++w) mx = fmaxf(mx, rmax[w * ROWS + lane]);
+        rmax[lane] = mx;
       }
-    if (t4 == 0) { tmax[warp * 16 + gid] = m_run[0]; tmax[warp * 16 + gid + 8] = m_run[1]; }
-    consumer_sync();
-    if (tid < a.NB * 16) {
-      const int tb = tid >> 4, g = tid & 15;
-      float mx = 0.f;
-      if (g < G && tb < nbv) {
-        mx = -INFINITY;
-        for (int rl = 0; rl < RB; ++rl)
-          if (r0 + rl < a.R)
-            for (int w = 0; w < FW; ++w) mx = fmaxf(mx, rmax[w * ROWS + (tb * RB + rl) * G + g]);
-        for (int w = tb * WPG; w < (tb + 1) * WPG; ++w) mx = fmaxf(mx, tmax[w * 16 + g]);
-      }
-      hmax[tid] = mx;
-    }
-    consumer_sync();
-    uint32_t pf[MT][KK][4];                         // P as A operand of the re-projection (bf16), this warp's columns
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
-#pragma unroll
-      for (int hr = 0; hr < 2; ++hr) {
-        const bool ok = rvalid[mt][hr];
-        const float M = hmax[rhead[mt][hr]];
-        float sum = 0.f;
-#pragma unroll
-        for (int nt = 0; nt < NTW; ++nt)
-#pragma unroll
-          for (int k = 0; k < 2; ++k) {
-            const float p = (ok && nt < ncg) ? fast_exp2(accL[mt][nt][2 * hr + k] - M) : 0.f;
-            accL[mt][nt][2 * hr + k] = p;
-            sum += p;
-          }
-        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-        if (t4 == 0) rsum[warp * ROWS + mt * 16 + gid + 8 * hr] = sum;
-      }
-#pragma unroll
-      for (int kk = 0; kk < KK; ++kk) {
-        pf[mt][kk][0] = pack2_bf16(accL[mt][2 * kk][0], accL[mt][2 * kk][1]);
-        pf[mt][kk][1] = pack2_bf16(accL[mt][2 * kk][2], accL[mt][2 * kk][3]);
-        const int n1 = 2 * kk + 1 < NTW ? 2 * kk + 1 : NTW - 1;
-        pf[mt][kk][2] = 2 * kk + 1 < NTW ? pack2_bf16(accL[mt][n1][0], accL[mt][n1][1]) : 0u;
-        pf[mt][kk][3] = 2 * kk + 1 < NTW ? pack2_bf16(accL[mt][n1][2], accL[mt][n1][3]) : 0u;
+      __syncwarp();
+      for (int x = lane; x < a.NB * 16; x += 32) {
+        const int tb = x >> 4, g = x & 15;
+        float mx = 0.f;
+        if (g < G && tb < nbv) {
+          mx = -INFINITY;
+          for (int rl = 0; rl < rbv; ++rl) mx = fmaxf(mx, rmax[(tb * RB + rl) * G + g]);
+          for (int w = tb * WPG; w < (tb + 1) * WPG; ++w) mx = fmaxf(mx, tmax[w * 16 + g]);
+        }
+        hmax[x] = mx;
       }
     }
-    // the text accumulators move to the same reference maximum
+    named_barrier_sync(1, FCONS);
+    uint32_t pf[KTW][4];                            // P (bf16) of this warp's column groups, as MMA operand fragments
 #pragma unroll
     for (int hr = 0; hr < 2; ++hr) {
-      const int head = gid + 8 * hr;
-      const float M = hmax[bl * 16 + head];
-      const float scl = m_run[hr] == -INFINITY ? 0.f : fast_exp2(m_run[hr] - M);
-      float l = l_run[hr] * scl;
-      l += __shfl_xor_sync(0xffffffffu, l, 1);
-      l += __shfl_xor_sync(0xffffffffu, l, 2);
+      const bool ok = rvalid[hr];
+      const float M = hmax[rhead[hr]];
+      float sum = 0.f;
 #pragma unroll
-      for (int nt = 0; nt < 16; ++nt) { yacc[nt][2 * hr] *= scl; yacc[nt][2 * hr + 1] *= scl; }
-      if (t4 == 0) tsum[warp * 16 + head] = l;
+      for (int nt = 0; nt < 2 * KTW; ++nt)
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+          const float p = (ok && nt < 2 * my_kt) ? fast_exp2(accL[nt][2 * hr + k] - M) : 0.f;
+          accL[nt][2 * hr + k] = p;
+          sum += p;
+        }
+      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+      if (t4 == 0) rsum[warp * ROWS + gid + 8 * hr] = sum;
     }
-    consumer_sync();
-    if (tid < a.NB * 16) {
-      const int tb = tid >> 4, g = tid & 15;
-      float vs = 0.f, tsm = 0.f;
-      if (g < G && tb < nbv) {
-        for (int rl = 0; rl < RB; ++rl)
-          if (r0 + rl < a.R)
-            for (int w = 0; w < FW; ++w) vs += rsum[w * ROWS + (tb * RB + rl) * G + g];
-        for (int w = tb * WPG; w < (tb + 1) * WPG; ++w) tsm += tsum[w * 16 + g];
+#pragma unroll
+    for (int kt = 0; kt < KTW; ++kt) {
+      pf[kt][0] = pack2_bf16(accL[2 * kt][0], accL[2 * kt][1]);
+      pf[kt][1] = pack2_bf16(accL[2 * kt][2], accL[2 * kt][3]);
+      pf[kt][2] = pack2_bf16(accL[2 * kt + 1][0], accL[2 * kt + 1][1]);
+      pf[kt][3] = pack2_bf16(accL[2 * kt + 1][2], accL[2 * kt + 1][3]);
+    }
+    // the text accumulators move to the same reference maximum
+    {
+      float scl[2];
+#pragma unroll
+      for (int hr = 0; hr < 2; ++hr) {
+        const int head = gid + 8 * hr;
+        const float M = hmax[bl * 16 + head];
+        scl[hr] = m_run[hr] == -INFINITY ? 0.f : fast_exp2(m_run[hr] - M);
+        float l = l_run[hr] * scl[hr];
+        l += __shfl_xor_sync(0xffffffffu, l, 1);
+        l += __shfl_xor_sync(0xffffffffu, l, 2);
+        if (t4 == 0) tsum[warp * 16 + head] = l;
       }
-      vsum[tid] = vs;
-      hsum[tid] = vs + tsm;
+#pragma unroll
+      for (int nh = 0; nh < NH; ++nh) {
+        const float c0s = __shfl_sync(0xffffffffu, scl[nh], (2 * t4) * 4);
+        const float c1s = __shfl_sync(0xffffffffu, scl[nh], (2 * t4 + 1) * 4);
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt) {
+          yacc[mt][nh][0] *= c0s; yacc[mt][nh][1] *= c1s;
+          yacc[mt][nh][2] *= c0s; yacc[mt][nh][3] *= c1s;
+        }
+      }
+    }
+    named_barrier_sync(1, FCONS);
+    if (warp == 0) {
+      if (lane < ROWS) {
+        float sm_ = 0.f;
+#pragma unroll
+        for (int w = 0; w < FWT; ++w) sm_ += rsum[w * ROWS + lane];
+        rsum[lane] = sm_;
+      }
+      __syncwarp();
+      for (int x = lane; x < a.NB * 16; x += 32) {
+        const int tb = x >> 4, g = x & 15;
+        float vs = 0.f, tsm = 0.f;
+        if (g < G && tb < nbv) {
+          for (int rl = 0; rl < rbv; ++rl) vs += rsum[(tb * RB + rl) * G + g];
+          for (int w = tb * WPG; w < (tb + 1) * WPG; ++w) tsm += tsum[w * 16 + g];
+        }
+        vsum[x] = vs;
+        hsum[x] = vs + tsm;
+      }
     }
 
     // =============================== pass C: re-projection by U^T and product with V_tilde ===============================
-    for (int c = 0; c < a.NJ; ++c, ++it) {
-      const uint32_t slot = it % a.stages, use = it / a.stages;
-      if (!dead && !mbar_wait_bounded(&full_bar[slot], use & 1u)) dead = true;
+    const int msplit = a.msplit, mshift = a.mshift;           // a task covers the row tiles mt with (mt >> mshift) == its group
+    for (int c = 0; c < a.NJ; ++c) {
+      if (!dead && !mbar_wait_bounded(&full_bar[slot], phase)) dead = true;
       const uint32_t par_u = sm_u + slot * a.stage_bytes, v_u = par_u + a.par_bytes;
-      for (int s = 0; s < JC; ++s) {
-        if ((c * JC + s) * 16 >= a.m) break;
-        // partial W_c[rows][16] over this warp's columns of P
-        float wc[MT][2][4];
+      const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);
+      for (int s = 0; s < nsub; ++s) {
+        // partial W[rows][16] over this warp's columns of P
+        float wc[2][4];
 #pragma unroll
-        for (int mt = 0; mt < MT; ++mt)
+        for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-          for (int nt = 0; nt < 2; ++nt)
+          for (int e = 0; e < 4; ++e) wc[nt][e] = 0.f;
+        {
+          uint32_t bu[KTW][4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) wc[mt][nt][e] = 0.f;
+          for (int kt = 0; kt < KTW; ++kt)
+            if (kt < my_kt) ldsm_x4(bu[kt], par_u + u_off[kt] + (uint32_t)(s * 2048));
 #pragma unroll
-        for (int kk = 0; kk < KK; ++kk) {
-          if (2 * kk < ncg) {
-            int col = c0 + kk * 16 + ((lane >> 3) & 1) * 8;
-            if (col >= a.n) col = c0;
-            const int row = (col >> 6) * rows16 + s * 16 + (lane & 7) + lhi * 8;
-            uint32_t bu[4];
-            ldsm_x4(bu, par_u + swz(row, (col & 63) >> 3));
+          for (int kt = 0; kt < KTW; ++kt)
+            if (kt < my_kt) {
+              mma_bf16_16816(wc[0], pf[kt], bu[kt][0], bu[kt][1]);
+              mma_bf16_16816(wc[1], pf[kt], bu[kt][2], bu[kt][3]);
+            }
+        }
+        float* wr = wred + warp * (ROWS * 16);
 #pragma unroll
-            for (int mt = 0; mt < MT; ++mt) {
-              mma_bf16_16816(wc[mt][0], pf[mt][kk], bu[0], bu[1]);
-              mma_bf16_16816(wc[mt][1], pf[mt][kk], bu[2], bu[3]);
+        for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+          for (int hr = 0; hr < 2; ++hr)
+            *reinterpret_cast<float2*>(&wr[(gid + 8 * hr) * 16 + nt * 8 + 2 * t4]) = make_float2(wc[nt][2 * hr], wc[nt][2 * hr + 1]);
+        named_barrier_sync(1, FCONS);
+        if (tid < ROWS * 16) {
+          const float* wp = wred + tid;
+          float w = 0.f;
+#pragma unroll
+          for (int x = 0; x < FWT; ++x) w += wp[x * ROWS * 16];
+          W_sm[(tid >> 4) * SLD + (tid & 15)] = __float2bfloat16_rn(w);
+        }
+        named_barrier_sync(1, FCONS);
+        // y^T[128][heads] += V^T[128][16 rows of block] W^T[16][heads of block], my (block, row-tile group) tasks
+        for (int task = wig; task < RB * msplit; task += WPG) {
+          const int rl = task >> (3 - mshift), mg = task & (msplit - 1);
+          if (rl >= rbv || bl >= nbv) continue;
+          const int bi = bl * RB + rl;
+          uint32_t bw[4];
+          ldsm_x4(bw, W_u + (uint32_t)(((bi * G + lrowB) * SLD + lmid * 8) * 2));
+          const uint32_t rowoff = v_u + (uint32_t)((bi * rows16 + s * 16 + lrowB) * 128);
+#pragma unroll
+          for (int mt = 0; mt < 8; ++mt) {
+            if ((mt >> mshift) == mg) {
+              uint32_t av[4];
+              ldsm_x4_t(av, rowoff + (mt >> 2) * a.k_half_bytes + (uint32_t)(((((mt & 3) * 2 + lmid)) ^ l7) << 4));
+#pragma unroll
+              for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(yacc[mt][nh], av, bw[2 * nh], bw[2 * nh + 1]);
             }
           }
         }
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-          for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-            for (int hr = 0; hr < 2; ++hr)
-              *reinterpret_cast<float2*>(&wred[(warp * ROWS + mt * 16 + gid + 8 * hr) * 16 + nt * 8 + 2 * t4]) =
-                  make_float2(wc[mt][nt][2 * hr], wc[mt][nt][2 * hr + 1]);
-        consumer_sync();
-        for (int idx = tid; idx < ROWS * 16; idx += FCONS) {
-          float w = 0.f;
-#pragma unroll
-          for (int x = 0; x < FW; ++x) w += wred[x * ROWS * 16 + idx];
-          W_sm[(idx >> 4) * SLD + (idx & 15)] = __float2bfloat16_rn(w);
-        }
-        consumer_sync();
-        // y[heads of sequence bl] += W_c[rows of block] V_c[block]
-        for (int rl = wig; rl < RB; rl += WPG) {
-          if (r0 + rl >= a.R || bl >= nbv) continue;
-          const int bi = bl * RB + rl;
-          uint32_t aw[4];
-          ldsm_x4(aw, W_u + (uint32_t)(((bi * G + lrow) * SLD + lhi * 8) * 2));
-          const int row = bi * rows16 + s * 16 + lrow;
-#pragma unroll
-          for (int np = 0; np < 8; ++np) {
-            const int col = np * 16 + lhi * 8;
-            uint32_t bv[4];
-            ldsm_x4_t(bv, v_u + (col >> 6) * a.k_half_bytes + swz(row, (col & 63) >> 3));
-            mma_bf16_16816(yacc[2 * np], aw, bv[0], bv[1]);
-            mma_bf16_16816(yacc[2 * np + 1], aw, bv[2], bv[3]);
-          }
-        }
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&empty_bar[slot]);
+      release();
     }
 
     // =============================== unit end: reduce over warps, mu term, normalise or leave a partial ===============================
-    for (int k = 0; k < WPG; ++k) {
-      if (wig == k) {
+    const int bh = b0 * a.H_kv + h;                    // used when the block axis is split (NB == 1)
+    const size_t pbase = ((size_t)bh * a.nrg + rg) * G;
+    for (int g0 = 0; g0 < G; g0 += YHG) {
+      // every warp parks its tile columns of heads g0 .. g0+YHG-1; then the warps of a sequence are summed
 #pragma unroll
-        for (int hr = 0; hr < 2; ++hr) {
-          const int head = gid + 8 * hr;
-          if (head < G) {
+      for (int nh = 0; nh < NH; ++nh)
 #pragma unroll
-            for (int nt = 0; nt < 16; ++nt) {
-              float2* p = reinterpret_cast<float2*>(&yred[(bl * 16 + head) * D + nt * 8 + 2 * t4]);
-              float2 v = make_float2(yacc[nt][2 * hr], yacc[nt][2 * hr + 1]);
-              if (k > 0) { const float2 o = *p; v.x += o.x; v.y += o.y; }
-              *p = v;
+        for (int e = 0; e < 2; ++e) {
+          const int head = nh * 8 + 2 * t4 + e;
+          if (head >= g0 && head < g0 + YHG && head < G) {
+            float* yp = yred + (warp * YHG + (head - g0)) * D;
+#pragma unroll
+            for (int mt = 0; mt < 8; ++mt) {
+              yp[mt * 16 + gid] = yacc[mt][nh][e];
+              yp[mt * 16 + gid + 8] = yacc[mt][nh][2 + e];
             }
           }
         }
+      named_barrier_sync(1, FCONS);
+      const int hg = min(YHG, G - g0);
+      for (int idx = tid; idx < nbv * hg * D; idx += FCONS) {
+        const int col = idx & (D - 1), gg = (idx >> 7) % hg, tb = idx / (D * hg);
+        const int g = g0 + gg;
+        float y = 0.f;
+        for (int w = tb * WPG; w < (tb + 1) * WPG; ++w) y += yred[(w * YHG + gg) * D + col];
+        y = fmaf(vsum[tb * 16 + g], __bfloat162float(a.mu[h * D + col]), y);
+        if (a.nrg == 1)
+          a.out[((size_t)(b0 + tb) * a.H_kv * G + (size_t)h * G + g) * D + col] = __float2bfloat16_rn(y / hsum[tb * 16 + g]);
+        else
+          a.part_y[(pbase + g) * D + col] = y;
       }
-      consumer_sync();
+      named_barrier_sync(1, FCONS);
     }
-    if (a.nrg == 1) {
-      for (int idx = tid; idx < nbv * G * 64; idx += FCONS) {
-        const int cp = idx & 63, g = (idx >> 6) % G, tb = idx / (64 * G);
-        const float2 y = *reinterpret_cast<const float2*>(&yred[(tb * 16 + g) * D + 2 * cp]);
-        const __nv_bfloat162 mu2 = *reinterpret_cast<const __nv_bfloat162*>(a.mu + h * D + 2 * cp);
-        const float vs = vsum[tb * 16 + g], inv = 1.f / hsum[tb * 16 + g];
-        const __nv_bfloat162 o = __floats2bfloat162_rn(fmaf(vs, __low2float(mu2), y.x) * inv, fmaf(vs, __high2float(mu2), y.y) * inv);
-        *reinterpret_cast<__nv_bfloat162*>(a.out + ((size_t)(b0 + tb) * a.H_kv * G + (size_t)h * G + g) * D + 2 * cp) = o;
-      }
-    } else {
-      // NB == 1 here: one sequence, several units along the block axis
-      const int bh = b0 * a.H_kv + h;
-      const size_t pbase = ((size_t)bh * a.nrg + rg) * G;
-      for (int idx = tid; idx < G * D; idx += FCONS) {
-        const int g = idx >> 7, col = idx & (D - 1);
-        a.part_y[(pbase + g) * D + col] = fmaf(vsum[g], __bfloat162float(a.mu[h * D + col]), yred[g * D + col]);
-      }
+    if (a.nrg > 1) {
+      // one sequence, several units along the block axis: the last unit to arrive merges the partials
       if (tid < G) a.part_ml[pbase + tid] = make_float2(hmax[tid], hsum[tid]);
       __threadfence();
-      consumer_sync();
+      named_barrier_sync(1, FCONS);
       if (tid == 0) {
         const int old = atomicAdd(&a.cnt[bh], 1);
         s_last = old == a.nrg - 1 ? 1 : 0;
         if (s_last) a.cnt[bh] = 0;                  // every unit of (sequence, head) has arrived: ready for the next call
       }
-      consumer_sync();
+      named_barrier_sync(1, FCONS);
       if (s_last) {
         __threadfence();
         const size_t p0 = (size_t)bh * a.nrg * G;
@@ -553,8 +604,8 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           a.out[((size_t)b0 * a.H_kv * G + (size_t)h * G + g) * D + col] = __float2bfloat16_rn(num / den);
         }
       }
+      named_barrier_sync(1, FCONS);
     }
-    consumer_sync();
   }
   if (dead && lane == 0) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
 }
@@ -591,21 +642,30 @@ bool encode_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// consumer warps for a block length n: the 16-column groups of the logits should divide evenly
+static int consumer_warps(int n) {
+  const int KT = n / 16;
+  if (KT % 12 == 0 && KT / 12 <= 3) return 12;   // n = 576 (24 x 24 grids): 3 groups per warp
+  return 8;
+}
+
 FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
   FusedPlan p{};
   const int G = L->G, n = L->desc.n, m = L->m, H_kv = L->desc.H_kv;
   if (L->desc.dtype != KVC_BF16 || L->passthrough || R < 1 || B < 1 || n % 64 != 0 || n > 1024 || G > 16) return p;
   if (reinterpret_cast<uintptr_t>(L->desc.theta) & 15 || reinterpret_cast<uintptr_t>(L->desc.U) & 15) return p;
   const int sms = L->num_sms > 0 ? L->num_sms : 148;
+  p.FW = consumer_warps(n);
+  p.ktw = ceil_div(n / 16, p.FW);
   p.MT = 1;
-  const int cap = 16 * p.MT;
+  const int cap = ROWS;
   p.RB = R < cap / G ? R : cap / G;
   p.NB = 1;
   if (p.RB == R) {
     // whole sequences per unit: more sequences per unit share one pass over theta[h] and U[h]
     double best = 0;
     for (int nb = 1; nb <= 4; nb *= 2) {
-      if (nb > 1 && (nb * R * G > cap || nb > B)) break;
+      if (nb > 1 && (nb * R * G > cap || nb > B || p.FW % nb != 0)) break;
       const long long units = (long long)H_kv * ceil_div(B, nb);
       const double cost = (double)ceil_div((int)units, sms) * ((double)nb * R * m * 512.0 + 4.0 * m * n);
       if (nb == 1 || cost < best) { best = cost; p.NB = nb; }
@@ -628,17 +688,26 @@ FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
   p.TCH = tch > 256 ? 256 : tch;
   if (p.TCH < 16) return p;
   p.txt_half_bytes = (uint32_t)p.NB * p.TCH * 128u;
-  const int rows = 16 * p.MT;
+  {
+    // the 8 row tiles of a value block go to `msplit` tasks so that the warps of a sequence share the work evenly
+    const int wpg = p.FW / p.NB;
+    int best = 1 << 30;
+    for (int sh = 3; sh >= 0; --sh) {            // sh = 3: one task per block
+      const int ms = 8 >> sh, cost = ceil_div(p.RB * ms, wpg) * ((1 << sh) + 1);
+      if (cost < best) { best = cost; p.msplit = ms; p.mshift = sh; }
+    }
+  }
+  p.sld = 16 * p.JC + 8;
   uint32_t off = 0;
   auto take = [&](uint32_t bytes) { uint32_t o = off; off = (off + bytes + 127u) & ~127u; return o; };
   p.off_q = take((uint32_t)p.NB * 16 * QLD * 2);
-  p.off_S = take((uint32_t)(2 * rows * SLD + (rows + 16) * SLD) * 2);
-  p.off_W = p.off_S + (uint32_t)2 * rows * SLD * 2;
-  p.off_wred = take((uint32_t)FW * rows * 16 * 4);
-  p.off_rstat = take((uint32_t)2 * FW * rows * 4);
-  p.off_tstat = take((uint32_t)2 * FW * 16 * 4);
+  p.off_S = take((uint32_t)(2 * ROWS * p.sld + (ROWS + 16) * SLD) * 2);
+  p.off_W = p.off_S + (uint32_t)2 * ROWS * p.sld * 2;
+  p.off_wred = take((uint32_t)p.FW * ROWS * 16 * 4);
+  p.off_rstat = take((uint32_t)2 * p.FW * ROWS * 4);
+  p.off_tstat = take((uint32_t)2 * p.FW * 16 * 4);
   p.off_hstat = take((uint32_t)3 * p.NB * 16 * 4);
-  p.off_yred = take((uint32_t)p.NB * 16 * D * 4);
+  p.off_yred = take((uint32_t)p.FW * YHG * D * 4);
   p.misc_bytes = off;
   const uint32_t avail = SMEM_LIMIT - 1024u - 2048u - p.misc_bytes;   // alignment slack; static shared memory and its padding
   int stages = (int)(avail / p.stage_bytes);
@@ -650,17 +719,24 @@ FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
   return p;
 }
 
-template <int MT, int NTW, int NH>
+template <int FWT, int KTW, int NH>
 static cudaError_t launch_inst(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
   static size_t configured = 0;
   if (p.smem_bytes > configured) {
-    cudaError_t e = cudaFuncSetAttribute(fused_decode_kernel<MT, NTW, NH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(fused_decode_kernel<FWT, KTW, NH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)p.smem_bytes);
     if (e != cudaSuccess) return e;
     configured = p.smem_bytes;
   }
-  return launch_dependent(fused_decode_kernel<MT, NTW, NH>, dim3(p.grid), dim3(FTHREADS), p.smem_bytes, st, tm[0], tm[1],
-                          tm[2], tm[3], tm[4], tm[5], fa);
+  return launch_dependent(fused_decode_kernel<FWT, KTW, NH>, dim3(p.grid), dim3((FWT + 1) * 32), p.smem_bytes, st, tm[0],
+                          tm[1], tm[2], tm[3], tm[4], tm[5], fa);
+}
+
+template <int NH>
+static cudaError_t launch_nh(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
+  if (p.FW == 12) return launch_inst<12, 3, NH>(tm, fa, p, st);
+  if (p.ktw <= 2) return launch_inst<8, 2, NH>(tm, fa, p, st);
+  return launch_inst<8, 8, NH>(tm, fa, p, st);
 }
 
 cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPlan& p, cudaStream_t st, bool* encoded) {
@@ -701,6 +777,7 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
   fa.B = B; fa.H_kv = H_kv; fa.G = a.G; fa.R = R; fa.m = m; fa.n = n; fa.T = a.T;
   fa.NB = p.NB; fa.RB = p.RB; fa.nbg = p.nbg; fa.nrg = p.nrg; fa.units = p.units; fa.JC = p.JC; fa.NJ = p.NJ;
   fa.TCH = p.TCH; fa.ncg = p.ncg; fa.stages = p.stages;
+  fa.ktw = p.ktw; fa.msplit = p.msplit; fa.mshift = p.mshift; fa.sld = p.sld;
   fa.Tper = (ceil_div(a.T > 0 ? a.T : 1, p.nrg) + 15) & ~15;
   fa.par_bytes = p.par_bytes; fa.k_half_bytes = p.k_half_bytes; fa.txt_half_bytes = p.txt_half_bytes;
   fa.stage_bytes = p.stage_bytes;
@@ -714,10 +791,7 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
   fa.status = a.status;
 
   ProfScope prof(KVC_KERNEL_FUSED, st);
-  const bool nh2 = a.G > 8;
-  if (p.ncg <= 4) return nh2 ? launch_inst<1, 4, 2>(tm, fa, p, st) : launch_inst<1, 4, 1>(tm, fa, p, st);
-  if (p.ncg <= 9) return nh2 ? launch_inst<1, 9, 2>(tm, fa, p, st) : launch_inst<1, 9, 1>(tm, fa, p, st);
-  return nh2 ? launch_inst<1, 16, 2>(tm, fa, p, st) : launch_inst<1, 16, 1>(tm, fa, p, st);
+  return a.G > 8 ? launch_nh<2>(tm, fa, p, st) : launch_nh<1>(tm, fa, p, st);
 }
 
 }  // namespace kvc

@@ -85,6 +85,9 @@ struct FusedPlan {
   int JC, NJ;        // 16-row sub-chunks of the m axis per stage; stages per pass over the m axis
   int TCH;           // text rows per stage and sequence
   int ncg;           // n / 64
+  int FW, ktw;       // consumer warps; 16-column groups of the logits per warp
+  int msplit, mshift;// the 8 row tiles of a value block go to msplit = 8 >> mshift tasks
+  int sld;           // row stride of the score tile
   int stages, grid;
   uint32_t par_bytes, k_half_bytes, txt_half_bytes, stage_bytes, misc_bytes;
   uint32_t off_q, off_S, off_W, off_wred, off_rstat, off_tstat, off_hstat, off_yred;   // relative to the end of the ring
@@ -108,6 +111,7 @@ struct kvc_layer {
 namespace kvc {
 
 WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap);
+int cuda_status(cudaError_t e);   // KVC_OK or KVC_ERR_CUDA, remembering the error for kvc_last_cuda_error
 FusedPlan plan_fused(const kvc_layer* L, int B, int R);
 
 struct DecodeArgs {
