@@ -3,22 +3,23 @@
 //
 // Work unit = one KV head h, NB sequences and RB vision blocks of each (NB*RB*G <= 16 expansion rows),
 // plus a slice of the sequences' text rows.  A persistent CTA streams, per unit, through a ring of large
-// shared-memory stages filled by the TMA engine (tiled tensor maps, 128-byte swizzle):
-//   pass A   stage c = rows [16 JC c, 16 JC (c+1)) of K_tilde of every block of the unit  +  the same rows
-//            of theta[h] (all n columns).  Scores S_c = sigma q K_c^T go through shared memory as bf16 and
-//            are multiplied into the logits L += S_c theta_c, which stay in registers (rows x n, fp32,
-//            every warp owning a range of 16-column groups).
-//   text     stage = TCH rows of K_txt and V_txt per sequence; every warp runs an online-softmax
-//            attention over its own 16-row tiles.
-//   softmax  one maximum per (sequence, head) over all blocks of the unit and its text rows; P = 2^(L - max).
-//   pass C   stage c = rows of V_tilde + the same rows of U[h]:  W_c = P U_c^T (split over the warps' column
-//            ranges, reduced through shared memory), then y^T += V_c^T W_c^T.
-// theta/U rows (L2-resident, shared by all sequences) and capsule rows (HBM) arrive interleaved in the same
-// stages, so both streams stay busy for the whole unit.  All matrix products run on mma.sync m16n8k16; the
-// products with value rows are taken transposed (head dimension as M, heads as N) so that a group of up to
-// 8 heads costs one 8-wide tile.  A unit that holds every block of its sequences writes `out` directly;
-// otherwise the units of a (sequence, KV head) leave (max, sum, y) partials and the last one to arrive
-// merges them.
+// shared-memory stages filled by the TMA engine (tiled tensor maps, 128-byte swizzle).  A stage of pass A holds
+// rows [16 JC c, 16 JC (c+1)) of K_tilde of every block of the unit and the same rows of theta[h] (all n
+// columns); a stage of pass C holds the same rows of V_tilde and of U[h]; a text stage holds TCH rows of K_txt
+// and V_txt per sequence.  theta/U rows (L2-resident, shared by all sequences) and capsule rows (HBM) thus
+// arrive interleaved and both streams stay busy for the whole unit.
+//
+// The consumer warps are specialised, and the two groups run one stage apart instead of meeting at a barrier:
+//   value warps      pass A: S_c = sigma q K_c^T (bf16 tile in shared memory)           -> expansion warps
+//                    text:   online-softmax attention over their own 16-row tiles
+//                    pass C: y^T += V_c^T W_c^T                                          <- expansion warps
+//   expansion warps  pass A: L += S_c theta_c, logits in registers (rows x n, fp32), each warp a column range
+//                    softmax: P = 2^(L - max), one maximum per (sequence, head) over the unit's blocks and text
+//                    pass C: W_c = P U_c^T, split over the column ranges and reduced through shared memory
+// All matrix products run on mma.sync m16n8k16; the products with value rows are taken transposed (head
+// dimension as M, heads as N) so that a group of up to 8 heads costs one 8-wide tile.  A unit that holds every
+// block of its sequences writes `out` directly; otherwise the units of a (sequence, KV head) leave
+// (max, sum, y) partials and the last one to arrive merges them.
 #include "kvc_tma.cuh"
 #include "kvc_internal.cuh"
 
@@ -37,7 +38,7 @@ struct FusedArgs {
   __nv_bfloat16* out;
   int B, H_kv, G, R, m, n, T;
   int NB, RB, nbg, nrg, units, JC, NJ, TCH, Tper, ncg, stages;
-  int ktw;            // 16-column groups of L per warp
+  int ktw;            // 16-column groups of L per expansion warp
   int msplit, mshift; // the 8 row tiles of a value block go to msplit = 8 >> mshift tasks
   int sld;            // row stride of the score tile in elements (16 JC + 8)
   uint32_t par_bytes, k_half_bytes, txt_half_bytes, stage_bytes;
@@ -48,37 +49,49 @@ struct FusedArgs {
   int* status;        // device status word
 };
 
-// FWT consumer warps + one producer warp.  Every consumer warp owns up to KTW 16-column groups of the logits;
-// NH = 8-head tiles of the group (1: G <= 8, 2: G <= 16)
-template <int FWT, int KTW, int NH>
-__global__ void __launch_bounds__((FWT + 1) * 32, 1)
+// shared-memory barriers of one CTA
+struct FusedBars {
+  uint64_t full[FMAX_STAGES], empty[FMAX_STAGES];   // ring: data landed / every consumer warp done
+  uint64_t s_ready[2], s_free[2];                   // score tile: written by the value warps / read by the expansion warps
+  uint64_t w_ready[2], w_free[2];                   // weight tile: written by the expansion warps / read by the value warps
+};
+
+// EW expansion warps, VW value warps, one producer warp.  Every expansion warp owns up to KTW 16-column groups of
+// the logits; NH = 8-head tiles of the group (1: G <= 8, 2: G <= 16)
+template <int EW, int VW, int KTW, int NH>
+__global__ void __launch_bounds__((EW + VW + 1) * 32, 1)
 fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                     const __grid_constant__ CUtensorMap tmKt, const __grid_constant__ CUtensorMap tmVt,
                     const __grid_constant__ CUtensorMap tmTh, const __grid_constant__ CUtensorMap tmU,
                     const FusedArgs a) {
-  constexpr int FCONS = FWT * 32;
+  constexpr int CW = EW + VW;                 // consumer warps
+  constexpr int FCONS = CW * 32;
   constexpr int FTHREADS = FCONS + 32;
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* sm = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
-  __shared__ __align__(8) uint64_t full_bar[FMAX_STAGES], empty_bar[FMAX_STAGES];
+  __shared__ __align__(8) FusedBars bars;
   __shared__ int s_last;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
-    for (int s = 0; s < a.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], FWT); }
+    for (int s = 0; s < a.stages; ++s) { mbar_init(&bars.full[s], 1); mbar_init(&bars.empty[s], CW); }
+    for (int x = 0; x < 2; ++x) {
+      mbar_init(&bars.s_ready[x], VW); mbar_init(&bars.s_free[x], EW);
+      mbar_init(&bars.w_ready[x], EW); mbar_init(&bars.w_free[x], VW);
+    }
     fence_mbar_init();
   }
   // score and weight tiles start as zeros: their padding rows and columns are read by the MMAs
   {
     uint32_t* z = reinterpret_cast<uint32_t*>(sm + a.off_S);
-    const int words = (2 * ROWS * a.sld + (ROWS + 16) * SLD) / 2;
+    const int words = (2 * ROWS * a.sld + 2 * (ROWS + 16) * SLD) / 2;
     for (int i = tid; i < words; i += FTHREADS) z[i] = 0u;
   }
   __syncthreads();
 
   const int per_h = a.nbg * a.nrg;
 
-  if (warp == FWT) {
+  if (warp == CW) {
     // ================= producer: one thread feeds the ring =================
     // It walks the stage sequence of this CTA's units: per unit NJ stages of pass A, the text stages, NJ stages
     // of pass C.  A slot is refilled as soon as every consumer warp has released it.
@@ -97,9 +110,9 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       for (int part = 0; part < 3; ++part) {
         const int count = part == 1 ? nts : a.NJ;
         for (int c = 0; c < count; ++c) {
-          if (!mbar_wait_bounded(&empty_bar[slot], phase)) { atomicExch(a.status, (int)KVC_ERR_TIMEOUT); return; }
+          if (!mbar_wait_bounded(&bars.empty[slot], phase)) { atomicExch(a.status, (int)KVC_ERR_TIMEOUT); return; }
           unsigned char* dst = sm + slot * a.stage_bytes;
-          uint64_t* bar = &full_bar[slot];
+          uint64_t* bar = &bars.full[slot];
           if (part == 1) {
             const int y = ts0 + c * a.TCH;
             mbar_expect_tx(bar, 4 * a.txt_half_bytes);
@@ -125,486 +138,569 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     return;
   }
 
-  // ================= consumers =================
+  // ================= consumers: common set-up =================
   const int gid = lane >> 2, t4 = lane & 3;
   const int G = a.G, RB = a.RB, JC = a.JC;
-  const int WPG = FWT / a.NB;                      // warps per sequence of the unit
-  const int bl = warp / WPG, wig = warp - bl * WPG;
   const int rows16 = 16 * JC;                      // rows of one block inside a stage
   const int sld = a.sld;
   const uint32_t sm_u = smem_addr(sm);
   const uint32_t q_u = sm_u + a.off_q, S_u = sm_u + a.off_S, W_u = sm_u + a.off_W;
   __nv_bfloat16* q_sm = reinterpret_cast<__nv_bfloat16*>(sm + a.off_q);
-  __nv_bfloat16* S_sm = reinterpret_cast<__nv_bfloat16*>(sm + a.off_S);
-  __nv_bfloat16* W_sm = reinterpret_cast<__nv_bfloat16*>(sm + a.off_W);
-  float* wred = reinterpret_cast<float*>(sm + a.off_wred);
-  float* rmax = reinterpret_cast<float*>(sm + a.off_rstat);
-  float* rsum = rmax + FWT * ROWS;
-  float* tmax = reinterpret_cast<float*>(sm + a.off_tstat);
-  float* tsum = tmax + FWT * 16;
-  float* hmax = reinterpret_cast<float*>(sm + a.off_hstat);
+  __nv_bfloat16* S_sm = reinterpret_cast<__nv_bfloat16*>(sm + a.off_S);      // [2][ROWS][sld]
+  __nv_bfloat16* W_sm = reinterpret_cast<__nv_bfloat16*>(sm + a.off_W);      // [2][ROWS + 16][SLD]
+  float* wred = reinterpret_cast<float*>(sm + a.off_wred);                   // [2][EW][ROWS][16]
+  float* rmax = reinterpret_cast<float*>(sm + a.off_rstat);                  // [EW][ROWS]
+  float* rsum = rmax + EW * ROWS;
+  float* tmax = reinterpret_cast<float*>(sm + a.off_tstat);                  // [VW][16]
+  float* tsum = tmax + VW * 16;
+  float* hmax = reinterpret_cast<float*>(sm + a.off_hstat);                  // [NB][16]
   float* hsum = hmax + a.NB * 16;
   float* vsum = hsum + a.NB * 16;
-  float* yred = reinterpret_cast<float*>(sm + a.off_yred);
+  float* yred = reinterpret_cast<float*>(sm + a.off_yred);                   // [VW][YHG][D]
   const float qscale = 0.08838834764831845f * 1.4426950408889634f;   // sigma = 1/sqrt(128), logits kept in log2 units
   const int l7 = lane & 7;
   const int lrow = l7 + ((lane >> 3) & 1) * 8;     // ldmatrix address pattern A: rows 0-15 by lanes 0-15, twice
   const int lhi = lane >> 4;
   const int lrowB = l7 + lhi * 8;                  // address pattern B: rows 0-7 | 0-7 | 8-15 | 8-15
   const int lmid = (lane >> 3) & 1;
-
-  // this warp's 16-column groups of the logits, and the byte offsets of its fragments inside a parameter tile
-  const int KT = a.n >> 4;
-  const int kt0 = warp * a.ktw;
-  const int my_kt = max(0, min(a.ktw, KT - kt0));
-  uint32_t th_off[KTW], u_off[KTW];                // theta: [k = row][n = col] read transposed;  U: [n = row][k = col]
-#pragma unroll
-  for (int kt = 0; kt < KTW; ++kt) {
-    const int ktc = kt < my_kt ? kt0 + kt : 0;
-    const int col_t = ktc * 16 + lhi * 8, col_u = ktc * 16 + lmid * 8;
-    th_off[kt] = (uint32_t)(((col_t >> 6) * rows16 + lrow) * 128 + ((((col_t & 63) >> 3) ^ l7) << 4));
-    u_off[kt] = (uint32_t)(((col_u >> 6) * rows16 + lrowB) * 128 + ((((col_u & 63) >> 3) ^ l7) << 4));
-  }
+  const int WPG = VW / a.NB;                       // value warps per sequence of the unit
 
   grid_dep_wait();
   grid_dep_launch();
   if (blockIdx.x == 0 && tid == 0) *a.status = 0;
 
   uint32_t slot = 0, phase = 0;
+  uint32_t si = 0, wi = 0;                         // score tiles and weight tiles handed over so far (buffer = count & 1)
   bool dead = false;
+  auto wait_on = [&](uint64_t* bar, uint32_t parity) { if (!dead && !mbar_wait_bounded(bar, parity)) dead = true; };
   // the stage in `slot` has been consumed by this warp
   auto release = [&]() {
     __syncwarp();
-    if (lane == 0) mbar_arrive(&empty_bar[slot]);
+    if (lane == 0) mbar_arrive(&bars.empty[slot]);
     if (++slot == (uint32_t)a.stages) { slot = 0; phase ^= 1u; }
   };
+  auto signal = [&](uint64_t* bar) { __syncwarp(); if (lane == 0) mbar_arrive(bar); };
 
-  for (int u = blockIdx.x; u < a.units; u += gridDim.x) {
-    const int h = u / per_h, rem = u - h * per_h;
-    const int bg = rem / a.nrg, rg = rem - bg * a.nrg;
-    const int b0 = bg * a.NB, r0 = rg * a.RB;
-    const int nbv = min(a.NB, a.B - b0);
-    const int rbv = min(RB, a.R - r0);
-    const int ts0 = rg * a.Tper;
-    const int ts1 = min(a.T, ts0 + a.Tper);
-    const int nts = ts1 > ts0 ? (ts1 - ts0 + a.TCH - 1) / a.TCH : 0;
-
-    // ---- queries of the unit's sequences: [NB][16 heads][128], heads >= G and absent sequences are zero rows
-    for (int idx = tid; idx < a.NB * 256; idx += FCONS) {
-      const int tb = idx >> 8, g = (idx >> 4) & 15, piece = idx & 15;
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (tb < nbv && g < G)
-        v = *reinterpret_cast<const uint4*>(a.q + ((size_t)(b0 + tb) * a.H_kv * G + (size_t)h * G + g) * D + piece * 8);
-      *reinterpret_cast<uint4*>(q_sm + (tb * 16 + g) * QLD + piece * 8) = v;
-    }
-    named_barrier_sync(1, FCONS);
-    uint32_t qf[NH][8][2];                          // B operand of the score MMA: heads of sequence bl
+  if (warp < EW) {
+    // ======================================================================================================
+    // expansion warps: L += S theta, softmax, W = P U^T
+    // ======================================================================================================
+    const int ETH = EW * 32;
+    const int KT = a.n >> 4;
+    const int kt0 = warp * a.ktw;
+    const int my_kt = max(0, min(a.ktw, KT - kt0));
+    // byte offsets of this warp's fragments inside a parameter tile [column group][row][64]
+    uint32_t th_off[KTW], u_off[KTW];              // theta: [k = row][n = col] read transposed;  U: [n = row][k = col]
 #pragma unroll
-    for (int nh = 0; nh < NH; ++nh)
-#pragma unroll
-      for (int k2 = 0; k2 < 4; ++k2) {
-        uint32_t r[4];
-        ldsm_x4(r, q_u + (uint32_t)(((bl * 16 + nh * 8 + l7) * QLD + k2 * 32 + (lane >> 3) * 8) * 2));
-        qf[nh][2 * k2][0] = r[0]; qf[nh][2 * k2][1] = r[1];
-        qf[nh][2 * k2 + 1][0] = r[2]; qf[nh][2 * k2 + 1][1] = r[3];
-      }
-
-    // expansion rows held by this lane: rho = gid + 8*hr  <->  (sequence, block, head)
-    bool rvalid[2];
-    int rhead[2];
-#pragma unroll
-    for (int hr = 0; hr < 2; ++hr) {
-      const int rho = gid + 8 * hr;
-      const int bi = rho / G, g = rho - bi * G;
-      const int rbl = bi / RB, rrl = bi - rbl * RB;
-      rvalid[hr] = rho < a.NB * RB * G && rbl < nbv && rrl < rbv;
-      rhead[hr] = rvalid[hr] ? rbl * 16 + g : 0;
+    for (int kt = 0; kt < KTW; ++kt) {
+      const int ktc = kt < my_kt ? kt0 + kt : 0;
+      const int col_t = ktc * 16 + lhi * 8, col_u = ktc * 16 + lmid * 8;
+      th_off[kt] = (uint32_t)(((col_t >> 6) * rows16 + lrow) * 128 + ((((col_t & 63) >> 3) ^ l7) << 4));
+      u_off[kt] = (uint32_t)(((col_u >> 6) * rows16 + lrowB) * 128 + ((((col_u & 63) >> 3) ^ l7) << 4));
     }
 
-    float accL[2 * KTW][4];
-#pragma unroll
-    for (int nt = 0; nt < 2 * KTW; ++nt)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) accL[nt][e] = 0.f;
+    for (int u = blockIdx.x; u < a.units; u += gridDim.x) {
+      const int h = u / per_h, rem = u - h * per_h;
+      const int bg = rem / a.nrg, rg = rem - bg * a.nrg;
+      const int b0 = bg * a.NB, r0 = rg * a.RB;
+      const int nbv = min(a.NB, a.B - b0);
+      const int rbv = min(RB, a.R - r0);
+      const int ts0 = rg * a.Tper;
+      const int ts1 = min(a.T, ts0 + a.Tper);
+      const int nts = ts1 > ts0 ? (ts1 - ts0 + a.TCH - 1) / a.TCH : 0;
+      (void)h;
 
-    // =============================== pass A: scores and expansion by theta ===============================
-    int buf = 0;
-    for (int c = 0; c < a.NJ; ++c) {
-      if (!dead && !mbar_wait_bounded(&full_bar[slot], phase)) dead = true;
-      const uint32_t par_u = sm_u + slot * a.stage_bytes, k_u = par_u + a.par_bytes;
-      const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);          // 16-row sub-chunks with rows below m
-      __nv_bfloat16* Sb = S_sm + buf * (ROWS * sld);
-      // S[rows of block][16] = sigma q K^T for my (block, sub-chunk) tasks
-      for (int task = wig; task < RB * nsub; task += WPG) {
-        const int rl = task / nsub, s = task - rl * nsub;
-        const int bi = bl * RB + rl;
-        const uint32_t rowoff = k_u + (uint32_t)((bi * rows16 + s * 16 + lrow) * 128);
-        uint32_t af[8][4];
+      // expansion rows held by this lane: rho = gid + 8*hr  <->  (sequence, block, head)
+      bool rvalid[2];
+      int rhead[2];
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          ldsm_x4(af[ks], rowoff + (ks >> 2) * a.k_half_bytes + (uint32_t)(((((ks & 3) * 2 + lhi)) ^ l7) << 4));
-        float sc[NH][2][4];
-#pragma unroll
-        for (int nh = 0; nh < NH; ++nh)
-#pragma unroll
-          for (int x = 0; x < 2; ++x)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) sc[nh][x][e] = 0.f;
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-#pragma unroll
-          for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(sc[nh][ks & 1], af[ks], qf[nh][ks][0], qf[nh][ks][1]);
-#pragma unroll
-        for (int nh = 0; nh < NH; ++nh)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int head = nh * 8 + 2 * t4 + (e & 1), j = gid + (e >> 1) * 8;
-            if (head < G) Sb[(bi * G + head) * sld + s * 16 + j] = __float2bfloat16_rn((sc[nh][0][e] + sc[nh][1][e]) * qscale);
-          }
+      for (int hr = 0; hr < 2; ++hr) {
+        const int rho = gid + 8 * hr;
+        const int bi = rho / G, g = rho - bi * G;
+        const int rbl = bi / RB, rrl = bi - rbl * RB;
+        rvalid[hr] = rho < a.NB * RB * G && rbl < nbv && rrl < rbv;
+        rhead[hr] = rvalid[hr] ? rbl * 16 + g : 0;
       }
-      named_barrier_sync(1, FCONS);
-      // L[:, my column groups] += S theta
-      for (int s = 0; s < nsub; ++s) {
-        uint32_t as[4];
-        ldsm_x4(as, S_u + (uint32_t)((buf * (ROWS * sld) + lrow * sld + s * 16 + lhi * 8) * 2));
-        uint32_t bf[KTW][4];
-#pragma unroll
-        for (int kt = 0; kt < KTW; ++kt)
-          if (kt < my_kt) ldsm_x4_t(bf[kt], par_u + th_off[kt] + (uint32_t)(s * 2048));
-#pragma unroll
-        for (int kt = 0; kt < KTW; ++kt)
-          if (kt < my_kt) {
-            mma_bf16_16816(accL[2 * kt], as, bf[kt][0], bf[kt][1]);
-            mma_bf16_16816(accL[2 * kt + 1], as, bf[kt][2], bf[kt][3]);
-          }
-      }
-      buf ^= 1;
-      release();
-    }
 
-    // =============================== text rows: online-softmax attention per warp ===============================
-    // yacc[mt][nh]: y^T tile, rows = head-dimension mt*16 + gid (+8), columns = heads nh*8 + 2*t4 (+1) of sequence bl
-    float yacc[8][NH][4];
+      float accL[2 * KTW][4];
 #pragma unroll
-    for (int mt = 0; mt < 8; ++mt)
+      for (int nt = 0; nt < 2 * KTW; ++nt)
 #pragma unroll
-      for (int nh = 0; nh < NH; ++nh)
+        for (int e = 0; e < 4; ++e) accL[nt][e] = 0.f;
+
+      // ---------------- pass A: L[:, my column groups] += S theta ----------------
+      for (int c = 0; c < a.NJ; ++c) {
+        wait_on(&bars.full[slot], phase);
+        const uint32_t par_u = sm_u + slot * a.stage_bytes;
+        const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);          // 16-row sub-chunks with rows below m
+        const uint32_t sbuf = si & 1u;
+        wait_on(&bars.s_ready[sbuf], (si >> 1) & 1u);
+        for (int s = 0; s < nsub; ++s) {
+          uint32_t as[4];
+          ldsm_x4(as, S_u + (uint32_t)((sbuf * (ROWS * sld) + lrow * sld + s * 16 + lhi * 8) * 2));
 #pragma unroll
-        for (int e = 0; e < 4; ++e) yacc[mt][nh][e] = 0.f;
-    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // heads gid and gid + 8
-    for (int ts = 0; ts < nts; ++ts) {
-      if (!dead && !mbar_wait_bounded(&full_bar[slot], phase)) dead = true;
-      const uint32_t kt_u = sm_u + slot * a.stage_bytes, vt_u = kt_u + 2 * a.txt_half_bytes;
-      for (int tile = wig; tile * 16 < a.TCH; tile += WPG) {
-        const int t_first = ts0 + ts * a.TCH + tile * 16;
-        if (t_first >= ts1) break;
-        const int row0 = bl * a.TCH + tile * 16;
-        const uint32_t rowB = (uint32_t)((row0 + lrowB) * 128);
-        // logits [16 heads][16 text rows] = q K_txt^T
-        float cc[2][4];
+          for (int kq = 0; kq < KTW; kq += 4) {                 // fragments of 4 column groups in flight at a time
+            uint32_t bf[4][4];
 #pragma unroll
-        for (int nt = 0; nt < 2; ++nt)
+            for (int x = 0; x < 4; ++x)
+              if (kq + x < KTW && kq + x < my_kt) ldsm_x4_t(bf[x], par_u + th_off[(kq + x < KTW) ? kq + x : 0] + (uint32_t)(s * 2048));
 #pragma unroll
-          for (int e = 0; e < 4; ++e) cc[nt][e] = 0.f;
-        {
-          uint32_t bk[8][4];
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks)
-            ldsm_x4(bk[ks], kt_u + (ks >> 2) * a.txt_half_bytes + rowB + (uint32_t)(((((ks & 3) * 2 + lmid)) ^ l7) << 4));
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            uint32_t aq[4];
-            ldsm_x4(aq, q_u + (uint32_t)(((bl * 16 + lrow) * QLD + ks * 16 + lhi * 8) * 2));
-            mma_bf16_16816(cc[0], aq, bk[ks][0], bk[ks][1]);
-            mma_bf16_16816(cc[1], aq, bk[ks][2], bk[ks][3]);
+            for (int x = 0; x < 4; ++x)
+              if (kq + x < KTW && kq + x < my_kt) {
+                const int kt = (kq + x < KTW) ? kq + x : 0;
+                mma_bf16_16816(accL[2 * kt], as, bf[x][0], bf[x][1]);
+                mma_bf16_16816(accL[2 * kt + 1], as, bf[x][2], bf[x][3]);
+              }
           }
         }
-        // cc[nt][e]: head gid + 8*(e>>1), text row t_first + nt*8 + 2*t4 + (e&1)
+        signal(&bars.s_free[sbuf]);
+        ++si;
+        release();
+      }
+      // ---------------- text stages belong to the value warps ----------------
+      for (int ts = 0; ts < nts; ++ts) {
+        wait_on(&bars.full[slot], phase);
+        release();
+      }
+
+      // ---------------- joint softmax over the unit's blocks and text rows ----------------
 #pragma unroll
-        for (int nt = 0; nt < 2; ++nt)
+      for (int hr = 0; hr < 2; ++hr) {
+        float mx = -INFINITY;
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int t = t_first + nt * 8 + 2 * t4 + (e & 1);
-            cc[nt][e] = t < ts1 ? cc[nt][e] * qscale : -INFINITY;
+        for (int nt = 0; nt < 2 * KTW; ++nt)
+          if (nt < 2 * my_kt) mx = fmaxf(mx, fmaxf(accL[nt][2 * hr], accL[nt][2 * hr + 1]));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        if (t4 == 0) rmax[warp * ROWS + gid + 8 * hr] = rvalid[hr] ? mx : -INFINITY;
+      }
+      named_barrier_sync(1, FCONS);                                   // B1: row maxima and text maxima are in place
+      if (warp == 0) {
+        // maximum of every expansion row over the warps, then of every (sequence, head) over its blocks and text rows
+        if (lane < ROWS) {
+          float mx = -INFINITY;
+#pragma unroll
+          for (int w = 0; w < EW; ++w) mx = fmaxf(mx, rmax[w * ROWS + lane]);
+          rmax[lane] = mx;
+        }
+        __syncwarp();
+        for (int x = lane; x < a.NB * 16; x += 32) {
+          const int tb = x >> 4, g = x & 15;
+          float mx = 0.f;
+          if (g < G && tb < nbv) {
+            mx = -INFINITY;
+            for (int rl = 0; rl < rbv; ++rl) mx = fmaxf(mx, rmax[(tb * RB + rl) * G + g]);
+            for (int w = tb * WPG; w < (tb + 1) * WPG; ++w) mx = fmaxf(mx, tmax[w * 16 + g]);
           }
-        float scl[2];
+          hmax[x] = mx;
+        }
+      }
+      named_barrier_sync(1, FCONS);                                   // B2: head maxima
+      uint32_t pf[KTW][4];                            // P (bf16) of this warp's column groups, as MMA operand fragments
 #pragma unroll
-        for (int hr = 0; hr < 2; ++hr) {
-          float mx = fmaxf(fmaxf(cc[0][2 * hr], cc[0][2 * hr + 1]), fmaxf(cc[1][2 * hr], cc[1][2 * hr + 1]));
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-          const float m_new = fmaxf(m_run[hr], mx);              // finite: the tile has at least one valid row
-          scl[hr] = fast_exp2(m_run[hr] - m_new);                // 0 on the first tile
-          m_run[hr] = m_new;
-          float ps = 0.f;
+      for (int hr = 0; hr < 2; ++hr) {
+        const bool ok = rvalid[hr];
+        const float M = hmax[rhead[hr]];
+        float sum = 0.f;
+#pragma unroll
+        for (int nt = 0; nt < 2 * KTW; ++nt)
+#pragma unroll
+          for (int k = 0; k < 2; ++k) {
+            const float p = (ok && nt < 2 * my_kt) ? fast_exp2(accL[nt][2 * hr + k] - M) : 0.f;
+            accL[nt][2 * hr + k] = p;
+            sum += p;
+          }
+        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+        if (t4 == 0) rsum[warp * ROWS + gid + 8 * hr] = sum;
+      }
+#pragma unroll
+      for (int kt = 0; kt < KTW; ++kt) {
+        pf[kt][0] = pack2_bf16(accL[2 * kt][0], accL[2 * kt][1]);
+        pf[kt][1] = pack2_bf16(accL[2 * kt][2], accL[2 * kt][3]);
+        pf[kt][2] = pack2_bf16(accL[2 * kt + 1][0], accL[2 * kt + 1][1]);
+        pf[kt][3] = pack2_bf16(accL[2 * kt + 1][2], accL[2 * kt + 1][3]);
+      }
+      named_barrier_sync(1, FCONS);                                   // B3: row sums and text sums are in place
+      if (warp == 0) {
+        if (lane < ROWS) {
+          float sm_ = 0.f;
+#pragma unroll
+          for (int w = 0; w < EW; ++w) sm_ += rsum[w * ROWS + lane];
+          rsum[lane] = sm_;
+        }
+        __syncwarp();
+        for (int x = lane; x < a.NB * 16; x += 32) {
+          const int tb = x >> 4, g = x & 15;
+          float vs = 0.f, tsm = 0.f;
+          if (g < G && tb < nbv) {
+            for (int rl = 0; rl < rbv; ++rl) vs += rsum[(tb * RB + rl) * G + g];
+            for (int w = tb * WPG; w < (tb + 1) * WPG; ++w) tsm += tsum[w * 16 + g];
+          }
+          vsum[x] = vs;
+          hsum[x] = vs + tsm;
+        }
+      }
+      named_barrier_sync(1, FCONS);                                   // B4: head sums
+
+      // ---------------- pass C: W = P U^T, reduced over the expansion warps ----------------
+      for (int c = 0; c < a.NJ; ++c) {
+        wait_on(&bars.full[slot], phase);
+        const uint32_t par_u = sm_u + slot * a.stage_bytes;
+        const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);
+        for (int s = 0; s < nsub; ++s) {
+          float wc[2][4];
 #pragma unroll
           for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-            for (int k = 0; k < 2; ++k) {
-              const float p = fast_exp2(cc[nt][2 * hr + k] - m_new);
-              cc[nt][2 * hr + k] = p;
-              ps += p;
-            }
-          l_run[hr] = l_run[hr] * scl[hr] + ps;
+            for (int e = 0; e < 4; ++e) wc[nt][e] = 0.f;
+#pragma unroll
+          for (int kq = 0; kq < KTW; kq += 4) {
+            uint32_t bu[4][4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x)
+              if (kq + x < KTW && kq + x < my_kt) ldsm_x4(bu[x], par_u + u_off[(kq + x < KTW) ? kq + x : 0] + (uint32_t)(s * 2048));
+#pragma unroll
+            for (int x = 0; x < 4; ++x)
+              if (kq + x < KTW && kq + x < my_kt) {
+                const int kt = (kq + x < KTW) ? kq + x : 0;
+                mma_bf16_16816(wc[0], pf[kt], bu[x][0], bu[x][1]);
+                mma_bf16_16816(wc[1], pf[kt], bu[x][2], bu[x][3]);
+              }
+          }
+          const uint32_t wbuf = wi & 1u;
+          float* wr = wred + (wbuf * EW + warp) * (ROWS * 16);
+#pragma unroll
+          for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+            for (int hr = 0; hr < 2; ++hr)
+              *reinterpret_cast<float2*>(&wr[(gid + 8 * hr) * 16 + nt * 8 + 2 * t4]) = make_float2(wc[nt][2 * hr], wc[nt][2 * hr + 1]);
+          named_barrier_sync(2, ETH);
+          wait_on(&bars.w_free[wbuf], ((wi >> 1) & 1u) ^ 1u);        // the value warps are done with this buffer's previous tile
+          for (int idx = tid; idx < ROWS * 16; idx += ETH) {
+            const float* wp = wred + wbuf * EW * (ROWS * 16) + idx;
+            float w = 0.f;
+#pragma unroll
+            for (int x = 0; x < EW; ++x) w += wp[x * ROWS * 16];
+            W_sm[wbuf * ((ROWS + 16) * SLD) + (idx >> 4) * SLD + (idx & 15)] = __float2bfloat16_rn(w);
+          }
+          signal(&bars.w_ready[wbuf]);
+          ++wi;
         }
-        // the accumulator's columns are heads: fetch their factors from the lanes that own those heads as rows
+        release();
+      }
+    }
+  } else {
+    // ======================================================================================================
+    // value warps: scores, text attention, y^T += V^T W^T, output
+    // ======================================================================================================
+    const int VTH = VW * 32;
+    const int vw = warp - EW, vtid = tid - EW * 32;
+    const int bl = vw / WPG, wig = vw - bl * WPG;
+    const int msplit = a.msplit, mshift = a.mshift;           // a task covers the row tiles mt with (mt >> mshift) == its group
+
+    for (int u = blockIdx.x; u < a.units; u += gridDim.x) {
+      const int h = u / per_h, rem = u - h * per_h;
+      const int bg = rem / a.nrg, rg = rem - bg * a.nrg;
+      const int b0 = bg * a.NB, r0 = rg * a.RB;
+      const int nbv = min(a.NB, a.B - b0);
+      const int rbv = min(RB, a.R - r0);
+      const int ts0 = rg * a.Tper;
+      const int ts1 = min(a.T, ts0 + a.Tper);
+      const int nts = ts1 > ts0 ? (ts1 - ts0 + a.TCH - 1) / a.TCH : 0;
+
+      // ---- queries of the unit's sequences: [NB][16 heads][128], heads >= G and absent sequences are zero rows
+      for (int idx = vtid; idx < a.NB * 256; idx += VTH) {
+        const int tb = idx >> 8, g = (idx >> 4) & 15, piece = idx & 15;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (tb < nbv && g < G)
+          v = *reinterpret_cast<const uint4*>(a.q + ((size_t)(b0 + tb) * a.H_kv * G + (size_t)h * G + g) * D + piece * 8);
+        *reinterpret_cast<uint4*>(q_sm + (tb * 16 + g) * QLD + piece * 8) = v;
+      }
+      named_barrier_sync(3, VTH);
+      uint32_t qf[NH][8][2];                          // B operand of the score MMA: heads of sequence bl
+#pragma unroll
+      for (int nh = 0; nh < NH; ++nh)
+#pragma unroll
+        for (int k2 = 0; k2 < 4; ++k2) {
+          uint32_t r[4];
+          ldsm_x4(r, q_u + (uint32_t)(((bl * 16 + nh * 8 + l7) * QLD + k2 * 32 + (lane >> 3) * 8) * 2));
+          qf[nh][2 * k2][0] = r[0]; qf[nh][2 * k2][1] = r[1];
+          qf[nh][2 * k2 + 1][0] = r[2]; qf[nh][2 * k2 + 1][1] = r[3];
+        }
+
+      // ---------------- pass A: S[rows of block][16] = sigma q K^T for my (block, sub-chunk) tasks ----------------
+      for (int c = 0; c < a.NJ; ++c) {
+        wait_on(&bars.full[slot], phase);
+        const uint32_t k_u = sm_u + slot * a.stage_bytes + a.par_bytes;
+        const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);
+        const uint32_t sbuf = si & 1u;
+        wait_on(&bars.s_free[sbuf], ((si >> 1) & 1u) ^ 1u);          // the expansion warps are done with this buffer's previous tile
+        __nv_bfloat16* Sb = S_sm + sbuf * (ROWS * sld);
+        for (int task = wig; task < RB * nsub; task += WPG) {
+          const int rl = task / nsub, s = task - rl * nsub;
+          const int bi = bl * RB + rl;
+          const uint32_t rowoff = k_u + (uint32_t)((bi * rows16 + s * 16 + lrow) * 128);
+          uint32_t af[8][4];
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks)
+            ldsm_x4(af[ks], rowoff + (ks >> 2) * a.k_half_bytes + (uint32_t)(((((ks & 3) * 2 + lhi)) ^ l7) << 4));
+          float sc[NH][2][4];
+#pragma unroll
+          for (int nh = 0; nh < NH; ++nh)
+#pragma unroll
+            for (int x = 0; x < 2; ++x)
+#pragma unroll
+              for (int e = 0; e < 4; ++e) sc[nh][x][e] = 0.f;
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks)
+#pragma unroll
+            for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(sc[nh][ks & 1], af[ks], qf[nh][ks][0], qf[nh][ks][1]);
+#pragma unroll
+          for (int nh = 0; nh < NH; ++nh)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const int head = nh * 8 + 2 * t4 + (e & 1), j = gid + (e >> 1) * 8;
+              if (head < G) Sb[(bi * G + head) * sld + s * 16 + j] = __float2bfloat16_rn((sc[nh][0][e] + sc[nh][1][e]) * qscale);
+            }
+        }
+        signal(&bars.s_ready[sbuf]);
+        ++si;
+        release();
+      }
+
+      // ---------------- text rows: online-softmax attention per warp ----------------
+      // yacc[mt][nh]: y^T tile, rows = head-dimension mt*16 + gid (+8), columns = heads nh*8 + 2*t4 (+1) of sequence bl
+      float yacc[8][NH][4];
+#pragma unroll
+      for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+        for (int nh = 0; nh < NH; ++nh)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) yacc[mt][nh][e] = 0.f;
+      float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // heads gid and gid + 8
+      for (int ts = 0; ts < nts; ++ts) {
+        wait_on(&bars.full[slot], phase);
+        const uint32_t kt_u = sm_u + slot * a.stage_bytes, vt_u = kt_u + 2 * a.txt_half_bytes;
+        for (int tile = wig; tile * 16 < a.TCH; tile += WPG) {
+          const int t_first = ts0 + ts * a.TCH + tile * 16;
+          if (t_first >= ts1) break;
+          const int row0 = bl * a.TCH + tile * 16;
+          const uint32_t rowB = (uint32_t)((row0 + lrowB) * 128);
+          // logits [16 heads][16 text rows] = q K_txt^T
+          float cc[2][4];
+          {
+            float c2[2][2][4];                       // two accumulation chains per tile column
+#pragma unroll
+            for (int x = 0; x < 2; ++x)
+#pragma unroll
+              for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) c2[x][nt][e] = 0.f;
+#pragma unroll
+            for (int kh = 0; kh < 2; ++kh) {
+              uint32_t bk[4][4], aq[4][4];
+#pragma unroll
+              for (int x = 0; x < 4; ++x) {
+                const int ks = kh * 4 + x;
+                ldsm_x4(bk[x], kt_u + kh * a.txt_half_bytes + rowB + (uint32_t)((((x * 2 + lmid)) ^ l7) << 4));
+                ldsm_x4(aq[x], q_u + (uint32_t)(((bl * 16 + lrow) * QLD + ks * 16 + lhi * 8) * 2));
+              }
+#pragma unroll
+              for (int x = 0; x < 4; ++x) {
+                mma_bf16_16816(c2[x & 1][0], aq[x], bk[x][0], bk[x][1]);
+                mma_bf16_16816(c2[x & 1][1], aq[x], bk[x][2], bk[x][3]);
+              }
+            }
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+              for (int e = 0; e < 4; ++e) cc[nt][e] = c2[0][nt][e] + c2[1][nt][e];
+          }
+          // cc[nt][e]: head gid + 8*(e>>1), text row t_first + nt*8 + 2*t4 + (e&1)
+#pragma unroll
+          for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const int t = t_first + nt * 8 + 2 * t4 + (e & 1);
+              cc[nt][e] = t < ts1 ? cc[nt][e] * qscale : -INFINITY;
+            }
+          float scl[2];
+#pragma unroll
+          for (int hr = 0; hr < 2; ++hr) {
+            float mx = fmaxf(fmaxf(cc[0][2 * hr], cc[0][2 * hr + 1]), fmaxf(cc[1][2 * hr], cc[1][2 * hr + 1]));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            const float m_new = fmaxf(m_run[hr], mx);              // finite: the tile has at least one valid row
+            scl[hr] = fast_exp2(m_run[hr] - m_new);                // 0 on the first tile
+            m_run[hr] = m_new;
+            float ps = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+              for (int k = 0; k < 2; ++k) {
+                const float p = fast_exp2(cc[nt][2 * hr + k] - m_new);
+                cc[nt][2 * hr + k] = p;
+                ps += p;
+              }
+            l_run[hr] = l_run[hr] * scl[hr] + ps;
+          }
+          // the accumulator's columns are heads: fetch their factors from the lanes that own those heads as rows
+#pragma unroll
+          for (int nh = 0; nh < NH; ++nh) {
+            const float c0s = __shfl_sync(0xffffffffu, scl[nh], (2 * t4) * 4);
+            const float c1s = __shfl_sync(0xffffffffu, scl[nh], (2 * t4 + 1) * 4);
+            if (c0s != 1.f || c1s != 1.f) {
+#pragma unroll
+              for (int mt = 0; mt < 8; ++mt) {
+                yacc[mt][nh][0] *= c0s; yacc[mt][nh][1] *= c1s;
+                yacc[mt][nh][2] *= c0s; yacc[mt][nh][3] *= c1s;
+              }
+            }
+          }
+          // y^T[128][heads] += V_txt^T[128][16 rows] P^T[16 rows][heads]
+          uint32_t pb[2][2];
+          pb[0][0] = pack2_bf16(cc[0][0], cc[0][1]); pb[0][1] = pack2_bf16(cc[1][0], cc[1][1]);
+          pb[1][0] = pack2_bf16(cc[0][2], cc[0][3]); pb[1][1] = pack2_bf16(cc[1][2], cc[1][3]);
+          uint32_t av[8][4];
+#pragma unroll
+          for (int mt = 0; mt < 8; ++mt)
+            ldsm_x4_t(av[mt], vt_u + (mt >> 2) * a.txt_half_bytes + rowB + (uint32_t)(((((mt & 3) * 2 + lmid)) ^ l7) << 4));
+#pragma unroll
+          for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+            for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(yacc[mt][nh], av[mt], pb[nh][0], pb[nh][1]);
+        }
+        release();
+      }
+
+      // ---------------- joint softmax: the text accumulators move to the unit's reference maximum ----------------
+      if (t4 == 0) { tmax[vw * 16 + gid] = m_run[0]; tmax[vw * 16 + gid + 8] = m_run[1]; }
+      named_barrier_sync(1, FCONS);                                   // B1
+      named_barrier_sync(1, FCONS);                                   // B2: head maxima
+      {
+        float scl[2];
+#pragma unroll
+        for (int hr = 0; hr < 2; ++hr) {
+          const int head = gid + 8 * hr;
+          const float M = hmax[bl * 16 + head];
+          scl[hr] = m_run[hr] == -INFINITY ? 0.f : fast_exp2(m_run[hr] - M);
+          float l = l_run[hr] * scl[hr];
+          l += __shfl_xor_sync(0xffffffffu, l, 1);
+          l += __shfl_xor_sync(0xffffffffu, l, 2);
+          if (t4 == 0) tsum[vw * 16 + head] = l;
+        }
 #pragma unroll
         for (int nh = 0; nh < NH; ++nh) {
           const float c0s = __shfl_sync(0xffffffffu, scl[nh], (2 * t4) * 4);
           const float c1s = __shfl_sync(0xffffffffu, scl[nh], (2 * t4 + 1) * 4);
-          if (c0s != 1.f || c1s != 1.f) {
-#pragma unroll
-            for (int mt = 0; mt < 8; ++mt) {
-              yacc[mt][nh][0] *= c0s; yacc[mt][nh][1] *= c1s;
-              yacc[mt][nh][2] *= c0s; yacc[mt][nh][3] *= c1s;
-            }
-          }
-        }
-        // y^T[128][heads] += V_txt^T[128][16 rows] P^T[16 rows][heads]
-        uint32_t pb[2][2];
-        pb[0][0] = pack2_bf16(cc[0][0], cc[0][1]); pb[0][1] = pack2_bf16(cc[1][0], cc[1][1]);
-        pb[1][0] = pack2_bf16(cc[0][2], cc[0][3]); pb[1][1] = pack2_bf16(cc[1][2], cc[1][3]);
-        uint32_t av[8][4];
-#pragma unroll
-        for (int mt = 0; mt < 8; ++mt)
-          ldsm_x4_t(av[mt], vt_u + (mt >> 2) * a.txt_half_bytes + rowB + (uint32_t)(((((mt & 3) * 2 + lmid)) ^ l7) << 4));
-#pragma unroll
-        for (int mt = 0; mt < 8; ++mt)
-#pragma unroll
-          for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(yacc[mt][nh], av[mt], pb[nh][0], pb[nh][1]);
-      }
-      release();
-    }
-
-    // =============================== joint softmax over the unit's blocks and text rows ===============================
-#pragma unroll
-    for (int hr = 0; hr < 2; ++hr) {
-      float mx = -INFINITY;
-#pragma unroll
-      for (int nt = 0; nt < 2 * KTW; ++nt)
-        if (nt < 2 * my_kt) mx = fmaxf(mx, fmaxf(accL[nt][2 * hr], accL[nt][2 * hr + 1]));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-      if (t4 == 0) rmax[warp * ROWS + gid + 8 * hr] = rvalid[hr] ? mx : -INFINITY;
-    }
-    if (t4 == 0) { tmax[warp * 16 + gid] = m_run[0]; tmax[warp * 16 + gid + 8] = m_run[1]; }
-    named_barrier_sync(1, FCONS);
-    if (warp == 0) {
-      // maximum of every expansion row over the warps, then of every (sequence, head) over its blocks and text rows
-      if (lane < ROWS) {
-        float mx = -INFINITY;
-#pragma unroll
-        for (int w = 0; w < FWT; ++w) mx = fmaxf(mx, rmax[w * ROWS + lane]);
-        rmax[lane] = mx;
-      }
-      __syncwarp();
-      for (int x = lane; x < a.NB * 16; x += 32) {
-        const int tb = x >> 4, g = x & 15;
-        float mx = 0.f;
-        if (g < G && tb < nbv) {
-          mx = -INFINITY;
-          for (int rl = 0; rl < rbv; ++rl) mx = fmaxf(mx, rmax[(tb * RB + rl) * G + g]);
-          for (int w = tb * WPG; w < (tb + 1) * WPG; ++w) mx = fmaxf(mx, tmax[w * 16 + g]);
-        }
-        hmax[x] = mx;
-      }
-    }
-    named_barrier_sync(1, FCONS);
-    uint32_t pf[KTW][4];                            // P (bf16) of this warp's column groups, as MMA operand fragments
-#pragma unroll
-    for (int hr = 0; hr < 2; ++hr) {
-      const bool ok = rvalid[hr];
-      const float M = hmax[rhead[hr]];
-      float sum = 0.f;
-#pragma unroll
-      for (int nt = 0; nt < 2 * KTW; ++nt)
-#pragma unroll
-        for (int k = 0; k < 2; ++k) {
-          const float p = (ok && nt < 2 * my_kt) ? fast_exp2(accL[nt][2 * hr + k] - M) : 0.f;
-          accL[nt][2 * hr + k] = p;
-          sum += p;
-        }
-      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-      if (t4 == 0) rsum[warp * ROWS + gid + 8 * hr] = sum;
-    }
-#pragma unroll
-    for (int kt = 0; kt < KTW; ++kt) {
-      pf[kt][0] = pack2_bf16(accL[2 * kt][0], accL[2 * kt][1]);
-      pf[kt][1] = pack2_bf16(accL[2 * kt][2], accL[2 * kt][3]);
-      pf[kt][2] = pack2_bf16(accL[2 * kt + 1][0], accL[2 * kt + 1][1]);
-      pf[kt][3] = pack2_bf16(accL[2 * kt + 1][2], accL[2 * kt + 1][3]);
-    }
-    // the text accumulators move to the same reference maximum
-    {
-      float scl[2];
-#pragma unroll
-      for (int hr = 0; hr < 2; ++hr) {
-        const int head = gid + 8 * hr;
-        const float M = hmax[bl * 16 + head];
-        scl[hr] = m_run[hr] == -INFINITY ? 0.f : fast_exp2(m_run[hr] - M);
-        float l = l_run[hr] * scl[hr];
-        l += __shfl_xor_sync(0xffffffffu, l, 1);
-        l += __shfl_xor_sync(0xffffffffu, l, 2);
-        if (t4 == 0) tsum[warp * 16 + head] = l;
-      }
-#pragma unroll
-      for (int nh = 0; nh < NH; ++nh) {
-        const float c0s = __shfl_sync(0xffffffffu, scl[nh], (2 * t4) * 4);
-        const float c1s = __shfl_sync(0xffffffffu, scl[nh], (2 * t4 + 1) * 4);
-#pragma unroll
-        for (int mt = 0; mt < 8; ++mt) {
-          yacc[mt][nh][0] *= c0s; yacc[mt][nh][1] *= c1s;
-          yacc[mt][nh][2] *= c0s; yacc[mt][nh][3] *= c1s;
-        }
-      }
-    }
-    named_barrier_sync(1, FCONS);
-    if (warp == 0) {
-      if (lane < ROWS) {
-        float sm_ = 0.f;
-#pragma unroll
-        for (int w = 0; w < FWT; ++w) sm_ += rsum[w * ROWS + lane];
-        rsum[lane] = sm_;
-      }
-      __syncwarp();
-      for (int x = lane; x < a.NB * 16; x += 32) {
-        const int tb = x >> 4, g = x & 15;
-        float vs = 0.f, tsm = 0.f;
-        if (g < G && tb < nbv) {
-          for (int rl = 0; rl < rbv; ++rl) vs += rsum[(tb * RB + rl) * G + g];
-          for (int w = tb * WPG; w < (tb + 1) * WPG; ++w) tsm += tsum[w * 16 + g];
-        }
-        vsum[x] = vs;
-        hsum[x] = vs + tsm;
-      }
-    }
-
-    // =============================== pass C: re-projection by U^T and product with V_tilde ===============================
-    const int msplit = a.msplit, mshift = a.mshift;           // a task covers the row tiles mt with (mt >> mshift) == its group
-    for (int c = 0; c < a.NJ; ++c) {
-      if (!dead && !mbar_wait_bounded(&full_bar[slot], phase)) dead = true;
-      const uint32_t par_u = sm_u + slot * a.stage_bytes, v_u = par_u + a.par_bytes;
-      const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);
-      for (int s = 0; s < nsub; ++s) {
-        // partial W[rows][16] over this warp's columns of P
-        float wc[2][4];
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) wc[nt][e] = 0.f;
-        {
-          uint32_t bu[KTW][4];
-#pragma unroll
-          for (int kt = 0; kt < KTW; ++kt)
-            if (kt < my_kt) ldsm_x4(bu[kt], par_u + u_off[kt] + (uint32_t)(s * 2048));
-#pragma unroll
-          for (int kt = 0; kt < KTW; ++kt)
-            if (kt < my_kt) {
-              mma_bf16_16816(wc[0], pf[kt], bu[kt][0], bu[kt][1]);
-              mma_bf16_16816(wc[1], pf[kt], bu[kt][2], bu[kt][3]);
-            }
-        }
-        float* wr = wred + warp * (ROWS * 16);
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-          for (int hr = 0; hr < 2; ++hr)
-            *reinterpret_cast<float2*>(&wr[(gid + 8 * hr) * 16 + nt * 8 + 2 * t4]) = make_float2(wc[nt][2 * hr], wc[nt][2 * hr + 1]);
-        named_barrier_sync(1, FCONS);
-        if (tid < ROWS * 16) {
-          const float* wp = wred + tid;
-          float w = 0.f;
-#pragma unroll
-          for (int x = 0; x < FWT; ++x) w += wp[x * ROWS * 16];
-          W_sm[(tid >> 4) * SLD + (tid & 15)] = __float2bfloat16_rn(w);
-        }
-        named_barrier_sync(1, FCONS);
-        // y^T[128][heads] += V^T[128][16 rows of block] W^T[16][heads of block], my (block, row-tile group) tasks
-        for (int task = wig; task < RB * msplit; task += WPG) {
-          const int rl = task >> (3 - mshift), mg = task & (msplit - 1);
-          if (rl >= rbv || bl >= nbv) continue;
-          const int bi = bl * RB + rl;
-          uint32_t bw[4];
-          ldsm_x4(bw, W_u + (uint32_t)(((bi * G + lrowB) * SLD + lmid * 8) * 2));
-          const uint32_t rowoff = v_u + (uint32_t)((bi * rows16 + s * 16 + lrowB) * 128);
 #pragma unroll
           for (int mt = 0; mt < 8; ++mt) {
-            if ((mt >> mshift) == mg) {
-              uint32_t av[4];
-              ldsm_x4_t(av, rowoff + (mt >> 2) * a.k_half_bytes + (uint32_t)(((((mt & 3) * 2 + lmid)) ^ l7) << 4));
-#pragma unroll
-              for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(yacc[mt][nh], av, bw[2 * nh], bw[2 * nh + 1]);
-            }
+            yacc[mt][nh][0] *= c0s; yacc[mt][nh][1] *= c1s;
+            yacc[mt][nh][2] *= c0s; yacc[mt][nh][3] *= c1s;
           }
         }
       }
-      release();
-    }
+      named_barrier_sync(1, FCONS);                                   // B3
+      named_barrier_sync(1, FCONS);                                   // B4: head sums
 
-    // =============================== unit end: reduce over warps, mu term, normalise or leave a partial ===============================
-    const int bh = b0 * a.H_kv + h;                    // used when the block axis is split (NB == 1)
-    const size_t pbase = ((size_t)bh * a.nrg + rg) * G;
-    for (int g0 = 0; g0 < G; g0 += YHG) {
-      // every warp parks its tile columns of heads g0 .. g0+YHG-1; then the warps of a sequence are summed
+      // ---------------- pass C: y^T[128][heads] += V^T[128][16 rows of block] W^T[16][heads of block] ----------------
+      for (int c = 0; c < a.NJ; ++c) {
+        wait_on(&bars.full[slot], phase);
+        const uint32_t v_u = sm_u + slot * a.stage_bytes + a.par_bytes;
+        const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);
+        for (int s = 0; s < nsub; ++s) {
+          const uint32_t wbuf = wi & 1u;
+          wait_on(&bars.w_ready[wbuf], (wi >> 1) & 1u);
+          for (int task = wig; task < RB * msplit; task += WPG) {          // my (block, row-tile group) tasks
+            const int rl = task >> (3 - mshift), mg = task & (msplit - 1);
+            if (rl >= rbv || bl >= nbv) continue;
+            const int bi = bl * RB + rl;
+            uint32_t bw[4];
+            ldsm_x4(bw, W_u + (uint32_t)((wbuf * ((ROWS + 16) * SLD) + (bi * G + lrowB) * SLD + lmid * 8) * 2));
+            const uint32_t rowoff = v_u + (uint32_t)((bi * rows16 + s * 16 + lrowB) * 128);
+            uint32_t av[8][4];
 #pragma unroll
-      for (int nh = 0; nh < NH; ++nh)
+            for (int mt = 0; mt < 8; ++mt)
+              if ((mt >> mshift) == mg)
+                ldsm_x4_t(av[mt], rowoff + (mt >> 2) * a.k_half_bytes + (uint32_t)(((((mt & 3) * 2 + lmid)) ^ l7) << 4));
 #pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          const int head = nh * 8 + 2 * t4 + e;
-          if (head >= g0 && head < g0 + YHG && head < G) {
-            float* yp = yred + (warp * YHG + (head - g0)) * D;
+            for (int mt = 0; mt < 8; ++mt)
+              if ((mt >> mshift) == mg) {
 #pragma unroll
-            for (int mt = 0; mt < 8; ++mt) {
-              yp[mt * 16 + gid] = yacc[mt][nh][e];
-              yp[mt * 16 + gid + 8] = yacc[mt][nh][2 + e];
+                for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(yacc[mt][nh], av[mt], bw[2 * nh], bw[2 * nh + 1]);
+              }
+          }
+          signal(&bars.w_free[wbuf]);
+          ++wi;
+        }
+        release();
+      }
+
+      // ---------------- unit end: reduce over the value warps, mu term, normalise or leave a partial ----------------
+      const int bh = b0 * a.H_kv + h;                    // used when the block axis is split (NB == 1)
+      const size_t pbase = ((size_t)bh * a.nrg + rg) * G;
+      for (int g0 = 0; g0 < G; g0 += YHG) {
+        // every warp parks its tile columns of heads g0 .. g0+YHG-1; then the warps of a sequence are summed
+#pragma unroll
+        for (int nh = 0; nh < NH; ++nh)
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int head = nh * 8 + 2 * t4 + e;
+            if (head >= g0 && head < g0 + YHG && head < G) {
+              float* yp = yred + (vw * YHG + (head - g0)) * D;
+#pragma unroll
+              for (int mt = 0; mt < 8; ++mt) {
+                yp[mt * 16 + gid] = yacc[mt][nh][e];
+                yp[mt * 16 + gid + 8] = yacc[mt][nh][2 + e];
+              }
             }
           }
+        named_barrier_sync(3, VTH);
+        const int hg = min(YHG, G - g0);
+        for (int idx = vtid; idx < nbv * hg * D; idx += VTH) {
+          const int col = idx & (D - 1), gg = (idx >> 7) % hg, tb = idx / (D * hg);
+          const int g = g0 + gg;
+          float y = 0.f;
+          for (int w = tb * WPG; w < (tb + 1) * WPG; ++w) y += yred[(w * YHG + gg) * D + col];
+          y = fmaf(vsum[tb * 16 + g], __bfloat162float(a.mu[h * D + col]), y);
+          if (a.nrg == 1)
+            a.out[((size_t)(b0 + tb) * a.H_kv * G + (size_t)h * G + g) * D + col] = __float2bfloat16_rn(y / hsum[tb * 16 + g]);
+          else
+            a.part_y[(pbase + g) * D + col] = y;
         }
-      named_barrier_sync(1, FCONS);
-      const int hg = min(YHG, G - g0);
-      for (int idx = tid; idx < nbv * hg * D; idx += FCONS) {
-        const int col = idx & (D - 1), gg = (idx >> 7) % hg, tb = idx / (D * hg);
-        const int g = g0 + gg;
-        float y = 0.f;
-        for (int w = tb * WPG; w < (tb + 1) * WPG; ++w) y += yred[(w * YHG + gg) * D + col];
-        y = fmaf(vsum[tb * 16 + g], __bfloat162float(a.mu[h * D + col]), y);
-        if (a.nrg == 1)
-          a.out[((size_t)(b0 + tb) * a.H_kv * G + (size_t)h * G + g) * D + col] = __float2bfloat16_rn(y / hsum[tb * 16 + g]);
-        else
-          a.part_y[(pbase + g) * D + col] = y;
+        named_barrier_sync(3, VTH);
       }
-      named_barrier_sync(1, FCONS);
-    }
-    if (a.nrg > 1) {
-      // one sequence, several units along the block axis: the last unit to arrive merges the partials
-      if (tid < G) a.part_ml[pbase + tid] = make_float2(hmax[tid], hsum[tid]);
-      __threadfence();
-      named_barrier_sync(1, FCONS);
-      if (tid == 0) {
-        const int old = atomicAdd(&a.cnt[bh], 1);
-        s_last = old == a.nrg - 1 ? 1 : 0;
-        if (s_last) a.cnt[bh] = 0;                  // every unit of (sequence, head) has arrived: ready for the next call
-      }
-      named_barrier_sync(1, FCONS);
-      if (s_last) {
+      if (a.nrg > 1) {
+        // one sequence, several units along the block axis: the last unit to arrive merges the partials
+        if (vtid < G) a.part_ml[pbase + vtid] = make_float2(hmax[vtid], hsum[vtid]);
         __threadfence();
-        const size_t p0 = (size_t)bh * a.nrg * G;
-        for (int idx = tid; idx < G * D; idx += FCONS) {
-          const int g = idx >> 7, col = idx & (D - 1);
-          float M = -INFINITY;
-          for (int p = 0; p < a.nrg; ++p) M = fmaxf(M, __ldcg(&a.part_ml[p0 + (size_t)p * G + g]).x);
-          float num = 0.f, den = 0.f;
-          for (int p = 0; p < a.nrg; ++p) {
-            const float2 ml = __ldcg(&a.part_ml[p0 + (size_t)p * G + g]);
-            const float w = fast_exp2(ml.x - M);
-            den = fmaf(w, ml.y, den);
-            num = fmaf(w, __ldcg(&a.part_y[(p0 + (size_t)p * G + g) * D + col]), num);
-          }
-          a.out[((size_t)b0 * a.H_kv * G + (size_t)h * G + g) * D + col] = __float2bfloat16_rn(num / den);
+        named_barrier_sync(3, VTH);
+        if (vtid == 0) {
+          const int old = atomicAdd(&a.cnt[bh], 1);
+          s_last = old == a.nrg - 1 ? 1 : 0;
+          if (s_last) a.cnt[bh] = 0;                  // every unit of (sequence, head) has arrived: ready for the next call
         }
+        named_barrier_sync(3, VTH);
+        if (s_last) {
+          __threadfence();
+          const size_t p0 = (size_t)bh * a.nrg * G;
+          for (int idx = vtid; idx < G * D; idx += VTH) {
+            const int g = idx >> 7, col = idx & (D - 1);
+            float M = -INFINITY;
+            for (int p = 0; p < a.nrg; ++p) M = fmaxf(M, __ldcg(&a.part_ml[p0 + (size_t)p * G + g]).x);
+            float num = 0.f, den = 0.f;
+            for (int p = 0; p < a.nrg; ++p) {
+              const float2 ml = __ldcg(&a.part_ml[p0 + (size_t)p * G + g]);
+              const float w = fast_exp2(ml.x - M);
+              den = fmaf(w, ml.y, den);
+              num = fmaf(w, __ldcg(&a.part_y[(p0 + (size_t)p * G + g) * D + col]), num);
+            }
+            a.out[((size_t)b0 * a.H_kv * G + (size_t)h * G + g) * D + col] = __float2bfloat16_rn(num / den);
+          }
+        }
+        named_barrier_sync(3, VTH);
       }
-      named_barrier_sync(1, FCONS);
     }
   }
   if (dead && lane == 0) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
@@ -642,11 +738,12 @@ bool encode_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// consumer warps for a block length n: the 16-column groups of the logits should divide evenly
-static int consumer_warps(int n) {
+// expansion and value warps for a block length n (the 16-column groups of the logits are dealt to the expansion warps)
+static void warp_split(int n, int* ew, int* vw, int* ktw_max) {
   const int KT = n / 16;
-  if (KT % 12 == 0 && KT / 12 <= 3) return 12;   // n = 576 (24 x 24 grids): 3 groups per warp
-  return 8;
+  if (KT <= 16) { *ew = 4; *vw = 8; *ktw_max = 4; }          // n <= 256
+  else if (KT <= 40) { *ew = 5; *vw = 10; *ktw_max = 8; }    // n <= 640 (24 x 24 grids: 576): the value warps carry most of the work
+  else { *ew = 8; *vw = 4; *ktw_max = 8; }                   // n <= 1024
 }
 
 FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
@@ -655,8 +752,9 @@ FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
   if (L->desc.dtype != KVC_BF16 || L->passthrough || R < 1 || B < 1 || n % 64 != 0 || n > 1024 || G > 16) return p;
   if (reinterpret_cast<uintptr_t>(L->desc.theta) & 15 || reinterpret_cast<uintptr_t>(L->desc.U) & 15) return p;
   const int sms = L->num_sms > 0 ? L->num_sms : 148;
-  p.FW = consumer_warps(n);
-  p.ktw = ceil_div(n / 16, p.FW);
+  int ktw_max = 0;
+  warp_split(n, &p.EW, &p.VW, &ktw_max);
+  p.ktw = ceil_div(n / 16, p.EW);
   p.MT = 1;
   const int cap = ROWS;
   p.RB = R < cap / G ? R : cap / G;
@@ -665,7 +763,7 @@ FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
     // whole sequences per unit: more sequences per unit share one pass over theta[h] and U[h]
     double best = 0;
     for (int nb = 1; nb <= 4; nb *= 2) {
-      if (nb > 1 && (nb * R * G > cap || nb > B || p.FW % nb != 0)) break;
+      if (nb > 1 && (nb * R * G > cap || nb > B || p.VW % nb != 0)) break;
       const long long units = (long long)H_kv * ceil_div(B, nb);
       const double cost = (double)ceil_div((int)units, sms) * ((double)nb * R * m * 512.0 + 4.0 * m * n);
       if (nb == 1 || cost < best) { best = cost; p.NB = nb; }
@@ -690,7 +788,7 @@ FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
   p.txt_half_bytes = (uint32_t)p.NB * p.TCH * 128u;
   {
     // the 8 row tiles of a value block go to `msplit` tasks so that the warps of a sequence share the work evenly
-    const int wpg = p.FW / p.NB;
+    const int wpg = p.VW / p.NB;
     int best = 1 << 30;
     for (int sh = 3; sh >= 0; --sh) {            // sh = 3: one task per block
       const int ms = 8 >> sh, cost = ceil_div(p.RB * ms, wpg) * ((1 << sh) + 1);
@@ -701,13 +799,13 @@ FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
   uint32_t off = 0;
   auto take = [&](uint32_t bytes) { uint32_t o = off; off = (off + bytes + 127u) & ~127u; return o; };
   p.off_q = take((uint32_t)p.NB * 16 * QLD * 2);
-  p.off_S = take((uint32_t)(2 * ROWS * p.sld + (ROWS + 16) * SLD) * 2);
+  p.off_S = take((uint32_t)(2 * ROWS * p.sld + 2 * (ROWS + 16) * SLD) * 2);
   p.off_W = p.off_S + (uint32_t)2 * ROWS * p.sld * 2;
-  p.off_wred = take((uint32_t)p.FW * ROWS * 16 * 4);
-  p.off_rstat = take((uint32_t)2 * p.FW * ROWS * 4);
-  p.off_tstat = take((uint32_t)2 * p.FW * 16 * 4);
+  p.off_wred = take((uint32_t)2 * p.EW * ROWS * 16 * 4);
+  p.off_rstat = take((uint32_t)2 * p.EW * ROWS * 4);
+  p.off_tstat = take((uint32_t)2 * p.VW * 16 * 4);
   p.off_hstat = take((uint32_t)3 * p.NB * 16 * 4);
-  p.off_yred = take((uint32_t)p.FW * YHG * D * 4);
+  p.off_yred = take((uint32_t)p.VW * YHG * D * 4);
   p.misc_bytes = off;
   const uint32_t avail = SMEM_LIMIT - 1024u - 2048u - p.misc_bytes;   // alignment slack; static shared memory and its padding
   int stages = (int)(avail / p.stage_bytes);
@@ -719,24 +817,24 @@ FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
   return p;
 }
 
-template <int FWT, int KTW, int NH>
+template <int EW, int VW, int KTW, int NH>
 static cudaError_t launch_inst(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
   static size_t configured = 0;
   if (p.smem_bytes > configured) {
-    cudaError_t e = cudaFuncSetAttribute(fused_decode_kernel<FWT, KTW, NH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(fused_decode_kernel<EW, VW, KTW, NH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)p.smem_bytes);
     if (e != cudaSuccess) return e;
     configured = p.smem_bytes;
   }
-  return launch_dependent(fused_decode_kernel<FWT, KTW, NH>, dim3(p.grid), dim3((FWT + 1) * 32), p.smem_bytes, st, tm[0],
+  return launch_dependent(fused_decode_kernel<EW, VW, KTW, NH>, dim3(p.grid), dim3((EW + VW + 1) * 32), p.smem_bytes, st, tm[0],
                           tm[1], tm[2], tm[3], tm[4], tm[5], fa);
 }
 
 template <int NH>
 static cudaError_t launch_nh(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
-  if (p.FW == 12) return launch_inst<12, 3, NH>(tm, fa, p, st);
-  if (p.ktw <= 2) return launch_inst<8, 2, NH>(tm, fa, p, st);
-  return launch_inst<8, 8, NH>(tm, fa, p, st);
+  if (p.EW == 4) return launch_inst<4, 8, 4, NH>(tm, fa, p, st);
+  if (p.EW == 5) return launch_inst<5, 10, 8, NH>(tm, fa, p, st);
+  return launch_inst<8, 4, 8, NH>(tm, fa, p, st);
 }
 
 cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPlan& p, cudaStream_t st, bool* encoded) {

@@ -85,7 +85,7 @@ struct FusedPlan {
   int JC, NJ;        // 16-row sub-chunks of the m axis per stage; stages per pass over the m axis
   int TCH;           // text rows per stage and sequence
   int ncg;           // n / 64
-  int FW, ktw;       // consumer warps; 16-column groups of the logits per warp
+  int EW, VW, ktw;   // expansion warps, value warps; 16-column groups of the logits per expansion warp
   int msplit, mshift;// the 8 row tiles of a value block go to msplit = 8 >> mshift tasks
   int sld;           // row stride of the score tile
   int stages, grid;
