@@ -148,15 +148,19 @@ int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out) {
   L->passthrough = pass ? 1 : 0;
   L->d_idx = nullptr;
   L->d_cnt = nullptr;
+  L->d_usum = nullptr;
   L->num_sms = 0;
   if (cudaGetDevice(&L->device) != cudaSuccess ||
       cudaDeviceGetAttribute(&L->num_sms, cudaDevAttrMultiProcessorCount, L->device) != cudaSuccess ||
       cudaMalloc(&L->d_idx, idx.size() * sizeof(int32_t)) != cudaSuccess ||
       cudaMemcpy(L->d_idx, idx.data(), idx.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess ||
-      cudaMalloc(&L->d_cnt, KVC_MAX_COUNTERS * sizeof(int)) != cudaSuccess ||
-      cudaMemset(L->d_cnt, 0, KVC_MAX_COUNTERS * sizeof(int)) != cudaSuccess) {
+      cudaMalloc(&L->d_cnt, (KVC_MAX_COUNTERS + 1) * sizeof(int)) != cudaSuccess ||
+      cudaMemset(L->d_cnt, 0, (KVC_MAX_COUNTERS + 1) * sizeof(int)) != cudaSuccess ||
+      (!pass && (cudaMalloc(&L->d_usum, idx.size() * sizeof(float)) != cudaSuccess ||
+                 compute_usum(L, L->d_usum) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess))) {
     if (L->d_idx) cudaFree(L->d_idx);
     if (L->d_cnt) cudaFree(L->d_cnt);
+    if (L->d_usum) cudaFree(L->d_usum);
     delete L;
     cudaGetLastError();
     return KVC_ERR_CUDA;
@@ -169,6 +173,7 @@ int kvc_layer_destroy(kvc_layer* L) {
   if (!L) return KVC_OK;
   if (L->d_idx) cudaFree(L->d_idx);
   if (L->d_cnt) cudaFree(L->d_cnt);
+  if (L->d_usum) cudaFree(L->d_usum);
   delete L;
   return KVC_OK;
 }

@@ -83,6 +83,11 @@ static cudaError_t launch_compress_t(const kvc_layer* L, const void* K_vis, cons
   }
   if (e != cudaSuccess) return e;
   ProfScope prof(KVC_KERNEL_PROJECT_VALUES, st);
+  {
+    bool used = false;
+    e = launch_project_values_mma(L, V_vis, B, R, Vc, st, &used);      // bf16: tensor cores
+    if (used || e != cudaSuccess) return e;
+  }
   dim3 grid((unsigned)(B * H_kv * R), (unsigned)ceil_div(m, 32));
   project_values_kernel<T><<<grid, 256, 0, st>>>(static_cast<const T*>(V_vis), static_cast<T*>(Vc),
                                                  static_cast<const T*>(L->desc.U),

@@ -105,7 +105,9 @@ struct kvc_layer {
   int device;
   int num_sms;
   int32_t* d_idx;        // device [H_kv][m]
-  int* d_cnt;            // device [KVC_MAX_COUNTERS] arrival counters of the one-kernel decode path; zero between calls
+  int* d_cnt;            // device [KVC_MAX_COUNTERS + 1] arrival counters of the one-kernel decode path (zero between
+                         // calls), then the status word of the compress kernels
+  float* d_usum;         // device [H_kv][m] row sums of U (value compression:  U (V - 1 mu^T) = U V - (U 1) mu^T)
 };
 
 namespace kvc {
@@ -183,6 +185,8 @@ cudaError_t launch_expand_mma(const DecodeArgs& a, cudaStream_t st);
 cudaError_t launch_output(const DecodeArgs& a, int dtype, cudaStream_t st);
 // one-kernel path; *encoded == false (and nothing launched) if the tensor maps could not be built
 cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPlan& p, cudaStream_t st, bool* encoded);
+cudaError_t compute_usum(const kvc_layer* L, float* usum);
+cudaError_t launch_project_values_mma(const kvc_layer* L, const void* V_vis, int B, int R, void* Vc, cudaStream_t st, bool* used);
 cudaError_t launch_compress(const kvc_layer* L, const void* K_vis, const void* V_vis, int B, int R,
                             void* Kc, void* Vc, cudaStream_t st);
 
