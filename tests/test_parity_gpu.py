@@ -222,3 +222,97 @@ def test_decode_steps_with_growing_text_tail():
         ps = dict(p); ps["T"] = T
         _, _, want = tl.oracle_run(shape, ps)
         assert np.abs(tl.np64(out) - want).max() <= tl.TOL["bf16"]
+
+
+# ------------------------------------------------------------------ one-kernel bf16 path: edge cases and coverage
+def _fused_launches(fn):
+    """Runs fn with the library's event brackets on and returns {kernel name: launches}."""
+    kvc.kvc_profile_start(64)
+    try:
+        fn()
+        torch.cuda.synchronize()
+    finally:
+        kvc.kvc_profile_stop()
+    out = {k: v[1] for k, v in kvc.kvc_profile_read().items()}
+    kvc.kvc_profile_start(0)
+    kvc.kvc_profile_stop()
+    return out
+
+
+def test_bf16_block_lengths_of_the_configurations_take_the_one_kernel_path():
+    shape = tl.small(wl.CONFIGS[1], B=2, H_q=4, H_kv=4)
+    p = tl.make_problem(shape, 131, T=40, T_cap=48)
+    counts = _fused_launches(lambda: tl.gpu_run(shape, p))
+    assert counts["fused"] == 1 and counts["scores"] == 0 and counts["output"] == 0
+    # a block length that is not a multiple of 64 goes through the three-phase kernels
+    shape2 = wl.Shape("odd-n", 1, 2, 4, 2, 128, 7, 2, 9, 1, "bf16")
+    p2 = tl.make_problem(shape2, 132)
+    counts2 = _fused_launches(lambda: tl.gpu_run(shape2, p2))
+    assert counts2["fused"] == 0 and counts2["scores"] == 1
+
+
+@pytest.mark.parametrize("B,H_q,H_kv,grid,R,T", [
+    (3, 2, 2, 8, 5, 0),        # odd batch with two sequences per unit, no text
+    (3, 2, 2, 8, 5, 1),        # one text row
+    (1, 2, 2, 8, 7, 255),      # text spanning several stages, ragged tail
+    (2, 2, 2, 8, 1, 257),
+    (1, 7, 1, 8, 5, 700),      # G = 7: units split the block axis, text rows split between the units
+    (2, 14, 2, 16, 3, 33),     # n = 256, blocks not a multiple of the blocks per unit
+    (5, 4, 4, 24, 2, 130),     # n = 576: 12 logit column groups per warp range, odd batch
+    (1, 16, 1, 8, 3, 20),      # G = 16: two head tiles, one block per unit
+    (1, 12, 2, 32, 2, 64),     # n = 1024
+])
+def test_one_kernel_path_edges(B, H_q, H_kv, grid, R, T):
+    shape = wl.Shape("fused-edge", 1, B, H_q, H_kv, 128, grid, R, T, 1, "bf16")
+    p = tl.make_problem(shape, 140 + B + 7 * R + T, T=T, T_cap=T + 5)
+    _check(shape, p)
+
+
+def test_more_units_than_sms_and_status_word_clean():
+    """Persistent CTAs walk several work units each (ring parity carried across units)."""
+    shape = wl.Shape("many-units", 1, 40, 8, 8, 128, 8, 2, 37, 1, "bf16")      # 8 * 40 = 320 units of one sequence
+    p = tl.make_problem(shape, 150, T=37, T_cap=40)
+    K_o, V_o, out_o = tl.oracle_run(shape, p)
+    layer = tl.gpu_layer(shape, p)
+    B, R = shape.B, shape.R
+    caps = kvc.alloc_capsules(layer, B, R)
+    kvc.kvc_compress(layer, p["K_vis"].cuda(), p["V_vis"].cuda(), B, R, caps)
+    ws = kvc.alloc_workspace(layer, B, R, 40)
+    out = torch.full((B, shape.H_q, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    kvc.kvc_decode_attend(layer, p["q"].cuda(), caps, B, R, p["K_txt"].cuda(), p["V_txt"].cuda(), 37, 40, out, ws)
+    torch.cuda.synchronize()
+    assert kvc.kvc_read_device_status(layer, B, R, 37, ws) == 0
+    assert np.abs(tl.np64(out) - out_o).max() <= tl.TOL["bf16"]
+
+
+@pytest.mark.parametrize("ci", [1, 2, 3])
+def test_full_size_configuration_sampled_heads(ci):
+    """One layer at the configuration's full size, in the launch configuration the benchmark times; the oracle
+    recomputes a sample of (sequence, KV head) pairs from slices of the same inputs."""
+    shape = wl.CONFIGS[ci]
+    m = orc.retained_len(shape.n, shape.ratio_permille)
+    T = shape.T0 + 7
+    p = wl.decode_inputs(shape, m, wl.layer_seed(ci, 1), "cuda", T=T, T_cap=T + 9)
+    dt = wl.torch_dtype(shape.dtype)
+    layer = kvc.Layer(shape.H_q, shape.H_kv, shape.d, shape.n, shape.ratio_permille, dt, idx=p["idx"], theta=p["theta"],
+                      U=p["U"], mu=p["mu"])
+    B, R, G = shape.B, shape.R, shape.G
+    caps = kvc.alloc_capsules(layer, B, R)
+    kvc.kvc_compress(layer, p["K_vis"], p["V_vis"], B, R, caps)
+    ws = kvc.alloc_workspace(layer, B, R, T + 9)
+    out = torch.full((B, shape.H_q, 128), float("nan"), dtype=dt, device="cuda")
+    kvc.kvc_decode_attend(layer, p["q"], caps, B, R, p["K_txt"], p["V_txt"], T, T + 9, out, ws)
+    torch.cuda.synchronize()
+    assert kvc.kvc_read_device_status(layer, B, R, T, ws) == 0
+    assert torch.isfinite(out.float()).all()
+    rng = np.random.default_rng(7 + ci)
+    pairs = {(0, 0), (B - 1, shape.H_kv - 1)} | {(int(rng.integers(B)), int(rng.integers(shape.H_kv))) for _ in range(4)}
+    for b, h in sorted(pairs):
+        sl = lambda t: tl.np64(t[b:b + 1, h:h + 1])
+        K_t, V_t = orc.compress(sl(p["K_vis"]), sl(p["V_vis"]), p["idx"].numpy(), tl.np64(p["U"][h:h + 1]),
+                                tl.np64(p["mu"][h:h + 1]), shape.n)
+        want = orc.decode_attend_fused(tl.np64(p["q"][b:b + 1, h * G:(h + 1) * G]), K_t, V_t, tl.np64(p["theta"][h:h + 1]),
+                                       tl.np64(p["U"][h:h + 1]), tl.np64(p["mu"][h:h + 1]), sl(p["K_txt"])[:, :, :T],
+                                       sl(p["V_txt"])[:, :, :T])
+        got = tl.np64(out[b:b + 1, h * G:(h + 1) * G])
+        assert np.abs(got - want).max() <= tl.TOL[shape.dtype], (b, h)
