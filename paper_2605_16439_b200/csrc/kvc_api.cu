@@ -70,8 +70,15 @@ WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap) {
   w.off_ypart = take(sizeof(float) * (size_t)B * H_kv * G * w.nsplit * D);
   w.off_ystat = take(sizeof(float2) * (size_t)B * H_kv * G * w.nsplit);
   {
-    const FusedPlan fp = (B > 0 && R > 0) ? plan_fused(L, B, R) : FusedPlan{};
-    const size_t np = (fp.ok && fp.nrg > 1) ? (size_t)B * H_kv * fp.nrg * G : 0;
+    // partial outputs of the one-kernel path: per (sequence, KV head) one per unit along the block axis, or, without
+    // vision blocks, one per slice of the text rows (at most 16, whatever T is)
+    size_t np = 0;
+    if (B > 0 && R > 0) {
+      const FusedPlan fp = plan_fused(L, B, R);
+      if (fp.ok && fp.nrg > 1) np = (size_t)B * H_kv * fp.nrg * G;
+    } else if (B > 0 && T_cap > 0 && plan_fused_text(L, B, T_cap).ok) {
+      np = (size_t)B * H_kv * 16 * G;
+    }
     w.off_fpy = take(sizeof(float) * np * D);
     w.off_fpml = take(sizeof(float2) * np);
   }
@@ -248,8 +255,9 @@ int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B
   a.fpart_ml = reinterpret_cast<float2*>(ws + a.ws.off_fpml);
 
   // bf16 storage with TMA-compatible shapes and pointers: the whole of Algorithm 1 in one kernel
-  if (R > 0) {
-    const FusedPlan fp = plan_fused(L, B, R);
+  {
+    // R == 0 (text rows only, the uncompressed comparator): the same kernel with text stages only
+    const FusedPlan fp = R > 0 ? plan_fused(L, B, R) : plan_fused_text(L, B, T);
     const uintptr_t align = reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(capsules) |
                             reinterpret_cast<uintptr_t>(out) | (T > 0 ? reinterpret_cast<uintptr_t>(K_txt) |
                             reinterpret_cast<uintptr_t>(V_txt) : 0) | reinterpret_cast<uintptr_t>(L->desc.mu);

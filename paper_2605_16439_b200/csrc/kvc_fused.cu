@@ -663,7 +663,7 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           const int g = g0 + gg;
           float y = 0.f;
           for (int w = tb * WPG; w < (tb + 1) * WPG; ++w) y += yred[(w * YHG + gg) * D + col];
-          y = fmaf(vsum[tb * 16 + g], __bfloat162float(a.mu[h * D + col]), y);
+          if (a.R > 0) y = fmaf(vsum[tb * 16 + g], __bfloat162float(a.mu[h * D + col]), y);
           if (a.nrg == 1)
             a.out[((size_t)(b0 + tb) * a.H_kv * G + (size_t)h * G + g) * D + col] = __float2bfloat16_rn(y / hsum[tb * 16 + g]);
           else
@@ -817,6 +817,53 @@ FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
   return p;
 }
 
+// Text-only attention (no vision blocks: the uncompressed comparator and R == 0 calls) through the same kernel:
+// only text stages, the rows of a (sequence, KV head) cut into `nrg` slices whose partials are merged.
+FusedPlan plan_fused_text(const kvc_layer* L, int B, int T) {
+  FusedPlan p{};
+  const int G = L->G, H_kv = L->desc.H_kv;
+  if (L->desc.dtype != KVC_BF16 || B < 1 || T < 1 || G > 16) return p;
+  const int sms = L->num_sms > 0 ? L->num_sms : 148;
+  p.EW = 4; p.VW = 8; p.ktw = 0; p.MT = 1;
+  p.NB = 1; p.RB = 1; p.nbg = B;
+  // slices: enough units for every SM, cut so that the persistent CTAs are evenly loaded, slices of >= 256 rows
+  const long long bh = (long long)B * H_kv;
+  int best_ns = 1;
+  double best_eff = 0;
+  for (int ns = 1; ns <= 16; ++ns) {
+    if (ns > 1 && (T / ns < 256 || bh > KVC_MAX_COUNTERS)) break;
+    const long long units = bh * ns;
+    const long long grid = units < sms ? units : sms;
+    const double eff = (double)units / (double)(((units + grid - 1) / grid) * sms);
+    if (eff > best_eff + 0.02) { best_eff = eff; best_ns = ns; }
+  }
+  p.nrg = best_ns;
+  p.units = (int)(bh * p.nrg);
+  p.ncg = 1; p.JC = 1; p.NJ = 0;
+  p.TCH = 128;
+  p.par_bytes = 0; p.k_half_bytes = 0;
+  p.txt_half_bytes = (uint32_t)p.TCH * 128u;
+  p.stage_bytes = 4 * p.txt_half_bytes;
+  p.msplit = 1; p.mshift = 3;
+  p.sld = 24;
+  uint32_t off = 0;
+  auto take = [&](uint32_t bytes) { uint32_t o = off; off = (off + bytes + 127u) & ~127u; return o; };
+  p.off_q = take((uint32_t)p.NB * 16 * QLD * 2);
+  p.off_S = take((uint32_t)(2 * ROWS * p.sld + 2 * (ROWS + 16) * SLD) * 2);
+  p.off_W = p.off_S + (uint32_t)2 * ROWS * p.sld * 2;
+  p.off_wred = take((uint32_t)2 * p.EW * ROWS * 16 * 4);
+  p.off_rstat = take((uint32_t)2 * p.EW * ROWS * 4);
+  p.off_tstat = take((uint32_t)2 * p.VW * 16 * 4);
+  p.off_hstat = take((uint32_t)3 * p.NB * 16 * 4);
+  p.off_yred = take((uint32_t)p.VW * YHG * D * 4);
+  p.misc_bytes = off;
+  p.stages = 3;
+  p.smem_bytes = (size_t)p.stages * p.stage_bytes + p.misc_bytes + 1024u;
+  p.grid = p.units < sms ? p.units : sms;
+  p.ok = 1;
+  return p;
+}
+
 template <int EW, int VW, int KTW, int NH>
 static cudaError_t launch_inst(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
   static size_t configured = 0;
@@ -841,7 +888,7 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
   const int H_kv = a.H_kv, m = a.m, n = a.n, R = a.R, B = a.B;
   CUtensorMap tm[6];
   *encoded = false;
-  {
+  if (R > 0) {
     const uint64_t dims[5] = {(uint64_t)D, (uint64_t)m, (uint64_t)R, (uint64_t)H_kv, (uint64_t)B};
     const uint64_t str[4] = {256ull, (uint64_t)m * 256, (uint64_t)R * m * 256, (uint64_t)H_kv * R * m * 256};
     const uint32_t box[5] = {64u, (uint32_t)(16 * p.JC), (uint32_t)p.RB, 1u, (uint32_t)p.NB};
@@ -858,7 +905,9 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
     tm[2] = tm[0];
     tm[3] = tm[1];
   }
-  {
+  if (R == 0) {
+    tm[0] = tm[2]; tm[1] = tm[3]; tm[4] = tm[2]; tm[5] = tm[3];          // never used: no vision stages
+  } else {
     // theta, U [H_kv][m][n] viewed as (64 columns, m rows, n/64 column groups, H_kv): a box lands as [group][row][64]
     const uint64_t dims[4] = {64ull, (uint64_t)m, (uint64_t)p.ncg, (uint64_t)H_kv};
     const uint64_t str[3] = {(uint64_t)n * 2, 128ull, (uint64_t)m * n * 2};
@@ -872,7 +921,7 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
   fa.q = static_cast<const __nv_bfloat16*>(a.q);
   fa.mu = static_cast<const __nv_bfloat16*>(a.mu);
   fa.out = static_cast<__nv_bfloat16*>(a.out);
-  fa.B = B; fa.H_kv = H_kv; fa.G = a.G; fa.R = R; fa.m = m; fa.n = n; fa.T = a.T;
+  fa.B = B; fa.H_kv = H_kv; fa.G = a.G; fa.R = R; fa.m = R > 0 ? m : 1; fa.n = R > 0 ? n : 64; fa.T = a.T;
   fa.NB = p.NB; fa.RB = p.RB; fa.nbg = p.nbg; fa.nrg = p.nrg; fa.units = p.units; fa.JC = p.JC; fa.NJ = p.NJ;
   fa.TCH = p.TCH; fa.ncg = p.ncg; fa.stages = p.stages;
   fa.ktw = p.ktw; fa.msplit = p.msplit; fa.mshift = p.mshift; fa.sld = p.sld;

@@ -115,6 +115,7 @@ namespace kvc {
 WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap);
 int cuda_status(cudaError_t e);   // KVC_OK or KVC_ERR_CUDA, remembering the error for kvc_last_cuda_error
 FusedPlan plan_fused(const kvc_layer* L, int B, int R);
+FusedPlan plan_fused_text(const kvc_layer* L, int B, int T);   // R == 0: text rows only
 
 struct DecodeArgs {
   const void* q;
