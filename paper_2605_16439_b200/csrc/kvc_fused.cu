@@ -52,9 +52,13 @@ struct FusedArgs {
 // shared-memory barriers of one CTA
 struct FusedBars {
   uint64_t full[FMAX_STAGES], empty[FMAX_STAGES];   // ring: data landed / every consumer warp done
-  uint64_t s_ready[2], s_free[2];                   // score tile: written by the value warps / read by the expansion warps
-  uint64_t w_ready[2], w_free[2];                   // weight tile: written by the expansion warps / read by the value warps
 };
+// Named barriers (bar.arrive by the writers or readers that move on, bar.sync by the side that has to wait), all
+// counting every consumer thread: 1 all consumers, 2 expansion warps, 3 value warps, then per tile buffer b:
+constexpr int BAR_S_READY = 4;   // + b: score tile written (value warps arrive, expansion warps wait)
+constexpr int BAR_S_FREE = 6;    // + b: score tile read     (expansion warps arrive, value warps wait)
+constexpr int BAR_W_READY = 8;   // + b: weight tile written (expansion warps arrive, value warps wait)
+constexpr int BAR_W_FREE = 10;   // + b: weight tile read    (value warps arrive, expansion warps wait)
 
 // EW expansion warps, VW value warps, one producer warp.  Every expansion warp owns up to KTW 16-column groups of
 // the logits; NH = 8-head tiles of the group (1: G <= 8, 2: G <= 16)
@@ -75,10 +79,6 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     for (int s = 0; s < a.stages; ++s) { mbar_init(&bars.full[s], 1); mbar_init(&bars.empty[s], CW); }
-    for (int x = 0; x < 2; ++x) {
-      mbar_init(&bars.s_ready[x], VW); mbar_init(&bars.s_free[x], EW);
-      mbar_init(&bars.w_ready[x], EW); mbar_init(&bars.w_free[x], VW);
-    }
     fence_mbar_init();
   }
   // score and weight tiles start as zeros: their padding rows and columns are read by the MMAs
@@ -179,7 +179,6 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     if (lane == 0) mbar_arrive(&bars.empty[slot]);
     if (++slot == (uint32_t)a.stages) { slot = 0; phase ^= 1u; }
   };
-  auto signal = [&](uint64_t* bar) { __syncwarp(); if (lane == 0) mbar_arrive(bar); };
 
   if (warp < EW) {
     // ======================================================================================================
@@ -234,7 +233,7 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const uint32_t par_u = sm_u + slot * a.stage_bytes;
         const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);          // 16-row sub-chunks with rows below m
         const uint32_t sbuf = si & 1u;
-        wait_on(&bars.s_ready[sbuf], (si >> 1) & 1u);
+        named_barrier_sync(BAR_S_READY + (int)sbuf, FCONS);
         for (int s = 0; s < nsub; ++s) {
           uint32_t as[4];
           ldsm_x4(as, S_u + (uint32_t)((sbuf * (ROWS * sld) + lrow * sld + s * 16 + lhi * 8) * 2));
@@ -253,7 +252,7 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
               }
           }
         }
-        signal(&bars.s_free[sbuf]);
+        named_barrier_arrive(BAR_S_FREE + (int)sbuf, FCONS);
         ++si;
         release();
       }
@@ -376,7 +375,7 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             for (int hr = 0; hr < 2; ++hr)
               *reinterpret_cast<float2*>(&wr[(gid + 8 * hr) * 16 + nt * 8 + 2 * t4]) = make_float2(wc[nt][2 * hr], wc[nt][2 * hr + 1]);
           named_barrier_sync(2, ETH);
-          wait_on(&bars.w_free[wbuf], ((wi >> 1) & 1u) ^ 1u);        // the value warps are done with this buffer's previous tile
+          if (wi >= 2) named_barrier_sync(BAR_W_FREE + (int)wbuf, FCONS);   // the value warps are done with this buffer's previous tile
           for (int idx = tid; idx < ROWS * 16; idx += ETH) {
             const float* wp = wred + wbuf * EW * (ROWS * 16) + idx;
             float w = 0.f;
@@ -384,7 +383,7 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             for (int x = 0; x < EW; ++x) w += wp[x * ROWS * 16];
             W_sm[wbuf * ((ROWS + 16) * SLD) + (idx >> 4) * SLD + (idx & 15)] = __float2bfloat16_rn(w);
           }
-          signal(&bars.w_ready[wbuf]);
+          named_barrier_arrive(BAR_W_READY + (int)wbuf, FCONS);
           ++wi;
         }
         release();
@@ -435,10 +434,10 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const uint32_t k_u = sm_u + slot * a.stage_bytes + a.par_bytes;
         const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);
         const uint32_t sbuf = si & 1u;
-        wait_on(&bars.s_free[sbuf], ((si >> 1) & 1u) ^ 1u);          // the expansion warps are done with this buffer's previous tile
+        if (si >= 2) named_barrier_sync(BAR_S_FREE + (int)sbuf, FCONS);   // the expansion warps are done with this buffer's previous tile
         __nv_bfloat16* Sb = S_sm + sbuf * (ROWS * sld);
         for (int task = wig; task < RB * nsub; task += WPG) {
-          const int rl = task / nsub, s = task - rl * nsub;
+          const int rl = nsub == 1 ? task : task / nsub, s = task - rl * nsub;
           const int bi = bl * RB + rl;
           const uint32_t rowoff = k_u + (uint32_t)((bi * rows16 + s * 16 + lrow) * 128);
           uint32_t af[8][4];
@@ -464,7 +463,7 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
               if (head < G) Sb[(bi * G + head) * sld + s * 16 + j] = __float2bfloat16_rn((sc[nh][0][e] + sc[nh][1][e]) * qscale);
             }
         }
-        signal(&bars.s_ready[sbuf]);
+        named_barrier_arrive(BAR_S_READY + (int)sbuf, FCONS);
         ++si;
         release();
       }
@@ -611,7 +610,7 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);
         for (int s = 0; s < nsub; ++s) {
           const uint32_t wbuf = wi & 1u;
-          wait_on(&bars.w_ready[wbuf], (wi >> 1) & 1u);
+          named_barrier_sync(BAR_W_READY + (int)wbuf, FCONS);
           for (int task = wig; task < RB * msplit; task += WPG) {          // my (block, row-tile group) tasks
             const int rl = task >> (3 - mshift), mg = task & (msplit - 1);
             if (rl >= rbv || bl >= nbv) continue;
@@ -631,7 +630,7 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(yacc[mt][nh], av[mt], bw[2 * nh], bw[2 * nh + 1]);
               }
           }
-          signal(&bars.w_free[wbuf]);
+          named_barrier_arrive(BAR_W_FREE + (int)wbuf, FCONS);
           ++wi;
         }
         release();
