@@ -35,7 +35,11 @@ NOMINAL_HBM_GBS = 8000.0        # the figure the task's metric quotes its percen
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
 # the ncu capture summarised under profiles/, keyed by (kernel, workload name); None = not captured.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # profiles/fused_decode_config1.md: 185.5 MB read + 5.5 MB written per launch at T = 130 text rows; a text row costs
+    # 2 * B * H_kv * d * 2 bytes = 131072 bytes more, so the mid-run launch (T = 255.5) moves 191.0 MB + 16.5 MB
+    ("fused", "config1-llava-next-7b"): 207.5e6,
+}
 
 
 def parse_args():
