@@ -28,8 +28,7 @@ namespace kvc {
 constexpr int FMAX_STAGES = 8;
 constexpr int QLD = 136;                     // row stride of the query tile in elements (272 B: conflict-free ldmatrix)
 constexpr int SLD = 24;                      // row stride of the 16-column weight tile (48 B)
-constexpr int ROWS = 16;                     // expansion rows per unit (one MMA row tile)
-constexpr int YHG = 2;                       // heads per round of the final cross-warp reduction
+constexpr int ROWS = 16;                     // expansion rows per MMA row tile; a unit holds MT of them
 constexpr uint32_t SMEM_LIMIT = 232448;      // 227 KB per CTA on sm_100
 
 struct FusedArgs {
@@ -41,6 +40,7 @@ struct FusedArgs {
   int ktw;            // 16-column groups of L per expansion warp
   int msplit, mshift; // the 8 row tiles of a value block go to msplit = 8 >> mshift tasks
   int sld;            // row stride of the score tile in elements (16 JC + 8)
+  int yhg;            // heads per round of the final reduction over the value warps
   uint32_t par_bytes, k_half_bytes, txt_half_bytes, stage_bytes;
   uint32_t off_q, off_S, off_W, off_wred, off_rstat, off_tstat, off_hstat, off_yred;
   float* part_y;      // [B*H_kv][nrg][G][D]  partial outputs (only when nrg > 1)
@@ -61,8 +61,8 @@ constexpr int BAR_W_READY = 8;   // + b: weight tile written (expansion warps ar
 constexpr int BAR_W_FREE = 10;   // + b: weight tile read    (value warps arrive, expansion warps wait)
 
 // EW expansion warps, VW value warps, one producer warp.  Every expansion warp owns up to KTW 16-column groups of
-// the logits; NH = 8-head tiles of the group (1: G <= 8, 2: G <= 16)
-template <int EW, int VW, int KTW, int NH>
+// the logits; NH = 8-head tiles of the group (1: G <= 8, 2: G <= 16); MT = 16-row tiles of expansion rows per unit
+template <int EW, int VW, int KTW, int NH, int MT>
 __global__ void __launch_bounds__((EW + VW + 1) * 32, 1)
 fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                     const __grid_constant__ CUtensorMap tmKt, const __grid_constant__ CUtensorMap tmVt,
@@ -71,6 +71,7 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   constexpr int CW = EW + VW;                 // consumer warps
   constexpr int FCONS = CW * 32;
   constexpr int FTHREADS = FCONS + 32;
+  constexpr int RT = ROWS * MT;               // expansion rows of a unit
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* sm = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
   __shared__ __align__(8) FusedBars bars;
@@ -84,7 +85,7 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   // score and weight tiles start as zeros: their padding rows and columns are read by the MMAs
   {
     uint32_t* z = reinterpret_cast<uint32_t*>(sm + a.off_S);
-    const int words = (2 * ROWS * a.sld + 2 * (ROWS + 16) * SLD) / 2;
+    const int words = (2 * RT * a.sld + 2 * (RT + 16) * SLD) / 2;
     for (int i = tid; i < words; i += FTHREADS) z[i] = 0u;
   }
   __syncthreads();
@@ -146,17 +147,17 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const uint32_t sm_u = smem_addr(sm);
   const uint32_t q_u = sm_u + a.off_q, S_u = sm_u + a.off_S, W_u = sm_u + a.off_W;
   __nv_bfloat16* q_sm = reinterpret_cast<__nv_bfloat16*>(sm + a.off_q);
-  __nv_bfloat16* S_sm = reinterpret_cast<__nv_bfloat16*>(sm + a.off_S);      // [2][ROWS][sld]
-  __nv_bfloat16* W_sm = reinterpret_cast<__nv_bfloat16*>(sm + a.off_W);      // [2][ROWS + 16][SLD]
-  float* wred = reinterpret_cast<float*>(sm + a.off_wred);                   // [2][EW][ROWS][16]
-  float* rmax = reinterpret_cast<float*>(sm + a.off_rstat);                  // [EW][ROWS]
-  float* rsum = rmax + EW * ROWS;
+  __nv_bfloat16* S_sm = reinterpret_cast<__nv_bfloat16*>(sm + a.off_S);      // [2][RT][sld]
+  __nv_bfloat16* W_sm = reinterpret_cast<__nv_bfloat16*>(sm + a.off_W);      // [2][RT + 16][SLD]
+  float* wred = reinterpret_cast<float*>(sm + a.off_wred);                   // [2][EW][RT][16]
+  float* rmax = reinterpret_cast<float*>(sm + a.off_rstat);                  // [EW][RT]
+  float* rsum = rmax + EW * RT;
   float* tmax = reinterpret_cast<float*>(sm + a.off_tstat);                  // [VW][16]
   float* tsum = tmax + VW * 16;
   float* hmax = reinterpret_cast<float*>(sm + a.off_hstat);                  // [NB][16]
   float* hsum = hmax + a.NB * 16;
   float* vsum = hsum + a.NB * 16;
-  float* yred = reinterpret_cast<float*>(sm + a.off_yred);                   // [VW][YHG][D]
+  float* yred = reinterpret_cast<float*>(sm + a.off_yred);                   // [VW][yhg][D]
   const float qscale = 0.08838834764831845f * 1.4426950408889634f;   // sigma = 1/sqrt(128), logits kept in log2 units
   const int l7 = lane & 7;
   const int lrow = l7 + ((lane >> 3) & 1) * 8;     // ldmatrix address pattern A: rows 0-15 by lanes 0-15, twice
@@ -209,23 +210,27 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       const int nts = ts1 > ts0 ? (ts1 - ts0 + a.TCH - 1) / a.TCH : 0;
       (void)h;
 
-      // expansion rows held by this lane: rho = gid + 8*hr  <->  (sequence, block, head)
-      bool rvalid[2];
-      int rhead[2];
+      // expansion rows held by this lane: rho = mt*16 + gid + 8*hr  <->  (sequence, block, head)
+      bool rvalid[MT][2];
+      int rhead[MT][2];
 #pragma unroll
-      for (int hr = 0; hr < 2; ++hr) {
-        const int rho = gid + 8 * hr;
-        const int bi = rho / G, g = rho - bi * G;
-        const int rbl = bi / RB, rrl = bi - rbl * RB;
-        rvalid[hr] = rho < a.NB * RB * G && rbl < nbv && rrl < rbv;
-        rhead[hr] = rvalid[hr] ? rbl * 16 + g : 0;
-      }
+      for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int hr = 0; hr < 2; ++hr) {
+          const int rho = mt * 16 + gid + 8 * hr;
+          const int bi = rho / G, g = rho - bi * G;
+          const int rbl = bi / RB, rrl = bi - rbl * RB;
+          rvalid[mt][hr] = rho < a.NB * RB * G && rbl < nbv && rrl < rbv;
+          rhead[mt][hr] = rvalid[mt][hr] ? rbl * 16 + g : 0;
+        }
 
-      float accL[2 * KTW][4];
+      float accL[MT][2 * KTW][4];
 #pragma unroll
-      for (int nt = 0; nt < 2 * KTW; ++nt)
+      for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) accL[nt][e] = 0.f;
+        for (int nt = 0; nt < 2 * KTW; ++nt)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) accL[mt][nt][e] = 0.f;
 
       // ---------------- pass A: L[:, my column groups] += S theta ----------------
       for (int c = 0; c < a.NJ; ++c) {
@@ -235,8 +240,10 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const uint32_t sbuf = si & 1u;
         named_barrier_sync(BAR_S_READY + (int)sbuf, FCONS);
         for (int s = 0; s < nsub; ++s) {
-          uint32_t as[4];
-          ldsm_x4(as, S_u + (uint32_t)((sbuf * (ROWS * sld) + lrow * sld + s * 16 + lhi * 8) * 2));
+          uint32_t as[MT][4];
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt)
+            ldsm_x4(as[mt], S_u + (uint32_t)((sbuf * (RT * sld) + (mt * 16 + lrow) * sld + s * 16 + lhi * 8) * 2));
 #pragma unroll
           for (int kq = 0; kq < KTW; kq += 4) {                 // fragments of 4 column groups in flight at a time
             uint32_t bf[4][4];
@@ -247,8 +254,11 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             for (int x = 0; x < 4; ++x)
               if (kq + x < KTW && kq + x < my_kt) {
                 const int kt = (kq + x < KTW) ? kq + x : 0;
-                mma_bf16_16816(accL[2 * kt], as, bf[x][0], bf[x][1]);
-                mma_bf16_16816(accL[2 * kt + 1], as, bf[x][2], bf[x][3]);
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                  mma_bf16_16816(accL[mt][2 * kt], as[mt], bf[x][0], bf[x][1]);
+                  mma_bf16_16816(accL[mt][2 * kt + 1], as[mt], bf[x][2], bf[x][3]);
+                }
               }
           }
         }
@@ -264,23 +274,25 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 
       // ---------------- joint softmax over the unit's blocks and text rows ----------------
 #pragma unroll
-      for (int hr = 0; hr < 2; ++hr) {
-        float mx = -INFINITY;
+      for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-        for (int nt = 0; nt < 2 * KTW; ++nt)
-          if (nt < 2 * my_kt) mx = fmaxf(mx, fmaxf(accL[nt][2 * hr], accL[nt][2 * hr + 1]));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-        if (t4 == 0) rmax[warp * ROWS + gid + 8 * hr] = rvalid[hr] ? mx : -INFINITY;
-      }
+        for (int hr = 0; hr < 2; ++hr) {
+          float mx = -INFINITY;
+#pragma unroll
+          for (int nt = 0; nt < 2 * KTW; ++nt)
+            if (nt < 2 * my_kt) mx = fmaxf(mx, fmaxf(accL[mt][nt][2 * hr], accL[mt][nt][2 * hr + 1]));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+          if (t4 == 0) rmax[warp * RT + mt * 16 + gid + 8 * hr] = rvalid[mt][hr] ? mx : -INFINITY;
+        }
       named_barrier_sync(1, FCONS);                                   // B1: row maxima and text maxima are in place
       if (warp == 0) {
         // maximum of every expansion row over the warps, then of every (sequence, head) over its blocks and text rows
-        if (lane < ROWS) {
+        for (int x = lane; x < RT; x += 32) {
           float mx = -INFINITY;
 #pragma unroll
-          for (int w = 0; w < EW; ++w) mx = fmaxf(mx, rmax[w * ROWS + lane]);
-          rmax[lane] = mx;
+          for (int w = 0; w < EW; ++w) mx = fmaxf(mx, rmax[w * RT + x]);
+          rmax[x] = mx;
         }
         __syncwarp();
         for (int x = lane; x < a.NB * 16; x += 32) {
@@ -295,38 +307,41 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         }
       }
       named_barrier_sync(1, FCONS);                                   // B2: head maxima
-      uint32_t pf[KTW][4];                            // P (bf16) of this warp's column groups, as MMA operand fragments
+      uint32_t pf[MT][KTW][4];                        // P (bf16) of this warp's column groups, as MMA operand fragments
 #pragma unroll
-      for (int hr = 0; hr < 2; ++hr) {
-        const bool ok = rvalid[hr];
-        const float M = hmax[rhead[hr]];
-        float sum = 0.f;
+      for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
-        for (int nt = 0; nt < 2 * KTW; ++nt)
+        for (int hr = 0; hr < 2; ++hr) {
+          const bool ok = rvalid[mt][hr];
+          const float M = hmax[rhead[mt][hr]];
+          float sum = 0.f;
 #pragma unroll
-          for (int k = 0; k < 2; ++k) {
-            const float p = (ok && nt < 2 * my_kt) ? fast_exp2(accL[nt][2 * hr + k] - M) : 0.f;
-            accL[nt][2 * hr + k] = p;
-            sum += p;
-          }
-        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-        if (t4 == 0) rsum[warp * ROWS + gid + 8 * hr] = sum;
-      }
+          for (int nt = 0; nt < 2 * KTW; ++nt)
 #pragma unroll
-      for (int kt = 0; kt < KTW; ++kt) {
-        pf[kt][0] = pack2_bf16(accL[2 * kt][0], accL[2 * kt][1]);
-        pf[kt][1] = pack2_bf16(accL[2 * kt][2], accL[2 * kt][3]);
-        pf[kt][2] = pack2_bf16(accL[2 * kt + 1][0], accL[2 * kt + 1][1]);
-        pf[kt][3] = pack2_bf16(accL[2 * kt + 1][2], accL[2 * kt + 1][3]);
+            for (int k = 0; k < 2; ++k) {
+              const float p = (ok && nt < 2 * my_kt) ? fast_exp2(accL[mt][nt][2 * hr + k] - M) : 0.f;
+              accL[mt][nt][2 * hr + k] = p;
+              sum += p;
+            }
+          sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+          sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+          if (t4 == 0) rsum[warp * RT + mt * 16 + gid + 8 * hr] = sum;
+        }
+#pragma unroll
+        for (int kt = 0; kt < KTW; ++kt) {
+          pf[mt][kt][0] = pack2_bf16(accL[mt][2 * kt][0], accL[mt][2 * kt][1]);
+          pf[mt][kt][1] = pack2_bf16(accL[mt][2 * kt][2], accL[mt][2 * kt][3]);
+          pf[mt][kt][2] = pack2_bf16(accL[mt][2 * kt + 1][0], accL[mt][2 * kt + 1][1]);
+          pf[mt][kt][3] = pack2_bf16(accL[mt][2 * kt + 1][2], accL[mt][2 * kt + 1][3]);
+        }
       }
       named_barrier_sync(1, FCONS);                                   // B3: row sums and text sums are in place
       if (warp == 0) {
-        if (lane < ROWS) {
+        for (int x = lane; x < RT; x += 32) {
           float sm_ = 0.f;
 #pragma unroll
-          for (int w = 0; w < EW; ++w) sm_ += rsum[w * ROWS + lane];
-          rsum[lane] = sm_;
+          for (int w = 0; w < EW; ++w) sm_ += rsum[w * RT + x];
+          rsum[x] = sm_;
         }
         __syncwarp();
         for (int x = lane; x < a.NB * 16; x += 32) {
@@ -348,11 +363,13 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const uint32_t par_u = sm_u + slot * a.stage_bytes;
         const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);
         for (int s = 0; s < nsub; ++s) {
-          float wc[2][4];
+          float wc[MT][2][4];
 #pragma unroll
-          for (int nt = 0; nt < 2; ++nt)
+          for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-            for (int e = 0; e < 4; ++e) wc[nt][e] = 0.f;
+            for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+              for (int e = 0; e < 4; ++e) wc[mt][nt][e] = 0.f;
 #pragma unroll
           for (int kq = 0; kq < KTW; kq += 4) {
             uint32_t bu[4][4];
@@ -363,25 +380,31 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             for (int x = 0; x < 4; ++x)
               if (kq + x < KTW && kq + x < my_kt) {
                 const int kt = (kq + x < KTW) ? kq + x : 0;
-                mma_bf16_16816(wc[0], pf[kt], bu[x][0], bu[x][1]);
-                mma_bf16_16816(wc[1], pf[kt], bu[x][2], bu[x][3]);
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                  mma_bf16_16816(wc[mt][0], pf[mt][kt], bu[x][0], bu[x][1]);
+                  mma_bf16_16816(wc[mt][1], pf[mt][kt], bu[x][2], bu[x][3]);
+                }
               }
           }
           const uint32_t wbuf = wi & 1u;
-          float* wr = wred + (wbuf * EW + warp) * (ROWS * 16);
+          float* wr = wred + (wbuf * EW + warp) * (RT * 16);
 #pragma unroll
-          for (int nt = 0; nt < 2; ++nt)
+          for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-            for (int hr = 0; hr < 2; ++hr)
-              *reinterpret_cast<float2*>(&wr[(gid + 8 * hr) * 16 + nt * 8 + 2 * t4]) = make_float2(wc[nt][2 * hr], wc[nt][2 * hr + 1]);
+            for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+              for (int hr = 0; hr < 2; ++hr)
+                *reinterpret_cast<float2*>(&wr[(mt * 16 + gid + 8 * hr) * 16 + nt * 8 + 2 * t4]) =
+                    make_float2(wc[mt][nt][2 * hr], wc[mt][nt][2 * hr + 1]);
           named_barrier_sync(2, ETH);
           if (wi >= 2) named_barrier_sync(BAR_W_FREE + (int)wbuf, FCONS);   // the value warps are done with this buffer's previous tile
-          for (int idx = tid; idx < ROWS * 16; idx += ETH) {
-            const float* wp = wred + wbuf * EW * (ROWS * 16) + idx;
+          for (int idx = tid; idx < RT * 16; idx += ETH) {
+            const float* wp = wred + wbuf * EW * (RT * 16) + idx;
             float w = 0.f;
 #pragma unroll
-            for (int x = 0; x < EW; ++x) w += wp[x * ROWS * 16];
-            W_sm[wbuf * ((ROWS + 16) * SLD) + (idx >> 4) * SLD + (idx & 15)] = __float2bfloat16_rn(w);
+            for (int x = 0; x < EW; ++x) w += wp[x * RT * 16];
+            W_sm[wbuf * ((RT + 16) * SLD) + (idx >> 4) * SLD + (idx & 15)] = __float2bfloat16_rn(w);
           }
           named_barrier_arrive(BAR_W_READY + (int)wbuf, FCONS);
           ++wi;
@@ -435,7 +458,7 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);
         const uint32_t sbuf = si & 1u;
         if (si >= 2) named_barrier_sync(BAR_S_FREE + (int)sbuf, FCONS);   // the expansion warps are done with this buffer's previous tile
-        __nv_bfloat16* Sb = S_sm + sbuf * (ROWS * sld);
+        __nv_bfloat16* Sb = S_sm + sbuf * (RT * sld);
         for (int task = wig; task < RB * nsub; task += WPG) {
           const int rl = nsub == 1 ? task : task / nsub, s = task - rl * nsub;
           const int bi = bl * RB + rl;
@@ -616,7 +639,7 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             if (rl >= rbv || bl >= nbv) continue;
             const int bi = bl * RB + rl;
             uint32_t bw[4];
-            ldsm_x4(bw, W_u + (uint32_t)((wbuf * ((ROWS + 16) * SLD) + (bi * G + lrowB) * SLD + lmid * 8) * 2));
+            ldsm_x4(bw, W_u + (uint32_t)((wbuf * ((RT + 16) * SLD) + (bi * G + lrowB) * SLD + lmid * 8) * 2));
             const uint32_t rowoff = v_u + (uint32_t)((bi * rows16 + s * 16 + lrowB) * 128);
             uint32_t av[8][4];
 #pragma unroll
@@ -639,6 +662,7 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       // ---------------- unit end: reduce over the value warps, mu term, normalise or leave a partial ----------------
       const int bh = b0 * a.H_kv + h;                    // used when the block axis is split (NB == 1)
       const size_t pbase = ((size_t)bh * a.nrg + rg) * G;
+      const int YHG = a.yhg;
       for (int g0 = 0; g0 < G; g0 += YHG) {
         // every warp parks its tile columns of heads g0 .. g0+YHG-1; then the warps of a sequence are summed
 #pragma unroll
@@ -684,18 +708,55 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         if (s_last) {
           __threadfence();
           const size_t p0 = (size_t)bh * a.nrg * G;
-          for (int idx = vtid; idx < G * D; idx += VTH) {
-            const int g = idx >> 7, col = idx & (D - 1);
-            float M = -INFINITY;
-            for (int p = 0; p < a.nrg; ++p) M = fmaxf(M, __ldcg(&a.part_ml[p0 + (size_t)p * G + g]).x);
-            float num = 0.f, den = 0.f;
-            for (int p = 0; p < a.nrg; ++p) {
-              const float2 ml = __ldcg(&a.part_ml[p0 + (size_t)p * G + g]);
-              const float w = fast_exp2(ml.x - M);
-              den = fmaf(w, ml.y, den);
-              num = fmaf(w, __ldcg(&a.part_y[(p0 + (size_t)p * G + g) * D + col]), num);
+          // weights of the partials, w[p][g] = 2^(max_p - max) / sum: first all (max, sum) pairs into shared memory
+          float* mlm = yred;                              // [nrg*G] maxima, then [nrg*G] sums, then [nrg*G] weights
+          const int npg = a.nrg * G;
+          const bool in_smem = 3 * npg <= VW * YHG * D;
+          if (in_smem) {
+            for (int idx = vtid; idx < npg; idx += VTH) {
+              const float2 ml = __ldcg(&a.part_ml[p0 + idx]);
+              mlm[idx] = ml.x;
+              mlm[npg + idx] = ml.y;
             }
-            a.out[((size_t)b0 * a.H_kv * G + (size_t)h * G + g) * D + col] = __float2bfloat16_rn(num / den);
+            named_barrier_sync(3, VTH);
+            if (vtid < G) {
+              float M = -INFINITY, den = 0.f;
+              for (int p = 0; p < a.nrg; ++p) M = fmaxf(M, mlm[p * G + vtid]);
+              for (int p = 0; p < a.nrg; ++p) den = fmaf(fast_exp2(mlm[p * G + vtid] - M), mlm[npg + p * G + vtid], den);
+              const float inv = 1.f / den;
+              for (int p = 0; p < a.nrg; ++p) mlm[2 * npg + p * G + vtid] = fast_exp2(mlm[p * G + vtid] - M) * inv;
+            }
+            named_barrier_sync(3, VTH);
+            for (int idx = vtid; idx < G * D; idx += VTH) {
+              const int g = idx >> 7, col = idx & (D - 1);
+              const float* yp = a.part_y + (p0 + g) * D + col;
+              float num = 0.f;
+              int p = 0;
+              for (; p + 4 <= a.nrg; p += 4) {            // four independent loads in flight
+                const float y0 = __ldcg(yp + (size_t)(p + 0) * G * D), y1 = __ldcg(yp + (size_t)(p + 1) * G * D);
+                const float y2 = __ldcg(yp + (size_t)(p + 2) * G * D), y3 = __ldcg(yp + (size_t)(p + 3) * G * D);
+                num = fmaf(mlm[2 * npg + (p + 0) * G + g], y0, num);
+                num = fmaf(mlm[2 * npg + (p + 1) * G + g], y1, num);
+                num = fmaf(mlm[2 * npg + (p + 2) * G + g], y2, num);
+                num = fmaf(mlm[2 * npg + (p + 3) * G + g], y3, num);
+              }
+              for (; p < a.nrg; ++p) num = fmaf(mlm[2 * npg + p * G + g], __ldcg(yp + (size_t)p * G * D), num);
+              a.out[((size_t)b0 * a.H_kv * G + (size_t)h * G + g) * D + col] = __float2bfloat16_rn(num);
+            }
+          } else {
+            for (int idx = vtid; idx < G * D; idx += VTH) {
+              const int g = idx >> 7, col = idx & (D - 1);
+              float M = -INFINITY;
+              for (int p = 0; p < a.nrg; ++p) M = fmaxf(M, __ldcg(&a.part_ml[p0 + (size_t)p * G + g]).x);
+              float num = 0.f, den = 0.f;
+              for (int p = 0; p < a.nrg; ++p) {
+                const float2 ml = __ldcg(&a.part_ml[p0 + (size_t)p * G + g]);
+                const float w = fast_exp2(ml.x - M);
+                den = fmaf(w, ml.y, den);
+                num = fmaf(w, __ldcg(&a.part_y[(p0 + (size_t)p * G + g) * D + col]), num);
+              }
+              a.out[((size_t)b0 * a.H_kv * G + (size_t)h * G + g) * D + col] = __float2bfloat16_rn(num / den);
+            }
           }
         }
         named_barrier_sync(3, VTH);
@@ -754,8 +815,9 @@ FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
   int ktw_max = 0;
   warp_split(n, &p.EW, &p.VW, &ktw_max);
   p.ktw = ceil_div(n / 16, p.EW);
-  p.MT = 1;
-  const int cap = ROWS;
+  // two row tiles per unit when the logits of both still fit the expansion warps' registers (n <= 256)
+  p.MT = (n <= 256 && G * R > ROWS) ? 2 : 1;
+  const int cap = ROWS * p.MT;
   p.RB = R < cap / G ? R : cap / G;
   p.NB = 1;
   if (p.RB == R) {
@@ -798,13 +860,15 @@ FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
   uint32_t off = 0;
   auto take = [&](uint32_t bytes) { uint32_t o = off; off = (off + bytes + 127u) & ~127u; return o; };
   p.off_q = take((uint32_t)p.NB * 16 * QLD * 2);
-  p.off_S = take((uint32_t)(2 * ROWS * p.sld + 2 * (ROWS + 16) * SLD) * 2);
-  p.off_W = p.off_S + (uint32_t)2 * ROWS * p.sld * 2;
-  p.off_wred = take((uint32_t)2 * p.EW * ROWS * 16 * 4);
-  p.off_rstat = take((uint32_t)2 * p.EW * ROWS * 4);
+  const int rt = ROWS * p.MT;
+  p.off_S = take((uint32_t)(2 * rt * p.sld + 2 * (rt + 16) * SLD) * 2);
+  p.off_W = p.off_S + (uint32_t)2 * rt * p.sld * 2;
+  p.off_wred = take((uint32_t)2 * p.EW * rt * 16 * 4);
+  p.off_rstat = take((uint32_t)2 * p.EW * rt * 4);
   p.off_tstat = take((uint32_t)2 * p.VW * 16 * 4);
   p.off_hstat = take((uint32_t)3 * p.NB * 16 * 4);
-  p.off_yred = take((uint32_t)p.VW * YHG * D * 4);
+  p.yhg = G > 4 ? 8 : (G > 2 ? 4 : 2);
+  p.off_yred = take((uint32_t)p.VW * p.yhg * D * 4);
   p.misc_bytes = off;
   const uint32_t avail = SMEM_LIMIT - 1024u - 2048u - p.misc_bytes;   // alignment slack; static shared memory and its padding
   int stages = (int)(avail / p.stage_bytes);
@@ -848,39 +912,43 @@ FusedPlan plan_fused_text(const kvc_layer* L, int B, int T) {
   uint32_t off = 0;
   auto take = [&](uint32_t bytes) { uint32_t o = off; off = (off + bytes + 127u) & ~127u; return o; };
   p.off_q = take((uint32_t)p.NB * 16 * QLD * 2);
-  p.off_S = take((uint32_t)(2 * ROWS * p.sld + 2 * (ROWS + 16) * SLD) * 2);
-  p.off_W = p.off_S + (uint32_t)2 * ROWS * p.sld * 2;
-  p.off_wred = take((uint32_t)2 * p.EW * ROWS * 16 * 4);
-  p.off_rstat = take((uint32_t)2 * p.EW * ROWS * 4);
+  const int rt = ROWS * p.MT;
+  p.off_S = take((uint32_t)(2 * rt * p.sld + 2 * (rt + 16) * SLD) * 2);
+  p.off_W = p.off_S + (uint32_t)2 * rt * p.sld * 2;
+  p.off_wred = take((uint32_t)2 * p.EW * rt * 16 * 4);
+  p.off_rstat = take((uint32_t)2 * p.EW * rt * 4);
   p.off_tstat = take((uint32_t)2 * p.VW * 16 * 4);
   p.off_hstat = take((uint32_t)3 * p.NB * 16 * 4);
-  p.off_yred = take((uint32_t)p.VW * YHG * D * 4);
+  p.yhg = G > 4 ? 8 : (G > 2 ? 4 : 2);
+  p.off_yred = take((uint32_t)p.VW * p.yhg * D * 4);
   p.misc_bytes = off;
-  p.stages = 3;
+  const uint32_t avail = SMEM_LIMIT - 1024u - 2048u - p.misc_bytes;
+  p.stages = (int)(avail / p.stage_bytes) > 3 ? 3 : (int)(avail / p.stage_bytes);
+  if (p.stages < 2) return p;
   p.smem_bytes = (size_t)p.stages * p.stage_bytes + p.misc_bytes + 1024u;
   p.grid = p.units < sms ? p.units : sms;
   p.ok = 1;
   return p;
 }
 
-template <int EW, int VW, int KTW, int NH>
+template <int EW, int VW, int KTW, int NH, int MT>
 static cudaError_t launch_inst(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
   static size_t configured = 0;
   if (p.smem_bytes > configured) {
-    cudaError_t e = cudaFuncSetAttribute(fused_decode_kernel<EW, VW, KTW, NH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(fused_decode_kernel<EW, VW, KTW, NH, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)p.smem_bytes);
     if (e != cudaSuccess) return e;
     configured = p.smem_bytes;
   }
-  return launch_dependent(fused_decode_kernel<EW, VW, KTW, NH>, dim3(p.grid), dim3((EW + VW + 1) * 32), p.smem_bytes, st, tm[0],
+  return launch_dependent(fused_decode_kernel<EW, VW, KTW, NH, MT>, dim3(p.grid), dim3((EW + VW + 1) * 32), p.smem_bytes, st, tm[0],
                           tm[1], tm[2], tm[3], tm[4], tm[5], fa);
 }
 
 template <int NH>
 static cudaError_t launch_nh(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
-  if (p.EW == 4) return launch_inst<4, 8, 4, NH>(tm, fa, p, st);
-  if (p.EW == 5) return launch_inst<5, 10, 8, NH>(tm, fa, p, st);
-  return launch_inst<8, 4, 8, NH>(tm, fa, p, st);
+  if (p.EW == 4) return p.MT == 2 ? launch_inst<4, 8, 4, NH, 2>(tm, fa, p, st) : launch_inst<4, 8, 4, NH, 1>(tm, fa, p, st);
+  if (p.EW == 5) return launch_inst<5, 10, 8, NH, 1>(tm, fa, p, st);
+  return launch_inst<8, 4, 8, NH, 1>(tm, fa, p, st);
 }
 
 cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPlan& p, cudaStream_t st, bool* encoded) {
@@ -923,7 +991,7 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
   fa.B = B; fa.H_kv = H_kv; fa.G = a.G; fa.R = R; fa.m = R > 0 ? m : 1; fa.n = R > 0 ? n : 64; fa.T = a.T;
   fa.NB = p.NB; fa.RB = p.RB; fa.nbg = p.nbg; fa.nrg = p.nrg; fa.units = p.units; fa.JC = p.JC; fa.NJ = p.NJ;
   fa.TCH = p.TCH; fa.ncg = p.ncg; fa.stages = p.stages;
-  fa.ktw = p.ktw; fa.msplit = p.msplit; fa.mshift = p.mshift; fa.sld = p.sld;
+  fa.ktw = p.ktw; fa.msplit = p.msplit; fa.mshift = p.mshift; fa.sld = p.sld; fa.yhg = p.yhg;
   fa.Tper = (ceil_div(a.T > 0 ? a.T : 1, p.nrg) + 15) & ~15;
   fa.par_bytes = p.par_bytes; fa.k_half_bytes = p.k_half_bytes; fa.txt_half_bytes = p.txt_half_bytes;
   fa.stage_bytes = p.stage_bytes;

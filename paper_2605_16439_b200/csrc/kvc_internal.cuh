@@ -88,6 +88,7 @@ struct FusedPlan {
   int EW, VW, ktw;   // expansion warps, value warps; 16-column groups of the logits per expansion warp
   int msplit, mshift;// the 8 row tiles of a value block go to msplit = 8 >> mshift tasks
   int sld;           // row stride of the score tile
+  int yhg;           // heads per round of the final reduction over the value warps
   int stages, grid;
   uint32_t par_bytes, k_half_bytes, txt_half_bytes, stage_bytes, misc_bytes;
   uint32_t off_q, off_S, off_W, off_wred, off_rstat, off_tstat, off_hstat, off_yred;   // relative to the end of the ring
