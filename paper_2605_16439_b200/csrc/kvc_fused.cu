@@ -803,7 +803,7 @@ static void warp_split(int n, int* ew, int* vw, int* ktw_max) {
   const int KT = n / 16;
   if (KT <= 16) { *ew = 4; *vw = 8; *ktw_max = 4; }          // n <= 256
   else if (KT <= 40) { *ew = 5; *vw = 10; *ktw_max = 8; }    // n <= 640 (24 x 24 grids: 576): the value warps carry most of the work
-  else { *ew = 8; *vw = 4; *ktw_max = 8; }                   // n <= 1024
+  else { *ew = 11; *vw = 4; *ktw_max = 6; }                  // n <= 1024: the expansion dominates
 }
 
 FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
@@ -948,7 +948,7 @@ template <int NH>
 static cudaError_t launch_nh(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
   if (p.EW == 4) return p.MT == 2 ? launch_inst<4, 8, 4, NH, 2>(tm, fa, p, st) : launch_inst<4, 8, 4, NH, 1>(tm, fa, p, st);
   if (p.EW == 5) return launch_inst<5, 10, 8, NH, 1>(tm, fa, p, st);
-  return launch_inst<8, 4, 8, NH, 1>(tm, fa, p, st);
+  return launch_inst<11, 4, 6, NH, 1>(tm, fa, p, st);
 }
 
 cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPlan& p, cudaStream_t st, bool* encoded) {
