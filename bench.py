@@ -58,6 +58,8 @@ def parse_args():
     ap.add_argument("--no-comparator", action="store_true")
     ap.add_argument("--no-profile", action="store_true", help="do not bracket kernels with events in the timed region")
     ap.add_argument("--oracle-decode-steps", type=int, default=96)
+    ap.add_argument("--sweep", action="store_true",
+                    help="configuration 4: ratio x batch x vision tokens on the Qwen2-VL shape; prints one JSON line per point")
     return ap.parse_args()
 
 
@@ -335,6 +337,64 @@ def run_reference(a, shape, rank):
     print(json.dumps(line))
 
 
+def run_sweep(a, dev):
+    """Configuration 4 of the task: ratio {0,.2,.4,.6,.8} x batch {1,8,32,64} x vision tokens {2048,8192,32768} on the
+    Qwen2-VL-7B shape (28 query / 4 KV heads, 32x32 grids), bf16, decode steps of the attention path only.  Two layer
+    buffers are rotated (every call still streams more than L2 at the larger points); the uncompressed comparator runs on
+    the same KV length.  One JSON line per point."""
+    from paper_2605_16439_b200 import binding as kvc
+    base = wl.CONFIGS[2]
+    dt = torch.bfloat16
+    steps, nl = 16, 2
+    for nv in (2048, 8192, 32768):
+        for B in (1, 8, 32, 64):
+            for ratio in (0, 200, 400, 600, 800):
+                shape = dataclasses.replace(base, B=B, R=nv // base.n, ratio_permille=ratio, layers=nl, steps=steps)
+                m = kvc.kvc_retained_len(shape.n, ratio)
+                T0, T_cap = shape.T0, shape.T0 + steps
+                layers = []
+                for l in range(nl):
+                    p = wl.decode_inputs(shape, m, 4000 + l, dev, T=T0, T_cap=T_cap)
+                    layer = (kvc.Layer(shape.H_q, shape.H_kv, shape.d, shape.n, 0, dt) if ratio == 0 else
+                             kvc.Layer(shape.H_q, shape.H_kv, shape.d, shape.n, ratio, dt, idx=p["idx"], theta=p["theta"],
+                                       U=p["U"], mu=p["mu"]))
+                    p["layer"] = layer
+                    p["caps"] = kvc.alloc_capsules(layer, B, shape.R, dev)
+                    kvc.kvc_compress(layer, p["K_vis"], p["V_vis"], B, shape.R, p["caps"])
+                    p["out"] = torch.empty((B, shape.H_q, shape.d), dtype=dt, device=dev)
+                    if l > 0 or ratio != 0:
+                        del p["V_vis"]
+                    layers.append(p)
+                ws = kvc.alloc_workspace(layers[0]["layer"], B, shape.R, T_cap, dev)
+
+                def run():
+                    for t in range(steps):
+                        for p in layers:
+                            kvc.kvc_decode_attend(p["layer"], p["q"], p["caps"], B, shape.R, p["K_txt"], p["V_txt"], T0 + t,
+                                                  T_cap, p["out"], ws)
+                run()
+                ms = timed(run, 1, dev) / (steps * nl)
+                contract = contract_bytes_per_layer_call(shape, m, T0 + (steps - 1) / 2.0)
+                # uncompressed comparator over the same sequence length (vision + text rows in one K/V buffer)
+                S = nv + T0 + steps // 2
+                full = kvc.Layer(shape.H_q, shape.H_kv, shape.d, shape.n, 0, dt)
+                Kf = layers[0]["K_vis"].new_empty((B, shape.H_kv, S, shape.d)).normal_()
+                Vf = torch.empty_like(Kf).normal_()
+                wsf = kvc.alloc_workspace(full, B, 0, S, dev)
+                outf = torch.empty((B, shape.H_q, shape.d), dtype=dt, device=dev)
+                fn = lambda: [kvc.kvc_attend_full(full, layers[0]["q"], Kf, Vf, B, S, S, outf, wsf) for _ in range(steps)]
+                fn()
+                ms_full = timed(fn, 1, dev) / steps
+                print(json.dumps({"sweep": "config4-qwen2-vl-7b", "vision_tokens": nv, "batch": B, "ratio": ratio / 1000.0, "m": m,
+                                  "us_per_layer_call": round(ms * 1e3, 2), "tokens_per_s_28_layers": round(B / (ms * 1e-3 * 28), 1),
+                                  "contract_gbs": round(contract / (ms * 1e-3) / 1e9, 1),
+                                  "frac_of_8tbs": round(contract / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS, 4),
+                                  "uncompressed_us_per_layer_call": round(ms_full * 1e3, 2),
+                                  "speedup_vs_uncompressed": round(ms_full / ms, 3)}), flush=True)
+                del layers, ws, Kf, Vf, wsf
+                torch.cuda.empty_cache()
+
+
 def main():
     a = parse_args()
     shape = pick_shape(a)
@@ -356,6 +416,11 @@ def main():
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
     from paper_2605_16439_b200 import binding as kvc
+
+    if a.sweep:
+        if rank == 0:
+            run_sweep(a, dev)
+        return
 
     job = Job(shape, a.config, dev, rank)
     m = job.m

@@ -76,8 +76,10 @@ WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap) {
     if (B > 0 && R > 0) {
       const FusedPlan fp = plan_fused(L, B, R);
       if (fp.ok && fp.nrg > 1) np = (size_t)B * H_kv * fp.nrg * G;
-    } else if (B > 0 && T_cap > 0 && plan_fused_text(L, B, T_cap).ok) {
-      np = (size_t)B * H_kv * 16 * G;
+    }
+    if ((R == 0 || L->passthrough) && B > 0 && R * n + T_cap > 0 && plan_fused_text(L, B, R * n + T_cap).ok) {
+      const size_t np_plain = (size_t)B * H_kv * 16 * G;
+      np = np > np_plain ? np : np_plain;
     }
     w.off_fpy = take(sizeof(float) * np * D);
     w.off_fpml = take(sizeof(float2) * np);
@@ -257,7 +259,9 @@ int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B
   // bf16 storage with TMA-compatible shapes and pointers: the whole of Algorithm 1 in one kernel
   {
     // R == 0 (text rows only, the uncompressed comparator): the same kernel with text stages only
-    const FusedPlan fp = R > 0 ? plan_fused(L, B, R) : plan_fused_text(L, B, T);
+    // rho = 0 stores K and V verbatim: vision rows and text rows are attended as plain rows by the text-only mode
+    const bool plain = R == 0 || L->passthrough;
+    const FusedPlan fp = plain ? plan_fused_text(L, B, R * L->desc.n + T) : plan_fused(L, B, R);
     const uintptr_t align = reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(capsules) |
                             reinterpret_cast<uintptr_t>(out) | (T > 0 ? reinterpret_cast<uintptr_t>(K_txt) |
                             reinterpret_cast<uintptr_t>(V_txt) : 0) | reinterpret_cast<uintptr_t>(L->desc.mu);

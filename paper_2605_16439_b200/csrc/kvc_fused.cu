@@ -36,6 +36,7 @@ struct FusedArgs {
   const __nv_bfloat16* mu;
   __nv_bfloat16* out;
   int B, H_kv, G, R, m, n, T;
+  int S0;             // text-only mode: rows of a leading K/V segment (verbatim vision rows of a rho = 0 store), else 0
   int NB, RB, nbg, nrg, units, JC, NJ, TCH, Tper, ncg, stages;
   int ktw;            // 16-column groups of L per expansion warp
   int msplit, mshift; // the 8 row tiles of a value block go to msplit = 8 >> mshift tasks
@@ -59,6 +60,19 @@ constexpr int BAR_S_READY = 4;   // + b: score tile written (value warps arrive,
 constexpr int BAR_S_FREE = 6;    // + b: score tile read     (expansion warps arrive, value warps wait)
 constexpr int BAR_W_READY = 8;   // + b: weight tile written (expansion warps arrive, value warps wait)
 constexpr int BAR_W_FREE = 10;   // + b: weight tile read    (value warps arrive, expansion warps wait)
+
+// The plain K/V rows a unit attends over: its slice [g0, g1) of the concatenation [leading segment | text rows], as a
+// range of the leading segment (a0, a1; tensor maps tmK / tmV) and a range of the text rows (b0, b1; tmKt / tmVt)
+struct RowRanges { int a0, a1, b0, b1, na, nb; };
+__device__ __forceinline__ RowRanges row_ranges(const FusedArgs& a, int rg) {
+  RowRanges r;
+  const int g0 = rg * a.Tper, g1 = min(a.S0 + a.T, g0 + a.Tper);
+  r.a0 = min(g0, a.S0); r.a1 = min(g1, a.S0);
+  r.b0 = max(g0, a.S0) - a.S0; r.b1 = max(g1, a.S0) - a.S0;
+  r.na = r.a1 > r.a0 ? (r.a1 - r.a0 + a.TCH - 1) / a.TCH : 0;
+  r.nb = r.b1 > r.b0 ? (r.b1 - r.b0 + a.TCH - 1) / a.TCH : 0;
+  return r;
+}
 
 // EW expansion warps, VW value warps, one producer warp.  Every expansion warp owns up to KTW 16-column groups of
 // the logits; NH = 8-head tiles of the group (1: G <= 8, 2: G <= 16); MT = 16-row tiles of expansion rows per unit
@@ -105,9 +119,8 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       const int h = u / per_h, rem = u - h * per_h;
       const int bg = rem / a.nrg, rg = rem - bg * a.nrg;
       const int b0 = bg * a.NB, r0 = rg * a.RB;
-      const int ts0 = rg * a.Tper;
-      const int ts1 = min(a.T, ts0 + a.Tper);
-      const int nts = ts1 > ts0 ? (ts1 - ts0 + a.TCH - 1) / a.TCH : 0;
+      const RowRanges tr = row_ranges(a, rg);
+      const int nts = tr.na + tr.nb;
       for (int part = 0; part < 3; ++part) {
         const int count = part == 1 ? nts : a.NJ;
         for (int c = 0; c < count; ++c) {
@@ -115,13 +128,16 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           unsigned char* dst = sm + slot * a.stage_bytes;
           uint64_t* bar = &bars.full[slot];
           if (part == 1) {
-            const int y = ts0 + c * a.TCH;
+            const bool lead = c < tr.na;
+            const int y = lead ? tr.a0 + c * a.TCH : tr.b0 + (c - tr.na) * a.TCH;
+            const CUtensorMap* mk = lead ? &tmK : &tmKt;
+            const CUtensorMap* mv = lead ? &tmV : &tmVt;
             mbar_expect_tx(bar, 4 * a.txt_half_bytes);
             if (first) { grid_dep_wait(); first = false; }
-            tma_load_4d(dst, &tmKt, 0, y, h, b0, bar);
-            tma_load_4d(dst + a.txt_half_bytes, &tmKt, 64, y, h, b0, bar);
-            tma_load_4d(dst + 2 * a.txt_half_bytes, &tmVt, 0, y, h, b0, bar);
-            tma_load_4d(dst + 3 * a.txt_half_bytes, &tmVt, 64, y, h, b0, bar);
+            tma_load_4d(dst, mk, 0, y, h, b0, bar);
+            tma_load_4d(dst + a.txt_half_bytes, mk, 64, y, h, b0, bar);
+            tma_load_4d(dst + 2 * a.txt_half_bytes, mv, 0, y, h, b0, bar);
+            tma_load_4d(dst + 3 * a.txt_half_bytes, mv, 64, y, h, b0, bar);
           } else {
             const CUtensorMap* tp = part == 0 ? &tmTh : &tmU;
             const CUtensorMap* tk = part == 0 ? &tmK : &tmV;
@@ -205,9 +221,8 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       const int b0 = bg * a.NB, r0 = rg * a.RB;
       const int nbv = min(a.NB, a.B - b0);
       const int rbv = min(RB, a.R - r0);
-      const int ts0 = rg * a.Tper;
-      const int ts1 = min(a.T, ts0 + a.Tper);
-      const int nts = ts1 > ts0 ? (ts1 - ts0 + a.TCH - 1) / a.TCH : 0;
+      const RowRanges tr = row_ranges(a, rg);
+      const int nts = tr.na + tr.nb;
       (void)h;
 
       // expansion rows held by this lane: rho = mt*16 + gid + 8*hr  <->  (sequence, block, head)
@@ -427,9 +442,8 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       const int b0 = bg * a.NB, r0 = rg * a.RB;
       const int nbv = min(a.NB, a.B - b0);
       const int rbv = min(RB, a.R - r0);
-      const int ts0 = rg * a.Tper;
-      const int ts1 = min(a.T, ts0 + a.Tper);
-      const int nts = ts1 > ts0 ? (ts1 - ts0 + a.TCH - 1) / a.TCH : 0;
+      const RowRanges tr = row_ranges(a, rg);
+      const int nts = tr.na + tr.nb;
 
       // ---- queries of the unit's sequences: [NB][16 heads][128], heads >= G and absent sequences are zero rows
       for (int idx = vtid; idx < a.NB * 256; idx += VTH) {
@@ -505,7 +519,8 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         wait_on(&bars.full[slot], phase);
         const uint32_t kt_u = sm_u + slot * a.stage_bytes, vt_u = kt_u + 2 * a.txt_half_bytes;
         for (int tile = wig; tile * 16 < a.TCH; tile += WPG) {
-          const int t_first = ts0 + ts * a.TCH + tile * 16;
+          const int ts1 = ts < tr.na ? tr.a1 : tr.b1;               // end of the row range this stage belongs to
+          const int t_first = (ts < tr.na ? tr.a0 + ts * a.TCH : tr.b0 + (ts - tr.na) * a.TCH) + tile * 16;
           if (t_first >= ts1) break;
           const int row0 = bl * a.TCH + tile * 16;
           const uint32_t rowB = (uint32_t)((row0 + lrowB) * 128);
@@ -882,7 +897,7 @@ FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
 
 // Text-only attention (no vision blocks: the uncompressed comparator and R == 0 calls) through the same kernel:
 // only text stages, the rows of a (sequence, KV head) cut into `nrg` slices whose partials are merged.
-FusedPlan plan_fused_text(const kvc_layer* L, int B, int T) {
+FusedPlan plan_fused_text(const kvc_layer* L, int B, int T) {   // T = all plain rows (leading segment + text)
   FusedPlan p{};
   const int G = L->G, H_kv = L->desc.H_kv;
   if (L->desc.dtype != KVC_BF16 || B < 1 || T < 1 || G > 16) return p;
@@ -955,7 +970,7 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
   const int H_kv = a.H_kv, m = a.m, n = a.n, R = a.R, B = a.B;
   CUtensorMap tm[6];
   *encoded = false;
-  if (R > 0) {
+  if (R > 0 && !a.passthrough) {
     const uint64_t dims[5] = {(uint64_t)D, (uint64_t)m, (uint64_t)R, (uint64_t)H_kv, (uint64_t)B};
     const uint64_t str[4] = {256ull, (uint64_t)m * 256, (uint64_t)R * m * 256, (uint64_t)H_kv * R * m * 256};
     const uint32_t box[5] = {64u, (uint32_t)(16 * p.JC), (uint32_t)p.RB, 1u, (uint32_t)p.NB};
@@ -972,7 +987,16 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
     tm[2] = tm[0];
     tm[3] = tm[1];
   }
-  if (R == 0) {
+  const int S0 = (R > 0 && a.passthrough) ? R * n : 0;   // rho = 0: the store holds K and V verbatim, attended as plain rows
+  if (S0 > 0) {
+    const uint64_t dims[4] = {(uint64_t)D, (uint64_t)S0, (uint64_t)H_kv, (uint64_t)B};
+    const uint64_t str[3] = {256ull, (uint64_t)S0 * 256, (uint64_t)H_kv * S0 * 256};
+    const uint32_t box[4] = {64u, (uint32_t)p.TCH, 1u, (uint32_t)p.NB};
+    if (!encode_tensor_map_bf16(&tm[0], a.Kc, 4, dims, str, box)) return cudaSuccess;
+    if (!encode_tensor_map_bf16(&tm[1], a.Vc, 4, dims, str, box)) return cudaSuccess;
+    if (a.T == 0) { tm[2] = tm[0]; tm[3] = tm[1]; }
+    tm[4] = tm[0]; tm[5] = tm[1];
+  } else if (R == 0) {
     tm[0] = tm[2]; tm[1] = tm[3]; tm[4] = tm[2]; tm[5] = tm[3];          // never used: no vision stages
   } else {
     // theta, U [H_kv][m][n] viewed as (64 columns, m rows, n/64 column groups, H_kv): a box lands as [group][row][64]
@@ -988,11 +1012,13 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
   fa.q = static_cast<const __nv_bfloat16*>(a.q);
   fa.mu = static_cast<const __nv_bfloat16*>(a.mu);
   fa.out = static_cast<__nv_bfloat16*>(a.out);
-  fa.B = B; fa.H_kv = H_kv; fa.G = a.G; fa.R = R; fa.m = R > 0 ? m : 1; fa.n = R > 0 ? n : 64; fa.T = a.T;
+  const bool plain = R == 0 || a.passthrough;            // text-only mode
+  fa.B = B; fa.H_kv = H_kv; fa.G = a.G; fa.R = plain ? 0 : R; fa.m = plain ? 1 : m; fa.n = plain ? 64 : n; fa.T = a.T;
+  fa.S0 = S0;
   fa.NB = p.NB; fa.RB = p.RB; fa.nbg = p.nbg; fa.nrg = p.nrg; fa.units = p.units; fa.JC = p.JC; fa.NJ = p.NJ;
   fa.TCH = p.TCH; fa.ncg = p.ncg; fa.stages = p.stages;
   fa.ktw = p.ktw; fa.msplit = p.msplit; fa.mshift = p.mshift; fa.sld = p.sld; fa.yhg = p.yhg;
-  fa.Tper = (ceil_div(a.T > 0 ? a.T : 1, p.nrg) + 15) & ~15;
+  fa.Tper = (ceil_div(S0 + a.T > 0 ? S0 + a.T : 1, p.nrg) + 15) & ~15;
   fa.par_bytes = p.par_bytes; fa.k_half_bytes = p.k_half_bytes; fa.txt_half_bytes = p.txt_half_bytes;
   fa.stage_bytes = p.stage_bytes;
   const uint32_t ring = (uint32_t)p.stages * p.stage_bytes;

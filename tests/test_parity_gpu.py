@@ -316,3 +316,13 @@ def test_full_size_configuration_sampled_heads(ci):
                                        sl(p["V_txt"])[:, :, :T])
         got = tl.np64(out[b:b + 1, h * G:(h + 1) * G])
         assert np.abs(got - want).max() <= tl.TOL[shape.dtype], (b, h)
+
+
+@pytest.mark.parametrize("B,H_q,H_kv,grid,R,T", [(1, 4, 1, 16, 3, 300), (2, 2, 2, 8, 5, 0), (3, 14, 2, 32, 2, 77)])
+def test_pass_through_store_is_attended_as_plain_rows(B, H_q, H_kv, grid, R, T):
+    """rho = 0 with bf16 storage: the verbatim vision rows and the text rows form one row sequence that is cut into
+    slices (a slice may straddle the two buffers) and merged."""
+    shape = wl.Shape("rho0", 1, B, H_q, H_kv, 128, grid, R, T, 1, "bf16", ratio_permille=0)
+    p = tl.make_problem(shape, 160 + B + R + T, T=T, T_cap=T + 3)
+    counts = _fused_launches(lambda: _check(shape, p))
+    assert counts["fused"] == 1 and counts["scores"] == 0
