@@ -199,7 +199,7 @@ def capsule_views(layer: Layer, capsules, B: int, R: int):
     return (capsules[:half].view(layer.dtype).view(shape), capsules[half:2 * half].view(layer.dtype).view(shape))
 
 
-KVC_KERNEL_COUNT = 8
+KVC_KERNEL_COUNT = 9
 
 
 def kvc_profile_start(max_launches: int) -> None:

@@ -1,5 +1,7 @@
 // Host side of the C ABI: validation, layer handles, workspace layout, kernel sequencing.
 #include <new>
+#include <cstdlib>
+#include <cstring>
 #include <vector>
 
 #include "kvc_internal.cuh"
@@ -159,6 +161,10 @@ int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out) {
   L->d_cnt = nullptr;
   L->d_usum = nullptr;
   L->num_sms = 0;
+  {
+    const char* ex = std::getenv("KVC_EXPANSION");
+    L->use_tc = ex && std::strcmp(ex, "tcgen05") == 0;
+  }
   if (cudaGetDevice(&L->device) != cudaSuccess ||
       cudaDeviceGetAttribute(&L->num_sms, cudaDevAttrMultiProcessorCount, L->device) != cudaSuccess ||
       cudaMalloc(&L->d_idx, idx.size() * sizeof(int32_t)) != cudaSuccess ||

@@ -8,7 +8,7 @@
 
 namespace kvc {
 
-constexpr uint32_t WAIT_SPIN_LIMIT = 1u << 24;   // polls; each try_wait already blocks for a HW-defined slice
+constexpr uint32_t WAIT_SPIN_LIMIT = 1u << 21;   // polls (tens of milliseconds at least; a legitimate wait is far below a millisecond)
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 

@@ -20,59 +20,9 @@
 // dimension as M, heads as N) so that a group of up to 8 heads costs one 8-wide tile.  A unit that holds every
 // block of its sequences writes `out` directly; otherwise the units of a (sequence, KV head) leave
 // (max, sum, y) partials and the last one to arrive merges them.
-#include "kvc_tma.cuh"
-#include "kvc_internal.cuh"
+#include "kvc_fused.cuh"
 
 namespace kvc {
-
-constexpr int FMAX_STAGES = 8;
-constexpr int QLD = 136;                     // row stride of the query tile in elements (272 B: conflict-free ldmatrix)
-constexpr int SLD = 24;                      // row stride of the 16-column weight tile (48 B)
-constexpr int ROWS = 16;                     // expansion rows per MMA row tile; a unit holds MT of them
-constexpr uint32_t SMEM_LIMIT = 232448;      // 227 KB per CTA on sm_100
-
-struct FusedArgs {
-  const __nv_bfloat16* q;
-  const __nv_bfloat16* mu;
-  __nv_bfloat16* out;
-  int B, H_kv, G, R, m, n, T;
-  int S0;             // text-only mode: rows of a leading K/V segment (verbatim vision rows of a rho = 0 store), else 0
-  int NB, RB, nbg, nrg, units, JC, NJ, TCH, Tper, ncg, stages;
-  int ktw;            // 16-column groups of L per expansion warp
-  int msplit, mshift; // the 8 row tiles of a value block go to msplit = 8 >> mshift tasks
-  int sld;            // row stride of the score tile in elements (16 JC + 8)
-  int yhg;            // heads per round of the final reduction over the value warps
-  uint32_t par_bytes, k_half_bytes, txt_half_bytes, stage_bytes;
-  uint32_t off_q, off_S, off_W, off_wred, off_rstat, off_tstat, off_hstat, off_yred;
-  float* part_y;      // [B*H_kv][nrg][G][D]  partial outputs (only when nrg > 1)
-  float2* part_ml;    // [B*H_kv][nrg][G]     (max in log2 units, sum)
-  int* cnt;           // [B*H_kv] arrival counters, zero between calls
-  int* status;        // device status word
-};
-
-// shared-memory barriers of one CTA
-struct FusedBars {
-  uint64_t full[FMAX_STAGES], empty[FMAX_STAGES];   // ring: data landed / every consumer warp done
-};
-// Named barriers (bar.arrive by the writers or readers that move on, bar.sync by the side that has to wait), all
-// counting every consumer thread: 1 all consumers, 2 expansion warps, 3 value warps, then per tile buffer b:
-constexpr int BAR_S_READY = 4;   // + b: score tile written (value warps arrive, expansion warps wait)
-constexpr int BAR_S_FREE = 6;    // + b: score tile read     (expansion warps arrive, value warps wait)
-constexpr int BAR_W_READY = 8;   // + b: weight tile written (expansion warps arrive, value warps wait)
-constexpr int BAR_W_FREE = 10;   // + b: weight tile read    (value warps arrive, expansion warps wait)
-
-// The plain K/V rows a unit attends over: its slice [g0, g1) of the concatenation [leading segment | text rows], as a
-// range of the leading segment (a0, a1; tensor maps tmK / tmV) and a range of the text rows (b0, b1; tmKt / tmVt)
-struct RowRanges { int a0, a1, b0, b1, na, nb; };
-__device__ __forceinline__ RowRanges row_ranges(const FusedArgs& a, int rg) {
-  RowRanges r;
-  const int g0 = rg * a.Tper, g1 = min(a.S0 + a.T, g0 + a.Tper);
-  r.a0 = min(g0, a.S0); r.a1 = min(g1, a.S0);
-  r.b0 = max(g0, a.S0) - a.S0; r.b1 = max(g1, a.S0) - a.S0;
-  r.na = r.a1 > r.a0 ? (r.a1 - r.a0 + a.TCH - 1) / a.TCH : 0;
-  r.nb = r.b1 > r.b0 ? (r.b1 - r.b0 + a.TCH - 1) / a.TCH : 0;
-  return r;
-}
 
 // EW expansion warps, VW value warps, one producer warp.  Every expansion warp owns up to KTW 16-column groups of
 // the logits; NH = 8-head tiles of the group (1: G <= 8, 2: G <= 16); MT = 16-row tiles of expansion rows per unit
@@ -822,6 +772,10 @@ static void warp_split(int n, int* ew, int* vw, int* ktw_max) {
 }
 
 FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
+  if (L->use_tc) {
+    const FusedPlan t = plan_fused_tc(L, B, R);
+    if (t.ok) return t;
+  }
   FusedPlan p{};
   const int G = L->G, n = L->desc.n, m = L->m, H_kv = L->desc.H_kv;
   if (L->desc.dtype != KVC_BF16 || L->passthrough || R < 1 || B < 1 || n % 64 != 0 || n > 1024 || G > 16) return p;
@@ -1025,12 +979,14 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
   fa.off_q = ring + p.off_q; fa.off_S = ring + p.off_S; fa.off_W = ring + p.off_W; fa.off_wred = ring + p.off_wred;
   fa.off_rstat = ring + p.off_rstat; fa.off_tstat = ring + p.off_tstat; fa.off_hstat = ring + p.off_hstat;
   fa.off_yred = ring + p.off_yred;
+  fa.off_P = ring + p.off_P; fa.off_rtab = ring + p.off_rtab; fa.tmem_cols = p.tmem_cols;
   fa.part_y = a.fpart_y;
   fa.part_ml = a.fpart_ml;
   fa.cnt = L->d_cnt;
   fa.status = a.status;
 
-  ProfScope prof(KVC_KERNEL_FUSED, st);
+  ProfScope prof(p.tc ? KVC_KERNEL_FUSED_TC : KVC_KERNEL_FUSED, st);
+  if (p.tc) return launch_fused_tc_kernel(tm, fa, p, st);
   return a.G > 8 ? launch_nh<2>(tm, fa, p, st) : launch_nh<1>(tm, fa, p, st);
 }
 

@@ -1,0 +1,883 @@
+// Algorithm 1 as one kernel for bf16 storage, with the two expansions on the 5th-generation tensor cores:
+//   L^T[n x rows] += theta_c^T[n x 16] S_c^T[16 x rows]      (Alg. 1 step 2; logits accumulate in tensor memory)
+//   W_c^T[rows of c x rows] = U_c[rows of c x n] P^T[n x rows]  (Alg. 1 step 3, re-projection of the probabilities)
+// `rows` = the expansion rows of a work unit (sequence, block, head), the N dimension of both products, so that the
+// large dimensions (n and the stage's rows of theta/U) are the M dimension of tcgen05.mma and the operand tiles are
+// read exactly as the TMA engine lays them down (128-byte swizzle): theta_c as an MN-major A operand, U_c as a
+// K-major A operand.  Work units, stages and the producer are those of kvc_fused.cu.  Warp roles:
+//   warps 0-3        softmax over the logits read back from tensor memory (one lane per column of L^T), P as a
+//                    bf16 operand in shared memory; in pass C they move W^T from tensor memory to the weight tile
+//   value warps      S_c = sigma q K_c^T (mma.sync, bf16 tile in shared memory in UMMA core-matrix order), text rows
+//                    flash-style, y^T += V_c^T W_c^T, unit end: reduction, mu term, output or partial + merge
+//   MMA warp         one thread issues every tcgen05.mma and commits completion to the mbarriers that free the
+//                    stage, the score tile and the accumulators
+//   producer warp    one thread feeds the ring through tensor maps
+//
+// Status: opt-in (KVC_EXPANSION=tcgen05 when the layer is created).  Measured on B200: one tcgen05.mma of K = 16
+// occupies the tensor pipe for about 85 cycles at M = 64 and about 129 cycles at M = 128 whatever N <= 128 is (one
+// row of A per cycle), so with N = 16 or 32 expansion rows the re-projection (n/16 MMAs per stage) is bound by the
+// MMA count, not by data; the products only pay off with >= 64 rows on both M and N, i.e. with work units that
+// batch the expansion rows of many sequences of a head.
+#include "kvc_fused.cuh"
+#include "kvc_tcgen05.cuh"
+
+namespace kvc {
+
+constexpr int TEW = 4;                         // softmax / conversion warps: one per tensor-memory lane quarter
+constexpr int BAR_P_READY = 12;                // probabilities written (warps 0-3 arrive, the MMA warp waits)
+constexpr int BAR_END = 13;                    // every tensor-memory user is done: the MMA warp may free it
+
+struct TcBars {
+  uint64_t full[FMAX_STAGES], empty[FMAX_STAGES];
+  uint64_t s_free[2];      // the MMAs that read score tile b have completed
+  uint64_t w_done[2];      // W^T of a stage is complete in accumulator b
+  uint64_t w_tfree[2];     // accumulator b has been read back (4 warps)
+  uint64_t l_done;         // the logits of the unit are complete
+  uint64_t l_free;         // the logits of the unit have been read back (4 warps)
+};
+
+template <int VW, int NH, int MT>
+__global__ void __launch_bounds__((TEW + VW + 2) * 32, 1)
+fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                       const __grid_constant__ CUtensorMap tmKt, const __grid_constant__ CUtensorMap tmVt,
+                       const __grid_constant__ CUtensorMap tmTh, const __grid_constant__ CUtensorMap tmU,
+                       const FusedArgs a) {
+  constexpr int CW = TEW + VW;                // warps that meet at the softmax barriers
+  constexpr int FCONS = CW * 32;
+  constexpr int MMA_WARP = CW, PROD_WARP = CW + 1;
+  constexpr int FTHREADS = (CW + 2) * 32;
+  constexpr int RT = ROWS * MT;               // expansion rows of a unit = N of the expansion MMAs
+  constexpr int SREADY = VW * 32 + 32;        // value warps arrive, the MMA warp waits
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  unsigned char* sm = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
+  __shared__ __align__(8) TcBars bars;
+  __shared__ int s_last;
+  __shared__ uint32_t s_tmem;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) {
+    for (int s = 0; s < a.stages; ++s) { mbar_init(&bars.full[s], 1); mbar_init(&bars.empty[s], VW + 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&bars.s_free[b], 1); mbar_init(&bars.w_done[b], 1); mbar_init(&bars.w_tfree[b], TEW); }
+    mbar_init(&bars.l_done, 1);
+    mbar_init(&bars.l_free, TEW);
+    fence_mbar_init();
+  }
+  if (warp == MMA_WARP) tmem_alloc(&s_tmem, (uint32_t)a.tmem_cols);
+  const int JC = a.JC;
+  const uint32_t s_buf_bytes = (uint32_t)(JC * RT * 32);            // score tile buffer: [JC][2 halves][RT/8][8][8]
+  const int w_buf_elems = JC * (RT + 16) * SLD;                      // weight tile buffer: [JC][RT + 16][SLD]
+  // score and weight tiles start as zeros: their padding rows and columns are read by the MMAs
+  {
+    uint32_t* z = reinterpret_cast<uint32_t*>(sm + a.off_S);
+    const int words = (int)(2 * s_buf_bytes) / 4 + w_buf_elems;      // 2 score buffers (bytes / 4) + 2 weight buffers (elements / 2)
+    for (int i = tid; i < words; i += FTHREADS) z[i] = 0u;
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tb = s_tmem;                  // tensor memory: L^T tiles at columns [0, NT*RT), W^T buffers after them
+  const int NT = (a.n + 127) >> 7;
+  const uint32_t w_col = (uint32_t)(NT * RT);
+
+  const int per_h = a.nbg * a.nrg;
+  const int rows16 = 16 * JC;                      // rows of one block inside a stage
+  const uint32_t sm_u = smem_addr(sm);
+
+  if (warp == PROD_WARP) {
+    // ================= producer: one thread feeds the ring =================
+    if (lane != 0) return;
+    tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmTh); tma_prefetch_desc(&tmU);
+    if (a.T > 0) { tma_prefetch_desc(&tmKt); tma_prefetch_desc(&tmVt); }
+    bool first = true;
+    uint32_t slot = 0, phase = 1;              // parity to wait for on the empty barrier: 1 passes on a fresh barrier
+    for (int u = blockIdx.x; u < a.units; u += gridDim.x) {
+      const int h = u / per_h, rem = u - h * per_h;
+      const int bg = rem / a.nrg, rg = rem - bg * a.nrg;
+      const int b0 = bg * a.NB, r0 = rg * a.RB;
+      const RowRanges tr = row_ranges(a, rg);
+      const int nts = tr.na + tr.nb;
+      for (int part = 0; part < 3; ++part) {
+        const int count = part == 1 ? nts : a.NJ;
+        for (int c = 0; c < count; ++c) {
+          if (!mbar_wait_bounded(&bars.empty[slot], phase)) { atomicExch(a.status, (int)KVC_ERR_TIMEOUT); return; }
+          unsigned char* dst = sm + slot * a.stage_bytes;
+          uint64_t* bar = &bars.full[slot];
+          if (part == 1) {
+            const int y = tr.b0 + c * a.TCH;
+            mbar_expect_tx(bar, 4 * a.txt_half_bytes);
+            if (first) { grid_dep_wait(); first = false; }
+            tma_load_4d(dst, &tmKt, 0, y, h, b0, bar);
+            tma_load_4d(dst + a.txt_half_bytes, &tmKt, 64, y, h, b0, bar);
+            tma_load_4d(dst + 2 * a.txt_half_bytes, &tmVt, 0, y, h, b0, bar);
+            tma_load_4d(dst + 3 * a.txt_half_bytes, &tmVt, 64, y, h, b0, bar);
+          } else {
+            const CUtensorMap* tp = part == 0 ? &tmTh : &tmU;
+            const CUtensorMap* tk = part == 0 ? &tmK : &tmV;
+            const int j0 = c * rows16;
+            mbar_expect_tx(bar, a.par_bytes + 2 * a.k_half_bytes);
+            tma_load_4d(dst, tp, 0, j0, 0, h, bar);                  // parameters: never written by this library
+            if (first) { grid_dep_wait(); first = false; }            // everything else may come from the stream's previous kernel
+            tma_load_5d(dst + a.par_bytes, tk, 0, j0, r0, h, b0, bar);
+            tma_load_5d(dst + a.par_bytes + a.k_half_bytes, tk, 64, j0, r0, h, b0, bar);
+          }
+          if (++slot == (uint32_t)a.stages) { slot = 0; phase ^= 1u; }
+        }
+      }
+    }
+    return;
+  }
+
+  grid_dep_wait();
+  grid_dep_launch();
+  if (blockIdx.x == 0 && tid == 0) *a.status = 0;
+
+  uint32_t slot = 0, phase = 0;
+  uint32_t si = 0, wi = 0;                         // score tiles and weight tiles (one per stage) handed over so far
+  uint32_t ucount = 0;                             // units this CTA has started
+  bool dead = false;
+  auto wait_on = [&](uint64_t* bar, uint32_t parity) { if (!dead && !mbar_wait_bounded(bar, parity)) dead = true; };
+  auto advance = [&]() { if (++slot == (uint32_t)a.stages) { slot = 0; phase ^= 1u; } };
+
+  if (warp == MMA_WARP) {
+    // ======================================================================================================
+    // MMA warp: lane 0 issues the expansion MMAs of every stage
+    // ======================================================================================================
+    const uint32_t S_u = sm_u + a.off_S, P_u = sm_u + a.off_P;
+    const uint32_t cg_bytes = (uint32_t)rows16 * 128u;            // one 64-column group of a parameter tile
+    const uint32_t idesc_L_full = umma_idesc_bf16(128, RT, 1, 0);
+    const uint32_t idesc_L_half = umma_idesc_bf16(64, RT, 1, 0);
+    const uint32_t idesc_W = umma_idesc_bf16(64, RT, 0, 0);
+    const bool half_tail = (a.n & 127) != 0;                      // n = 64 (mod 128): the last tile of L^T has 64 rows
+    for (int u = blockIdx.x; u < a.units; u += gridDim.x, ++ucount) {
+      const int rem = u % per_h;
+      const int rg = rem % a.nrg;
+      const RowRanges tr = row_ranges(a, rg);
+      const int nts = tr.na + tr.nb;
+      // ---------------- pass A ----------------
+      if (ucount > 0) wait_on(&bars.l_free, (ucount - 1) & 1u);    // the previous unit's logits have been read back
+      for (int c = 0; c < a.NJ; ++c) {
+        wait_on(&bars.full[slot], phase);
+        const uint32_t sbuf = si & 1u;
+        named_barrier_sync(BAR_S_READY + (int)sbuf, SREADY);
+        tc_fence_after();
+        if (lane == 0) {
+          const uint32_t par_u = sm_u + slot * a.stage_bytes;
+          const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);
+          for (int s = 0; s < nsub; ++s) {
+            const uint64_t bdesc = umma_smem_desc(S_u + sbuf * s_buf_bytes + (uint32_t)(s * RT * 32), (uint32_t)(RT * 16), 128u, UMMA_LAYOUT_NONE);
+            for (int t = 0; t < NT; ++t) {
+              const uint64_t adesc = umma_smem_desc(par_u + (uint32_t)(2 * t) * cg_bytes + (uint32_t)(s * 2048), cg_bytes, 1024u, UMMA_LAYOUT_SW128);
+              umma_bf16(tb + (uint32_t)(t * RT), adesc, bdesc, (half_tail && t == NT - 1) ? idesc_L_half : idesc_L_full, (c | s) ? 1u : 0u);
+            }
+          }
+          umma_commit(&bars.empty[slot]);
+          umma_commit(&bars.s_free[sbuf]);
+          if (c == a.NJ - 1) umma_commit(&bars.l_done);
+        }
+        __syncwarp();
+        ++si;
+        advance();
+      }
+      // ---------------- text stages belong to the value warps ----------------
+      for (int ts = 0; ts < nts; ++ts) {
+        wait_on(&bars.full[slot], phase);
+        if (lane == 0) mbar_arrive(&bars.empty[slot]);
+        advance();
+      }
+      // ---------------- pass C ----------------
+      named_barrier_sync(BAR_P_READY, TEW * 32 + 32);
+      for (int c = 0; c < a.NJ; ++c) {
+        wait_on(&bars.full[slot], phase);
+        const uint32_t wbuf = wi & 1u;
+        if (wi >= 2) wait_on(&bars.w_tfree[wbuf], ((wi >> 1) - 1) & 1u);
+        tc_fence_after();
+        if (lane == 0) {
+          const uint32_t par_u = sm_u + slot * a.stage_bytes;
+          for (int cg = 0; cg < a.ncg; ++cg)
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+              const uint64_t adesc = umma_smem_desc(par_u + (uint32_t)cg * cg_bytes + (uint32_t)(kk * 32), 16u, 1024u, UMMA_LAYOUT_SW128);
+              const uint64_t bdesc = umma_smem_desc(P_u + (uint32_t)(cg * RT * 128 + kk * 32), 16u, 1024u, UMMA_LAYOUT_SW128);
+              umma_bf16(tb + w_col + wbuf * RT, adesc, bdesc, idesc_W, (cg | kk) ? 1u : 0u);
+            }
+          umma_commit(&bars.w_done[wbuf]);
+          umma_commit(&bars.empty[slot]);
+        }
+        __syncwarp();
+        ++wi;
+        advance();
+      }
+    }
+    tc_fence_before();
+    named_barrier_sync(BAR_END, (CW + 1) * 32);
+    tmem_dealloc(tb, (uint32_t)a.tmem_cols);
+    if (dead && lane == 0) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
+    return;
+  }
+
+  // ================= softmax / conversion warps and value warps: common set-up =================
+  const int gid = lane >> 2, t4 = lane & 3;
+  const int G = a.G, RB = a.RB;
+  const uint32_t q_u = sm_u + a.off_q, W_u = sm_u + a.off_W;
+  __nv_bfloat16* q_sm = reinterpret_cast<__nv_bfloat16*>(sm + a.off_q);
+  unsigned char* S_sm = sm + a.off_S;                                        // [2][JC][2][RT/8][8][8] bf16
+  __nv_bfloat16* W_sm = reinterpret_cast<__nv_bfloat16*>(sm + a.off_W);      // [2][JC][RT + 16][SLD]
+  float* rmax = reinterpret_cast<float*>(sm + a.off_rstat);                  // [TEW][RT]
+  float* rsum = rmax + TEW * RT;
+  float* tmax = reinterpret_cast<float*>(sm + a.off_tstat);                  // [VW][16]
+  float* tsum = tmax + VW * 16;
+  float* hmax = reinterpret_cast<float*>(sm + a.off_hstat);                  // [NB][16]
+  float* hsum = hmax + a.NB * 16;
+  float* vsum = hsum + a.NB * 16;
+  int* rtab = reinterpret_cast<int*>(sm + a.off_rtab);                       // [RT] head slot of an expansion row, -1 if unused
+  float* yred = reinterpret_cast<float*>(sm + a.off_yred);                   // [VW][yhg][D]
+  const float qscale = 0.08838834764831845f * 1.4426950408889634f;   // sigma = 1/sqrt(128), logits kept in log2 units
+  const int l7 = lane & 7;
+  const int lrow = l7 + ((lane >> 3) & 1) * 8;     // ldmatrix address pattern A: rows 0-15 by lanes 0-15, twice
+  const int lhi = lane >> 4;
+  const int lrowB = l7 + lhi * 8;                  // address pattern B: rows 0-7 | 0-7 | 8-15 | 8-15
+  const int lmid = (lane >> 3) & 1;
+  const int WPG = VW / a.NB;                       // value warps per sequence of the unit
+
+  if (warp < TEW) {
+    // ======================================================================================================
+    // warps 0-3: joint softmax on the logits in tensor memory, then W^T -> weight tiles
+    // ======================================================================================================
+    const uint32_t tq = tb + ((uint32_t)(warp * 32) << 16);       // this warp's lane quarter
+    const bool half_tail = (a.n & 127) != 0;
+    unsigned char* P_sm = sm + a.off_P;                           // [n/64][RT][64] bf16, 128-byte swizzle
+    for (int u = blockIdx.x; u < a.units; u += gridDim.x, ++ucount) {
+      const int h = u / per_h, rem = u - h * per_h;
+      const int bg = rem / a.nrg, rg = rem - bg * a.nrg;
+      const int b0 = bg * a.NB, r0 = rg * a.RB;
+      const int nbv = min(a.NB, a.B - b0);
+      const int rbv = min(RB, a.R - r0);
+      (void)h;
+      // expansion row rho <-> (sequence, block, head); this lane's own row for the statistics: rho = lane
+      bool my_valid = false;
+      {
+        const int rho = lane;
+        const int bi = rho / G, g = rho - bi * G;
+        const int rbl = bi / RB, rrl = bi - rbl * RB;
+        my_valid = rho < RT && rho < a.NB * RB * G && rbl < nbv && rrl < rbv;
+        if (warp == 0 && rho < RT) rtab[rho] = my_valid ? rbl * 16 + g : -1;
+      }
+
+      // ---------------- maxima of the logits ----------------
+      wait_on(&bars.l_done, ucount & 1u);
+      __syncwarp();
+      tc_fence_after();
+      float mx[RT];
+#pragma unroll
+      for (int r = 0; r < RT; ++r) mx[r] = -INFINITY;
+      for (int t = 0; t < NT; ++t) {
+        float v[RT];
+        __syncwarp();
+        tmem_ld<RT>(tq + (uint32_t)(t * RT), v);
+        const bool lane_ok = !(half_tail && t == NT - 1) || lane < 16;
+        if (lane_ok) {
+#pragma unroll
+          for (int r = 0; r < RT; ++r) mx[r] = fmaxf(mx[r], v[r]);
+        }
+      }
+      {
+        float mine = -INFINITY;
+#pragma unroll
+        for (int r = 0; r < RT; ++r) {
+          float x = mx[r];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+          if (lane == r) mine = x;
+        }
+        if (lane < RT) rmax[warp * RT + lane] = my_valid ? mine : -INFINITY;
+      }
+      named_barrier_sync(1, FCONS);                                   // B1: row maxima and text maxima are in place
+      if (warp == 0) {
+        for (int x = lane; x < RT; x += 32) {
+          float m_ = -INFINITY;
+#pragma unroll
+          for (int w = 0; w < TEW; ++w) m_ = fmaxf(m_, rmax[w * RT + x]);
+          rmax[x] = m_;
+        }
+        __syncwarp();
+        for (int x = lane; x < a.NB * 16; x += 32) {
+          const int tb_ = x >> 4, g = x & 15;
+          float m_ = 0.f;
+          if (g < G && tb_ < nbv) {
+            m_ = -INFINITY;
+            for (int rl = 0; rl < rbv; ++rl) m_ = fmaxf(m_, rmax[(tb_ * RB + rl) * G + g]);
+            for (int w = tb_ * WPG; w < (tb_ + 1) * WPG; ++w) m_ = fmaxf(m_, tmax[w * 16 + g]);
+          }
+          hmax[x] = m_;
+        }
+      }
+      named_barrier_sync(1, FCONS);                                   // B2: head maxima
+
+      // ---------------- P = 2^(L - max) as the bf16 operand of the re-projection; row sums ----------------
+      float Mr[RT];
+      uint32_t vmask = 0;
+#pragma unroll
+      for (int r = 0; r < RT; ++r) {
+        const int slot_ = rtab[r];
+        Mr[r] = slot_ >= 0 ? hmax[slot_] : 0.f;
+        vmask |= slot_ >= 0 ? (1u << r) : 0u;
+      }
+      float sum[RT];
+#pragma unroll
+      for (int r = 0; r < RT; ++r) sum[r] = 0.f;
+      for (int t = 0; t < NT; ++t) {
+        float v[RT];
+        __syncwarp();
+        tmem_ld<RT>(tq + (uint32_t)(t * RT), v);
+        const bool tail = half_tail && t == NT - 1;
+        const bool lane_ok = !tail || lane < 16;
+        const int i = t * 128 + (tail ? warp * 16 : warp * 32) + lane;          // column of L = row of L^T
+        const uint32_t cgo = (uint32_t)((i >> 6) * (RT * 128)), c8 = (uint32_t)((i & 63) >> 3), cl = (uint32_t)((i & 7) * 2);
+        if (lane_ok) {
+#pragma unroll
+          for (int r = 0; r < RT; ++r) {
+            const float p = (vmask >> r & 1u) ? fast_exp2(v[r] - Mr[r]) : 0.f;
+            sum[r] += p;
+            *reinterpret_cast<__nv_bfloat16*>(P_sm + cgo + (uint32_t)(r * 128) + ((c8 ^ (uint32_t)(r & 7)) << 4) + cl) = __float2bfloat16_rn(p);
+          }
+        }
+      }
+      {
+        float mine = 0.f;
+#pragma unroll
+        for (int r = 0; r < RT; ++r) {
+          float x = sum[r];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+          if (lane == r) mine = x;
+        }
+        if (lane < RT) rsum[warp * RT + lane] = mine;
+      }
+      fence_proxy_async();                                             // P is read by the tensor core (async proxy)
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars.l_free);
+      named_barrier_arrive(BAR_P_READY, TEW * 32 + 32);
+      named_barrier_sync(1, FCONS);                                   // B3: row sums and text sums are in place
+      if (warp == 0) {
+        for (int x = lane; x < RT; x += 32) {
+          float s_ = 0.f;
+#pragma unroll
+          for (int w = 0; w < TEW; ++w) s_ += rsum[w * RT + x];
+          rsum[x] = s_;
+        }
+        __syncwarp();
+        for (int x = lane; x < a.NB * 16; x += 32) {
+          const int tb_ = x >> 4, g = x & 15;
+          float vs = 0.f, tsm = 0.f;
+          if (g < G && tb_ < nbv) {
+            for (int rl = 0; rl < rbv; ++rl) vs += rsum[(tb_ * RB + rl) * G + g];
+            for (int w = tb_ * WPG; w < (tb_ + 1) * WPG; ++w) tsm += tsum[w * 16 + g];
+          }
+          vsum[x] = vs;
+          hsum[x] = vs + tsm;
+        }
+      }
+      named_barrier_sync(1, FCONS);                                   // B4: head sums
+
+      // ---------------- pass C: W^T of every stage from tensor memory to the weight tile ----------------
+      for (int c = 0; c < a.NJ; ++c) {
+        const uint32_t wbuf = wi & 1u;
+        const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);
+        wait_on(&bars.w_done[wbuf], (wi >> 1) & 1u);
+        __syncwarp();
+        tc_fence_after();
+        float v[RT];
+        if (warp < nsub) tmem_ld<RT>(tq + w_col + wbuf * RT, v);      // lane j < 16: row j of sub-chunk `warp`
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars.w_tfree[wbuf]);
+        if (wi >= 2) named_barrier_sync(BAR_W_FREE + (int)wbuf, FCONS);   // the value warps are done with this buffer's previous tile
+        if (warp < nsub && lane < 16) {
+          __nv_bfloat16* wt = W_sm + wbuf * w_buf_elems + warp * ((RT + 16) * SLD) + lane;
+#pragma unroll
+          for (int r = 0; r < RT; ++r) wt[r * SLD] = __float2bfloat16_rn(v[r]);
+        }
+        named_barrier_arrive(BAR_W_READY + (int)wbuf, FCONS);
+        ++wi;
+      }
+    }
+    named_barrier_sync(BAR_END, (CW + 1) * 32);
+    if (dead && lane == 0) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
+    return;
+  }
+
+  // ======================================================================================================
+  // value warps: scores, text attention, y^T += V^T W^T, output
+  // ======================================================================================================
+  // the stage in `slot` has been consumed by this warp
+  auto release = [&]() {
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&bars.empty[slot]);
+    advance();
+  };
+  const int VTH = VW * 32;
+  const int vw = warp - TEW, vtid = tid - TEW * 32;
+  const int bl = vw / WPG, wig = vw - bl * WPG;
+  const int msplit = a.msplit, mshift = a.mshift;           // a task covers the row tiles mt with (mt >> mshift) == its group
+
+  for (int u = blockIdx.x; u < a.units; u += gridDim.x) {
+    const int h = u / per_h, rem = u - h * per_h;
+    const int bg = rem / a.nrg, rg = rem - bg * a.nrg;
+    const int b0 = bg * a.NB, r0 = rg * a.RB;
+    const int nbv = min(a.NB, a.B - b0);
+    const int rbv = min(RB, a.R - r0);
+    const RowRanges tr = row_ranges(a, rg);
+    const int nts = tr.na + tr.nb;
+
+    // ---- queries of the unit's sequences: [NB][16 heads][128], heads >= G and absent sequences are zero rows
+    for (int idx = vtid; idx < a.NB * 256; idx += VTH) {
+      const int tb = idx >> 8, g = (idx >> 4) & 15, piece = idx & 15;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (tb < nbv && g < G)
+        v = *reinterpret_cast<const uint4*>(a.q + ((size_t)(b0 + tb) * a.H_kv * G + (size_t)h * G + g) * D + piece * 8);
+      *reinterpret_cast<uint4*>(q_sm + (tb * 16 + g) * QLD + piece * 8) = v;
+    }
+    named_barrier_sync(3, VTH);
+    uint32_t qf[NH][8][2];                          // B operand of the score MMA: heads of sequence bl
+#pragma unroll
+    for (int nh = 0; nh < NH; ++nh)
+#pragma unroll
+      for (int k2 = 0; k2 < 4; ++k2) {
+        uint32_t r[4];
+        ldsm_x4(r, q_u + (uint32_t)(((bl * 16 + nh * 8 + l7) * QLD + k2 * 32 + (lane >> 3) * 8) * 2));
+        qf[nh][2 * k2][0] = r[0]; qf[nh][2 * k2][1] = r[1];
+        qf[nh][2 * k2 + 1][0] = r[2]; qf[nh][2 * k2 + 1][1] = r[3];
+      }
+
+    // ---------------- pass A: S[rows of block][16] = sigma q K^T for my (block, sub-chunk) tasks ----------------
+    for (int c = 0; c < a.NJ; ++c) {
+      wait_on(&bars.full[slot], phase);
+      const uint32_t k_u = sm_u + slot * a.stage_bytes + a.par_bytes;
+      const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);
+      const uint32_t sbuf = si & 1u;
+      if (si >= 2) wait_on(&bars.s_free[sbuf], ((si >> 1) - 1) & 1u);   // the MMAs that read this buffer's previous tile are complete
+      unsigned char* Sb = S_sm + sbuf * s_buf_bytes;
+      for (int task = wig; task < RB * nsub; task += WPG) {
+        const int rl = nsub == 1 ? task : task / nsub, s = task - rl * nsub;
+        const int bi = bl * RB + rl;
+        const uint32_t rowoff = k_u + (uint32_t)((bi * rows16 + s * 16 + lrow) * 128);
+        uint32_t af[8][4];
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+          ldsm_x4(af[ks], rowoff + (ks >> 2) * a.k_half_bytes + (uint32_t)(((((ks & 3) * 2 + lhi)) ^ l7) << 4));
+        float sc[NH][2][4];
+#pragma unroll
+        for (int nh = 0; nh < NH; ++nh)
+#pragma unroll
+          for (int x = 0; x < 2; ++x)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) sc[nh][x][e] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+#pragma unroll
+          for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(sc[nh][ks & 1], af[ks], qf[nh][ks][0], qf[nh][ks][1]);
+#pragma unroll
+        for (int nh = 0; nh < NH; ++nh)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int head = nh * 8 + 2 * t4 + (e & 1), j = gid + (e >> 1) * 8;
+            if (head < G) {
+              // element (row rho, column j) of sub-chunk s, K-major core matrices of 8 rows x 8 columns
+              const int rho = bi * G + head;
+              *reinterpret_cast<__nv_bfloat16*>(Sb + s * (RT * 32) + (j >> 3) * (RT * 16) + (rho >> 3) * 128 + (rho & 7) * 16 + (j & 7) * 2) =
+                  __float2bfloat16_rn((sc[nh][0][e] + sc[nh][1][e]) * qscale);
+            }
+          }
+      }
+      fence_proxy_async();                                              // the tile is read by the tensor core (async proxy)
+      named_barrier_arrive(BAR_S_READY + (int)sbuf, SREADY);
+      ++si;
+      release();
+    }
+
+    // ---------------- text rows: online-softmax attention per warp ----------------
+    // yacc[mt][nh]: y^T tile, rows = head-dimension mt*16 + gid (+8), columns = heads nh*8 + 2*t4 (+1) of sequence bl
+    float yacc[8][NH][4];
+#pragma unroll
+    for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+      for (int nh = 0; nh < NH; ++nh)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) yacc[mt][nh][e] = 0.f;
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // heads gid and gid + 8
+    for (int ts = 0; ts < nts; ++ts) {
+      wait_on(&bars.full[slot], phase);
+      const uint32_t kt_u = sm_u + slot * a.stage_bytes, vt_u = kt_u + 2 * a.txt_half_bytes;
+      for (int tile = wig; tile * 16 < a.TCH; tile += WPG) {
+        const int ts1 = ts < tr.na ? tr.a1 : tr.b1;               // end of the row range this stage belongs to
+        const int t_first = (ts < tr.na ? tr.a0 + ts * a.TCH : tr.b0 + (ts - tr.na) * a.TCH) + tile * 16;
+        if (t_first >= ts1) break;
+        const int row0 = bl * a.TCH + tile * 16;
+        const uint32_t rowB = (uint32_t)((row0 + lrowB) * 128);
+        // logits [16 heads][16 text rows] = q K_txt^T
+        float cc[2][4];
+        {
+          float c2[2][2][4];                       // two accumulation chains per tile column
+#pragma unroll
+          for (int x = 0; x < 2; ++x)
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+              for (int e = 0; e < 4; ++e) c2[x][nt][e] = 0.f;
+#pragma unroll
+          for (int kh = 0; kh < 2; ++kh) {
+            uint32_t bk[4][4], aq[4][4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+              const int ks = kh * 4 + x;
+              ldsm_x4(bk[x], kt_u + kh * a.txt_half_bytes + rowB + (uint32_t)((((x * 2 + lmid)) ^ l7) << 4));
+              ldsm_x4(aq[x], q_u + (uint32_t)(((bl * 16 + lrow) * QLD + ks * 16 + lhi * 8) * 2));
+            }
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+              mma_bf16_16816(c2[x & 1][0], aq[x], bk[x][0], bk[x][1]);
+              mma_bf16_16816(c2[x & 1][1], aq[x], bk[x][2], bk[x][3]);
+            }
+          }
+#pragma unroll
+          for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) cc[nt][e] = c2[0][nt][e] + c2[1][nt][e];
+        }
+        // cc[nt][e]: head gid + 8*(e>>1), text row t_first + nt*8 + 2*t4 + (e&1)
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int t = t_first + nt * 8 + 2 * t4 + (e & 1);
+            cc[nt][e] = t < ts1 ? cc[nt][e] * qscale : -INFINITY;
+          }
+        float scl[2];
+#pragma unroll
+        for (int hr = 0; hr < 2; ++hr) {
+          float mx = fmaxf(fmaxf(cc[0][2 * hr], cc[0][2 * hr + 1]), fmaxf(cc[1][2 * hr], cc[1][2 * hr + 1]));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+          const float m_new = fmaxf(m_run[hr], mx);              // finite: the tile has at least one valid row
+          scl[hr] = fast_exp2(m_run[hr] - m_new);                // 0 on the first tile
+          m_run[hr] = m_new;
+          float ps = 0.f;
+#pragma unroll
+          for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+              const float p = fast_exp2(cc[nt][2 * hr + k] - m_new);
+              cc[nt][2 * hr + k] = p;
+              ps += p;
+            }
+          l_run[hr] = l_run[hr] * scl[hr] + ps;
+        }
+        // the accumulator's columns are heads: fetch their factors from the lanes that own those heads as rows
+#pragma unroll
+        for (int nh = 0; nh < NH; ++nh) {
+          const float c0s = __shfl_sync(0xffffffffu, scl[nh], (2 * t4) * 4);
+          const float c1s = __shfl_sync(0xffffffffu, scl[nh], (2 * t4 + 1) * 4);
+          if (c0s != 1.f || c1s != 1.f) {
+#pragma unroll
+            for (int mt = 0; mt < 8; ++mt) {
+              yacc[mt][nh][0] *= c0s; yacc[mt][nh][1] *= c1s;
+              yacc[mt][nh][2] *= c0s; yacc[mt][nh][3] *= c1s;
+            }
+          }
+        }
+        // y^T[128][heads] += V_txt^T[128][16 rows] P^T[16 rows][heads]
+        uint32_t pb[2][2];
+        pb[0][0] = pack2_bf16(cc[0][0], cc[0][1]); pb[0][1] = pack2_bf16(cc[1][0], cc[1][1]);
+        pb[1][0] = pack2_bf16(cc[0][2], cc[0][3]); pb[1][1] = pack2_bf16(cc[1][2], cc[1][3]);
+        uint32_t av[8][4];
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt)
+          ldsm_x4_t(av[mt], vt_u + (mt >> 2) * a.txt_half_bytes + rowB + (uint32_t)(((((mt & 3) * 2 + lmid)) ^ l7) << 4));
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+          for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(yacc[mt][nh], av[mt], pb[nh][0], pb[nh][1]);
+      }
+      release();
+    }
+
+    // ---------------- joint softmax: the text accumulators move to the unit's reference maximum ----------------
+    if (t4 == 0) { tmax[vw * 16 + gid] = m_run[0]; tmax[vw * 16 + gid + 8] = m_run[1]; }
+    named_barrier_sync(1, FCONS);                                   // B1
+    named_barrier_sync(1, FCONS);                                   // B2: head maxima
+    {
+      float scl[2];
+#pragma unroll
+      for (int hr = 0; hr < 2; ++hr) {
+        const int head = gid + 8 * hr;
+        const float M = hmax[bl * 16 + head];
+        scl[hr] = m_run[hr] == -INFINITY ? 0.f : fast_exp2(m_run[hr] - M);
+        float l = l_run[hr] * scl[hr];
+        l += __shfl_xor_sync(0xffffffffu, l, 1);
+        l += __shfl_xor_sync(0xffffffffu, l, 2);
+        if (t4 == 0) tsum[vw * 16 + head] = l;
+      }
+#pragma unroll
+      for (int nh = 0; nh < NH; ++nh) {
+        const float c0s = __shfl_sync(0xffffffffu, scl[nh], (2 * t4) * 4);
+        const float c1s = __shfl_sync(0xffffffffu, scl[nh], (2 * t4 + 1) * 4);
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt) {
+          yacc[mt][nh][0] *= c0s; yacc[mt][nh][1] *= c1s;
+          yacc[mt][nh][2] *= c0s; yacc[mt][nh][3] *= c1s;
+        }
+      }
+    }
+    named_barrier_sync(1, FCONS);                                   // B3
+    named_barrier_sync(1, FCONS);                                   // B4: head sums
+
+    // ---------------- pass C: y^T[128][heads] += V^T[128][16 rows of block] W^T[16][heads of block] ----------------
+    for (int c = 0; c < a.NJ; ++c) {
+      wait_on(&bars.full[slot], phase);
+      const uint32_t v_u = sm_u + slot * a.stage_bytes + a.par_bytes;
+      const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);
+      const uint32_t wbuf = wi & 1u;
+      named_barrier_sync(BAR_W_READY + (int)wbuf, FCONS);
+      const int ntask = RB * msplit;
+      for (int task = wig; task < nsub * ntask; task += WPG) {          // my (sub-chunk, block, row-tile group) tasks
+        const int s = task / ntask, tk = task - s * ntask;
+        const int rl = tk >> (3 - mshift), mg = tk & (msplit - 1);
+        if (rl >= rbv || bl >= nbv) continue;
+        const int bi = bl * RB + rl;
+        uint32_t bw[4];
+        ldsm_x4(bw, W_u + (uint32_t)((wbuf * w_buf_elems + s * ((RT + 16) * SLD) + (bi * G + lrowB) * SLD + lmid * 8) * 2));
+        const uint32_t rowoff = v_u + (uint32_t)((bi * rows16 + s * 16 + lrowB) * 128);
+        uint32_t av[8][4];
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt)
+          if ((mt >> mshift) == mg)
+            ldsm_x4_t(av[mt], rowoff + (mt >> 2) * a.k_half_bytes + (uint32_t)(((((mt & 3) * 2 + lmid)) ^ l7) << 4));
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt)
+          if ((mt >> mshift) == mg) {
+#pragma unroll
+            for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(yacc[mt][nh], av[mt], bw[2 * nh], bw[2 * nh + 1]);
+          }
+      }
+      named_barrier_arrive(BAR_W_FREE + (int)wbuf, FCONS);
+      ++wi;
+      release();
+    }
+
+    // ---------------- unit end: reduce over the value warps, mu term, normalise or leave a partial ----------------
+    const int bh = b0 * a.H_kv + h;                    // used when the block axis is split (NB == 1)
+    const size_t pbase = ((size_t)bh * a.nrg + rg) * G;
+    const int YHG = a.yhg;
+    for (int g0 = 0; g0 < G; g0 += YHG) {
+      // every warp parks its tile columns of heads g0 .. g0+YHG-1; then the warps of a sequence are summed
+#pragma unroll
+      for (int nh = 0; nh < NH; ++nh)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int head = nh * 8 + 2 * t4 + e;
+          if (head >= g0 && head < g0 + YHG && head < G) {
+            float* yp = yred + (vw * YHG + (head - g0)) * D;
+#pragma unroll
+            for (int mt = 0; mt < 8; ++mt) {
+              yp[mt * 16 + gid] = yacc[mt][nh][e];
+              yp[mt * 16 + gid + 8] = yacc[mt][nh][2 + e];
+            }
+          }
+        }
+      named_barrier_sync(3, VTH);
+      const int hg = min(YHG, G - g0);
+      for (int idx = vtid; idx < nbv * hg * D; idx += VTH) {
+        const int col = idx & (D - 1), gg = (idx >> 7) % hg, tb = idx / (D * hg);
+        const int g = g0 + gg;
+        float y = 0.f;
+        for (int w = tb * WPG; w < (tb + 1) * WPG; ++w) y += yred[(w * YHG + gg) * D + col];
+        if (a.R > 0) y = fmaf(vsum[tb * 16 + g], __bfloat162float(a.mu[h * D + col]), y);
+        if (a.nrg == 1)
+          a.out[((size_t)(b0 + tb) * a.H_kv * G + (size_t)h * G + g) * D + col] = __float2bfloat16_rn(y / hsum[tb * 16 + g]);
+        else
+          a.part_y[(pbase + g) * D + col] = y;
+      }
+      named_barrier_sync(3, VTH);
+    }
+    if (a.nrg > 1) {
+      // one sequence, several units along the block axis: the last unit to arrive merges the partials
+      if (vtid < G) a.part_ml[pbase + vtid] = make_float2(hmax[vtid], hsum[vtid]);
+      __threadfence();
+      named_barrier_sync(3, VTH);
+      if (vtid == 0) {
+        const int old = atomicAdd(&a.cnt[bh], 1);
+        s_last = old == a.nrg - 1 ? 1 : 0;
+        if (s_last) a.cnt[bh] = 0;                  // every unit of (sequence, head) has arrived: ready for the next call
+      }
+      named_barrier_sync(3, VTH);
+      if (s_last) {
+        __threadfence();
+        const size_t p0 = (size_t)bh * a.nrg * G;
+        // weights of the partials, w[p][g] = 2^(max_p - max) / sum: first all (max, sum) pairs into shared memory
+        float* mlm = yred;                              // [nrg*G] maxima, then [nrg*G] sums, then [nrg*G] weights
+        const int npg = a.nrg * G;
+        const bool in_smem = 3 * npg <= VW * YHG * D;
+        if (in_smem) {
+          for (int idx = vtid; idx < npg; idx += VTH) {
+            const float2 ml = __ldcg(&a.part_ml[p0 + idx]);
+            mlm[idx] = ml.x;
+            mlm[npg + idx] = ml.y;
+          }
+          named_barrier_sync(3, VTH);
+          if (vtid < G) {
+            float M = -INFINITY, den = 0.f;
+            for (int p = 0; p < a.nrg; ++p) M = fmaxf(M, mlm[p * G + vtid]);
+            for (int p = 0; p < a.nrg; ++p) den = fmaf(fast_exp2(mlm[p * G + vtid] - M), mlm[npg + p * G + vtid], den);
+            const float inv = 1.f / den;
+            for (int p = 0; p < a.nrg; ++p) mlm[2 * npg + p * G + vtid] = fast_exp2(mlm[p * G + vtid] - M) * inv;
+          }
+          named_barrier_sync(3, VTH);
+          for (int idx = vtid; idx < G * D; idx += VTH) {
+            const int g = idx >> 7, col = idx & (D - 1);
+            const float* yp = a.part_y + (p0 + g) * D + col;
+            float num = 0.f;
+            int p = 0;
+            for (; p + 4 <= a.nrg; p += 4) {            // four independent loads in flight
+              const float y0 = __ldcg(yp + (size_t)(p + 0) * G * D), y1 = __ldcg(yp + (size_t)(p + 1) * G * D);
+              const float y2 = __ldcg(yp + (size_t)(p + 2) * G * D), y3 = __ldcg(yp + (size_t)(p + 3) * G * D);
+              num = fmaf(mlm[2 * npg + (p + 0) * G + g], y0, num);
+              num = fmaf(mlm[2 * npg + (p + 1) * G + g], y1, num);
+              num = fmaf(mlm[2 * npg + (p + 2) * G + g], y2, num);
+              num = fmaf(mlm[2 * npg + (p + 3) * G + g], y3, num);
+            }
+            for (; p < a.nrg; ++p) num = fmaf(mlm[2 * npg + p * G + g], __ldcg(yp + (size_t)p * G * D), num);
+            a.out[((size_t)b0 * a.H_kv * G + (size_t)h * G + g) * D + col] = __float2bfloat16_rn(num);
+          }
+        } else {
+          for (int idx = vtid; idx < G * D; idx += VTH) {
+            const int g = idx >> 7, col = idx & (D - 1);
+            float M = -INFINITY;
+            for (int p = 0; p < a.nrg; ++p) M = fmaxf(M, __ldcg(&a.part_ml[p0 + (size_t)p * G + g]).x);
+            float num = 0.f, den = 0.f;
+            for (int p = 0; p < a.nrg; ++p) {
+              const float2 ml = __ldcg(&a.part_ml[p0 + (size_t)p * G + g]);
+              const float w = fast_exp2(ml.x - M);
+              den = fmaf(w, ml.y, den);
+              num = fmaf(w, __ldcg(&a.part_y[(p0 + (size_t)p * G + g) * D + col]), num);
+            }
+            a.out[((size_t)b0 * a.H_kv * G + (size_t)h * G + g) * D + col] = __float2bfloat16_rn(num / den);
+          }
+        }
+      }
+      named_barrier_sync(3, VTH);
+    }
+  }
+  named_barrier_sync(BAR_END, (CW + 1) * 32);
+  if (dead && lane == 0) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------------------ host side
+FusedPlan plan_fused_tc(const kvc_layer* L, int B, int R) {
+  FusedPlan p{};
+  const int G = L->G, n = L->desc.n, m = L->m, H_kv = L->desc.H_kv;
+  if (L->desc.dtype != KVC_BF16 || L->passthrough || R < 1 || B < 1 || n % 64 != 0 || n > 1024 || G > 16) return p;
+  if (reinterpret_cast<uintptr_t>(L->desc.theta) & 15 || reinterpret_cast<uintptr_t>(L->desc.U) & 15) return p;
+  const int sms = L->num_sms > 0 ? L->num_sms : 148;
+  p.tc = 1;
+  p.EW = TEW;
+  p.VW = n <= 256 ? 8 : 10;
+  p.ktw = 0;
+  // the logits live in tensor memory: two row tiles per unit whenever a sequence has more than 16 expansion rows
+  p.MT = G * R > ROWS ? 2 : 1;
+  const int cap = ROWS * p.MT;
+  p.RB = R < cap / G ? R : cap / G;
+  p.NB = 1;
+  if (p.RB == R) {
+    // whole sequences per unit: more sequences per unit share one pass over theta[h] and U[h]
+    double best = 0;
+    for (int nb = 1; nb <= 4; nb *= 2) {
+      if (nb > 1 && (nb * R * G > cap || nb > B || p.VW % nb != 0)) break;
+      const long long units = (long long)H_kv * ceil_div(B, nb);
+      const double cost = (double)ceil_div((int)units, sms) * ((double)nb * R * m * 512.0 + 4.0 * m * n);
+      if (nb == 1 || cost < best) { best = cost; p.NB = nb; }
+    }
+  }
+  p.nbg = ceil_div(B, p.NB);
+  p.nrg = ceil_div(R, p.RB);
+  p.units = H_kv * p.nbg * p.nrg;
+  if (p.nrg > 1 && (long long)B * H_kv > KVC_MAX_COUNTERS) return p;
+  p.ncg = n / 64;
+  const uint32_t chunk = (uint32_t)p.NB * p.RB * 4096u + (uint32_t)n * 32u;
+  int jc = (int)(65536u / chunk);
+  const int jmax = ceil_div(m, 16) < 4 ? ceil_div(m, 16) : 4;          // at most 64 rows of U per stage: M of the re-projection MMA
+  p.JC = jc < 1 ? 1 : (jc > jmax ? jmax : jc);
+  p.NJ = ceil_div(m, 16 * p.JC);
+  p.par_bytes = (uint32_t)p.ncg * p.JC * 2048u;
+  p.k_half_bytes = (uint32_t)p.NB * p.RB * p.JC * 2048u;
+  p.stage_bytes = p.par_bytes + 2 * p.k_half_bytes;
+  int tch = (int)(p.stage_bytes / (p.NB * 512u)) & ~15;
+  p.TCH = tch > 256 ? 256 : tch;
+  if (p.TCH < 16) return p;
+  p.txt_half_bytes = (uint32_t)p.NB * p.TCH * 128u;
+  {
+    const int wpg = p.VW / p.NB;
+    int best = 1 << 30;
+    for (int sh = 3; sh >= 0; --sh) {            // sh = 3: one task per block
+      const int ms = 8 >> sh, cost = ceil_div(p.JC * p.RB * ms, wpg) * ((1 << sh) + 1);
+      if (cost < best) { best = cost; p.msplit = ms; p.mshift = sh; }
+    }
+  }
+  p.sld = 0;
+  const int rt = ROWS * p.MT;
+  p.yhg = G > 4 ? 8 : (G > 2 ? 4 : 2);
+  uint32_t off = 0;
+  auto take = [&](uint32_t bytes) { uint32_t o = off; off = (off + bytes + 127u) & ~127u; return o; };
+  // P (read by the MMAs of pass C) and the reduction buffer of the unit end (used after them) share one region that
+  // starts right after the ring, 1024-byte aligned
+  const uint32_t p_bytes = (uint32_t)rt * n * 2, yred_bytes = (uint32_t)p.VW * p.yhg * D * 4;
+  p.off_P = take(p_bytes > yred_bytes ? p_bytes : yred_bytes);
+  p.off_yred = p.off_P;
+  p.off_q = take((uint32_t)p.NB * 16 * QLD * 2);
+  p.off_S = take((uint32_t)(2 * p.JC * rt * 32 + 2 * p.JC * (rt + 16) * SLD * 2));
+  p.off_W = p.off_S + (uint32_t)(2 * p.JC * rt * 32);
+  p.off_wred = 0;
+  p.off_rstat = take((uint32_t)2 * TEW * rt * 4);
+  p.off_tstat = take((uint32_t)2 * p.VW * 16 * 4);
+  p.off_hstat = take((uint32_t)3 * p.NB * 16 * 4);
+  p.off_rtab = take((uint32_t)rt * 4);
+  p.misc_bytes = off;
+  const int nt = (n + 127) / 128;
+  int cols = 32;
+  while (cols < nt * rt + 2 * rt) cols *= 2;
+  p.tmem_cols = cols;
+  if (cols > 512) return p;
+  if (SMEM_LIMIT < 1024u + 2048u + p.misc_bytes + 2 * p.stage_bytes) return p;
+  const uint32_t avail = SMEM_LIMIT - 1024u - 2048u - p.misc_bytes;   // alignment slack; static shared memory and its padding
+  int stages = (int)(avail / p.stage_bytes);
+  p.stages = stages > FMAX_STAGES ? FMAX_STAGES : stages;
+  if (p.stages < 2) return p;
+  p.smem_bytes = (size_t)p.stages * p.stage_bytes + p.misc_bytes + 1024u;
+  p.grid = p.units < sms ? p.units : sms;
+  p.ok = 1;
+  return p;
+}
+
+template <int VW, int NH, int MT>
+static cudaError_t launch_tc_inst(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
+  static size_t configured = 0;
+  if (p.smem_bytes > configured) {
+    cudaError_t e = cudaFuncSetAttribute(fused_decode_tc_kernel<VW, NH, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
+    if (e != cudaSuccess) return e;
+    configured = p.smem_bytes;
+  }
+  return launch_dependent(fused_decode_tc_kernel<VW, NH, MT>, dim3(p.grid), dim3((TEW + VW + 2) * 32), p.smem_bytes, st, tm[0], tm[1],
+                          tm[2], tm[3], tm[4], tm[5], fa);
+}
+
+template <int NH>
+static cudaError_t launch_tc_nh(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
+  if (p.VW == 8) return p.MT == 2 ? launch_tc_inst<8, NH, 2>(tm, fa, p, st) : launch_tc_inst<8, NH, 1>(tm, fa, p, st);
+  return p.MT == 2 ? launch_tc_inst<10, NH, 2>(tm, fa, p, st) : launch_tc_inst<10, NH, 1>(tm, fa, p, st);
+}
+
+cudaError_t launch_fused_tc_kernel(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
+  return fa.G > 8 ? launch_tc_nh<2>(tm, fa, p, st) : launch_tc_nh<1>(tm, fa, p, st);
+}
+
+}  // namespace kvc

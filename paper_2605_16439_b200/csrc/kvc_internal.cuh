@@ -92,6 +92,9 @@ struct FusedPlan {
   int stages, grid;
   uint32_t par_bytes, k_half_bytes, txt_half_bytes, stage_bytes, misc_bytes;
   uint32_t off_q, off_S, off_W, off_wred, off_rstat, off_tstat, off_hstat, off_yred;   // relative to the end of the ring
+  int tc;            // 1: the expansions run on tcgen05 with the logits in tensor memory (kvc_fused_tc.cu)
+  uint32_t off_P, off_rtab;
+  int tmem_cols;
   size_t smem_bytes;
 };
 
@@ -105,6 +108,7 @@ struct kvc_layer {
   int passthrough;       // ratio_permille == 0
   int device;
   int num_sms;
+  int use_tc;            // 1: expansions of the one-kernel decode path on tcgen05 (environment KVC_EXPANSION=tcgen05 at creation)
   int32_t* d_idx;        // device [H_kv][m]
   int* d_cnt;            // device [KVC_MAX_COUNTERS + 1] arrival counters of the one-kernel decode path (zero between
                          // calls), then the status word of the compress kernels
@@ -116,6 +120,7 @@ namespace kvc {
 WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap);
 int cuda_status(cudaError_t e);   // KVC_OK or KVC_ERR_CUDA, remembering the error for kvc_last_cuda_error
 FusedPlan plan_fused(const kvc_layer* L, int B, int R);
+FusedPlan plan_fused_tc(const kvc_layer* L, int B, int R);     // tensor-memory variant; ok == 0 if the shape does not fit it
 FusedPlan plan_fused_text(const kvc_layer* L, int B, int T);   // R == 0: text rows only
 
 struct DecodeArgs {

@@ -79,6 +79,7 @@ const char* kvc_kernel_name(int kernel_id) {
     case KVC_KERNEL_MERGE: return "merge";
     case KVC_KERNEL_COMBINE: return "combine";
     case KVC_KERNEL_FUSED: return "fused";
+    case KVC_KERNEL_FUSED_TC: return "fused_tc";
     default: return "?";
   }
 }

@@ -1,0 +1,87 @@
+// 5th-generation tensor core (tcgen05) helpers for sm_100a: tensor-memory allocation, shared-memory matrix
+// descriptors, the instruction descriptor of kind::f16 (bf16 operands, fp32 accumulation in tensor memory),
+// MMA issue, commit to an mbarrier, and tensor-memory loads.
+//
+// Operand layouts in shared memory (16-bit elements), all tile bases 1024-byte aligned when swizzled:
+//   K-major,  128-byte swizzle: rows of 64 elements (128 B) along K; 8 rows form a 1024-byte atom; SBO = byte
+//             distance between 8-row groups; a K step of 16 elements advances the start address by 32 B.
+//   MN-major, 128-byte swizzle: rows of 64 elements along M (or N), one row per k; 8 k-rows form an atom;
+//             LBO = byte distance between 64-element groups along M/N, SBO = between 8-row groups along K.
+//   K-major, no swizzle: 8 rows x 16 B core matrices; SBO = distance between 8-row groups, LBO = between the
+//             two 8-element halves of a K step.
+// This is the layout the TMA engine produces for a {64, rows} box with CU_TENSOR_MAP_SWIZZLE_128B.
+// Accumulator layout in tensor memory: M = 128: row i <-> lane i; M = 64: row i <-> lane (i % 16) + 32 (i / 16);
+// column j of the tile <-> column base + j (fp32).
+#pragma once
+
+#include <stdint.h>
+
+#include "kvc_async.cuh"
+
+namespace kvc {
+
+constexpr uint32_t UMMA_LAYOUT_NONE = 0, UMMA_LAYOUT_SW128 = 2;
+
+__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFFu);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1 << 46;                    // descriptor version of this architecture
+  d |= (uint64_t)layout << 61;
+  return d;
+}
+// kind::f16 instruction descriptor: D fp32, A and B bf16; a_mn / b_mn = 1 for an MN-major operand
+__device__ __forceinline__ uint32_t umma_idesc_bf16(int M, int N, int a_mn, int b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+         ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+// D[tmem] (+)= A[smem] B[smem]; issued by ONE thread; accumulate == 0 overwrites D
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// the mbarrier receives one arrival when every MMA issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+
+// whole warp; cols a power of two in [32, 512]; the base address lands in *dst (shared memory)
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_addr(dst)), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t base, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(base), "r"(cols) : "memory");
+}
+
+// whole warp: lane l receives columns [col, col + N) of tensor-memory lane (quarter of the warp) * 32 + l
+__device__ __forceinline__ void tmem_ld_x16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+template <int N>
+__device__ __forceinline__ void tmem_ld(uint32_t taddr, float (&v)[N]) {
+  static_assert(N % 16 == 0, "columns per load");
+#pragma unroll
+  for (int c = 0; c < N; c += 16) {
+    float t[16];
+    tmem_ld_x16(taddr + (uint32_t)c, t);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[c + i] = t[i];
+  }
+}
+
+}  // namespace kvc

@@ -268,6 +268,25 @@ def test_one_kernel_path_edges(B, H_q, H_kv, grid, R, T):
     _check(shape, p)
 
 
+@pytest.mark.parametrize("B,H_q,H_kv,grid,R,T", [
+    (3, 2, 2, 8, 5, 1),        # two sequences per unit, odd batch, one text row
+    (1, 7, 1, 8, 5, 700),      # G = 7: two row tiles of expansion rows, units split the block axis
+    (2, 14, 2, 16, 3, 33),     # n = 256
+    (5, 4, 4, 24, 2, 130),     # n = 576: last tile of the transposed logits has 64 rows
+    (1, 16, 1, 8, 3, 20),      # G = 16: two head tiles
+    (1, 12, 2, 32, 2, 64),     # n = 1024: eight logit tiles in tensor memory
+    (40, 8, 8, 8, 2, 37),      # more units than SMs: accumulators and barriers reused across units
+])
+def test_tensor_memory_variant_of_the_expansions(B, H_q, H_kv, grid, R, T, monkeypatch):
+    """The opt-in variant that runs Alg. 1 steps 2-3 on tcgen05 with the logits in tensor memory (chosen when the
+    layer is created with KVC_EXPANSION=tcgen05 in the environment) against the oracle."""
+    monkeypatch.setenv("KVC_EXPANSION", "tcgen05")
+    shape = wl.Shape("tc-variant", 1, B, H_q, H_kv, 128, grid, R, T, 1, "bf16")
+    p = tl.make_problem(shape, 170 + B + 7 * R + T, T=T, T_cap=T + 5)
+    counts = _fused_launches(lambda: _check(shape, p))
+    assert counts["fused_tc"] >= 1 and counts["fused"] == 0 and counts["scores"] == 0
+
+
 def test_more_units_than_sms_and_status_word_clean():
     """Persistent CTAs walk several work units each (ring parity carried across units)."""
     shape = wl.Shape("many-units", 1, 40, 8, 8, 128, 8, 2, 37, 1, "bf16")      # 8 * 40 = 320 units of one sequence
