@@ -81,9 +81,9 @@ KVC_API int kvc_retained_len(int n, int ratio_permille);
  * unchanged while the handle is in use.  ratio_permille == 0 is the pass-through limit: m = n,
  * capsules hold K and V verbatim, idx / theta / U / mu are ignored.
  * The device that is current at this call must be current for every later call with the handle.
- * If the environment variable KVC_EXPANSION is "tcgen05" when the handle is created, bf16 decode calls
- * of this handle run Alg. 1 steps 2-3 on the tcgen05 tensor cores with the logits in tensor memory
- * (same results within the bf16 tolerance; slower than the default at the shapes measured so far). */
+ * bf16 decode calls run Alg. 1 steps 2-3 either on mma.sync with the logits in registers or on tcgen05 with the
+ * logits in tensor memory; the library picks per shape (same results within the bf16 tolerance).  The environment
+ * variable KVC_EXPANSION = "tcgen05" | "mma", read when the handle is created, forces one of them where it applies. */
 KVC_API int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out);
 KVC_API int kvc_layer_destroy(kvc_layer* layer);
 
@@ -182,7 +182,7 @@ typedef enum {
   KVC_KERNEL_MERGE = 5,           /* log-sum-exp merge of partials */
   KVC_KERNEL_COMBINE = 6,         /* n-split partials of Alg. 1 step 3 combined per row */
   KVC_KERNEL_FUSED = 7,           /* Alg. 1 steps 1-4 + text + normalisation in one kernel (bf16) */
-  KVC_KERNEL_FUSED_TC = 8,        /* the same kernel with steps 2-3 on tcgen05 / tensor memory (opt-in, see kvc_layer_create) */
+  KVC_KERNEL_FUSED_TC = 8,        /* the same kernel with steps 2-3 on tcgen05 / tensor memory (see kvc_layer_create) */
   KVC_KERNEL_COUNT = 9
 } kvc_kernel_id;
 KVC_API int kvc_profile_start(int max_launches);

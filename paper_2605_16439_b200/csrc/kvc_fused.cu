@@ -139,7 +139,11 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   uint32_t slot = 0, phase = 0;
   uint32_t si = 0, wi = 0;                         // score tiles and weight tiles handed over so far (buffer = count & 1)
   bool dead = false;
-  auto wait_on = [&](uint64_t* bar, uint32_t parity) { if (!dead && !mbar_wait_bounded(bar, parity)) dead = true; };
+  // every lane of the calling warp waits; the lanes leave the polling loop together again before any warp-wide instruction
+  auto wait_on = [&](uint64_t* bar, uint32_t parity) {
+    if (!dead && !mbar_wait_bounded(bar, parity)) dead = true;
+    __syncwarp();
+  };
   // the stage in `slot` has been consumed by this warp
   auto release = [&]() {
     __syncwarp();
@@ -772,9 +776,12 @@ static void warp_split(int n, int* ew, int* vw, int* ktw_max) {
 }
 
 FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
-  if (L->use_tc) {
+  if (L->use_tc >= 0) {
+    // The tensor-memory variant pays per tcgen05.mma, not per expansion row: it wins for long blocks once two row
+    // tiles per unit still give most SMs a unit (measured on the n = 1024, G = 7 shape: ahead from batch 16 on,
+    // behind at batches 1-4 where units of half the size halve the latency).
     const FusedPlan t = plan_fused_tc(L, B, R);
-    if (t.ok) return t;
+    if (t.ok && (L->use_tc > 0 || (L->desc.n > 640 && t.MT == 2 && t.units >= 96))) return t;
   }
   FusedPlan p{};
   const int G = L->G, n = L->desc.n, m = L->m, H_kv = L->desc.H_kv;
@@ -957,8 +964,9 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
     const uint64_t dims[4] = {64ull, (uint64_t)m, (uint64_t)p.ncg, (uint64_t)H_kv};
     const uint64_t str[3] = {(uint64_t)n * 2, 128ull, (uint64_t)m * n * 2};
     const uint32_t box[4] = {64u, (uint32_t)(16 * p.JC), (uint32_t)p.ncg, 1u};
+    const uint32_t box_tc[4] = {64u, 128u, 1u, 1u};     // tensor-memory variant: U by 64-column groups, 128 rows at a time
     if (!encode_tensor_map_bf16(&tm[4], a.theta, 4, dims, str, box)) return cudaSuccess;
-    if (!encode_tensor_map_bf16(&tm[5], a.U, 4, dims, str, box)) return cudaSuccess;
+    if (!encode_tensor_map_bf16(&tm[5], a.U, 4, dims, str, p.tc ? box_tc : box)) return cudaSuccess;
   }
   *encoded = true;
 
@@ -979,7 +987,7 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
   fa.off_q = ring + p.off_q; fa.off_S = ring + p.off_S; fa.off_W = ring + p.off_W; fa.off_wred = ring + p.off_wred;
   fa.off_rstat = ring + p.off_rstat; fa.off_tstat = ring + p.off_tstat; fa.off_hstat = ring + p.off_hstat;
   fa.off_yred = ring + p.off_yred;
-  fa.off_P = ring + p.off_P; fa.off_rtab = ring + p.off_rtab; fa.tmem_cols = p.tmem_cols;
+  fa.off_P = ring + p.off_P; fa.off_rtab = ring + p.off_rtab; fa.tmem_cols = p.tmem_cols; fa.UT = p.UT; fa.nu = p.nu;
   fa.part_y = a.fpart_y;
   fa.part_ml = a.fpart_ml;
   fa.cnt = L->d_cnt;

@@ -27,14 +27,39 @@ constexpr int TEW = 4;                         // softmax / conversion warps: on
 constexpr int BAR_P_READY = 12;                // probabilities written (warps 0-3 arrive, the MMA warp waits)
 constexpr int BAR_END = 13;                    // every tensor-memory user is done: the MMA warp may free it
 
+// Order of the stages between pass A and the V_tilde stages: `nu` stages of U (tensor core) and `nts` text stages
+// (value warps).  The first TEXT_LEAD text stages go first, because the re-projection cannot start before the softmax
+// is done; after that the two kinds alternate.  (iu, it) = stages of either kind issued so far.
+constexpr int TEXT_LEAD = 3;
+__device__ __forceinline__ bool next_is_text(int iu, int it, int nu, int nts) {
+  return it < nts && (it < TEXT_LEAD || iu >= nu || it - TEXT_LEAD < iu);
+}
+
 struct TcBars {
   uint64_t full[FMAX_STAGES], empty[FMAX_STAGES];
   uint64_t s_free[2];      // the MMAs that read score tile b have completed
-  uint64_t w_done[2];      // W^T of a stage is complete in accumulator b
-  uint64_t w_tfree[2];     // accumulator b has been read back (4 warps)
+  uint64_t w_done;         // W^T of the unit is complete
   uint64_t l_done;         // the logits of the unit are complete
   uint64_t l_free;         // the logits of the unit have been read back (4 warps)
 };
+
+// Reduces 16 per-lane values over the 32 lanes of a warp (maximum or sum) in 31 shuffles: after the first exchange
+// every step halves the rows a lane keeps; lane l (and l + 16) returns the total of row l & 15.
+template <bool IS_MAX>
+__device__ __forceinline__ float lane_reduce16(float (&x)[16], int lane) {
+  auto op = [](float p, float q) { return IS_MAX ? fmaxf(p, q) : p + q; };
+#pragma unroll
+  for (int r = 0; r < 16; ++r) x[r] = op(x[r], __shfl_xor_sync(0xffffffffu, x[r], 16));
+  float y8[8], y4[4], y2[2];
+  const bool u8 = lane & 8, u4 = lane & 4, u2 = lane & 2, u1 = lane & 1;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) y8[k] = op(u8 ? x[8 + k] : x[k], __shfl_xor_sync(0xffffffffu, u8 ? x[k] : x[8 + k], 8));
+#pragma unroll
+  for (int k = 0; k < 4; ++k) y4[k] = op(u4 ? y8[4 + k] : y8[k], __shfl_xor_sync(0xffffffffu, u4 ? y8[k] : y8[4 + k], 4));
+#pragma unroll
+  for (int k = 0; k < 2; ++k) y2[k] = op(u2 ? y4[2 + k] : y4[k], __shfl_xor_sync(0xffffffffu, u2 ? y4[k] : y4[2 + k], 2));
+  return op(u1 ? y2[1] : y2[0], __shfl_xor_sync(0xffffffffu, u1 ? y2[0] : y2[1], 1));
+}
 
 template <int VW, int NH, int MT>
 __global__ void __launch_bounds__((TEW + VW + 2) * 32, 1)
@@ -57,7 +82,8 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     for (int s = 0; s < a.stages; ++s) { mbar_init(&bars.full[s], 1); mbar_init(&bars.empty[s], VW + 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&bars.s_free[b], 1); mbar_init(&bars.w_done[b], 1); mbar_init(&bars.w_tfree[b], TEW); }
+    for (int b = 0; b < 2; ++b) mbar_init(&bars.s_free[b], 1);
+    mbar_init(&bars.w_done, 1);
     mbar_init(&bars.l_done, 1);
     mbar_init(&bars.l_free, TEW);
     fence_mbar_init();
@@ -65,19 +91,20 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   if (warp == MMA_WARP) tmem_alloc(&s_tmem, (uint32_t)a.tmem_cols);
   const int JC = a.JC;
   const uint32_t s_buf_bytes = (uint32_t)(JC * RT * 32);            // score tile buffer: [JC][2 halves][RT/8][8][8]
-  const int w_buf_elems = JC * (RT + 16) * SLD;                      // weight tile buffer: [JC][RT + 16][SLD]
-  // score and weight tiles start as zeros: their padding rows and columns are read by the MMAs
+  // score tiles start as zeros: the rows of absent (sequence, block, head) triples are read by the MMAs
   {
     uint32_t* z = reinterpret_cast<uint32_t*>(sm + a.off_S);
-    const int words = (int)(2 * s_buf_bytes) / 4 + w_buf_elems;      // 2 score buffers (bytes / 4) + 2 weight buffers (elements / 2)
+    const int words = (int)(2 * s_buf_bytes) / 4;
     for (int i = tid; i < words; i += FTHREADS) z[i] = 0u;
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tb = s_tmem;                  // tensor memory: L^T tiles at columns [0, NT*RT), W^T buffers after them
+  const uint32_t tb = s_tmem;                  // tensor memory: L^T tiles at columns [0, NT*RT), W^T tiles after them
   const int NT = (a.n + 127) >> 7;
+  const int MTL = (a.m + 127) >> 7;            // 128-row tiles of W^T (rows of U)
   const uint32_t w_col = (uint32_t)(NT * RT);
+  const int ugroups = (MTL + a.UT - 1) / a.UT; // stages per 64-column group of U: UT row tiles each
 
   const int per_h = a.nbg * a.nrg;
   const int rows16 = 16 * JC;                      // rows of one block inside a stage
@@ -96,29 +123,43 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       const int b0 = bg * a.NB, r0 = rg * a.RB;
       const RowRanges tr = row_ranges(a, rg);
       const int nts = tr.na + tr.nb;
+      // stage sequence of a unit: NJ stages of pass A (theta rows + K_tilde rows); then the column groups of U and
+      // the text stages, interleaved so that the tensor core (U) and the value warps (text) both have work; then
+      // NJ stages of V_tilde rows
       for (int part = 0; part < 3; ++part) {
-        const int count = part == 1 ? nts : a.NJ;
-        for (int c = 0; c < count; ++c) {
+        const int count = part == 1 ? a.nu + nts : a.NJ;
+        int iu = 0, it = 0;
+        for (int cc = 0; cc < count; ++cc) {
+          const bool is_text = part == 1 && next_is_text(iu, it, a.nu, nts);
+          const int c = part == 1 ? (is_text ? it++ : iu++) : cc;
           if (!mbar_wait_bounded(&bars.empty[slot], phase)) { atomicExch(a.status, (int)KVC_ERR_TIMEOUT); return; }
           unsigned char* dst = sm + slot * a.stage_bytes;
           uint64_t* bar = &bars.full[slot];
-          if (part == 1) {
+          if (is_text) {
             const int y = tr.b0 + c * a.TCH;
             mbar_expect_tx(bar, 4 * a.txt_half_bytes);
-            if (first) { grid_dep_wait(); first = false; }
             tma_load_4d(dst, &tmKt, 0, y, h, b0, bar);
             tma_load_4d(dst + a.txt_half_bytes, &tmKt, 64, y, h, b0, bar);
             tma_load_4d(dst + 2 * a.txt_half_bytes, &tmVt, 0, y, h, b0, bar);
             tma_load_4d(dst + 3 * a.txt_half_bytes, &tmVt, 64, y, h, b0, bar);
-          } else {
-            const CUtensorMap* tp = part == 0 ? &tmTh : &tmU;
-            const CUtensorMap* tk = part == 0 ? &tmK : &tmV;
+          } else if (part == 1) {
+            // 64 columns of U[h], row tiles [t0, t0 + nt_) of 128 rows each (rows past m are zero-filled)
+            const int cg = c / ugroups, t0 = (c - cg * ugroups) * a.UT;
+            const int nt_ = min(a.UT, MTL - t0);
+            mbar_expect_tx(bar, (uint32_t)nt_ * 16384u);
+            for (int t = 0; t < nt_; ++t) tma_load_4d(dst + t * 16384, &tmU, 0, (t0 + t) * 128, cg, h, bar);
+          } else if (part == 0) {
             const int j0 = c * rows16;
             mbar_expect_tx(bar, a.par_bytes + 2 * a.k_half_bytes);
-            tma_load_4d(dst, tp, 0, j0, 0, h, bar);                  // parameters: never written by this library
+            tma_load_4d(dst, &tmTh, 0, j0, 0, h, bar);               // parameters: never written by this library
             if (first) { grid_dep_wait(); first = false; }            // everything else may come from the stream's previous kernel
-            tma_load_5d(dst + a.par_bytes, tk, 0, j0, r0, h, b0, bar);
-            tma_load_5d(dst + a.par_bytes + a.k_half_bytes, tk, 64, j0, r0, h, b0, bar);
+            tma_load_5d(dst + a.par_bytes, &tmK, 0, j0, r0, h, b0, bar);
+            tma_load_5d(dst + a.par_bytes + a.k_half_bytes, &tmK, 64, j0, r0, h, b0, bar);
+          } else {
+            const int j0 = c * rows16;
+            mbar_expect_tx(bar, 2 * a.k_half_bytes);
+            tma_load_5d(dst + a.par_bytes, &tmV, 0, j0, r0, h, b0, bar);
+            tma_load_5d(dst + a.par_bytes + a.k_half_bytes, &tmV, 64, j0, r0, h, b0, bar);
           }
           if (++slot == (uint32_t)a.stages) { slot = 0; phase ^= 1u; }
         }
@@ -132,10 +173,14 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   if (blockIdx.x == 0 && tid == 0) *a.status = 0;
 
   uint32_t slot = 0, phase = 0;
-  uint32_t si = 0, wi = 0;                         // score tiles and weight tiles (one per stage) handed over so far
+  uint32_t si = 0;                                 // score tiles handed over so far (buffer = si & 1)
   uint32_t ucount = 0;                             // units this CTA has started
   bool dead = false;
-  auto wait_on = [&](uint64_t* bar, uint32_t parity) { if (!dead && !mbar_wait_bounded(bar, parity)) dead = true; };
+  // every lane of the calling warp waits; the lanes leave the polling loop together again before any warp-wide instruction
+  auto wait_on = [&](uint64_t* bar, uint32_t parity) {
+    if (!dead && !mbar_wait_bounded(bar, parity)) dead = true;
+    __syncwarp();
+  };
   auto advance = [&]() { if (++slot == (uint32_t)a.stages) { slot = 0; phase ^= 1u; } };
 
   if (warp == MMA_WARP) {
@@ -146,7 +191,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     const uint32_t cg_bytes = (uint32_t)rows16 * 128u;            // one 64-column group of a parameter tile
     const uint32_t idesc_L_full = umma_idesc_bf16(128, RT, 1, 0);
     const uint32_t idesc_L_half = umma_idesc_bf16(64, RT, 1, 0);
-    const uint32_t idesc_W = umma_idesc_bf16(64, RT, 0, 0);
+    const uint32_t idesc_W = umma_idesc_bf16(128, RT, 0, 0);
     const bool half_tail = (a.n & 127) != 0;                      // n = 64 (mod 128): the last tile of L^T has 64 rows
     for (int u = blockIdx.x; u < a.units; u += gridDim.x, ++ucount) {
       const int rem = u % per_h;
@@ -178,33 +223,40 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         ++si;
         advance();
       }
-      // ---------------- text stages belong to the value warps ----------------
-      for (int ts = 0; ts < nts; ++ts) {
-        wait_on(&bars.full[slot], phase);
-        if (lane == 0) mbar_arrive(&bars.empty[slot]);
-        advance();
+      // ---------------- W^T[m x rows] = U P^T: one stage = 64 columns of U, UT row tiles; text stages pass by ----------------
+      for (int iu = 0, it = 0; iu + it < a.nu + nts;) {
+        if (!next_is_text(iu, it, a.nu, nts)) {
+          const int i = iu++;
+          wait_on(&bars.full[slot], phase);
+          if (i == 0) named_barrier_sync(BAR_P_READY, TEW * 32 + 32);    // the probabilities of the unit are in shared memory
+          tc_fence_after();
+          if (lane == 0) {
+            const uint32_t par_u = sm_u + slot * a.stage_bytes;
+            const int cg = i / ugroups, t0 = (i - cg * ugroups) * a.UT;
+            const int nt_ = min(a.UT, MTL - t0);
+            for (int t = 0; t < nt_; ++t)
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk) {
+                const uint64_t adesc = umma_smem_desc(par_u + (uint32_t)(t * 16384 + kk * 32), 16u, 1024u, UMMA_LAYOUT_SW128);
+                const uint64_t bdesc = umma_smem_desc(P_u + (uint32_t)(cg * RT * 128 + kk * 32), 16u, 1024u, UMMA_LAYOUT_SW128);
+                umma_bf16(tb + w_col + (uint32_t)((t0 + t) * RT), adesc, bdesc, idesc_W, (cg | kk) ? 1u : 0u);
+              }
+            umma_commit(&bars.empty[slot]);
+            if (i == a.nu - 1) umma_commit(&bars.w_done);
+          }
+          __syncwarp();
+          advance();
+        } else {
+          ++it;
+          wait_on(&bars.full[slot], phase);
+          if (lane == 0) mbar_arrive(&bars.empty[slot]);
+          advance();
+        }
       }
-      // ---------------- pass C ----------------
-      named_barrier_sync(BAR_P_READY, TEW * 32 + 32);
+      // ---------------- the V_tilde stages belong to the value warps ----------------
       for (int c = 0; c < a.NJ; ++c) {
         wait_on(&bars.full[slot], phase);
-        const uint32_t wbuf = wi & 1u;
-        if (wi >= 2) wait_on(&bars.w_tfree[wbuf], ((wi >> 1) - 1) & 1u);
-        tc_fence_after();
-        if (lane == 0) {
-          const uint32_t par_u = sm_u + slot * a.stage_bytes;
-          for (int cg = 0; cg < a.ncg; ++cg)
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-              const uint64_t adesc = umma_smem_desc(par_u + (uint32_t)cg * cg_bytes + (uint32_t)(kk * 32), 16u, 1024u, UMMA_LAYOUT_SW128);
-              const uint64_t bdesc = umma_smem_desc(P_u + (uint32_t)(cg * RT * 128 + kk * 32), 16u, 1024u, UMMA_LAYOUT_SW128);
-              umma_bf16(tb + w_col + wbuf * RT, adesc, bdesc, idesc_W, (cg | kk) ? 1u : 0u);
-            }
-          umma_commit(&bars.w_done[wbuf]);
-          umma_commit(&bars.empty[slot]);
-        }
-        __syncwarp();
-        ++wi;
+        if (lane == 0) mbar_arrive(&bars.empty[slot]);
         advance();
       }
     }
@@ -221,7 +273,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   const uint32_t q_u = sm_u + a.off_q, W_u = sm_u + a.off_W;
   __nv_bfloat16* q_sm = reinterpret_cast<__nv_bfloat16*>(sm + a.off_q);
   unsigned char* S_sm = sm + a.off_S;                                        // [2][JC][2][RT/8][8][8] bf16
-  __nv_bfloat16* W_sm = reinterpret_cast<__nv_bfloat16*>(sm + a.off_W);      // [2][JC][RT + 16][SLD]
+  __nv_bfloat16* W_sm = reinterpret_cast<__nv_bfloat16*>(sm + a.off_W);      // [ceil(m/16)][RT + 16][SLD]; shares its region with P
   float* rmax = reinterpret_cast<float*>(sm + a.off_rstat);                  // [TEW][RT]
   float* rsum = rmax + TEW * RT;
   float* tmax = reinterpret_cast<float*>(sm + a.off_tstat);                  // [VW][16]
@@ -229,6 +281,8 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   float* hmax = reinterpret_cast<float*>(sm + a.off_hstat);                  // [NB][16]
   float* hsum = hmax + a.NB * 16;
   float* vsum = hsum + a.NB * 16;
+  float* hvmax = vsum + a.NB * 16;                                           // maximum over the vision logits only
+  float* hfv = hvmax + a.NB * 16;                                            // 2^(hvmax - hmax): moves the vision weights to the joint maximum
   int* rtab = reinterpret_cast<int*>(sm + a.off_rtab);                       // [RT] head slot of an expansion row, -1 if unused
   float* yred = reinterpret_cast<float*>(sm + a.off_yred);                   // [VW][yhg][D]
   const float qscale = 0.08838834764831845f * 1.4426950408889634f;   // sigma = 1/sqrt(128), logits kept in log2 units
@@ -253,46 +307,45 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       const int nbv = min(a.NB, a.B - b0);
       const int rbv = min(RB, a.R - r0);
       (void)h;
-      // expansion row rho <-> (sequence, block, head); this lane's own row for the statistics: rho = lane
-      bool my_valid = false;
-      {
-        const int rho = lane;
+      named_barrier_sync(2, TEW * 32);           // every warp is done with the previous unit's tables
+      // expansion row rho <-> (sequence, block, head): head slot of the row, -1 if the unit has no such row
+      auto row_slot = [&](int rho) {
         const int bi = rho / G, g = rho - bi * G;
         const int rbl = bi / RB, rrl = bi - rbl * RB;
-        my_valid = rho < RT && rho < a.NB * RB * G && rbl < nbv && rrl < rbv;
-        if (warp == 0 && rho < RT) rtab[rho] = my_valid ? rbl * 16 + g : -1;
-      }
+        return (rho < a.NB * RB * G && rbl < nbv && rrl < rbv) ? rbl * 16 + g : -1;
+      };
+      if (warp == 0)
+        for (int x = lane; x < RT; x += 32) rtab[x] = row_slot(x);
 
-      // ---------------- maxima of the logits ----------------
+      // ---------------- maxima of the logits, 16 expansion rows (one tensor-memory load) at a time ----------------
       wait_on(&bars.l_done, ucount & 1u);
-      __syncwarp();
       tc_fence_after();
-      float mx[RT];
 #pragma unroll
-      for (int r = 0; r < RT; ++r) mx[r] = -INFINITY;
-      for (int t = 0; t < NT; ++t) {
-        float v[RT];
+      for (int hh = 0; hh < MT; ++hh) {
+        float mx[16];
+#pragma unroll
+        for (int r = 0; r < 16; ++r) mx[r] = -INFINITY;
+        uint32_t nx[16];
         __syncwarp();
-        tmem_ld<RT>(tq + (uint32_t)(t * RT), v);
-        const bool lane_ok = !(half_tail && t == NT - 1) || lane < 16;
-        if (lane_ok) {
+        tmem_ld_issue_x16(tq + (uint32_t)(hh * 16), nx);
+        for (int t = 0; t < NT; ++t) {
+          float v[16];
+          tmem_ld_wait_x16(nx);
 #pragma unroll
-          for (int r = 0; r < RT; ++r) mx[r] = fmaxf(mx[r], v[r]);
+          for (int r = 0; r < 16; ++r) v[r] = __uint_as_float(nx[r]);
+          if (t + 1 < NT) tmem_ld_issue_x16(tq + (uint32_t)((t + 1) * RT + hh * 16), nx);   // in flight while tile t is reduced
+          if (!(half_tail && t == NT - 1) || lane < 16) {
+#pragma unroll
+            for (int r = 0; r < 16; ++r) mx[r] = fmaxf(mx[r], v[r]);
+          }
         }
+        const float mine = lane_reduce16<true>(mx, lane);            // row hh*16 + (lane & 15)
+        if (lane < 16) rmax[warp * RT + hh * 16 + lane] = row_slot(hh * 16 + lane) >= 0 ? mine : -INFINITY;
       }
-      {
-        float mine = -INFINITY;
-#pragma unroll
-        for (int r = 0; r < RT; ++r) {
-          float x = mx[r];
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
-          if (lane == r) mine = x;
-        }
-        if (lane < RT) rmax[warp * RT + lane] = my_valid ? mine : -INFINITY;
-      }
-      named_barrier_sync(1, FCONS);                                   // B1: row maxima and text maxima are in place
+      named_barrier_sync(2, TEW * 32);
       if (warp == 0) {
+        // maximum of every expansion row over the warps, then of every (sequence, head) over its blocks: the softmax of
+        // the vision logits is taken relative to it, the text rows join at the unit's weight hand-over
         for (int x = lane; x < RT; x += 32) {
           float m_ = -INFINITY;
 #pragma unroll
@@ -306,59 +359,55 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
           if (g < G && tb_ < nbv) {
             m_ = -INFINITY;
             for (int rl = 0; rl < rbv; ++rl) m_ = fmaxf(m_, rmax[(tb_ * RB + rl) * G + g]);
-            for (int w = tb_ * WPG; w < (tb_ + 1) * WPG; ++w) m_ = fmaxf(m_, tmax[w * 16 + g]);
           }
-          hmax[x] = m_;
+          hvmax[x] = m_;
         }
       }
-      named_barrier_sync(1, FCONS);                                   // B2: head maxima
+      named_barrier_sync(2, TEW * 32);
 
       // ---------------- P = 2^(L - max) as the bf16 operand of the re-projection; row sums ----------------
-      float Mr[RT];
-      uint32_t vmask = 0;
 #pragma unroll
-      for (int r = 0; r < RT; ++r) {
-        const int slot_ = rtab[r];
-        Mr[r] = slot_ >= 0 ? hmax[slot_] : 0.f;
-        vmask |= slot_ >= 0 ? (1u << r) : 0u;
-      }
-      float sum[RT];
+      for (int hh = 0; hh < MT; ++hh) {
+        float Mr[16], sum[16];                        // rows without a (sequence, block, head) get the reference +inf: P = 0
 #pragma unroll
-      for (int r = 0; r < RT; ++r) sum[r] = 0.f;
-      for (int t = 0; t < NT; ++t) {
-        float v[RT];
+        for (int r = 0; r < 16; ++r) {
+          const int slot_ = rtab[hh * 16 + r];
+          Mr[r] = slot_ >= 0 ? hvmax[slot_] : INFINITY;
+          sum[r] = 0.f;
+        }
+        uint32_t nx[16];
         __syncwarp();
-        tmem_ld<RT>(tq + (uint32_t)(t * RT), v);
-        const bool tail = half_tail && t == NT - 1;
-        const bool lane_ok = !tail || lane < 16;
-        const int i = t * 128 + (tail ? warp * 16 : warp * 32) + lane;          // column of L = row of L^T
-        const uint32_t cgo = (uint32_t)((i >> 6) * (RT * 128)), c8 = (uint32_t)((i & 63) >> 3), cl = (uint32_t)((i & 7) * 2);
-        if (lane_ok) {
+        tmem_ld_issue_x16(tq + (uint32_t)(hh * 16), nx);
+        for (int t = 0; t < NT; ++t) {
+          float v[16];
+          tmem_ld_wait_x16(nx);
 #pragma unroll
-          for (int r = 0; r < RT; ++r) {
-            const float p = (vmask >> r & 1u) ? fast_exp2(v[r] - Mr[r]) : 0.f;
-            sum[r] += p;
-            *reinterpret_cast<__nv_bfloat16*>(P_sm + cgo + (uint32_t)(r * 128) + ((c8 ^ (uint32_t)(r & 7)) << 4) + cl) = __float2bfloat16_rn(p);
+          for (int r = 0; r < 16; ++r) v[r] = __uint_as_float(nx[r]);
+          if (t + 1 < NT) tmem_ld_issue_x16(tq + (uint32_t)((t + 1) * RT + hh * 16), nx);   // in flight while tile t is processed
+          const bool tail = half_tail && t == NT - 1;
+          const bool lane_ok = !tail || lane < 16;
+          const int i = t * 128 + (tail ? warp * 16 : warp * 32) + lane;          // column of L = row of L^T
+          // element (row, column i) of P: column group i / 64, 128-byte rows, 16-byte pieces XOR-ed with the row modulo 8
+          unsigned char* pb = P_sm + (uint32_t)((i >> 6) * (RT * 128) + hh * 2048) + (uint32_t)((i & 7) * 2);
+          const uint32_t c8s = (uint32_t)(((i & 63) >> 3) << 4);
+          if (lane_ok) {
+#pragma unroll
+            for (int r = 0; r < 16; ++r) {
+              const float p = fast_exp2(v[r] - Mr[r]);
+              sum[r] += p;
+              *reinterpret_cast<__nv_bfloat16*>(pb + r * 128 + (c8s ^ (uint32_t)((r & 7) << 4))) = __float2bfloat16_rn(p);
+            }
           }
         }
-      }
-      {
-        float mine = 0.f;
-#pragma unroll
-        for (int r = 0; r < RT; ++r) {
-          float x = sum[r];
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-          if (lane == r) mine = x;
-        }
-        if (lane < RT) rsum[warp * RT + lane] = mine;
+        const float mine = lane_reduce16<false>(sum, lane);
+        if (lane < 16) rsum[warp * RT + hh * 16 + lane] = mine;
       }
       fence_proxy_async();                                             // P is read by the tensor core (async proxy)
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars.l_free);
       named_barrier_arrive(BAR_P_READY, TEW * 32 + 32);
-      named_barrier_sync(1, FCONS);                                   // B3: row sums and text sums are in place
+      named_barrier_sync(1, FCONS);                                   // B1: row sums here, maxima and sums of the text rows from the value warps
       if (warp == 0) {
         for (int x = lane; x < RT; x += 32) {
           float s_ = 0.f;
@@ -369,38 +418,50 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         __syncwarp();
         for (int x = lane; x < a.NB * 16; x += 32) {
           const int tb_ = x >> 4, g = x & 15;
-          float vs = 0.f, tsm = 0.f;
+          float M = 0.f, fv = 0.f, vs = 0.f, tsm = 0.f;
           if (g < G && tb_ < nbv) {
+            M = hvmax[x];
+            for (int w = tb_ * WPG; w < (tb_ + 1) * WPG; ++w) M = fmaxf(M, tmax[w * 16 + g]);
+            fv = fast_exp2(hvmax[x] - M);
             for (int rl = 0; rl < rbv; ++rl) vs += rsum[(tb_ * RB + rl) * G + g];
-            for (int w = tb_ * WPG; w < (tb_ + 1) * WPG; ++w) tsm += tsum[w * 16 + g];
+            vs *= fv;
+            for (int w = tb_ * WPG; w < (tb_ + 1) * WPG; ++w) {
+              const float tm_ = tmax[w * 16 + g];
+              if (tm_ != -INFINITY) tsm = fmaf(tsum[w * 16 + g], fast_exp2(tm_ - M), tsm);
+            }
           }
+          hmax[x] = M;
+          hfv[x] = fv;
           vsum[x] = vs;
           hsum[x] = vs + tsm;
         }
       }
-      named_barrier_sync(1, FCONS);                                   // B4: head sums
+      named_barrier_sync(1, FCONS);                                   // B2: joint maxima, sums and the vision factor
 
-      // ---------------- pass C: W^T of every stage from tensor memory to the weight tile ----------------
-      for (int c = 0; c < a.NJ; ++c) {
-        const uint32_t wbuf = wi & 1u;
-        const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);
-        wait_on(&bars.w_done[wbuf], (wi >> 1) & 1u);
-        __syncwarp();
-        tc_fence_after();
-        float v[RT];
-        if (warp < nsub) tmem_ld<RT>(tq + w_col + wbuf * RT, v);      // lane j < 16: row j of sub-chunk `warp`
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&bars.w_tfree[wbuf]);
-        if (wi >= 2) named_barrier_sync(BAR_W_FREE + (int)wbuf, FCONS);   // the value warps are done with this buffer's previous tile
-        if (warp < nsub && lane < 16) {
-          __nv_bfloat16* wt = W_sm + wbuf * w_buf_elems + warp * ((RT + 16) * SLD) + lane;
+      // ---------------- W^T (all m rows) from tensor memory to the weight tiles, at the joint maximum ----------------
+      float fvr[RT];
 #pragma unroll
-          for (int r = 0; r < RT; ++r) wt[r * SLD] = __float2bfloat16_rn(v[r]);
-        }
-        named_barrier_arrive(BAR_W_READY + (int)wbuf, FCONS);
-        ++wi;
+      for (int r = 0; r < RT; ++r) {
+        const int slot_ = rtab[r];
+        fvr[r] = slot_ >= 0 ? hfv[slot_] : 0.f;
       }
+      wait_on(&bars.w_done, ucount & 1u);
+      __syncwarp();
+      tc_fence_after();
+      const int NS = (a.m + 15) >> 4;
+      for (int t = 0; t < MTL; ++t) {
+        float v[RT];
+        __syncwarp();
+        tmem_ld<RT>(tq + w_col + (uint32_t)(t * RT), v);
+        const int j = t * 128 + warp * 32 + lane;                    // row of U
+        if (j < NS * 16) {
+          __nv_bfloat16* wt = W_sm + (j >> 4) * ((RT + 16) * SLD) + (j & 15);
+#pragma unroll
+          for (int r = 0; r < RT; ++r) wt[r * SLD] = __float2bfloat16_rn(v[r] * fvr[r]);
+        }
+      }
+      tc_fence_before();
+      named_barrier_arrive(BAR_W_READY, FCONS);
     }
     named_barrier_sync(BAR_END, (CW + 1) * 32);
     if (dead && lane == 0) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
@@ -506,7 +567,14 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
 #pragma unroll
         for (int e = 0; e < 4; ++e) yacc[mt][nh][e] = 0.f;
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // heads gid and gid + 8
-    for (int ts = 0; ts < nts; ++ts) {
+    for (int iu = 0, it = 0; iu + it < a.nu + nts;) {
+      if (!next_is_text(iu, it, a.nu, nts)) {            // a stage of U: the tensor core's
+        ++iu;
+        wait_on(&bars.full[slot], phase);
+        release();
+        continue;
+      }
+      const int ts = it++;
       wait_on(&bars.full[slot], phase);
       const uint32_t kt_u = sm_u + slot * a.stage_bytes, vt_u = kt_u + 2 * a.txt_half_bytes;
       for (int tile = wig; tile * 16 < a.TCH; tile += WPG) {
@@ -602,21 +670,22 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       release();
     }
 
-    // ---------------- joint softmax: the text accumulators move to the unit's reference maximum ----------------
-    if (t4 == 0) { tmax[vw * 16 + gid] = m_run[0]; tmax[vw * 16 + gid + 8] = m_run[1]; }
+    // ---------------- joint softmax: maxima and sums of this warp's text rows out, the joint maximum back ----------------
+#pragma unroll
+    for (int hr = 0; hr < 2; ++hr) {
+      float l = l_run[hr];
+      l += __shfl_xor_sync(0xffffffffu, l, 1);
+      l += __shfl_xor_sync(0xffffffffu, l, 2);
+      if (t4 == 0) { tmax[vw * 16 + gid + 8 * hr] = m_run[hr]; tsum[vw * 16 + gid + 8 * hr] = l; }
+    }
     named_barrier_sync(1, FCONS);                                   // B1
-    named_barrier_sync(1, FCONS);                                   // B2: head maxima
+    named_barrier_sync(1, FCONS);                                   // B2: joint maxima and sums
     {
       float scl[2];
 #pragma unroll
       for (int hr = 0; hr < 2; ++hr) {
-        const int head = gid + 8 * hr;
-        const float M = hmax[bl * 16 + head];
+        const float M = hmax[bl * 16 + gid + 8 * hr];
         scl[hr] = m_run[hr] == -INFINITY ? 0.f : fast_exp2(m_run[hr] - M);
-        float l = l_run[hr] * scl[hr];
-        l += __shfl_xor_sync(0xffffffffu, l, 1);
-        l += __shfl_xor_sync(0xffffffffu, l, 2);
-        if (t4 == 0) tsum[vw * 16 + head] = l;
       }
 #pragma unroll
       for (int nh = 0; nh < NH; ++nh) {
@@ -629,16 +698,13 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         }
       }
     }
-    named_barrier_sync(1, FCONS);                                   // B3
-    named_barrier_sync(1, FCONS);                                   // B4: head sums
 
-    // ---------------- pass C: y^T[128][heads] += V^T[128][16 rows of block] W^T[16][heads of block] ----------------
+    // ---------------- y^T[128][heads] += V^T[128][16 rows of block] W^T[16][heads of block], all weights in place ----------------
+    named_barrier_sync(BAR_W_READY, FCONS);
     for (int c = 0; c < a.NJ; ++c) {
       wait_on(&bars.full[slot], phase);
       const uint32_t v_u = sm_u + slot * a.stage_bytes + a.par_bytes;
       const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);
-      const uint32_t wbuf = wi & 1u;
-      named_barrier_sync(BAR_W_READY + (int)wbuf, FCONS);
       const int ntask = RB * msplit;
       for (int task = wig; task < nsub * ntask; task += WPG) {          // my (sub-chunk, block, row-tile group) tasks
         const int s = task / ntask, tk = task - s * ntask;
@@ -646,7 +712,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         if (rl >= rbv || bl >= nbv) continue;
         const int bi = bl * RB + rl;
         uint32_t bw[4];
-        ldsm_x4(bw, W_u + (uint32_t)((wbuf * w_buf_elems + s * ((RT + 16) * SLD) + (bi * G + lrowB) * SLD + lmid * 8) * 2));
+        ldsm_x4(bw, W_u + (uint32_t)(((c * JC + s) * ((RT + 16) * SLD) + (bi * G + lrowB) * SLD + lmid * 8) * 2));
         const uint32_t rowoff = v_u + (uint32_t)((bi * rows16 + s * 16 + lrowB) * 128);
         uint32_t av[8][4];
 #pragma unroll
@@ -660,10 +726,9 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
             for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(yacc[mt][nh], av[mt], bw[2 * nh], bw[2 * nh + 1]);
           }
       }
-      named_barrier_arrive(BAR_W_FREE + (int)wbuf, FCONS);
-      ++wi;
       release();
     }
+    named_barrier_sync(3, VTH);                                     // the weight tiles share their region with the reduction buffer
 
     // ---------------- unit end: reduce over the value warps, mu term, normalise or leave a partial ----------------
     const int bh = b0 * a.H_kv + h;                    // used when the block axis is split (NB == 1)
@@ -805,12 +870,16 @@ FusedPlan plan_fused_tc(const kvc_layer* L, int B, int R) {
   p.ncg = n / 64;
   const uint32_t chunk = (uint32_t)p.NB * p.RB * 4096u + (uint32_t)n * 32u;
   int jc = (int)(65536u / chunk);
-  const int jmax = ceil_div(m, 16) < 4 ? ceil_div(m, 16) : 4;          // at most 64 rows of U per stage: M of the re-projection MMA
+  const int jmax = ceil_div(m, 16) < 16 ? ceil_div(m, 16) : 16;
   p.JC = jc < 1 ? 1 : (jc > jmax ? jmax : jc);
   p.NJ = ceil_div(m, 16 * p.JC);
   p.par_bytes = (uint32_t)p.ncg * p.JC * 2048u;
   p.k_half_bytes = (uint32_t)p.NB * p.RB * p.JC * 2048u;
   p.stage_bytes = p.par_bytes + 2 * p.k_half_bytes;
+  if (p.stage_bytes < 16384u) p.stage_bytes = 16384u;                  // a stage also holds 128 rows x 64 columns of U
+  const int mtiles = ceil_div(m, 128);
+  p.UT = (int)(p.stage_bytes / 16384u) < mtiles ? (int)(p.stage_bytes / 16384u) : mtiles;
+  p.nu = p.ncg * ceil_div(mtiles, p.UT);
   int tch = (int)(p.stage_bytes / (p.NB * 512u)) & ~15;
   p.TCH = tch > 256 ? 256 : tch;
   if (p.TCH < 16) return p;
@@ -828,23 +897,26 @@ FusedPlan plan_fused_tc(const kvc_layer* L, int B, int R) {
   p.yhg = G > 4 ? 8 : (G > 2 ? 4 : 2);
   uint32_t off = 0;
   auto take = [&](uint32_t bytes) { uint32_t o = off; off = (off + bytes + 127u) & ~127u; return o; };
-  // P (read by the MMAs of pass C) and the reduction buffer of the unit end (used after them) share one region that
-  // starts right after the ring, 1024-byte aligned
+  // one region right after the ring (1024-byte aligned) serves, in turn: P (operand of the re-projection MMAs), the
+  // weight tiles of all m rows (written once those MMAs are complete), the reduction buffer of the unit end
   const uint32_t p_bytes = (uint32_t)rt * n * 2, yred_bytes = (uint32_t)p.VW * p.yhg * D * 4;
-  p.off_P = take(p_bytes > yred_bytes ? p_bytes : yred_bytes);
+  const uint32_t w_bytes = (uint32_t)ceil_div(m, 16) * (rt + 16) * SLD * 2;
+  uint32_t r0_bytes = p_bytes > yred_bytes ? p_bytes : yred_bytes;
+  if (w_bytes > r0_bytes) r0_bytes = w_bytes;
+  p.off_P = take(r0_bytes);
   p.off_yred = p.off_P;
+  p.off_W = p.off_P;
   p.off_q = take((uint32_t)p.NB * 16 * QLD * 2);
-  p.off_S = take((uint32_t)(2 * p.JC * rt * 32 + 2 * p.JC * (rt + 16) * SLD * 2));
-  p.off_W = p.off_S + (uint32_t)(2 * p.JC * rt * 32);
+  p.off_S = take((uint32_t)(2 * p.JC * rt * 32));
   p.off_wred = 0;
   p.off_rstat = take((uint32_t)2 * TEW * rt * 4);
   p.off_tstat = take((uint32_t)2 * p.VW * 16 * 4);
-  p.off_hstat = take((uint32_t)3 * p.NB * 16 * 4);
+  p.off_hstat = take((uint32_t)5 * p.NB * 16 * 4);
   p.off_rtab = take((uint32_t)rt * 4);
   p.misc_bytes = off;
   const int nt = (n + 127) / 128;
   int cols = 32;
-  while (cols < nt * rt + 2 * rt) cols *= 2;
+  while (cols < nt * rt + mtiles * rt) cols *= 2;
   p.tmem_cols = cols;
   if (cols > 512) return p;
   if (SMEM_LIMIT < 1024u + 2048u + p.misc_bytes + 2 * p.stage_bytes) return p;

@@ -95,6 +95,7 @@ struct FusedPlan {
   int tc;            // 1: the expansions run on tcgen05 with the logits in tensor memory (kvc_fused_tc.cu)
   uint32_t off_P, off_rtab;
   int tmem_cols;
+  int UT, nu;        // 128-row tiles of U per stage and stages of U per unit (tensor-memory variant)
   size_t smem_bytes;
 };
 
@@ -108,7 +109,8 @@ struct kvc_layer {
   int passthrough;       // ratio_permille == 0
   int device;
   int num_sms;
-  int use_tc;            // 1: expansions of the one-kernel decode path on tcgen05 (environment KVC_EXPANSION=tcgen05 at creation)
+  int use_tc;            // expansions of the one-kernel decode path: 0 chosen per shape, 1 tcgen05, -1 mma.sync (environment
+                         // KVC_EXPANSION=tcgen05 | mma when the handle is created)
   int32_t* d_idx;        // device [H_kv][m]
   int* d_cnt;            // device [KVC_MAX_COUNTERS + 1] arrival counters of the one-kernel decode path (zero between
                          // calls), then the status word of the compress kernels
