@@ -36,9 +36,12 @@ NOMINAL_HBM_GBS = 8000.0        # the figure the task's metric quotes its percen
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
 # the ncu capture summarised under profiles/, keyed by (kernel, workload name); None = not captured.
 NCU_TRAFFIC_BYTES = {
-    # profiles/fused_decode_config1.md: 185.5 MB read + 5.5 MB written per launch at T = 130 text rows; a text row costs
-    # 2 * B * H_kv * d * 2 bytes = 131072 bytes more, so the mid-run launch (T = 255.5) moves 191.0 MB + 16.5 MB
-    ("fused", "config1-llava-next-7b"): 207.5e6,
+    # profiles/fused_decode_config1.md: 185.7 MB read + 6.6 MB written per launch at T = 130 text rows; a text row costs
+    # 2 * B * H_kv * d * 2 bytes = 131072 bytes more, so the mid-run launch (T = 255.5) moves 192.3 MB + 16.4 MB
+    ("fused", "config1-llava-next-7b"): 208.7e6,
+    # profiles/fused_decode_tc_config2.md: 123.0 MB read + 4.6 MB written per launch at T = 258; 32768 bytes per text
+    # row more up to the mid-run launch (T = 511.5)
+    ("fused_tc", "config2-qwen2-vl-7b"): 136.0e6,
 }
 
 
