@@ -1,23 +1,25 @@
 // Algorithm 1 as one kernel for bf16 storage, with the two expansions on the 5th-generation tensor cores:
-//   L^T[n x rows] += theta_c^T[n x 16] S_c^T[16 x rows]      (Alg. 1 step 2; logits accumulate in tensor memory)
-//   W_c^T[rows of c x rows] = U_c[rows of c x n] P^T[n x rows]  (Alg. 1 step 3, re-projection of the probabilities)
-// `rows` = the expansion rows of a work unit (sequence, block, head), the N dimension of both products, so that the
-// large dimensions (n and the stage's rows of theta/U) are the M dimension of tcgen05.mma and the operand tiles are
-// read exactly as the TMA engine lays them down (128-byte swizzle): theta_c as an MN-major A operand, U_c as a
-// K-major A operand.  Work units, stages and the producer are those of kvc_fused.cu.  Warp roles:
-//   warps 0-3        softmax over the logits read back from tensor memory (one lane per column of L^T), P as a
-//                    bf16 operand in shared memory; in pass C they move W^T from tensor memory to the weight tile
-//   value warps      S_c = sigma q K_c^T (mma.sync, bf16 tile in shared memory in UMMA core-matrix order), text rows
+//   L^T[n x rows] += theta_c^T[n x 16] S_c^T[16 x rows]   (Alg. 1 step 2; logits accumulate in tensor memory)
+//   W^T[m x rows]  = U[m x n] P^T[n x rows]                (Alg. 1 step 3, re-projection of the probabilities)
+// `rows` = the expansion rows of a work unit (sequence, block, head) = the N dimension of both products; the large
+// dimensions (n for the logits, m for the weights) are the M dimension of tcgen05.mma, in tiles of 128, and the
+// operand tiles are read exactly as the TMA engine lays them down (128-byte swizzle): theta_c as an MN-major A
+// operand, 128-row tiles of a 64-column group of U as a K-major A operand.  Work units and the ring are those of
+// kvc_fused.cu; the stage sequence of a unit is: pass A (theta rows + K_tilde rows), then the column groups of U
+// interleaved with the text stages, then the V_tilde stages.  Warp roles:
+//   warps 0-3        softmax of the vision logits read back from tensor memory (one lane per column of L^T), relative
+//                    to the vision-only maximum; P as a bf16 operand in shared memory; when W^T is complete they move
+//                    it to the weight tiles, scaled to the joint maximum of vision and text rows
+//   value warps      S_c = sigma q K_c^T (mma.sync; bf16 tile in shared memory in UMMA core-matrix order), text rows
 //                    flash-style, y^T += V_c^T W_c^T, unit end: reduction, mu term, output or partial + merge
 //   MMA warp         one thread issues every tcgen05.mma and commits completion to the mbarriers that free the
 //                    stage, the score tile and the accumulators
 //   producer warp    one thread feeds the ring through tensor maps
 //
-// Status: opt-in (KVC_EXPANSION=tcgen05 when the layer is created).  Measured on B200: one tcgen05.mma of K = 16
-// occupies the tensor pipe for about 85 cycles at M = 64 and about 129 cycles at M = 128 whatever N <= 128 is (one
-// row of A per cycle), so with N = 16 or 32 expansion rows the re-projection (n/16 MMAs per stage) is bound by the
-// MMA count, not by data; the products only pay off with >= 64 rows on both M and N, i.e. with work units that
-// batch the expansion rows of many sequences of a head.
+// Measured on B200: one tcgen05.mma of K = 16 occupies the tensor pipe for about 129 cycles at M = 128 and about 85
+// at M = 64 whatever N <= 128 is (one row of A per cycle, A from shared or tensor memory alike).  The cost of a unit
+// is therefore (n/128) (m/16) + (m/128) (n/16) MMAs whatever its number of expansion rows: the variant pays off
+// for long blocks with as many rows per unit as the grid allows (see plan_fused in kvc_fused.cu).
 #include "kvc_fused.cuh"
 #include "kvc_tcgen05.cuh"
 
