@@ -25,7 +25,6 @@
 
 namespace kvc {
 
-constexpr int TEW = 4;                         // softmax / conversion warps: one per tensor-memory lane quarter
 constexpr int BAR_P_READY = 12;                // probabilities written (warps 0-3 arrive, the MMA warp waits)
 constexpr int BAR_END = 13;                    // every tensor-memory user is done: the MMA warp may free it
 
@@ -63,12 +62,15 @@ __device__ __forceinline__ float lane_reduce16(float (&x)[16], int lane) {
   return op(u1 ? y2[1] : y2[0], __shfl_xor_sync(0xffffffffu, u1 ? y2[0] : y2[1], 1));
 }
 
-template <int VW, int NH, int MT>
-__global__ void __launch_bounds__((TEW + VW + 2) * 32, 1)
+// EW = 4 or 8 softmax / conversion warps (warps 0 .. EW-1: one or two per tensor-memory lane quarter), VW value warps
+template <int EW, int VW, int NH, int MT>
+__global__ void __launch_bounds__((EW + VW + 2) * 32, 1)
 fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                        const __grid_constant__ CUtensorMap tmKt, const __grid_constant__ CUtensorMap tmVt,
                        const __grid_constant__ CUtensorMap tmTh, const __grid_constant__ CUtensorMap tmU,
                        const FusedArgs a) {
+  constexpr int TEW = EW;
+  constexpr int TSTEP = EW / 4;               // the tiles of a lane quarter are dealt to its TSTEP warps
   constexpr int CW = TEW + VW;                // warps that meet at the softmax barriers
   constexpr int FCONS = CW * 32;
   constexpr int MMA_WARP = CW, PROD_WARP = CW + 1;
@@ -106,6 +108,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   const int NT = (a.n + 127) >> 7;
   const int MTL = (a.m + 127) >> 7;            // 128-row tiles of W^T (rows of U)
   const uint32_t w_col = (uint32_t)(NT * RT);
+  const bool w_tail64 = a.m - 128 * (MTL - 1) <= 64;   // the last tile of W^T holds at most 64 rows of U: M = 64
   const int ugroups = (MTL + a.UT - 1) / a.UT; // stages per 64-column group of U: UT row tiles each
 
   const int per_h = a.nbg * a.nrg;
@@ -193,7 +196,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     const uint32_t cg_bytes = (uint32_t)rows16 * 128u;            // one 64-column group of a parameter tile
     const uint32_t idesc_L_full = umma_idesc_bf16(128, RT, 1, 0);
     const uint32_t idesc_L_half = umma_idesc_bf16(64, RT, 1, 0);
-    const uint32_t idesc_W = umma_idesc_bf16(128, RT, 0, 0);
+    const uint32_t idesc_W = umma_idesc_bf16(128, RT, 0, 0), idesc_W64 = umma_idesc_bf16(64, RT, 0, 0);
     const bool half_tail = (a.n & 127) != 0;                      // n = 64 (mod 128): the last tile of L^T has 64 rows
     for (int u = blockIdx.x; u < a.units; u += gridDim.x, ++ucount) {
       const int rem = u % per_h;
@@ -241,7 +244,8 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
               for (int kk = 0; kk < 4; ++kk) {
                 const uint64_t adesc = umma_smem_desc(par_u + (uint32_t)(t * 16384 + kk * 32), 16u, 1024u, UMMA_LAYOUT_SW128);
                 const uint64_t bdesc = umma_smem_desc(P_u + (uint32_t)(cg * RT * 128 + kk * 32), 16u, 1024u, UMMA_LAYOUT_SW128);
-                umma_bf16(tb + w_col + (uint32_t)((t0 + t) * RT), adesc, bdesc, idesc_W, (cg | kk) ? 1u : 0u);
+                umma_bf16(tb + w_col + (uint32_t)((t0 + t) * RT), adesc, bdesc, (w_tail64 && t0 + t == MTL - 1) ? idesc_W64 : idesc_W,
+                          (cg | kk) ? 1u : 0u);
               }
             umma_commit(&bars.empty[slot]);
             if (i == a.nu - 1) umma_commit(&bars.w_done);
@@ -299,7 +303,8 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     // ======================================================================================================
     // warps 0-3: joint softmax on the logits in tensor memory, then W^T -> weight tiles
     // ======================================================================================================
-    const uint32_t tq = tb + ((uint32_t)(warp * 32) << 16);       // this warp's lane quarter
+    const int wq = warp & 3, wh = warp >> 2;                      // lane quarter; which of the quarter's warps
+    const uint32_t tq = tb + ((uint32_t)(wq * 32) << 16);
     const bool half_tail = (a.n & 127) != 0;
     unsigned char* P_sm = sm + a.off_P;                           // [n/64][RT][64] bf16, 128-byte swizzle
     for (int u = blockIdx.x; u < a.units; u += gridDim.x, ++ucount) {
@@ -329,13 +334,13 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         for (int r = 0; r < 16; ++r) mx[r] = -INFINITY;
         uint32_t nx[16];
         __syncwarp();
-        tmem_ld_issue_x16(tq + (uint32_t)(hh * 16), nx);
-        for (int t = 0; t < NT; ++t) {
+        if (wh < NT) tmem_ld_issue_x16(tq + (uint32_t)(wh * RT + hh * 16), nx);
+        for (int t = wh; t < NT; t += TSTEP) {
           float v[16];
           tmem_ld_wait_x16(nx);
 #pragma unroll
           for (int r = 0; r < 16; ++r) v[r] = __uint_as_float(nx[r]);
-          if (t + 1 < NT) tmem_ld_issue_x16(tq + (uint32_t)((t + 1) * RT + hh * 16), nx);   // in flight while tile t is reduced
+          if (t + TSTEP < NT) tmem_ld_issue_x16(tq + (uint32_t)((t + TSTEP) * RT + hh * 16), nx);   // in flight while tile t is reduced
           if (!(half_tail && t == NT - 1) || lane < 16) {
 #pragma unroll
             for (int r = 0; r < 16; ++r) mx[r] = fmaxf(mx[r], v[r]);
@@ -379,16 +384,16 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         }
         uint32_t nx[16];
         __syncwarp();
-        tmem_ld_issue_x16(tq + (uint32_t)(hh * 16), nx);
-        for (int t = 0; t < NT; ++t) {
+        if (wh < NT) tmem_ld_issue_x16(tq + (uint32_t)(wh * RT + hh * 16), nx);
+        for (int t = wh; t < NT; t += TSTEP) {
           float v[16];
           tmem_ld_wait_x16(nx);
 #pragma unroll
           for (int r = 0; r < 16; ++r) v[r] = __uint_as_float(nx[r]);
-          if (t + 1 < NT) tmem_ld_issue_x16(tq + (uint32_t)((t + 1) * RT + hh * 16), nx);   // in flight while tile t is processed
+          if (t + TSTEP < NT) tmem_ld_issue_x16(tq + (uint32_t)((t + TSTEP) * RT + hh * 16), nx);   // in flight while tile t is processed
           const bool tail = half_tail && t == NT - 1;
           const bool lane_ok = !tail || lane < 16;
-          const int i = t * 128 + (tail ? warp * 16 : warp * 32) + lane;          // column of L = row of L^T
+          const int i = t * 128 + (tail ? wq * 16 : wq * 32) + lane;          // column of L = row of L^T
           // element (row, column i) of P: column group i / 64, 128-byte rows, 16-byte pieces XOR-ed with the row modulo 8
           unsigned char* pb = P_sm + (uint32_t)((i >> 6) * (RT * 128) + hh * 2048) + (uint32_t)((i & 7) * 2);
           const uint32_t c8s = (uint32_t)(((i & 63) >> 3) << 4);
@@ -451,12 +456,13 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       __syncwarp();
       tc_fence_after();
       const int NS = (a.m + 15) >> 4;
-      for (int t = 0; t < MTL; ++t) {
+      for (int t = wh; t < MTL; t += TSTEP) {
         float v[RT];
         __syncwarp();
         tmem_ld<RT>(tq + w_col + (uint32_t)(t * RT), v);
-        const int j = t * 128 + warp * 32 + lane;                    // row of U
-        if (j < NS * 16) {
+        const bool t64 = w_tail64 && t == MTL - 1;                   // a 64-row tile: 16 rows in the first lanes of every quarter
+        const int j = t * 128 + (t64 ? wq * 16 : wq * 32) + lane;    // row of U
+        if (j < NS * 16 && (!t64 || lane < 16)) {
           __nv_bfloat16* wt = W_sm + (j >> 4) * ((RT + 16) * SLD) + (j & 15);
 #pragma unroll
           for (int r = 0; r < RT; ++r) wt[r * SLD] = __float2bfloat16_rn(v[r] * fvr[r]);
@@ -847,11 +853,12 @@ FusedPlan plan_fused_tc(const kvc_layer* L, int B, int R) {
   if (reinterpret_cast<uintptr_t>(L->desc.theta) & 15 || reinterpret_cast<uintptr_t>(L->desc.U) & 15) return p;
   const int sms = L->num_sms > 0 ? L->num_sms : 148;
   p.tc = 1;
-  p.EW = TEW;
+  p.EW = 4;
   p.VW = n <= 256 ? 8 : 10;
   p.ktw = 0;
   // the logits live in tensor memory: two row tiles per unit whenever a sequence has more than 16 expansion rows
   p.MT = G * R > ROWS ? 2 : 1;
+  if (p.MT == 2 && n > 256) { p.EW = 8; p.VW = 6; }     // 32 rows x long blocks: the softmax is the larger share, the value warps have slack
   const int cap = ROWS * p.MT;
   p.RB = R < cap / G ? R : cap / G;
   p.NB = 1;
@@ -911,7 +918,7 @@ FusedPlan plan_fused_tc(const kvc_layer* L, int B, int R) {
   p.off_q = take((uint32_t)p.NB * 16 * QLD * 2);
   p.off_S = take((uint32_t)(2 * p.JC * rt * 32));
   p.off_wred = 0;
-  p.off_rstat = take((uint32_t)2 * TEW * rt * 4);
+  p.off_rstat = take((uint32_t)2 * p.EW * rt * 4);
   p.off_tstat = take((uint32_t)2 * p.VW * 16 * 4);
   p.off_hstat = take((uint32_t)5 * p.NB * 16 * 4);
   p.off_rtab = take((uint32_t)rt * 4);
@@ -932,22 +939,23 @@ FusedPlan plan_fused_tc(const kvc_layer* L, int B, int R) {
   return p;
 }
 
-template <int VW, int NH, int MT>
+template <int EW, int VW, int NH, int MT>
 static cudaError_t launch_tc_inst(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
   static size_t configured = 0;
   if (p.smem_bytes > configured) {
-    cudaError_t e = cudaFuncSetAttribute(fused_decode_tc_kernel<VW, NH, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
+    cudaError_t e = cudaFuncSetAttribute(fused_decode_tc_kernel<EW, VW, NH, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
     if (e != cudaSuccess) return e;
     configured = p.smem_bytes;
   }
-  return launch_dependent(fused_decode_tc_kernel<VW, NH, MT>, dim3(p.grid), dim3((TEW + VW + 2) * 32), p.smem_bytes, st, tm[0], tm[1],
+  return launch_dependent(fused_decode_tc_kernel<EW, VW, NH, MT>, dim3(p.grid), dim3((EW + VW + 2) * 32), p.smem_bytes, st, tm[0], tm[1],
                           tm[2], tm[3], tm[4], tm[5], fa);
 }
 
 template <int NH>
 static cudaError_t launch_tc_nh(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
-  if (p.VW == 8) return p.MT == 2 ? launch_tc_inst<8, NH, 2>(tm, fa, p, st) : launch_tc_inst<8, NH, 1>(tm, fa, p, st);
-  return p.MT == 2 ? launch_tc_inst<10, NH, 2>(tm, fa, p, st) : launch_tc_inst<10, NH, 1>(tm, fa, p, st);
+  if (p.EW == 8) return launch_tc_inst<8, 6, NH, 2>(tm, fa, p, st);
+  if (p.VW == 8) return p.MT == 2 ? launch_tc_inst<4, 8, NH, 2>(tm, fa, p, st) : launch_tc_inst<4, 8, NH, 1>(tm, fa, p, st);
+  return launch_tc_inst<4, 10, NH, 1>(tm, fa, p, st);
 }
 
 cudaError_t launch_fused_tc_kernel(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
