@@ -268,6 +268,21 @@ def test_one_kernel_path_edges(B, H_q, H_kv, grid, R, T):
     _check(shape, p)
 
 
+@pytest.mark.parametrize("B,H_q,H_kv,grid,R,T,ratio", [
+    (2, 14, 2, 32, 4, 0, 600),      # no text rows: only stages of U between the two passes
+    (1, 14, 2, 32, 5, 300, 950),    # m = 52: one tile of W^T, taken with M = 64
+    (1, 14, 2, 32, 3, 17, 850),     # m = 154: a full tile and a 26-row tile
+    (2, 8, 8, 16, 1, 40, 100),      # m = 231 of n = 256, one block, MHA: a single expansion row per unit and sequence
+    (3, 6, 2, 8, 9, 5, 500),        # n = 64 (half a logit tile), G = 3, blocks not a multiple of the blocks per unit
+])
+def test_tensor_memory_variant_edges(B, H_q, H_kv, grid, R, T, ratio, monkeypatch):
+    monkeypatch.setenv("KVC_EXPANSION", "tcgen05")
+    shape = wl.Shape("tc-edge", 1, B, H_q, H_kv, 128, grid, R, T, 1, "bf16", ratio_permille=ratio)
+    p = tl.make_problem(shape, 190 + B + 7 * R + T, T=T, T_cap=T + 5)
+    counts = _fused_launches(lambda: _check(shape, p))
+    assert counts["fused_tc"] >= 1 and counts["fused"] == 0 and counts["scores"] == 0
+
+
 @pytest.mark.parametrize("B,H_q,H_kv,grid,R,T", [
     (3, 2, 2, 8, 5, 1),        # two sequences per unit, odd batch, one text row
     (1, 7, 1, 8, 5, 700),      # G = 7: two row tiles of expansion rows, units split the block axis
