@@ -483,9 +483,9 @@ def main():
             if n:
                 kernels[k] = {"launches": n, "total_ms": round(t, 3), "avg_us": round(t / n * 1e3, 3),
                               "share": round(t / tot, 4)}
-        dom = max(("scores", "output", "fused", "fused_tc"), key=lambda k: prof.get(k, (0.0, 0))[0])
+        dom = max(("scores", "output", "fused", "fused_tc", "fused_pair"), key=lambda k: prof.get(k, (0.0, 0))[0])
         t_dom, n_dom = prof[dom]
-        if dom in ("fused", "fused_tc"):
+        if dom in ("fused", "fused_tc", "fused_pair"):
             # one kernel per layer call: its launch duration is the decode loop's device time over its launches
             # (CUDA events around the whole loop on the launching stream; consecutive launches overlap their
             # prologues, which the per-launch event brackets of the second pass would forbid)

@@ -83,7 +83,8 @@ KVC_API int kvc_retained_len(int n, int ratio_permille);
  * The device that is current at this call must be current for every later call with the handle.
  * bf16 decode calls run Alg. 1 steps 2-3 either on mma.sync with the logits in registers or on tcgen05 with the
  * logits in tensor memory; the library picks per shape (same results within the bf16 tolerance).  The environment
- * variable KVC_EXPANSION = "tcgen05" | "mma", read when the handle is created, forces one of them where it applies. */
+ * variable KVC_EXPANSION = "tcgen05" | "mma", read when the handle is created, forces one of them where it applies;
+ * "pair" selects the tcgen05 path run by clusters of two CTAs per (sequence, KV head) (experimental: correct, slower). */
 KVC_API int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out);
 KVC_API int kvc_layer_destroy(kvc_layer* layer);
 
@@ -183,7 +184,8 @@ typedef enum {
   KVC_KERNEL_COMBINE = 6,         /* n-split partials of Alg. 1 step 3 combined per row */
   KVC_KERNEL_FUSED = 7,           /* Alg. 1 steps 1-4 + text + normalisation in one kernel (bf16) */
   KVC_KERNEL_FUSED_TC = 8,        /* the same kernel with steps 2-3 on tcgen05 / tensor memory (see kvc_layer_create) */
-  KVC_KERNEL_COUNT = 9
+  KVC_KERNEL_FUSED_PAIR = 9,      /* the tensor-memory kernel run by clusters of two CTAs per (sequence, KV head) */
+  KVC_KERNEL_COUNT = 10
 } kvc_kernel_id;
 KVC_API int kvc_profile_start(int max_launches);
 KVC_API int kvc_profile_stop(void);

@@ -780,6 +780,10 @@ FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
     // The tensor-memory variant pays per tcgen05.mma, not per expansion row: it wins for long blocks once two row
     // tiles per unit still give most SMs a unit (measured on the n = 1024, G = 7 shape: ahead from batch 16 on,
     // behind at batches 1-4 where units of half the size halve the latency).
+    if (L->use_tc == 2) {
+      const FusedPlan t2 = plan_fused_pair(L, B, R);
+      if (t2.ok) return t2;
+    }
     const FusedPlan t = plan_fused_tc(L, B, R);
     if (t.ok && (L->use_tc > 0 || (L->desc.n > 640 && t.MT == 2 && t.units >= 96))) return t;
   }
@@ -963,7 +967,7 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
     // theta, U [H_kv][m][n] viewed as (64 columns, m rows, n/64 column groups, H_kv): a box lands as [group][row][64]
     const uint64_t dims[4] = {64ull, (uint64_t)m, (uint64_t)p.ncg, (uint64_t)H_kv};
     const uint64_t str[3] = {(uint64_t)n * 2, 128ull, (uint64_t)m * n * 2};
-    const uint32_t box[4] = {64u, (uint32_t)(16 * p.JC), (uint32_t)p.ncg, 1u};
+    const uint32_t box[4] = {64u, (uint32_t)(16 * p.JC), (uint32_t)(p.tc == 2 ? p.ncg / 2 : p.ncg), 1u};
     const uint32_t box_tc[4] = {64u, 128u, 1u, 1u};     // tensor-memory variant: U by 64-column groups, 128 rows at a time
     if (!encode_tensor_map_bf16(&tm[4], a.theta, 4, dims, str, box)) return cudaSuccess;
     if (!encode_tensor_map_bf16(&tm[5], a.U, 4, dims, str, p.tc ? box_tc : box)) return cudaSuccess;
@@ -988,12 +992,13 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
   fa.off_rstat = ring + p.off_rstat; fa.off_tstat = ring + p.off_tstat; fa.off_hstat = ring + p.off_hstat;
   fa.off_yred = ring + p.off_yred;
   fa.off_P = ring + p.off_P; fa.off_rtab = ring + p.off_rtab; fa.tmem_cols = p.tmem_cols; fa.UT = p.UT; fa.nu = p.nu;
+  fa.off_xstat = ring + p.off_xstat; fa.off_wrecv = ring + p.off_wrecv;
   fa.part_y = a.fpart_y;
   fa.part_ml = a.fpart_ml;
   fa.cnt = L->d_cnt;
   fa.status = a.status;
 
-  ProfScope prof(p.tc ? KVC_KERNEL_FUSED_TC : KVC_KERNEL_FUSED, st);
+  ProfScope prof(p.tc == 2 ? KVC_KERNEL_FUSED_PAIR : (p.tc ? KVC_KERNEL_FUSED_TC : KVC_KERNEL_FUSED), st);
   if (p.tc) return launch_fused_tc_kernel(tm, fa, p, st);
   return a.G > 8 ? launch_nh<2>(tm, fa, p, st) : launch_nh<1>(tm, fa, p, st);
 }

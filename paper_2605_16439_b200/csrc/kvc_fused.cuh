@@ -29,6 +29,7 @@ struct FusedArgs {
   uint32_t off_P, off_rtab;   // tensor-memory variant: probabilities as an MMA operand; head slot of every expansion row
   int tmem_cols;              // tensor-memory variant: columns to allocate (power of two >= 32)
   int UT, nu;                 // tensor-memory variant: 128-row tiles of U per stage; stages of U per unit
+  uint32_t off_xstat, off_wrecv;   // pair mode of the tensor-memory variant: what the peer CTA writes
   float* part_y;      // [B*H_kv][nrg][G][D]  partial outputs (only when nrg > 1)
   float2* part_ml;    // [B*H_kv][nrg][G]     (max in log2 units, sum)
   int* cnt;           // [B*H_kv] arrival counters, zero between calls

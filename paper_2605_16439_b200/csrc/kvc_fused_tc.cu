@@ -42,6 +42,8 @@ struct TcBars {
   uint64_t w_done;         // W^T of the unit is complete
   uint64_t l_done;         // the logits of the unit are complete
   uint64_t l_free;         // the logits of the unit have been read back (4 warps)
+  uint64_t x_data;         // pair mode: the peer's statistics and partial weights of the unit have landed here
+  uint64_t x_ack;          // pair mode: the peer has consumed what this CTA sent for the unit
 };
 
 // Reduces 16 per-lane values over the 32 lanes of a warp (maximum or sum) in 31 shuffles: after the first exchange
@@ -63,7 +65,11 @@ __device__ __forceinline__ float lane_reduce16(float (&x)[16], int lane) {
 }
 
 // EW = 4 or 8 softmax / conversion warps (warps 0 .. EW-1: one or two per tensor-memory lane quarter), VW value warps
-template <int EW, int VW, int NH, int MT>
+// PAIR: the two CTAs of a cluster share a (sequence, KV head): both compute the scores of all its blocks, CTA c keeps
+// the logits and the partial weights of columns [c n/2, (c+1) n/2) (its half of theta and U), the partial weights of the
+// other CTA's half of the m rows are sent to it through distributed shared memory, and each CTA multiplies its half of
+// the V_tilde rows (and attends its half of the text rows); the two outputs are merged like those of any split sequence.
+template <int EW, int VW, int NH, int MT, bool PAIR>
 __global__ void __launch_bounds__((EW + VW + 2) * 32, 1)
 fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                        const __grid_constant__ CUtensorMap tmKt, const __grid_constant__ CUtensorMap tmVt,
@@ -90,6 +96,8 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     mbar_init(&bars.w_done, 1);
     mbar_init(&bars.l_done, 1);
     mbar_init(&bars.l_free, TEW);
+    mbar_init(&bars.x_data, 1);
+    mbar_init(&bars.x_ack, 1);
     fence_mbar_init();
   }
   if (warp == MMA_WARP) tmem_alloc(&s_tmem, (uint32_t)a.tmem_cols);
@@ -104,8 +112,11 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if constexpr (PAIR) cluster_sync_all();      // the peer's barriers exist before anything is sent to them
   const uint32_t tb = s_tmem;                  // tensor memory: L^T tiles at columns [0, NT*RT), W^T tiles after them
-  const int NT = (a.n + 127) >> 7;
+  const int ncgl = PAIR ? a.ncg >> 1 : a.ncg;  // 64-column groups of theta / U this CTA works on
+  const int NT = PAIR ? a.n >> 8 : (a.n + 127) >> 7;
+  const int NJ0 = PAIR ? (a.NJ + 1) >> 1 : a.NJ;   // pair mode: CTA 0 takes the first NJ0 stages of the m axis in the value pass
   const int MTL = (a.m + 127) >> 7;            // 128-row tiles of W^T (rows of U)
   const uint32_t w_col = (uint32_t)(NT * RT);
   const bool w_tail64 = a.m - 128 * (MTL - 1) <= 64;   // the last tile of W^T holds at most 64 rows of U: M = 64
@@ -125,14 +136,16 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     for (int u = blockIdx.x; u < a.units; u += gridDim.x) {
       const int h = u / per_h, rem = u - h * per_h;
       const int bg = rem / a.nrg, rg = rem - bg * a.nrg;
-      const int b0 = bg * a.NB, r0 = rg * a.RB;
+      const int b0 = bg * a.NB, r0 = PAIR ? 0 : rg * a.RB;
       const RowRanges tr = row_ranges(a, rg);
       const int nts = tr.na + tr.nb;
+      const int cg0 = PAIR ? rg * ncgl : 0;          // first column group of this CTA
+      const int c2first = (PAIR && rg) ? NJ0 : 0, c2count = PAIR ? (rg ? a.NJ - NJ0 : NJ0) : a.NJ;
       // stage sequence of a unit: NJ stages of pass A (theta rows + K_tilde rows); then the column groups of U and
       // the text stages, interleaved so that the tensor core (U) and the value warps (text) both have work; then
       // NJ stages of V_tilde rows
       for (int part = 0; part < 3; ++part) {
-        const int count = part == 1 ? a.nu + nts : a.NJ;
+        const int count = part == 1 ? a.nu + nts : (part == 0 ? a.NJ : c2count);
         int iu = 0, it = 0;
         for (int cc = 0; cc < count; ++cc) {
           const bool is_text = part == 1 && next_is_text(iu, it, a.nu, nts);
@@ -152,16 +165,16 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
             const int cg = c / ugroups, t0 = (c - cg * ugroups) * a.UT;
             const int nt_ = min(a.UT, MTL - t0);
             mbar_expect_tx(bar, (uint32_t)nt_ * 16384u);
-            for (int t = 0; t < nt_; ++t) tma_load_4d(dst + t * 16384, &tmU, 0, (t0 + t) * 128, cg, h, bar);
+            for (int t = 0; t < nt_; ++t) tma_load_4d(dst + t * 16384, &tmU, 0, (t0 + t) * 128, cg0 + cg, h, bar);
           } else if (part == 0) {
             const int j0 = c * rows16;
             mbar_expect_tx(bar, a.par_bytes + 2 * a.k_half_bytes);
-            tma_load_4d(dst, &tmTh, 0, j0, 0, h, bar);               // parameters: never written by this library
+            tma_load_4d(dst, &tmTh, 0, j0, cg0, h, bar);             // parameters: never written by this library
             if (first) { grid_dep_wait(); first = false; }            // everything else may come from the stream's previous kernel
             tma_load_5d(dst + a.par_bytes, &tmK, 0, j0, r0, h, b0, bar);
             tma_load_5d(dst + a.par_bytes + a.k_half_bytes, &tmK, 64, j0, r0, h, b0, bar);
           } else {
-            const int j0 = c * rows16;
+            const int j0 = (c2first + c) * rows16;
             mbar_expect_tx(bar, 2 * a.k_half_bytes);
             tma_load_5d(dst + a.par_bytes, &tmV, 0, j0, r0, h, b0, bar);
             tma_load_5d(dst + a.par_bytes + a.k_half_bytes, &tmV, 64, j0, r0, h, b0, bar);
@@ -197,7 +210,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     const uint32_t idesc_L_full = umma_idesc_bf16(128, RT, 1, 0);
     const uint32_t idesc_L_half = umma_idesc_bf16(64, RT, 1, 0);
     const uint32_t idesc_W = umma_idesc_bf16(128, RT, 0, 0), idesc_W64 = umma_idesc_bf16(64, RT, 0, 0);
-    const bool half_tail = (a.n & 127) != 0;                      // n = 64 (mod 128): the last tile of L^T has 64 rows
+    const bool half_tail = !PAIR && (a.n & 127) != 0;             // n = 64 (mod 128): the last tile of L^T has 64 rows
     for (int u = blockIdx.x; u < a.units; u += gridDim.x, ++ucount) {
       const int rem = u % per_h;
       const int rg = rem % a.nrg;
@@ -260,7 +273,8 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         }
       }
       // ---------------- the V_tilde stages belong to the value warps ----------------
-      for (int c = 0; c < a.NJ; ++c) {
+      const int c2count = PAIR ? (rg ? a.NJ - NJ0 : NJ0) : a.NJ;
+      for (int c = 0; c < c2count; ++c) {
         wait_on(&bars.full[slot], phase);
         if (lane == 0) mbar_arrive(&bars.empty[slot]);
         advance();
@@ -289,6 +303,10 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   float* vsum = hsum + a.NB * 16;
   float* hvmax = vsum + a.NB * 16;                                           // maximum over the vision logits only
   float* hfv = hvmax + a.NB * 16;                                            // 2^(hvmax - hmax): moves the vision weights to the joint maximum
+  float* hfp = hfv + a.NB * 16;                                              // pair mode: the same for the peer's partial weights
+  float* rowf = hfp + a.NB * 16;                                             // [2][RT] those factors per expansion row
+  float* xstat = reinterpret_cast<float*>(sm + a.off_xstat);                 // pair mode, written by the peer: [16] maxima, [RT] row sums
+  __nv_bfloat16* wrecv = reinterpret_cast<__nv_bfloat16*>(sm + a.off_wrecv); // pair mode, written by the peer: [my rows of W^T][RT]
   int* rtab = reinterpret_cast<int*>(sm + a.off_rtab);                       // [RT] head slot of an expansion row, -1 if unused
   float* yred = reinterpret_cast<float*>(sm + a.off_yred);                   // [VW][yhg][D]
   const float qscale = 0.08838834764831845f * 1.4426950408889634f;   // sigma = 1/sqrt(128), logits kept in log2 units
@@ -310,7 +328,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     for (int u = blockIdx.x; u < a.units; u += gridDim.x, ++ucount) {
       const int h = u / per_h, rem = u - h * per_h;
       const int bg = rem / a.nrg, rg = rem - bg * a.nrg;
-      const int b0 = bg * a.NB, r0 = rg * a.RB;
+      const int b0 = bg * a.NB, r0 = PAIR ? 0 : rg * a.RB;
       const int nbv = min(a.NB, a.B - b0);
       const int rbv = min(RB, a.R - r0);
       (void)h;
@@ -414,7 +432,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars.l_free);
       named_barrier_arrive(BAR_P_READY, TEW * 32 + 32);
-      named_barrier_sync(1, FCONS);                                   // B1: row sums here, maxima and sums of the text rows from the value warps
+      named_barrier_sync(2, TEW * 32);                                // row sums of every warp
       if (warp == 0) {
         for (int x = lane; x < RT; x += 32) {
           float s_ = 0.f;
@@ -422,54 +440,127 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
           for (int w = 0; w < TEW; ++w) s_ += rsum[w * RT + x];
           rsum[x] = s_;
         }
+      }
+      const int NS = (a.m + 15) >> 4;
+      // rows of W^T this CTA turns into weight tiles; in pair mode the other rows go to the peer
+      const int oj0 = (PAIR && rg) ? NJ0 * rows16 : 0;
+      const int oj1 = PAIR ? min(NS * 16, (rg ? a.NJ : NJ0) * rows16) : NS * 16;
+      wait_on(&bars.w_done, ucount & 1u);
+      tc_fence_after();
+      if constexpr (PAIR) {
+        // ---- send: maxima and row sums of my columns, and my partial weights of the peer's rows (bf16) ----
+        const uint32_t peer = (uint32_t)rg ^ 1u;
+        if (ucount > 0 && !dead && !mbar_wait_cluster_bounded(&bars.x_ack, (ucount - 1) & 1u)) dead = true;   // the peer is done with my previous send
         __syncwarp();
+        if (warp == 0) {
+          const uint32_t xs = map_to_cta(smem_addr(xstat), peer);
+          for (int x = lane; x < 16; x += 32) st_cluster_f32(xs + 4u * x, hvmax[x]);
+          for (int x = lane; x < RT; x += 32) st_cluster_f32(xs + 4u * (16 + x), rsum[x]);
+        }
+        const int pj0 = rg ? 0 : NJ0 * rows16, pj1 = rg ? min(NS * 16, NJ0 * rows16) : NS * 16;
+        const uint32_t wr = map_to_cta(smem_addr(wrecv), peer);
+        for (int t = wh; t < MTL; t += TSTEP) {
+          const bool t64 = w_tail64 && t == MTL - 1;
+          const int j = t * 128 + (t64 ? wq * 16 : wq * 32) + lane;
+          const bool mine = j >= pj0 && j < pj1 && (!t64 || lane < 16);
+#pragma unroll
+          for (int hh = 0; hh < MT; ++hh) {
+            float v[16];
+            __syncwarp();
+            tmem_ld_x16(tq + w_col + (uint32_t)(t * RT + hh * 16), v);
+            if (mine) {
+              const uint32_t dst = wr + (uint32_t)(((j - pj0) * RT + hh * 16) * 2);
+#pragma unroll
+              for (int k = 0; k < 8; ++k) st_cluster_u32(dst + 4u * k, pack2_bf16(v[2 * k], v[2 * k + 1]));
+            }
+          }
+        }
+        named_barrier_sync(2, TEW * 32);                              // every warp has sent
+        if (tid == 0) mbar_arrive_cluster(map_to_cta(smem_addr(&bars.x_data), peer));
+        if (!dead && !mbar_wait_cluster_bounded(&bars.x_data, ucount & 1u)) dead = true;   // the peer's half has landed
+        __syncwarp();
+      }
+      named_barrier_sync(1, FCONS);                                   // B1: maxima and sums of the text rows from the value warps
+      if (warp == 0) {
         for (int x = lane; x < a.NB * 16; x += 32) {
           const int tb_ = x >> 4, g = x & 15;
-          float M = 0.f, fv = 0.f, vs = 0.f, tsm = 0.f;
+          float M = 0.f, fo = 0.f, fp = 0.f, vs = 0.f, tsm = 0.f;
           if (g < G && tb_ < nbv) {
-            M = hvmax[x];
+            float Mv = hvmax[x];
+            if constexpr (PAIR) Mv = fmaxf(Mv, xstat[x]);            // vision maximum over both halves of the columns
+            M = Mv;
             for (int w = tb_ * WPG; w < (tb_ + 1) * WPG; ++w) M = fmaxf(M, tmax[w * 16 + g]);
-            fv = fast_exp2(hvmax[x] - M);
+            fo = fast_exp2(hvmax[x] - M);
             for (int rl = 0; rl < rbv; ++rl) vs += rsum[(tb_ * RB + rl) * G + g];
-            vs *= fv;
+            vs *= fo;
+            if constexpr (PAIR) {
+              fp = fast_exp2(xstat[x] - M);
+              float vp = 0.f;
+              for (int rl = 0; rl < rbv; ++rl) vp += xstat[16 + (tb_ * RB + rl) * G + g];
+              vs = rg ? 0.f : fmaf(vp, fp, vs);                      // the sum of the vision probabilities is counted by CTA 0 alone
+            }
             for (int w = tb_ * WPG; w < (tb_ + 1) * WPG; ++w) {
               const float tm_ = tmax[w * 16 + g];
               if (tm_ != -INFINITY) tsm = fmaf(tsum[w * 16 + g], fast_exp2(tm_ - M), tsm);
             }
           }
           hmax[x] = M;
-          hfv[x] = fv;
+          hfv[x] = fo;
+          hfp[x] = fp;
           vsum[x] = vs;
           hsum[x] = vs + tsm;
         }
-      }
-      named_barrier_sync(1, FCONS);                                   // B2: joint maxima, sums and the vision factor
-
-      // ---------------- W^T (all m rows) from tensor memory to the weight tiles, at the joint maximum ----------------
-      float fvr[RT];
-#pragma unroll
-      for (int r = 0; r < RT; ++r) {
-        const int slot_ = rtab[r];
-        fvr[r] = slot_ >= 0 ? hfv[slot_] : 0.f;
-      }
-      wait_on(&bars.w_done, ucount & 1u);
-      __syncwarp();
-      tc_fence_after();
-      const int NS = (a.m + 15) >> 4;
-      for (int t = wh; t < MTL; t += TSTEP) {
-        float v[RT];
         __syncwarp();
-        tmem_ld<RT>(tq + w_col + (uint32_t)(t * RT), v);
+        for (int x = lane; x < RT; x += 32) {                        // factors of every expansion row
+          const int slot_ = rtab[x];
+          rowf[x] = slot_ >= 0 ? hfv[slot_] : 0.f;
+          rowf[RT + x] = slot_ >= 0 ? hfp[slot_] : 0.f;
+        }
+      }
+      named_barrier_sync(1, FCONS);                                   // B2: joint maxima, sums and the factors
+
+      // ---------------- my rows of W^T from tensor memory to the weight tiles, at the joint maximum ----------------
+      for (int t = wh; t < MTL; t += TSTEP) {
         const bool t64 = w_tail64 && t == MTL - 1;                   // a 64-row tile: 16 rows in the first lanes of every quarter
         const int j = t * 128 + (t64 ? wq * 16 : wq * 32) + lane;    // row of U
-        if (j < NS * 16 && (!t64 || lane < 16)) {
-          __nv_bfloat16* wt = W_sm + (j >> 4) * ((RT + 16) * SLD) + (j & 15);
+        const bool mine = j >= oj0 && j < oj1 && (!t64 || lane < 16);
+        __nv_bfloat16* wt = W_sm + ((j - oj0) >> 4) * ((RT + 16) * SLD) + (j & 15);
 #pragma unroll
-          for (int r = 0; r < RT; ++r) wt[r * SLD] = __float2bfloat16_rn(v[r] * fvr[r]);
+        for (int hh = 0; hh < MT; ++hh) {
+          float v[16];
+          __syncwarp();
+          tmem_ld_x16(tq + w_col + (uint32_t)(t * RT + hh * 16), v);
+          if (mine) {
+            if constexpr (PAIR) {
+              const uint4* rp = reinterpret_cast<const uint4*>(wrecv + (j - oj0) * RT + hh * 16);
+              const uint4 r0_ = rp[0], r1_ = rp[1];
+              const uint32_t rw[8] = {r0_.x, r0_.y, r0_.z, r0_.w, r1_.x, r1_.y, r1_.z, r1_.w};
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {
+                const float2 pr = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&rw[k]));
+                v[2 * k] = fmaf(pr.x, rowf[RT + hh * 16 + 2 * k], v[2 * k] * rowf[hh * 16 + 2 * k]);
+                v[2 * k + 1] = fmaf(pr.y, rowf[RT + hh * 16 + 2 * k + 1], v[2 * k + 1] * rowf[hh * 16 + 2 * k + 1]);
+              }
+            } else {
+#pragma unroll
+              for (int r = 0; r < 16; ++r) v[r] *= rowf[hh * 16 + r];
+            }
+#pragma unroll
+            for (int r = 0; r < 16; ++r) wt[(hh * 16 + r) * SLD] = __float2bfloat16_rn(v[r]);
+          }
         }
       }
       tc_fence_before();
+      if constexpr (PAIR) {
+        named_barrier_sync(2, TEW * 32);                              // what the peer sent has been consumed
+        if (tid == 0) mbar_arrive_cluster(map_to_cta(smem_addr(&bars.x_ack), (uint32_t)rg ^ 1u));
+      }
       named_barrier_arrive(BAR_W_READY, FCONS);
+    }
+    if constexpr (PAIR) {
+      // the peer's last acknowledgement arrives in this CTA's shared memory: stay until it is there
+      if (ucount > 0 && !dead && !mbar_wait_cluster_bounded(&bars.x_ack, (ucount - 1) & 1u)) dead = true;
+      __syncwarp();
     }
     named_barrier_sync(BAR_END, (CW + 1) * 32);
     if (dead && lane == 0) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
@@ -493,11 +584,13 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   for (int u = blockIdx.x; u < a.units; u += gridDim.x) {
     const int h = u / per_h, rem = u - h * per_h;
     const int bg = rem / a.nrg, rg = rem - bg * a.nrg;
-    const int b0 = bg * a.NB, r0 = rg * a.RB;
+    const int b0 = bg * a.NB, r0 = PAIR ? 0 : rg * a.RB;
     const int nbv = min(a.NB, a.B - b0);
     const int rbv = min(RB, a.R - r0);
     const RowRanges tr = row_ranges(a, rg);
     const int nts = tr.na + tr.nb;
+    const int c2first = (PAIR && rg) ? NJ0 : 0, c2count = PAIR ? (rg ? a.NJ - NJ0 : NJ0) : a.NJ;
+    (void)r0;
 
     // ---- queries of the unit's sequences: [NB][16 heads][128], heads >= G and absent sequences are zero rows
     for (int idx = vtid; idx < a.NB * 256; idx += VTH) {
@@ -709,10 +802,10 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
 
     // ---------------- y^T[128][heads] += V^T[128][16 rows of block] W^T[16][heads of block], all weights in place ----------------
     named_barrier_sync(BAR_W_READY, FCONS);
-    for (int c = 0; c < a.NJ; ++c) {
+    for (int c = 0; c < c2count; ++c) {
       wait_on(&bars.full[slot], phase);
       const uint32_t v_u = sm_u + slot * a.stage_bytes + a.par_bytes;
-      const int nsub = min(JC, (a.m - c * rows16 + 15) >> 4);
+      const int nsub = min(JC, (a.m - (c2first + c) * rows16 + 15) >> 4);
       const int ntask = RB * msplit;
       for (int task = wig; task < nsub * ntask; task += WPG) {          // my (sub-chunk, block, row-tile group) tasks
         const int s = task / ntask, tk = task - s * ntask;
@@ -920,7 +1013,7 @@ FusedPlan plan_fused_tc(const kvc_layer* L, int B, int R) {
   p.off_wred = 0;
   p.off_rstat = take((uint32_t)2 * p.EW * rt * 4);
   p.off_tstat = take((uint32_t)2 * p.VW * 16 * 4);
-  p.off_hstat = take((uint32_t)5 * p.NB * 16 * 4);
+  p.off_hstat = take((uint32_t)(6 * p.NB * 16 + 2 * rt) * 4);
   p.off_rtab = take((uint32_t)rt * 4);
   p.misc_bytes = off;
   const int nt = (n + 127) / 128;
@@ -939,23 +1032,117 @@ FusedPlan plan_fused_tc(const kvc_layer* L, int B, int R) {
   return p;
 }
 
-template <int EW, int VW, int NH, int MT>
+// Pair mode: one (sequence, KV head) per cluster of two CTAs, all its blocks in one unit of up to 64 expansion rows.
+FusedPlan plan_fused_pair(const kvc_layer* L, int B, int R) {
+  FusedPlan p{};
+  const int G = L->G, n = L->desc.n, m = L->m, H_kv = L->desc.H_kv;
+  if (L->desc.dtype != KVC_BF16 || L->passthrough || R < 1 || B < 1 || n % 256 != 0 || n > 1024 || G > 16 || R * G > 64 || m < 32) return p;
+  if (reinterpret_cast<uintptr_t>(L->desc.theta) & 15 || reinterpret_cast<uintptr_t>(L->desc.U) & 15) return p;
+  if ((long long)B * H_kv > KVC_MAX_COUNTERS) return p;
+  const int sms = L->num_sms > 0 ? L->num_sms : 148;
+  p.tc = 2;
+  p.EW = 8; p.VW = 6; p.ktw = 0;
+  p.MT = 4;
+  const int rt = ROWS * p.MT;
+  p.NB = 1; p.RB = R; p.nbg = B;
+  p.nrg = 2;                                   // the two CTAs of a pair leave two partial outputs per (sequence, head)
+  p.units = H_kv * B * 2;
+  p.ncg = n / 64;
+  const int ncgl = p.ncg / 2;
+  const uint32_t chunk = (uint32_t)R * 4096u + (uint32_t)(n / 2) * 32u;
+  int jc = (int)(49152u / chunk);
+  const int jmax = ceil_div(m, 32) < 16 ? ceil_div(m, 32) : 16;       // at least two stages along m: one per CTA in the value pass
+  p.JC = jc < 1 ? 1 : (jc > jmax ? jmax : jc);
+  p.NJ = ceil_div(m, 16 * p.JC);
+  if (p.NJ < 2) return p;
+  p.par_bytes = (uint32_t)ncgl * p.JC * 2048u;
+  p.k_half_bytes = (uint32_t)R * p.JC * 2048u;
+  p.stage_bytes = p.par_bytes + 2 * p.k_half_bytes;
+  if (p.stage_bytes < 16384u) p.stage_bytes = 16384u;
+  const int mtiles = ceil_div(m, 128);
+  p.UT = (int)(p.stage_bytes / 16384u) < mtiles ? (int)(p.stage_bytes / 16384u) : mtiles;
+  p.nu = ncgl * ceil_div(mtiles, p.UT);
+  int tch = (int)(p.stage_bytes / 512u) & ~15;
+  p.TCH = tch > 256 ? 256 : tch;
+  if (p.TCH < 16) return p;
+  p.txt_half_bytes = (uint32_t)p.TCH * 128u;
+  {
+    int best = 1 << 30;
+    for (int sh = 3; sh >= 0; --sh) {
+      const int ms = 8 >> sh, cost = ceil_div(p.JC * p.RB * ms, p.VW) * ((1 << sh) + 1);
+      if (cost < best) { best = cost; p.msplit = ms; p.mshift = sh; }
+    }
+  }
+  p.sld = 0;
+  p.yhg = G > 4 ? 8 : (G > 2 ? 4 : 2);
+  uint32_t off = 0;
+  auto take = [&](uint32_t bytes) { uint32_t o = off; off = (off + bytes + 127u) & ~127u; return o; };
+  const int nj0 = (p.NJ + 1) / 2;                                      // stages of the m axis of CTA 0 (the larger share)
+  const uint32_t p_bytes = (uint32_t)rt * (n / 2) * 2, yred_bytes = (uint32_t)p.VW * p.yhg * D * 4;
+  const uint32_t w_bytes = (uint32_t)nj0 * p.JC * (rt + 16) * SLD * 2;
+  uint32_t r0_bytes = p_bytes > yred_bytes ? p_bytes : yred_bytes;
+  if (w_bytes > r0_bytes) r0_bytes = w_bytes;
+  p.off_P = take(r0_bytes);
+  p.off_yred = p.off_P;
+  p.off_W = p.off_P;
+  p.off_wrecv = take((uint32_t)nj0 * p.JC * 16 * rt * 2);
+  p.off_xstat = take((uint32_t)(16 + rt) * 4);
+  p.off_q = take((uint32_t)16 * QLD * 2);
+  p.off_S = take((uint32_t)(2 * p.JC * rt * 32));
+  p.off_wred = 0;
+  p.off_rstat = take((uint32_t)2 * p.EW * rt * 4);
+  p.off_tstat = take((uint32_t)2 * p.VW * 16 * 4);
+  p.off_hstat = take((uint32_t)(6 * 16 + 2 * rt) * 4);
+  p.off_rtab = take((uint32_t)rt * 4);
+  p.misc_bytes = off;
+  int cols = 32;
+  while (cols < (n / 256) * rt + mtiles * rt) cols *= 2;
+  p.tmem_cols = cols;
+  if (cols > 512) return p;
+  if (SMEM_LIMIT < 1024u + 2048u + p.misc_bytes + 2 * p.stage_bytes) return p;
+  const uint32_t avail = SMEM_LIMIT - 1024u - 2048u - p.misc_bytes;
+  int stages = (int)(avail / p.stage_bytes);
+  p.stages = stages > FMAX_STAGES ? FMAX_STAGES : stages;
+  if (p.stages < 2) return p;
+  p.smem_bytes = (size_t)p.stages * p.stage_bytes + p.misc_bytes + 1024u;
+  const int pairs = p.units / 2, slots = sms / 2;
+  p.grid = 2 * (pairs < slots ? pairs : slots);
+  p.ok = 1;
+  return p;
+}
+
+template <int EW, int VW, int NH, int MT, bool PAIR>
 static cudaError_t launch_tc_inst(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
   static size_t configured = 0;
   if (p.smem_bytes > configured) {
-    cudaError_t e = cudaFuncSetAttribute(fused_decode_tc_kernel<EW, VW, NH, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
+    cudaError_t e = cudaFuncSetAttribute(fused_decode_tc_kernel<EW, VW, NH, MT, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
     if (e != cudaSuccess) return e;
     configured = p.smem_bytes;
   }
-  return launch_dependent(fused_decode_tc_kernel<EW, VW, NH, MT>, dim3(p.grid), dim3((EW + VW + 2) * 32), p.smem_bytes, st, tm[0], tm[1],
-                          tm[2], tm[3], tm[4], tm[5], fa);
+  if (!PAIR)
+    return launch_dependent(fused_decode_tc_kernel<EW, VW, NH, MT, PAIR>, dim3(p.grid), dim3((EW + VW + 2) * 32), p.smem_bytes, st, tm[0],
+                            tm[1], tm[2], tm[3], tm[4], tm[5], fa);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(p.grid);
+  cfg.blockDim = dim3((EW + VW + 2) * 32);
+  cfg.dynamicSmemBytes = p.smem_bytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = 2; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, fused_decode_tc_kernel<EW, VW, NH, MT, PAIR>, tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], fa);
 }
 
 template <int NH>
 static cudaError_t launch_tc_nh(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
-  if (p.EW == 8) return launch_tc_inst<8, 6, NH, 2>(tm, fa, p, st);
-  if (p.VW == 8) return p.MT == 2 ? launch_tc_inst<4, 8, NH, 2>(tm, fa, p, st) : launch_tc_inst<4, 8, NH, 1>(tm, fa, p, st);
-  return launch_tc_inst<4, 10, NH, 1>(tm, fa, p, st);
+  if (p.tc == 2) return launch_tc_inst<8, 6, NH, 4, true>(tm, fa, p, st);
+  if (p.EW == 8) return launch_tc_inst<8, 6, NH, 2, false>(tm, fa, p, st);
+  if (p.VW == 8) return p.MT == 2 ? launch_tc_inst<4, 8, NH, 2, false>(tm, fa, p, st) : launch_tc_inst<4, 8, NH, 1, false>(tm, fa, p, st);
+  return launch_tc_inst<4, 10, NH, 1, false>(tm, fa, p, st);
 }
 
 cudaError_t launch_fused_tc_kernel(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {

@@ -92,8 +92,8 @@ struct FusedPlan {
   int stages, grid;
   uint32_t par_bytes, k_half_bytes, txt_half_bytes, stage_bytes, misc_bytes;
   uint32_t off_q, off_S, off_W, off_wred, off_rstat, off_tstat, off_hstat, off_yred;   // relative to the end of the ring
-  int tc;            // 1: the expansions run on tcgen05 with the logits in tensor memory (kvc_fused_tc.cu)
-  uint32_t off_P, off_rtab;
+  int tc;            // 1: the expansions run on tcgen05 with the logits in tensor memory (kvc_fused_tc.cu); 2: its pair mode
+  uint32_t off_P, off_rtab, off_xstat, off_wrecv;
   int tmem_cols;
   int UT, nu;        // 128-row tiles of U per stage and stages of U per unit (tensor-memory variant)
   size_t smem_bytes;
@@ -109,8 +109,8 @@ struct kvc_layer {
   int passthrough;       // ratio_permille == 0
   int device;
   int num_sms;
-  int use_tc;            // expansions of the one-kernel decode path: 0 chosen per shape, 1 tcgen05, -1 mma.sync (environment
-                         // KVC_EXPANSION=tcgen05 | mma when the handle is created)
+  int use_tc;            // expansions of the one-kernel decode path: 0 chosen per shape, 1 tcgen05, 2 tcgen05 in pairs of CTAs,
+                         // -1 mma.sync (environment KVC_EXPANSION=tcgen05 | pair | mma when the handle is created)
   int32_t* d_idx;        // device [H_kv][m]
   int* d_cnt;            // device [KVC_MAX_COUNTERS + 1] arrival counters of the one-kernel decode path (zero between
                          // calls), then the status word of the compress kernels
@@ -123,6 +123,7 @@ WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap);
 int cuda_status(cudaError_t e);   // KVC_OK or KVC_ERR_CUDA, remembering the error for kvc_last_cuda_error
 FusedPlan plan_fused(const kvc_layer* L, int B, int R);
 FusedPlan plan_fused_tc(const kvc_layer* L, int B, int R);     // tensor-memory variant; ok == 0 if the shape does not fit it
+FusedPlan plan_fused_pair(const kvc_layer* L, int B, int R);   // its pair mode (clusters of two CTAs)
 FusedPlan plan_fused_text(const kvc_layer* L, int B, int T);   // R == 0: text rows only
 
 struct DecodeArgs {

@@ -80,6 +80,7 @@ const char* kvc_kernel_name(int kernel_id) {
     case KVC_KERNEL_COMBINE: return "combine";
     case KVC_KERNEL_FUSED: return "fused";
     case KVC_KERNEL_FUSED_TC: return "fused_tc";
+    case KVC_KERNEL_FUSED_PAIR: return "fused_pair";
     default: return "?";
   }
 }

@@ -269,6 +269,24 @@ def test_one_kernel_path_edges(B, H_q, H_kv, grid, R, T):
 
 
 @pytest.mark.parametrize("B,H_q,H_kv,grid,R,T,ratio", [
+    (2, 14, 2, 32, 8, 70, 600),     # the Qwen2-VL head layout: 56 expansion rows per (sequence, KV head)
+    (1, 14, 2, 16, 3, 0, 600),      # n = 256: one logit tile per CTA; no text rows
+    (3, 4, 4, 16, 5, 33, 600),      # MHA, odd batch
+    (1, 16, 1, 32, 4, 20, 800),     # G = 16: two head tiles, 64 expansion rows, m = 205
+    (1, 14, 2, 32, 2, 300, 950),    # m = 52: one stage of the m axis per CTA, a 64-row tile of W^T
+    (20, 8, 8, 16, 2, 37, 600),     # more pairs than SM pairs: buffers, barriers and acknowledgements reused across units
+])
+def test_tensor_memory_variant_in_pairs_of_ctas(B, H_q, H_kv, grid, R, T, ratio, monkeypatch):
+    """Clusters of two CTAs per (sequence, KV head): each keeps half of the columns of the logits, partial weights cross
+    through distributed shared memory (chosen with KVC_EXPANSION=pair)."""
+    monkeypatch.setenv("KVC_EXPANSION", "pair")
+    shape = wl.Shape("tc-pair", 1, B, H_q, H_kv, 128, grid, R, T, 1, "bf16", ratio_permille=ratio)
+    p = tl.make_problem(shape, 210 + B + 7 * R + T, T=T, T_cap=T + 5)
+    counts = _fused_launches(lambda: _check(shape, p))
+    assert counts["fused_pair"] >= 1 and counts["fused_tc"] == 0 and counts["fused"] == 0 and counts["scores"] == 0
+
+
+@pytest.mark.parametrize("B,H_q,H_kv,grid,R,T,ratio", [
     (2, 14, 2, 32, 4, 0, 600),      # no text rows: only stages of U between the two passes
     (1, 14, 2, 32, 5, 300, 950),    # m = 52: one tile of W^T, taken with M = 64
     (1, 14, 2, 32, 3, 17, 850),     # m = 154: a full tile and a 26-row tile
