@@ -39,9 +39,9 @@ NCU_TRAFFIC_BYTES = {
     # profiles/fused_decode_config1.md: 185.7 MB read + 6.6 MB written per launch at T = 130 text rows; a text row costs
     # 2 * B * H_kv * d * 2 bytes = 131072 bytes more, so the mid-run launch (T = 255.5) moves 192.3 MB + 16.4 MB
     ("fused", "config1-llava-next-7b"): 208.7e6,
-    # profiles/fused_decode_tc_config2.md: 123.0 MB read + 4.6 MB written per launch at T = 258; 32768 bytes per text
+    # profiles/fused_decode_tc_config2.md: 123.0 MB read + 4.2 MB written per launch at T = 258; 32768 bytes per text
     # row more up to the mid-run launch (T = 511.5)
-    ("fused_tc", "config2-qwen2-vl-7b"): 136.0e6,
+    ("fused_tc", "config2-qwen2-vl-7b"): 135.5e6,
 }
 
 
