@@ -154,6 +154,12 @@ KVC_API int kvc_decode_attend_static(const kvc_layer* layer, const void* q, cons
 KVC_API int kvc_read_device_status(const kvc_layer* layer, int B, int R, int T, const void* workspace,
                                    int* status_out);
 
+/* Self-test of the bounded device-side waits: one warp waits on a shared-memory barrier that nothing ever
+ * completes, with the wait every kernel of this library uses.  Returns KVC_ERR_TIMEOUT when the wait gave up
+ * as designed (after about a second) and KVC_OK if it returned as complete (a defect); the CUDA context stays
+ * usable either way.  Allocates and frees 4 bytes of device memory and synchronises `stream`. */
+KVC_API int kvc_selftest_bounded_wait(void* stream);
+
 /* Integer maps as the device path uses them (read back from the device copy):
  * idx_out: HOST [H_kv][m] retained indices per KV head; group_out: HOST [R*n][2] = (block r,
  * offset i) of vision token t = r*n + i (the Reshape of Alg. 1 step 1).  Either may be NULL. */

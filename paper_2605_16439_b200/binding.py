@@ -58,6 +58,7 @@ def _lib() -> C.CDLL:
         lib.kvc_static_scratch_bytes.argtypes = []; lib.kvc_static_scratch_bytes.restype = C.c_size_t
         lib.kvc_read_device_status.argtypes = [vp, i, i, i, vp, C.POINTER(i)]
         lib.kvc_read_device_status.restype = i
+        lib.kvc_selftest_bounded_wait.argtypes = [vp]; lib.kvc_selftest_bounded_wait.restype = i
         lib.kvc_export_maps.argtypes = [vp, i, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         lib.kvc_export_maps.restype = i
         lib.kvc_strerror.argtypes = [i]; lib.kvc_strerror.restype = C.c_char_p
@@ -181,6 +182,11 @@ def kvc_read_device_status(layer: Layer, B: int, R: int, T: int, workspace) -> i
     _check(_lib().kvc_read_device_status(layer.handle, B, R, T, _ptr(workspace), C.byref(out)),
            "kvc_read_device_status")
     return out.value
+
+
+def kvc_selftest_bounded_wait(stream=None) -> int:
+    """Status of a device-side wait that nothing completes: KVC_ERR_TIMEOUT (-7) when the bound works."""
+    return int(_lib().kvc_selftest_bounded_wait(_stream(stream)))
 
 
 def kvc_export_maps(layer: Layer, R: int):

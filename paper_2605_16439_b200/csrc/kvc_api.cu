@@ -298,6 +298,24 @@ int kvc_attend_full(const kvc_layer* L, const void* q, const void* K, const void
   return decode_common(L, q, nullptr, B, 0, K, V, S, S_cap, out, workspace, static_cast<cudaStream_t>(stream));
 }
 
+int kvc_selftest_bounded_wait(void* stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int* d_status = nullptr;
+  cudaError_t e = cudaMalloc(&d_status, sizeof(int));
+  if (e != cudaSuccess) return cuda_status(e);
+  int h_status = KVC_ERR_CUDA;
+  e = cudaMemsetAsync(d_status, 0, sizeof(int), st);
+  if (e == cudaSuccess) {
+    kvc::launch_wait_selftest(d_status, st);
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) e = cudaMemcpyAsync(&h_status, d_status, sizeof(int), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  cudaFree(d_status);
+  if (e != cudaSuccess) return cuda_status(e);
+  return h_status;
+}
+
 int kvc_read_device_status(const kvc_layer* L, int B, int R, int T, const void* workspace, int* status_out) {
   if (!L || !workspace || !status_out || B < 0 || R < 0 || T < 0) return KVC_ERR_ARG;
   const WsLayout w = ws_layout(L, B, R, T);

@@ -320,6 +320,15 @@ def test_tensor_memory_variant_of_the_expansions(B, H_q, H_kv, grid, R, T, monke
     assert counts["fused_tc"] >= 1 and counts["fused"] == 0 and counts["scores"] == 0
 
 
+def test_a_wait_that_nothing_completes_gives_up_and_the_context_stays_usable():
+    """Every device-side wait of the library is bounded: the self-test kernel waits on a barrier nobody arrives on and
+    must come back with KVC_ERR_TIMEOUT (about a second); afterwards an ordinary decode call still runs and is correct."""
+    assert kvc.kvc_selftest_bounded_wait() == -7
+    shape = tl.small(wl.CONFIGS[1], B=2, H_q=4, H_kv=4)
+    p = tl.make_problem(shape, 161, T=40, T_cap=48)
+    _check(shape, p)
+
+
 def test_more_units_than_sms_and_status_word_clean():
     """Persistent CTAs walk several work units each (ring parity carried across units)."""
     shape = wl.Shape("many-units", 1, 40, 8, 8, 128, 8, 2, 37, 1, "bf16")      # 8 * 40 = 320 units of one sequence
