@@ -85,7 +85,9 @@ static cudaError_t launch_compress_t(const kvc_layer* L, const void* K_vis, cons
   ProfScope prof(KVC_KERNEL_PROJECT_VALUES, st);
   {
     bool used = false;
-    e = launch_project_values_mma(L, V_vis, B, R, Vc, st, &used);      // bf16: tensor cores
+    e = launch_project_values_tc(L, V_vis, B, R, Vc, st, &used);       // bf16: tcgen05, accumulator in tensor memory
+    if (used || e != cudaSuccess) return e;
+    e = launch_project_values_mma(L, V_vis, B, R, Vc, st, &used);      // bf16: mma.sync (kept as the comparison kernel)
     if (used || e != cudaSuccess) return e;
   }
   dim3 grid((unsigned)(B * H_kv * R), (unsigned)ceil_div(m, 32));

@@ -197,6 +197,7 @@ cudaError_t launch_output(const DecodeArgs& a, int dtype, cudaStream_t st);
 cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPlan& p, cudaStream_t st, bool* encoded);
 void launch_wait_selftest(int* status, cudaStream_t st);   // one warp, a wait that runs out: *status = KVC_ERR_TIMEOUT
 cudaError_t compute_usum(const kvc_layer* L, float* usum);
+cudaError_t launch_project_values_tc(const kvc_layer* L, const void* V_vis, int B, int R, void* Vc, cudaStream_t st, bool* used);
 cudaError_t launch_project_values_mma(const kvc_layer* L, const void* V_vis, int B, int R, void* Vc, cudaStream_t st, bool* used);
 cudaError_t launch_compress(const kvc_layer* L, const void* K_vis, const void* V_vis, int B, int R,
                             void* Kc, void* Vc, cudaStream_t st);
