@@ -320,6 +320,35 @@ def test_tensor_memory_variant_of_the_expansions(B, H_q, H_kv, grid, R, T, monke
     assert counts["fused_tc"] >= 1 and counts["fused"] == 0 and counts["scores"] == 0
 
 
+def _random_shapes(count, seed):
+    """Seeded random shapes the one-kernel path serves: block lengths that are multiples of 64, up to 16 heads per KV head."""
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < count:
+        grid = int(rng.choice([8, 16, 24, 32]))
+        G = int(rng.choice([1, 2, 4, 7, 8, 12, 16]))
+        H_kv = int(rng.integers(1, 4))
+        B = int(rng.integers(1, 6))
+        R = int(rng.integers(1, 10))
+        T = int(rng.choice([0, 1, 15, 16, 17, 100, 333]))
+        ratio = int(rng.choice([100, 350, 600, 800, 950]))
+        if B * H_kv * R * grid * grid > 60000:        # keep the oracle fast
+            continue
+        out.append((B, G * H_kv, H_kv, grid, R, T, ratio))
+    return out
+
+
+@pytest.mark.parametrize("variant", ["mma", "tcgen05", "pair"])
+def test_random_shapes_through_every_variant_of_the_one_kernel_path(variant, monkeypatch):
+    """The same seeded random shapes through the mma.sync kernel, the tensor-memory kernel and its pair mode (a shape
+    a variant does not serve falls to the next one: the result must be right whichever kernel ran)."""
+    monkeypatch.setenv("KVC_EXPANSION", variant)
+    for k, (B, H_q, H_kv, grid, R, T, ratio) in enumerate(_random_shapes(10, 20260 + len(variant))):
+        shape = wl.Shape(f"rand-{variant}-{k}", 1, B, H_q, H_kv, 128, grid, R, T, 1, "bf16", ratio_permille=ratio)
+        p = tl.make_problem(shape, 300 + k, T=T, T_cap=T + 3)
+        _check(shape, p)
+
+
 def test_a_wait_that_nothing_completes_gives_up_and_the_context_stays_usable():
     """Every device-side wait of the library is bounded: the self-test kernel waits on a barrier nobody arrives on and
     must come back with KVC_ERR_TIMEOUT (about a second); afterwards an ordinary decode call still runs and is correct."""
