@@ -84,7 +84,7 @@ KVC_API int kvc_retained_len(int n, int ratio_permille);
  * bf16 decode calls run Alg. 1 steps 2-3 either on mma.sync with the logits in registers or on tcgen05 with the
  * logits in tensor memory; the library picks per shape (same results within the bf16 tolerance).  The environment
  * variable KVC_EXPANSION = "tcgen05" | "mma", read when the handle is created, forces one of them where it applies;
- * "pair" selects the tcgen05 path run by clusters of two CTAs per (sequence, KV head) (experimental: correct, slower). */
+ * "pair" the tcgen05 path run by clusters of two CTAs per (sequence, KV head). */
 KVC_API int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out);
 KVC_API int kvc_layer_destroy(kvc_layer* layer);
 

@@ -780,9 +780,10 @@ FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
     // The tensor-memory variant pays per tcgen05.mma, not per expansion row: it wins for long blocks once two row
     // tiles per unit still give most SMs a unit (measured on the n = 1024, G = 7 shape: ahead from batch 16 on,
     // behind at batches 1-4 where units of half the size halve the latency).
-    if (L->use_tc == 2) {
+    if (L->use_tc != 1) {
+      // pairs of CTAs per (sequence, KV head): ahead of the single-CTA variant on the n = 1024, G = 7 shape from batch 16 on
       const FusedPlan t2 = plan_fused_pair(L, B, R);
-      if (t2.ok) return t2;
+      if (t2.ok && (L->use_tc == 2 || (L->desc.n > 640 && t2.units >= 96))) return t2;
     }
     const FusedPlan t = plan_fused_tc(L, B, R);
     if (t.ok && (L->use_tc > 0 || (L->desc.n > 640 && t.MT == 2 && t.units >= 96))) return t;

@@ -343,9 +343,11 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         for (int x = lane; x < RT; x += 32) rtab[x] = row_slot(x);
 
       // ---------------- maxima of the logits, 16 expansion rows (one tensor-memory load) at a time ----------------
+      // (the loops over the 16-row groups are kept rolled: this code runs once per unit, and instruction fetch of the
+      // unrolled copies cost more than the loop overhead saves)
       wait_on(&bars.l_done, ucount & 1u);
       tc_fence_after();
-#pragma unroll
+#pragma unroll 1
       for (int hh = 0; hh < MT; ++hh) {
         float mx[16];
 #pragma unroll
@@ -391,7 +393,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       named_barrier_sync(2, TEW * 32);
 
       // ---------------- P = 2^(L - max) as the bf16 operand of the re-projection; row sums ----------------
-#pragma unroll
+#pragma unroll 1
       for (int hh = 0; hh < MT; ++hh) {
         float Mr[16], sum[16];                        // rows without a (sequence, block, head) get the reference +inf: P = 0
 #pragma unroll
@@ -463,15 +465,15 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
           const bool t64 = w_tail64 && t == MTL - 1;
           const int j = t * 128 + (t64 ? wq * 16 : wq * 32) + lane;
           const bool mine = j >= pj0 && j < pj1 && (!t64 || lane < 16);
-#pragma unroll
+#pragma unroll 1
           for (int hh = 0; hh < MT; ++hh) {
             float v[16];
             __syncwarp();
             tmem_ld_x16(tq + w_col + (uint32_t)(t * RT + hh * 16), v);
             if (mine) {
               const uint32_t dst = wr + (uint32_t)(((j - pj0) * RT + hh * 16) * 2);
-#pragma unroll
-              for (int k = 0; k < 8; ++k) st_cluster_u32(dst + 4u * k, pack2_bf16(v[2 * k], v[2 * k + 1]));
+              st_cluster_v4(dst, pack2_bf16(v[0], v[1]), pack2_bf16(v[2], v[3]), pack2_bf16(v[4], v[5]), pack2_bf16(v[6], v[7]));
+              st_cluster_v4(dst + 16u, pack2_bf16(v[8], v[9]), pack2_bf16(v[10], v[11]), pack2_bf16(v[12], v[13]), pack2_bf16(v[14], v[15]));
             }
           }
         }
@@ -525,7 +527,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         const int j = t * 128 + (t64 ? wq * 16 : wq * 32) + lane;    // row of U
         const bool mine = j >= oj0 && j < oj1 && (!t64 || lane < 16);
         __nv_bfloat16* wt = W_sm + ((j - oj0) >> 4) * ((RT + 16) * SLD) + (j & 15);
-#pragma unroll
+#pragma unroll 1
         for (int hh = 0; hh < MT; ++hh) {
           float v[16];
           __syncwarp();
@@ -1041,7 +1043,7 @@ FusedPlan plan_fused_pair(const kvc_layer* L, int B, int R) {
   if ((long long)B * H_kv > KVC_MAX_COUNTERS) return p;
   const int sms = L->num_sms > 0 ? L->num_sms : 148;
   p.tc = 2;
-  p.EW = 8; p.VW = 6; p.ktw = 0;
+  p.EW = 4; p.VW = 8; p.ktw = 0;
   p.MT = 4;
   const int rt = ROWS * p.MT;
   p.NB = 1; p.RB = R; p.nbg = B;
@@ -1139,7 +1141,7 @@ static cudaError_t launch_tc_inst(const CUtensorMap* tm, const FusedArgs& fa, co
 
 template <int NH>
 static cudaError_t launch_tc_nh(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
-  if (p.tc == 2) return launch_tc_inst<8, 6, NH, 4, true>(tm, fa, p, st);
+  if (p.tc == 2) return launch_tc_inst<4, 8, NH, 4, true>(tm, fa, p, st);
   if (p.EW == 8) return launch_tc_inst<8, 6, NH, 2, false>(tm, fa, p, st);
   if (p.VW == 8) return p.MT == 2 ? launch_tc_inst<4, 8, NH, 2, false>(tm, fa, p, st) : launch_tc_inst<4, 8, NH, 1, false>(tm, fa, p, st);
   return launch_tc_inst<4, 10, NH, 1, false>(tm, fa, p, st);
