@@ -43,7 +43,7 @@ struct TcBars {
   uint64_t l_done;         // the logits of the unit are complete
   uint64_t l_free;         // the logits of the unit have been read back (4 warps)
   uint64_t x_data;         // pair mode: the peer's statistics and partial weights of the unit have landed here
-  uint64_t x_ack;          // pair mode: the peer has consumed what this CTA sent for the unit
+  uint64_t x_ready;        // pair mode: the peer's re-projection of the unit is complete: its weight tiles may be written
 };
 
 // Reduces 16 per-lane values over the 32 lanes of a warp (maximum or sum) in 31 shuffles: after the first exchange
@@ -97,7 +97,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     mbar_init(&bars.l_done, 1);
     mbar_init(&bars.l_free, TEW);
     mbar_init(&bars.x_data, 1);
-    mbar_init(&bars.x_ack, 1);
+    mbar_init(&bars.x_ready, 1);
     fence_mbar_init();
   }
   if (warp == MMA_WARP) tmem_alloc(&s_tmem, (uint32_t)a.tmem_cols);
@@ -306,7 +306,6 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   float* hfp = hfv + a.NB * 16;                                              // pair mode: the same for the peer's partial weights
   float* rowf = hfp + a.NB * 16;                                             // [2][RT] those factors per expansion row
   float* xstat = reinterpret_cast<float*>(sm + a.off_xstat);                 // pair mode, written by the peer: [16] maxima, [RT] row sums
-  __nv_bfloat16* wrecv = reinterpret_cast<__nv_bfloat16*>(sm + a.off_wrecv); // pair mode, written by the peer: [my rows of W^T][RT]
   int* rtab = reinterpret_cast<int*>(sm + a.off_rtab);                       // [RT] head slot of an expansion row, -1 if unused
   float* yred = reinterpret_cast<float*>(sm + a.off_yred);                   // [VW][yhg][D]
   const float qscale = 0.08838834764831845f * 1.4426950408889634f;   // sigma = 1/sqrt(128), logits kept in log2 units
@@ -316,6 +315,10 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   const int lrowB = l7 + lhi * 8;                  // address pattern B: rows 0-7 | 0-7 | 8-15 | 8-15
   const int lmid = (lane >> 3) & 1;
   const int WPG = VW / a.NB;                       // value warps per sequence of the unit
+  // expansion rows of a block: G heads; pair mode pads them to 8 or 16 so that a block's rows start a 16-byte piece of the
+  // weight tiles, which it keeps as [row of U][expansion row] (the layout the peer CTA sends and this CTA adds to in place)
+  const int GP = PAIR ? (G <= 8 ? 8 : 16) : G;
+  constexpr int WLD = RT + 8;                      // pair mode: row stride of the weight tiles in elements
 
   if (warp < TEW) {
     // ======================================================================================================
@@ -335,9 +338,9 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       named_barrier_sync(2, TEW * 32);           // every warp is done with the previous unit's tables
       // expansion row rho <-> (sequence, block, head): head slot of the row, -1 if the unit has no such row
       auto row_slot = [&](int rho) {
-        const int bi = rho / G, g = rho - bi * G;
+        const int bi = rho / GP, g = rho - bi * GP;
         const int rbl = bi / RB, rrl = bi - rbl * RB;
-        return (rho < a.NB * RB * G && rbl < nbv && rrl < rbv) ? rbl * 16 + g : -1;
+        return (g < G && rho < a.NB * RB * GP && rbl < nbv && rrl < rbv) ? rbl * 16 + g : -1;
       };
       if (warp == 0)
         for (int x = lane; x < RT; x += 32) rtab[x] = row_slot(x);
@@ -385,7 +388,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
           float m_ = 0.f;
           if (g < G && tb_ < nbv) {
             m_ = -INFINITY;
-            for (int rl = 0; rl < rbv; ++rl) m_ = fmaxf(m_, rmax[(tb_ * RB + rl) * G + g]);
+            for (int rl = 0; rl < rbv; ++rl) m_ = fmaxf(m_, rmax[(tb_ * RB + rl) * GP + g]);
           }
           hvmax[x] = m_;
         }
@@ -450,9 +453,12 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       wait_on(&bars.w_done, ucount & 1u);
       tc_fence_after();
       if constexpr (PAIR) {
-        // ---- send: maxima and row sums of my columns, and my partial weights of the peer's rows (bf16) ----
+        // ---- my re-projection is complete and P is dead: the peer may write into my weight tiles (they share P's region);
+        // then send: maxima and row sums of my columns, and my partial weights of the peer's rows (bf16), straight into
+        // the peer's weight tiles ----
         const uint32_t peer = (uint32_t)rg ^ 1u;
-        if (ucount > 0 && !dead && !mbar_wait_cluster_bounded(&bars.x_ack, (ucount - 1) & 1u)) dead = true;   // the peer is done with my previous send
+        if (tid == 0) mbar_arrive_cluster(map_to_cta(smem_addr(&bars.x_ready), peer));
+        if (!dead && !mbar_wait_cluster_bounded(&bars.x_ready, ucount & 1u)) dead = true;
         __syncwarp();
         if (warp == 0) {
           const uint32_t xs = map_to_cta(smem_addr(xstat), peer);
@@ -460,7 +466,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
           for (int x = lane; x < RT; x += 32) st_cluster_f32(xs + 4u * (16 + x), rsum[x]);
         }
         const int pj0 = rg ? 0 : NJ0 * rows16, pj1 = rg ? min(NS * 16, NJ0 * rows16) : NS * 16;
-        const uint32_t wr = map_to_cta(smem_addr(wrecv), peer);
+        const uint32_t wr = map_to_cta(smem_addr(W_sm), peer);
         for (int t = wh; t < MTL; t += TSTEP) {
           const bool t64 = w_tail64 && t == MTL - 1;
           const int j = t * 128 + (t64 ? wq * 16 : wq * 32) + lane;
@@ -471,7 +477,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
             __syncwarp();
             tmem_ld_x16(tq + w_col + (uint32_t)(t * RT + hh * 16), v);
             if (mine) {
-              const uint32_t dst = wr + (uint32_t)(((j - pj0) * RT + hh * 16) * 2);
+              const uint32_t dst = wr + (uint32_t)(((j - pj0) * WLD + hh * 16) * 2);
               st_cluster_v4(dst, pack2_bf16(v[0], v[1]), pack2_bf16(v[2], v[3]), pack2_bf16(v[4], v[5]), pack2_bf16(v[6], v[7]));
               st_cluster_v4(dst + 16u, pack2_bf16(v[8], v[9]), pack2_bf16(v[10], v[11]), pack2_bf16(v[12], v[13]), pack2_bf16(v[14], v[15]));
             }
@@ -493,12 +499,12 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
             M = Mv;
             for (int w = tb_ * WPG; w < (tb_ + 1) * WPG; ++w) M = fmaxf(M, tmax[w * 16 + g]);
             fo = fast_exp2(hvmax[x] - M);
-            for (int rl = 0; rl < rbv; ++rl) vs += rsum[(tb_ * RB + rl) * G + g];
+            for (int rl = 0; rl < rbv; ++rl) vs += rsum[(tb_ * RB + rl) * GP + g];
             vs *= fo;
             if constexpr (PAIR) {
               fp = fast_exp2(xstat[x] - M);
               float vp = 0.f;
-              for (int rl = 0; rl < rbv; ++rl) vp += xstat[16 + (tb_ * RB + rl) * G + g];
+              for (int rl = 0; rl < rbv; ++rl) vp += xstat[16 + (tb_ * RB + rl) * GP + g];
               vs = rg ? 0.f : fmaf(vp, fp, vs);                      // the sum of the vision probabilities is counted by CTA 0 alone
             }
             for (int w = tb_ * WPG; w < (tb_ + 1) * WPG; ++w) {
@@ -526,7 +532,8 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         const bool t64 = w_tail64 && t == MTL - 1;                   // a 64-row tile: 16 rows in the first lanes of every quarter
         const int j = t * 128 + (t64 ? wq * 16 : wq * 32) + lane;    // row of U
         const bool mine = j >= oj0 && j < oj1 && (!t64 || lane < 16);
-        __nv_bfloat16* wt = W_sm + ((j - oj0) >> 4) * ((RT + 16) * SLD) + (j & 15);
+        __nv_bfloat16* wt = W_sm + ((j - oj0) >> 4) * ((RT + 16) * SLD) + (j & 15);      // [expansion row][row of U] tiles
+        __nv_bfloat16* wp = W_sm + (j - oj0) * WLD;                                       // pair mode: [row of U][expansion row]
 #pragma unroll 1
         for (int hh = 0; hh < MT; ++hh) {
           float v[16];
@@ -534,35 +541,28 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
           tmem_ld_x16(tq + w_col + (uint32_t)(t * RT + hh * 16), v);
           if (mine) {
             if constexpr (PAIR) {
-              const uint4* rp = reinterpret_cast<const uint4*>(wrecv + (j - oj0) * RT + hh * 16);
+              // the peer's partial sits where the result goes: add in place
+              uint4* rp = reinterpret_cast<uint4*>(wp + hh * 16);
               const uint4 r0_ = rp[0], r1_ = rp[1];
               const uint32_t rw[8] = {r0_.x, r0_.y, r0_.z, r0_.w, r1_.x, r1_.y, r1_.z, r1_.w};
+              uint32_t ow[8];
 #pragma unroll
               for (int k = 0; k < 8; ++k) {
                 const float2 pr = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&rw[k]));
-                v[2 * k] = fmaf(pr.x, rowf[RT + hh * 16 + 2 * k], v[2 * k] * rowf[hh * 16 + 2 * k]);
-                v[2 * k + 1] = fmaf(pr.y, rowf[RT + hh * 16 + 2 * k + 1], v[2 * k + 1] * rowf[hh * 16 + 2 * k + 1]);
+                ow[k] = pack2_bf16(fmaf(pr.x, rowf[RT + hh * 16 + 2 * k], v[2 * k] * rowf[hh * 16 + 2 * k]),
+                                   fmaf(pr.y, rowf[RT + hh * 16 + 2 * k + 1], v[2 * k + 1] * rowf[hh * 16 + 2 * k + 1]));
               }
+              rp[0] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+              rp[1] = make_uint4(ow[4], ow[5], ow[6], ow[7]);
             } else {
 #pragma unroll
-              for (int r = 0; r < 16; ++r) v[r] *= rowf[hh * 16 + r];
+              for (int r = 0; r < 16; ++r) wt[(hh * 16 + r) * SLD] = __float2bfloat16_rn(v[r] * rowf[hh * 16 + r]);
             }
-#pragma unroll
-            for (int r = 0; r < 16; ++r) wt[(hh * 16 + r) * SLD] = __float2bfloat16_rn(v[r]);
           }
         }
       }
       tc_fence_before();
-      if constexpr (PAIR) {
-        named_barrier_sync(2, TEW * 32);                              // what the peer sent has been consumed
-        if (tid == 0) mbar_arrive_cluster(map_to_cta(smem_addr(&bars.x_ack), (uint32_t)rg ^ 1u));
-      }
       named_barrier_arrive(BAR_W_READY, FCONS);
-    }
-    if constexpr (PAIR) {
-      // the peer's last acknowledgement arrives in this CTA's shared memory: stay until it is there
-      if (ucount > 0 && !dead && !mbar_wait_cluster_bounded(&bars.x_ack, (ucount - 1) & 1u)) dead = true;
-      __syncwarp();
     }
     named_barrier_sync(BAR_END, (CW + 1) * 32);
     if (dead && lane == 0) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
@@ -648,7 +648,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
             const int head = nh * 8 + 2 * t4 + (e & 1), j = gid + (e >> 1) * 8;
             if (head < G) {
               // element (row rho, column j) of sub-chunk s, K-major core matrices of 8 rows x 8 columns
-              const int rho = bi * G + head;
+              const int rho = bi * GP + head;
               *reinterpret_cast<__nv_bfloat16*>(Sb + s * (RT * 32) + (j >> 3) * (RT * 16) + (rho >> 3) * 128 + (rho & 7) * 16 + (j & 7) * 2) =
                   __float2bfloat16_rn((sc[nh][0][e] + sc[nh][1][e]) * qscale);
             }
@@ -815,7 +815,10 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         if (rl >= rbv || bl >= nbv) continue;
         const int bi = bl * RB + rl;
         uint32_t bw[4];
-        ldsm_x4(bw, W_u + (uint32_t)(((c * JC + s) * ((RT + 16) * SLD) + (bi * G + lrowB) * SLD + lmid * 8) * 2));
+        if constexpr (PAIR)      // tiles kept as [row of U][expansion row]: transposing load; rows of U by lmid, heads by lhi
+          ldsm_x4_t(bw, W_u + (uint32_t)((((c * JC + s) * 16 + lmid * 8 + l7) * WLD + bi * GP + lhi * 8) * 2));
+        else
+          ldsm_x4(bw, W_u + (uint32_t)(((c * JC + s) * ((RT + 16) * SLD) + (bi * G + lrowB) * SLD + lmid * 8) * 2));
         const uint32_t rowoff = v_u + (uint32_t)((bi * rows16 + s * 16 + lrowB) * 128);
         uint32_t av[8][4];
 #pragma unroll
@@ -1038,7 +1041,8 @@ FusedPlan plan_fused_tc(const kvc_layer* L, int B, int R) {
 FusedPlan plan_fused_pair(const kvc_layer* L, int B, int R) {
   FusedPlan p{};
   const int G = L->G, n = L->desc.n, m = L->m, H_kv = L->desc.H_kv;
-  if (L->desc.dtype != KVC_BF16 || L->passthrough || R < 1 || B < 1 || n % 256 != 0 || n > 1024 || G > 16 || R * G > 64 || m < 32) return p;
+  const int GP = G <= 8 ? 8 : 16;                                      // expansion rows per block, padded
+  if (L->desc.dtype != KVC_BF16 || L->passthrough || R < 1 || B < 1 || n % 256 != 0 || n > 1024 || G > 16 || R * GP > 64 || m < 32) return p;
   if (reinterpret_cast<uintptr_t>(L->desc.theta) & 15 || reinterpret_cast<uintptr_t>(L->desc.U) & 15) return p;
   if ((long long)B * H_kv > KVC_MAX_COUNTERS) return p;
   const int sms = L->num_sms > 0 ? L->num_sms : 148;
@@ -1081,13 +1085,13 @@ FusedPlan plan_fused_pair(const kvc_layer* L, int B, int R) {
   auto take = [&](uint32_t bytes) { uint32_t o = off; off = (off + bytes + 127u) & ~127u; return o; };
   const int nj0 = (p.NJ + 1) / 2;                                      // stages of the m axis of CTA 0 (the larger share)
   const uint32_t p_bytes = (uint32_t)rt * (n / 2) * 2, yred_bytes = (uint32_t)p.VW * p.yhg * D * 4;
-  const uint32_t w_bytes = (uint32_t)nj0 * p.JC * (rt + 16) * SLD * 2;
+  const uint32_t w_bytes = (uint32_t)nj0 * p.JC * 16 * (rt + 8) * 2;     // [rows of U of CTA 0][expansion rows + 8]
   uint32_t r0_bytes = p_bytes > yred_bytes ? p_bytes : yred_bytes;
   if (w_bytes > r0_bytes) r0_bytes = w_bytes;
   p.off_P = take(r0_bytes);
   p.off_yred = p.off_P;
   p.off_W = p.off_P;
-  p.off_wrecv = take((uint32_t)nj0 * p.JC * 16 * rt * 2);
+  p.off_wrecv = 0;
   p.off_xstat = take((uint32_t)(16 + rt) * 4);
   p.off_q = take((uint32_t)16 * QLD * 2);
   p.off_S = take((uint32_t)(2 * p.JC * rt * 32));
