@@ -782,8 +782,10 @@ FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
     // behind at batches 1-4 where units of half the size halve the latency).
     if (L->use_tc != 1) {
       // pairs of CTAs per (sequence, KV head): ahead of the single-CTA variant on the n = 1024, G = 7 shape from batch 16 on
+      // when a sequence has more expansion rows than one CTA's two row tiles (8 blocks: 122 vs 154 us at batch 32; with 2
+      // blocks the 64-row unit is mostly padding: 105 vs 45 us)
       const FusedPlan t2 = plan_fused_pair(L, B, R);
-      if (t2.ok && (L->use_tc == 2 || (L->desc.n > 640 && t2.units >= 96))) return t2;
+      if (t2.ok && (L->use_tc == 2 || (L->desc.n > 640 && R * L->G > 32 && t2.units >= 96))) return t2;
     }
     const FusedPlan t = plan_fused_tc(L, B, R);
     if (t.ok && (L->use_tc > 0 || (L->desc.n > 640 && t.MT == 2 && t.units >= 96))) return t;
