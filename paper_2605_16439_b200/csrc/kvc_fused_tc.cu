@@ -136,11 +136,13 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     for (int u = blockIdx.x; u < a.units; u += gridDim.x) {
       const int h = u / per_h, rem = u - h * per_h;
       const int bg = rem / a.nrg, rg = rem - bg * a.nrg;
-      const int b0 = bg * a.NB, r0 = PAIR ? 0 : rg * a.RB;
+      // pair mode: the units 2k, 2k+1 of a (sequence, head) are the two CTAs (rank rk) of a cluster on block group k
+      const int rk = PAIR ? (rg & 1) : 0;
+      const int b0 = bg * a.NB, r0 = PAIR ? (rg >> 1) * a.RB : rg * a.RB;
       const RowRanges tr = row_ranges(a, rg);
       const int nts = tr.na + tr.nb;
-      const int cg0 = PAIR ? rg * ncgl : 0;          // first column group of this CTA
-      const int c2first = (PAIR && rg) ? NJ0 : 0, c2count = PAIR ? (rg ? a.NJ - NJ0 : NJ0) : a.NJ;
+      const int cg0 = PAIR ? rk * ncgl : 0;          // first column group of this CTA
+      const int c2first = (PAIR && rk) ? NJ0 : 0, c2count = PAIR ? (rk ? a.NJ - NJ0 : NJ0) : a.NJ;
       // stage sequence of a unit: NJ stages of pass A (theta rows + K_tilde rows); then the column groups of U and
       // the text stages, interleaved so that the tensor core (U) and the value warps (text) both have work; then
       // NJ stages of V_tilde rows
@@ -273,7 +275,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         }
       }
       // ---------------- the V_tilde stages belong to the value warps ----------------
-      const int c2count = PAIR ? (rg ? a.NJ - NJ0 : NJ0) : a.NJ;
+      const int c2count = PAIR ? ((rg & 1) ? a.NJ - NJ0 : NJ0) : a.NJ;
       for (int c = 0; c < c2count; ++c) {
         wait_on(&bars.full[slot], phase);
         if (lane == 0) mbar_arrive(&bars.empty[slot]);
@@ -331,7 +333,8 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     for (int u = blockIdx.x; u < a.units; u += gridDim.x, ++ucount) {
       const int h = u / per_h, rem = u - h * per_h;
       const int bg = rem / a.nrg, rg = rem - bg * a.nrg;
-      const int b0 = bg * a.NB, r0 = PAIR ? 0 : rg * a.RB;
+      const int rk = PAIR ? (rg & 1) : 0;           // pair mode: rank in the cluster; block group rg >> 1
+      const int b0 = bg * a.NB, r0 = PAIR ? (rg >> 1) * a.RB : rg * a.RB;
       const int nbv = min(a.NB, a.B - b0);
       const int rbv = min(RB, a.R - r0);
       (void)h;
@@ -448,15 +451,15 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       }
       const int NS = (a.m + 15) >> 4;
       // rows of W^T this CTA turns into weight tiles; in pair mode the other rows go to the peer
-      const int oj0 = (PAIR && rg) ? NJ0 * rows16 : 0;
-      const int oj1 = PAIR ? min(NS * 16, (rg ? a.NJ : NJ0) * rows16) : NS * 16;
+      const int oj0 = (PAIR && rk) ? NJ0 * rows16 : 0;
+      const int oj1 = PAIR ? min(NS * 16, (rk ? a.NJ : NJ0) * rows16) : NS * 16;
       wait_on(&bars.w_done, ucount & 1u);
       tc_fence_after();
       if constexpr (PAIR) {
         // ---- my re-projection is complete and P is dead: the peer may write into my weight tiles (they share P's region);
         // then send: maxima and row sums of my columns, and my partial weights of the peer's rows (bf16), straight into
         // the peer's weight tiles ----
-        const uint32_t peer = (uint32_t)rg ^ 1u;
+        const uint32_t peer = (uint32_t)rk ^ 1u;
         if (tid == 0) mbar_arrive_cluster(map_to_cta(smem_addr(&bars.x_ready), peer));
         if (!dead && !mbar_wait_cluster_bounded(&bars.x_ready, ucount & 1u)) dead = true;
         __syncwarp();
@@ -465,7 +468,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
           for (int x = lane; x < 16; x += 32) st_cluster_f32(xs + 4u * x, hvmax[x]);
           for (int x = lane; x < RT; x += 32) st_cluster_f32(xs + 4u * (16 + x), rsum[x]);
         }
-        const int pj0 = rg ? 0 : NJ0 * rows16, pj1 = rg ? min(NS * 16, NJ0 * rows16) : NS * 16;
+        const int pj0 = rk ? 0 : NJ0 * rows16, pj1 = rk ? min(NS * 16, NJ0 * rows16) : NS * 16;
         const uint32_t wr = map_to_cta(smem_addr(W_sm), peer);
         for (int t = wh; t < MTL; t += TSTEP) {
           const bool t64 = w_tail64 && t == MTL - 1;
@@ -505,7 +508,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
               fp = fast_exp2(xstat[x] - M);
               float vp = 0.f;
               for (int rl = 0; rl < rbv; ++rl) vp += xstat[16 + (tb_ * RB + rl) * GP + g];
-              vs = rg ? 0.f : fmaf(vp, fp, vs);                      // the sum of the vision probabilities is counted by CTA 0 alone
+              vs = rk ? 0.f : fmaf(vp, fp, vs);                      // the sum of the vision probabilities is counted by CTA 0 alone
             }
             for (int w = tb_ * WPG; w < (tb_ + 1) * WPG; ++w) {
               const float tm_ = tmax[w * 16 + g];
@@ -586,12 +589,13 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   for (int u = blockIdx.x; u < a.units; u += gridDim.x) {
     const int h = u / per_h, rem = u - h * per_h;
     const int bg = rem / a.nrg, rg = rem - bg * a.nrg;
-    const int b0 = bg * a.NB, r0 = PAIR ? 0 : rg * a.RB;
+    const int rk = PAIR ? (rg & 1) : 0;
+    const int b0 = bg * a.NB, r0 = PAIR ? (rg >> 1) * a.RB : rg * a.RB;
     const int nbv = min(a.NB, a.B - b0);
     const int rbv = min(RB, a.R - r0);
     const RowRanges tr = row_ranges(a, rg);
     const int nts = tr.na + tr.nb;
-    const int c2first = (PAIR && rg) ? NJ0 : 0, c2count = PAIR ? (rg ? a.NJ - NJ0 : NJ0) : a.NJ;
+    const int c2first = (PAIR && rk) ? NJ0 : 0, c2count = PAIR ? (rk ? a.NJ - NJ0 : NJ0) : a.NJ;
     (void)r0;
 
     // ---- queries of the unit's sequences: [NB][16 heads][128], heads >= G and absent sequences are zero rows
@@ -1042,7 +1046,7 @@ FusedPlan plan_fused_pair(const kvc_layer* L, int B, int R) {
   FusedPlan p{};
   const int G = L->G, n = L->desc.n, m = L->m, H_kv = L->desc.H_kv;
   const int GP = G <= 8 ? 8 : 16;                                      // expansion rows per block, padded
-  if (L->desc.dtype != KVC_BF16 || L->passthrough || R < 1 || B < 1 || n % 256 != 0 || n > 1024 || G > 16 || R * GP > 64 || m < 32) return p;
+  if (L->desc.dtype != KVC_BF16 || L->passthrough || R < 1 || B < 1 || n % 256 != 0 || n > 1024 || G > 16 || m < 32) return p;
   if (reinterpret_cast<uintptr_t>(L->desc.theta) & 15 || reinterpret_cast<uintptr_t>(L->desc.U) & 15) return p;
   if ((long long)B * H_kv > KVC_MAX_COUNTERS) return p;
   const int sms = L->num_sms > 0 ? L->num_sms : 148;
@@ -1050,19 +1054,20 @@ FusedPlan plan_fused_pair(const kvc_layer* L, int B, int R) {
   p.EW = 4; p.VW = 8; p.ktw = 0;
   p.MT = 4;
   const int rt = ROWS * p.MT;
-  p.NB = 1; p.RB = R; p.nbg = B;
-  p.nrg = 2;                                   // the two CTAs of a pair leave two partial outputs per (sequence, head)
-  p.units = H_kv * B * 2;
+  p.NB = 1; p.nbg = B;
+  p.RB = R < 64 / GP ? R : 64 / GP;            // blocks per pair: up to 64 padded expansion rows
+  p.nrg = 2 * ceil_div(R, p.RB);               // every pair leaves two partial outputs per (sequence, head)
+  p.units = H_kv * B * p.nrg;
   p.ncg = n / 64;
   const int ncgl = p.ncg / 2;
-  const uint32_t chunk = (uint32_t)R * 4096u + (uint32_t)(n / 2) * 32u;
+  const uint32_t chunk = (uint32_t)p.RB * 4096u + (uint32_t)(n / 2) * 32u;
   int jc = (int)(49152u / chunk);
   const int jmax = ceil_div(m, 32) < 16 ? ceil_div(m, 32) : 16;       // at least two stages along m: one per CTA in the value pass
   p.JC = jc < 1 ? 1 : (jc > jmax ? jmax : jc);
   p.NJ = ceil_div(m, 16 * p.JC);
   if (p.NJ < 2) return p;
   p.par_bytes = (uint32_t)ncgl * p.JC * 2048u;
-  p.k_half_bytes = (uint32_t)R * p.JC * 2048u;
+  p.k_half_bytes = (uint32_t)p.RB * p.JC * 2048u;
   p.stage_bytes = p.par_bytes + 2 * p.k_half_bytes;
   if (p.stage_bytes < 16384u) p.stage_bytes = 16384u;
   const int mtiles = ceil_div(m, 128);

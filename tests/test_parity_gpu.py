@@ -275,6 +275,8 @@ def test_one_kernel_path_edges(B, H_q, H_kv, grid, R, T):
     (1, 16, 1, 32, 4, 20, 800),     # G = 16: two head tiles, 64 expansion rows, m = 205
     (1, 14, 2, 32, 2, 300, 950),    # m = 52: one stage of the m axis per CTA, a 64-row tile of W^T
     (20, 8, 8, 16, 2, 37, 600),     # more pairs than SM pairs: buffers, barriers and acknowledgements reused across units
+    (1, 14, 2, 32, 20, 50, 600),    # 20 blocks: three block groups (8, 8, 4 blocks), one pair each, six partial outputs merged
+    (2, 4, 4, 16, 11, 9, 600),      # MHA, 11 blocks: two block groups (8, 3)
 ])
 def test_tensor_memory_variant_in_pairs_of_ctas(B, H_q, H_kv, grid, R, T, ratio, monkeypatch):
     """Clusters of two CTAs per (sequence, KV head): each keeps half of the columns of the logits, partial weights cross
