@@ -44,6 +44,7 @@ struct TcBars {
   uint64_t l_free;         // the logits of the unit have been read back (4 warps)
   uint64_t x_data;         // pair mode: the peer's statistics and partial weights of the unit have landed here
   uint64_t x_ready;        // pair mode: the peer's re-projection of the unit is complete: its weight tiles may be written
+  uint64_t m_data;         // pair mode, CTA 0: the peer's partial output of the unit has landed here
 };
 
 // Reduces 16 per-lane values over the 32 lanes of a warp (maximum or sum) in 31 shuffles: after the first exchange
@@ -88,6 +89,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   __shared__ __align__(8) TcBars bars;
   __shared__ int s_last;
   __shared__ uint32_t s_tmem;
+  __shared__ float2 s_mlpeer[8];            // pair mode, CTA 0: (maximum, sum) of the peer's partial output per head
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
@@ -98,6 +100,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     mbar_init(&bars.l_free, TEW);
     mbar_init(&bars.x_data, 1);
     mbar_init(&bars.x_ready, 1);
+    mbar_init(&bars.m_data, 1);
     fence_mbar_init();
   }
   if (warp == MMA_WARP) tmem_alloc(&s_tmem, (uint32_t)a.tmem_cols);
@@ -195,6 +198,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   uint32_t slot = 0, phase = 0;
   uint32_t si = 0;                                 // score tiles handed over so far (buffer = si & 1)
   uint32_t ucount = 0;                             // units this CTA has started
+  uint32_t vunit = 0;                              // units whose outputs the value warps have merged through the pair (pair mode)
   bool dead = false;
   // every lane of the calling warp waits; the lanes leave the polling loop together again before any warp-wide instruction
   auto wait_on = [&](uint64_t* bar, uint32_t parity) {
@@ -844,6 +848,13 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     const int bh = b0 * a.H_kv + h;                    // used when the block axis is split (NB == 1)
     const size_t pbase = ((size_t)bh * a.nrg + rg) * G;
     const int YHG = a.yhg;
+    // pair mode, one block group per sequence: the two outputs of the pair are merged through distributed shared memory
+    // (CTA 1 sends, CTA 0 merges and writes); the buffers are regions that are dead by now: the query tile for this CTA's
+    // output, the score tiles for the peer's
+    const bool pmerge = PAIR && a.nrg == 2 && G <= 8;
+    float* ybuf0 = reinterpret_cast<float*>(sm + a.off_q);
+    float* ybuf1 = reinterpret_cast<float*>(sm + a.off_S);
+    const uint32_t ypeer = PAIR ? map_to_cta(smem_addr(ybuf1), 0u) : 0u;
     for (int g0 = 0; g0 < G; g0 += YHG) {
       // every warp parks its tile columns of heads g0 .. g0+YHG-1; then the warps of a sequence are summed
 #pragma unroll
@@ -870,12 +881,37 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         if (a.R > 0) y = fmaf(vsum[tb * 16 + g], __bfloat162float(a.mu[h * D + col]), y);
         if (a.nrg == 1)
           a.out[((size_t)(b0 + tb) * a.H_kv * G + (size_t)h * G + g) * D + col] = __float2bfloat16_rn(y / hsum[tb * 16 + g]);
-        else
+        else if (pmerge) {
+          if (rk) st_cluster_f32(ypeer + (uint32_t)((g * D + col) * 4), y); else ybuf0[g * D + col] = y;
+        } else
           a.part_y[(pbase + g) * D + col] = y;
       }
       named_barrier_sync(3, VTH);
     }
-    if (a.nrg > 1) {
+    if (pmerge) {
+      if (rk) {
+        if (vtid < G) {
+          const uint32_t mp = map_to_cta(smem_addr(&s_mlpeer[vtid]), 0u);
+          st_cluster_f32(mp, hmax[vtid]);
+          st_cluster_f32(mp + 4u, hsum[vtid]);
+        }
+        named_barrier_sync(3, VTH);                                   // every value of this CTA's output has been sent
+        if (vtid == 0) mbar_arrive_cluster(map_to_cta(smem_addr(&bars.m_data), 0u));
+      } else {
+        named_barrier_sync(3, VTH);                                   // this CTA's output is in its buffer
+        if (!dead && !mbar_wait_cluster_bounded(&bars.m_data, vunit & 1u)) dead = true;
+        __syncwarp();
+        for (int idx = vtid; idx < G * D; idx += VTH) {
+          const int g = idx >> 7, col = idx & (D - 1);
+          const float M0 = hmax[g], M1 = s_mlpeer[g].x, M = fmaxf(M0, M1);
+          const float w0 = fast_exp2(M0 - M), w1 = fast_exp2(M1 - M);
+          const float num = fmaf(ybuf0[idx], w0, ybuf1[idx] * w1), den = fmaf(hsum[g], w0, s_mlpeer[g].y * w1);
+          a.out[((size_t)b0 * a.H_kv * G + (size_t)h * G + g) * D + col] = __float2bfloat16_rn(num / den);
+        }
+        named_barrier_sync(3, VTH);                                   // the buffers are read: the next unit may overwrite them
+      }
+      ++vunit;
+    } else if (a.nrg > 1) {
       // one sequence, several units along the block axis: the last unit to arrive merges the partials
       if (vtid < G) a.part_ml[pbase + vtid] = make_float2(hmax[vtid], hsum[vtid]);
       __threadfence();
