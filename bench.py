@@ -42,8 +42,8 @@ NCU_TRAFFIC_BYTES = {
     # profiles/fused_decode_tc_config2.md: 123.0 MB read + 4.2 MB written per launch at T = 258; 32768 bytes per text
     # row more up to the mid-run launch (T = 511.5)
     ("fused_tc", "config2-qwen2-vl-7b"): 135.5e6,
-    # profiles/fused_decode_pair_config2.md: 123.0 MB read + 3.9 MB written per launch at T = 258, scaled the same way
-    ("fused_pair", "config2-qwen2-vl-7b"): 135.2e6,
+    # profiles/fused_decode_pair_config2.md: 123.0 MB read + 4.4 MB written per launch at T = 258, scaled the same way
+    ("fused_pair", "config2-qwen2-vl-7b"): 135.7e6,
 }
 
 
