@@ -63,6 +63,9 @@ def parse_args():
     ap.add_argument("--no-comparator", action="store_true")
     ap.add_argument("--no-profile", action="store_true", help="do not bracket kernels with events in the timed region")
     ap.add_argument("--oracle-decode-steps", type=int, default=96)
+    ap.add_argument("--pyramid", type=str, default=None, metavar="LO,HI",
+                    help="decode loop with a per-layer ratio rising linearly from LO to HI permille (first to last layer), "
+                         "beside the same loop at the uniform mean ratio; one JSON line (not the headline metric)")
     ap.add_argument("--sweep", action="store_true",
                     help="configuration 4: ratio x batch x vision tokens on the Qwen2-VL shape; prints one JSON line per point")
     return ap.parse_args()
@@ -145,33 +148,40 @@ class ClockSampler:
 class Job:
     """All device state of one rank's batch: per-layer inputs, parameters, capsule stores, text tails."""
 
-    def __init__(self, shape: wl.Shape, config_index: int, dev, rank: int):
+    def __init__(self, shape: wl.Shape, config_index: int, dev, rank: int, ratios=None):
+        """ratios: compression ratio in permille per layer (a pyramid schedule); None = the shape's ratio everywhere."""
         from paper_2605_16439_b200 import binding as kvc
         self.kvc, self.shape, self.dev = kvc, shape, dev
         dt = wl.torch_dtype(shape.dtype)
+        self.ratios = list(ratios) if ratios is not None else [shape.ratio_permille] * shape.layers
         self.m = kvc.kvc_retained_len(shape.n, shape.ratio_permille)
         self.T_cap = shape.T0 + shape.steps
         self.layers = []
-        for l in range(shape.layers):
+        self.ws = None
+        for l, ratio in enumerate(self.ratios):
             seed = wl.layer_seed(config_index, l) + 100000 * rank
-            p = wl.decode_inputs(shape, self.m, seed, dev, T=shape.T0, T_cap=self.T_cap)
-            if shape.ratio_permille == 0:
+            m = kvc.kvc_retained_len(shape.n, ratio)
+            p = wl.decode_inputs(shape, m, seed, dev, T=shape.T0, T_cap=self.T_cap)
+            if ratio == 0:
                 layer = kvc.Layer(shape.H_q, shape.H_kv, shape.d, shape.n, 0, dt, layer=l)
             else:
-                layer = kvc.Layer(shape.H_q, shape.H_kv, shape.d, shape.n, shape.ratio_permille, dt, idx=p["idx"],
+                layer = kvc.Layer(shape.H_q, shape.H_kv, shape.d, shape.n, ratio, dt, idx=p["idx"],
                                   theta=p["theta"], U=p["U"], mu=p["mu"], layer=l)
-            p["layer"] = layer
+            p["layer"], p["m"], p["ratio"] = layer, m, ratio
             p["caps"] = kvc.alloc_capsules(layer, shape.B, shape.R, dev)
             p["out"] = torch.zeros((shape.B, shape.H_q, shape.d), dtype=dt, device=dev)
             self.layers.append(p)
-        self.ws = kvc.alloc_workspace(self.layers[0]["layer"], shape.B, shape.R, self.T_cap, dev)
+            if ratios is not None or l == 0:       # one workspace serves every layer: the largest request
+                ws = kvc.alloc_workspace(layer, shape.B, shape.R, self.T_cap, dev)
+                if self.ws is None or ws.numel() * ws.element_size() > self.ws.numel() * self.ws.element_size():
+                    self.ws = ws
         self.launches = 0
 
     def compress_all(self):
         s = self.shape
         for p in self.layers:
             self.kvc.kvc_compress(p["layer"], p["K_vis"], p["V_vis"], s.B, s.R, p["caps"])
-        self.launches += (0 if s.ratio_permille == 0 else 2) * len(self.layers)
+        self.launches += sum(0 if r == 0 else 2 for r in self.ratios)
 
     def decode_step(self, t: int):
         s = self.shape
@@ -400,6 +410,58 @@ def run_sweep(a, dev):
                 torch.cuda.empty_cache()
 
 
+def run_pyramid(a, shape, dev):
+    """Pyramid retention schedule (Sec. 2.4, Sec. 3.2: early layers keep more, deep layers less; the paper prints no
+    schedule, so a linear one from LO to HI permille is taken, whose mean is the uniform comparison ratio).  Times the
+    decode loop (all layers in model order, every layer its own buffers) once with the schedule and once with the mean
+    ratio everywhere, and gives each layer's launch time from events placed between the layers."""
+    lo, hi = (int(x) for x in a.pyramid.split(","))
+    L = shape.layers
+    ratios = [lo + (hi - lo) * l // max(L - 1, 1) for l in range(L)]
+    mean = round(sum(ratios) / L)
+    out = {"pyramid": shape.name, "schedule": f"linear {lo}..{hi} permille over {L} layers", "mean_ratio_permille": mean,
+           "batch": shape.B, "decode_steps": shape.steps}
+    for tag, rr in (("pyramid", ratios), ("uniform", [mean] * L)):
+        job = Job(dataclasses.replace(shape, ratio_permille=mean), a.config, dev, 0, ratios=rr)
+        job.compress_all()
+        for p in job.layers:                       # the full-size vision K/V is not needed after compression
+            del p["K_vis"], p["V_vis"]
+        torch.cuda.empty_cache()
+        loop = lambda: [job.decode_step(t) for t in range(shape.steps)]
+        loop()
+        ms = timed(loop, 1, dev)
+        T_mid = shape.T0 + (shape.steps - 1) / 2.0
+        contract = sum(contract_bytes_per_layer_call(shape, p["m"], T_mid) for p in job.layers)
+        out[tag] = {"ms_per_decode_step": round(ms / shape.steps, 4),
+                    "tokens_per_s": round(shape.B * shape.steps / (ms * 1e-3), 1),
+                    "contract_gbs": round(contract * shape.steps / (ms * 1e-3) / 1e9, 1),
+                    "capsule_mb": round(sum(p["caps"].numel() * p["caps"].element_size() for p in job.layers) / 1e6, 1)}
+        if tag == "pyramid":
+            # per-layer launch times: events between the layers (the programmatic overlap of consecutive launches is
+            # off in this pass, so the sum is a little above the loop time)
+            ev = [[torch.cuda.Event(enable_timing=True) for _ in range(L + 1)] for _ in range(shape.steps)]
+            s = shape
+            torch.cuda.synchronize(dev)
+            for t in range(s.steps):
+                ev[t][0].record()
+                for l, p in enumerate(job.layers):
+                    job.kvc.kvc_decode_attend(p["layer"], p["q"], p["caps"], s.B, s.R, p["K_txt"], p["V_txt"], s.T0 + t,
+                                              job.T_cap, p["out"], job.ws)
+                    ev[t][l + 1].record()
+            torch.cuda.synchronize(dev)
+            per = []
+            for l, p in enumerate(job.layers):
+                us = sum(ev[t][l].elapsed_time(ev[t][l + 1]) for t in range(s.steps)) / s.steps * 1e3
+                c = contract_bytes_per_layer_call(shape, p["m"], T_mid)
+                per.append({"layer": l, "ratio": p["ratio"] / 1000.0, "m": p["m"], "us": round(us, 1),
+                            "frac_of_8tbs": round(c / (us * 1e-6) / 1e9 / NOMINAL_HBM_GBS, 3)})
+            out["per_layer"] = per
+        del job
+        torch.cuda.empty_cache()
+    out["pyramid_vs_uniform"] = round(out["uniform"]["ms_per_decode_step"] / out["pyramid"]["ms_per_decode_step"], 3)
+    print(json.dumps(out))
+
+
 def main():
     a = parse_args()
     shape = pick_shape(a)
@@ -425,6 +487,11 @@ def main():
     if a.sweep:
         if rank == 0:
             run_sweep(a, dev)
+        return
+
+    if a.pyramid:
+        if rank == 0:
+            run_pyramid(a, shape, dev)
         return
 
     job = Job(shape, a.config, dev, rank)

@@ -122,6 +122,11 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   const int NJ0 = PAIR ? (a.NJ + 1) >> 1 : a.NJ;   // pair mode: CTA 0 takes the first NJ0 stages of the m axis in the value pass
   const int MTL = (a.m + 127) >> 7;            // 128-row tiles of W^T (rows of U)
   const uint32_t w_col = (uint32_t)(NT * RT);
+  // W^T tiles beyond the allocated columns take the columns of L^T, whose logits are dead once P is in shared memory
+  // (long retained lengths in pair mode: 4 + 4 tiles of 64 columns fill the 512, tiles 4.. of W^T overlay L^T)
+  const int wown = (a.tmem_cols - NT * RT) / RT;
+  const bool overlay = MTL > wown;
+  auto wcol = [&](int t) -> uint32_t { return t < wown ? w_col + (uint32_t)(t * RT) : (uint32_t)((t - wown) * RT); };
   const bool w_tail64 = a.m - 128 * (MTL - 1) <= 64;   // the last tile of W^T holds at most 64 rows of U: M = 64
   const int ugroups = (MTL + a.UT - 1) / a.UT; // stages per 64-column group of U: UT row tiles each
 
@@ -263,7 +268,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
               for (int kk = 0; kk < 4; ++kk) {
                 const uint64_t adesc = umma_smem_desc(par_u + (uint32_t)(t * 16384 + kk * 32), 16u, 1024u, UMMA_LAYOUT_SW128);
                 const uint64_t bdesc = umma_smem_desc(P_u + (uint32_t)(cg * RT * 128 + kk * 32), 16u, 1024u, UMMA_LAYOUT_SW128);
-                umma_bf16(tb + w_col + (uint32_t)((t0 + t) * RT), adesc, bdesc, (w_tail64 && t0 + t == MTL - 1) ? idesc_W64 : idesc_W,
+                umma_bf16(tb + wcol(t0 + t), adesc, bdesc, (w_tail64 && t0 + t == MTL - 1) ? idesc_W64 : idesc_W,
                           (cg | kk) ? 1u : 0u);
               }
             umma_commit(&bars.empty[slot]);
@@ -442,7 +447,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       fence_proxy_async();                                             // P is read by the tensor core (async proxy)
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&bars.l_free);
+      if (lane == 0 && !overlay) mbar_arrive(&bars.l_free);          // (with W^T tiles over L^T: after they have been read)
       named_barrier_arrive(BAR_P_READY, TEW * 32 + 32);
       named_barrier_sync(2, TEW * 32);                                // row sums of every warp
       if (warp == 0) {
@@ -482,7 +487,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
           for (int hh = 0; hh < MT; ++hh) {
             float v[16];
             __syncwarp();
-            tmem_ld_x16(tq + w_col + (uint32_t)(t * RT + hh * 16), v);
+            tmem_ld_x16(tq + wcol(t) + (uint32_t)(hh * 16), v);
             if (mine) {
               const uint32_t dst = wr + (uint32_t)(((j - pj0) * WLD + hh * 16) * 2);
               st_cluster_v4(dst, pack2_bf16(v[0], v[1]), pack2_bf16(v[2], v[3]), pack2_bf16(v[4], v[5]), pack2_bf16(v[6], v[7]));
@@ -545,7 +550,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         for (int hh = 0; hh < MT; ++hh) {
           float v[16];
           __syncwarp();
-          tmem_ld_x16(tq + w_col + (uint32_t)(t * RT + hh * 16), v);
+          tmem_ld_x16(tq + wcol(t) + (uint32_t)(hh * 16), v);
           if (mine) {
             if constexpr (PAIR) {
               // the peer's partial sits where the result goes: add in place
@@ -569,6 +574,10 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         }
       }
       tc_fence_before();
+      if (overlay) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars.l_free);
+      }
       named_barrier_arrive(BAR_W_READY, FCONS);
     }
     named_barrier_sync(BAR_END, (CW + 1) * 32);
@@ -1142,10 +1151,13 @@ FusedPlan plan_fused_pair(const kvc_layer* L, int B, int R) {
   p.off_hstat = take((uint32_t)(6 * 16 + 2 * rt) * 4);
   p.off_rtab = take((uint32_t)rt * 4);
   p.misc_bytes = off;
+  // tensor memory: n/256 tiles of L^T, then the tiles of W^T; W^T tiles that do not fit behind them take the columns of
+  // L^T (dead by then), so up to n/256 more
+  const int lcols = (n / 256) * rt;
   int cols = 32;
-  while (cols < (n / 256) * rt + mtiles * rt) cols *= 2;
+  while (cols < lcols + mtiles * rt && cols < 512) cols *= 2;
   p.tmem_cols = cols;
-  if (cols > 512) return p;
+  if (lcols + mtiles * rt > 512 && mtiles - (512 - lcols) / rt > n / 256) return p;
   if (SMEM_LIMIT < 1024u + 2048u + p.misc_bytes + 2 * p.stage_bytes) return p;
   const uint32_t avail = SMEM_LIMIT - 1024u - 2048u - p.misc_bytes;
   int stages = (int)(avail / p.stage_bytes);

@@ -268,6 +268,17 @@ def test_one_kernel_path_edges(B, H_q, H_kv, grid, R, T):
     _check(shape, p)
 
 
+# per-layer ratios of a pyramid schedule (Sec. 2.4, Sec. 3.2: shallow layers compress less, deep layers more): every retained
+# length between 0.3 and 0.9 on the 7B block lengths goes through the same one-kernel path as the uniform 0.6
+@pytest.mark.parametrize("ratio", [300, 375, 450, 525, 600, 675, 750, 825, 900])
+@pytest.mark.parametrize("ci,kw", [(1, dict(B=2, H_q=4, H_kv=4, R=3)), (2, dict(B=1, H_q=14, H_kv=2, R=3))])
+def test_pyramid_schedule_ratios_on_the_7b_block_lengths(ci, kw, ratio):
+    shape = tl.small(wl.CONFIGS[ci], ratio_permille=ratio, **kw)
+    p = tl.make_problem(shape, 900 + ci + ratio, T=70, T_cap=80)
+    counts = _fused_launches(lambda: _check(shape, p))
+    assert counts["fused"] + counts["fused_tc"] + counts["fused_pair"] == 1 and counts["scores"] == 0
+
+
 @pytest.mark.parametrize("B,H_q,H_kv,grid,R,T,ratio", [
     (2, 14, 2, 32, 8, 70, 600),     # the Qwen2-VL head layout: 56 expansion rows per (sequence, KV head)
     (1, 14, 2, 16, 3, 0, 600),      # n = 256: one logit tile per CTA; no text rows
@@ -277,6 +288,9 @@ def test_one_kernel_path_edges(B, H_q, H_kv, grid, R, T):
     (20, 8, 8, 16, 2, 37, 600),     # more pairs than SM pairs: buffers, barriers and acknowledgements reused across units
     (1, 14, 2, 32, 20, 50, 600),    # 20 blocks: three block groups (8, 8, 4 blocks), one pair each, six partial outputs merged
     (2, 4, 4, 16, 11, 9, 600),      # MHA, 11 blocks: two block groups (8, 3)
+    (2, 14, 2, 32, 8, 70, 300),     # m = 717: six tiles of W^T, the last two take the tensor-memory columns of the logits
+    (1, 14, 2, 32, 3, 33, 200),     # m = 820: seven tiles, the last (52 rows, M = 64) among the overlaid ones
+    (20, 4, 4, 32, 2, 37, 450),     # m = 564 and more pairs than SM pairs: the next unit's logits wait for the overlaid tiles
 ])
 def test_tensor_memory_variant_in_pairs_of_ctas(B, H_q, H_kv, grid, R, T, ratio, monkeypatch):
     """Clusters of two CTAs per (sequence, KV head): each keeps half of the columns of the logits, partial weights cross
