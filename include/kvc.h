@@ -160,6 +160,17 @@ KVC_API int kvc_read_device_status(const kvc_layer* layer, int B, int R, int T, 
  * usable either way.  Allocates and frees 4 bytes of device memory and synchronises `stream`. */
 KVC_API int kvc_selftest_bounded_wait(void* stream);
 
+/* Collapse of a factored key reconstructor, once per (layer, ratio) before kvc_layer_create.  Sec. 3.1 describes the
+ * reconstructor f_theta as a two-layer network while Alg. 1 (step 2) applies a single matrix theta[h] of m x n per KV
+ * head to the compressed scores; the two agree when both layers are linear along the token axis, and then
+ *   theta[h] = W1[h] W2[h],   W1: DEVICE [H_kv][m][k],  W2: DEVICE [H_kv][k][n],  theta_out: DEVICE [H_kv][m][n],
+ * all contiguous, of type `dtype`, caller-owned; theta_out must not overlap the inputs.  fp32 accumulation, one rounding
+ * to `dtype`.  m = kvc_retained_len(n, ratio); k >= 1 is the hidden width.  Asynchronous on `stream`; no allocation.
+ * Errors: KVC_ERR_ARG (null pointer), KVC_ERR_SHAPE (a size < 1 or a grid dimension beyond 65535), KVC_ERR_DTYPE,
+ * KVC_ERR_CUDA (launch failure). */
+KVC_API int kvc_collapse_theta(const void* W1, const void* W2, int H_kv, int m, int k, int n, kvc_dtype dtype,
+                               void* theta_out, void* stream);
+
 /* Integer maps as the device path uses them (read back from the device copy):
  * idx_out: HOST [H_kv][m] retained indices per KV head; group_out: HOST [R*n][2] = (block r,
  * offset i) of vision token t = r*n + i (the Reshape of Alg. 1 step 1).  Either may be NULL. */

@@ -142,6 +142,22 @@ def reconstruct(K_t, V_t, theta, U, mu, passthrough: bool = False):
     return K_hat, V_hat
 
 
+def collapse_reconstructor(W1, W2) -> np.ndarray:
+    """A key reconstructor of two layers that are linear along the token axis (Sec. 3.1 calls f_theta a two-layer
+    network; Alg. 1 step 2 and App. D use one m x n matrix theta per KV head):
+        K_hat = W2^T (W1^T K_tilde) = (W1 W2)^T K_tilde,  so  theta[h] = W1[h] W2[h].
+    W1 [H_kv, m, k], W2 [H_kv, k, n] -> theta [H_kv, m, n], the definition of the matrix product written out."""
+    W1, W2 = np.asarray(W1, F64), np.asarray(W2, F64)
+    H_kv, m, k = W1.shape
+    n = W2.shape[2]
+    theta = np.zeros((H_kv, m, n), F64)
+    for h in range(H_kv):
+        for j in range(m):
+            for l in range(k):
+                theta[h, j] += W1[h, j, l] * W2[h, l]
+    return theta
+
+
 def decode_attend_definition(q, K_t, V_t, theta, U, mu, K_txt, V_txt, passthrough: bool = False):
     """Form 1: reconstruct, concatenate with text K/V, run the original attention."""
     K_hat, V_hat = reconstruct(K_t, V_t, theta, U, mu, passthrough)

@@ -59,6 +59,7 @@ def _lib() -> C.CDLL:
         lib.kvc_read_device_status.argtypes = [vp, i, i, i, vp, C.POINTER(i)]
         lib.kvc_read_device_status.restype = i
         lib.kvc_selftest_bounded_wait.argtypes = [vp]; lib.kvc_selftest_bounded_wait.restype = i
+        lib.kvc_collapse_theta.argtypes = [vp, vp, i, i, i, i, i, vp, vp]; lib.kvc_collapse_theta.restype = i
         lib.kvc_export_maps.argtypes = [vp, i, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         lib.kvc_export_maps.restype = i
         lib.kvc_strerror.argtypes = [i]; lib.kvc_strerror.restype = C.c_char_p
@@ -182,6 +183,19 @@ def kvc_read_device_status(layer: Layer, B: int, R: int, T: int, workspace) -> i
     _check(_lib().kvc_read_device_status(layer.handle, B, R, T, _ptr(workspace), C.byref(out)),
            "kvc_read_device_status")
     return out.value
+
+
+def kvc_collapse_theta(W1: torch.Tensor, W2: torch.Tensor, stream=None) -> torch.Tensor:
+    """theta [H_kv, m, n] = W1 [H_kv, m, k] @ W2 [H_kv, k, n] on the device (a factored key reconstructor collapsed once,
+    before kvc_layer_create)."""
+    assert W1.is_cuda and W2.is_cuda and W1.dtype == W2.dtype and W1.is_contiguous() and W2.is_contiguous()
+    H, m, k = W1.shape
+    assert W2.shape[0] == H and W2.shape[1] == k
+    n = W2.shape[2]
+    theta = torch.empty((H, m, n), dtype=W1.dtype, device=W1.device)
+    _check(_lib().kvc_collapse_theta(W1.data_ptr(), W2.data_ptr(), H, m, k, n, _DTYPES[W1.dtype], theta.data_ptr(), _stream(stream)),
+           "kvc_collapse_theta")
+    return theta
 
 
 def kvc_selftest_bounded_wait(stream=None) -> int:

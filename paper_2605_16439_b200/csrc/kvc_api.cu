@@ -298,6 +298,14 @@ int kvc_attend_full(const kvc_layer* L, const void* q, const void* K, const void
   return decode_common(L, q, nullptr, B, 0, K, V, S, S_cap, out, workspace, static_cast<cudaStream_t>(stream));
 }
 
+int kvc_collapse_theta(const void* W1, const void* W2, int H_kv, int m, int k, int n, kvc_dtype dtype, void* theta_out,
+                       void* stream) {
+  if (!W1 || !W2 || !theta_out) return KVC_ERR_ARG;
+  if (H_kv < 1 || m < 1 || k < 1 || n < 1 || H_kv > 65535 || (m + 63) / 64 > 65535) return KVC_ERR_SHAPE;
+  if (dtype != KVC_F32 && dtype != KVC_BF16) return KVC_ERR_DTYPE;
+  return cuda_status(kvc::launch_collapse_theta(W1, W2, theta_out, H_kv, m, k, n, (int)dtype, static_cast<cudaStream_t>(stream)));
+}
+
 int kvc_selftest_bounded_wait(void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int* d_status = nullptr;

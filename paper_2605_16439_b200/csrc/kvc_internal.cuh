@@ -195,6 +195,9 @@ cudaError_t launch_expand_mma(const DecodeArgs& a, cudaStream_t st);
 cudaError_t launch_output(const DecodeArgs& a, int dtype, cudaStream_t st);
 // one-kernel path; *encoded == false (and nothing launched) if the tensor maps could not be built
 cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPlan& p, cudaStream_t st, bool* encoded);
+// theta[h] = W1[h] W2[h] (m x k times k x n), fp32 accumulation, one rounding to the storage type
+cudaError_t launch_collapse_theta(const void* W1, const void* W2, void* theta, int H_kv, int m, int k, int n, int dtype,
+                                  cudaStream_t st);
 void launch_wait_selftest(int* status, cudaStream_t st);   // one warp, a wait that runs out: *status = KVC_ERR_TIMEOUT
 cudaError_t compute_usum(const kvc_layer* L, float* usum);
 cudaError_t launch_project_values_tc(const kvc_layer* L, const void* V_vis, int B, int R, void* Vc, cudaStream_t st, bool* used);

@@ -284,6 +284,35 @@ def test_scalar_closed_form():
         assert abs(got[0, 0, 0] - want) < 1e-14
 
 
+# ---------------------------------------------------------------- factored key reconstructor
+def test_collapsed_two_layer_reconstructor():
+    """theta = W1 W2: (i) with k = m and W1 = I it is W2 itself; (ii) the keys reconstructed layer by layer with scalar
+    loops (first the k hidden rows, then the n positions) are theta^T K_tilde; (iii) its rank is at most k; (iv) a decode
+    step with the collapsed theta equals one whose scores are expanded in two skinny steps, (S W1) W2."""
+    r = _rng(31)
+    H, m, k, n, d = 2, 5, 3, 7, 4
+    W1 = r.standard_normal((H, m, k)); W2 = r.standard_normal((H, k, n))
+    th = orc.collapse_reconstructor(W1, W2)
+    eye = np.broadcast_to(np.eye(m), (H, m, m))
+    W2m = r.standard_normal((H, m, n))
+    assert np.array_equal(orc.collapse_reconstructor(eye, W2m), W2m)
+    Kt = r.standard_normal((m, d))
+    for h in range(H):
+        hidden = [[sum(W1[h][j][l] * Kt[j][c] for j in range(m)) for c in range(d)] for l in range(k)]
+        Kh = [[sum(W2[h][l][i] * hidden[l][c] for l in range(k)) for c in range(d)] for i in range(n)]
+        np.testing.assert_allclose(th[h].T @ Kt, np.array(Kh), atol=1e-13)
+        assert np.linalg.matrix_rank(th[h]) <= k
+    # (iv): Alg. 1 with L = (S W1) W2 taken in two steps, one head, one block, no text
+    q = r.standard_normal(d); V = r.standard_normal((n, d)); U = r.standard_normal((1, m, n)); mu = r.standard_normal((1, d))
+    K_t = Kt[None, None, None]; V_t = (U[0] @ (V - mu[0]))[None, None, None]
+    S = Kt @ q / math.sqrt(d)
+    L = (S @ W1[0]) @ W2[0]
+    P = np.exp(L - L.max()); P /= P.sum()
+    want = (P @ U[0].T) @ V_t[0, 0, 0] + P.sum() * mu[0]
+    got = orc.decode_attend_fused(q[None, None], K_t, V_t, th[:1], U, mu, np.zeros((1, 1, 0, d)), np.zeros((1, 1, 0, d)))
+    np.testing.assert_allclose(got[0, 0], want, atol=1e-13)
+
+
 # ---------------------------------------------------------------- sizes (App. D)
 def _golden(name):
     vals = {}

@@ -424,6 +424,37 @@ def test_full_size_configuration_sampled_heads(ci):
         assert np.abs(got - want).max() <= tl.TOL[shape.dtype], (b, h)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("H,m,k,n", [(3, 231, 96, 576), (1, 1, 1, 1), (2, 65, 17, 130), (4, 410, 128, 1024)])
+def test_factored_reconstructor_collapses_to_theta(dtype, H, m, k, n):
+    """theta = W1 W2 on the device against the written-out product in fp64: fp32 accumulation over k terms, then one
+    rounding to the storage type (bf16: 2^-9 relative)."""
+    dt = wl.torch_dtype(dtype)
+    W1 = wl.gaussian((H, m, k), 601, "cpu", dt, std=1.0)
+    W2 = wl.gaussian((H, k, n), 602, "cpu", dt, std=k ** -0.5)
+    want = orc.collapse_reconstructor(tl.np64(W1), tl.np64(W2))
+    got = tl.np64(kvc.kvc_collapse_theta(W1.cuda(), W2.cuda()))
+    torch.cuda.synchronize()
+    scale = max(1.0, float(np.abs(want).max()))
+    assert np.abs(got - want).max() <= (1e-5 if dtype == "f32" else 2.0 ** -8) * scale
+
+
+def test_decode_with_a_collapsed_reconstructor():
+    """A layer built from the device-collapsed theta decodes like the oracle with its own collapsed theta (rounded to
+    the storage type as every parameter is)."""
+    shape = tl.small(wl.CONFIGS[1], B=2, H_q=4, H_kv=4, R=2)
+    p = tl.make_problem(shape, 611, T=40, T_cap=48)
+    m, n, k = p["m"], shape.n, 64
+    W1 = wl.gaussian((shape.H_kv, m, k), 612, "cpu", torch.bfloat16, std=1.0)
+    W2 = wl.gaussian((shape.H_kv, k, n), 613, "cpu", torch.bfloat16, std=(k * shape.d) ** -0.5)
+    theta_dev = kvc.kvc_collapse_theta(W1.cuda(), W2.cuda())
+    p_gpu = dict(p, theta=theta_dev.cpu())
+    p_orc = dict(p, theta=torch.from_numpy(orc.collapse_reconstructor(tl.np64(W1), tl.np64(W2))).to(torch.bfloat16))
+    _, _, out_o = tl.oracle_run(shape, p_orc)
+    _, _, _, out_g = tl.gpu_run(shape, p_gpu)
+    assert np.abs(tl.np64(out_g) - out_o).max() <= tl.TOL["bf16"]
+
+
 @pytest.mark.parametrize("B,H_q,H_kv,grid,R,T", [(1, 4, 1, 16, 3, 300), (2, 2, 2, 8, 5, 0), (3, 14, 2, 32, 2, 77)])
 def test_pass_through_store_is_attended_as_plain_rows(B, H_q, H_kv, grid, R, T):
     """rho = 0 with bf16 storage: the verbatim vision rows and the text rows form one row sequence that is cut into
