@@ -210,39 +210,47 @@ def timed(fn, reps: int, dev) -> float:
 
 
 def run_e2e(job: Job, dev) -> dict:
-    """The same job driven from HOST buffers: per step the vision K/V of every layer, and per decode step
-    and layer the query and the new text K/V row, are copied from pinned host memory, and the attention
-    output is copied back, all inside the timed region."""
+    """The same job driven from HOST buffers: per step the vision K/V of every layer, and per decode step the queries
+    and the new text K/V rows of all layers, are copied from pinned host memory, and the attention outputs of all
+    layers are copied back, all inside the timed region.  The per-decode-step inputs of the layers travel as one packed
+    buffer each (queries, key rows, value rows) and the outputs as one: the text tails, queries and outputs of the
+    layers are slices of one device tensor each."""
     s, kvc = job.shape, job.kvc
     dt = wl.torch_dtype(s.dtype)
-    host = []
-    for p in job.layers:
-        host.append(dict(K_vis=p["K_vis"].to("cpu").pin_memory(), V_vis=p["V_vis"].to("cpu").pin_memory(),
-                         q=p["q"].to("cpu").pin_memory(),
-                         k_row=p["K_txt"][:, :, 0].contiguous().to("cpu").pin_memory(),
-                         v_row=p["V_txt"][:, :, 0].contiguous().to("cpu").pin_memory(),
-                         out=torch.empty((s.B, s.H_q, s.d), dtype=dt).pin_memory()))
+    L = len(job.layers)
+    q_all = torch.stack([p["q"] for p in job.layers])                    # [L, B, H_q, d]
+    out_all = torch.zeros_like(q_all)
+    Kt_all = torch.stack([p["K_txt"] for p in job.layers])               # [L, B, H_kv, T_cap, d]
+    Vt_all = torch.stack([p["V_txt"] for p in job.layers])
+    for l, p in enumerate(job.layers):                                   # the job's layers now live in the packed tensors
+        p["q"], p["out"], p["K_txt"], p["V_txt"] = q_all[l], out_all[l], Kt_all[l], Vt_all[l]
+    torch.cuda.empty_cache()
+    host_vis = [(p["K_vis"].to("cpu").pin_memory(), p["V_vis"].to("cpu").pin_memory()) for p in job.layers]
+    h_q = q_all.to("cpu").pin_memory()
+    h_k = Kt_all[:, :, :, 0].contiguous().to("cpu").pin_memory()         # [L, B, H_kv, d]: the row appended per decode step
+    h_v = Vt_all[:, :, :, 0].contiguous().to("cpu").pin_memory()
+    h_out = torch.empty(out_all.shape, dtype=dt).pin_memory()
     h2d = d2h = 0
 
     def one_step():
         nonlocal h2d, d2h
         h2d = d2h = 0
-        for p, h in zip(job.layers, host):
-            p["K_vis"].copy_(h["K_vis"], non_blocking=True)
-            p["V_vis"].copy_(h["V_vis"], non_blocking=True)
-            h2d += h["K_vis"].numel() * h["K_vis"].element_size() * 2
+        for p, (hk, hv) in zip(job.layers, host_vis):
+            p["K_vis"].copy_(hk, non_blocking=True)
+            p["V_vis"].copy_(hv, non_blocking=True)
+            h2d += hk.numel() * hk.element_size() * 2
             kvc.kvc_compress(p["layer"], p["K_vis"], p["V_vis"], s.B, s.R, p["caps"])
         for t in range(s.steps):
             T = s.T0 + t
-            for p, h in zip(job.layers, host):
-                p["q"].copy_(h["q"], non_blocking=True)
-                p["K_txt"][:, :, T - 1].copy_(h["k_row"], non_blocking=True)
-                p["V_txt"][:, :, T - 1].copy_(h["v_row"], non_blocking=True)
+            q_all.copy_(h_q, non_blocking=True)
+            Kt_all[:, :, :, T - 1].copy_(h_k, non_blocking=True)
+            Vt_all[:, :, :, T - 1].copy_(h_v, non_blocking=True)
+            for p in job.layers:
                 kvc.kvc_decode_attend(p["layer"], p["q"], p["caps"], s.B, s.R, p["K_txt"], p["V_txt"], T, job.T_cap,
                                       p["out"], job.ws)
-                h["out"].copy_(p["out"], non_blocking=True)
-                h2d += (h["q"].numel() + 2 * h["k_row"].numel()) * h["q"].element_size()
-                d2h += h["out"].numel() * h["out"].element_size()
+            h_out.copy_(out_all, non_blocking=True)
+            h2d += (h_q.numel() + 2 * h_k.numel()) * h_q.element_size()
+            d2h += h_out.numel() * h_out.element_size()
 
     one_step()                                   # warm-up (also pages the pinned buffers in)
     torch.cuda.synchronize(dev)
