@@ -31,7 +31,7 @@ import torch
 from paper_2605_16439_b200 import workloads as wl
 
 FALLBACK_HBM_GBS = 6650.0       # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
-NOMINAL_HBM_GBS = 8000.0        # the figure the task's metric quotes its percentage against
+NOMINAL_HBM_GBS = 8000.0        # nominal HBM3e bandwidth: the roofline fraction of the metric is quoted against it
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
 # the ncu capture summarised under profiles/, keyed by (kernel, workload name); None = not captured.
@@ -53,7 +53,7 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--config", type=int, default=1, help="index into the task's configurations (1 = LLaVA-NeXT-7B shape)")
+    ap.add_argument("--config", type=int, default=1, help="index into the benchmark configurations (1 = LLaVA-NeXT-7B shape)")
     ap.add_argument("--decode-steps", type=int, default=None, help="override the configuration's decode steps")
     ap.add_argument("--layers", type=int, default=None)
     ap.add_argument("--batch", type=int, default=None)
@@ -361,7 +361,7 @@ def run_reference(a, shape, rank):
 
 
 def run_sweep(a, dev):
-    """Configuration 4 of the task: ratio {0,.2,.4,.6,.8} x batch {1,8,32,64} x vision tokens {2048,8192,32768} on the
+    """Configuration 4 (the sweep): ratio {0,.2,.4,.6,.8} x batch {1,8,32,64} x vision tokens {2048,8192,32768} on the
     Qwen2-VL-7B shape (28 query / 4 KV heads, 32x32 grids), bf16, decode steps of the attention path only.  Two layer
     buffers are rotated (every call still streams more than L2 at the larger points); the uncompressed comparator runs on
     the same KV length.  One JSON line per point."""

@@ -60,7 +60,7 @@ class Shape:
         return self.R * self.n
 
 
-# The five configurations of the benchmark spec (index = config number).
+# The five benchmark configurations (index = config number).
 CONFIGS = (
     Shape("config0-single-layer-fp32", 1, 1, 8, 2, 128, 24, 1, 32, 1, "f32"),
     Shape("config1-llava-next-7b", 32, 8, 32, 32, 128, 24, 5, 128, 256, "bf16"),

@@ -1,6 +1,6 @@
 """CUDA path vs CPU oracle, element by element, on the same seeded inputs (through the C ABI).
 
-Bounds (task statement): max-abs 1e-4 for fp32 storage, 2e-2 for bf16 storage with fp32
+Bounds: max-abs 1e-4 for fp32 storage, 2e-2 for bf16 storage with fp32
 accumulation (end to end: compress + decode, oracle in fp64 on the bf16-rounded inputs); the
 selected key rows and the integer maps bit-exact.
 """
@@ -42,7 +42,7 @@ def _check(shape, p, form="fused"):
     return err
 
 
-# ------------------------------------------------------------------ the task's configurations
+# ------------------------------------------------------------------ the benchmark configurations
 def test_config0_fp32_exact_shape():
     shape = wl.CONFIGS[0]
     p = tl.make_problem(shape, wl.layer_seed(0, 0))
