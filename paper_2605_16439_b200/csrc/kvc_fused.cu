@@ -71,6 +71,14 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       const int b0 = bg * a.NB, r0 = rg * a.RB;
       const RowRanges tr = row_ranges(a, rg);
       const int nts = tr.na + tr.nb;
+      if (first && a.R > 0) {
+        // while the stream's previous kernel drains: the K_tilde rows of the first ring of stages are asked into L2 (a
+        // prefetch consumes no data, so it need not wait for that kernel; the loads below do)
+        for (int c = 0; c < a.NJ && c < a.stages; ++c) {
+          tma_prefetch_l2_5d(&tmK, 0, c * 16 * a.JC, r0, h, b0);
+          tma_prefetch_l2_5d(&tmK, 64, c * 16 * a.JC, r0, h, b0);
+        }
+      }
       for (int part = 0; part < 3; ++part) {
         const int count = part == 1 ? nts : a.NJ;
         for (int c = 0; c < count; ++c) {
@@ -123,6 +131,9 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   float* hmax = reinterpret_cast<float*>(sm + a.off_hstat);                  // [NB][16]
   float* hsum = hmax + a.NB * 16;
   float* vsum = hsum + a.NB * 16;
+  float* hvmax = vsum + a.NB * 16;                                           // maximum over the vision logits only
+  float* hfv = hvmax + a.NB * 16;                                            // 2^(hvmax - hmax): moves the vision weights to the joint maximum
+  float* rowf = hfv + a.NB * 16;                                             // [RT] that factor per expansion row
   float* yred = reinterpret_cast<float*>(sm + a.off_yred);                   // [VW][yhg][D]
   const float qscale = 0.08838834764831845f * 1.4426950408889634f;   // sigma = 1/sqrt(128), logits kept in log2 units
   const int l7 = lane & 7;
@@ -132,6 +143,15 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const int lmid = (lane >> 3) & 1;
   const int WPG = VW / a.NB;                       // value warps per sequence of the unit
 
+  if (warp >= EW && blockIdx.x < a.units) {
+    // the queries of the first unit: into L2 (and the TLB) before the wait, read after it
+    const int u = blockIdx.x, h = u / per_h, rem = u - h * per_h, b0 = (rem / a.nrg) * a.NB;
+    const int vt = tid - EW * 32;
+    if (vt < a.NB * 32) {
+      const int tb = vt >> 5, g = (vt >> 1) & 15, half = vt & 1;     // 128-byte halves of a 256-byte query row
+      if (b0 + tb < a.B && g < a.G) prefetch_l2(a.q + ((size_t)(b0 + tb) * a.H_kv * a.G + (size_t)h * a.G + g) * D + half * 64);
+    }
+  }
   grid_dep_wait();
   grid_dep_launch();
   if (blockIdx.x == 0 && tid == 0) *a.status = 0;
@@ -235,13 +255,25 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         ++si;
         release();
       }
-      // ---------------- text stages belong to the value warps ----------------
-      for (int ts = 0; ts < nts; ++ts) {
-        wait_on(&bars.full[slot], phase);
-        release();
-      }
+      // ---------------- the text stages belong to the value warps: this warp only hands their slots back, as they
+      // fill, between the steps of the softmax below (a look at the barrier, no wait, until the last step) ----------------
+      int ts_done = 0;
+      auto pass_text = [&](bool block) {
+        while (ts_done < nts) {
+          if (block) {
+            wait_on(&bars.full[slot], phase);
+          } else {
+            int ok = 0;
+            if (lane == 0) ok = mbar_test_wait(&bars.full[slot], phase) ? 1 : 0;
+            if (!__shfl_sync(0xffffffffu, ok, 0)) break;
+          }
+          release();
+          ++ts_done;
+        }
+      };
 
-      // ---------------- joint softmax over the unit's blocks and text rows ----------------
+      // ---------------- softmax of the vision logits relative to the vision-only maximum, while the value warps attend
+      // the text rows; the text rows' maxima and sums join afterwards through one factor per (sequence, head) ----------------
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
@@ -254,9 +286,10 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
           if (t4 == 0) rmax[warp * RT + mt * 16 + gid + 8 * hr] = rvalid[mt][hr] ? mx : -INFINITY;
         }
-      named_barrier_sync(1, FCONS);                                   // B1: row maxima and text maxima are in place
+      pass_text(false);
+      named_barrier_sync(2, ETH);                                     // row maxima of every expansion warp
       if (warp == 0) {
-        // maximum of every expansion row over the warps, then of every (sequence, head) over its blocks and text rows
+        // maximum of every expansion row over the warps, then of every (sequence, head) over its blocks
         for (int x = lane; x < RT; x += 32) {
           float mx = -INFINITY;
 #pragma unroll
@@ -270,19 +303,19 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           if (g < G && tb < nbv) {
             mx = -INFINITY;
             for (int rl = 0; rl < rbv; ++rl) mx = fmaxf(mx, rmax[(tb * RB + rl) * G + g]);
-            for (int w = tb * WPG; w < (tb + 1) * WPG; ++w) mx = fmaxf(mx, tmax[w * 16 + g]);
           }
-          hmax[x] = mx;
+          hvmax[x] = mx;
         }
       }
-      named_barrier_sync(1, FCONS);                                   // B2: head maxima
+      pass_text(false);
+      named_barrier_sync(2, ETH);                                     // vision maxima per (sequence, head)
       uint32_t pf[MT][KTW][4];                        // P (bf16) of this warp's column groups, as MMA operand fragments
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
         for (int hr = 0; hr < 2; ++hr) {
           const bool ok = rvalid[mt][hr];
-          const float M = hmax[rhead[mt][hr]];
+          const float M = hvmax[rhead[mt][hr]];
           float sum = 0.f;
 #pragma unroll
           for (int nt = 0; nt < 2 * KTW; ++nt)
@@ -304,7 +337,8 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           pf[mt][kt][3] = pack2_bf16(accL[mt][2 * kt + 1][2], accL[mt][2 * kt + 1][3]);
         }
       }
-      named_barrier_sync(1, FCONS);                                   // B3: row sums and text sums are in place
+      pass_text(false);
+      named_barrier_sync(2, ETH);                                     // row sums of every expansion warp
       if (warp == 0) {
         for (int x = lane; x < RT; x += 32) {
           float sm_ = 0.f;
@@ -312,12 +346,37 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           for (int w = 0; w < EW; ++w) sm_ += rsum[w * RT + x];
           rsum[x] = sm_;
         }
-        __syncwarp();
+      }
+      pass_text(true);
+      named_barrier_sync(1, FCONS);                                   // B1: the text maxima are in place
+      if (warp == 0) {
+        // joint maximum of every (sequence, head) and the factor that moves its vision weights to it
+        for (int x = lane; x < a.NB * 16; x += 32) {
+          const int tb = x >> 4, g = x & 15;
+          float mx = 0.f, f = 0.f;
+          if (g < G && tb < nbv) {
+            mx = hvmax[x];
+            for (int w = tb * WPG; w < (tb + 1) * WPG; ++w) mx = fmaxf(mx, tmax[w * 16 + g]);
+            f = fast_exp2(hvmax[x] - mx);
+          }
+          hmax[x] = mx;
+          hfv[x] = f;
+        }
+      }
+      named_barrier_sync(1, FCONS);                                   // B2: head maxima
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int hr = 0; hr < 2; ++hr)
+          if (warp == 0 && t4 == 0) rowf[mt * 16 + gid + 8 * hr] = rvalid[mt][hr] ? hfv[rhead[mt][hr]] : 0.f;
+      named_barrier_sync(1, FCONS);                                   // B3: text sums are in place
+      if (warp == 0) {
         for (int x = lane; x < a.NB * 16; x += 32) {
           const int tb = x >> 4, g = x & 15;
           float vs = 0.f, tsm = 0.f;
           if (g < G && tb < nbv) {
             for (int rl = 0; rl < rbv; ++rl) vs += rsum[(tb * RB + rl) * G + g];
+            vs *= hfv[x];
             for (int w = tb * WPG; w < (tb + 1) * WPG; ++w) tsm += tsum[w * 16 + g];
           }
           vsum[x] = vs;
@@ -373,7 +432,7 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             float w = 0.f;
 #pragma unroll
             for (int x = 0; x < EW; ++x) w += wp[x * RT * 16];
-            W_sm[wbuf * ((RT + 16) * SLD) + (idx >> 4) * SLD + (idx & 15)] = __float2bfloat16_rn(w);
+            W_sm[wbuf * ((RT + 16) * SLD) + (idx >> 4) * SLD + (idx & 15)] = __float2bfloat16_rn(w * rowf[idx >> 4]);
           }
           named_barrier_arrive(BAR_W_READY + (int)wbuf, FCONS);
           ++wi;
@@ -849,7 +908,7 @@ FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
   p.off_wred = take((uint32_t)2 * p.EW * rt * 16 * 4);
   p.off_rstat = take((uint32_t)2 * p.EW * rt * 4);
   p.off_tstat = take((uint32_t)2 * p.VW * 16 * 4);
-  p.off_hstat = take((uint32_t)3 * p.NB * 16 * 4);
+  p.off_hstat = take((uint32_t)(5 * p.NB * 16 + rt) * 4);
   p.yhg = G > 4 ? 8 : (G > 2 ? 4 : 2);
   p.off_yred = take((uint32_t)p.VW * p.yhg * D * 4);
   p.misc_bytes = off;
@@ -901,7 +960,7 @@ FusedPlan plan_fused_text(const kvc_layer* L, int B, int T) {   // T = all plain
   p.off_wred = take((uint32_t)2 * p.EW * rt * 16 * 4);
   p.off_rstat = take((uint32_t)2 * p.EW * rt * 4);
   p.off_tstat = take((uint32_t)2 * p.VW * 16 * 4);
-  p.off_hstat = take((uint32_t)3 * p.NB * 16 * 4);
+  p.off_hstat = take((uint32_t)(5 * p.NB * 16 + rt) * 4);
   p.yhg = G > 4 ? 8 : (G > 2 ? 4 : 2);
   p.off_yred = take((uint32_t)p.VW * p.yhg * D * 4);
   p.misc_bytes = off;
