@@ -953,21 +953,34 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
             for (int p = 0; p < a.nrg; ++p) mlm[2 * npg + p * G + vtid] = fast_exp2(mlm[p * G + vtid] - M) * inv;
           }
           named_barrier_sync(3, VTH);
-          for (int idx = vtid; idx < G * D; idx += VTH) {
-            const int g = idx >> 7, col = idx & (D - 1);
+          // four output columns per thread, up to eight partials' loads in flight: the merge is a chain of L2 round trips
+          for (int idx = vtid; idx < G * (D / 4); idx += VTH) {
+            const int g = idx >> 5, col = (idx & 31) * 4;
             const float* yp = a.part_y + (p0 + g) * D + col;
-            float num = 0.f;
+            const float* wp = mlm + 2 * npg + g;
+            float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+            auto acc = [&](const float4& y, float w) {
+              num.x = fmaf(w, y.x, num.x); num.y = fmaf(w, y.y, num.y); num.z = fmaf(w, y.z, num.z); num.w = fmaf(w, y.w, num.w);
+            };
             int p = 0;
-            for (; p + 4 <= a.nrg; p += 4) {            // four independent loads in flight
-              const float y0 = __ldcg(yp + (size_t)(p + 0) * G * D), y1 = __ldcg(yp + (size_t)(p + 1) * G * D);
-              const float y2 = __ldcg(yp + (size_t)(p + 2) * G * D), y3 = __ldcg(yp + (size_t)(p + 3) * G * D);
-              num = fmaf(mlm[2 * npg + (p + 0) * G + g], y0, num);
-              num = fmaf(mlm[2 * npg + (p + 1) * G + g], y1, num);
-              num = fmaf(mlm[2 * npg + (p + 2) * G + g], y2, num);
-              num = fmaf(mlm[2 * npg + (p + 3) * G + g], y3, num);
+            for (; p + 8 <= a.nrg; p += 8) {
+              float4 y[8];
+#pragma unroll
+              for (int k = 0; k < 8; ++k) y[k] = __ldcg(reinterpret_cast<const float4*>(yp + (size_t)(p + k) * G * D));
+#pragma unroll
+              for (int k = 0; k < 8; ++k) acc(y[k], wp[(p + k) * G]);
             }
-            for (; p < a.nrg; ++p) num = fmaf(mlm[2 * npg + p * G + g], __ldcg(yp + (size_t)p * G * D), num);
-            a.out[((size_t)b0 * a.H_kv * G + (size_t)h * G + g) * D + col] = __float2bfloat16_rn(num);
+            for (; p + 4 <= a.nrg; p += 4) {
+              float4 y[4];
+#pragma unroll
+              for (int k = 0; k < 4; ++k) y[k] = __ldcg(reinterpret_cast<const float4*>(yp + (size_t)(p + k) * G * D));
+#pragma unroll
+              for (int k = 0; k < 4; ++k) acc(y[k], wp[(p + k) * G]);
+            }
+            for (; p < a.nrg; ++p) acc(__ldcg(reinterpret_cast<const float4*>(yp + (size_t)p * G * D)), wp[p * G]);
+            uint2 o;
+            o.x = pack2_bf16(num.x, num.y); o.y = pack2_bf16(num.z, num.w);
+            *reinterpret_cast<uint2*>(a.out + ((size_t)b0 * a.H_kv * G + (size_t)h * G + g) * D + col) = o;
           }
         } else {
           for (int idx = vtid; idx < G * D; idx += VTH) {
