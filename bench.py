@@ -36,9 +36,9 @@ NOMINAL_HBM_GBS = 8000.0        # nominal HBM3e bandwidth: the roofline fraction
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
 # the ncu capture summarised under profiles/, keyed by (kernel, workload name); None = not captured.
 NCU_TRAFFIC_BYTES = {
-    # profiles/fused_decode_config1.md: 185.8 MB read + 6.5 MB written per launch at T = 130 text rows; a text row costs
-    # 2 * B * H_kv * d * 2 bytes = 131072 bytes more, so the mid-run launch (T = 255.5) moves 192.3 MB + 16.4 MB
-    ("fused", "config1-llava-next-7b"): 208.7e6,
+    # profiles/fused_decode_config1.md: 185.8 MB read + 7.2 MB written per launch at T = 130 text rows; a text row costs
+    # 2 * B * H_kv * d * 2 bytes = 131072 bytes more, so the mid-run launch (T = 255.5) moves 193.0 MB + 16.4 MB
+    ("fused", "config1-llava-next-7b"): 209.4e6,
     # profiles/fused_decode_tc_config2.md: 123.0 MB read + 4.2 MB written per launch at T = 258; 32768 bytes per text
     # row more up to the mid-run launch (T = 511.5)
     ("fused_tc", "config2-qwen2-vl-7b"): 135.5e6,
