@@ -170,45 +170,55 @@ def decode_attend_definition(q, K_t, V_t, theta, U, mu, K_txt, V_txt, passthroug
 # Algorithm 1 (fused KVCapsule), with the text tail in the same softmax
 # --------------------------------------------------------------------------
 def decode_attend_fused(q, K_t, V_t, theta, U, mu, K_txt, V_txt, passthrough: bool = False):
-    """Form 2: Alg. 1's four steps, text logits joined before the softmax."""
+    """Form 2: the associative order of Alg. 1 (steps 1-4) for one decode query per sequence.
+
+    Nothing of length n x d is formed.  Per (sequence b, KV head h) and for the G query heads that read h:
+      step 1  the query meets the m retained keys of every block:           s_c[g, r, j]
+      step 2  those m scores are spread over the block's n positions by theta[h], and all R*n vision
+              logits take part in ONE softmax together with the T text logits (Sec. 3.2, decoding stage)
+      step 3  the vision probabilities are folded back to m weights per block by U[h]:  w_c[g, r, j]
+      step 4  the weights meet the compressed values; the centring vector returns with the total vision
+              probability as its coefficient; the text rows add their ordinary attention term.
+    """
     q, K_t, V_t = np.asarray(q, F64), np.asarray(K_t, F64), np.asarray(V_t, F64)
     K_txt, V_txt = np.asarray(K_txt, F64), np.asarray(V_txt, F64)
     B, H_q, d = q.shape
-    _, H_kv, R, m, _ = K_t.shape
+    H_kv, R, m = K_t.shape[1], K_t.shape[2], K_t.shape[3]
     G = H_q // H_kv
-    T = K_txt.shape[2]
-    sigma = 1.0 / np.sqrt(F64(d))
-    if passthrough:
-        n = m
-        theta = np.broadcast_to(np.eye(m, dtype=F64), (H_kv, m, m))
-        U = theta
+    if passthrough:                      # rho = 0: theta = U = I, mu = 0
+        theta = U = np.broadcast_to(np.eye(m, dtype=F64), (H_kv, m, m))
         mu = np.zeros((H_kv, d), F64)
     else:
         theta, U, mu = np.asarray(theta, F64), np.asarray(U, F64), np.asarray(mu, F64)
-        n = theta.shape[2]
-    Y = np.zeros((B, H_q, d), F64)
+    n = theta.shape[2]
+    scale = 1.0 / np.sqrt(F64(d))
+    out = np.zeros((B, H_q, d), F64)
     for b in range(B):
         for h in range(H_kv):
-            Q_bh = q[b, h * G:(h + 1) * G]                                  # [G,d]
-            # Step 1: scores in compressed sequence space, shaped [G,R,m]
-            S_full = np.stack([Q_bh @ K_t[b, h, r].T for r in range(R)], axis=1) * sigma if R else np.zeros((G, 0, m))
-            # Step 2: expand to spatial resolution, softmax (jointly with the text logits)
-            L_img = S_full @ theta[h]                                       # [G,R,n]
-            L_txt = (Q_bh @ K_txt[b, h].T) * sigma                          # [G,T]
-            L_all = np.concatenate([L_img.reshape(G, R * n), L_txt], axis=1)
-            P_all = np.stack([softmax(L_all[g]) for g in range(G)], axis=0)
-            P = P_all[:, :R * n].reshape(G, R, n)
-            P_txt = P_all[:, R * n:]
-            # Step 3: associative re-projection with transposed U
-            W = P @ U[h].T                                                  # [G,R,m]
-            # Step 4: multiply with compressed values, add the P mu term and the text values
-            y = np.zeros((G, d), F64)
-            for r in range(R):
-                y += W[:, r, :] @ V_t[b, h, r]
-            y += P.sum(axis=(1, 2))[:, None] * mu[h][None, :]
-            y += P_txt @ V_txt[b, h]
-            Y[b, h * G:(h + 1) * G] = y
-    return Y
+            for g in range(G):
+                hq = h * G + g
+                query = q[b, hq]
+                # step 1
+                s_c = np.zeros((R, m), F64)
+                for r in range(R):
+                    s_c[r] = (K_t[b, h, r] @ query) * scale
+                # step 2
+                logit_v = np.zeros((R, n), F64)
+                for r in range(R):
+                    logit_v[r] = s_c[r] @ theta[h]
+                logit_t = (K_txt[b, h] @ query) * scale
+                prob = softmax(np.concatenate([logit_v.reshape(R * n), logit_t]))
+                prob_v, prob_t = prob[:R * n].reshape(R, n), prob[R * n:]
+                # step 3
+                w_c = np.zeros((R, m), F64)
+                for r in range(R):
+                    w_c[r] = U[h] @ prob_v[r]
+                # step 4
+                y = prob_v.sum() * mu[h]
+                for r in range(R):
+                    y = y + w_c[r] @ V_t[b, h, r]
+                out[b, hq] = y + prob_t @ V_txt[b, h]
+    return out
 
 
 # --------------------------------------------------------------------------

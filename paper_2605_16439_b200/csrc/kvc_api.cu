@@ -163,7 +163,7 @@ int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out) {
   L->num_sms = 0;
   {
     const char* ex = std::getenv("KVC_EXPANSION");
-    L->use_tc = !ex ? 0 : (std::strcmp(ex, "tcgen05") == 0 ? 1 : (std::strcmp(ex, "pair") == 0 ? 2 : (std::strcmp(ex, "mma") == 0 ? -1 : 0)));
+    L->use_tc = !ex ? 0 : (std::strcmp(ex, "tcgen05") == 0 ? 1 : (std::strcmp(ex, "pair") == 0 ? 2 : (std::strcmp(ex, "mma") == 0 ? -1 : (std::strcmp(ex, "phases") == 0 ? -2 : 0))));
   }
   if (cudaGetDevice(&L->device) != cudaSuccess ||
       cudaDeviceGetAttribute(&L->num_sms, cudaDevAttrMultiProcessorCount, L->device) != cudaSuccess ||

@@ -848,6 +848,7 @@ static void warp_split(int n, int* ew, int* vw, int* ktw_max) {
 }
 
 FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
+  if (L->use_tc == -2) return FusedPlan{};      // the three-phase kernels were asked for
   if (L->use_tc >= 0) {
     // The tensor-memory variant pays per tcgen05.mma, not per expansion row: it wins for long blocks once two row
     // tiles per unit still give most SMs a unit (measured on the n = 1024, G = 7 shape: ahead from batch 16 on,

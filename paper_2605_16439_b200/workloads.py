@@ -16,7 +16,14 @@ InternVL3-shaped models, which are not available offline):
     rho_t: x_0 = e_0, x_f = rho_t x_{f-1} + sqrt(1 - rho_t^2) e_f, each e_f a
     smoothed field as above.
   * text K/V and the decode query: N(0,1).
-  * parameters theta, U [H_kv,m,n] and mu [H_kv,d]: N(0, 1/d).
+  * parameters theta, U [H_kv,m,n] and mu [H_kv,d]: N(0, 1/d) (recipe "flat": near-uniform softmaxes).
+  * recipe "peaked": theta ~ N(0, 75/m) instead, which gives the expanded vision logits a standard
+    deviation of about 3 on the smoothed fields (a few positions dominate every softmax); text keys
+    ~ N(0, 3.5^2) so that the text logits are as peaked and both sides carry probability mass.
+  * recipe "structured": theta[j, i] = 1 where idx[j] is the retained position nearest to i (every
+    position copies the score of its nearest retained key; theta[:, idx] = I), U with orthonormal
+    rows (QR of a Gaussian matrix), the query scaled by 8 (logit standard deviation about 3) and the
+    text keys ~ N(0, 0.45^2) (the scale of the smoothed vision keys, so text logits are alike).
   * retained indices: evenly spaced, idx[j] = floor(j n / m); or a sorted seeded
     random subset (irregular gathers).
 bf16 workloads are rounded to bf16 once, here, and both sides start from the
@@ -123,6 +130,31 @@ def params(H_kv: int, m: int, n: int, d: int, seed: int, device="cpu", dtype=tor
     return theta, U, mu
 
 
+def peaked_params(H_kv: int, m: int, n: int, d: int, seed: int, device="cpu", dtype=torch.float32):
+    """Recipe "peaked": as `params`, with theta ~ N(0, 75/m)."""
+    theta = gaussian((H_kv, m, n), seed * 7 + 1, device, dtype, math.sqrt(75.0 / m))
+    U = gaussian((H_kv, m, n), seed * 7 + 2, device, dtype, 1.0 / math.sqrt(d))
+    mu = gaussian((H_kv, d), seed * 7 + 3, device, dtype, 1.0 / math.sqrt(d))
+    return theta, U, mu
+
+
+def structured_params(H_kv: int, m: int, n: int, d: int, idx: torch.Tensor, seed: int, device="cpu",
+                      dtype=torch.float32):
+    """Recipe "structured": nearest-retained-position one-hot theta, orthonormal rows in U, Gaussian mu."""
+    idx2 = idx.to(torch.int64).reshape(-1, m)                       # [1 or H_kv, m]
+    pos = torch.arange(n, dtype=torch.int64)
+    theta = torch.zeros((H_kv, m, n), dtype=torch.float32)
+    for h in range(H_kv):
+        ih = idx2[h if idx2.shape[0] > 1 else 0]
+        nearest = torch.argmin((pos[None, :] - ih[:, None]).abs(), dim=0)   # [n] -> row j of the nearest retained key
+        theta[h, nearest, pos] = 1.0
+    gen = _gen(seed * 7 + 2, "cpu")
+    U = torch.stack([torch.linalg.qr(torch.randn((n, m), generator=gen, dtype=torch.float64))[0].T for _ in range(H_kv)])
+    mu = gaussian((H_kv, d), seed * 7 + 3, "cpu", torch.float32, 1.0 / math.sqrt(d))
+    return (theta.to(dtype).to(device).contiguous(), U.to(torch.float32).to(dtype).to(device).contiguous(),
+            mu.to(dtype).to(device).contiguous())
+
+
 def evenly_spaced_idx(n: int, m: int) -> torch.Tensor:
     """idx[j] = floor(j n / m), strictly increasing for m <= n; int32 [m]."""
     j = torch.arange(m, dtype=torch.int64)
@@ -143,25 +175,38 @@ def layer_seed(config_index: int, layer: int) -> int:
 
 
 def decode_inputs(shape: Shape, m: int, seed: int, device="cpu", T: int | None = None,
-                  T_cap: int | None = None):
+                  T_cap: int | None = None, recipe: str = "flat", idx: torch.Tensor | None = None):
     """All tensors of one layer's decode problem, in the storage dtype of `shape`.
 
     Returns a dict: K_vis, V_vis [B,H_kv,N_v,d]; K_txt, V_txt [B,H_kv,T_cap,d] (rows >= T are
     filled too, they must not influence the result); q [B,H_q,d]; theta, U, mu; idx [m].
+    recipe: "flat" (the benchmark configurations), "peaked" or "structured" (module docstring); idx: the retained
+    index set to use instead of the evenly spaced one.
     """
     dt = torch_dtype(shape.dtype)
     T = shape.T0 if T is None else T
     T_cap = T if T_cap is None else T_cap
     s = seed * 16
-    theta, U, mu = params(shape.H_kv, m, shape.n, shape.d, s + 5, device, dt)
+    idx = evenly_spaced_idx(shape.n, m) if idx is None else idx
+    q_gain, kt_gain = 1.0, 1.0
+    if recipe == "flat":
+        theta, U, mu = params(shape.H_kv, m, shape.n, shape.d, s + 5, device, dt)
+    elif recipe == "peaked":
+        theta, U, mu = peaked_params(shape.H_kv, m, shape.n, shape.d, s + 5, device, dt)
+        kt_gain = 3.5
+    elif recipe == "structured":
+        theta, U, mu = structured_params(shape.H_kv, m, shape.n, shape.d, idx, s + 5, device, dt)
+        q_gain, kt_gain = 8.0, 0.45
+    else:
+        raise ValueError(f"unknown recipe {recipe!r}")
     return dict(
         K_vis=vision_kv(shape.B, shape.H_kv, shape.R, shape.grid, shape.d, s + 0, device, dt, shape.ar1),
         V_vis=vision_kv(shape.B, shape.H_kv, shape.R, shape.grid, shape.d, s + 1, device, dt, shape.ar1),
-        K_txt=gaussian((shape.B, shape.H_kv, T_cap, shape.d), s + 2, device, dt),
+        K_txt=gaussian((shape.B, shape.H_kv, T_cap, shape.d), s + 2, device, dt, kt_gain),
         V_txt=gaussian((shape.B, shape.H_kv, T_cap, shape.d), s + 3, device, dt),
-        q=gaussian((shape.B, shape.H_q, shape.d), s + 4, device, dt),
+        q=gaussian((shape.B, shape.H_q, shape.d), s + 4, device, dt, q_gain),
         theta=theta, U=U, mu=mu,
-        idx=evenly_spaced_idx(shape.n, m),
+        idx=idx,
         T=T, T_cap=T_cap,
     )
 

@@ -267,6 +267,42 @@ def test_tiny_grid_brute_force():
         np.testing.assert_allclose(got[0, 0], want, atol=1e-13)
 
 
+def test_two_heads_two_blocks_brute_force():
+    """G = 2 query heads per KV head, H_kv = 2, R = 2 blocks, T = 2 text rows, per-head index sets: every step with
+    scalar loops over plain Python lists, so that the head map hq -> hq // G, the block offsets r*n + i and the
+    per-head parameters are all written out independently of the oracle's array code."""
+    r = _rng(15)
+    B, H_kv, G, R, n, m, d, T = 1, 2, 2, 2, 3, 2, 2, 2
+    H_q = H_kv * G
+    K = r.standard_normal((B, H_kv, R * n, d)); V = r.standard_normal((B, H_kv, R * n, d))
+    Kx = r.standard_normal((B, H_kv, T, d)); Vx = r.standard_normal((B, H_kv, T, d))
+    q = r.standard_normal((B, H_q, d))
+    th = r.standard_normal((H_kv, m, n)); U = r.standard_normal((H_kv, m, n)); mu = r.standard_normal((H_kv, d))
+    idx = [[0, 2], [1, 2]]
+    want = [[0.0] * d for _ in range(H_q)]
+    for hq in range(H_q):
+        h = hq // G
+        rowsK, rowsV = [], []
+        for blk in range(R):
+            Kc = [[K[0][h][blk * n + idx[h][j]][c] for c in range(d)] for j in range(m)]
+            Vc = [[sum(U[h][j][i] * (V[0][h][blk * n + i][c] - mu[h][c]) for i in range(n)) for c in range(d)] for j in range(m)]
+            for i in range(n):
+                rowsK.append([sum(th[h][j][i] * Kc[j][c] for j in range(m)) for c in range(d)])
+                rowsV.append([sum(U[h][j][i] * Vc[j][c] for j in range(m)) + mu[h][c] for c in range(d)])
+        for t in range(T):
+            rowsK.append([Kx[0][h][t][c] for c in range(d)])
+            rowsV.append([Vx[0][h][t][c] for c in range(d)])
+        logits = [sum(q[0][hq][c] * rk[c] for c in range(d)) / math.sqrt(d) for rk in rowsK]
+        mx = max(logits)
+        ex = [math.exp(l - mx) for l in logits]
+        Z = sum(ex)
+        want[hq] = [sum(ex[i] / Z * rowsV[i][c] for i in range(len(rowsV))) for c in range(d)]
+    K_t, V_t = orc.compress(K, V, np.array(idx), U, mu, n)
+    for f in (orc.decode_attend_definition, orc.decode_attend_fused):
+        got = f(q, K_t, V_t, th, U, mu, Kx, Vx)
+        np.testing.assert_allclose(got[0], np.array(want), atol=1e-13)
+
+
 def test_scalar_closed_form():
     """n = 2, m = 1, d = 1: the whole path is a three-way logistic mixture in closed form."""
     k0, k1, v0, v1 = 0.7, -0.4, 1.5, -2.0
@@ -323,6 +359,22 @@ def _golden(name):
                 k, v = line.split()
                 vals[k] = float(v)
     return vals
+
+
+def test_memory_footprint_hand_written_integers():
+    """App. D Eq. 2 on sizes small enough to count by hand (bytes): B = 1, H_kv = 1, one block of n = 4 tokens kept at
+    m = 2 (rho = 0.5), d = 2, 2-byte elements, c = 1 prompt token, t = 1 generated token.
+      compressed cache : K and V, (1 + 2 + 1) tokens x 2 channels x 2 bytes      = 2 * 16 = 32
+      S_recon(theta)   : 1 head x 2 x 4 entries x 2 bytes                         = 16
+      S_PCA(U, mu)     : U 1 x 2 x 4 x 2 bytes = 16, mu 1 x 2 x 2 bytes = 4        = 20
+    and Eq. 1 for the same sequence: (1 + 4 + 1) tokens x 2 x 2 bytes, K and V    = 48."""
+    assert orc.footprint_kvcapsule(1, 1, 1, 4, 1, 1, 2, 2, 500) == 32 + 16 + 20 == 68
+    assert orc.footprint_base(1, 1, 1, 4, 1, 2, 2) == 48
+    # three blocks, two KV heads, batch 3, 4-byte parameters beside 2-byte cache entries:
+    #   cache 2 * 3 * 2 * (1 + 3*2 + 1) * 2 * 2 = 384;  theta 2*2*4*4 = 64;  U 64 + mu 2*2*4 = 16
+    assert orc.footprint_kvcapsule(3, 2, 1, 4, 3, 1, 2, 2, 500, b_param=4) == 384 + 64 + 80 == 528
+    # the parameter terms do not grow with the batch (Sec. 4.3): only the cache term does
+    assert orc.footprint_kvcapsule(6, 2, 1, 4, 3, 1, 2, 2, 500, b_param=4) == 768 + 144
 
 
 def test_memory_footprint_closed_forms_and_paper_ratio():

@@ -51,7 +51,7 @@ def test_static_scratch_entry_point_matches_workspace_entry_point(ci, kw):
         assert float((out.float() - want.float()).abs().max()) <= tol
     # and against the CPU oracle, like every other parity test
     _, _, ref = tl.oracle_run(shape, p)
-    assert np.abs(tl.np64(outs[1]) - ref).max() <= tol
+    tl.assert_close(tl.np64(outs[1]), ref, shape.dtype)
 
 
 def test_static_scratch_rejects_shapes_beyond_its_fixed_size():
