@@ -31,20 +31,39 @@ import torch
 from paper_2605_16439_b200 import workloads as wl
 
 FALLBACK_HBM_GBS = 6650.0       # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
+FALLBACK_BF16_TFLOPS = 1400.0   # sustained dense bf16 of the same earlier measurement
 NOMINAL_HBM_GBS = 8000.0        # nominal HBM3e bandwidth: the roofline fraction of the metric is quoted against it
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from
-# the ncu capture summarised under profiles/, keyed by (kernel, workload name); None = not captured.
-NCU_TRAFFIC_BYTES = {
-    # profiles/fused_decode_config1.md: 185.8 MB read + 7.2 MB written per launch at T = 130 text rows; a text row costs
-    # 2 * B * H_kv * d * 2 bytes = 131072 bytes more, so the mid-run launch (T = 255.5) moves 193.0 MB + 16.4 MB
-    ("fused", "config1-llava-next-7b"): 209.4e6,
-    # profiles/fused_decode_tc_config2.md: 123.0 MB read + 4.2 MB written per launch at T = 258; 32768 bytes per text
-    # row more up to the mid-run launch (T = 511.5)
-    ("fused_tc", "config2-qwen2-vl-7b"): 135.5e6,
-    # profiles/fused_decode_pair_config2.md: 123.0 MB read + 4.4 MB written per launch at T = 258, scaled the same way
-    ("fused_pair", "config2-qwen2-vl-7b"): 135.7e6,
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from one ncu capture,
+# keyed by (kernel, workload name): (bytes, digest of the kernel's source files when the counters were taken).  The
+# captures ran at 4 decode steps (text length 130 / 258); a text row adds exactly 2 * B * H_kv * d * 2 bytes, and the
+# figure here is scaled by that amount to the mid-run text length.  When the sources no longer match the digest the
+# bench reports traffic = null: the counters belong to another kernel.
+KERNEL_SOURCES = {
+    "fused": ("kvc_fused.cu", "kvc_fused.cuh", "kvc_tma.cuh", "kvc_async.cuh"),
+    "fused_tc": ("kvc_fused_tc.cu", "kvc_fused.cuh", "kvc_tcgen05.cuh", "kvc_tma.cuh", "kvc_async.cuh"),
+    "fused_pair": ("kvc_fused_tc.cu", "kvc_fused.cuh", "kvc_tcgen05.cuh", "kvc_tma.cuh", "kvc_async.cuh"),
 }
+NCU_TRAFFIC_BYTES = {
+    ("fused", "config1-llava-next-7b"): (209.4e6, "stale"),
+    ("fused_pair", "config2-qwen2-vl-7b"): (135.7e6, "stale"),
+}
+
+
+def source_digest(kernel: str) -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for f in KERNEL_SOURCES.get(kernel, ()):
+        with open(os.path.join(ROOT, "paper_2605_16439_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:12]
+
+
+def ncu_traffic(kernel: str, workload: str):
+    rec = NCU_TRAFFIC_BYTES.get((kernel, workload))
+    if rec is None or rec[1] != source_digest(kernel):
+        return None
+    return rec[0]
 
 
 def parse_args():
@@ -62,10 +81,13 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-comparator", action="store_true")
     ap.add_argument("--no-profile", action="store_true", help="do not bracket kernels with events in the timed region")
+    ap.add_argument("--no-other-configs", dest="other_configs", action="store_false",
+                    help="headline configuration only (the default run also times configurations 2 and 3 for two steps each)")
     ap.add_argument("--oracle-decode-steps", type=int, default=96)
     ap.add_argument("--pyramid", type=str, default=None, metavar="LO,HI",
                     help="decode loop with a per-layer ratio rising linearly from LO to HI permille (first to last layer), "
                          "beside the same loop at the uniform mean ratio; one JSON line (not the headline metric)")
+    ap.add_argument("--sweep-steps", type=int, default=128, help="decode steps per sweep point (the configuration states 128)")
     ap.add_argument("--sweep", action="store_true",
                     help="configuration 4: ratio x batch x vision tokens on the Qwen2-VL shape; prints one JSON line per point")
     return ap.parse_args()
@@ -191,10 +213,18 @@ class Job:
                                        self.T_cap, p["out"], self.ws)
         self.launches += len(self.layers)          # lower bound (one-kernel path); the event-bracket pass counts exactly
 
-    def step(self):
+    def step(self, marks=None):
+        """One bench step.  marks: a list that receives (start, after compress, end) events of this step, recorded on the
+        launching stream between the library calls (they add no synchronisation)."""
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)] if marks is not None else None
+        if ev: ev[0].record()
         self.compress_all()
+        if ev: ev[1].record()
         for t in range(self.shape.steps):
             self.decode_step(t)
+        if ev:
+            ev[2].record()
+            marks.append(tuple(ev))
 
 
 def timed(fn, reps: int, dev) -> float:
@@ -292,33 +322,46 @@ def run_comparator(shape: wl.Shape, dev, reps_layers: int = 8, steps: int = 16) 
 
 
 # --------------------------------------------------------------------------------------------- CPU oracle arm
-def oracle_sample(shape: wl.Shape, config_index: int, decode_steps: int) -> dict:
-    """Times the CPU oracle, as it stands, on ONE layer: one compress plus `decode_steps` decode steps of
-    Algorithm 1's order, and scales to the full job (layers x steps) by the per-call averages."""
+def oracle_sample(shape: wl.Shape, config_index: int, decode_steps: int, budget_s: float = 14.0, threads=None) -> dict:
+    """Times the CPU oracle, as it stands, on ONE layer: one compress plus up to `decode_steps` decode steps of
+    Algorithm 1's order spread over the run (stopping once `budget_s` seconds of decode work are spent, two steps at
+    least), and scales to the full job (layers x steps) by the per-call averages.  threads: limit of the BLAS thread
+    pool (None = as the host provides)."""
+    import contextlib
     import numpy as np
     from oracle import kvcapsule_oracle as orc
     try:
-        from threadpoolctl import threadpool_info
-        cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+        from threadpoolctl import threadpool_info, threadpool_limits
+        limit = threadpool_limits(limits=threads) if threads else contextlib.nullcontext()
     except Exception:
-        cores = os.cpu_count() or 1
-    m = orc.retained_len(shape.n, shape.ratio_permille)
-    T_cap = shape.T0 + shape.steps
-    p = wl.decode_inputs(shape, m, wl.layer_seed(config_index, 0), "cpu", T=shape.T0, T_cap=T_cap)
-    f64 = lambda t: t.float().numpy().astype(np.float64)
-    a = {k: f64(p[k]) for k in ("K_vis", "V_vis", "K_txt", "V_txt", "q", "theta", "U", "mu")}
-    passthrough = shape.ratio_permille == 0
-    t0 = time.perf_counter()
-    K_t, V_t = orc.compress(a["K_vis"], a["V_vis"], p["idx"].numpy(), a["U"], a["mu"], shape.n, passthrough)
-    t_comp = time.perf_counter() - t0
-    ts = []
-    stride = max(1, shape.steps // decode_steps)
-    for t in list(range(0, shape.steps, stride))[:decode_steps]:
-        T = shape.T0 + t
+        threadpool_info, limit = None, contextlib.nullcontext()
+    with limit:
+        try:
+            cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+        except Exception:
+            cores = threads or os.cpu_count() or 1
+        m = orc.retained_len(shape.n, shape.ratio_permille)
+        T_cap = shape.T0 + shape.steps
+        p = wl.decode_inputs(shape, m, wl.layer_seed(config_index, 0), "cpu", T=shape.T0, T_cap=T_cap)
+        f64 = lambda t: t.float().numpy().astype(np.float64)
+        a = {k: f64(p[k]) for k in ("K_vis", "V_vis", "K_txt", "V_txt", "q", "theta", "U", "mu")}
+        passthrough = shape.ratio_permille == 0
         t0 = time.perf_counter()
-        orc.decode_attend_fused(a["q"], K_t, V_t, a["theta"], a["U"], a["mu"], a["K_txt"][:, :, :T],
-                                a["V_txt"][:, :, :T], passthrough)
-        ts.append(time.perf_counter() - t0)
+        K_t, V_t = orc.compress(a["K_vis"], a["V_vis"], p["idx"].numpy(), a["U"], a["mu"], shape.n, passthrough)
+        t_comp = time.perf_counter() - t0
+        ts = []
+        stride = max(1, shape.steps // decode_steps)
+        picks = list(range(0, shape.steps, stride))[:decode_steps]
+        # visit the picked steps from both ends inwards so that a run cut short by the budget still spans the text lengths
+        order = [picks[i // 2] if i % 2 == 0 else picks[-1 - i // 2] for i in range(len(picks))]
+        for t in order:
+            T = shape.T0 + t
+            t0 = time.perf_counter()
+            orc.decode_attend_fused(a["q"], K_t, V_t, a["theta"], a["U"], a["mu"], a["K_txt"][:, :, :T],
+                                    a["V_txt"][:, :, :T], passthrough)
+            ts.append(time.perf_counter() - t0)
+            if len(ts) >= 2 and sum(ts) >= budget_s:
+                break
     t_dec = sum(ts) / len(ts)
     total = shape.layers * (t_comp + shape.steps * t_dec)
     return {"value": shape.B * shape.steps / total, "unit": "tokens/s", "cores": cores, "kind": "oracle",
@@ -368,7 +411,7 @@ def run_sweep(a, dev):
     from paper_2605_16439_b200 import binding as kvc
     base = wl.CONFIGS[2]
     dt = torch.bfloat16
-    steps, nl = 16, 2
+    steps, nl = a.sweep_steps, 2
     for nv in (2048, 8192, 32768):
         for B in (1, 8, 32, 64):
             for ratio in (0, 200, 400, 600, 800):
@@ -409,6 +452,7 @@ def run_sweep(a, dev):
                 fn()
                 ms_full = timed(fn, 1, dev) / steps
                 print(json.dumps({"sweep": "config4-qwen2-vl-7b", "vision_tokens": nv, "batch": B, "ratio": ratio / 1000.0, "m": m,
+                                  "decode_steps": steps,
                                   "us_per_layer_call": round(ms * 1e3, 2), "tokens_per_s_28_layers": round(B / (ms * 1e-3 * 28), 1),
                                   "contract_gbs": round(contract / (ms * 1e-3) / 1e9, 1),
                                   "frac_of_8tbs": round(contract / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS, 4),
@@ -470,6 +514,115 @@ def run_pyramid(a, shape, dev):
     print(json.dumps(out))
 
 
+def load_peaks() -> dict:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm": float(p["hbm_gbs"]), "hbm_src": "measured (MEASURED_PEAKS.json hbm_gbs)",
+                "tensor": float(p.get("bf16_tflops_sustained", p.get("bf16_tflops", FALLBACK_BF16_TFLOPS))),
+                "tensor_src": "measured (MEASURED_PEAKS.json bf16_tflops_sustained)"}
+    return {"hbm": FALLBACK_HBM_GBS, "hbm_src": "fallback", "tensor": FALLBACK_BF16_TFLOPS, "tensor_src": "fallback"}
+
+
+def measure(shape, config_index, dev, rank, world, local, steps, warmup, profile, peaks, dist=None) -> dict:
+    """Warm-up, then `steps` timed bench steps of one configuration on this rank: whole-step time (max over ranks),
+    the compress and decode parts of the SAME timed region from events recorded inside it, per-kernel event brackets
+    from a second pass, and the roofline objects.  Returns the keys of the JSON line that describe the run (plus the
+    job itself under "job")."""
+    from paper_2605_16439_b200 import binding as kvc
+    job = Job(shape, config_index, dev, rank)
+    m = job.m
+    for _ in range(warmup):
+        job.step()
+    torch.cuda.synchronize(dev)
+    calls = shape.layers * shape.steps
+    job.launches = 0
+    sampler = ClockSampler(local)
+    if dist is not None:
+        dist.barrier()
+    sampler.start()
+    marks = []
+    ms = timed(lambda: job.step(marks), steps, dev)
+    clocks = sampler.stop()
+    if dist is not None:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.barrier()
+        ms = float(t.item())
+    ms_compress = sum(e0.elapsed_time(e1) for e0, e1, _ in marks) / steps      # per step, inside the timed region
+    ms_decode = sum(e1.elapsed_time(e2) for _, e1, e2 in marks) / steps
+    # per-kernel durations: the same steps again with every launch bracketed by two CUDA events on the launching
+    # stream (the brackets sit between the kernels, so the programmatic overlap of consecutive kernels is off in this
+    # pass and the pass is a little slower than the timed region above)
+    prof, ms_bracketed = {}, None
+    if profile:
+        kvc.kvc_profile_start(steps * (5 * calls + 2 * shape.layers))
+        ms_bracketed = timed(job.step, steps, dev) / steps
+        kvc.kvc_profile_stop()
+        prof = kvc.kvc_profile_read()
+        kvc.kvc_profile_start(0)
+        kvc.kvc_profile_stop()
+        job.launches = int(sum(v[1] for v in prof.values())) // max(steps, 1) * steps
+    launches = job.launches
+
+    ms_step = ms / steps
+    tokens_per_s = world * shape.B * shape.steps / (ms_step * 1e-3)
+    T_mid = shape.T0 + (shape.steps - 1) / 2.0
+    contract = contract_bytes_per_layer_call(shape, m, T_mid)
+    decode_gbs = contract * calls / (ms_decode * 1e-3) / 1e9
+    peak, peak_src = peaks["hbm"], peaks["hbm_src"]
+
+    roofline, kernels = None, {}
+    decode_kernels = ("scores", "output", "fused", "fused_tc", "fused_pair", "split_scores", "split_expand", "split_output")
+    if prof:
+        tot = sum(v[0] for v in prof.values()) or 1.0
+        for k, (t, n) in prof.items():
+            if n:
+                kernels[k] = {"launches": n, "total_ms": round(t, 3), "avg_us": round(t / n * 1e3, 3),
+                              "share": round(t / tot, 4)}
+        dom = max(decode_kernels, key=lambda k: prof.get(k, (0.0, 0))[0])
+        t_dom, n_dom = prof[dom]
+        if dom in ("fused", "fused_tc", "fused_pair"):
+            # one kernel per layer call: its launch duration is the decode part of the timed region over its launches
+            # (events recorded inside the timed region, on the launching stream; consecutive launches overlap their
+            # prologues, which the per-launch brackets of the second pass forbid)
+            alg = contract
+            avg_us = ms_decode / calls * 1e3
+        else:
+            # several kernels per layer call: the dominant one against its own stream (one of K_tilde / V_tilde, the
+            # text rows it reads, q or out), from its event brackets
+            alg = stream_kernel_bytes(shape, m, T_mid) + (
+                shape.B * shape.H_kv * int(T_mid) * shape.d * elem_bytes(shape) if dom == "split_output" else 0)
+            avg_us = t_dom / n_dom * 1e3
+        achieved = alg / (avg_us * 1e-6) / 1e9
+        roofline = {"kernel": dom, "bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                    "frac": round(achieved / peak, 4), "traffic": ncu_traffic(dom, shape.name), "peak_source": peak_src,
+                    "algorithmic_bytes_per_launch": int(alg), "avg_launch_us": round(avg_us, 3),
+                    "launches_in_timed_region": calls * steps,
+                    "avg_launch_us_bracketed": round(t_dom / n_dom * 1e3, 3)}
+    # the prefill-side compress on its own: K and V read in full, capsules written; the value projection is a dense
+    # contraction of 2 B H_kv R m n d flop per layer
+    b = elem_bytes(shape)
+    c_bytes = 2 * shape.B * shape.H_kv * shape.R * shape.n * shape.d * b + 2 * shape.B * shape.H_kv * shape.R * m * shape.d * b
+    c_flop = 2.0 * shape.B * shape.H_kv * shape.R * m * shape.n * shape.d
+    c_us = ms_compress / shape.layers * 1e3
+    compress = {"us_per_layer": round(c_us, 2), "algorithmic_bytes_per_layer": int(c_bytes),
+                "achieved_gbs": round(c_bytes / (c_us * 1e-6) / 1e9, 1), "frac_of_hbm_peak": round(c_bytes / (c_us * 1e-6) / 1e9 / peak, 4),
+                "flop_per_layer": c_flop, "achieved_tflops": round(c_flop / (c_us * 1e-6) / 1e12, 1),
+                "frac_of_tensor_peak": round(c_flop / (c_us * 1e-6) / 1e12 / peaks["tensor"], 4),
+                "tensor_peak": peaks["tensor"], "tensor_peak_source": peaks["tensor_src"],
+                "bound": "hbm (K and V are read in full; the projection runs on tcgen05 beside the stream)"}
+    return {"job": job, "value": round(tokens_per_s, 2), "ms_per_step": round(ms_step, 3),
+            "config": config_dict(shape, m), "clocks": clocks, "gpu_launches": launches,
+            "ms_per_decode_step": round(ms_decode / shape.steps, 4),
+            "ms_per_layer_call": round(ms_decode / calls, 5),
+            "ms_compress_all_layers": round(ms_compress, 3),
+            "decode_contract_gbs": round(decode_gbs, 1),
+            "decode_frac_of_8tbs": round(decode_gbs / NOMINAL_HBM_GBS, 4),
+            "decode_frac_of_measured_peak": round(decode_gbs / peak, 4),
+            "kernels": kernels, "ms_per_step_bracketed": ms_bracketed, "roofline": roofline, "compress": compress}
+
+
 def main():
     a = parse_args()
     shape = pick_shape(a)
@@ -502,95 +655,16 @@ def main():
             run_pyramid(a, shape, dev)
         return
 
-    job = Job(shape, a.config, dev, rank)
-    m = job.m
-    for _ in range(max(a.warmup, 3)):
-        job.step()
-    torch.cuda.synchronize(dev)
-
-    calls = shape.layers * shape.steps
-    job.launches = 0
-    sampler = ClockSampler(local)
-    if world > 1:
-        dist.barrier()
-    sampler.start()
-    ms = timed(job.step, a.steps, dev)
-    clocks = sampler.stop()
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dist.barrier()
-        ms = float(t.item())
-    # per-kernel durations: the same steps again with every launch bracketed by two CUDA events on the
-    # launching stream (the brackets sit between the kernels, so the programmatic overlap of consecutive
-    # kernels is off in this pass and the pass is a little slower than the timed region above)
-    prof = {}
-    ms_bracketed = None
-    if not a.no_profile:
-        kvc.kvc_profile_start(a.steps * (5 * calls + 2 * shape.layers))
-        ms_bracketed = timed(job.step, a.steps, dev) / a.steps
-        kvc.kvc_profile_stop()
-        prof = kvc.kvc_profile_read()
-        kvc.kvc_profile_start(0)
-        kvc.kvc_profile_stop()
-        job.launches = int(sum(v[1] for v in prof.values())) // max(a.steps, 1) * a.steps
-    launches = job.launches
-
-    ms_step = ms / a.steps
-    tokens_per_s = world * shape.B * shape.steps / (ms_step * 1e-3)
-
-    # decode-only and compress-only figures (context for the whole-step value)
-    ms_compress = timed(job.compress_all, 1, dev)
-    ms_decode = timed(lambda: [job.decode_step(t) for t in range(shape.steps)], 1, dev)
-    T_mid = shape.T0 + (shape.steps - 1) / 2.0
-    contract = contract_bytes_per_layer_call(shape, m, T_mid)
-    decode_gbs = contract * calls / (ms_decode * 1e-3) / 1e9
-
-    # roofline of the dominant kernel, from the event brackets recorded inside the timed region
-    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(peaks_path):
-        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
-    else:
-        peak, peak_src = FALLBACK_HBM_GBS, "fallback"
-    roofline = None
-    kernels = {}
-    if prof:
-        tot = sum(v[0] for v in prof.values()) or 1.0
-        for k, (t, n) in prof.items():
-            if n:
-                kernels[k] = {"launches": n, "total_ms": round(t, 3), "avg_us": round(t / n * 1e3, 3),
-                              "share": round(t / tot, 4)}
-        dom = max(("scores", "output", "fused", "fused_tc", "fused_pair"), key=lambda k: prof.get(k, (0.0, 0))[0])
-        t_dom, n_dom = prof[dom]
-        if dom in ("fused", "fused_tc", "fused_pair"):
-            # one kernel per layer call: its launch duration is the decode loop's device time over its launches
-            # (CUDA events around the whole loop on the launching stream; consecutive launches overlap their
-            # prologues, which the per-launch event brackets of the second pass would forbid)
-            alg = contract_bytes_per_layer_call(shape, m, T_mid)
-            avg_us = ms_decode / calls * 1e3
-        else:
-            alg = stream_kernel_bytes(shape, m, T_mid)
-            avg_us = t_dom / n_dom * 1e3
-        achieved = alg / (avg_us * 1e-6) / 1e9
-        traffic = NCU_TRAFFIC_BYTES.get((dom, shape.name))
-        roofline = {"kernel": dom, "bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
-                    "frac": round(achieved / peak, 4), "traffic": traffic, "peak_source": peak_src,
-                    "algorithmic_bytes_per_launch": int(alg), "avg_launch_us": round(avg_us, 3),
-                    "avg_launch_us_bracketed": round(t_dom / n_dom * 1e3, 3)}
-
-    line = {"metric": "decode tokens/s", "value": round(tokens_per_s, 2), "unit": "tokens/s", "n_gpus": world,
-            "steps": a.steps, "warmup": max(a.warmup, 3), "ms_per_step": round(ms_step, 3),
+    peaks = load_peaks()
+    res = measure(shape, a.config, dev, rank, world, local, a.steps, max(a.warmup, 3), not a.no_profile, peaks,
+                  dist if world > 1 else None)
+    job, m = res.pop("job"), res["config"]["m"]
+    line = {"metric": "decode tokens/s", "value": res["value"], "unit": "tokens/s", "n_gpus": world,
+            "steps": a.steps, "warmup": max(a.warmup, 3), "ms_per_step": res["ms_per_step"],
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": shape.dtype,
-            "data": "synthetic", "config": config_dict(shape, m, {"global_batch": world * shape.B,
-                                                                   "parallelism": f"batch-sharded x{world}"}),
-            "clocks": clocks, "gpu_launches": launches,
-            "ms_per_decode_step": round(ms_decode / shape.steps, 4),
-            "ms_per_layer_call": round(ms_decode / calls, 5),
-            "ms_compress_all_layers": round(ms_compress, 3),
-            "decode_contract_gbs": round(decode_gbs, 1),
-            "decode_frac_of_8tbs": round(decode_gbs / NOMINAL_HBM_GBS, 4),
-            "decode_frac_of_measured_peak": round(decode_gbs / peak, 4),
-            "kernels": kernels, "ms_per_step_bracketed": ms_bracketed, "roofline": roofline}
+            "data": "synthetic"}
+    line.update({k: v for k, v in res.items() if k not in ("value", "ms_per_step")})
+    line["config"].update({"global_batch": world * shape.B, "parallelism": f"batch-sharded x{world}"})
 
     if rank == 0 and world == 1:
         if not a.no_comparator:
@@ -602,6 +676,32 @@ def main():
                            "ms_per_step": round(e["ms"], 3)}
         if not a.no_cpu_baseline:
             line["cpu_baseline"] = oracle_sample(shape, a.config, a.oracle_decode_steps)
+            one = oracle_sample(shape, a.config, 4, budget_s=6.0, threads=1)
+            line["cpu_baseline"]["single_thread"] = {"value": one["value"], "unit": "tokens/s", "cores": 1,
+                                                     "sample": one["sample"]}
+        if a.other_configs and all(x is None for x in (a.layers, a.decode_steps, a.batch, a.ratio)):
+            # the other 7B-shaped configurations, a few bench steps each in the same process, each under its own clock
+            # sampler: per-layer-call time, roofline and the uncompressed comparator on the same shape
+            del job
+            torch.cuda.empty_cache()
+            line["other_configs"] = []
+            for ci in (2, 3):
+                if ci == a.config:
+                    continue
+                oshape = wl.CONFIGS[ci]
+                r = measure(oshape, ci, dev, rank, 1, local, 2, 1, not a.no_profile, peaks)
+                ojob = r.pop("job")
+                del ojob
+                torch.cuda.empty_cache()
+                comp = run_comparator(oshape, dev) if not a.no_comparator else None
+                line["other_configs"].append({
+                    "workload": oshape.name, "steps": 2, "warmup": 1, "value": r["value"], "unit": "tokens/s",
+                    "ms_per_step": r["ms_per_step"], "us_per_layer_call": round(r["ms_per_layer_call"] * 1e3, 2),
+                    "decode_frac_of_measured_peak": r["decode_frac_of_measured_peak"],
+                    "decode_frac_of_8tbs": r["decode_frac_of_8tbs"], "roofline": r["roofline"], "compress": r["compress"],
+                    "kernels": r["kernels"], "config": r["config"], "clocks": r["clocks"],
+                    "comparator_us": round(comp["ms_per_layer_call"] * 1e3, 2) if comp else None})
+                torch.cuda.empty_cache()
     elif world > 1 and not a.no_e2e:
         e = run_e2e(job, dev)
         t = torch.tensor([e["ms"]], device=dev)

@@ -84,7 +84,8 @@ KVC_API int kvc_retained_len(int n, int ratio_permille);
  * bf16 decode calls run Alg. 1 steps 2-3 either on mma.sync with the logits in registers or on tcgen05 with the
  * logits in tensor memory; the library picks per shape (same results within the bf16 tolerance).  The environment
  * variable KVC_EXPANSION = "tcgen05" | "mma", read when the handle is created, forces one of them where it applies;
- * "pair" the tcgen05 path run by clusters of two CTAs per (sequence, KV head). */
+ * "pair" the tcgen05 path run by clusters of two CTAs per (sequence, KV head); "phases" the three-kernel path
+ * (scores, expansion, output) that also serves fp32 storage. */
 KVC_API int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out);
 KVC_API int kvc_layer_destroy(kvc_layer* layer);
 
@@ -112,7 +113,9 @@ KVC_API int kvc_compress(const kvc_layer* layer, const void* K_vis, const void* 
  * q, out: [B][H_q][d].  K_txt, V_txt: [B][H_kv][T_cap][d] of which the first T rows are valid
  * (may be NULL when T == 0).  R == 0 attends over text only; R == 0 and T == 0 is KVC_ERR_SHAPE.
  * workspace: kvc_workspace_bytes(layer, B, R, T_max) bytes for the same B and R and any
- * T_max >= T; calls sharing a workspace must be stream-ordered. */
+ * T_max >= T; calls sharing a workspace must be stream-ordered.  All per-call device state (partials, arrival
+ * words, status word) lives in the workspace, none in the layer handle: calls on one handle with different
+ * workspaces may run concurrently on different streams. */
 KVC_API int kvc_decode_attend(const kvc_layer* layer, const void* q, const void* capsules, int B, int R,
                       const void* K_txt, const void* V_txt, int T, int T_cap, void* out,
                       void* workspace, void* stream);
@@ -149,10 +152,17 @@ KVC_API int kvc_decode_attend_static(const kvc_layer* layer, const void* q, cons
 
 /* Device status word of the last kvc_decode_attend call that used `workspace` with these B, R, T:
  * 0, or KVC_ERR_TIMEOUT if a bounded device-side wait (bulk-copy completion) gave up, in which case
- * that call's output is invalid.  Synchronous (copies one int to the host); the kernels never trap
+ * that call's output is invalid.  workspace == NULL reads the word of the last kvc_decode_attend_static
+ * call on the current device.  Synchronous (copies one int to the host); the kernels never trap
  * or spin without limit. */
 KVC_API int kvc_read_device_status(const kvc_layer* layer, int B, int R, int T, const void* workspace,
                                    int* status_out);
+
+/* Device status word of the last kvc_compress call on this handle (cleared when a compress call starts):
+ * 0, or KVC_ERR_TIMEOUT if a bounded wait of the value-projection kernel gave up, in which case the capsules
+ * of that call are invalid.  Synchronous; call it after the stream of that kvc_compress has been synchronised.
+ * Compress calls on one handle must be stream-ordered (they share this word and nothing else). */
+KVC_API int kvc_read_compress_status(const kvc_layer* layer, int* status_out);
 
 /* Self-test of the bounded device-side waits: one warp waits on a shared-memory barrier that nothing ever
  * completes, with the wait every kernel of this library uses.  Returns KVC_ERR_TIMEOUT when the wait gave up
@@ -171,9 +181,11 @@ KVC_API int kvc_selftest_bounded_wait(void* stream);
 KVC_API int kvc_collapse_theta(const void* W1, const void* W2, int H_kv, int m, int k, int n, kvc_dtype dtype,
                                void* theta_out, void* stream);
 
-/* Integer maps as the device path uses them (read back from the device copy):
- * idx_out: HOST [H_kv][m] retained indices per KV head; group_out: HOST [R*n][2] = (block r,
- * offset i) of vision token t = r*n + i (the Reshape of Alg. 1 step 1).  Either may be NULL. */
+/* Integer maps as the device path uses them: idx_out: HOST [H_kv][m] retained indices per KV head, read back
+ * from the device copy the kernels index with; group_out: HOST [R*n][2] = (block r, offset i) of vision token
+ * t = r*n + i (the Reshape of Alg. 1 step 1), written on the device by a kernel that uses the row arithmetic of
+ * the key selection and copied back.  Either may be NULL.  Synchronous; allocates and frees a temporary of
+ * 8*R*n bytes when group_out is given. */
 KVC_API int kvc_export_maps(const kvc_layer* layer, int R, int32_t* idx_out, int32_t* group_out);
 
 /* Retained length m and the row stride (in elements) of internal score buffers. */

@@ -58,6 +58,7 @@ def _lib() -> C.CDLL:
         lib.kvc_static_scratch_bytes.argtypes = []; lib.kvc_static_scratch_bytes.restype = C.c_size_t
         lib.kvc_read_device_status.argtypes = [vp, i, i, i, vp, C.POINTER(i)]
         lib.kvc_read_device_status.restype = i
+        lib.kvc_read_compress_status.argtypes = [vp, C.POINTER(i)]; lib.kvc_read_compress_status.restype = i
         lib.kvc_selftest_bounded_wait.argtypes = [vp]; lib.kvc_selftest_bounded_wait.restype = i
         lib.kvc_collapse_theta.argtypes = [vp, vp, i, i, i, i, i, vp, vp]; lib.kvc_collapse_theta.restype = i
         lib.kvc_export_maps.argtypes = [vp, i, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
@@ -182,6 +183,12 @@ def kvc_read_device_status(layer: Layer, B: int, R: int, T: int, workspace) -> i
     out = C.c_int(-99)
     _check(_lib().kvc_read_device_status(layer.handle, B, R, T, _ptr(workspace), C.byref(out)),
            "kvc_read_device_status")
+    return out.value
+
+
+def kvc_read_compress_status(layer: Layer) -> int:
+    out = C.c_int(-99)
+    _check(_lib().kvc_read_compress_status(layer.handle, C.byref(out)), "kvc_read_compress_status")
     return out.value
 
 

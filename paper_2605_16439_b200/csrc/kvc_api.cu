@@ -1,4 +1,7 @@
 // Host side of the C ABI: validation, layer handles, workspace layout, kernel sequencing.
+#include <atomic>
+#include <map>
+#include <mutex>
 #include <new>
 #include <cstdlib>
 #include <cstring>
@@ -85,6 +88,7 @@ WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap) {
     }
     w.off_fpy = take(sizeof(float) * np * D);
     w.off_fpml = take(sizeof(float2) * np);
+    w.off_fcnt = take(sizeof(unsigned long long) * (np ? (size_t)B * H_kv : 0));
   }
   w.total = off;
   return w;
@@ -95,6 +99,20 @@ WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap) {
 using namespace kvc;
 
 namespace kvc {
+cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes) {
+  static std::mutex mu;
+  static std::map<std::pair<const void*, int>, size_t> set_to;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  std::lock_guard<std::mutex> lock(mu);
+  size_t& have = set_to[std::make_pair(kernel, dev)];
+  if (have >= bytes) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess) have = bytes;
+  return e;
+}
+
 static thread_local cudaError_t g_last_cuda = cudaSuccess;
 // KVC_OK, or KVC_ERR_CUDA after remembering the error for kvc_last_cuda_error (the runtime's own slot is cleared)
 int cuda_status(cudaError_t e) {
@@ -158,8 +176,9 @@ int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out) {
   L->G = desc->H_q / desc->H_kv;
   L->passthrough = pass ? 1 : 0;
   L->d_idx = nullptr;
-  L->d_cnt = nullptr;
+  L->d_cstatus = nullptr;
   L->d_usum = nullptr;
+  L->maps = map_cache_create();
   L->num_sms = 0;
   {
     const char* ex = std::getenv("KVC_EXPANSION");
@@ -169,13 +188,14 @@ int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out) {
       cudaDeviceGetAttribute(&L->num_sms, cudaDevAttrMultiProcessorCount, L->device) != cudaSuccess ||
       cudaMalloc(&L->d_idx, idx.size() * sizeof(int32_t)) != cudaSuccess ||
       cudaMemcpy(L->d_idx, idx.data(), idx.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess ||
-      cudaMalloc(&L->d_cnt, (KVC_MAX_COUNTERS + 1) * sizeof(int)) != cudaSuccess ||
-      cudaMemset(L->d_cnt, 0, (KVC_MAX_COUNTERS + 1) * sizeof(int)) != cudaSuccess ||
+      cudaMalloc(&L->d_cstatus, sizeof(int)) != cudaSuccess ||
+      cudaMemset(L->d_cstatus, 0, sizeof(int)) != cudaSuccess ||
       (!pass && (cudaMalloc(&L->d_usum, idx.size() * sizeof(float)) != cudaSuccess ||
                  compute_usum(L, L->d_usum) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess))) {
     if (L->d_idx) cudaFree(L->d_idx);
-    if (L->d_cnt) cudaFree(L->d_cnt);
+    if (L->d_cstatus) cudaFree(L->d_cstatus);
     if (L->d_usum) cudaFree(L->d_usum);
+    map_cache_destroy(L->maps);
     delete L;
     cudaGetLastError();
     return KVC_ERR_CUDA;
@@ -187,8 +207,9 @@ int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out) {
 int kvc_layer_destroy(kvc_layer* L) {
   if (!L) return KVC_OK;
   if (L->d_idx) cudaFree(L->d_idx);
-  if (L->d_cnt) cudaFree(L->d_cnt);
+  if (L->d_cstatus) cudaFree(L->d_cstatus);
   if (L->d_usum) cudaFree(L->d_usum);
+  map_cache_destroy(L->maps);
   delete L;
   return KVC_OK;
 }
@@ -214,7 +235,8 @@ int kvc_compress(const kvc_layer* L, const void* K_vis, const void* V_vis, int B
   const size_t half = kvc_capsule_bytes(L, B, R) / 2;
   void* Kc = capsules;
   void* Vc = static_cast<char*>(capsules) + half;
-  cudaError_t e;
+  cudaError_t e = cudaMemsetAsync(L->d_cstatus, 0, sizeof(int), st);   // status word of this compress call
+  if (e != cudaSuccess) return cuda_status(e);
   if (L->passthrough) {
     e = cudaMemcpyAsync(Kc, K_vis, half, cudaMemcpyDeviceToDevice, st);
     if (e == cudaSuccess) e = cudaMemcpyAsync(Vc, V_vis, half, cudaMemcpyDeviceToDevice, st);
@@ -227,6 +249,18 @@ int kvc_compress(const kvc_layer* L, const void* K_vis, const void* V_vis, int B
 }  // extern "C"
 
 namespace kvc {
+// One token per decode call, process-wide: never 0 and never one of the byte patterns a caller is likely to have
+// filled a fresh workspace with, so that stale workspace contents cannot pass for arrivals of this call.
+static unsigned int next_token() {
+  static std::atomic<unsigned int> counter{0x1000u};
+  for (;;) {
+    const unsigned int t = counter.fetch_add(1u, std::memory_order_relaxed) + 1u;
+    const unsigned int b0 = t & 0xffu;
+    const bool uniform = ((t >> 8) & 0xffu) == b0 && ((t >> 16) & 0xffu) == b0 && (t >> 24) == b0;
+    if (t != 0u && !uniform) return t;
+  }
+}
+
 int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B, int R, const void* K_txt,
                   const void* V_txt, int T, int T_cap, void* out, void* workspace, cudaStream_t st) {
   if (!L || B < 0 || R < 0 || T < 0 || T_cap < T) return KVC_ERR_ARG;
@@ -258,6 +292,8 @@ int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B
   a.ypart = reinterpret_cast<float*>(ws + a.ws.off_ypart);
   a.ystat = reinterpret_cast<float2*>(ws + a.ws.off_ystat);
   a.cnt = reinterpret_cast<int*>(ws + a.ws.off_cnt);
+  a.fcnt = reinterpret_cast<unsigned long long*>(ws + a.ws.off_fcnt);
+  a.token = next_token();
   a.status = a.cnt + (size_t)B * L->desc.H_kv;
   a.fpart_y = reinterpret_cast<float*>(ws + a.ws.off_fpy);
   a.fpart_ml = reinterpret_cast<float2*>(ws + a.ws.off_fpml);
@@ -325,10 +361,21 @@ int kvc_selftest_bounded_wait(void* stream) {
 }
 
 int kvc_read_device_status(const kvc_layer* L, int B, int R, int T, const void* workspace, int* status_out) {
-  if (!L || !workspace || !status_out || B < 0 || R < 0 || T < 0) return KVC_ERR_ARG;
+  if (!L || !status_out || B < 0 || R < 0 || T < 0) return KVC_ERR_ARG;
+  if (!workspace) {                           // the fixed scratch array of kvc_decode_attend_static on this device
+    void* p = nullptr;
+    const int s = kvc::static_scratch(&p);
+    if (s != KVC_OK) return s;
+    workspace = p;
+  }
   const WsLayout w = ws_layout(L, B, R, T);
   const char* p = static_cast<const char*>(workspace) + w.off_cnt + sizeof(int) * (size_t)B * L->desc.H_kv;
   return cudaMemcpy(status_out, p, sizeof(int), cudaMemcpyDeviceToHost) == cudaSuccess ? KVC_OK : KVC_ERR_CUDA;
+}
+
+int kvc_read_compress_status(const kvc_layer* L, int* status_out) {
+  if (!L || !status_out) return KVC_ERR_ARG;
+  return cudaMemcpy(status_out, L->d_cstatus, sizeof(int), cudaMemcpyDeviceToHost) == cudaSuccess ? KVC_OK : KVC_ERR_CUDA;
 }
 
 int kvc_export_maps(const kvc_layer* L, int R, int32_t* idx_out, int32_t* group_out) {
@@ -338,12 +385,16 @@ int kvc_export_maps(const kvc_layer* L, int R, int32_t* idx_out, int32_t* group_
         cudaSuccess)
       return KVC_ERR_CUDA;
   }
-  if (group_out) {
-    const int n = L->desc.n;
-    for (long long t = 0; t < (long long)R * n; ++t) {
-      group_out[2 * t] = (int32_t)(t / n);
-      group_out[2 * t + 1] = (int32_t)(t % n);
-    }
+  if (group_out && R > 0) {
+    // written by a kernel with the row arithmetic of the key selection (block r, offset i -> row r*n + i)
+    const size_t bytes = (size_t)R * L->desc.n * 2 * sizeof(int32_t);
+    int32_t* d = nullptr;
+    if (cudaMalloc(&d, bytes) != cudaSuccess) return cuda_status(cudaGetLastError());
+    cudaError_t e = cudaMemset(d, 0xff, bytes);
+    if (e == cudaSuccess) e = kvc::launch_export_groups(d, R, L->desc.n, nullptr);
+    if (e == cudaSuccess) e = cudaMemcpy(group_out, d, bytes, cudaMemcpyDeviceToHost);
+    cudaFree(d);
+    if (e != cudaSuccess) return cuda_status(e);
   }
   return KVC_OK;
 }

@@ -106,6 +106,13 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
 }
 
+// every thread of every CTA of the cluster, diverged or not: no CTA leaves while a peer may still store into its
+// shared memory or arrive on its barriers
+__device__ __forceinline__ void cluster_exit_sync() {
+  asm volatile("barrier.cluster.arrive.release;\n" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire;\n" ::: "memory");
+}
+
 // programmatic dependent launch: wait for the preceding kernel of the stream to complete and flush;
 // allow the next kernel of the stream to begin launching
 __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }

@@ -4,6 +4,25 @@
 
 namespace kvc {
 
+// Row of vision token (block r, offset i) inside a (sequence, KV head)'s vision K/V: the grouping of Alg. 1 step 1.
+__host__ __device__ __forceinline__ long long vision_row(long long r, int n, int i) { return r * n + i; }
+
+// (block, offset) of every vision token as the key selection addresses them: thread (r, i) writes to entry vision_row(r, n, i)
+__global__ void export_groups_kernel(int32_t* __restrict__ out, int R, int n) {
+  const long long x = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (x >= (long long)R * n) return;
+  const int r = (int)(x / n), i = (int)(x - (long long)r * n);
+  const long long t = vision_row(r, n, i);
+  out[2 * t] = r;
+  out[2 * t + 1] = i;
+}
+
+cudaError_t launch_export_groups(int32_t* d_out, int R, int n, cudaStream_t st) {
+  const long long total = (long long)R * n;
+  export_groups_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(d_out, R, n);
+  return cudaGetLastError();
+}
+
 // K_tilde[b,h,r,j,:] = K_vis[b,h,r*n + idx[h][j],:].  One warp copies RPI rows per step.
 template <typename T>
 __global__ void __launch_bounds__(256) gather_keys_kernel(const T* __restrict__ K_vis, T* __restrict__ Kc,
@@ -20,7 +39,8 @@ __global__ void __launch_bounds__(256) gather_keys_kernel(const T* __restrict__ 
   const long long bhr = row / m;
   const int h = (int)((bhr / R) % H_kv);
   const int src = idx[h * m + j];
-  const uint4 v = __ldg(reinterpret_cast<const uint4*>(K_vis + (bhr * n + src) * D + c * EPV));
+  const long long blk = bhr % R, seq_head = bhr / R;
+  const uint4 v = __ldg(reinterpret_cast<const uint4*>(K_vis + (seq_head * R * n + vision_row(blk, n, src)) * D + c * EPV));
   *reinterpret_cast<uint4*>(Kc + row * D + c * EPV) = v;
 }
 

@@ -173,13 +173,11 @@ cudaError_t launch_project_values_mma(const kvc_layer* L, const void* V_vis, int
   a.H_kv = H_kv; a.R = R; a.n = n; a.m = m;
   a.mtiles = ceil_div(m, CM_BM);
   a.blocks = B * H_kv * R;
-  a.status = L->d_cnt + KVC_MAX_COUNTERS;          // the word behind the counters
+  a.status = L->d_cstatus;
   const size_t smem = (size_t)CM_STAGES * CM_STAGE + 1024;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(project_values_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  {
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(project_values_mma_kernel), smem);
     if (e != cudaSuccess) return e;
-    configured = true;
   }
   project_values_mma_kernel<<<(unsigned)(a.blocks * a.mtiles), (CM_WARPS + 1) * 32, smem, st>>>(tmU, tmV, a);
   return cudaGetLastError();

@@ -161,13 +161,11 @@ cudaError_t launch_project_values_tc(const kvc_layer* L, const void* V_vis, int 
   a.H_kv = H_kv; a.R = R; a.n = n; a.m = m;
   a.mtiles = ceil_div(m, CT_BM);
   a.blocks = B * H_kv * R;
-  a.status = L->d_cnt + KVC_MAX_COUNTERS;          // the word behind the counters
+  a.status = L->d_cstatus;
   const size_t smem = (size_t)CT_STAGES * CT_STAGE + 1024;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(project_values_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  {
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(project_values_tc_kernel), smem);
     if (e != cudaSuccess) return e;
-    configured = true;
   }
   project_values_tc_kernel<<<(unsigned)(a.blocks * a.mtiles), 6 * 32, smem, st>>>(tmU, tmV, a);
   return cudaGetLastError();

@@ -215,11 +215,9 @@ __global__ void __launch_bounds__(128) expand_mma_kernel(DecodeArgs a) {
 template <int NT_W>
 static cudaError_t launch_nt(const DecodeArgs& a, cudaStream_t st) {
   const size_t smem = sizeof(__nv_bfloat16) * ((size_t)XM_ROWS * (a.ms + 8) + (size_t)a.ms * XM_LD + (size_t)a.ws.cgw * XM_LD);
-  static size_t configured = 0;
-  if (smem > configured) {
-    cudaError_t e = cudaFuncSetAttribute(expand_mma_kernel<NT_W>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  {
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(expand_mma_kernel<NT_W>), smem);
     if (e != cudaSuccess) return e;
-    configured = smem;
   }
   dim3 grid(a.ws.NS, ceil_div(a.B * a.G * a.R, XM_ROWS) * a.ws.CG, a.H_kv);
   return launch_dependent(expand_mma_kernel<NT_W>, grid, dim3(128), smem, st, a);

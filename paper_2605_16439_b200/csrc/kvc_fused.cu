@@ -20,6 +20,9 @@
 // dimension as M, heads as N) so that a group of up to 8 heads costs one 8-wide tile.  A unit that holds every
 // block of its sequences writes `out` directly; otherwise the units of a (sequence, KV head) leave
 // (max, sum, y) partials and the last one to arrive merges them.
+#include <mutex>
+#include <new>
+
 #include "kvc_fused.cuh"
 
 namespace kvc {
@@ -728,9 +731,7 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         __threadfence();
         named_barrier_sync(3, VTH);
         if (vtid == 0) {
-          const int old = atomicAdd(&a.cnt[bh], 1);
-          s_last = old == a.nrg - 1 ? 1 : 0;
-          if (s_last) a.cnt[bh] = 0;                  // every unit of (sequence, head) has arrived: ready for the next call
+          s_last = arrive_is_last(&a.cnt[bh], a.token, a.nrg) ? 1 : 0;
         }
         named_barrier_sync(3, VTH);
         if (s_last) {
@@ -806,6 +807,31 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   }
   if (dead && lane == 0) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
 }
+
+}  // namespace kvc
+
+// The tensor maps over the capsule store and the parameters depend only on (B, R, capsule pointer, box shape), not on
+// the text length: a decode loop re-encodes them for the same few stores again and again, so a handle keeps the last few.
+struct kvc_map_cache {
+  struct Entry {
+    bool valid;
+    int B, R, tc, JC, RB, NB;
+    const void* Kc;
+    CUtensorMap tm[4];          // K_tilde, V_tilde, theta, U
+  };
+  std::mutex mu;
+  Entry e[8];
+  int next;
+};
+
+namespace kvc {
+
+kvc_map_cache* map_cache_create() {
+  kvc_map_cache* c = new (std::nothrow) kvc_map_cache();
+  if (c) { for (auto& x : c->e) x.valid = false; c->next = 0; }
+  return c;
+}
+void map_cache_destroy(kvc_map_cache* c) { delete c; }
 
 // ------------------------------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -889,7 +915,6 @@ FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
   p.nbg = ceil_div(B, p.NB);
   p.nrg = ceil_div(R, p.RB);
   p.units = H_kv * p.nbg * p.nrg;
-  if (p.nrg > 1 && (long long)B * H_kv > KVC_MAX_COUNTERS) return p;
   p.ncg = n / 64;
   const uint32_t chunk = (uint32_t)p.NB * p.RB * 4096u + (uint32_t)n * 32u;
   int jc = (int)(65536u / chunk);
@@ -950,7 +975,7 @@ FusedPlan plan_fused_text(const kvc_layer* L, int B, int T) {   // T = all plain
   int best_ns = 1;
   double best_eff = 0;
   for (int ns = 1; ns <= 16; ++ns) {
-    if (ns > 1 && (T / ns < 256 || bh > KVC_MAX_COUNTERS)) break;
+    if (ns > 1 && T / ns < 256) break;
     const long long units = bh * ns;
     const long long grid = units < sms ? units : sms;
     const double eff = (double)units / (double)(((units + grid - 1) / grid) * sms);
@@ -989,12 +1014,9 @@ FusedPlan plan_fused_text(const kvc_layer* L, int B, int T) {   // T = all plain
 
 template <int EW, int VW, int KTW, int NH, int MT>
 static cudaError_t launch_inst(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
-  static size_t configured = 0;
-  if (p.smem_bytes > configured) {
-    cudaError_t e = cudaFuncSetAttribute(fused_decode_kernel<EW, VW, KTW, NH, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)p.smem_bytes);
+  {
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(fused_decode_kernel<EW, VW, KTW, NH, MT>), p.smem_bytes);
     if (e != cudaSuccess) return e;
-    configured = p.smem_bytes;
   }
   return launch_dependent(fused_decode_kernel<EW, VW, KTW, NH, MT>, dim3(p.grid), dim3((EW + VW + 1) * 32), p.smem_bytes, st, tm[0],
                           tm[1], tm[2], tm[3], tm[4], tm[5], fa);
@@ -1011,7 +1033,18 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
   const int H_kv = a.H_kv, m = a.m, n = a.n, R = a.R, B = a.B;
   CUtensorMap tm[6];
   *encoded = false;
-  if (R > 0 && !a.passthrough) {
+  const bool compressed = R > 0 && !a.passthrough;
+  bool cached = false;
+  if (compressed && L->maps) {
+    std::lock_guard<std::mutex> lock(L->maps->mu);
+    for (const auto& x : L->maps->e)
+      if (x.valid && x.B == B && x.R == R && x.tc == p.tc && x.JC == p.JC && x.RB == p.RB && x.NB == p.NB && x.Kc == a.Kc) {
+        tm[0] = x.tm[0]; tm[1] = x.tm[1]; tm[4] = x.tm[2]; tm[5] = x.tm[3];
+        cached = true;
+        break;
+      }
+  }
+  if (compressed && !cached) {
     const uint64_t dims[5] = {(uint64_t)D, (uint64_t)m, (uint64_t)R, (uint64_t)H_kv, (uint64_t)B};
     const uint64_t str[4] = {256ull, (uint64_t)m * 256, (uint64_t)R * m * 256, (uint64_t)H_kv * R * m * 256};
     const uint32_t box[5] = {64u, (uint32_t)(16 * p.JC), (uint32_t)p.RB, 1u, (uint32_t)p.NB};
@@ -1039,7 +1072,7 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
     tm[4] = tm[0]; tm[5] = tm[1];
   } else if (R == 0) {
     tm[0] = tm[2]; tm[1] = tm[3]; tm[4] = tm[2]; tm[5] = tm[3];          // never used: no vision stages
-  } else {
+  } else if (!cached) {
     // theta, U [H_kv][m][n] viewed as (64 columns, m rows, n/64 column groups, H_kv): a box lands as [group][row][64]
     const uint64_t dims[4] = {64ull, (uint64_t)m, (uint64_t)p.ncg, (uint64_t)H_kv};
     const uint64_t str[3] = {(uint64_t)n * 2, 128ull, (uint64_t)m * n * 2};
@@ -1047,6 +1080,14 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
     const uint32_t box_tc[4] = {64u, 128u, 1u, 1u};     // tensor-memory variant: U by 64-column groups, 128 rows at a time
     if (!encode_tensor_map_bf16(&tm[4], a.theta, 4, dims, str, box)) return cudaSuccess;
     if (!encode_tensor_map_bf16(&tm[5], a.U, 4, dims, str, p.tc ? box_tc : box)) return cudaSuccess;
+    if (L->maps) {
+      std::lock_guard<std::mutex> lock(L->maps->mu);
+      auto& x = L->maps->e[L->maps->next];
+      L->maps->next = (L->maps->next + 1) % 8;
+      x.B = B; x.R = R; x.tc = p.tc; x.JC = p.JC; x.RB = p.RB; x.NB = p.NB; x.Kc = a.Kc;
+      x.tm[0] = tm[0]; x.tm[1] = tm[1]; x.tm[2] = tm[4]; x.tm[3] = tm[5];
+      x.valid = true;
+    }
   }
   *encoded = true;
 
@@ -1071,7 +1112,8 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
   fa.off_xstat = ring + p.off_xstat; fa.off_wrecv = ring + p.off_wrecv;
   fa.part_y = a.fpart_y;
   fa.part_ml = a.fpart_ml;
-  fa.cnt = L->d_cnt;
+  fa.cnt = a.fcnt;
+  fa.token = a.token;
   fa.status = a.status;
 
   ProfScope prof(p.tc == 2 ? KVC_KERNEL_FUSED_PAIR : (p.tc ? KVC_KERNEL_FUSED_TC : KVC_KERNEL_FUSED), st);

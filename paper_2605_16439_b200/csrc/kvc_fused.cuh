@@ -32,7 +32,8 @@ struct FusedArgs {
   uint32_t off_xstat, off_wrecv;   // pair mode of the tensor-memory variant: what the peer CTA writes
   float* part_y;      // [B*H_kv][nrg][G][D]  partial outputs (only when nrg > 1)
   float2* part_ml;    // [B*H_kv][nrg][G]     (max in log2 units, sum)
-  int* cnt;           // [B*H_kv] arrival counters, zero between calls
+  unsigned long long* cnt;   // [B*H_kv] arrival words in the caller's workspace (see arrive_is_last)
+  unsigned int token;        // this call's token, never 0
   int* status;        // device status word
 };
 
@@ -58,6 +59,22 @@ __device__ __forceinline__ RowRanges row_ranges(const FusedArgs& a, int rg) {
   r.na = r.a1 > r.a0 ? (r.a1 - r.a0 + a.TCH - 1) / a.TCH : 0;
   r.nb = r.b1 > r.b0 ? (r.b1 - r.b0 + a.TCH - 1) / a.TCH : 0;
   return r;
+}
+
+// Arrival of one unit of a (sequence, KV head) whose partials are merged by the last unit to arrive.  The word lives in
+// the caller's workspace, which is never initialised: it packs (token of the call that last touched it, arrivals of
+// that call), so whatever an earlier call or nobody left there reads as "no arrivals yet" for a new token.  The last
+// arriver clears the word, which also keeps a replayed launch (same token) correct.  Call after __threadfence().
+__device__ __forceinline__ bool arrive_is_last(unsigned long long* word, unsigned int token, int expected) {
+  unsigned long long seen = *reinterpret_cast<volatile unsigned long long*>(word);
+  for (;;) {
+    const unsigned int count = (unsigned int)(seen >> 32) == token ? (unsigned int)seen : 0u;
+    const bool last = (int)count + 1 == expected;
+    const unsigned long long want = last ? 0ull : (((unsigned long long)token << 32) | (count + 1u));
+    const unsigned long long prev = atomicCAS(word, seen, want);
+    if (prev == seen) return last;
+    seen = prev;
+  }
 }
 
 // tensor-memory variant of the kernel (kvc_fused_tc.cu): tm = the six tensor maps in the order of the kernel arguments

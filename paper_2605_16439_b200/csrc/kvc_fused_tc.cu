@@ -136,7 +136,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
 
   if (warp == PROD_WARP) {
     // ================= producer: one thread feeds the ring =================
-    if (lane != 0) return;
+    if (lane != 0) { if constexpr (PAIR) cluster_exit_sync(); return; }
     tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmTh); tma_prefetch_desc(&tmU);
     if (a.T > 0) { tma_prefetch_desc(&tmKt); tma_prefetch_desc(&tmVt); }
     bool first = true;
@@ -160,7 +160,11 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         for (int cc = 0; cc < count; ++cc) {
           const bool is_text = part == 1 && next_is_text(iu, it, a.nu, nts);
           const int c = part == 1 ? (is_text ? it++ : iu++) : cc;
-          if (!mbar_wait_bounded(&bars.empty[slot], phase)) { atomicExch(a.status, (int)KVC_ERR_TIMEOUT); return; }
+          if (!mbar_wait_bounded(&bars.empty[slot], phase)) {
+            atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
+            if constexpr (PAIR) cluster_exit_sync();
+            return;
+          }
           unsigned char* dst = sm + slot * a.stage_bytes;
           uint64_t* bar = &bars.full[slot];
           if (is_text) {
@@ -193,6 +197,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         }
       }
     }
+    if constexpr (PAIR) cluster_exit_sync();
     return;
   }
 
@@ -295,6 +300,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     named_barrier_sync(BAR_END, (CW + 1) * 32);
     tmem_dealloc(tb, (uint32_t)a.tmem_cols);
     if (dead && lane == 0) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
+    if constexpr (PAIR) cluster_exit_sync();
     return;
   }
 
@@ -582,6 +588,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     }
     named_barrier_sync(BAR_END, (CW + 1) * 32);
     if (dead && lane == 0) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
+    if constexpr (PAIR) cluster_exit_sync();
     return;
   }
 
@@ -926,9 +933,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       __threadfence();
       named_barrier_sync(3, VTH);
       if (vtid == 0) {
-        const int old = atomicAdd(&a.cnt[bh], 1);
-        s_last = old == a.nrg - 1 ? 1 : 0;
-        if (s_last) a.cnt[bh] = 0;                  // every unit of (sequence, head) has arrived: ready for the next call
+        s_last = arrive_is_last(&a.cnt[bh], a.token, a.nrg) ? 1 : 0;
       }
       named_barrier_sync(3, VTH);
       if (s_last) {
@@ -1003,6 +1008,7 @@ fused_decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   }
   named_barrier_sync(BAR_END, (CW + 1) * 32);
   if (dead && lane == 0) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
+  if constexpr (PAIR) cluster_exit_sync();
 }
 
 // ------------------------------------------------------------------------------------------ host side
@@ -1035,7 +1041,6 @@ FusedPlan plan_fused_tc(const kvc_layer* L, int B, int R) {
   p.nbg = ceil_div(B, p.NB);
   p.nrg = ceil_div(R, p.RB);
   p.units = H_kv * p.nbg * p.nrg;
-  if (p.nrg > 1 && (long long)B * H_kv > KVC_MAX_COUNTERS) return p;
   p.ncg = n / 64;
   const uint32_t chunk = (uint32_t)p.NB * p.RB * 4096u + (uint32_t)n * 32u;
   int jc = (int)(65536u / chunk);
@@ -1106,7 +1111,6 @@ FusedPlan plan_fused_pair(const kvc_layer* L, int B, int R) {
   const int GP = G <= 8 ? 8 : 16;                                      // expansion rows per block, padded
   if (L->desc.dtype != KVC_BF16 || L->passthrough || R < 1 || B < 1 || n % 256 != 0 || n > 1024 || G > 16 || m < 32) return p;
   if (reinterpret_cast<uintptr_t>(L->desc.theta) & 15 || reinterpret_cast<uintptr_t>(L->desc.U) & 15) return p;
-  if ((long long)B * H_kv > KVC_MAX_COUNTERS) return p;
   const int sms = L->num_sms > 0 ? L->num_sms : 148;
   p.tc = 2;
   p.EW = 4; p.VW = 8; p.ktw = 0;
@@ -1185,11 +1189,9 @@ FusedPlan plan_fused_pair(const kvc_layer* L, int B, int R) {
 
 template <int EW, int VW, int NH, int MT, bool PAIR>
 static cudaError_t launch_tc_inst(const CUtensorMap* tm, const FusedArgs& fa, const FusedPlan& p, cudaStream_t st) {
-  static size_t configured = 0;
-  if (p.smem_bytes > configured) {
-    cudaError_t e = cudaFuncSetAttribute(fused_decode_tc_kernel<EW, VW, NH, MT, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes);
+  {
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(fused_decode_tc_kernel<EW, VW, NH, MT, PAIR>), p.smem_bytes);
     if (e != cudaSuccess) return e;
-    configured = p.smem_bytes;
   }
   if (!PAIR)
     return launch_dependent(fused_decode_tc_kernel<EW, VW, NH, MT, PAIR>, dim3(p.grid), dim3((EW + VW + 2) * 32), p.smem_bytes, st, tm[0],

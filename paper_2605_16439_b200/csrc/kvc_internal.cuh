@@ -17,7 +17,6 @@ constexpr int EXP_ROWS = 16;        // rows per CTA in the generic expansion ker
 constexpr int EXP_IC = 64;          // vision positions per inner chunk of the expansion
 constexpr int EXP_TARGET_CTAS = 296;
 constexpr int MAX_NS = 16;          // upper bound of the n-axis splits of the expansion
-constexpr int KVC_MAX_COUNTERS = 8192;  // (sequence, KV head) arrival counters owned by a layer handle
 
 inline __host__ __device__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline __host__ __device__ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -71,6 +70,7 @@ struct WsLayout {
   size_t off_cnt;  // int [B*H_kv] arrival counters, then one int device status word
   size_t off_fpy;  // fp32 [B*H_kv][nrg][G][D]  partial outputs of the one-kernel path (units that split the block axis)
   size_t off_fpml; // float2 [B*H_kv][nrg][G]   their (max, sum)
+  size_t off_fcnt; // u64 [B*H_kv]              arrival words of the one-kernel path: (call token, arrivals)
   size_t total;
 };
 
@@ -101,6 +101,8 @@ struct FusedPlan {
 
 }  // namespace kvc
 
+struct kvc_map_cache;     // tensor maps of recent decode calls on a handle (kvc_fused.cu)
+
 struct kvc_layer {
   kvc_layer_desc desc;   // idx pointer cleared after the copy
   int m;                 // retained length
@@ -112,9 +114,9 @@ struct kvc_layer {
   int use_tc;            // expansions of the one-kernel decode path: 0 chosen per shape, 1 tcgen05, 2 tcgen05 in pairs of CTAs,
                          // -1 mma.sync (environment KVC_EXPANSION=tcgen05 | pair | mma when the handle is created)
   int32_t* d_idx;        // device [H_kv][m]
-  int* d_cnt;            // device [KVC_MAX_COUNTERS + 1] arrival counters of the one-kernel decode path (zero between
-                         // calls), then the status word of the compress kernels
+  int* d_cstatus;        // device status word of the compress kernels (cleared by every kvc_compress call)
   float* d_usum;         // device [H_kv][m] row sums of U (value compression:  U (V - 1 mu^T) = U V - (U 1) mu^T)
+  kvc_map_cache* maps;   // host: tensor maps keyed by (B, R, capsule pointer, launch plan); guarded by its own mutex
 };
 
 namespace kvc {
@@ -149,6 +151,8 @@ struct DecodeArgs {
   float* ypart;
   float2* ystat;
   int* cnt;
+  unsigned long long* fcnt;   // arrival words of the one-kernel path
+  unsigned int token;         // this call's token (never 0)
   int* status;         // device status word (0 = ok, else a kvc_status), cleared by the first kernel of the call
   float* fpart_y;      // partials of the one-kernel path
   float2* fpart_ml;
@@ -159,6 +163,10 @@ struct DecodeArgs {
 // scratch of ws_layout(L, B, R, T).total bytes
 int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B, int R, const void* K_txt,
                   const void* V_txt, int T, int T_cap, void* out, void* workspace, cudaStream_t st);
+
+// Raises a kernel's dynamic shared-memory limit to at least `bytes` on the current device.  The attribute is per device
+// (and per kernel), so the record of what has been set is keyed by (kernel, device ordinal); safe from several host threads.
+cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes);
 
 // optional event brackets around a launch (kvc_profile_*)
 bool prof_begin(int kernel_id, cudaStream_t st);
@@ -198,7 +206,11 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
 // theta[h] = W1[h] W2[h] (m x k times k x n), fp32 accumulation, one rounding to the storage type
 cudaError_t launch_collapse_theta(const void* W1, const void* W2, void* theta, int H_kv, int m, int k, int n, int dtype,
                                   cudaStream_t st);
+cudaError_t launch_export_groups(int32_t* d_out, int R, int n, cudaStream_t st);   // (block, offset) of every vision token
+int static_scratch(void** out);     // device address of the fixed scratch array on the current device (kvc_static.cu)
 void launch_wait_selftest(int* status, cudaStream_t st);   // one warp, a wait that runs out: *status = KVC_ERR_TIMEOUT
+kvc_map_cache* map_cache_create();
+void map_cache_destroy(kvc_map_cache* c);
 cudaError_t compute_usum(const kvc_layer* L, float* usum);
 cudaError_t launch_project_values_tc(const kvc_layer* L, const void* V_vis, int B, int R, void* Vc, cudaStream_t st, bool* used);
 cudaError_t launch_project_values_mma(const kvc_layer* L, const void* V_vis, int B, int R, void* Vc, cudaStream_t st, bool* used);

@@ -309,11 +309,9 @@ __global__ void __launch_bounds__(256) merge_kernel(DecodeArgs a) {
 template <typename T, int GT>
 static cudaError_t launch_output_g(const DecodeArgs& a, cudaStream_t st) {
   const size_t smem = OutSmem<T, GT>::TOTAL;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(output_kernel<T, GT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  {
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(output_kernel<T, GT>), smem);
     if (e != cudaSuccess) return e;
-    configured = true;
   }
   for (int g_base = 0; g_base < a.G; g_base += GT) {
     cudaError_t e = launch_dependent(output_kernel<T, GT>, dim3(a.ws.out_ctas), dim3(OUT_THREADS), smem, st, a, g_base);

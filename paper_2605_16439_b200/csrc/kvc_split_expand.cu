@@ -1,0 +1,222 @@
+// Split path, second kernel: Alg. 1 steps 2 and 3 for 128 expansion rows of a KV head and one range [n0, n0 + NW) of
+// the n positions of a block, as two dense products on tcgen05 with the accumulators in tensor memory:
+//   L[128 x NW]  = S[128 x m] theta[h][m x range]            A = S tile (K-major), B = theta rows (MN-major)
+//   P = 2^(L - rowmax) (bf16, in shared memory as the next A operand), rowsum
+//   Wp[128 x m]  = P[128 x NW] U[h][m x range]^T              A = P (K-major), B = rows of U (K-major), in passes of
+//                                                             at most 512 columns; the logits' columns are reused
+// Every operand tile is read as the TMA engine lays it down (128-byte swizzle).  The partial weights of the range, still
+// relative to the range's own row maximum, go to the workspace as bf16 with (rowmax, rowsum); the output kernel joins the
+// ranges of a row.  One CTA per (KV head, row tile, range); warps 0-3 = one lane per expansion row (softmax, epilogue),
+// warp 4 = MMA issue, warp 5 = TMA producer.
+#include "kvc_split.cuh"
+#include "kvc_tcgen05.cuh"
+
+namespace kvc {
+
+constexpr int SE_THREADS = 6 * 32;
+
+struct ExpandBars {
+  uint64_t full[SP_MAX_STAGES], empty[SP_MAX_STAGES];
+  uint64_t l_done;      // the logits are complete in tensor memory
+  uint64_t p_ready;     // the probabilities are in shared memory and the logits have been read (4 warps)
+  uint64_t w_done;      // a pass of the weights is complete
+  uint64_t w_free;      // a pass of the weights has been read back (4 warps)
+};
+
+__global__ void __launch_bounds__(SE_THREADS, 1)
+split_expand_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUtensorMap tmTh,
+                    const __grid_constant__ CUtensorMap tmU, const SplitArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  unsigned char* sm = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
+  __shared__ __align__(8) ExpandBars bars;
+  __shared__ uint32_t s_tmem;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  // CTA -> (KV head, row tile, range): the ranges of a tile are neighbours (they share the S tile in L2)
+  const int s = blockIdx.x % a.NS;
+  const int ht = blockIdx.x / a.NS;
+  const int tile = ht % a.ntile, h = ht / a.ntile;
+  const int n0 = s * a.NW;
+  const int ngrp = a.NW >> 6;                          // 64-column groups of the range
+  const uint32_t p_bytes = (uint32_t)a.NW * 256u;      // P: [NW/64][128 rows][128 B]
+  unsigned char* ring = sm + p_bytes;
+
+  if (tid == 0) {
+    for (int i = 0; i < a.e_stages; ++i) { mbar_init(&bars.full[i], 1); mbar_init(&bars.empty[i], 1); }
+    mbar_init(&bars.l_done, 1);
+    mbar_init(&bars.p_ready, 4);
+    mbar_init(&bars.w_done, 1);
+    mbar_init(&bars.w_free, 4);
+    fence_mbar_init();
+  }
+  if (warp == 4) tmem_alloc(&s_tmem, (uint32_t)a.tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tb = s_tmem;
+  const uint32_t th_bytes = (uint32_t)ngrp * 8192u;    // theta rows of a chunk: [group][64 rows][128 B]
+  const uint32_t u_box = (uint32_t)a.brow * 128u;
+
+  if (warp == 5) {
+    // ---------------- producer ----------------
+    if (lane == 0) {
+      tma_prefetch_desc(&tmS); tma_prefetch_desc(&tmTh); tma_prefetch_desc(&tmU);
+      uint32_t slot = 0, phase = 1;
+      bool waited = false;
+      bool ok = true;
+      for (int kc = 0; kc < a.nk1 && ok; ++kc) {
+        if (!mbar_wait_bounded(&bars.empty[slot], phase)) { ok = false; break; }
+        unsigned char* dst = ring + slot * a.e_stage_bytes;
+        mbar_expect_tx(&bars.full[slot], 16384u + th_bytes);
+        tma_load_4d(dst + 16384, &tmTh, 0, kc * 64, n0 >> 6, h, &bars.full[slot]);   // parameters: never written by the library
+        if (!waited) { grid_dep_wait(); waited = true; }                             // the scores come from the kernel before
+        tma_load_3d(dst, &tmS, kc * 64, tile * SP_TILE_ROWS, h, &bars.full[slot]);
+        if (++slot == (uint32_t)a.e_stages) { slot = 0; phase ^= 1u; }
+      }
+      for (int wp = 0; wp < a.npass && ok; ++wp)
+        for (int kc = 0; kc < ngrp && ok; ++kc) {
+          if (!mbar_wait_bounded(&bars.empty[slot], phase)) { ok = false; break; }
+          unsigned char* dst = ring + slot * a.e_stage_bytes;
+          mbar_expect_tx(&bars.full[slot], (uint32_t)a.nbox * u_box);
+          for (int bx = 0; bx < a.nbox; ++bx)
+            tma_load_3d(dst + bx * u_box, &tmU, n0 + kc * 64, wp * a.prow + bx * a.brow, h, &bars.full[slot]);
+          if (++slot == (uint32_t)a.e_stages) { slot = 0; phase ^= 1u; }
+        }
+      if (!ok) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
+    }
+  } else if (warp == 4) {
+    // ---------------- MMA issue ----------------
+    grid_dep_launch();
+    const uint32_t sm_u = smem_addr(sm), ring_u = sm_u + p_bytes;
+    const uint32_t idesc_L = umma_idesc_bf16(128, a.NW, 0, 1);
+    const uint32_t idesc_W = umma_idesc_bf16(128, a.brow, 0, 0);
+    uint32_t slot = 0, phase = 0;
+    bool dead = false;
+    auto wait_on = [&](uint64_t* bar, uint32_t parity) {
+      if (!dead && !mbar_wait_bounded(bar, parity)) dead = true;
+      __syncwarp();
+    };
+    for (int kc = 0; kc < a.nk1; ++kc) {
+      wait_on(&bars.full[slot], phase);
+      tc_fence_after();
+      if (lane == 0) {
+        const uint32_t s_u = ring_u + slot * a.e_stage_bytes, th_u = s_u + 16384u;
+        const int ksteps = min(4, (a.m - kc * 64 + 15) >> 4);
+        for (int ks = 0; ks < ksteps; ++ks) {
+          const uint64_t adesc = umma_smem_desc(s_u + (uint32_t)(ks * 32), 16u, 1024u, UMMA_LAYOUT_SW128);
+          const uint64_t bdesc = umma_smem_desc(th_u + (uint32_t)(ks * 2048), 8192u, 1024u, UMMA_LAYOUT_SW128);
+          umma_bf16(tb, adesc, bdesc, idesc_L, (kc | ks) ? 1u : 0u);
+        }
+        umma_commit(&bars.empty[slot]);
+        if (kc == a.nk1 - 1) umma_commit(&bars.l_done);
+      }
+      __syncwarp();
+      if (++slot == (uint32_t)a.e_stages) { slot = 0; phase ^= 1u; }
+    }
+    wait_on(&bars.p_ready, 0);
+    for (int wp = 0; wp < a.npass; ++wp) {
+      if (wp > 0) wait_on(&bars.w_free, (uint32_t)((wp - 1) & 1));
+      tc_fence_after();
+      for (int kc = 0; kc < ngrp; ++kc) {
+        wait_on(&bars.full[slot], phase);
+        tc_fence_after();
+        if (lane == 0) {
+          const uint32_t u_u = ring_u + slot * a.e_stage_bytes;
+          const uint32_t p_u = sm_u + (uint32_t)kc * 16384u;
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks) {
+            const uint64_t adesc = umma_smem_desc(p_u + (uint32_t)(ks * 32), 16u, 1024u, UMMA_LAYOUT_SW128);
+            for (int bx = 0; bx < a.nbox; ++bx) {
+              const uint64_t bdesc = umma_smem_desc(u_u + bx * u_box + (uint32_t)(ks * 32), 16u, 1024u, UMMA_LAYOUT_SW128);
+              umma_bf16(tb + (uint32_t)(bx * a.brow), adesc, bdesc, idesc_W, (kc | ks) ? 1u : 0u);
+            }
+          }
+          umma_commit(&bars.empty[slot]);
+          if (kc == ngrp - 1) umma_commit(&bars.w_done);
+        }
+        __syncwarp();
+        if (++slot == (uint32_t)a.e_stages) { slot = 0; phase ^= 1u; }
+      }
+    }
+    if (dead && lane == 0) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
+  } else {
+    // ---------------- warps 0-3: lane <-> expansion row ----------------
+    const int row = warp * 32 + lane;                          // row of the tile = tensor-memory lane
+    const long long rho = (long long)tile * SP_TILE_ROWS + row;
+    const bool valid = rho < a.rows_h;
+    const uint32_t trow = tb + ((uint32_t)(warp * 32) << 16);
+    bool ok = mbar_wait_bounded(&bars.l_done, 0);
+    __syncwarp();
+    tc_fence_after();
+    // pass 1: row maximum over the range
+    float mx = -INFINITY;
+    for (int c0 = 0; c0 < a.NW; c0 += 16) {
+      float v[16];
+      tmem_ld_x16(trow + (uint32_t)c0, v);
+#pragma unroll
+      for (int k = 0; k < 16; ++k) mx = fmaxf(mx, v[k]);
+    }
+    // pass 2: probabilities relative to it, as the K-major A operand of the second product
+    float sum = 0.f;
+    unsigned char* prow = sm + (uint32_t)row * 128u;
+    for (int c0 = 0; c0 < a.NW; c0 += 16) {
+      float v[16];
+      tmem_ld_x16(trow + (uint32_t)c0, v);
+      uint32_t w[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const float p0 = fast_exp2(v[2 * k] - mx), p1 = fast_exp2(v[2 * k + 1] - mx);
+        sum += p0 + p1;
+        w[k] = pack2_bf16(p0, p1);
+      }
+      const int grp = c0 >> 6, piece = (c0 & 63) >> 3;        // two 16-byte pieces: piece, piece + 1
+      unsigned char* g = prow + (uint32_t)grp * 16384u;
+      *reinterpret_cast<uint4*>(g + (((piece) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+      *reinterpret_cast<uint4*>(g + (((piece + 1) ^ (row & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+    }
+    if (valid && ok) a.stat[((size_t)h * a.NS + s) * a.rows_h + rho] = make_float2(mx, sum);
+    fence_proxy_async();                                       // P is read by the tensor core (async proxy)
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&bars.p_ready);
+    // the weights of the range, pass by pass
+    __nv_bfloat16* wrow = a.Wp + (((size_t)h * a.NS + s) * a.rows_h + (valid ? rho : 0)) * a.ms;
+    for (int wp = 0; wp < a.npass; ++wp) {
+      if (ok && !mbar_wait_bounded(&bars.w_done, (uint32_t)(wp & 1))) ok = false;
+      __syncwarp();
+      tc_fence_after();
+      const int j0 = wp * a.prow;
+      for (int c0 = 0; c0 < a.prow && j0 + c0 < a.ms; c0 += 16) {
+        float v[16];
+        tmem_ld_x16(trow + (uint32_t)c0, v);
+        if (valid && ok) {
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            const int j = j0 + c0 + 8 * half;
+            if (j < a.ms)
+              *reinterpret_cast<uint4*>(wrow + j) =
+                  make_uint4(pack2_bf16(v[8 * half], v[8 * half + 1]), pack2_bf16(v[8 * half + 2], v[8 * half + 3]),
+                             pack2_bf16(v[8 * half + 4], v[8 * half + 5]), pack2_bf16(v[8 * half + 6], v[8 * half + 7]));
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars.w_free);
+    }
+    if (!ok && lane == 0) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) tmem_dealloc(tb, (uint32_t)a.tmem_cols);
+}
+
+cudaError_t launch_split_expand(const CUtensorMap& tmS, const CUtensorMap& tmTh, const CUtensorMap& tmU, const SplitArgs& a,
+                                const SplitPlan& p, cudaStream_t st) {
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(split_expand_kernel), p.e_smem);
+  if (e != cudaSuccess) return e;
+  ProfScope prof(KVC_KERNEL_SPLIT_EXPAND, st);
+  return launch_dependent(split_expand_kernel, dim3(p.e_grid), dim3(SE_THREADS), p.e_smem, st, tmS, tmTh, tmU, a);
+}
+
+}  // namespace kvc

@@ -38,6 +38,10 @@ int scratch_for_current_device(void** out) {
 
 }  // namespace
 
+namespace kvc {
+int static_scratch(void** out) { return scratch_for_current_device(out); }
+}  // namespace kvc
+
 extern "C" {
 
 size_t kvc_static_scratch_bytes(void) { return (size_t)KVC_STATIC_SCRATCH_BYTES; }

@@ -239,6 +239,35 @@ def test_repeat_calls_are_bitwise_deterministic_and_workspace_needs_no_init():
     assert torch.equal(outs[0].view(torch.int16), outs[2].view(torch.int16))
 
 
+def test_two_streams_on_one_handle_with_separate_workspaces():
+    """All per-call device state lives in the workspace: two decode calls on the same layer handle, each with its own
+    workspace, on two streams at once, on shapes whose units leave partials that the last arriver merges."""
+    shape = wl.Shape("two-streams", 1, 3, 14, 2, 128, 8, 9, 600, 1, "bf16")       # G = 7: the block axis is split
+    pa = tl.make_problem(shape, 98, T=600, T_cap=608, recipe="peaked")
+    pb = tl.make_problem(shape, 99, T=333, T_cap=608, recipe="peaked")
+    pb["theta"], pb["U"], pb["mu"], pb["idx"] = pa["theta"], pa["U"], pa["mu"], pa["idx"]   # one parameter set, one handle
+    layer = tl.gpu_layer(shape, pa)
+    B, R = shape.B, shape.R
+    runs = []
+    for p in (pa, pb):
+        caps = kvc.alloc_capsules(layer, B, R)
+        kvc.kvc_compress(layer, p["K_vis"].cuda(), p["V_vis"].cuda(), B, R, caps)
+        runs.append(dict(p=p, caps=caps, ws=kvc.alloc_workspace(layer, B, R, 608), q=p["q"].cuda(), Kt=p["K_txt"].cuda(),
+                         Vt=p["V_txt"].cuda(), out=torch.empty((B, shape.H_q, 128), dtype=torch.bfloat16, device="cuda"),
+                         stream=torch.cuda.Stream()))
+    torch.cuda.synchronize()
+    assert kvc.kvc_read_compress_status(layer) == 0
+    for _ in range(20):                                   # interleaved launches: the kernels of the two streams overlap
+        for r in runs:
+            kvc.kvc_decode_attend(layer, r["q"], r["caps"], B, R, r["Kt"], r["Vt"], r["p"]["T"], 608, r["out"], r["ws"],
+                                  stream=r["stream"])
+    torch.cuda.synchronize()
+    for r in runs:
+        assert kvc.kvc_read_device_status(layer, B, R, r["p"]["T"], r["ws"]) == 0
+        _, _, want = tl.oracle_run(shape, r["p"])
+        tl.assert_close(tl.np64(r["out"]), want, "bf16")
+
+
 def test_decode_steps_with_growing_text_tail():
     """A few decode steps: the text tail grows by one row per step inside a fixed-capacity buffer."""
     shape = tl.small(wl.CONFIGS[1], B=1, H_q=2, H_kv=2, R=2, grid=8)

@@ -45,6 +45,8 @@ def test_static_scratch_entry_point_matches_workspace_entry_point(ci, kw):
         if i == 0:
             kvc.kvc_decode_attend_static(layer, q2, caps, B, R, Kt, Vt, T, T_cap, torch.empty_like(want))
     torch.cuda.synchronize()
+    # the status word of the static call sits in the fixed array: read with no workspace pointer
+    assert kvc.kvc_read_device_status(layer, B, R, T, None) == 0
     tol = tl.TOL[shape.dtype]
     for out in outs:
         assert torch.isfinite(out.float()).all()
