@@ -214,7 +214,10 @@ typedef enum {
   KVC_KERNEL_FUSED = 7,           /* Alg. 1 steps 1-4 + text + normalisation in one kernel (bf16) */
   KVC_KERNEL_FUSED_TC = 8,        /* the same kernel with steps 2-3 on tcgen05 / tensor memory (see kvc_layer_create) */
   KVC_KERNEL_FUSED_PAIR = 9,      /* the tensor-memory kernel run by clusters of two CTAs per (sequence, KV head) */
-  KVC_KERNEL_COUNT = 10
+  KVC_KERNEL_SPLIT_SCORES = 10,   /* three-kernel bf16 path: Alg. 1 step 1, one pass over K_tilde */
+  KVC_KERNEL_SPLIT_EXPAND = 11,   /* its steps 2-3 on tcgen05, per 128 expansion rows and range of the n axis */
+  KVC_KERNEL_SPLIT_OUTPUT = 12,   /* its step 4, the text rows and the normalisation, one pass over V_tilde and text K/V */
+  KVC_KERNEL_COUNT = 13
 } kvc_kernel_id;
 KVC_API int kvc_profile_start(int max_launches);
 KVC_API int kvc_profile_stop(void);

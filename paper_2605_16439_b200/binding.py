@@ -226,7 +226,7 @@ def capsule_views(layer: Layer, capsules, B: int, R: int):
     return (capsules[:half].view(layer.dtype).view(shape), capsules[half:2 * half].view(layer.dtype).view(shape))
 
 
-KVC_KERNEL_COUNT = 10
+KVC_KERNEL_COUNT = 13
 
 
 def kvc_profile_start(max_launches: int) -> None:

@@ -8,6 +8,7 @@
 #include <vector>
 
 #include "kvc_internal.cuh"
+#include "kvc_split.cuh"
 
 namespace kvc {
 
@@ -89,6 +90,14 @@ WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap) {
     w.off_fpy = take(sizeof(float) * np * D);
     w.off_fpml = take(sizeof(float2) * np);
     w.off_fcnt = take(sizeof(unsigned long long) * (np ? (size_t)B * H_kv : 0));
+  }
+  {
+    size_t sb = 0;
+    if (B > 0 && R > 0) {
+      const SplitPlan sp = plan_split(L, B, R);
+      if (sp.ok) sb = split_ws(L, sp, B, R).bytes;
+    }
+    w.off_split = take(sb);
   }
   w.total = off;
   return w;
@@ -182,7 +191,7 @@ int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out) {
   L->num_sms = 0;
   {
     const char* ex = std::getenv("KVC_EXPANSION");
-    L->use_tc = !ex ? 0 : (std::strcmp(ex, "tcgen05") == 0 ? 1 : (std::strcmp(ex, "pair") == 0 ? 2 : (std::strcmp(ex, "mma") == 0 ? -1 : (std::strcmp(ex, "phases") == 0 ? -2 : 0))));
+    L->use_tc = !ex ? 0 : (std::strcmp(ex, "tcgen05") == 0 ? 1 : (std::strcmp(ex, "pair") == 0 ? 2 : (std::strcmp(ex, "mma") == 0 ? -1 : (std::strcmp(ex, "phases") == 0 ? -2 : (std::strcmp(ex, "split") == 0 ? 3 : 0)))));
   }
   if (cudaGetDevice(&L->device) != cudaSuccess ||
       cudaDeviceGetAttribute(&L->num_sms, cudaDevAttrMultiProcessorCount, L->device) != cudaSuccess ||
@@ -249,6 +258,12 @@ int kvc_compress(const kvc_layer* L, const void* K_vis, const void* V_vis, int B
 }  // extern "C"
 
 namespace kvc {
+// Which bf16 shapes take the three-kernel path (the others take the one-kernel path): forced by KVC_EXPANSION=split.
+static bool use_split(const kvc_layer* L, int B, int R) {
+  if (L->use_tc != 3) return false;
+  return plan_split(L, B, R).ok != 0;
+}
+
 // One token per decode call, process-wide: never 0 and never one of the byte patterns a caller is likely to have
 // filled a fresh workspace with, so that stale workspace contents cannot pass for arrivals of this call.
 static unsigned int next_token() {
@@ -297,16 +312,23 @@ int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B
   a.status = a.cnt + (size_t)B * L->desc.H_kv;
   a.fpart_y = reinterpret_cast<float*>(ws + a.ws.off_fpy);
   a.fpart_ml = reinterpret_cast<float2*>(ws + a.ws.off_fpml);
+  a.split_base = ws + a.ws.off_split;
 
   // bf16 storage with TMA-compatible shapes and pointers: the whole of Algorithm 1 in one kernel
   {
     // R == 0 (text rows only, the uncompressed comparator): the same kernel with text stages only
     // rho = 0 stores K and V verbatim: vision rows and text rows are attended as plain rows by the text-only mode
     const bool plain = R == 0 || L->passthrough;
-    const FusedPlan fp = plain ? plan_fused_text(L, B, R * L->desc.n + T) : plan_fused(L, B, R);
     const uintptr_t align = reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(capsules) |
                             reinterpret_cast<uintptr_t>(out) | (T > 0 ? reinterpret_cast<uintptr_t>(K_txt) |
                             reinterpret_cast<uintptr_t>(V_txt) : 0) | reinterpret_cast<uintptr_t>(L->desc.mu);
+    if (!plain && (align & 15) == 0 && use_split(L, B, R)) {
+      const SplitPlan sp = plan_split(L, B, R);
+      bool encoded = false;
+      const cudaError_t se = launch_split(L, a, sp, st, &encoded);
+      if (encoded) return cuda_status(se);
+    }
+    const FusedPlan fp = plain ? plan_fused_text(L, B, R * L->desc.n + T) : plan_fused(L, B, R);
     if (fp.ok && (align & 15) == 0) {
       bool encoded = false;
       const cudaError_t fe = launch_fused(L, a, fp, st, &encoded);

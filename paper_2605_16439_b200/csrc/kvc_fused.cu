@@ -853,7 +853,7 @@ static EncodeTiledFn encode_fn() {
 }
 
 bool encode_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
-                            const uint64_t* strides_bytes, const uint32_t* box) {
+                            const uint64_t* strides_bytes, const uint32_t* box, bool swizzle128) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t gd[5], gs[4];
@@ -861,7 +861,8 @@ bool encode_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const 
   for (int i = 0; i < rank; ++i) { gd[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
   for (int i = 0; i + 1 < rank; ++i) gs[i] = strides_bytes[i];
   return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gd, gs, bx, es,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -875,7 +876,7 @@ static void warp_split(int n, int* ew, int* vw, int* ktw_max) {
 
 FusedPlan plan_fused(const kvc_layer* L, int B, int R) {
   if (L->use_tc == -2) return FusedPlan{};      // the three-phase kernels were asked for
-  if (L->use_tc >= 0) {
+  if (L->use_tc >= 0 && L->use_tc != 3) {
     // The tensor-memory variant pays per tcgen05.mma, not per expansion row: it wins for long blocks once two row
     // tiles per unit still give most SMs a unit (measured on the n = 1024, G = 7 shape: ahead from batch 16 on,
     // behind at batches 1-4 where units of half the size halve the latency).

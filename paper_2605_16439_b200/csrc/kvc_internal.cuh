@@ -71,6 +71,7 @@ struct WsLayout {
   size_t off_fpy;  // fp32 [B*H_kv][nrg][G][D]  partial outputs of the one-kernel path (units that split the block axis)
   size_t off_fpml; // float2 [B*H_kv][nrg][G]   their (max, sum)
   size_t off_fcnt; // u64 [B*H_kv]              arrival words of the one-kernel path: (call token, arrivals)
+  size_t off_split;// the regions of the three-kernel bf16 path (kvc_split.cuh), 0 bytes when the shape does not take it
   size_t total;
 };
 
@@ -156,6 +157,7 @@ struct DecodeArgs {
   int* status;         // device status word (0 = ok, else a kvc_status), cleared by the first kernel of the call
   float* fpart_y;      // partials of the one-kernel path
   float2* fpart_ml;
+  void* split_base;    // regions of the three-kernel bf16 path
   WsLayout ws;
 };
 

@@ -81,6 +81,9 @@ const char* kvc_kernel_name(int kernel_id) {
     case KVC_KERNEL_FUSED: return "fused";
     case KVC_KERNEL_FUSED_TC: return "fused_tc";
     case KVC_KERNEL_FUSED_PAIR: return "fused_pair";
+    case KVC_KERNEL_SPLIT_SCORES: return "split_scores";
+    case KVC_KERNEL_SPLIT_EXPAND: return "split_expand";
+    case KVC_KERNEL_SPLIT_OUTPUT: return "split_output";
     default: return "?";
   }
 }

@@ -1,0 +1,190 @@
+// Host side of the three-kernel bf16 decode path: launch plan, workspace regions, tensor maps, the three launches.
+#include "kvc_split.cuh"
+
+namespace kvc {
+
+cudaError_t launch_split_scores(const CUtensorMap& tmK, const SplitArgs& a, const SplitPlan& p, cudaStream_t st);
+cudaError_t launch_split_expand(const CUtensorMap& tmS, const CUtensorMap& tmTh, const CUtensorMap& tmU, const SplitArgs& a,
+                                const SplitPlan& p, cudaStream_t st);
+cudaError_t launch_split_output(const CUtensorMap* tm, const SplitArgs& a, const SplitPlan& p, cudaStream_t st);
+
+constexpr uint32_t SP_SMEM_LIMIT = 232448;      // 227 KB per CTA on sm_100
+
+SplitPlan plan_split(const kvc_layer* L, int B, int R) {
+  SplitPlan p{};
+  const int G = L->G, n = L->desc.n, m = L->m, H_kv = L->desc.H_kv;
+  if (L->desc.dtype != KVC_BF16 || L->passthrough || R < 1 || B < 1 || n % 64 != 0 || G > 16) return p;
+  if ((reinterpret_cast<uintptr_t>(L->desc.theta) | reinterpret_cast<uintptr_t>(L->desc.U)) & 15) return p;
+  const int sms = L->num_sms > 0 ? L->num_sms : 148;
+  p.rows_h = B * R * G;
+  p.ntile = ceil_div(p.rows_h, SP_TILE_ROWS);
+  p.ms = (m + 7) & ~7;
+  p.nk1 = ceil_div(m, 64);
+  // ranges of the n axis: widths of 64..256 columns that divide n; the fewest ranges that still give most SMs a CTA
+  const int ncg = n / 64;
+  p.NS = 0;
+  for (int ns = 1; ns <= ncg; ++ns) {
+    if (ncg % ns != 0 || n / ns > 256) continue;
+    p.NS = ns;
+    if ((long long)H_kv * p.ntile * ns >= (sms * 2) / 3) break;
+  }
+  if (p.NS == 0) return p;
+  p.NW = n / p.NS;
+  if ((long long)R * p.NS > 128) return p;            // the output kernel keeps a factor per (block, range, head) in shared memory
+  // passes over the weights: at most 512 tensor-memory columns each, cut into one or two boxes of rows of U
+  const int mpad = (m + 15) & ~15;
+  p.npass = ceil_div(mpad, 512);
+  p.prow = (ceil_div(mpad, p.npass) + 31) & ~31;
+  p.nbox = p.prow > 256 ? 2 : 1;
+  p.brow = p.prow / p.nbox;
+  int cols = p.prow > p.NW ? p.prow : p.NW;
+  p.tmem_cols = 32;
+  while (p.tmem_cols < cols) p.tmem_cols <<= 1;
+  p.e_p_bytes = (uint32_t)p.NW * 256u;
+  const uint32_t st1 = 16384u + (uint32_t)(p.NW / 64) * 8192u, st2 = (uint32_t)p.prow * 128u;
+  p.e_stage_bytes = ((st1 > st2 ? st1 : st2) + 1023u) & ~1023u;
+  p.e_stages = (int)((SP_SMEM_LIMIT - 2048u - p.e_p_bytes) / p.e_stage_bytes);
+  if (p.e_stages > 4) p.e_stages = 4;
+  if (p.e_stages < 2) return p;
+  p.e_smem = (size_t)p.e_p_bytes + (size_t)p.e_stages * p.e_stage_bytes + 1024;
+  p.e_grid = H_kv * p.ntile * p.NS;
+  // score kernel
+  p.s_tiles_bh = ceil_div(R * m, SP_TILE_ROWS);
+  p.s_stages = 6;
+  p.s_smem = (size_t)p.s_stages * 32768 + 1024;
+  {
+    const long long items = (long long)B * H_kv * p.s_tiles_bh;
+    p.s_grid = (int)(items < sms ? items : sms);
+  }
+  // output kernel
+  p.vt = ceil_div(m, SP_OUT_ROWS);
+  p.o_w_bytes = (uint32_t)(p.NS * G) * 128u;
+  p.o_stage_bytes = 32768u;
+  if (16384u + p.o_w_bytes > p.o_stage_bytes) return p;
+  {
+    const int NH = G > 8 ? 2 : 1;
+    uint32_t off = 0;
+    auto take = [&](uint32_t bytes) { uint32_t o = off; off = (off + bytes + 127u) & ~127u; return o; };
+    p.o_off_q = take(16 * 136 * 2);
+    p.o_off_fac = take((uint32_t)(R * p.NS) * 16u * 8u);
+    p.o_off_red = take(8u * NH * 8u * 64u * 4u);
+    p.o_off_stat = take((2 * 8 * 16 + 32) * 4);
+    p.o_stages = (int)((SP_SMEM_LIMIT - 2048u - off) / p.o_stage_bytes);
+    if (p.o_stages > SP_MAX_STAGES) p.o_stages = SP_MAX_STAGES;
+    if (p.o_stages < 2) return p;
+    const uint32_t ring = (uint32_t)p.o_stages * p.o_stage_bytes;
+    p.o_off_q += ring; p.o_off_fac += ring; p.o_off_red += ring; p.o_off_stat += ring;
+    p.o_smem = (size_t)ring + off + 1024;
+  }
+  {
+    const long long items = (long long)B * H_kv * R * p.vt;
+    p.o_grid = (int)(items < sms ? items : sms);
+    const long long bh = (long long)B * H_kv;
+    p.nslot_v = (int)((p.o_grid + bh - 1) / bh) + 1;
+    p.nslot_t = p.nslot_v;
+  }
+  p.ok = 1;
+  return p;
+}
+
+SplitWs split_ws(const kvc_layer* L, const SplitPlan& p, int B, int R) {
+  SplitWs w{};
+  (void)R;
+  const int H_kv = L->desc.H_kv, G = L->G;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  w.off_S = take(sizeof(__nv_bfloat16) * (size_t)H_kv * p.rows_h * p.ms);
+  w.off_Wp = take(sizeof(__nv_bfloat16) * (size_t)H_kv * p.NS * p.rows_h * p.ms);
+  w.off_stat = take(sizeof(float2) * (size_t)H_kv * p.NS * p.rows_h);
+  const size_t nslot = (size_t)p.nslot_v + p.nslot_t;
+  w.off_py = take(sizeof(float) * (size_t)B * H_kv * nslot * G * D);
+  w.off_pml = take(sizeof(float2) * (size_t)B * H_kv * nslot * G);
+  w.off_cnt = take(sizeof(int) * (size_t)B * H_kv);
+  w.bytes = off;
+  return w;
+}
+
+cudaError_t launch_split(const kvc_layer* L, const DecodeArgs& a, const SplitPlan& p, cudaStream_t st, bool* encoded) {
+  const int H_kv = a.H_kv, m = a.m, n = a.n, R = a.R, B = a.B, G = a.G;
+  *encoded = false;
+  char* ws = reinterpret_cast<char*>(a.split_base);
+  const SplitWs w = split_ws(L, p, B, R);
+  CUtensorMap tmK, tmS, tmTh, tmU, tmO[4];
+  {
+    // K_tilde as (channels, R m rows of a pair, pairs): rows past the pair's last are zero-filled, not read
+    const uint64_t dims[3] = {(uint64_t)D, (uint64_t)R * m, (uint64_t)B * H_kv};
+    const uint64_t str[2] = {256ull, (uint64_t)R * m * 256};
+    const uint32_t box[3] = {64u, (uint32_t)SP_TILE_ROWS, 1u};
+    if (!encode_tensor_map_bf16(&tmK, a.Kc, 3, dims, str, box)) return cudaSuccess;
+  }
+  {
+    const uint64_t dims[3] = {(uint64_t)m, (uint64_t)p.rows_h, (uint64_t)H_kv};
+    const uint64_t str[2] = {(uint64_t)p.ms * 2, (uint64_t)p.rows_h * p.ms * 2};
+    const uint32_t box[3] = {64u, (uint32_t)SP_TILE_ROWS, 1u};
+    if (!encode_tensor_map_bf16(&tmS, ws + w.off_S, 3, dims, str, box)) return cudaSuccess;
+  }
+  {
+    // theta [H_kv][m][n] viewed as (64 columns, m rows, n/64 column groups, H_kv): a box lands as [group][row][64]
+    const uint64_t dims[4] = {64ull, (uint64_t)m, (uint64_t)(n / 64), (uint64_t)H_kv};
+    const uint64_t str[3] = {(uint64_t)n * 2, 128ull, (uint64_t)m * n * 2};
+    const uint32_t box[4] = {64u, 64u, (uint32_t)(p.NW / 64), 1u};
+    if (!encode_tensor_map_bf16(&tmTh, a.theta, 4, dims, str, box)) return cudaSuccess;
+  }
+  {
+    const uint64_t dims[3] = {(uint64_t)n, (uint64_t)m, (uint64_t)H_kv};
+    const uint64_t str[2] = {(uint64_t)n * 2, (uint64_t)m * n * 2};
+    const uint32_t box[3] = {64u, (uint32_t)p.brow, 1u};
+    if (!encode_tensor_map_bf16(&tmU, a.U, 3, dims, str, box)) return cudaSuccess;
+  }
+  {
+    const uint64_t dims[5] = {(uint64_t)D, (uint64_t)m, (uint64_t)R, (uint64_t)H_kv, (uint64_t)B};
+    const uint64_t str[4] = {256ull, (uint64_t)m * 256, (uint64_t)R * m * 256, (uint64_t)H_kv * R * m * 256};
+    const uint32_t box[5] = {64u, (uint32_t)SP_OUT_ROWS, 1u, 1u, 1u};
+    if (!encode_tensor_map_bf16(&tmO[0], a.Vc, 5, dims, str, box)) return cudaSuccess;
+  }
+  if (a.T > 0) {
+    const uint64_t dims[4] = {(uint64_t)D, (uint64_t)a.T, (uint64_t)H_kv, (uint64_t)B};
+    const uint64_t str[3] = {256ull, (uint64_t)a.T_cap * 256, (uint64_t)H_kv * a.T_cap * 256};
+    const uint32_t box[4] = {64u, (uint32_t)SP_OUT_ROWS, 1u, 1u};
+    if (!encode_tensor_map_bf16(&tmO[1], a.K_txt, 4, dims, str, box)) return cudaSuccess;
+    if (!encode_tensor_map_bf16(&tmO[2], a.V_txt, 4, dims, str, box)) return cudaSuccess;
+  } else {
+    tmO[1] = tmO[0];
+    tmO[2] = tmO[0];
+  }
+  {
+    // partial weights as (m columns, expansion rows, ranges, H_kv): a box = 64 columns of the G rows of a block, all ranges
+    const uint64_t dims[4] = {(uint64_t)m, (uint64_t)p.rows_h, (uint64_t)p.NS, (uint64_t)H_kv};
+    const uint64_t str[3] = {(uint64_t)p.ms * 2, (uint64_t)p.rows_h * p.ms * 2, (uint64_t)p.NS * p.rows_h * p.ms * 2};
+    const uint32_t box[4] = {64u, (uint32_t)G, (uint32_t)p.NS, 1u};
+    if (!encode_tensor_map_bf16(&tmO[3], ws + w.off_Wp, 4, dims, str, box, false)) return cudaSuccess;
+  }
+  *encoded = true;
+
+  SplitArgs sa{};
+  sa.q = static_cast<const __nv_bfloat16*>(a.q);
+  sa.mu = static_cast<const __nv_bfloat16*>(a.mu);
+  sa.out = static_cast<__nv_bfloat16*>(a.out);
+  sa.S = reinterpret_cast<__nv_bfloat16*>(ws + w.off_S);
+  sa.Wp = reinterpret_cast<__nv_bfloat16*>(ws + w.off_Wp);
+  sa.stat = reinterpret_cast<float2*>(ws + w.off_stat);
+  sa.py = reinterpret_cast<float*>(ws + w.off_py);
+  sa.pml = reinterpret_cast<float2*>(ws + w.off_pml);
+  sa.cnt = reinterpret_cast<int*>(ws + w.off_cnt);
+  sa.status = a.status;
+  sa.B = B; sa.H_kv = H_kv; sa.G = G; sa.R = R; sa.m = m; sa.n = n; sa.T = a.T;
+  sa.rows_h = p.rows_h; sa.ntile = p.ntile; sa.NS = p.NS; sa.NW = p.NW; sa.ms = p.ms; sa.nk1 = p.nk1;
+  sa.npass = p.npass; sa.prow = p.prow; sa.nbox = p.nbox; sa.brow = p.brow; sa.tmem_cols = p.tmem_cols;
+  sa.e_stages = p.e_stages; sa.e_stage_bytes = p.e_stage_bytes;
+  sa.s_tiles_bh = p.s_tiles_bh; sa.s_stages = p.s_stages;
+  sa.vt = p.vt; sa.o_stages = p.o_stages; sa.o_stage_bytes = p.o_stage_bytes;
+  sa.nslot_v = p.nslot_v; sa.nslot_t = p.nslot_t;
+  sa.o_off_q = p.o_off_q; sa.o_off_fac = p.o_off_fac; sa.o_off_red = p.o_off_red; sa.o_off_stat = p.o_off_stat;
+
+  cudaError_t e = launch_split_scores(tmK, sa, p, st);
+  if (e == cudaSuccess) e = launch_split_expand(tmS, tmTh, tmU, sa, p, st);
+  if (e == cudaSuccess) e = launch_split_output(tmO, sa, p, st);
+  return e;
+}
+
+}  // namespace kvc

@@ -69,7 +69,11 @@ split_expand_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_consta
         unsigned char* dst = ring + slot * a.e_stage_bytes;
         mbar_expect_tx(&bars.full[slot], 16384u + th_bytes);
         tma_load_4d(dst + 16384, &tmTh, 0, kc * 64, n0 >> 6, h, &bars.full[slot]);   // parameters: never written by the library
-        if (!waited) { grid_dep_wait(); waited = true; }                             // the scores come from the kernel before
+        if (!waited) {
+          grid_dep_wait();                    // the scores come from the kernel before
+          grid_dep_launch();                  // only now: the output kernel relies on that kernel being complete
+          waited = true;
+        }
         tma_load_3d(dst, &tmS, kc * 64, tile * SP_TILE_ROWS, h, &bars.full[slot]);
         if (++slot == (uint32_t)a.e_stages) { slot = 0; phase ^= 1u; }
       }
@@ -86,7 +90,6 @@ split_expand_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_consta
     }
   } else if (warp == 4) {
     // ---------------- MMA issue ----------------
-    grid_dep_launch();
     const uint32_t sm_u = smem_addr(sm), ring_u = sm_u + p_bytes;
     const uint32_t idesc_L = umma_idesc_bf16(128, a.NW, 0, 1);
     const uint32_t idesc_W = umma_idesc_bf16(128, a.brow, 0, 0);
@@ -158,7 +161,7 @@ split_expand_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_consta
     }
     // pass 2: probabilities relative to it, as the K-major A operand of the second product
     float sum = 0.f;
-    unsigned char* prow = sm + (uint32_t)row * 128u;
+    unsigned char* p_row = sm + (uint32_t)row * 128u;
     for (int c0 = 0; c0 < a.NW; c0 += 16) {
       float v[16];
       tmem_ld_x16(trow + (uint32_t)c0, v);
@@ -170,7 +173,7 @@ split_expand_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_consta
         w[k] = pack2_bf16(p0, p1);
       }
       const int grp = c0 >> 6, piece = (c0 & 63) >> 3;        // two 16-byte pieces: piece, piece + 1
-      unsigned char* g = prow + (uint32_t)grp * 16384u;
+      unsigned char* g = p_row + (uint32_t)grp * 16384u;
       *reinterpret_cast<uint4*>(g + (((piece) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
       *reinterpret_cast<uint4*>(g + (((piece + 1) ^ (row & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
     }

@@ -44,8 +44,13 @@ split_output_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
   const int tt = (a.T + SP_OUT_ROWS - 1) / SP_OUT_ROWS;          // text tiles per (sequence, KV head)
   const int vb = R * vt;                                          // value tiles per (sequence, KV head)
   const long long tot_t = BH * tt, tot_v = BH * vb;
-  const long long tlo = run_begin(blockIdx.x, tot_t, gridDim.x), thi = run_begin(blockIdx.x + 1, tot_t, gridDim.x);
-  const long long vlo = run_begin(blockIdx.x, tot_v, gridDim.x), vhi = run_begin(blockIdx.x + 1, tot_v, gridDim.x);
+  // each list is dealt to the first min(grid, items) CTAs, so that every CTA that takes part owns at least one item and
+  // the runs that hold tiles of one pair belong to consecutive CTAs
+  const long long gt = tot_t < (long long)gridDim.x ? tot_t : (long long)gridDim.x;
+  const long long gv = tot_v < (long long)gridDim.x ? tot_v : (long long)gridDim.x;
+  const bool in_t = (long long)blockIdx.x < gt, in_v = (long long)blockIdx.x < gv;
+  const long long tlo = in_t ? run_begin(blockIdx.x, tot_t, gt) : 0, thi = in_t ? run_begin(blockIdx.x + 1, tot_t, gt) : 0;
+  const long long vlo = in_v ? run_begin(blockIdx.x, tot_v, gv) : 0, vhi = in_v ? run_begin(blockIdx.x + 1, tot_v, gv) : 0;
   const uint32_t w_bytes = (uint32_t)(NS * G) * 128u;
 
   if (warp == SO_WARPS) {
@@ -153,10 +158,10 @@ split_output_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     __threadfence();
     named_barrier_sync(1, SO_CONS);
     // how many runs hold tiles of this pair: those of the CTAs that own its first and last tile, per kind
-    const int cv0 = vb > 0 ? run_owner((long long)bh * vb, tot_v, gridDim.x) : 0;
-    const int nsv = vb > 0 ? run_owner((long long)(bh + 1) * vb - 1, tot_v, gridDim.x) - cv0 + 1 : 0;
-    const int ct0 = tt > 0 ? run_owner((long long)bh * tt, tot_t, gridDim.x) : 0;
-    const int nst = tt > 0 ? run_owner((long long)(bh + 1) * tt - 1, tot_t, gridDim.x) - ct0 + 1 : 0;
+    const int cv0 = vb > 0 ? run_owner((long long)bh * vb, tot_v, gv) : 0;
+    const int nsv = vb > 0 ? run_owner((long long)(bh + 1) * vb - 1, tot_v, gv) - cv0 + 1 : 0;
+    const int ct0 = tt > 0 ? run_owner((long long)bh * tt, tot_t, gt) : 0;
+    const int nst = tt > 0 ? run_owner((long long)(bh + 1) * tt - 1, tot_t, gt) - ct0 + 1 : 0;
     if (tid == 0) s_last = atomicAdd(&a.cnt[bh], 1) + 1 == nsv + nst ? 1 : 0;
     named_barrier_sync(1, SO_CONS);
     if (s_last) {
@@ -227,7 +232,7 @@ split_output_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         hsum[tid] = l;
       }
       named_barrier_sync(1, SO_CONS);
-      const int ct0 = run_owner((long long)bh * tt, tot_t, gridDim.x);
+      const int ct0 = run_owner((long long)bh * tt, tot_t, gt);
       flush(bh, a.nslot_v + (int)blockIdx.x - ct0, false);
     };
 
@@ -353,7 +358,7 @@ split_output_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
       // probability mass of the vision positions (and with it the mu term), the others none
       if (!has_first && tid < 16) hsum[tid] = 0.f;
       named_barrier_sync(1, SO_CONS);
-      const int cv0 = run_owner((long long)bh * vb, tot_v, gridDim.x);
+      const int cv0 = run_owner((long long)bh * vb, tot_v, gv);
       flush(bh, (int)blockIdx.x - cv0, has_first);
     };
     for (long long i = vlo; i < vhi; ++i) {

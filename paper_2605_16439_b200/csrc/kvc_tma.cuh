@@ -75,7 +75,8 @@ __device__ __forceinline__ float fast_exp2(float x) {
 }
 
 // ---- host: encode a tiled bf16 tensor map (returns false if the driver entry point is missing or refuses)
+// swizzle128 == false: rows of the box land one after the other, unswizzled
 bool encode_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
-                            const uint64_t* strides_bytes, const uint32_t* box);
+                            const uint64_t* strides_bytes, const uint32_t* box, bool swizzle128 = true);
 
 }  // namespace kvc

@@ -79,12 +79,13 @@ def test_reduced_7b_shapes_bf16(ci, kw):
     _check(shape, p)
 
 
-@pytest.mark.parametrize("variant", ["mma", "tcgen05", "pair", "phases"])
+@pytest.mark.parametrize("variant", ["mma", "tcgen05", "pair", "split", "phases"])
 @pytest.mark.parametrize("recipe", ["peaked", "structured"])
 @pytest.mark.parametrize("ci,kw", tl.REDUCED_7B)
 def test_sharp_recipes_through_every_kernel_variant(ci, kw, recipe, variant, monkeypatch):
     """Peaked softmaxes and O(1) outputs on the block lengths of the 7B-shaped configurations, through the mma.sync
-    kernel, the tensor-memory kernel, its pair mode and the three-phase kernels: the inputs on which the mutations of
+    kernel, the tensor-memory kernel, its pair mode, the three-kernel bf16 path and the generic three-phase kernels: the
+    inputs on which the mutations of
     tests/test_sensitivity_cpu.py move the result by 14 to 280 times the bound asserted here."""
     monkeypatch.setenv("KVC_EXPANSION", variant)
     shape = tl.small(wl.CONFIGS[ci], **kw)
@@ -92,6 +93,8 @@ def test_sharp_recipes_through_every_kernel_variant(ci, kw, recipe, variant, mon
     counts = _fused_launches(lambda: _check(shape, p))
     if variant == "phases":
         assert counts["scores"] == 1 and counts["fused"] + counts["fused_tc"] + counts["fused_pair"] == 0
+    elif variant == "split":
+        assert counts["split_scores"] == counts["split_expand"] == counts["split_output"] == 1 and counts["fused"] == 0
     else:
         assert counts["fused"] + counts["fused_tc"] + counts["fused_pair"] == 1
 
@@ -418,7 +421,7 @@ def _random_shapes(count, seed):
     return out
 
 
-@pytest.mark.parametrize("variant", ["mma", "tcgen05", "pair"])
+@pytest.mark.parametrize("variant", ["mma", "tcgen05", "pair", "split"])
 def test_random_shapes_through_every_variant_of_the_one_kernel_path(variant, monkeypatch):
     """The same seeded random shapes through the mma.sync kernel, the tensor-memory kernel and its pair mode (a shape
     a variant does not serve falls to the next one: the result must be right whichever kernel ran)."""
