@@ -62,26 +62,26 @@ SplitPlan plan_split(const kvc_layer* L, int B, int R) {
   p.o_stage_bytes = 32768u;
   if (16384u + p.o_w_bytes > p.o_stage_bytes) return p;
   {
-    const int NH = G > 8 ? 2 : 1;
-    uint32_t off = 0;
-    auto take = [&](uint32_t bytes) { uint32_t o = off; off = (off + bytes + 127u) & ~127u; return o; };
-    p.o_off_q = take(16 * 136 * 2);
-    p.o_off_fac = take((uint32_t)(R * p.NS) * 16u * 8u);
-    p.o_off_red = take(8u * NH * 8u * 64u * 4u);
-    p.o_off_stat = take((2 * 8 * 16 + 32) * 4);
-    p.o_stages = (int)((SP_SMEM_LIMIT - 2048u - off) / p.o_stage_bytes);
-    if (p.o_stages > SP_MAX_STAGES) p.o_stages = SP_MAX_STAGES;
-    if (p.o_stages < 2) return p;
-    const uint32_t ring = (uint32_t)p.o_stages * p.o_stage_bytes;
-    p.o_off_q += ring; p.o_off_fac += ring; p.o_off_red += ring; p.o_off_stat += ring;
-    p.o_smem = (size_t)ring + off + 1024;
-  }
-  {
     const long long items = (long long)B * H_kv * R * p.vt;
     p.o_grid = (int)(items < sms ? items : sms);
     const long long bh = (long long)B * H_kv;
     p.nslot_v = (int)((p.o_grid + bh - 1) / bh) + 1;
     p.nslot_t = p.nslot_v;
+  }
+  {
+    const int NH = G > 8 ? 2 : 1;
+    uint32_t off = 0;
+    auto take = [&](uint32_t bytes) { uint32_t o = off; off = (off + bytes + 127u) & ~127u; return o; };
+    p.o_off_q = 0;
+    p.o_off_fac = take((uint32_t)(R * p.NS) * 16u * 8u);
+    p.o_off_red = take(8u * NH * 8u * (uint32_t)D * 4u);
+    p.o_off_stat = take((uint32_t)(2 * 8 * 16 + 32 + 2 * (p.nslot_v + p.nslot_t) * 16) * 4u);
+    if (off + 2048u + 2 * p.o_stage_bytes > SP_SMEM_LIMIT) return p;
+    p.o_stages = (int)((SP_SMEM_LIMIT - 2048u - off) / p.o_stage_bytes);
+    if (p.o_stages > SP_MAX_STAGES) p.o_stages = SP_MAX_STAGES;
+    const uint32_t ring = (uint32_t)p.o_stages * p.o_stage_bytes;
+    p.o_off_fac += ring; p.o_off_red += ring; p.o_off_stat += ring;
+    p.o_smem = (size_t)ring + off + 1024;
   }
   p.ok = 1;
   return p;

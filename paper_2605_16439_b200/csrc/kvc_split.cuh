@@ -76,6 +76,23 @@ struct SplitArgs {
 // sigma = 1/sqrt(128), logits kept in log2 units
 constexpr float SP_QSCALE = 0.08838834764831845f * 1.4426950408889634f;
 
+// Stage rings whose tiles go to groups of SP_GROUP warps (tile k of a CTA's list to group k mod 2, ring slot k mod stages):
+// a group may reach the full barrier of its slot before the slot's previous round has even been filled, and the barrier's
+// parity alone cannot tell round w from round w - 2.  So every slot carries a count of the warps that have released it
+// over all rounds; the consumers of round w first wait (bounded) until every warp of the rounds before has released,
+// which pins the barrier's current phase to round w.
+constexpr int SP_GROUP = 4;            // warps that share a tile
+__device__ __forceinline__ bool wait_round(const volatile uint32_t* released, uint32_t slot, uint32_t round) {
+  for (uint32_t i = 0; i < (1u << 24); ++i)
+    if (released[slot] >= round * SP_GROUP) return true;
+  return false;
+}
+__device__ __forceinline__ void release_slot(uint32_t* released, uint64_t* empty_bar, uint32_t slot) {
+  atomicAdd(&released[slot], 1u);
+  __threadfence_block();
+  mbar_arrive(&empty_bar[slot]);
+}
+
 // Item i of `tot` items dealt in contiguous runs to `grid` CTAs: CTA c owns [c tot / grid, (c+1) tot / grid).
 __host__ __device__ __forceinline__ long long run_begin(long long c, long long tot, long long grid) { return c * tot / grid; }
 // the CTA that owns item i

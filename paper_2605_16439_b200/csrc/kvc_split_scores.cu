@@ -2,9 +2,11 @@
 //   S[h][(b R + r) G + g][j] = sigma log2(e) q[b, hG + g, :] . K_tilde[b, h, r, j, :]      (bf16, fp32 accumulation)
 // One streaming pass over K_tilde, bound by HBM bandwidth.  The R m key rows of a (sequence, KV head) are contiguous in
 // the capsule store; they are cut into tiles of 128 rows and the flat tile list is dealt in contiguous runs to one
-// persistent CTA per SM.  A producer thread keeps a ring of TMA-filled 32 KB stages full (128-byte swizzle); eight consumer
-// warps take 16 rows each: the queries of the KV head (up to 16, zero-padded) are the A operand held in registers, the key
-// rows the B operand read with ldmatrix, so a lane ends up with two consecutive rows of one head and stores them as bf16.
+// persistent CTA per SM.  A producer thread keeps a ring of TMA-filled 32 KB stages full (128-byte swizzle).  The eight
+// consumer warps form two groups of four; tile k of the CTA's run goes to group k mod 2 and each warp of the group takes
+// 32 of its rows (a stage is held only for that short time, and two tiles are in work at once): the queries of the KV
+// head (up to 16, zero-padded) are the A operand held in registers, the key rows the B operand read with ldmatrix, and a
+// lane ends up with two consecutive key rows of one head.
 #include "kvc_split.cuh"
 
 namespace kvc {
@@ -19,9 +21,10 @@ split_scores_kernel(const __grid_constant__ CUtensorMap tmK, const SplitArgs a) 
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* sm = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
   __shared__ __align__(8) uint64_t full_bar[SP_MAX_STAGES], empty_bar[SP_MAX_STAGES];
+  __shared__ uint32_t released[SP_MAX_STAGES];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
-    for (int s = 0; s < a.s_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], SS_WARPS); }
+    for (int s = 0; s < a.s_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], SP_GROUP); released[s] = 0u; }
     fence_mbar_init();
   }
   __syncthreads();
@@ -29,6 +32,7 @@ split_scores_kernel(const __grid_constant__ CUtensorMap tmK, const SplitArgs a) 
   const long long BH = (long long)a.B * a.H_kv;
   const long long total = BH * a.s_tiles_bh;
   const long long lo = run_begin(blockIdx.x, total, gridDim.x), hi = run_begin(blockIdx.x + 1, total, gridDim.x);
+  const int nst = a.s_stages;
 
   if (warp == SS_WARPS) {
     if (lane != 0) return;
@@ -42,25 +46,27 @@ split_scores_kernel(const __grid_constant__ CUtensorMap tmK, const SplitArgs a) 
       mbar_expect_tx(&full_bar[slot], SS_STAGE);
       tma_load_3d(dst, &tmK, 0, t * SP_TILE_ROWS, bh, &full_bar[slot]);
       tma_load_3d(dst + SS_HALF, &tmK, 64, t * SP_TILE_ROWS, bh, &full_bar[slot]);
-      if (++slot == (uint32_t)a.s_stages) { slot = 0; phase ^= 1u; }
+      if (++slot == (uint32_t)nst) { slot = 0; phase ^= 1u; }
     }
     return;
   }
 
   grid_dep_wait();
   grid_dep_launch();
-  // per-call device state of the path: status word, arrival counters of the output kernel's segments
+  // per-call device state of the path: status word, arrival counters of the output kernel's runs
   if (blockIdx.x == 0 && tid == 0) *a.status = 0;
   for (long long i = (long long)blockIdx.x * (SS_WARPS * 32) + tid; i < BH; i += (long long)gridDim.x * (SS_WARPS * 32)) a.cnt[i] = 0;
 
   const int gid = lane >> 2, t4 = lane & 3;
   const int G = a.G, m = a.m, Rm = a.R * a.m;
   const uint32_t sm_u = smem_addr(sm);
-  uint32_t slot = 0, phase = 0;
   bool dead = false;
   int cur_bh = -1;
   uint32_t qa[8][4];
-  for (long long i = lo; i < hi; ++i) {
+  const int grp = warp / SP_GROUP, wj = warp % SP_GROUP;
+  for (long long k = grp; lo + k < hi; k += SS_WARPS / SP_GROUP) {
+    const long long i = lo + k;
+    const uint32_t slot = (uint32_t)(k % nst), round = (uint32_t)(k / nst), phase = round & 1u;
     const int bh = (int)(i / a.s_tiles_bh), t = (int)(i - (long long)bh * a.s_tiles_bh);
     const int b = bh / a.H_kv, h = bh - b * a.H_kv;
     if (bh != cur_bh) {
@@ -76,42 +82,61 @@ split_scores_kernel(const __grid_constant__ CUtensorMap tmK, const SplitArgs a) 
         qa[ks][3] = gid + 8 < G ? *reinterpret_cast<const uint32_t*>(q0 + (size_t)(gid + 8) * D + k0 + 8) : 0u;
       }
     }
-    if (!dead && !mbar_wait_bounded(&full_bar[slot], phase)) dead = true;
+    if (!dead && !(wait_round(released, slot, round) && mbar_wait_bounded(&full_bar[slot], phase))) dead = true;
     __syncwarp();
     const uint32_t st_u = sm_u + slot * SS_STAGE;
-    float acc[2][4];
+    // (block, row in block) of the tile's first key row; the rows of a lane follow by small steps
+    const int g0 = t * SP_TILE_ROWS;
+    const int r_t = g0 / m, j_t = g0 - r_t * m;
+    __nv_bfloat16* S_h = a.S + (size_t)h * a.rows_h * a.ms;
+    const int bR = b * a.R;
 #pragma unroll
-    for (int nt = 0; nt < 2; ++nt) {
+    for (int np = 2 * wj; np < 2 * wj + 2; ++np) { // 16 rows per step as two 8-row groups: independent accumulation chains
+      float acc[2][4];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
-      const int row = warp * 16 + nt * 8 + (lane & 7);
+      for (int nt = 0; nt < 2; ++nt) {
 #pragma unroll
-      for (int x = 0; x < 4; ++x) {
-        // four 8 x 8 matrices: the 16-byte pieces 4x .. 4x+3 of rows row0 .. row0+7 (pieces 0-7 in the first half)
-        const int c = 4 * x + (lane >> 3);
-        uint32_t bf[4];
-        ldsm_x4(bf, st_u + (uint32_t)(c >> 3) * SS_HALF + (uint32_t)row * 128u + (uint32_t)((((c & 7) ^ (row & 7))) << 4));
-        mma_bf16_16816(acc[nt], qa[2 * x], bf[0], bf[1]);
-        mma_bf16_16816(acc[nt], qa[2 * x + 1], bf[2], bf[3]);
+        for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
+        const int row = np * 16 + nt * 8 + (lane & 7);
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+          // four 8 x 8 matrices: the 16-byte pieces 4x .. 4x+3 of rows row0 .. row0+7 (pieces 0-7 in the first half)
+          const int c = 4 * x + (lane >> 3);
+          uint32_t bf[4];
+          ldsm_x4(bf, st_u + (uint32_t)(c >> 3) * SS_HALF + (uint32_t)row * 128u + (uint32_t)((((c & 7) ^ (row & 7))) << 4));
+          mma_bf16_16816(acc[nt], qa[2 * x], bf[0], bf[1]);
+          mma_bf16_16816(acc[nt], qa[2 * x + 1], bf[2], bf[3]);
+        }
+      }
+      if (dead) continue;
+      // acc[nt][e]: head gid + 8 (e >> 1), key row g0 + np*16 + nt*8 + 2 t4 + (e & 1) of the (sequence, KV head)
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) {
+        const int off = np * 16 + nt * 8 + 2 * t4;
+        if (g0 + off >= Rm) continue;
+        int r = r_t, j = j_t + off;
+        if (m >= SP_TILE_ROWS) { if (j >= m) { j -= m; ++r; } }
+        else { const int dr = j / m; r += dr; j -= dr * m; }
+        int r1 = r, j1 = j + 1;
+        if (j1 == m) { j1 = 0; ++r1; }
+        const bool second = g0 + off + 1 < Rm;
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+          const int head = gid + 8 * hh;
+          if (head >= G) continue;
+          const float v0 = acc[nt][2 * hh] * SP_QSCALE, v1 = acc[nt][2 * hh + 1] * SP_QSCALE;
+          __nv_bfloat16* p0 = S_h + ((size_t)(bR + r) * G + head) * a.ms + j;
+          if (second && r1 == r && (j & 1) == 0) {
+            *reinterpret_cast<uint32_t*>(p0) = pack2_bf16(v0, v1);
+          } else {
+            *p0 = __float2bfloat16_rn(v0);
+            if (second) S_h[((size_t)(bR + r1) * G + head) * a.ms + j1] = __float2bfloat16_rn(v1);
+          }
+        }
       }
     }
     __syncwarp();
-    if (lane == 0) mbar_arrive(&empty_bar[slot]);
-    if (++slot == (uint32_t)a.s_stages) { slot = 0; phase ^= 1u; }
-    if (dead) continue;
-    // acc[nt][e]: head gid + 8 (e >> 1), key row t*128 + warp*16 + nt*8 + 2 t4 + (e & 1) of the (sequence, KV head)
-#pragma unroll
-    for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int head = gid + 8 * (e >> 1);
-        const int gr = t * SP_TILE_ROWS + warp * 16 + nt * 8 + 2 * t4 + (e & 1);
-        if (head < G && gr < Rm) {
-          const int r = gr / m, j = gr - r * m;
-          const size_t rho = (size_t)(b * a.R + r) * G + head;
-          a.S[((size_t)h * a.rows_h + rho) * a.ms + j] = __float2bfloat16_rn(acc[nt][e] * SP_QSCALE);
-        }
-      }
+    if (lane == 0) release_slot(released, empty_bar, slot);
   }
   if (dead && lane == 0) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
 }
