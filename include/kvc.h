@@ -81,11 +81,12 @@ KVC_API int kvc_retained_len(int n, int ratio_permille);
  * unchanged while the handle is in use.  ratio_permille == 0 is the pass-through limit: m = n,
  * capsules hold K and V verbatim, idx / theta / U / mu are ignored.
  * The device that is current at this call must be current for every later call with the handle.
- * bf16 decode calls run Alg. 1 steps 2-3 either on mma.sync with the logits in registers or on tcgen05 with the
- * logits in tensor memory; the library picks per shape (same results within the bf16 tolerance).  The environment
- * variable KVC_EXPANSION = "tcgen05" | "mma", read when the handle is created, forces one of them where it applies;
- * "pair" the tcgen05 path run by clusters of two CTAs per (sequence, KV head); "phases" the three-kernel path
- * (scores, expansion, output) that also serves fp32 storage. */
+ * bf16 decode calls run Alg. 1 either as one kernel (steps 2-3 on mma.sync with the logits in registers, or on tcgen05
+ * with the logits in tensor memory) or, for block lengths above 640, as three kernels (streaming scores, tcgen05
+ * expansion per 128 rows and range of the n axis, streaming output); the library picks per shape (same results within
+ * the bf16 tolerance).  The environment variable KVC_EXPANSION = "tcgen05" | "mma" | "pair" | "split", read when the
+ * handle is created, forces one of them where it applies ("pair": the tcgen05 one-kernel path run by clusters of two
+ * CTAs per (sequence, KV head)); "phases" forces the generic three-phase kernels that also serve fp32 storage. */
 KVC_API int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out);
 KVC_API int kvc_layer_destroy(kvc_layer* layer);
 

@@ -258,9 +258,13 @@ int kvc_compress(const kvc_layer* L, const void* K_vis, const void* V_vis, int B
 }  // extern "C"
 
 namespace kvc {
-// Which bf16 shapes take the three-kernel path (the others take the one-kernel path): forced by KVC_EXPANSION=split.
+// Which bf16 shapes take the three-kernel path (the others take the one-kernel path).  Measured on B200 over batch 1-64,
+// 2-32 blocks and ratios 0.2-0.8 at n = 1024, G = 7: ahead of the one-kernel variants at 31 of 33 points (by 1.0-2.1 x;
+// behind by at most 12 % at ratio 0.8 with few rows); behind them for short blocks (n = 256: 35 vs 21 us, n = 576: 74 vs
+// 41 us at the 7B shapes), where the logits of a unit fit the registers of the one-kernel path.
+// KVC_EXPANSION=split forces it where its plan applies, any other value of the variable keeps it off.
 static bool use_split(const kvc_layer* L, int B, int R) {
-  if (L->use_tc != 3) return false;
+  if (L->use_tc != 3 && !(L->use_tc == 0 && L->desc.n > 640)) return false;
   return plan_split(L, B, R).ok != 0;
 }
 

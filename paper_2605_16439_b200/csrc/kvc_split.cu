@@ -4,8 +4,8 @@
 namespace kvc {
 
 cudaError_t launch_split_scores(const CUtensorMap& tmK, const SplitArgs& a, const SplitPlan& p, cudaStream_t st);
-cudaError_t launch_split_expand(const CUtensorMap& tmS, const CUtensorMap& tmTh, const CUtensorMap& tmU, const SplitArgs& a,
-                                const SplitPlan& p, cudaStream_t st);
+cudaError_t launch_split_expand(const CUtensorMap& tmS, const CUtensorMap& tmTh, const CUtensorMap& tmU, const CUtensorMap& tmWs,
+                                const SplitArgs& a, const SplitPlan& p, cudaStream_t st);
 cudaError_t launch_split_output(const CUtensorMap* tm, const SplitArgs& a, const SplitPlan& p, cudaStream_t st);
 
 constexpr uint32_t SP_SMEM_LIMIT = 232448;      // 227 KB per CTA on sm_100
@@ -34,7 +34,8 @@ SplitPlan plan_split(const kvc_layer* L, int B, int R) {
   // passes over the weights: at most 512 tensor-memory columns each, cut into one or two boxes of rows of U
   const int mpad = (m + 15) & ~15;
   p.npass = ceil_div(mpad, 512);
-  p.prow = (ceil_div(mpad, p.npass) + 31) & ~31;
+  // one pass: whole 32-column steps; several: whole 64-column tiles, so that no pass stores into the next one's columns
+  p.prow = p.npass == 1 ? ((mpad + 31) & ~31) : ((ceil_div(mpad, p.npass) + 63) & ~63);
   p.nbox = p.prow > 256 ? 2 : 1;
   p.brow = p.prow / p.nbox;
   int cols = p.prow > p.NW ? p.prow : p.NW;
@@ -62,25 +63,28 @@ SplitPlan plan_split(const kvc_layer* L, int B, int R) {
   p.o_stage_bytes = 32768u;
   if (16384u + p.o_w_bytes > p.o_stage_bytes) return p;
   {
-    const long long items = (long long)B * H_kv * R * p.vt;
-    p.o_grid = (int)(items < sms ? items : sms);
+    // CTAs per (sequence, KV head): as many as the SMs allow (the same for every pair), at most one per value tile
     const long long bh = (long long)B * H_kv;
-    p.nslot_v = (int)((p.o_grid + bh - 1) / bh) + 1;
-    p.nslot_t = p.nslot_v;
+    const long long vb = (long long)R * p.vt;
+    long long cpb = sms / bh;
+    if (cpb < 1) cpb = 1;
+    if (cpb > vb) cpb = vb;
+    p.o_cpb = (int)cpb;
+    p.o_grid = (int)(cpb > 1 ? bh * cpb : (bh < sms ? bh : sms));
   }
   {
     const int NH = G > 8 ? 2 : 1;
     uint32_t off = 0;
     auto take = [&](uint32_t bytes) { uint32_t o = off; off = (off + bytes + 127u) & ~127u; return o; };
-    p.o_off_q = 0;
+    p.o_off_q = take(16u * (uint32_t)D * 4u);                       // text part of a pair
     p.o_off_fac = take((uint32_t)(R * p.NS) * 16u * 8u);
     p.o_off_red = take(8u * NH * 8u * (uint32_t)D * 4u);
-    p.o_off_stat = take((uint32_t)(2 * 8 * 16 + 32 + 2 * (p.nslot_v + p.nslot_t) * 16) * 4u);
+    p.o_off_stat = take((uint32_t)(2 * 8 * 16 + 64 + 2 * p.o_cpb * 16) * 4u);
     if (off + 2048u + 2 * p.o_stage_bytes > SP_SMEM_LIMIT) return p;
     p.o_stages = (int)((SP_SMEM_LIMIT - 2048u - off) / p.o_stage_bytes);
     if (p.o_stages > SP_MAX_STAGES) p.o_stages = SP_MAX_STAGES;
     const uint32_t ring = (uint32_t)p.o_stages * p.o_stage_bytes;
-    p.o_off_fac += ring; p.o_off_red += ring; p.o_off_stat += ring;
+    p.o_off_q += ring; p.o_off_fac += ring; p.o_off_red += ring; p.o_off_stat += ring;
     p.o_smem = (size_t)ring + off + 1024;
   }
   p.ok = 1;
@@ -96,7 +100,7 @@ SplitWs split_ws(const kvc_layer* L, const SplitPlan& p, int B, int R) {
   w.off_S = take(sizeof(__nv_bfloat16) * (size_t)H_kv * p.rows_h * p.ms);
   w.off_Wp = take(sizeof(__nv_bfloat16) * (size_t)H_kv * p.NS * p.rows_h * p.ms);
   w.off_stat = take(sizeof(float2) * (size_t)H_kv * p.NS * p.rows_h);
-  const size_t nslot = (size_t)p.nslot_v + p.nslot_t;
+  const size_t nslot = p.o_cpb > 1 ? (size_t)p.o_cpb : 0;
   w.off_py = take(sizeof(float) * (size_t)B * H_kv * nslot * G * D);
   w.off_pml = take(sizeof(float2) * (size_t)B * H_kv * nslot * G);
   w.off_cnt = take(sizeof(int) * (size_t)B * H_kv);
@@ -109,7 +113,7 @@ cudaError_t launch_split(const kvc_layer* L, const DecodeArgs& a, const SplitPla
   *encoded = false;
   char* ws = reinterpret_cast<char*>(a.split_base);
   const SplitWs w = split_ws(L, p, B, R);
-  CUtensorMap tmK, tmS, tmTh, tmU, tmO[4];
+  CUtensorMap tmK, tmS, tmTh, tmU, tmWs, tmO[4];
   {
     // K_tilde as (channels, R m rows of a pair, pairs): rows past the pair's last are zero-filled, not read
     const uint64_t dims[3] = {(uint64_t)D, (uint64_t)R * m, (uint64_t)B * H_kv};
@@ -158,6 +162,9 @@ cudaError_t launch_split(const kvc_layer* L, const DecodeArgs& a, const SplitPla
     const uint64_t str[3] = {(uint64_t)p.ms * 2, (uint64_t)p.rows_h * p.ms * 2, (uint64_t)p.NS * p.rows_h * p.ms * 2};
     const uint32_t box[4] = {64u, (uint32_t)G, (uint32_t)p.NS, 1u};
     if (!encode_tensor_map_bf16(&tmO[3], ws + w.off_Wp, 4, dims, str, box, false)) return cudaSuccess;
+    // the same tensor as the expansion kernel stores it: 64 columns of the 128 rows of a tile, swizzled rows
+    const uint32_t sbox[4] = {64u, (uint32_t)SP_TILE_ROWS, 1u, 1u};
+    if (!encode_tensor_map_bf16(&tmWs, ws + w.off_Wp, 4, dims, str, sbox)) return cudaSuccess;
   }
   *encoded = true;
 
@@ -178,11 +185,11 @@ cudaError_t launch_split(const kvc_layer* L, const DecodeArgs& a, const SplitPla
   sa.e_stages = p.e_stages; sa.e_stage_bytes = p.e_stage_bytes;
   sa.s_tiles_bh = p.s_tiles_bh; sa.s_stages = p.s_stages;
   sa.vt = p.vt; sa.o_stages = p.o_stages; sa.o_stage_bytes = p.o_stage_bytes;
-  sa.nslot_v = p.nslot_v; sa.nslot_t = p.nslot_t;
+  sa.o_cpb = p.o_cpb;
   sa.o_off_q = p.o_off_q; sa.o_off_fac = p.o_off_fac; sa.o_off_red = p.o_off_red; sa.o_off_stat = p.o_off_stat;
 
   cudaError_t e = launch_split_scores(tmK, sa, p, st);
-  if (e == cudaSuccess) e = launch_split_expand(tmS, tmTh, tmU, sa, p, st);
+  if (e == cudaSuccess) e = launch_split_expand(tmS, tmTh, tmU, tmWs, sa, p, st);
   if (e == cudaSuccess) e = launch_split_output(tmO, sa, p, st);
   return e;
 }

@@ -34,7 +34,7 @@ struct SplitPlan {
   int s_stages, s_grid; size_t s_smem;
   int vt;              // 64-row tiles per block of V_tilde
   int o_stages, o_grid; uint32_t o_stage_bytes, o_w_bytes; size_t o_smem;
-  int nslot_v, nslot_t;   // partial slots per (sequence, KV head): vision segments, text segments
+  int o_cpb;              // CTAs of the output kernel per (sequence, KV head) = its partial slots (1: no partials)
   uint32_t o_off_q, o_off_fac, o_off_red, o_off_stat;   // behind the ring
 };
 
@@ -43,8 +43,8 @@ struct SplitWs {
   size_t off_S;      // bf16 [H_kv][rows_h][ms]
   size_t off_Wp;     // bf16 [H_kv][NS][rows_h][ms]
   size_t off_stat;   // float2 [H_kv][NS][rows_h]  (row maximum in log2 units, row sum)
-  size_t off_py;     // fp32 [B*H_kv][nslot][G][D]
-  size_t off_pml;    // float2 [B*H_kv][nslot][G]
+  size_t off_py;     // fp32 [B*H_kv][o_cpb][G][D]
+  size_t off_pml;    // float2 [B*H_kv][o_cpb][G]
   size_t off_cnt;    // int [B*H_kv]  arrivals of the output kernel's segments, cleared by the score kernel
   size_t bytes;
 };
@@ -69,7 +69,7 @@ struct SplitArgs {
   int e_stages; uint32_t e_stage_bytes;
   int s_tiles_bh, s_stages;
   int vt, o_stages; uint32_t o_stage_bytes;
-  int nslot_v, nslot_t;
+  int o_cpb;
   uint32_t o_off_q, o_off_fac, o_off_red, o_off_stat;
 };
 

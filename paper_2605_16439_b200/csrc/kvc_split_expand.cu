@@ -25,7 +25,7 @@ struct ExpandBars {
 
 __global__ void __launch_bounds__(SE_THREADS, 1)
 split_expand_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUtensorMap tmTh,
-                    const __grid_constant__ CUtensorMap tmU, const SplitArgs a) {
+                    const __grid_constant__ CUtensorMap tmU, const __grid_constant__ CUtensorMap tmWs, const SplitArgs a) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* sm = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
   __shared__ __align__(8) ExpandBars bars;
@@ -151,55 +151,106 @@ split_expand_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_consta
     bool ok = mbar_wait_bounded(&bars.l_done, 0);
     __syncwarp();
     tc_fence_after();
-    // pass 1: row maximum over the range
+    // pass 1: row maximum over the range (32 columns per load, the next load in flight while one is reduced)
     float mx = -INFINITY;
-    for (int c0 = 0; c0 < a.NW; c0 += 16) {
-      float v[16];
-      tmem_ld_x16(trow + (uint32_t)c0, v);
+    {
+      uint32_t ra[32], rb[32];
+      tmem_ld_issue_x32(trow, ra);
+      for (int c0 = 0; c0 < a.NW; c0 += 64) {
+        tmem_ld_wait_x32(ra);
+        tmem_ld_issue_x32(trow + (uint32_t)(c0 + 32), rb);
 #pragma unroll
-      for (int k = 0; k < 16; ++k) mx = fmaxf(mx, v[k]);
+        for (int k = 0; k < 32; ++k) mx = fmaxf(mx, __uint_as_float(ra[k]));
+        tmem_ld_wait_x32(rb);
+        if (c0 + 64 < a.NW) tmem_ld_issue_x32(trow + (uint32_t)(c0 + 64), ra);
+#pragma unroll
+        for (int k = 0; k < 32; ++k) mx = fmaxf(mx, __uint_as_float(rb[k]));
+      }
     }
     // pass 2: probabilities relative to it, as the K-major A operand of the second product
     float sum = 0.f;
     unsigned char* p_row = sm + (uint32_t)row * 128u;
-    for (int c0 = 0; c0 < a.NW; c0 += 16) {
-      float v[16];
-      tmem_ld_x16(trow + (uint32_t)c0, v);
-      uint32_t w[8];
+    {
+      uint32_t ra[32];
+      auto emit = [&](int c0, const uint32_t (&r)[32]) {       // 32 columns -> four 16-byte pieces of the row
+        uint32_t w[16];
 #pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        const float p0 = fast_exp2(v[2 * k] - mx), p1 = fast_exp2(v[2 * k + 1] - mx);
-        sum += p0 + p1;
-        w[k] = pack2_bf16(p0, p1);
+        for (int k = 0; k < 16; ++k) {
+          const float p0 = fast_exp2(__uint_as_float(r[2 * k]) - mx), p1 = fast_exp2(__uint_as_float(r[2 * k + 1]) - mx);
+          sum += p0 + p1;
+          w[k] = pack2_bf16(p0, p1);
+        }
+        unsigned char* g = p_row + (uint32_t)(c0 >> 6) * 16384u;
+        const int piece = (c0 & 63) >> 3;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          *reinterpret_cast<uint4*>(g + (((piece + q) ^ (row & 7)) << 4)) = make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+      };
+      for (int c0 = 0; c0 < a.NW; c0 += 32) {
+        tmem_ld_issue_x32(trow + (uint32_t)c0, ra);
+        tmem_ld_wait_x32(ra);
+        emit(c0, ra);
       }
-      const int grp = c0 >> 6, piece = (c0 & 63) >> 3;        // two 16-byte pieces: piece, piece + 1
-      unsigned char* g = p_row + (uint32_t)grp * 16384u;
-      *reinterpret_cast<uint4*>(g + (((piece) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-      *reinterpret_cast<uint4*>(g + (((piece + 1) ^ (row & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
     }
     if (valid && ok) a.stat[((size_t)h * a.NS + s) * a.rows_h + rho] = make_float2(mx, sum);
     fence_proxy_async();                                       // P is read by the tensor core (async proxy)
     tc_fence_before();
     __syncwarp();
     if (lane == 0) mbar_arrive(&bars.p_ready);
-    // the weights of the range, pass by pass
+    // the weights of the range, pass by pass.  The last pass goes through the shared memory of P (dead by then): 64-column
+    // tiles in the swizzled row layout, stored by the TMA engine (rows and columns outside the tensor are clipped);
+    // earlier passes (retained lengths above 512) store from registers.
     __nv_bfloat16* wrow = a.Wp + (((size_t)h * a.NS + s) * a.rows_h + (valid ? rho : 0)) * a.ms;
+    const int ntile = a.NW >> 6;                                 // staging tiles of 16 KB in the region of P
     for (int wp = 0; wp < a.npass; ++wp) {
       if (ok && !mbar_wait_bounded(&bars.w_done, (uint32_t)(wp & 1))) ok = false;
       __syncwarp();
       tc_fence_after();
       const int j0 = wp * a.prow;
-      for (int c0 = 0; c0 < a.prow && j0 + c0 < a.ms; c0 += 16) {
-        float v[16];
-        tmem_ld_x16(trow + (uint32_t)c0, v);
-        if (valid && ok) {
+      if (wp == a.npass - 1) {
+        int cg = 0;
+        for (int c0 = 0; c0 < a.prow && j0 + c0 < a.m; c0 += 64, ++cg) {
+          unsigned char* tile_sm = sm + (uint32_t)(cg % ntile) * 16384u;
+          if (cg >= ntile) {                                     // the store that last read this tile has to be done with it
+            if (tid == 0) { if (ntile >= 4) bulk_wait_group_read<3>(); else if (ntile >= 2) bulk_wait_group_read<1>(); else bulk_wait_group_read<0>(); }
+            named_barrier_sync(2, 128);
+          }
+          const int ncol = min(64, a.prow - c0);
+          uint32_t ra[32];
+          for (int cc = 0; cc < ncol; cc += 32) {
+            tmem_ld_issue_x32(trow + (uint32_t)(c0 + cc), ra);
+            tmem_ld_wait_x32(ra);
+            unsigned char* g = tile_sm + (uint32_t)row * 128u;
+            const int piece = cc >> 3;
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            const int j = j0 + c0 + 8 * half;
-            if (j < a.ms)
-              *reinterpret_cast<uint4*>(wrow + j) =
-                  make_uint4(pack2_bf16(v[8 * half], v[8 * half + 1]), pack2_bf16(v[8 * half + 2], v[8 * half + 3]),
-                             pack2_bf16(v[8 * half + 4], v[8 * half + 5]), pack2_bf16(v[8 * half + 6], v[8 * half + 7]));
+            for (int q = 0; q < 4; ++q)
+              *reinterpret_cast<uint4*>(g + (((piece + q) ^ (row & 7)) << 4)) =
+                  make_uint4(pack2_bf16(__uint_as_float(ra[8 * q]), __uint_as_float(ra[8 * q + 1])),
+                             pack2_bf16(__uint_as_float(ra[8 * q + 2]), __uint_as_float(ra[8 * q + 3])),
+                             pack2_bf16(__uint_as_float(ra[8 * q + 4]), __uint_as_float(ra[8 * q + 5])),
+                             pack2_bf16(__uint_as_float(ra[8 * q + 6]), __uint_as_float(ra[8 * q + 7])));
+          }
+          fence_proxy_async();
+          named_barrier_sync(2, 128);
+          if (tid == 0 && ok) {
+            tma_store_4d(&tmWs, tile_sm, j0 + c0, tile * SP_TILE_ROWS, s, h);
+            bulk_commit_group();
+          }
+        }
+        if (tid == 0) bulk_wait_group_all();
+      } else {
+        for (int c0 = 0; c0 < a.prow && j0 + c0 < a.ms; c0 += 16) {
+          float v[16];
+          tmem_ld_x16(trow + (uint32_t)c0, v);
+          if (valid && ok) {
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              const int j = j0 + c0 + 8 * half;
+              if (j < a.ms)
+                *reinterpret_cast<uint4*>(wrow + j) =
+                    make_uint4(pack2_bf16(v[8 * half], v[8 * half + 1]), pack2_bf16(v[8 * half + 2], v[8 * half + 3]),
+                               pack2_bf16(v[8 * half + 4], v[8 * half + 5]), pack2_bf16(v[8 * half + 6], v[8 * half + 7]));
+            }
           }
         }
       }
@@ -214,12 +265,12 @@ split_expand_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_consta
   if (warp == 4) tmem_dealloc(tb, (uint32_t)a.tmem_cols);
 }
 
-cudaError_t launch_split_expand(const CUtensorMap& tmS, const CUtensorMap& tmTh, const CUtensorMap& tmU, const SplitArgs& a,
-                                const SplitPlan& p, cudaStream_t st) {
+cudaError_t launch_split_expand(const CUtensorMap& tmS, const CUtensorMap& tmTh, const CUtensorMap& tmU, const CUtensorMap& tmWs,
+                                const SplitArgs& a, const SplitPlan& p, cudaStream_t st) {
   cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(split_expand_kernel), p.e_smem);
   if (e != cudaSuccess) return e;
   ProfScope prof(KVC_KERNEL_SPLIT_EXPAND, st);
-  return launch_dependent(split_expand_kernel, dim3(p.e_grid), dim3(SE_THREADS), p.e_smem, st, tmS, tmTh, tmU, a);
+  return launch_dependent(split_expand_kernel, dim3(p.e_grid), dim3(SE_THREADS), p.e_smem, st, tmS, tmTh, tmU, tmWs, a);
 }
 
 }  // namespace kvc

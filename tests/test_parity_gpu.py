@@ -343,7 +343,8 @@ def test_pyramid_schedule_ratios_on_the_7b_block_lengths(ci, kw, ratio):
     shape = tl.small(wl.CONFIGS[ci], ratio_permille=ratio, **kw)
     p = tl.make_problem(shape, 900 + ci + ratio, T=70, T_cap=80)
     counts = _fused_launches(lambda: _check(shape, p))
-    assert counts["fused"] + counts["fused_tc"] + counts["fused_pair"] == 1 and counts["scores"] == 0
+    # one kernel per call for the LLaVA-NeXT block length, the three-kernel bf16 path for the Qwen2-VL one
+    assert counts["fused"] + counts["fused_tc"] + counts["fused_pair"] + counts["split_output"] == 1 and counts["scores"] == 0
 
 
 @pytest.mark.parametrize("B,H_q,H_kv,grid,R,T,ratio", [
