@@ -216,8 +216,8 @@ typedef enum {
   KVC_KERNEL_FUSED_TC = 8,        /* the same kernel with steps 2-3 on tcgen05 / tensor memory (see kvc_layer_create) */
   KVC_KERNEL_FUSED_PAIR = 9,      /* the tensor-memory kernel run by clusters of two CTAs per (sequence, KV head) */
   KVC_KERNEL_SPLIT_SCORES = 10,   /* three-kernel bf16 path: Alg. 1 step 1, one pass over K_tilde */
-  KVC_KERNEL_SPLIT_EXPAND = 11,   /* its steps 2-3 on tcgen05, per 128 expansion rows and range of the n axis */
-  KVC_KERNEL_SPLIT_OUTPUT = 12,   /* its step 4, the text rows and the normalisation, one pass over V_tilde and text K/V */
+  KVC_KERNEL_SPLIT_EXPAND = 11,   /* its steps 2-3 on tcgen05, per 128 expansion rows and range of the n axis; the text rows on idle SMs */
+  KVC_KERNEL_SPLIT_OUTPUT = 12,   /* its step 4 and the normalisation, one pass over V_tilde, merged with the text partials */
   KVC_KERNEL_COUNT = 13
 } kvc_kernel_id;
 KVC_API int kvc_profile_start(int max_launches);

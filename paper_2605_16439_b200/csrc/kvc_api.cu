@@ -95,7 +95,7 @@ WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap) {
     size_t sb = 0;
     if (B > 0 && R > 0) {
       const SplitPlan sp = plan_split(L, B, R);
-      if (sp.ok) sb = split_ws(L, sp, B, R).bytes;
+      if (sp.ok) sb = split_ws(L, sp, B, R, T_cap).bytes;
     }
     w.off_split = take(sb);
   }
@@ -326,7 +326,7 @@ int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B
     const uintptr_t align = reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(capsules) |
                             reinterpret_cast<uintptr_t>(out) | (T > 0 ? reinterpret_cast<uintptr_t>(K_txt) |
                             reinterpret_cast<uintptr_t>(V_txt) : 0) | reinterpret_cast<uintptr_t>(L->desc.mu);
-    if (!plain && (align & 15) == 0 && use_split(L, B, R)) {
+    if (!plain && (align & 15) == 0 && T <= 64 * SP_OUT_ROWS * SP_TEXT_CHUNK && use_split(L, B, R)) {
       const SplitPlan sp = plan_split(L, B, R);
       bool encoded = false;
       const cudaError_t se = launch_split(L, a, sp, st, &encoded);

@@ -4,8 +4,7 @@
 namespace kvc {
 
 cudaError_t launch_split_scores(const CUtensorMap& tmK, const SplitArgs& a, const SplitPlan& p, cudaStream_t st);
-cudaError_t launch_split_expand(const CUtensorMap& tmS, const CUtensorMap& tmTh, const CUtensorMap& tmU, const CUtensorMap& tmWs,
-                                const SplitArgs& a, const SplitPlan& p, cudaStream_t st);
+cudaError_t launch_split_expand(const CUtensorMap* tm, const SplitArgs& a, const SplitPlan& p, cudaStream_t st);
 cudaError_t launch_split_output(const CUtensorMap* tm, const SplitArgs& a, const SplitPlan& p, cudaStream_t st);
 
 constexpr uint32_t SP_SMEM_LIMIT = 232448;      // 227 KB per CTA on sm_100
@@ -44,7 +43,7 @@ SplitPlan plan_split(const kvc_layer* L, int B, int R) {
   p.e_p_bytes = (uint32_t)p.NW * 256u;
   const uint32_t st1 = 16384u + (uint32_t)(p.NW / 64) * 8192u, st2 = (uint32_t)p.prow * 128u;
   p.e_stage_bytes = ((st1 > st2 ? st1 : st2) + 1023u) & ~1023u;
-  p.e_stages = (int)((SP_SMEM_LIMIT - 2048u - p.e_p_bytes) / p.e_stage_bytes);
+  p.e_stages = (int)((SP_SMEM_LIMIT - 5120u - p.e_p_bytes) / p.e_stage_bytes);
   if (p.e_stages > 4) p.e_stages = 4;
   if (p.e_stages < 2) return p;
   p.e_smem = (size_t)p.e_p_bytes + (size_t)p.e_stages * p.e_stage_bytes + 1024;
@@ -60,8 +59,7 @@ SplitPlan plan_split(const kvc_layer* L, int B, int R) {
   // output kernel
   p.vt = ceil_div(m, SP_OUT_ROWS);
   p.o_w_bytes = (uint32_t)(p.NS * G) * 128u;
-  p.o_stage_bytes = 32768u;
-  if (16384u + p.o_w_bytes > p.o_stage_bytes) return p;
+  p.o_stage_bytes = (16384u + p.o_w_bytes + 1023u) & ~1023u;
   {
     // CTAs per (sequence, KV head): as many as the SMs allow (the same for every pair), at most one per value tile
     const long long bh = (long long)B * H_kv;
@@ -76,10 +74,10 @@ SplitPlan plan_split(const kvc_layer* L, int B, int R) {
     const int NH = G > 8 ? 2 : 1;
     uint32_t off = 0;
     auto take = [&](uint32_t bytes) { uint32_t o = off; off = (off + bytes + 127u) & ~127u; return o; };
-    p.o_off_q = take(16u * (uint32_t)D * 4u);                       // text part of a pair
+    p.o_off_q = take(16u * (uint32_t)D * 4u);                       // summed accumulators of a pair
     p.o_off_fac = take((uint32_t)(R * p.NS) * 16u * 8u);
     p.o_off_red = take(8u * NH * 8u * (uint32_t)D * 4u);
-    p.o_off_stat = take((uint32_t)(2 * 8 * 16 + 64 + 2 * p.o_cpb * 16) * 4u);
+    p.o_off_stat = take((uint32_t)(32 + 2 * (p.o_cpb + 64) * 16) * 4u);   // up to 64 text chunks (16384 text rows)
     if (off + 2048u + 2 * p.o_stage_bytes > SP_SMEM_LIMIT) return p;
     p.o_stages = (int)((SP_SMEM_LIMIT - 2048u - off) / p.o_stage_bytes);
     if (p.o_stages > SP_MAX_STAGES) p.o_stages = SP_MAX_STAGES;
@@ -91,7 +89,7 @@ SplitPlan plan_split(const kvc_layer* L, int B, int R) {
   return p;
 }
 
-SplitWs split_ws(const kvc_layer* L, const SplitPlan& p, int B, int R) {
+SplitWs split_ws(const kvc_layer* L, const SplitPlan& p, int B, int R, int T) {
   SplitWs w{};
   (void)R;
   const int H_kv = L->desc.H_kv, G = L->G;
@@ -104,6 +102,9 @@ SplitWs split_ws(const kvc_layer* L, const SplitPlan& p, int B, int R) {
   w.off_py = take(sizeof(float) * (size_t)B * H_kv * nslot * G * D);
   w.off_pml = take(sizeof(float2) * (size_t)B * H_kv * nslot * G);
   w.off_cnt = take(sizeof(int) * (size_t)B * H_kv);
+  const size_t nct = (size_t)ceil_div(ceil_div(T > 0 ? T : 0, SP_OUT_ROWS), SP_TEXT_CHUNK);
+  w.off_tpy = take(sizeof(float) * (size_t)B * H_kv * nct * G * D);
+  w.off_tpml = take(sizeof(float2) * (size_t)B * H_kv * nct * G);
   w.bytes = off;
   return w;
 }
@@ -112,7 +113,7 @@ cudaError_t launch_split(const kvc_layer* L, const DecodeArgs& a, const SplitPla
   const int H_kv = a.H_kv, m = a.m, n = a.n, R = a.R, B = a.B, G = a.G;
   *encoded = false;
   char* ws = reinterpret_cast<char*>(a.split_base);
-  const SplitWs w = split_ws(L, p, B, R);
+  const SplitWs w = split_ws(L, p, B, R, a.T);
   CUtensorMap tmK, tmS, tmTh, tmU, tmWs, tmO[4];
   {
     // K_tilde as (channels, R m rows of a pair, pairs): rows past the pair's last are zero-filled, not read
@@ -178,6 +179,8 @@ cudaError_t launch_split(const kvc_layer* L, const DecodeArgs& a, const SplitPla
   sa.py = reinterpret_cast<float*>(ws + w.off_py);
   sa.pml = reinterpret_cast<float2*>(ws + w.off_pml);
   sa.cnt = reinterpret_cast<int*>(ws + w.off_cnt);
+  sa.tpy = reinterpret_cast<float*>(ws + w.off_tpy);
+  sa.tpml = reinterpret_cast<float2*>(ws + w.off_tpml);
   sa.status = a.status;
   sa.B = B; sa.H_kv = H_kv; sa.G = G; sa.R = R; sa.m = m; sa.n = n; sa.T = a.T;
   sa.rows_h = p.rows_h; sa.ntile = p.ntile; sa.NS = p.NS; sa.NW = p.NW; sa.ms = p.ms; sa.nk1 = p.nk1;
@@ -188,8 +191,18 @@ cudaError_t launch_split(const kvc_layer* L, const DecodeArgs& a, const SplitPla
   sa.o_cpb = p.o_cpb;
   sa.o_off_q = p.o_off_q; sa.o_off_fac = p.o_off_fac; sa.o_off_red = p.o_off_red; sa.o_off_stat = p.o_off_stat;
 
+  sa.e_grid = p.e_grid;
+  {
+    // text CTAs: the SMs the expansion CTAs leave idle in their last wave (a dozen at least), one item each at most
+    const int sms = L->num_sms > 0 ? L->num_sms : 148;
+    const long long items = (long long)B * H_kv * ceil_div(ceil_div(a.T, SP_OUT_ROWS), SP_TEXT_CHUNK);
+    int idle = sms - p.e_grid % sms;
+    if (idle < 12) idle = 12;
+    sa.tx_grid = a.T > 0 ? (int)(items < idle ? items : idle) : 0;
+  }
+  const CUtensorMap tmE[6] = {tmS, tmTh, tmU, tmWs, tmO[1], tmO[2]};
   cudaError_t e = launch_split_scores(tmK, sa, p, st);
-  if (e == cudaSuccess) e = launch_split_expand(tmS, tmTh, tmU, tmWs, sa, p, st);
+  if (e == cudaSuccess) e = launch_split_expand(tmE, sa, p, st);
   if (e == cudaSuccess) e = launch_split_output(tmO, sa, p, st);
   return e;
 }

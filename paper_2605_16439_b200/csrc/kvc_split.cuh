@@ -17,7 +17,8 @@ namespace kvc {
 
 constexpr int SP_TILE_ROWS = 128;      // retained key rows per stage of the score kernel; expansion rows per expansion CTA
 constexpr int SP_OUT_ROWS = 64;        // value rows (and text rows) per stage of the output kernel
-constexpr int SP_MAX_STAGES = 8;
+constexpr int SP_MAX_STAGES = 12;
+constexpr int SP_TEXT_CHUNK = 3;       // 64-row tiles of text per CTA of the text kernel (96 KB of stages: two CTAs per SM)
 
 struct SplitPlan {
   int ok;
@@ -45,12 +46,14 @@ struct SplitWs {
   size_t off_stat;   // float2 [H_kv][NS][rows_h]  (row maximum in log2 units, row sum)
   size_t off_py;     // fp32 [B*H_kv][o_cpb][G][D]
   size_t off_pml;    // float2 [B*H_kv][o_cpb][G]
-  size_t off_cnt;    // int [B*H_kv]  arrivals of the output kernel's segments, cleared by the score kernel
+  size_t off_cnt;    // int [B*H_kv]  arrivals of the output kernel's CTAs, cleared by the score kernel
+  size_t off_tpy;    // fp32 [B*H_kv][chunks][G][D]   partials of the text kernel
+  size_t off_tpml;   // float2 [B*H_kv][chunks][G]
   size_t bytes;
 };
 
 SplitPlan plan_split(const kvc_layer* L, int B, int R);
-SplitWs split_ws(const kvc_layer* L, const SplitPlan& p, int B, int R);
+SplitWs split_ws(const kvc_layer* L, const SplitPlan& p, int B, int R, int T);
 cudaError_t launch_split(const kvc_layer* L, const DecodeArgs& a, const SplitPlan& p, cudaStream_t st, bool* encoded);
 
 struct SplitArgs {
@@ -62,11 +65,14 @@ struct SplitArgs {
   float2* stat;
   float* py;
   float2* pml;
+  float* tpy;        // text kernel: [B*H_kv][chunks][G][D]
+  float2* tpml;      // [B*H_kv][chunks][G]
   int* cnt;
   int* status;
   int B, H_kv, G, R, m, n, T;
   int rows_h, ntile, NS, NW, ms, nk1, npass, prow, nbox, brow, tmem_cols;
   int e_stages; uint32_t e_stage_bytes;
+  int e_grid, tx_grid;   // expansion CTAs; text CTAs behind them in the same grid
   int s_tiles_bh, s_stages;
   int vt, o_stages; uint32_t o_stage_bytes;
   int o_cpb;
@@ -82,9 +88,9 @@ constexpr float SP_QSCALE = 0.08838834764831845f * 1.4426950408889634f;
 // over all rounds; the consumers of round w first wait (bounded) until every warp of the rounds before has released,
 // which pins the barrier's current phase to round w.
 constexpr int SP_GROUP = 4;            // warps that share a tile
-__device__ __forceinline__ bool wait_round(const volatile uint32_t* released, uint32_t slot, uint32_t round) {
+__device__ __forceinline__ bool wait_round(const volatile uint32_t* released, uint32_t slot, uint32_t round, uint32_t group = SP_GROUP) {
   for (uint32_t i = 0; i < (1u << 24); ++i)
-    if (released[slot] >= round * SP_GROUP) return true;
+    if (released[slot] >= round * group) return true;
   return false;
 }
 __device__ __forceinline__ void release_slot(uint32_t* released, uint64_t* empty_bar, uint32_t slot) {

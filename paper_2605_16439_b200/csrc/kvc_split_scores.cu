@@ -2,16 +2,16 @@
 //   S[h][(b R + r) G + g][j] = sigma log2(e) q[b, hG + g, :] . K_tilde[b, h, r, j, :]      (bf16, fp32 accumulation)
 // One streaming pass over K_tilde, bound by HBM bandwidth.  The R m key rows of a (sequence, KV head) are contiguous in
 // the capsule store; they are cut into tiles of 128 rows and the flat tile list is dealt in contiguous runs to one
-// persistent CTA per SM.  A producer thread keeps a ring of TMA-filled 32 KB stages full (128-byte swizzle).  The eight
-// consumer warps form two groups of four; tile k of the CTA's run goes to group k mod 2 and each warp of the group takes
-// 32 of its rows (a stage is held only for that short time, and two tiles are in work at once): the queries of the KV
-// head (up to 16, zero-padded) are the A operand held in registers, the key rows the B operand read with ldmatrix, and a
-// lane ends up with two consecutive key rows of one head.
+// persistent CTA per SM.  A producer thread keeps a ring of TMA-filled 32 KB stages full (128-byte swizzle).  Each of
+// the sixteen consumer warps takes 8 rows of every tile (a tile is a chain of dependent steps per warp, so its latency,
+// not its instruction count, sets the pace: more and shorter chains): the queries of the KV head (up to 16, zero-padded) are the A
+// operand held in registers, the key rows the B operand read with ldmatrix, and a lane ends up with two consecutive key
+// rows of one head.
 #include "kvc_split.cuh"
 
 namespace kvc {
 
-constexpr int SS_WARPS = 8;
+constexpr int SS_WARPS = 16;
 constexpr int SS_THREADS = (SS_WARPS + 1) * 32;
 constexpr uint32_t SS_HALF = SP_TILE_ROWS * 128;      // one 64-channel half of a tile
 constexpr uint32_t SS_STAGE = 2 * SS_HALF;
@@ -21,10 +21,9 @@ split_scores_kernel(const __grid_constant__ CUtensorMap tmK, const SplitArgs a) 
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* sm = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
   __shared__ __align__(8) uint64_t full_bar[SP_MAX_STAGES], empty_bar[SP_MAX_STAGES];
-  __shared__ uint32_t released[SP_MAX_STAGES];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
-    for (int s = 0; s < a.s_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], SP_GROUP); released[s] = 0u; }
+    for (int s = 0; s < a.s_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], SS_WARPS); }
     fence_mbar_init();
   }
   __syncthreads();
@@ -37,10 +36,21 @@ split_scores_kernel(const __grid_constant__ CUtensorMap tmK, const SplitArgs a) 
   if (warp == SS_WARPS) {
     if (lane != 0) return;
     tma_prefetch_desc(&tmK);
+    {
+      // while the stream's previous kernel drains: the first ring of tiles is asked into L2 (a prefetch consumes no
+      // data, so it need not wait for that kernel; the loads below do)
+      int pbh = (int)(lo / a.s_tiles_bh), pt = (int)(lo - (long long)pbh * a.s_tiles_bh);
+      for (int k = 0; k < nst && lo + k < hi; ++k) {
+        tma_prefetch_l2_3d(&tmK, 0, pt * SP_TILE_ROWS, pbh);
+        tma_prefetch_l2_3d(&tmK, 64, pt * SP_TILE_ROWS, pbh);
+        if (++pt == a.s_tiles_bh) { pt = 0; ++pbh; }
+      }
+    }
     grid_dep_wait();                              // the capsules and the queries may come from the stream's previous kernel
     uint32_t slot = 0, phase = 1;
-    for (long long i = lo; i < hi; ++i) {
-      const int bh = (int)(i / a.s_tiles_bh), t = (int)(i - (long long)bh * a.s_tiles_bh);
+    int bh = (int)(lo / a.s_tiles_bh), t = (int)(lo - (long long)bh * a.s_tiles_bh) - 1;
+    for (int it = (int)(hi - lo); it > 0; --it) {
+      if (++t == a.s_tiles_bh) { t = 0; ++bh; }
       if (!mbar_wait_bounded(&empty_bar[slot], phase)) { atomicExch(a.status, (int)KVC_ERR_TIMEOUT); return; }
       unsigned char* dst = sm + slot * SS_STAGE;
       mbar_expect_tx(&full_bar[slot], SS_STAGE);
@@ -63,11 +73,10 @@ split_scores_kernel(const __grid_constant__ CUtensorMap tmK, const SplitArgs a) 
   bool dead = false;
   int cur_bh = -1;
   uint32_t qa[8][4];
-  const int grp = warp / SP_GROUP, wj = warp % SP_GROUP;
-  for (long long k = grp; lo + k < hi; k += SS_WARPS / SP_GROUP) {
-    const long long i = lo + k;
-    const uint32_t slot = (uint32_t)(k % nst), round = (uint32_t)(k / nst), phase = round & 1u;
-    const int bh = (int)(i / a.s_tiles_bh), t = (int)(i - (long long)bh * a.s_tiles_bh);
+  uint32_t slot = 0, phase = 0;
+  int bh = (int)(lo / a.s_tiles_bh), t = (int)(lo - (long long)bh * a.s_tiles_bh) - 1;
+  for (int it = (int)(hi - lo); it > 0; --it) {
+    if (++t == a.s_tiles_bh) { t = 0; ++bh; }
     const int b = bh / a.H_kv, h = bh - b * a.H_kv;
     if (bh != cur_bh) {
       cur_bh = bh;
@@ -82,7 +91,7 @@ split_scores_kernel(const __grid_constant__ CUtensorMap tmK, const SplitArgs a) 
         qa[ks][3] = gid + 8 < G ? *reinterpret_cast<const uint32_t*>(q0 + (size_t)(gid + 8) * D + k0 + 8) : 0u;
       }
     }
-    if (!dead && !(wait_round(released, slot, round) && mbar_wait_bounded(&full_bar[slot], phase))) dead = true;
+    if (!dead && !mbar_wait_bounded(&full_bar[slot], phase)) dead = true;
     __syncwarp();
     const uint32_t st_u = sm_u + slot * SS_STAGE;
     // (block, row in block) of the tile's first key row; the rows of a lane follow by small steps
@@ -90,30 +99,26 @@ split_scores_kernel(const __grid_constant__ CUtensorMap tmK, const SplitArgs a) 
     const int r_t = g0 / m, j_t = g0 - r_t * m;
     __nv_bfloat16* S_h = a.S + (size_t)h * a.rows_h * a.ms;
     const int bR = b * a.R;
+    {
+      const int row0 = warp * 8;                   // this warp's 8 rows: two accumulation chains over the channel halves
+      float acc2[2][4];
 #pragma unroll
-    for (int np = 2 * wj; np < 2 * wj + 2; ++np) { // 16 rows per step as two 8-row groups: independent accumulation chains
-      float acc[2][4];
+      for (int x = 0; x < 2; ++x)
 #pragma unroll
-      for (int nt = 0; nt < 2; ++nt) {
+        for (int e = 0; e < 4; ++e) acc2[x][e] = 0.f;
+      const int row = row0 + (lane & 7);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
-        const int row = np * 16 + nt * 8 + (lane & 7);
-#pragma unroll
-        for (int x = 0; x < 4; ++x) {
-          // four 8 x 8 matrices: the 16-byte pieces 4x .. 4x+3 of rows row0 .. row0+7 (pieces 0-7 in the first half)
-          const int c = 4 * x + (lane >> 3);
-          uint32_t bf[4];
-          ldsm_x4(bf, st_u + (uint32_t)(c >> 3) * SS_HALF + (uint32_t)row * 128u + (uint32_t)((((c & 7) ^ (row & 7))) << 4));
-          mma_bf16_16816(acc[nt], qa[2 * x], bf[0], bf[1]);
-          mma_bf16_16816(acc[nt], qa[2 * x + 1], bf[2], bf[3]);
-        }
+      for (int x = 0; x < 4; ++x) {
+        // four 8 x 8 matrices: the 16-byte pieces 4x .. 4x+3 of rows row0 .. row0+7 (pieces 0-7 in the first half)
+        const int c = 4 * x + (lane >> 3);
+        uint32_t bf[4];
+        ldsm_x4(bf, st_u + (uint32_t)(c >> 3) * SS_HALF + (uint32_t)row * 128u + (uint32_t)((((c & 7) ^ (row & 7))) << 4));
+        mma_bf16_16816(acc2[x & 1], qa[2 * x], bf[0], bf[1]);
+        mma_bf16_16816(acc2[x & 1], qa[2 * x + 1], bf[2], bf[3]);
       }
-      if (dead) continue;
-      // acc[nt][e]: head gid + 8 (e >> 1), key row g0 + np*16 + nt*8 + 2 t4 + (e & 1) of the (sequence, KV head)
-#pragma unroll
-      for (int nt = 0; nt < 2; ++nt) {
-        const int off = np * 16 + nt * 8 + 2 * t4;
-        if (g0 + off >= Rm) continue;
+      // acc[e]: head gid + 8 (e >> 1), key row g0 + row0 + 2 t4 + (e & 1) of the (sequence, KV head)
+      const int off = row0 + 2 * t4;
+      if (!dead && g0 + off < Rm) {
         int r = r_t, j = j_t + off;
         if (m >= SP_TILE_ROWS) { if (j >= m) { j -= m; ++r; } }
         else { const int dr = j / m; r += dr; j -= dr * m; }
@@ -124,7 +129,7 @@ split_scores_kernel(const __grid_constant__ CUtensorMap tmK, const SplitArgs a) 
         for (int hh = 0; hh < 2; ++hh) {
           const int head = gid + 8 * hh;
           if (head >= G) continue;
-          const float v0 = acc[nt][2 * hh] * SP_QSCALE, v1 = acc[nt][2 * hh + 1] * SP_QSCALE;
+          const float v0 = (acc2[0][2 * hh] + acc2[1][2 * hh]) * SP_QSCALE, v1 = (acc2[0][2 * hh + 1] + acc2[1][2 * hh + 1]) * SP_QSCALE;
           __nv_bfloat16* p0 = S_h + ((size_t)(bR + r) * G + head) * a.ms + j;
           if (second && r1 == r && (j & 1) == 0) {
             *reinterpret_cast<uint32_t*>(p0) = pack2_bf16(v0, v1);
@@ -136,7 +141,8 @@ split_scores_kernel(const __grid_constant__ CUtensorMap tmK, const SplitArgs a) 
       }
     }
     __syncwarp();
-    if (lane == 0) release_slot(released, empty_bar, slot);
+    if (lane == 0) mbar_arrive(&empty_bar[slot]);
+    if (++slot == (uint32_t)nst) { slot = 0; phase ^= 1u; }
   }
   if (dead && lane == 0) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
 }
