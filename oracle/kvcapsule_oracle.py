@@ -29,6 +29,9 @@ Readings of the paper taken here (each also listed in the design document):
   - compression ratio rho = 1 - l_r;  m = ceil(l_r n) in integer arithmetic on
     rho expressed in permille.
   - rho = 0 is a pass-through: capsules hold K and V verbatim.
+  - the one-sided variants of App. G (Table 6) compress one side and keep the other verbatim:
+    mode "k" stores the retained key rows and the full values (theta only), mode "v" the full keys
+    and the projected values (U, mu only); mode "kv" is the method itself.
 
 Parity pins: every function below is pinned by tests/test_oracle_pins.py
 (library attention, lossless constructions, Eckart-Young, closed forms, brute
@@ -96,8 +99,10 @@ def attention(q, K, V) -> np.ndarray:
 # --------------------------------------------------------------------------
 # prefill-stage compression (Sec. 3.2 "Prefilling Stage")
 # --------------------------------------------------------------------------
-def compress(K_vis, V_vis, idx, U, mu, n: int, passthrough: bool = False):
-    """K_tilde = rows idx of each block's keys; V_tilde = U (V - 1 mu^T) per block."""
+def compress(K_vis, V_vis, idx, U, mu, n: int, passthrough: bool = False, mode: str = "kv"):
+    """K_tilde = rows idx of each block's keys; V_tilde = U (V - 1 mu^T) per block.
+    mode "k": only the keys are compressed (V_tilde = the block's values verbatim, n rows);
+    mode "v": only the values (K_tilde = the block's keys verbatim, n rows)."""
     K_vis, V_vis = np.asarray(K_vis, F64), np.asarray(V_vis, F64)
     B, H_kv, N_v, d = K_vis.shape
     if N_v % n != 0:
@@ -105,40 +110,55 @@ def compress(K_vis, V_vis, idx, U, mu, n: int, passthrough: bool = False):
     R = N_v // n
     if passthrough:
         return (K_vis.reshape(B, H_kv, R, n, d).copy(), V_vis.reshape(B, H_kv, R, n, d).copy())
-    U, mu = np.asarray(U, F64), np.asarray(mu, F64)
-    m = U.shape[1]
-    K_t = np.zeros((B, H_kv, R, m, d), F64)
-    V_t = np.zeros((B, H_kv, R, m, d), F64)
+    if mode != "k":
+        U, mu = np.asarray(U, F64), np.asarray(mu, F64)
+    m_k = n if mode == "v" else len(_idx_for_head(idx, 0))
+    m_v = n if mode == "k" else U.shape[1]
+    K_t = np.zeros((B, H_kv, R, m_k, d), F64)
+    V_t = np.zeros((B, H_kv, R, m_v, d), F64)
     for b in range(B):
         for h in range(H_kv):
-            sel = _idx_for_head(idx, h)
             for r in range(R):
                 K_blk = K_vis[b, h, r * n:(r + 1) * n]
                 V_blk = V_vis[b, h, r * n:(r + 1) * n]
-                K_t[b, h, r] = K_blk[sel]                       # row selection by M_l
-                V_center = V_blk - np.ones((n, 1), F64) * mu[h][None, :]
-                V_t[b, h, r] = U[h] @ V_center                  # sequence-level PCA projection
+                if mode == "v":
+                    K_t[b, h, r] = K_blk
+                else:
+                    K_t[b, h, r] = K_blk[_idx_for_head(idx, h)]  # row selection by M_l
+                if mode == "k":
+                    V_t[b, h, r] = V_blk
+                else:
+                    V_center = V_blk - np.ones((n, 1), F64) * mu[h][None, :]
+                    V_t[b, h, r] = U[h] @ V_center              # sequence-level PCA projection
     return K_t, V_t
 
 
 # --------------------------------------------------------------------------
 # decode-stage reconstruction (Sec. 3.2 "Decoding Stage")
 # --------------------------------------------------------------------------
-def reconstruct(K_t, V_t, theta, U, mu, passthrough: bool = False):
-    """K_hat = theta^T K_tilde,  V_hat = U^T V_tilde + 1 mu^T;  returns [B,H_kv,R*n,d] each."""
+def reconstruct(K_t, V_t, theta, U, mu, passthrough: bool = False, mode: str = "kv"):
+    """K_hat = theta^T K_tilde,  V_hat = U^T V_tilde + 1 mu^T;  returns [B,H_kv,R*n,d] each.
+    The side a one-sided mode keeps verbatim is returned as stored."""
     K_t, V_t = np.asarray(K_t, F64), np.asarray(V_t, F64)
-    B, H_kv, R, m, d = K_t.shape
+    B, H_kv, R, _, d = K_t.shape
     if passthrough:
+        m = K_t.shape[3]
         return K_t.reshape(B, H_kv, R * m, d).copy(), V_t.reshape(B, H_kv, R * m, d).copy()
-    theta, U, mu = np.asarray(theta, F64), np.asarray(U, F64), np.asarray(mu, F64)
-    n = theta.shape[2]
+    n = K_t.shape[3] if mode == "v" else np.asarray(theta).shape[2]
     K_hat = np.zeros((B, H_kv, R * n, d), F64)
     V_hat = np.zeros((B, H_kv, R * n, d), F64)
     for b in range(B):
         for h in range(H_kv):
             for r in range(R):
-                K_hat[b, h, r * n:(r + 1) * n] = theta[h].T @ K_t[b, h, r]
-                V_hat[b, h, r * n:(r + 1) * n] = U[h].T @ V_t[b, h, r] + np.ones((n, 1), F64) * mu[h][None, :]
+                if mode == "v":
+                    K_hat[b, h, r * n:(r + 1) * n] = K_t[b, h, r]
+                else:
+                    K_hat[b, h, r * n:(r + 1) * n] = np.asarray(theta[h], F64).T @ K_t[b, h, r]
+                if mode == "k":
+                    V_hat[b, h, r * n:(r + 1) * n] = V_t[b, h, r]
+                else:
+                    V_hat[b, h, r * n:(r + 1) * n] = (np.asarray(U[h], F64).T @ V_t[b, h, r]
+                                                      + np.ones((n, 1), F64) * np.asarray(mu[h], F64)[None, :])
     return K_hat, V_hat
 
 
@@ -158,9 +178,9 @@ def collapse_reconstructor(W1, W2) -> np.ndarray:
     return theta
 
 
-def decode_attend_definition(q, K_t, V_t, theta, U, mu, K_txt, V_txt, passthrough: bool = False):
+def decode_attend_definition(q, K_t, V_t, theta, U, mu, K_txt, V_txt, passthrough: bool = False, mode: str = "kv"):
     """Form 1: reconstruct, concatenate with text K/V, run the original attention."""
-    K_hat, V_hat = reconstruct(K_t, V_t, theta, U, mu, passthrough)
+    K_hat, V_hat = reconstruct(K_t, V_t, theta, U, mu, passthrough, mode)
     K_all = np.concatenate([K_hat, np.asarray(K_txt, F64)], axis=2)
     V_all = np.concatenate([V_hat, np.asarray(V_txt, F64)], axis=2)
     return attention(q, K_all, V_all)
@@ -169,8 +189,11 @@ def decode_attend_definition(q, K_t, V_t, theta, U, mu, K_txt, V_txt, passthroug
 # --------------------------------------------------------------------------
 # Algorithm 1 (fused KVCapsule), with the text tail in the same softmax
 # --------------------------------------------------------------------------
-def decode_attend_fused(q, K_t, V_t, theta, U, mu, K_txt, V_txt, passthrough: bool = False):
+def decode_attend_fused(q, K_t, V_t, theta, U, mu, K_txt, V_txt, passthrough: bool = False, mode: str = "kv"):
     """Form 2: the associative order of Alg. 1 (steps 1-4) for one decode query per sequence.
+    In a one-sided mode the side kept verbatim skips its step: mode "k" has no re-projection (the
+    probabilities meet the n stored value rows directly), mode "v" no score expansion (the query meets
+    all n stored keys).
 
     Nothing of length n x d is formed.  Per (sequence b, KV head h) and for the G query heads that read h:
       step 1  the query meets the m retained keys of every block:           s_c[g, r, j]
@@ -189,7 +212,16 @@ def decode_attend_fused(q, K_t, V_t, theta, U, mu, K_txt, V_txt, passthrough: bo
         theta = U = np.broadcast_to(np.eye(m, dtype=F64), (H_kv, m, m))
         mu = np.zeros((H_kv, d), F64)
     else:
-        theta, U, mu = np.asarray(theta, F64), np.asarray(U, F64), np.asarray(mu, F64)
+        if mode == "v":                  # keys verbatim: the expansion is the identity on the n stored keys
+            theta = np.broadcast_to(np.eye(m, dtype=F64), (H_kv, m, m))
+        else:
+            theta = np.asarray(theta, F64)
+        if mode == "k":                  # values verbatim: no re-projection, no centring term
+            nv = V_t.shape[3]
+            U = np.broadcast_to(np.eye(nv, dtype=F64), (H_kv, nv, nv))
+            mu = np.zeros((H_kv, d), F64)
+        else:
+            U, mu = np.asarray(U, F64), np.asarray(mu, F64)
     n = theta.shape[2]
     scale = 1.0 / np.sqrt(F64(d))
     out = np.zeros((B, H_q, d), F64)
@@ -210,7 +242,7 @@ def decode_attend_fused(q, K_t, V_t, theta, U, mu, K_txt, V_txt, passthrough: bo
                 prob = softmax(np.concatenate([logit_v.reshape(R * n), logit_t]))
                 prob_v, prob_t = prob[:R * n].reshape(R, n), prob[R * n:]
                 # step 3
-                w_c = np.zeros((R, m), F64)
+                w_c = np.zeros((R, U.shape[1]), F64)
                 for r in range(R):
                     w_c[r] = U[h] @ prob_v[r]
                 # step 4

@@ -195,6 +195,49 @@ def test_value_pca_is_eckart_young_optimal():
     np.testing.assert_allclose(resid, np.sum(s[m:] ** 2), rtol=1e-10)
 
 
+# ---------------------------------------------------------------- one-sided variants (App. G)
+def test_one_sided_modes():
+    """Mode "k" (keys compressed, values verbatim) and mode "v" (values compressed, keys verbatim): (i) each equals the
+    two-sided method given the identity on the side it keeps (U = I_n, mu = 0, or theta = I_n with every index
+    retained), which ties them to the pinned two-sided path; (ii) with the lossless construction on the compressed
+    side they reproduce full attention through the library routine; (iii) definition == Alg. 1 order."""
+    p = _problem(21)
+    r = _rng(210)
+    n, m, H_kv, d = p["n"], p["m"], 2, 8
+    eye_n = np.broadcast_to(np.eye(n), (H_kv, n, n))
+    K_all = lambda Kv: np.concatenate([Kv, p["K_txt"]], axis=2)
+    V_all = lambda Vv: np.concatenate([Vv, p["V_txt"]], axis=2)
+    # ---- mode "k"
+    K_t, V_t = orc.compress(p["K_vis"], p["V_vis"], p["idx"], None, None, n, mode="k")
+    assert K_t.shape[3] == m and V_t.shape[3] == n
+    assert np.array_equal(V_t.reshape(p["V_vis"].shape), p["V_vis"])
+    a = orc.decode_attend_definition(p["q"], K_t, V_t, p["theta"], None, None, p["K_txt"], p["V_txt"], mode="k")
+    b = orc.decode_attend_fused(p["q"], K_t, V_t, p["theta"], None, None, p["K_txt"], p["V_txt"], mode="k")
+    np.testing.assert_allclose(a, b, atol=1e-10)
+    K2, V2 = orc.compress(p["K_vis"], p["V_vis"], p["idx"], eye_n, np.zeros((H_kv, d)), n)
+    c = orc.decode_attend_definition(p["q"], K2, V2, p["theta"], eye_n, np.zeros((H_kv, d)), p["K_txt"], p["V_txt"])
+    np.testing.assert_allclose(a, c, atol=1e-12)
+    theta_l, K_l = _lossless_key_side(p, r)
+    K_t, V_t = orc.compress(K_l, p["V_vis"], p["idx"], None, None, n, mode="k")
+    got = orc.decode_attend_fused(p["q"], K_t, V_t, theta_l, None, None, p["K_txt"], p["V_txt"], mode="k")
+    np.testing.assert_allclose(got, _library_attention(p["q"], K_all(K_l), V_all(p["V_vis"])), atol=1e-11)
+    # ---- mode "v"
+    K_t, V_t = orc.compress(p["K_vis"], p["V_vis"], None, p["U"], p["mu"], n, mode="v")
+    assert K_t.shape[3] == n and V_t.shape[3] == m
+    assert np.array_equal(K_t.reshape(p["K_vis"].shape), p["K_vis"])
+    a = orc.decode_attend_definition(p["q"], K_t, V_t, None, p["U"], p["mu"], p["K_txt"], p["V_txt"], mode="v")
+    b = orc.decode_attend_fused(p["q"], K_t, V_t, None, p["U"], p["mu"], p["K_txt"], p["V_txt"], mode="v")
+    np.testing.assert_allclose(a, b, atol=1e-10)
+    # the two-sided method with every key retained and theta = I_n, on the same U and mu
+    K2 = p["K_vis"].reshape(2, H_kv, p["R"], n, d)
+    c = orc.decode_attend_definition(p["q"], K2, V_t, eye_n, p["U"], p["mu"], p["K_txt"], p["V_txt"])
+    np.testing.assert_allclose(a, c, atol=1e-12)
+    U_l, V_l = _lossless_value_side(p, r)
+    K_t, V_t = orc.compress(p["K_vis"], V_l, None, U_l, p["mu"], n, mode="v")
+    got = orc.decode_attend_fused(p["q"], K_t, V_t, None, U_l, p["mu"], p["K_txt"], p["V_txt"], mode="v")
+    np.testing.assert_allclose(got, _library_attention(p["q"], K_all(p["K_vis"]), V_all(V_l)), atol=1e-11)
+
+
 # ---------------------------------------------------------------- fused algebra
 @pytest.mark.parametrize("seed,kw", [(10, {}), (11, dict(B=1, H_q=4, H_kv=4, R=1, T=0)),
                                      (12, dict(H_q=8, H_kv=1, n=9, m=9, R=2, T=1))])
