@@ -588,11 +588,19 @@ def measure(shape, config_index, dev, rank, world, local, steps, warmup, profile
             # prologues, which the per-launch brackets of the second pass forbid)
             alg = contract
             avg_us = ms_decode / calls * 1e3
+        elif dom.startswith("split_"):
+            # three dependent kernels per layer call that overlap their ramps (programmatic dependent launch): the unit
+            # the roofline is taken over is the layer call, against the bytes the whole call must move; per-kernel
+            # brackets forbid that overlap and are listed under "kernels" for the shares only
+            dom = "split_scores+split_expand+split_output"
+            alg = contract
+            avg_us = ms_decode / calls * 1e3
+            t_dom = sum(prof.get(k, (0.0, 0))[0] for k in ("split_scores", "split_expand", "split_output"))
+            n_dom = prof["split_scores"][1]
         else:
             # several kernels per layer call: the dominant one against its own stream (one of K_tilde / V_tilde, the
             # text rows it reads, q or out), from its event brackets
-            alg = stream_kernel_bytes(shape, m, T_mid) + (
-                shape.B * shape.H_kv * int(T_mid) * shape.d * elem_bytes(shape) if dom == "split_output" else 0)
+            alg = stream_kernel_bytes(shape, m, T_mid)
             avg_us = t_dom / n_dom * 1e3
         achieved = alg / (avg_us * 1e-6) / 1e9
         roofline = {"kernel": dom, "bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",

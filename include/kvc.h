@@ -53,6 +53,14 @@ typedef enum {
 
 typedef enum { KVC_F32 = 0, KVC_BF16 = 1 } kvc_dtype;
 
+/* Which sides of the cache are compressed.  KVC_MODE_KV is the method (Sec. 3.1).  The one-sided settings of the
+ * ablation on K-side and V-side reconstruction (App. G, Table 6) keep the other side verbatim:
+ *   KVC_MODE_K_ONLY  K_tilde = the m retained key rows (theta expands the scores), V stored with all n rows per block:
+ *                    out = softmax(sigma q [theta^T K_tilde ; K_txt]^T) [V ; V_txt]          (no U, no mu)
+ *   KVC_MODE_V_ONLY  K stored with all n rows per block, V_tilde = U (V - 1 mu^T):
+ *                    out = softmax(sigma q [K ; K_txt]^T) [U^T V_tilde + 1 mu^T ; V_txt]     (no idx, no theta) */
+typedef enum { KVC_MODE_KV = 0, KVC_MODE_K_ONLY = 1, KVC_MODE_V_ONLY = 2 } kvc_mode;
+
 /* One parameter set = one (layer, compression ratio); the paper trains M_l, theta_l, U_l, mu_l
  * per layer for a given retention ratio (App. C, Algorithm 2) and fixes them at inference
  * (Sec. 3.2).  Shapes follow App. D: theta, U in R^{H_kv x m x n}, mu in R^{H_kv x d}. */
@@ -68,6 +76,8 @@ typedef struct {
   const void* theta;      /* [H_kv][m][n]  key / score reconstruction matrix (borrowed)        */
   const void* U;          /* [H_kv][m][n]  value PCA basis (borrowed); rows need not be orthonormal */
   const void* mu;         /* [H_kv][d]     value centering vector (borrowed)                   */
+  int mode;               /* kvc_mode; 0 = both sides compressed.  K_ONLY ignores U and mu,    */
+                          /*   V_ONLY ignores idx and theta (they may be NULL)                 */
 } kvc_layer_desc;
 
 typedef struct kvc_layer kvc_layer;
@@ -90,9 +100,14 @@ KVC_API int kvc_retained_len(int n, int ratio_permille);
 KVC_API int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out);
 KVC_API int kvc_layer_destroy(kvc_layer* layer);
 
-/* Bytes of the capsule store for B sequences of R blocks:  K_tilde [B][H_kv][R][m][d] followed
- * by V_tilde [B][H_kv][R][m][d] (the compressed-cache term of App. D, Eq. 2, vision part). */
+/* Bytes of the capsule store for B sequences of R blocks:  K_tilde [B][H_kv][R][m_k][d] followed
+ * by V_tilde [B][H_kv][R][m_v][d] (the compressed-cache term of App. D, Eq. 2, vision part), with m_k = m_v = m
+ * unless a one-sided mode keeps a side verbatim (then n rows per block on that side). */
 KVC_API size_t kvc_capsule_bytes(const kvc_layer* layer, int B, int R);
+
+/* Rows per block the capsule store holds on the key side (m_k) and on the value side (m_v); either pointer may be
+ * NULL.  KVC_ERR_ARG for a NULL handle. */
+KVC_API int kvc_layer_rows(const kvc_layer* layer, int* key_rows, int* value_rows);
 
 /* Bytes of scratch kvc_decode_attend needs for B sequences of R blocks and up to T_cap text rows
  * (the figure grows with T_cap but is not monotone in B and R: size it for the B and R you call

@@ -29,7 +29,11 @@ class KvcError(RuntimeError):
 class kvc_layer_desc(C.Structure):
     _fields_ = [("layer", C.c_int), ("H_q", C.c_int), ("H_kv", C.c_int), ("d", C.c_int), ("n", C.c_int),
                 ("ratio_permille", C.c_int), ("dtype", C.c_int), ("idx", C.POINTER(C.c_int32)),
-                ("idx_per_head", C.c_int), ("theta", C.c_void_p), ("U", C.c_void_p), ("mu", C.c_void_p)]
+                ("idx_per_head", C.c_int), ("theta", C.c_void_p), ("U", C.c_void_p), ("mu", C.c_void_p),
+                ("mode", C.c_int)]
+
+
+KVC_MODE_KV, KVC_MODE_K_ONLY, KVC_MODE_V_ONLY = 0, 1, 2
 
 
 _LIB = None
@@ -47,6 +51,7 @@ def _lib() -> C.CDLL:
         lib.kvc_layer_create.argtypes = [C.POINTER(kvc_layer_desc), C.POINTER(vp)]; lib.kvc_layer_create.restype = i
         lib.kvc_layer_destroy.argtypes = [vp]; lib.kvc_layer_destroy.restype = i
         lib.kvc_layer_m.argtypes = [vp]; lib.kvc_layer_m.restype = i
+        lib.kvc_layer_rows.argtypes = [vp, C.POINTER(i), C.POINTER(i)]; lib.kvc_layer_rows.restype = i
         lib.kvc_capsule_bytes.argtypes = [vp, i, i]; lib.kvc_capsule_bytes.restype = C.c_size_t
         lib.kvc_workspace_bytes.argtypes = [vp, i, i, i]; lib.kvc_workspace_bytes.restype = C.c_size_t
         lib.kvc_compress.argtypes = [vp, vp, vp, i, i, vp, vp]; lib.kvc_compress.restype = i
@@ -100,7 +105,7 @@ class Layer:
     """Owns one kvc_layer handle and keeps the borrowed parameter tensors alive."""
 
     def __init__(self, H_q: int, H_kv: int, d: int, n: int, ratio_permille: int, dtype: torch.dtype,
-                 idx=None, theta=None, U=None, mu=None, layer: int = 0):
+                 idx=None, theta=None, U=None, mu=None, layer: int = 0, mode: int = KVC_MODE_KV):
         if dtype not in _DTYPES:
             raise KvcError(-3, "kvc_layer_create") if _LIB else ValueError("unsupported dtype")
         self.H_q, self.H_kv, self.d, self.n, self.dtype = H_q, H_kv, d, n, dtype
@@ -109,6 +114,7 @@ class Layer:
         desc = kvc_layer_desc()
         desc.layer, desc.H_q, desc.H_kv, desc.d, desc.n = layer, H_q, H_kv, d, n
         desc.ratio_permille, desc.dtype = ratio_permille, _DTYPES[dtype]
+        desc.mode = mode
         idx_host = None
         if idx is not None:
             idx_host = idx.detach().to("cpu", torch.int32).contiguous()
@@ -122,6 +128,9 @@ class Layer:
         _check(_lib().kvc_layer_create(C.byref(desc), C.byref(h)), "kvc_layer_create")
         self.handle = h
         self.m = _lib().kvc_layer_m(h)
+        mk, mv = C.c_int(), C.c_int()
+        _check(_lib().kvc_layer_rows(h, C.byref(mk), C.byref(mv)), "kvc_layer_rows")
+        self.m_k, self.m_v = mk.value, mv.value
 
     def close(self):
         if getattr(self, "handle", None) and _LIB is not None:      # at interpreter exit the library may be gone already
@@ -220,10 +229,11 @@ def kvc_export_maps(layer: Layer, R: int):
 
 
 def capsule_views(layer: Layer, capsules, B: int, R: int):
-    """(K_tilde, V_tilde) [B,H_kv,R,m,d] typed views of a capsule store (no copy)."""
-    half = kvc_capsule_bytes(layer, B, R) // 2
-    shape = (B, layer.H_kv, R, layer.m, layer.d)
-    return (capsules[:half].view(layer.dtype).view(shape), capsules[half:2 * half].view(layer.dtype).view(shape))
+    """(K_tilde [B,H_kv,R,m_k,d], V_tilde [B,H_kv,R,m_v,d]) typed views of a capsule store (no copy)."""
+    total = kvc_capsule_bytes(layer, B, R)
+    kb = total // (layer.m_k + layer.m_v) * layer.m_k
+    return (capsules[:kb].view(layer.dtype).view(B, layer.H_kv, R, layer.m_k, layer.d),
+            capsules[kb:total].view(layer.dtype).view(B, layer.H_kv, R, layer.m_v, layer.d))
 
 
 KVC_KERNEL_COUNT = 13

@@ -16,10 +16,11 @@ static size_t elem_bytes(int dtype) { return dtype == KVC_BF16 ? 2 : 4; }
 
 WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap) {
   WsLayout w{};
-  const int H_kv = L->desc.H_kv, G = L->G, n = L->desc.n, ms = L->ms;
+  const int H_kv = L->desc.H_kv, G = L->G, n = L->desc.n;
+  const int ms = (L->mk + 15) / 16 * 16, msv = (L->mv + 15) / 16 * 16;
   const int rows_h = B * G * R;
   // tensor-core expansion: bf16 storage and 16-byte aligned rows of theta / U
-  w.use_mma = (!L->passthrough && L->desc.dtype == KVC_BF16 && n % 8 == 0) ? 1 : 0;
+  w.use_mma = (!L->passthrough && L->mode == KVC_MODE_KV && L->desc.dtype == KVC_BF16 && n % 8 == 0) ? 1 : 0;
   w.CG = 1;
   w.cgw = ms;
   int row_tiles;
@@ -42,7 +43,7 @@ WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap) {
     w.IR = (int)align_up((size_t)ceil_div(n, ns), EXP_IC);
     w.NS = ceil_div(n, w.IR);
   }
-  w.cpb = ceil_div(L->m, OUT_CHUNK);
+  w.cpb = ceil_div(L->mv, OUT_CHUNK);
   w.ct = ceil_div(T_cap, OUT_CHUNK);
   w.chunks_per_bh = R * w.cpb + w.ct;
   w.GT = G == 1 ? 1 : (G == 2 ? 2 : (G <= 4 ? 4 : 8));
@@ -69,9 +70,9 @@ WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap) {
   w.off_cnt = take(sizeof(int) * ((size_t)B * H_kv + 1));
   w.off_S = take((w.use_mma ? sizeof(__nv_bfloat16) : sizeof(float)) * (size_t)H_kv * rows_h * ms);
   w.off_stxt = take(sizeof(float) * (size_t)B * H_kv * G * w.Ts);
-  w.off_W = take(sizeof(float) * (size_t)w.NS * H_kv * rows_h * ms);
+  w.off_W = take(sizeof(float) * (size_t)w.NS * H_kv * rows_h * msv);
   w.off_wstat = take(sizeof(float2) * (size_t)w.NS * H_kv * rows_h);
-  w.off_Wc = take(sizeof(float) * (size_t)H_kv * rows_h * ms);
+  w.off_Wc = take(sizeof(float) * (size_t)H_kv * rows_h * msv);
   w.off_statc = take(sizeof(float4) * (size_t)H_kv * rows_h);
   w.off_ypart = take(sizeof(float) * (size_t)B * H_kv * G * w.nsplit * D);
   w.off_ystat = take(sizeof(float2) * (size_t)B * H_kv * G * w.nsplit);
@@ -81,7 +82,7 @@ WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap) {
     size_t np = 0;
     if (B > 0 && R > 0) {
       const FusedPlan fp = plan_fused(L, B, R);
-      if (fp.ok && fp.nrg > 1) np = (size_t)B * H_kv * fp.nrg * G;
+      if (fp.ok && L->mode == KVC_MODE_KV && fp.nrg > 1) np = (size_t)B * H_kv * fp.nrg * G;
     }
     if ((R == 0 || L->passthrough) && B > 0 && R * n + T_cap > 0 && plan_fused_text(L, B, R * n + T_cap).ok) {
       const size_t np_plain = (size_t)B * H_kv * 16 * G;
@@ -95,7 +96,7 @@ WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap) {
     size_t sb = 0;
     if (B > 0 && R > 0) {
       const SplitPlan sp = plan_split(L, B, R);
-      if (sp.ok) sb = split_ws(L, sp, B, R, T_cap).bytes;
+      if (sp.ok && L->mode == KVC_MODE_KV) sb = split_ws(L, sp, B, R, T_cap).bytes;
     }
     w.off_split = take(sb);
   }
@@ -166,12 +167,15 @@ int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out) {
   const int m = kvc_retained_len(desc->n, desc->ratio_permille);
   if (m < 1) return KVC_ERR_SHAPE;
   const bool pass = desc->ratio_permille == 0;
-  if (!pass && (!desc->idx || !desc->theta || !desc->U || !desc->mu)) return KVC_ERR_NO_PARAMS;
+  const int mode = pass ? KVC_MODE_KV : desc->mode;
+  if (mode != KVC_MODE_KV && mode != KVC_MODE_K_ONLY && mode != KVC_MODE_V_ONLY) return KVC_ERR_ARG;
+  const bool key_side = mode != KVC_MODE_V_ONLY, value_side = mode != KVC_MODE_K_ONLY;   // sides that are compressed
+  if (!pass && ((key_side && (!desc->idx || !desc->theta)) || (value_side && (!desc->U || !desc->mu)))) return KVC_ERR_NO_PARAMS;
 
   std::vector<int32_t> idx((size_t)desc->H_kv * m);
   for (int h = 0; h < desc->H_kv; ++h)
     for (int j = 0; j < m; ++j) {
-      const int32_t v = pass ? j : desc->idx[(desc->idx_per_head ? (size_t)h * m : 0) + j];
+      const int32_t v = (pass || !key_side) ? j : desc->idx[(desc->idx_per_head ? (size_t)h * m : 0) + j];
       if (v < 0 || v >= desc->n || (j > 0 && v <= idx[(size_t)h * m + j - 1])) return KVC_ERR_BOUNDS;
       idx[(size_t)h * m + j] = v;
     }
@@ -184,6 +188,9 @@ int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out) {
   L->ms = (m + 15) / 16 * 16;
   L->G = desc->H_q / desc->H_kv;
   L->passthrough = pass ? 1 : 0;
+  L->mode = mode;
+  L->mk = key_side ? m : desc->n;
+  L->mv = value_side ? m : desc->n;
   L->d_idx = nullptr;
   L->d_cstatus = nullptr;
   L->d_usum = nullptr;
@@ -199,7 +206,7 @@ int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out) {
       cudaMemcpy(L->d_idx, idx.data(), idx.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMalloc(&L->d_cstatus, sizeof(int)) != cudaSuccess ||
       cudaMemset(L->d_cstatus, 0, sizeof(int)) != cudaSuccess ||
-      (!pass && (cudaMalloc(&L->d_usum, idx.size() * sizeof(float)) != cudaSuccess ||
+      (!pass && value_side && (cudaMalloc(&L->d_usum, idx.size() * sizeof(float)) != cudaSuccess ||
                  compute_usum(L, L->d_usum) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess))) {
     if (L->d_idx) cudaFree(L->d_idx);
     if (L->d_cstatus) cudaFree(L->d_cstatus);
@@ -225,9 +232,21 @@ int kvc_layer_destroy(kvc_layer* L) {
 
 int kvc_layer_m(const kvc_layer* L) { return L ? L->m : -1; }
 
+int kvc_layer_rows(const kvc_layer* L, int* key_rows, int* value_rows) {
+  if (!L) return KVC_ERR_ARG;
+  if (key_rows) *key_rows = L->mk;
+  if (value_rows) *value_rows = L->mv;
+  return KVC_OK;
+}
+
+// bytes of the key part of a capsule store (the value part follows it)
+static size_t key_part_bytes(const kvc_layer* L, int B, int R) {
+  return (size_t)B * L->desc.H_kv * R * L->mk * D * elem_bytes(L->desc.dtype);
+}
+
 size_t kvc_capsule_bytes(const kvc_layer* L, int B, int R) {
   if (!L || B < 0 || R < 0) return 0;
-  return (size_t)2 * B * L->desc.H_kv * R * L->m * D * elem_bytes(L->desc.dtype);
+  return (size_t)B * L->desc.H_kv * R * ((size_t)L->mk + L->mv) * D * elem_bytes(L->desc.dtype);
 }
 
 size_t kvc_workspace_bytes(const kvc_layer* L, int B, int R, int T_cap) {
@@ -241,17 +260,17 @@ int kvc_compress(const kvc_layer* L, const void* K_vis, const void* V_vis, int B
   if (B == 0 || R == 0) return KVC_OK;
   if (!K_vis || !V_vis || !capsules) return KVC_ERR_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const size_t half = kvc_capsule_bytes(L, B, R) / 2;
+  const size_t kbytes = key_part_bytes(L, B, R), vbytes = kvc_capsule_bytes(L, B, R) - kbytes;
   void* Kc = capsules;
-  void* Vc = static_cast<char*>(capsules) + half;
+  void* Vc = static_cast<char*>(capsules) + kbytes;
   cudaError_t e = cudaMemsetAsync(L->d_cstatus, 0, sizeof(int), st);   // status word of this compress call
   if (e != cudaSuccess) return cuda_status(e);
-  if (L->passthrough) {
-    e = cudaMemcpyAsync(Kc, K_vis, half, cudaMemcpyDeviceToDevice, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(Vc, V_vis, half, cudaMemcpyDeviceToDevice, st);
-  } else {
-    e = launch_compress(L, K_vis, V_vis, B, R, Kc, Vc, st);
-  }
+  // a side kept verbatim (rho = 0, or the one-sided modes) is a plain copy of its n rows per block
+  if (L->passthrough || L->mode == KVC_MODE_V_ONLY) e = cudaMemcpyAsync(Kc, K_vis, kbytes, cudaMemcpyDeviceToDevice, st);
+  else e = launch_compress_keys(L, K_vis, B, R, Kc, st);
+  if (e != cudaSuccess) return cuda_status(e);
+  if (L->passthrough || L->mode == KVC_MODE_K_ONLY) e = cudaMemcpyAsync(Vc, V_vis, vbytes, cudaMemcpyDeviceToDevice, st);
+  else e = launch_compress_values(L, V_vis, B, R, Vc, st);
   return cuda_status(e);
 }
 
@@ -291,14 +310,15 @@ int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B
   DecodeArgs a{};
   a.ws = ws_layout(L, B, R, T);
   char* ws = static_cast<char*>(workspace);
-  const size_t half = kvc_capsule_bytes(L, B, R) / 2;
   a.q = q;
   a.Kc = capsules;
-  a.Vc = capsules ? static_cast<const char*>(capsules) + half : nullptr;
+  a.Vc = capsules ? static_cast<const char*>(capsules) + key_part_bytes(L, B, R) : nullptr;
   a.K_txt = K_txt; a.V_txt = V_txt;
   a.theta = L->desc.theta; a.U = L->desc.U; a.mu = L->desc.mu;
   a.out = out;
-  a.B = B; a.H_kv = L->desc.H_kv; a.G = L->G; a.R = R; a.m = L->m; a.ms = L->ms; a.n = L->desc.n;
+  a.B = B; a.H_kv = L->desc.H_kv; a.G = L->G; a.R = R; a.m = L->mk; a.ms = (L->mk + 15) / 16 * 16; a.n = L->desc.n;
+  a.mv = L->mv; a.msv = (L->mv + 15) / 16 * 16;
+  a.id_theta = L->mode == KVC_MODE_V_ONLY; a.id_U = L->mode == KVC_MODE_K_ONLY;
   a.T = T; a.T_cap = T_cap > 0 ? T_cap : 1; a.Ts = a.ws.Ts;
   a.passthrough = L->passthrough;
   a.S = reinterpret_cast<float*>(ws + a.ws.off_S);
@@ -323,16 +343,18 @@ int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B
     // R == 0 (text rows only, the uncompressed comparator): the same kernel with text stages only
     // rho = 0 stores K and V verbatim: vision rows and text rows are attended as plain rows by the text-only mode
     const bool plain = R == 0 || L->passthrough;
+    const bool one_sided = R > 0 && L->mode != KVC_MODE_KV;      // served by the three-phase kernels below
     const uintptr_t align = reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(capsules) |
                             reinterpret_cast<uintptr_t>(out) | (T > 0 ? reinterpret_cast<uintptr_t>(K_txt) |
                             reinterpret_cast<uintptr_t>(V_txt) : 0) | reinterpret_cast<uintptr_t>(L->desc.mu);
-    if (!plain && (align & 15) == 0 && T <= 64 * SP_OUT_ROWS * SP_TEXT_CHUNK && use_split(L, B, R)) {
+    if (!plain && !one_sided && (align & 15) == 0 && T <= 64 * SP_OUT_ROWS * SP_TEXT_CHUNK && use_split(L, B, R)) {
       const SplitPlan sp = plan_split(L, B, R);
       bool encoded = false;
       const cudaError_t se = launch_split(L, a, sp, st, &encoded);
       if (encoded) return cuda_status(se);
     }
-    const FusedPlan fp = plain ? plan_fused_text(L, B, R * L->desc.n + T) : plan_fused(L, B, R);
+    FusedPlan fp = plain ? plan_fused_text(L, B, R * L->desc.n + T) : plan_fused(L, B, R);
+    if (one_sided) fp.ok = 0;
     if (fp.ok && (align & 15) == 0) {
       bool encoded = false;
       const cudaError_t fe = launch_fused(L, a, fp, st, &encoded);

@@ -88,20 +88,21 @@ __global__ void __launch_bounds__(256) project_values_kernel(const T* __restrict
 }
 
 template <typename T>
-static cudaError_t launch_compress_t(const kvc_layer* L, const void* K_vis, const void* V_vis, int B, int R,
-                                     void* Kc, void* Vc, cudaStream_t st) {
+static cudaError_t launch_keys_t(const kvc_layer* L, const void* K_vis, int B, int R, void* Kc, cudaStream_t st) {
   constexpr int RPI = 32 / (D / Elems16<T>::N);
   const int H_kv = L->desc.H_kv, n = L->desc.n, m = L->m;
   const long long total_rows = (long long)B * H_kv * R * m;
   const long long warps = (total_rows + RPI - 1) / RPI;
+  ProfScope prof(KVC_KERNEL_GATHER_KEYS, st);
+  gather_keys_kernel<T><<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(
+      static_cast<const T*>(K_vis), static_cast<T*>(Kc), L->d_idx, H_kv, R, n, m, total_rows);
+  return cudaGetLastError();
+}
+
+template <typename T>
+static cudaError_t launch_values_t(const kvc_layer* L, const void* V_vis, int B, int R, void* Vc, cudaStream_t st) {
+  const int H_kv = L->desc.H_kv, n = L->desc.n, m = L->m;
   cudaError_t e;
-  {
-    ProfScope prof(KVC_KERNEL_GATHER_KEYS, st);
-    gather_keys_kernel<T><<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(
-        static_cast<const T*>(K_vis), static_cast<T*>(Kc), L->d_idx, H_kv, R, n, m, total_rows);
-    e = cudaGetLastError();
-  }
-  if (e != cudaSuccess) return e;
   ProfScope prof(KVC_KERNEL_PROJECT_VALUES, st);
   {
     bool used = false;
@@ -117,10 +118,13 @@ static cudaError_t launch_compress_t(const kvc_layer* L, const void* K_vis, cons
   return cudaGetLastError();
 }
 
-cudaError_t launch_compress(const kvc_layer* L, const void* K_vis, const void* V_vis, int B, int R, void* Kc,
-                            void* Vc, cudaStream_t st) {
-  return L->desc.dtype == KVC_BF16 ? launch_compress_t<__nv_bfloat16>(L, K_vis, V_vis, B, R, Kc, Vc, st)
-                                   : launch_compress_t<float>(L, K_vis, V_vis, B, R, Kc, Vc, st);
+cudaError_t launch_compress_keys(const kvc_layer* L, const void* K_vis, int B, int R, void* Kc, cudaStream_t st) {
+  return L->desc.dtype == KVC_BF16 ? launch_keys_t<__nv_bfloat16>(L, K_vis, B, R, Kc, st)
+                                   : launch_keys_t<float>(L, K_vis, B, R, Kc, st);
+}
+cudaError_t launch_compress_values(const kvc_layer* L, const void* V_vis, int B, int R, void* Vc, cudaStream_t st) {
+  return L->desc.dtype == KVC_BF16 ? launch_values_t<__nv_bfloat16>(L, V_vis, B, R, Vc, st)
+                                   : launch_values_t<float>(L, V_vis, B, R, Vc, st);
 }
 
 }  // namespace kvc

@@ -5,7 +5,10 @@
 // several CTAs, each emitting an unnormalised partial (W, max, sum).
 //
 // This translation unit holds the CUDA-core fp32 version, used for fp32 storage (1e-4 parity) and
-// as the fallback shape-agnostic path.
+// as the fallback shape-agnostic path.  It also serves the one-sided variants (App. G): with verbatim
+// keys the score row already has n entries and the expansion is the identity (id_theta); with verbatim
+// values the weight row has n entries and equals P (id_U).  The score row has a.m entries (pitch a.ms),
+// the weight row a.mv entries (pitch a.msv).
 #include "kvc_async.cuh"
 #include "kvc_internal.cuh"
 
@@ -14,10 +17,10 @@ namespace kvc {
 template <typename T>
 __global__ void __launch_bounds__(256) expand_kernel(DecodeArgs a) {
   extern __shared__ __align__(16) float smem[];
-  const int ms = a.ms, m = a.m, n = a.n;
+  const int ms = a.ms, m = a.m, n = a.n, msv = a.msv, mv = a.mv;
   float* Ssm = smem;                          // [EXP_ROWS][ms]
-  float* Wacc = Ssm + EXP_ROWS * ms;          // [EXP_ROWS][ms]
-  float* Lsm = Wacc + EXP_ROWS * ms;          // [EXP_ROWS][EXP_IC]
+  float* Wacc = Ssm + EXP_ROWS * ms;          // [EXP_ROWS][msv]
+  float* Lsm = Wacc + EXP_ROWS * msv;         // [EXP_ROWS][EXP_IC]
   float* Usm = Lsm + EXP_ROWS * EXP_IC;       // [64][EXP_IC + 1]
   float* rowmax = Usm + 64 * (EXP_IC + 1);    // [EXP_ROWS]
   float* rowsum = rowmax + EXP_ROWS;
@@ -29,14 +32,14 @@ __global__ void __launch_bounds__(256) expand_kernel(DecodeArgs a) {
   const int i_begin = split * a.ws.IR, i_end = min(n, i_begin + a.ws.IR);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const T* theta = static_cast<const T*>(a.theta) + (size_t)h * m * n;
-  const T* U = static_cast<const T*>(a.U) + (size_t)h * m * n;
+  const T* U = static_cast<const T*>(a.U) + (size_t)h * mv * n;
   const float* S = a.S + (size_t)h * nrows_h * ms;
 
   for (int x = tid; x < EXP_ROWS * ms; x += 256) {
     const int r = x / ms, j = x - r * ms;
     Ssm[x] = (row0 + r < nrows_h && j < m) ? S[(size_t)(row0 + r) * ms + j] : 0.f;
-    Wacc[x] = 0.f;
   }
+  for (int x = tid; x < EXP_ROWS * msv; x += 256) Wacc[x] = 0.f;
   if (tid < EXP_ROWS) { rowmax[tid] = -INFINITY; rowsum[tid] = 0.f; }
   __syncthreads();
 
@@ -46,7 +49,10 @@ __global__ void __launch_bounds__(256) expand_kernel(DecodeArgs a) {
     {
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
       const bool ok = i0 + ii < i_end;
-      if (ok) {
+      if (ok && a.id_theta) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) acc[k] = Ssm[(rg * 4 + k) * ms + i0 + ii];
+      } else if (ok) {
         const T* tp = theta + i0 + ii;
         for (int j = 0; j < m; ++j) {
           const float t = to_f32(tp[(size_t)j * n]);
@@ -81,11 +87,23 @@ __global__ void __launch_bounds__(256) expand_kernel(DecodeArgs a) {
       }
     }
     __syncthreads();
+    if (a.id_U) {
+      // W = P: the columns of this CTA's range written so far follow the running maximum, the chunk's columns are P
+      for (int x = tid; x < EXP_ROWS * (i0 - i_begin); x += 256) {
+        const int r = x / (i0 - i_begin), j = i_begin + (x - r * (i0 - i_begin));
+        Wacc[r * msv + j] *= rowscale[r];
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (i0 + ii < i_end) Wacc[(rg * 4 + k) * msv + i0 + ii] = Lsm[(rg * 4 + k) * EXP_IC + ii];
+      __syncthreads();
+      continue;
+    }
     // ---- W[:, j] = W[:, j] * scale + P . U[j, i0:i0+IC]^T, 64 rows of U at a time
-    for (int j0 = 0; j0 < m; j0 += 64) {
+    for (int j0 = 0; j0 < mv; j0 += 64) {
       for (int x = tid; x < 64 * EXP_IC; x += 256) {
         const int jj = x >> 6, i2 = x & 63;
-        const bool ok = (j0 + jj < m) && (i0 + i2 < i_end);
+        const bool ok = (j0 + jj < mv) && (i0 + i2 < i_end);
         Usm[jj * (EXP_IC + 1) + i2] = ok ? to_f32(U[(size_t)(j0 + jj) * n + i0 + i2]) : 0.f;
       }
       __syncthreads();
@@ -97,11 +115,11 @@ __global__ void __launch_bounds__(256) expand_kernel(DecodeArgs a) {
 #pragma unroll
           for (int k = 0; k < 4; ++k) acc[k] = fmaf(Lsm[(rg * 4 + k) * EXP_IC + i2], u, acc[k]);
         }
-        if (j0 + jj < m) {
+        if (j0 + jj < mv) {
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
             const int r = rg * 4 + k;
-            Wacc[r * ms + j0 + jj] = Wacc[r * ms + j0 + jj] * rowscale[r] + acc[k];
+            Wacc[r * msv + j0 + jj] = Wacc[r * msv + j0 + jj] * rowscale[r] + acc[k];
           }
         }
       }
@@ -109,10 +127,10 @@ __global__ void __launch_bounds__(256) expand_kernel(DecodeArgs a) {
     }
   }
 
-  float* Wout = a.W + ((size_t)split * a.H_kv + h) * nrows_h * ms;
-  for (int x = tid; x < EXP_ROWS * ms; x += 256) {
-    const int r = x / ms;
-    if (row0 + r < nrows_h) Wout[(size_t)(row0 + r) * ms + (x - r * ms)] = Wacc[x];
+  float* Wout = a.W + ((size_t)split * a.H_kv + h) * nrows_h * msv;
+  for (int x = tid; x < EXP_ROWS * msv; x += 256) {
+    const int r = x / msv;
+    if (row0 + r < nrows_h) Wout[(size_t)(row0 + r) * msv + (x - r * msv)] = Wacc[x];
   }
   if (tid < EXP_ROWS && row0 + tid < nrows_h)
     a.wstat[((size_t)split * a.H_kv + h) * nrows_h + row0 + tid] = make_float2(rowmax[tid], rowsum[tid]);
@@ -164,10 +182,10 @@ __global__ void __launch_bounds__(256) combine_kernel(DecodeArgs a) {
   float sc[MAX_NS];
 #pragma unroll
   for (int s = 0; s < MAX_NS; ++s) sc[s] = __shfl_sync(0xffffffffu, my_sc, s);
-  const size_t sstride = (size_t)nrows * a.ms;
-  const float* wp = a.W + (size_t)row * a.ms;
-  float* wo = a.Wcomb + (size_t)row * a.ms;
-  for (int j = lane; j < a.ms; j += 32) {
+  const size_t sstride = (size_t)nrows * a.msv;
+  const float* wp = a.W + (size_t)row * a.msv;
+  float* wo = a.Wcomb + (size_t)row * a.msv;
+  for (int j = lane; j < a.msv; j += 32) {
     float v[MAX_NS];
 #pragma unroll
     for (int s = 0; s < MAX_NS; ++s) v[s] = s < NS ? __ldcg(wp + s * sstride + j) : 0.f;
@@ -179,14 +197,14 @@ __global__ void __launch_bounds__(256) combine_kernel(DecodeArgs a) {
   if (lane == 0) a.statc[row] = make_float4(mx, sum, 0.f, 0.f);
 }
 
-static size_t expand_smem_bytes(int ms) {
-  return sizeof(float) * ((size_t)2 * EXP_ROWS * ms + EXP_ROWS * EXP_IC + 64 * (EXP_IC + 1) + 3 * EXP_ROWS);
+static size_t expand_smem_bytes(int ms, int msv) {
+  return sizeof(float) * ((size_t)EXP_ROWS * (ms + msv) + EXP_ROWS * EXP_IC + 64 * (EXP_IC + 1) + 3 * EXP_ROWS);
 }
 
 template <typename T>
 static cudaError_t launch_expand_t(const DecodeArgs& a, cudaStream_t st) {
-  const size_t smem = expand_smem_bytes(a.ms);
-  cudaError_t e = cudaFuncSetAttribute(expand_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const size_t smem = expand_smem_bytes(a.ms, a.msv);
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(expand_kernel<T>), smem);
   if (e != cudaSuccess) return e;
   dim3 grid(a.ws.NS, ceil_div(a.B * a.G * a.R, EXP_ROWS), a.H_kv);
   expand_kernel<T><<<grid, 256, smem, st>>>(a);

@@ -61,9 +61,9 @@ struct WsLayout {
   int Ts;          // row stride of the text logits (T rounded up to a multiple of 4)
   size_t off_S;    // fp32 or bf16 [H_kv][B][G][R][ms]   compressed scores, sigma applied
   size_t off_stxt; // fp32 [B][H_kv][G][T]       text logits
-  size_t off_W;    // fp32 [NS][H_kv][B*G*R][ms] unnormalised P U^T per split
+  size_t off_W;    // fp32 [NS][H_kv][B*G*R][msv] unnormalised P U^T per split (msv: pitch of a weight row)
   size_t off_wstat;// float2 [NS][H_kv][B*G*R]   (max, sum) per row and split
-  size_t off_Wc;   // fp32 [H_kv][B*G*R][ms]     the splits combined, relative to one maximum per row
+  size_t off_Wc;   // fp32 [H_kv][B*G*R][msv]    the splits combined, relative to one maximum per row
   size_t off_statc;// float4 [H_kv][B*G*R]       (max, sum, 0, 0) of the combined row
   size_t off_ypart;// fp32 [B][H_kv][G][nsplit][D]
   size_t off_ystat;// float2 [B][H_kv][G][nsplit]
@@ -108,6 +108,8 @@ struct kvc_layer {
   kvc_layer_desc desc;   // idx pointer cleared after the copy
   int m;                 // retained length
   int ms;                // row stride of score buffers (m rounded up to 16)
+  int mode;              // KVC_MODE_KV, or one side kept verbatim (App. G): KVC_MODE_K_ONLY, KVC_MODE_V_ONLY
+  int mk, mv;            // stored rows per block on the key side (n in the V-only mode) and on the value side (n in the K-only mode)
   int G;
   int passthrough;       // ratio_permille == 0
   int device;
@@ -139,9 +141,11 @@ struct DecodeArgs {
   const void* U;
   const void* mu;
   void* out;
-  int B, H_kv, G, R, m, ms, n, T, T_cap;
+  int B, H_kv, G, R, m, ms, n, T, T_cap;   // m, ms: key rows per block = length of a compressed score row, and its pitch
+  int mv, msv;         // value rows per block = length of a weight row, and its pitch (= m, ms unless one side is verbatim)
   int Ts;              // row stride of s_txt
   int passthrough;
+  int id_theta, id_U;  // the score expansion / the re-projection is the identity (verbatim keys / verbatim values)
   float* S;            // fp32 scores (CUDA-core expansion)
   __nv_bfloat16* Sb;   // bf16 scores (tensor-core expansion); exactly one of S / Sb is used
   float* s_txt;
@@ -216,7 +220,7 @@ void map_cache_destroy(kvc_map_cache* c);
 cudaError_t compute_usum(const kvc_layer* L, float* usum);
 cudaError_t launch_project_values_tc(const kvc_layer* L, const void* V_vis, int B, int R, void* Vc, cudaStream_t st, bool* used);
 cudaError_t launch_project_values_mma(const kvc_layer* L, const void* V_vis, int B, int R, void* Vc, cudaStream_t st, bool* used);
-cudaError_t launch_compress(const kvc_layer* L, const void* K_vis, const void* V_vis, int B, int R,
-                            void* Kc, void* Vc, cudaStream_t st);
+cudaError_t launch_compress_keys(const kvc_layer* L, const void* K_vis, int B, int R, void* Kc, cudaStream_t st);
+cudaError_t launch_compress_values(const kvc_layer* L, const void* V_vis, int B, int R, void* Vc, cudaStream_t st);
 
 }  // namespace kvc

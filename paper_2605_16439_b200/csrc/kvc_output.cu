@@ -44,7 +44,7 @@ __device__ __forceinline__ ChunkRef chunk_ref(const DecodeArgs& a, int q) {
   } else {
     c.r = lc / a.ws.cpb;
     c.j0 = (lc - c.r * a.ws.cpb) * OUT_CHUNK;
-    c.rows = min(OUT_CHUNK, a.m - c.j0);
+    c.rows = min(OUT_CHUNK, a.mv - c.j0);
   }
   return c;
 }
@@ -104,7 +104,7 @@ __global__ void __launch_bounds__(OUT_THREADS) output_kernel(DecodeArgs a, int g
           mbar_expect_tx(&full_bar[stage], data_bytes + gcount * wbytes +
                                                (c.is_txt ? 0u : (uint32_t)gcount * (uint32_t)sizeof(float4)));
           const T* src = c.is_txt ? static_cast<const T*>(a.V_txt) + ((size_t)c.bh * a.T_cap + c.j0) * D
-                                  : static_cast<const T*>(a.Vc) + (((size_t)c.bh * a.R + c.r) * a.m + c.j0) * D;
+                                  : static_cast<const T*>(a.Vc) + (((size_t)c.bh * a.R + c.r) * a.mv + c.j0) * D;
           bulk_g2s(sbase, src, data_bytes, &full_bar[stage]);
         }
         if (weights) {
@@ -116,7 +116,7 @@ __global__ void __launch_bounds__(OUT_THREADS) output_kernel(DecodeArgs a, int g
                        &full_bar[stage]);
             } else {
               const size_t row_id = (size_t)c.h * nrows_h + (size_t)(c.b * a.G + g_base + g) * a.R + c.r;
-              bulk_g2s(wdst + g * OUT_CHUNK, a.Wcomb + row_id * a.ms + c.j0, wbytes, &full_bar[stage]);
+              bulk_g2s(wdst + g * OUT_CHUNK, a.Wcomb + row_id * a.msv + c.j0, wbytes, &full_bar[stage]);
               bulk_g2s(sdst + g, a.statc + row_id, (uint32_t)sizeof(float4), &full_bar[stage]);
             }
           }
@@ -253,7 +253,7 @@ __global__ void __launch_bounds__(OUT_THREADS) output_kernel(DecodeArgs a, int g
           float ms_g = 0.f;
 #pragma unroll
           for (int k = 0; k < GT; ++k) if (k == g) ms_g = mu_sum[k];
-          if (!a.passthrough) y = fmaf(ms_g, to_f32(static_cast<const T*>(a.mu)[c.h * D + col]), y);
+          if (!a.passthrough && !a.id_U) y = fmaf(ms_g, to_f32(static_cast<const T*>(a.mu)[c.h * D + col]), y);
           a.ypart[(((size_t)c.bh * a.G + g_base + g) * a.ws.nsplit + slot) * D + col] = y;
         }
       }

@@ -54,29 +54,35 @@ def make_problem(shape: wl.Shape, seed: int, T=None, T_cap=None, idx=None, recip
     return p
 
 
-def oracle_run(shape: wl.Shape, p, form: str = "fused"):
+MODES = {"kv": kvc.KVC_MODE_KV, "k": kvc.KVC_MODE_K_ONLY, "v": kvc.KVC_MODE_V_ONLY}
+
+
+def oracle_run(shape: wl.Shape, p, form: str = "fused", mode: str = "kv"):
     """(K_tilde, V_tilde, out) in fp64 from the (already rounded) storage-dtype inputs."""
     passthrough = shape.ratio_permille == 0
     T = p["T"]
     args = [np64(p[k]) for k in ("K_vis", "V_vis")]
-    K_t, V_t = orc.compress(args[0], args[1], p["idx"].numpy(), np64(p["U"]), np64(p["mu"]), shape.n, passthrough)
+    K_t, V_t = orc.compress(args[0], args[1], p["idx"].numpy(), np64(p["U"]), np64(p["mu"]), shape.n, passthrough, mode)
     f = orc.decode_attend_fused if form == "fused" else orc.decode_attend_definition
     out = f(np64(p["q"]), K_t, V_t, np64(p["theta"]), np64(p["U"]), np64(p["mu"]),
-            np64(p["K_txt"])[:, :, :T], np64(p["V_txt"])[:, :, :T], passthrough)
+            np64(p["K_txt"])[:, :, :T], np64(p["V_txt"])[:, :, :T], passthrough, mode)
     return K_t, V_t, out
 
 
-def gpu_layer(shape: wl.Shape, p, dev="cuda"):
+def gpu_layer(shape: wl.Shape, p, dev="cuda", mode: str = "kv"):
     dt = wl.torch_dtype(shape.dtype)
     if shape.ratio_permille == 0:
         return kvc.Layer(shape.H_q, shape.H_kv, shape.d, shape.n, 0, dt)
-    return kvc.Layer(shape.H_q, shape.H_kv, shape.d, shape.n, shape.ratio_permille, dt, idx=p["idx"],
-                     theta=p["theta"].to(dev), U=p["U"].to(dev), mu=p["mu"].to(dev))
+    # a one-sided mode gets only the parameters of the side it compresses
+    return kvc.Layer(shape.H_q, shape.H_kv, shape.d, shape.n, shape.ratio_permille, dt,
+                     idx=p["idx"] if mode != "v" else None, theta=p["theta"].to(dev) if mode != "v" else None,
+                     U=p["U"].to(dev) if mode != "k" else None, mu=p["mu"].to(dev) if mode != "k" else None,
+                     mode=MODES[mode])
 
 
-def gpu_run(shape: wl.Shape, p, dev="cuda"):
+def gpu_run(shape: wl.Shape, p, dev="cuda", mode: str = "kv"):
     """(K_tilde, V_tilde, out) from the CUDA library through the C ABI."""
-    layer = gpu_layer(shape, p, dev)
+    layer = gpu_layer(shape, p, dev, mode)
     B, R, T, T_cap = shape.B, shape.R, p["T"], p["T_cap"]
     caps = kvc.alloc_capsules(layer, B, R, dev)
     kvc.kvc_compress(layer, p["K_vis"].to(dev), p["V_vis"].to(dev), B, R, caps)

@@ -39,12 +39,14 @@ def _log_error(shape, err, out_max, v_err=None, v_max=None):
                                 "out_max": out_max, "v_err": v_err, "v_max": v_max}) + "\n")
 
 
-def _check(shape, p, form="fused"):
+def _check(shape, p, form="fused", mode="kv"):
     tol = tl.TOL[shape.dtype]
-    K_o, V_o, out_o = tl.oracle_run(shape, p, form)
-    layer, K_g, V_g, out_g = tl.gpu_run(shape, p)
+    K_o, V_o, out_o = tl.oracle_run(shape, p, form, mode)
+    layer, K_g, V_g, out_g = tl.gpu_run(shape, p, mode=mode)
     v_err = v_max = None
-    if shape.R > 0:
+    if shape.R > 0 and mode == "k":
+        assert np.array_equal(tl.np64(K_g), K_o) and np.array_equal(tl.np64(V_g), V_o)    # both sides are copies of rows
+    elif shape.R > 0:
         # key capsules are copies of input rows: bit-exact
         assert np.array_equal(tl.np64(K_g), K_o)
         # value capsules: fp32 accumulation over n terms, then one rounding to the storage type (bf16: half an ulp of
@@ -97,6 +99,49 @@ def test_sharp_recipes_through_every_kernel_variant(ci, kw, recipe, variant, mon
         assert counts["split_scores"] == counts["split_expand"] == counts["split_output"] == 1 and counts["fused"] == 0
     else:
         assert counts["fused"] + counts["fused_tc"] + counts["fused_pair"] == 1
+
+
+@pytest.mark.parametrize("mode", ["k", "v"])
+@pytest.mark.parametrize("recipe", ["peaked", "structured"])
+@pytest.mark.parametrize("ci,kw", tl.REDUCED_7B + [(0, dict(B=2, H_q=4, H_kv=2, R=2))])
+def test_one_sided_modes(ci, kw, recipe, mode):
+    """App. G: only the keys (mode k) or only the values (mode v) compressed, the other side stored verbatim; the
+    capsule store has n rows per block on the verbatim side, and the side's parameters are not even passed."""
+    shape = tl.small(wl.CONFIGS[ci], **kw)
+    p = tl.make_problem(shape, wl.layer_seed(ci, 17), T=shape.T0 + 3, T_cap=shape.T0 + 64, recipe=recipe)
+    _check(shape, p, "fused", mode)
+    _check(shape, p, "definition", mode)
+
+
+@pytest.mark.parametrize("mode", ["k", "v"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("B,H_q,H_kv,grid,R,T,ratio", [(1, 3, 3, 6, 1, 0, 600), (2, 8, 1, 14, 3, 1, 300), (3, 12, 2, 11, 2, 257, 875),
+                                                      (1, 16, 1, 9, 5, 64, 950)])
+def test_one_sided_modes_ragged_shapes(B, H_q, H_kv, grid, R, T, ratio, dtype, mode):
+    shape = wl.Shape("one-sided", 1, B, H_q, H_kv, 128, grid, R, T, 1, dtype, ratio)
+    p = tl.make_problem(shape, 4242 + grid, T=T, T_cap=T + 9, recipe="peaked")
+    _check(shape, p, "fused", mode)
+
+
+def test_one_sided_mode_argument_errors():
+    shape = tl.small(wl.CONFIGS[0], B=1, H_q=2, H_kv=2, R=1)
+    p = tl.make_problem(shape, 5)
+    dev = "cuda"
+    with pytest.raises(kvc.KvcError) as e:       # K-only still needs idx and theta
+        kvc.Layer(2, 2, 128, shape.n, 600, torch.float32, U=p["U"].to(dev), mu=p["mu"].to(dev), mode=kvc.KVC_MODE_K_ONLY)
+    assert e.value.status == -4
+    with pytest.raises(kvc.KvcError) as e:       # V-only still needs U and mu
+        kvc.Layer(2, 2, 128, shape.n, 600, torch.float32, idx=p["idx"], theta=p["theta"].to(dev), mode=kvc.KVC_MODE_V_ONLY)
+    assert e.value.status == -4
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.Layer(2, 2, 128, shape.n, 600, torch.float32, idx=p["idx"], theta=p["theta"].to(dev), U=p["U"].to(dev),
+                  mu=p["mu"].to(dev), mode=7)
+    assert e.value.status == -1
+    lk = tl.gpu_layer(shape, p, dev, "k")
+    lv = tl.gpu_layer(shape, p, dev, "v")
+    m, n, per_row = lk.m, shape.n, 2 * 128 * 4
+    assert (lk.m_k, lk.m_v, lv.m_k, lv.m_v) == (m, n, n, m)
+    assert kvc.kvc_capsule_bytes(lk, 3, 2) == 3 * 2 * 2 * (m + n) * 128 * 4 == kvc.kvc_capsule_bytes(lv, 3, 2)
 
 
 @pytest.mark.parametrize("ratio", [0, 200, 400, 600, 800, 950])
