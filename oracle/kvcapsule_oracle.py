@@ -32,6 +32,12 @@ Readings of the paper taken here (each also listed in the design document):
   - the one-sided variants of App. G (Table 6) compress one side and keep the other verbatim:
     mode "k" stores the retained key rows and the full values (theta only), mode "v" the full keys
     and the projected values (U, mu only); mode "kv" is the method itself.
+  - batches with per-sequence lengths (App. D: c, n, t are per-request quantities): sequence b has
+    N_v[b] vision tokens and T[b] text tokens.  Compression works on whole n-token blocks (Sec. 3.1
+    "an image with size n"); the paper does not say what happens to a vision run that is not a whole
+    number of blocks.  Reading: the first floor(N_v[b] / n) blocks are compressed, the remaining
+    N_v[b] mod n tokens are kept uncompressed and attended like text rows (placed in front of them).
+    A sequence with no token at all gets a zero output row.
 
 Parity pins: every function below is pinned by tests/test_oracle_pins.py
 (library attention, lossless constructions, Eckart-Young, closed forms, brute
@@ -250,6 +256,64 @@ def decode_attend_fused(q, K_t, V_t, theta, U, mu, K_txt, V_txt, passthrough: bo
                 for r in range(R):
                     y = y + w_c[r] @ V_t[b, h, r]
                 out[b, hq] = y + prob_t @ V_txt[b, h]
+    return out
+
+
+# --------------------------------------------------------------------------
+# batches with per-sequence lengths
+# --------------------------------------------------------------------------
+def compress_ragged(K_vis, V_vis, N_v, idx, U, mu, n: int, R_max: int, mode: str = "kv"):
+    """K_vis, V_vis [B,H_kv,N_cap,d] of which sequence b uses its first N_v[b] rows.
+    Returns (K_tilde, V_tilde [B,H_kv,R_max,.,d] with zeros in the unused blocks, R_b [B] = whole blocks per
+    sequence, K_tail, V_tail = lists of [H_kv, N_v[b] mod n, d] arrays: the rows left uncompressed)."""
+    K_vis, V_vis = np.asarray(K_vis, F64), np.asarray(V_vis, F64)
+    B = K_vis.shape[0]
+    R_b = np.zeros(B, np.int64)
+    K_t = V_t = None
+    K_tail, V_tail = [], []
+    for b in range(B):
+        R_b[b] = int(N_v[b]) // n
+        if R_b[b] > R_max:
+            raise ValueError("R_max is smaller than a sequence's block count")
+        whole = int(R_b[b]) * n
+        # the sequence's whole blocks, compressed as a batch of one
+        Kb, Vb = compress(K_vis[b:b + 1, :, :whole], V_vis[b:b + 1, :, :whole], idx, U, mu, n, False, mode)
+        if K_t is None:
+            K_t = np.zeros((B, Kb.shape[1], R_max, Kb.shape[3], Kb.shape[4]), F64)
+            V_t = np.zeros((B, Vb.shape[1], R_max, Vb.shape[3], Vb.shape[4]), F64)
+        K_t[b, :, :R_b[b]] = Kb[0]
+        V_t[b, :, :R_b[b]] = Vb[0]
+        K_tail.append(K_vis[b, :, whole:int(N_v[b])].copy())
+        V_tail.append(V_vis[b, :, whole:int(N_v[b])].copy())
+    return K_t, V_t, R_b, K_tail, V_tail
+
+
+def decode_attend_ragged(q, K_t, V_t, theta, U, mu, K_txt, V_txt, R_b, T_b, mode: str = "kv"):
+    """Decode step on a padded batch: sequence b attends to its first R_b[b] blocks of the capsule store
+    [B,H_kv,R_max,.,d] and to the first T_b[b] rows of K_txt, V_txt [B,H_kv,T_cap,d].  Written as ONE masked
+    softmax over the padded axis (positions a sequence does not have get probability exactly zero); the pin is that
+    this equals running every sequence alone with its own lengths."""
+    q = np.asarray(q, F64)
+    K_txt, V_txt = np.asarray(K_txt, F64), np.asarray(V_txt, F64)
+    K_hat, V_hat = reconstruct(K_t, V_t, theta, U, mu, False, mode)        # [B,H_kv,R_max*n,d]
+    B, H_q, d = q.shape
+    H_kv = K_hat.shape[1]
+    G = H_q // H_kv
+    n = K_hat.shape[2] // np.asarray(K_t).shape[2] if np.asarray(K_t).shape[2] else 0
+    out = np.zeros((B, H_q, d), F64)
+    for b in range(B):
+        have_v = np.arange(K_hat.shape[2]) < int(R_b[b]) * n
+        have_t = np.arange(K_txt.shape[2]) < int(T_b[b])
+        have = np.concatenate([have_v, have_t])
+        if not have.any():
+            continue
+        for hq in range(H_q):
+            h = hq // G
+            K_all = np.concatenate([K_hat[b, h], K_txt[b, h]], axis=0)
+            V_all = np.where(have[:, None], np.concatenate([V_hat[b, h], V_txt[b, h]], axis=0), 0.0)
+            logit = np.where(have, (K_all @ q[b, hq]) / np.sqrt(d), -np.inf)
+            prob = np.where(have, np.exp(logit - logit[have].max()), 0.0)
+            out[b, hq] = (prob / prob.sum()) @ V_all
     return out
 
 

@@ -238,6 +238,73 @@ def test_one_sided_modes():
     np.testing.assert_allclose(got, _library_attention(p["q"], K_all(p["K_vis"]), V_all(V_l)), atol=1e-11)
 
 
+# ---------------------------------------------------------------- per-sequence lengths
+def test_ragged_batch_equals_the_sequences_run_one_by_one():
+    """A padded batch with per-sequence block counts and text lengths (masked softmax) gives, for every sequence, what
+    the uniform functions give for that sequence alone with its own R and T; padding contents (NaN here) never leak;
+    the limits R = 0 (text only), T = 0 (vision only) and an empty sequence (zero row) are in the batch; a vision run
+    that is not a whole number of blocks leaves its remainder uncompressed in front of the text rows."""
+    r = _rng(77)
+    n, m, d, H_kv, H_q, R_max, T_cap, N_cap = 12, 5, 8, 2, 4, 5, 9, 64
+    N_v = [0, 12, 60, 31, 0, 29]            # blocks 0, 1, 5, 2 (+7 left over), 0, 2 (+5)
+    T_own = [4, 0, 1, 2, 0, 0]              # text rows of each sequence (before the left-over vision rows)
+    B = len(N_v)
+    idx = np.sort(r.choice(n, m, replace=False))
+    theta, U = r.normal(size=(H_kv, m, n)), r.normal(size=(H_kv, m, n))
+    mu = r.normal(size=(H_kv, d))
+    q = r.normal(size=(B, H_q, d))
+    K_vis, V_vis = r.normal(size=(B, H_kv, N_cap, d)), r.normal(size=(B, H_kv, N_cap, d))
+    for b in range(B):                      # rows a sequence does not have must never be read into a result
+        K_vis[b, :, N_v[b]:] = np.nan
+        V_vis[b, :, N_v[b]:] = np.nan
+    K_t, V_t, R_b, K_tail, V_tail = orc.compress_ragged(np.nan_to_num(K_vis, nan=1e30), np.nan_to_num(V_vis, nan=1e30),
+                                                        N_v, idx, U, mu, n, R_max)
+    assert list(R_b) == [0, 1, 5, 2, 0, 2] and [k.shape[1] for k in K_tail] == [0, 0, 0, 7, 0, 5]
+    K_txt, V_txt = np.full((B, H_kv, T_cap, d), np.nan), np.full((B, H_kv, T_cap, d), np.nan)
+    T_b = []
+    own = [(r.normal(size=(H_kv, t, d)), r.normal(size=(H_kv, t, d))) for t in T_own]
+    for b in range(B):
+        t0 = K_tail[b].shape[1]
+        K_txt[b, :, :t0], V_txt[b, :, :t0] = K_tail[b], V_tail[b]
+        K_txt[b, :, t0:t0 + T_own[b]], V_txt[b, :, t0:t0 + T_own[b]] = own[b]
+        T_b.append(t0 + T_own[b])
+    K_pad, V_pad = K_t.copy(), V_t.copy()
+    for b in range(B):
+        K_pad[b, :, R_b[b]:] = np.nan
+        V_pad[b, :, R_b[b]:] = np.nan
+    got = orc.decode_attend_ragged(q, K_pad, V_pad, theta, U, mu, K_txt, V_txt, R_b, T_b)
+    assert np.isfinite(got).all()
+    for b in range(B):
+        Rb, Tb = int(R_b[b]), T_b[b]
+        if Rb == 0 and Tb == 0:
+            assert not got[b].any()
+            continue
+        # the sequence alone: its whole blocks compressed by the uniform function, then the uniform decode forms
+        Kb, Vb = orc.compress(K_vis[b:b + 1, :, :Rb * n], V_vis[b:b + 1, :, :Rb * n], idx, U, mu, n)
+        assert np.array_equal(Kb[0], K_t[b, :, :Rb]) and np.array_equal(Vb[0], V_t[b, :, :Rb])
+        for f in (orc.decode_attend_definition, orc.decode_attend_fused):
+            want = f(q[b:b + 1], Kb, Vb, theta, U, mu, K_txt[b:b + 1, :, :Tb], V_txt[b:b + 1, :, :Tb])
+            np.testing.assert_allclose(got[b:b + 1], want, atol=1e-11)
+        # and against the library routine on the reconstructed blocks + left-over rows + text rows
+        K_hat, V_hat = orc.reconstruct(Kb, Vb, theta, U, mu)
+        K_all = np.concatenate([K_hat, K_txt[b:b + 1, :, :Tb]], axis=2)
+        V_all = np.concatenate([V_hat, V_txt[b:b + 1, :, :Tb]], axis=2)
+        np.testing.assert_allclose(got[b:b + 1], _library_attention(q[b:b + 1], K_all, V_all), atol=1e-11)
+
+
+def test_uniform_lengths_reduce_to_the_uniform_functions():
+    p = _problem(31)
+    B = p["q"].shape[0]
+    K_t, V_t = orc.compress(p["K_vis"], p["V_vis"], p["idx"], p["U"], p["mu"], p["n"])
+    want = orc.decode_attend_definition(p["q"], K_t, V_t, p["theta"], p["U"], p["mu"], p["K_txt"], p["V_txt"])
+    got = orc.decode_attend_ragged(p["q"], K_t, V_t, p["theta"], p["U"], p["mu"], p["K_txt"], p["V_txt"],
+                                   [p["R"]] * B, [p["K_txt"].shape[2]] * B)
+    np.testing.assert_allclose(got, want, atol=1e-12)
+    K2, V2, R_b, K_tail, V_tail = orc.compress_ragged(p["K_vis"], p["V_vis"], [p["R"] * p["n"]] * B, p["idx"], p["U"],
+                                                      p["mu"], p["n"], p["R"])
+    assert np.array_equal(K2, K_t) and np.array_equal(V2, V_t) and all(k.shape[1] == 0 for k in K_tail)
+
+
 # ---------------------------------------------------------------- fused algebra
 @pytest.mark.parametrize("seed,kw", [(10, {}), (11, dict(B=1, H_q=4, H_kv=4, R=1, T=0)),
                                      (12, dict(H_q=8, H_kv=1, n=9, m=9, R=2, T=1))])
