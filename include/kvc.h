@@ -136,6 +136,33 @@ KVC_API int kvc_decode_attend(const kvc_layer* layer, const void* q, const void*
                       const void* K_txt, const void* V_txt, int T, int T_cap, void* out,
                       void* workspace, void* stream);
 
+/* Batches with per-sequence lengths (App. D, Eqs. 1-2 count c, n and t per request; Sec. 3.2 "Prefilling Stage"
+ * compresses each request's own vision tokens).
+ *
+ * kvc_compress_ragged: K_vis, V_vis [B][H_kv][N_cap][d], sequence b using its first N_v[b] rows (N_v: DEVICE int[B]).
+ * The floor(N_v[b] / n) whole blocks of a sequence are compressed into blocks [0, R_b[b]) of a capsule store laid out
+ * for R_max blocks per sequence (kvc_capsule_bytes(layer, B, R_max) bytes; blocks a sequence does not have are left
+ * untouched).  The paper compresses whole n-token blocks and is silent about a vision run that is not a whole number
+ * of them: here the N_v[b] mod n rows left over stay uncompressed and are copied to rows [0, T_b[b]) of K_tail, V_tail
+ * [B][H_kv][T_cap][d], the caller's text buffers, in front of which they are attended like text rows; the caller
+ * appends the text rows behind them and adds their count to T_b.  R_b, T_b: DEVICE int[B], written by the call.
+ * A length that does not fit (N_v[b] outside [0, N_cap], more than R_max blocks, more than T_cap rows left over) is
+ * clamped and reported as KVC_ERR_BOUNDS by kvc_read_compress_status.
+ *
+ * kvc_decode_attend_ragged: kvc_decode_attend where sequence b attends to its first R_b[b] <= R_max blocks and its
+ * first T_b[b] <= T_max <= T_cap text rows (DEVICE int[B] arrays read by the kernels, so the call can be replayed
+ * with new lengths; a NULL array means R_max, or T_max, for every sequence).  T_max is an upper bound of T_b the caller
+ * knows (T_cap if nothing better).  A sequence with R_b[b] == 0 and T_b[b] == 0 gets a zero output row.  Lengths
+ * outside their range are clamped and reported as KVC_ERR_BOUNDS by kvc_read_device_status(layer, B, R_max, T_max, ..).
+ * workspace: kvc_workspace_bytes(layer, B, R_max, T_cap).  Every sequence's result equals the call made for that
+ * sequence alone. */
+KVC_API int kvc_compress_ragged(const kvc_layer* layer, const void* K_vis, const void* V_vis, int B, int N_cap,
+                        const int* N_v, int R_max, void* capsules, void* K_tail, void* V_tail, int T_cap,
+                        int* R_b, int* T_b, void* stream);
+KVC_API int kvc_decode_attend_ragged(const kvc_layer* layer, const void* q, const void* capsules, int B, int R_max,
+                             const int* R_b, const void* K_txt, const void* V_txt, int T_max, const int* T_b,
+                             int T_cap, void* out, void* workspace, void* stream);
+
 /* Uncompressed decode attention over K, V [B][H_kv][S_cap][d] (first S rows valid), the standard
  * attention of Sec. 3.1; the comparator the compressed path is measured against.  Uses the same
  * workspace rule with R = 0, T_cap = S_cap. */

@@ -57,6 +57,10 @@ def _lib() -> C.CDLL:
         lib.kvc_compress.argtypes = [vp, vp, vp, i, i, vp, vp]; lib.kvc_compress.restype = i
         lib.kvc_decode_attend.argtypes = [vp, vp, vp, i, i, vp, vp, i, i, vp, vp, vp]
         lib.kvc_decode_attend.restype = i
+        lib.kvc_compress_ragged.argtypes = [vp, vp, vp, i, i, vp, i, vp, vp, vp, i, vp, vp, vp]
+        lib.kvc_compress_ragged.restype = i
+        lib.kvc_decode_attend_ragged.argtypes = [vp, vp, vp, i, i, vp, vp, vp, i, vp, i, vp, vp, vp]
+        lib.kvc_decode_attend_ragged.restype = i
         lib.kvc_attend_full.argtypes = [vp, vp, vp, vp, i, i, i, vp, vp, vp]; lib.kvc_attend_full.restype = i
         lib.kvc_decode_attend_static.argtypes = [vp, vp, vp, i, i, vp, vp, i, i, vp, vp]
         lib.kvc_decode_attend_static.restype = i
@@ -168,6 +172,21 @@ def kvc_decode_attend(layer: Layer, q, capsules, B: int, R: int, K_txt, V_txt, T
                       workspace, stream=None) -> None:
     _check(_lib().kvc_decode_attend(layer.handle, _ptr(q), _ptr(capsules), B, R, _ptr(K_txt), _ptr(V_txt), T,
                                     T_cap, _ptr(out), _ptr(workspace), _stream(stream)), "kvc_decode_attend")
+
+
+def kvc_compress_ragged(layer: Layer, K_vis, V_vis, B: int, N_cap: int, N_v, R_max: int, capsules, K_tail, V_tail,
+                        T_cap: int, R_b, T_b, stream=None) -> None:
+    """N_v, R_b, T_b: int32 device tensors of B entries (R_b and T_b are written)."""
+    _check(_lib().kvc_compress_ragged(layer.handle, _ptr(K_vis), _ptr(V_vis), B, N_cap, _ptr(N_v), R_max, _ptr(capsules),
+                                      _ptr(K_tail), _ptr(V_tail), T_cap, _ptr(R_b), _ptr(T_b), _stream(stream)),
+           "kvc_compress_ragged")
+
+
+def kvc_decode_attend_ragged(layer: Layer, q, capsules, B: int, R_max: int, R_b, K_txt, V_txt, T_max: int, T_b,
+                             T_cap: int, out, workspace, stream=None) -> None:
+    _check(_lib().kvc_decode_attend_ragged(layer.handle, _ptr(q), _ptr(capsules), B, R_max, _ptr(R_b), _ptr(K_txt),
+                                           _ptr(V_txt), T_max, _ptr(T_b), T_cap, _ptr(out), _ptr(workspace),
+                                           _stream(stream)), "kvc_decode_attend_ragged")
 
 
 def kvc_decode_attend_static(layer: Layer, q, capsules, B: int, R: int, K_txt, V_txt, T: int, T_cap: int, out,

@@ -300,7 +300,8 @@ static unsigned int next_token() {
 }
 
 int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B, int R, const void* K_txt,
-                  const void* V_txt, int T, int T_cap, void* out, void* workspace, cudaStream_t st) {
+                  const void* V_txt, int T, int T_cap, void* out, void* workspace, cudaStream_t st, const int* R_b,
+                  const int* T_b) {
   if (!L || B < 0 || R < 0 || T < 0 || T_cap < T) return KVC_ERR_ARG;
   if (B == 0) return KVC_OK;
   if (R == 0 && T == 0) return KVC_ERR_SHAPE;
@@ -337,13 +338,15 @@ int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B
   a.fpart_y = reinterpret_cast<float*>(ws + a.ws.off_fpy);
   a.fpart_ml = reinterpret_cast<float2*>(ws + a.ws.off_fpml);
   a.split_base = ws + a.ws.off_split;
+  a.R_b = R_b; a.T_b = T_b;
 
   // bf16 storage with TMA-compatible shapes and pointers: the whole of Algorithm 1 in one kernel
   {
     // R == 0 (text rows only, the uncompressed comparator): the same kernel with text stages only
     // rho = 0 stores K and V verbatim: vision rows and text rows are attended as plain rows by the text-only mode
     const bool plain = R == 0 || L->passthrough;
-    const bool one_sided = R > 0 && L->mode != KVC_MODE_KV;      // served by the three-phase kernels below
+    // one-sided modes and per-sequence lengths are served by the three-phase kernels below
+    const bool one_sided = (R > 0 && L->mode != KVC_MODE_KV) || R_b || T_b;
     const uintptr_t align = reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(capsules) |
                             reinterpret_cast<uintptr_t>(out) | (T > 0 ? reinterpret_cast<uintptr_t>(K_txt) |
                             reinterpret_cast<uintptr_t>(V_txt) : 0) | reinterpret_cast<uintptr_t>(L->desc.mu);
@@ -375,6 +378,28 @@ int kvc_decode_attend(const kvc_layer* L, const void* q, const void* capsules, i
                       const void* V_txt, int T, int T_cap, void* out, void* workspace, void* stream) {
   return decode_common(L, q, capsules, B, R, K_txt, V_txt, T, T_cap, out, workspace,
                        static_cast<cudaStream_t>(stream));
+}
+
+int kvc_decode_attend_ragged(const kvc_layer* L, const void* q, const void* capsules, int B, int R_max, const int* R_b,
+                             const void* K_txt, const void* V_txt, int T_max, const int* T_b, int T_cap, void* out,
+                             void* workspace, void* stream) {
+  return decode_common(L, q, capsules, B, R_max, K_txt, V_txt, T_max, T_cap, out, workspace,
+                       static_cast<cudaStream_t>(stream), R_b, T_b);
+}
+
+int kvc_compress_ragged(const kvc_layer* L, const void* K_vis, const void* V_vis, int B, int N_cap, const int* N_v,
+                        int R_max, void* capsules, void* K_tail, void* V_tail, int T_cap, int* R_b, int* T_b, void* stream) {
+  if (!L || B < 0 || N_cap < 0 || R_max < 0 || T_cap < 0) return KVC_ERR_ARG;
+  if (B == 0) return KVC_OK;
+  if (!N_v || !R_b || !T_b || (N_cap > 0 && (!K_vis || !V_vis)) || (R_max > 0 && !capsules) ||
+      (T_cap > 0 && (!K_tail || !V_tail)))
+    return KVC_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemsetAsync(L->d_cstatus, 0, sizeof(int), st);
+  if (e != cudaSuccess) return cuda_status(e);
+  void* Vc = capsules ? static_cast<char*>(capsules) + key_part_bytes(L, B, R_max) : nullptr;
+  return cuda_status(launch_compress_ragged(L, K_vis, V_vis, B, N_cap, N_v, R_max, capsules, Vc, K_tail, V_tail, T_cap,
+                                            R_b, T_b, st));
 }
 
 int kvc_attend_full(const kvc_layer* L, const void* q, const void* K, const void* V, int B, int S, int S_cap,

@@ -158,6 +158,8 @@ struct DecodeArgs {
   int* cnt;
   unsigned long long* fcnt;   // arrival words of the one-kernel path
   unsigned int token;         // this call's token (never 0)
+  const int* R_b;      // per-sequence block counts (<= R) and text lengths (<= T), device arrays; nullptr: R and T for all
+  const int* T_b;
   int* status;         // device status word (0 = ok, else a kvc_status), cleared by the first kernel of the call
   float* fpart_y;      // partials of the one-kernel path
   float2* fpart_ml;
@@ -165,10 +167,33 @@ struct DecodeArgs {
   WsLayout ws;
 };
 
+#ifdef __CUDACC__
+// blocks and text rows sequence b takes part with (clamped to the call's bounds; the first kernel reports a clamp)
+__device__ __forceinline__ int seq_R(const DecodeArgs& a, int b) {
+  if (!a.R_b) return a.R;
+  const int r = a.R_b[b];
+  return r < 0 ? 0 : (r > a.R ? a.R : r);
+}
+__device__ __forceinline__ int seq_T(const DecodeArgs& a, int b) {
+  if (!a.T_b) return a.T;
+  const int t = a.T_b[b];
+  return t < 0 ? 0 : (t > a.T ? a.T : t);
+}
+// after the status word has been cleared: lengths outside [0, R] x [0, T] are reported (and clamped by seq_R / seq_T)
+__device__ __forceinline__ void check_seq_lengths(const DecodeArgs& a, int tid, int nthreads) {
+  if (!a.R_b && !a.T_b) return;
+  for (int b = tid; b < a.B; b += nthreads) {
+    const bool bad = (a.R_b && (a.R_b[b] < 0 || a.R_b[b] > a.R)) || (a.T_b && (a.T_b[b] < 0 || a.T_b[b] > a.T));
+    if (bad) atomicExch(a.status, (int)KVC_ERR_BOUNDS);
+  }
+}
+#endif
+
 // validation + the three launches of one decode call; `workspace` is any 256-byte aligned device
 // scratch of ws_layout(L, B, R, T).total bytes
 int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B, int R, const void* K_txt,
-                  const void* V_txt, int T, int T_cap, void* out, void* workspace, cudaStream_t st);
+                  const void* V_txt, int T, int T_cap, void* out, void* workspace, cudaStream_t st,
+                  const int* R_b = nullptr, const int* T_b = nullptr);
 
 // Raises a kernel's dynamic shared-memory limit to at least `bytes` on the current device.  The attribute is per device
 // (and per kernel), so the record of what has been set is keyed by (kernel, device ordinal); safe from several host threads.
@@ -220,6 +245,9 @@ void map_cache_destroy(kvc_map_cache* c);
 cudaError_t compute_usum(const kvc_layer* L, float* usum);
 cudaError_t launch_project_values_tc(const kvc_layer* L, const void* V_vis, int B, int R, void* Vc, cudaStream_t st, bool* used);
 cudaError_t launch_project_values_mma(const kvc_layer* L, const void* V_vis, int B, int R, void* Vc, cudaStream_t st, bool* used);
+cudaError_t launch_compress_ragged(const kvc_layer* L, const void* K_vis, const void* V_vis, int B, int N_cap,
+                                   const int* N_v, int R_max, void* Kc, void* Vc, void* K_tail, void* V_tail, int T_cap,
+                                   int* R_b, int* T_b, cudaStream_t st);
 cudaError_t launch_compress_keys(const kvc_layer* L, const void* K_vis, int B, int R, void* Kc, cudaStream_t st);
 cudaError_t launch_compress_values(const kvc_layer* L, const void* V_vis, int B, int R, void* Vc, cudaStream_t st);
 

@@ -40,11 +40,11 @@ __device__ __forceinline__ ChunkRef chunk_ref(const DecodeArgs& a, int q) {
   if (c.is_txt) {
     c.r = 0;
     c.j0 = (lc - nvis) * OUT_CHUNK;
-    c.rows = min(OUT_CHUNK, a.T - c.j0);       // <= 0 for chunks beyond the current text length
+    c.rows = min(OUT_CHUNK, seq_T(a, c.b) - c.j0);   // <= 0 for chunks beyond the sequence's text length
   } else {
     c.r = lc / a.ws.cpb;
     c.j0 = (lc - c.r * a.ws.cpb) * OUT_CHUNK;
-    c.rows = min(OUT_CHUNK, a.mv - c.j0);
+    c.rows = c.r < seq_R(a, c.b) ? min(OUT_CHUNK, a.mv - c.j0) : 0;   // 0 for a block the sequence does not have
   }
   return c;
 }
@@ -300,7 +300,7 @@ __global__ void __launch_bounds__(256) merge_kernel(DecodeArgs a) {
     num.x = fmaf(sc, y.x, num.x); num.y = fmaf(sc, y.y, num.y);
     num.z = fmaf(sc, y.z, num.z); num.w = fmaf(sc, y.w, num.w);
   }
-  const float inv = 1.f / den;
+  const float inv = den > 0.f ? 1.f / den : 0.f;     // a sequence without any row: a zero output row
   T* o = static_cast<T*>(a.out) + (size_t)head * D + lane * 4;
   store_elem(o, num.x * inv); store_elem(o + 1, num.y * inv);
   store_elem(o + 2, num.z * inv); store_elem(o + 3, num.w * inv);

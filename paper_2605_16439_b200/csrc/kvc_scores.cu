@@ -25,11 +25,14 @@ __global__ void __launch_bounds__(256) scores_kernel(DecodeArgs a, int tiles_vis
   const int sub = lane / LPR, c = lane % LPR;
 
   // the arrival counters of the output kernel's split merge are cleared here, one launch earlier
-  if (blockIdx.x == 0)
+  if (blockIdx.x == 0) {
     for (int i = threadIdx.x; i <= a.B * a.H_kv; i += blockDim.x) a.cnt[i] = 0;   // counters + status word
+    __syncthreads();
+    check_seq_lengths(a, threadIdx.x, blockDim.x);
+  }
 
   const bool is_txt = tile >= tiles_vis;
-  const int nrows = is_txt ? a.T : a.R * a.m;
+  const int nrows = is_txt ? seq_T(a, b) : seq_R(a, b) * a.m;
   const int row0 = (is_txt ? tile - tiles_vis : tile) * SCORE_TILE_ROWS + warp * ROWS_PER_WARP;
   const T* base = is_txt
       ? static_cast<const T*>(a.K_txt) + (size_t)bh * a.T_cap * D
@@ -122,8 +125,11 @@ __global__ void __launch_bounds__(256, 4) scores_mma_kernel(DecodeArgs a, int tv
   // the expansion kernel may start now: it prefetches parameters, then waits for this grid to finish
   grid_dep_launch();
 
-  if (blockIdx.x == 0)
+  if (blockIdx.x == 0) {
     for (int i = threadIdx.x; i <= a.B * a.H_kv; i += blockDim.x) a.cnt[i] = 0;   // counters + status word
+    __syncthreads();
+    check_seq_lengths(a, threadIdx.x, blockDim.x);
+  }
 
   int cur_bh = -1;
   uint4 qf[NG][4];
@@ -131,7 +137,7 @@ __global__ void __launch_bounds__(256, 4) scores_mma_kernel(DecodeArgs a, int tv
     const int bh = tile / tiles_per_bh, lt = tile - bh * tiles_per_bh;
     const bool is_txt = lt >= tv;
     const int row0 = (is_txt ? lt - tv : lt) * SM_TILE;
-    const int nrows = is_txt ? a.T : VR;
+    const int nrows = is_txt ? seq_T(a, bh / a.H_kv) : seq_R(a, bh / a.H_kv) * a.m;
     const T* base = is_txt ? static_cast<const T*>(a.K_txt) + (size_t)bh * a.T_cap * D
                            : static_cast<const T*>(a.Kc) + (size_t)bh * VR * D;
     const int ra = row0 + g, rb = row0 + g + 8;
