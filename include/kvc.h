@@ -163,6 +163,30 @@ KVC_API int kvc_decode_attend_ragged(const kvc_layer* layer, const void* q, cons
                              const int* R_b, const void* K_txt, const void* V_txt, int T_max, const int* T_b,
                              int T_cap, void* out, void* workspace, void* stream);
 
+/* Parameter fits from activations (App. C, Algorithm 2), on the device in fp64.  Calibration-time calls: each one
+ * SYNCHRONISES the stream several times (the eigen-solver checks convergence on the host) and returns with its outputs
+ * complete.  X_vis: [B][H_kv][R*n][d] device, storage type `dtype`; every n-row block of every sequence is one sample.
+ * workspace: kvc_fit_workspace_bytes(H_kv, n) bytes, 256-byte aligned, device.  sweeps_out (may be NULL): sweeps the
+ * eigen-solver took.  Errors: KVC_ERR_ARG / _SHAPE (m outside [1, n]) / _DTYPE / _WORKSPACE / _BOUNDS (index set) / _CUDA.
+ *
+ * kvc_fit_value_pca: FitValuePCA (Sec. 3.1 "Sequence-Level Low-Rank Compression for Values"): mu_out [H_kv][d] = the
+ * mean of the value rows over samples and positions; U_out [H_kv][m][n] = the top-m principal directions along the
+ * token axis of the centred values (eigenvectors of the n x n token covariance by a hand-written cyclic Jacobi solver;
+ * rows orthonormal, each with its entry of largest magnitude positive), both written in `dtype`.  eig_out (may be
+ * NULL): DEVICE double [H_kv][n], the covariance eigenvalues in descending order (squared singular values of the
+ * pooled centred columns; the energy the projection loses is the sum of entries m..n-1).
+ *
+ * kvc_fit_key_reconstructor: for the fixed retained index set idx (HOST, as in kvc_layer_desc), theta_out [H_kv][m][n]
+ * minimising sum over samples of || K - theta^T K[idx] ||_F^2, the reconstruction term of Algorithm 2 for a reconstructor
+ * that is linear along the token axis; minimum-norm solution: eigen-directions of the retained rows' second-moment
+ * matrix with eigenvalue <= rcond * the largest are dropped. */
+KVC_API size_t kvc_fit_workspace_bytes(int H_kv, int n);
+KVC_API int kvc_fit_value_pca(const void* V_vis, int B, int R, int H_kv, int n, int m, kvc_dtype dtype, void* U_out,
+                      void* mu_out, double* eig_out, void* workspace, void* stream, int* sweeps_out);
+KVC_API int kvc_fit_key_reconstructor(const void* K_vis, int B, int R, int H_kv, int n, int m, const int32_t* idx,
+                              int idx_per_head, double rcond, kvc_dtype dtype, void* theta_out, void* workspace,
+                              void* stream, int* sweeps_out);
+
 /* Uncompressed decode attention over K, V [B][H_kv][S_cap][d] (first S rows valid), the standard
  * attention of Sec. 3.1; the comparator the compressed path is measured against.  Uses the same
  * workspace rule with R = 0, T_cap = S_cap. */

@@ -61,6 +61,12 @@ def _lib() -> C.CDLL:
         lib.kvc_compress_ragged.restype = i
         lib.kvc_decode_attend_ragged.argtypes = [vp, vp, vp, i, i, vp, vp, vp, i, vp, i, vp, vp, vp]
         lib.kvc_decode_attend_ragged.restype = i
+        lib.kvc_fit_workspace_bytes.argtypes = [i, i]; lib.kvc_fit_workspace_bytes.restype = C.c_size_t
+        lib.kvc_fit_value_pca.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, vp, C.POINTER(i)]
+        lib.kvc_fit_value_pca.restype = i
+        lib.kvc_fit_key_reconstructor.argtypes = [vp, i, i, i, i, i, C.POINTER(C.c_int32), i, C.c_double, i, vp, vp, vp,
+                                                  C.POINTER(i)]
+        lib.kvc_fit_key_reconstructor.restype = i
         lib.kvc_attend_full.argtypes = [vp, vp, vp, vp, i, i, i, vp, vp, vp]; lib.kvc_attend_full.restype = i
         lib.kvc_decode_attend_static.argtypes = [vp, vp, vp, i, i, vp, vp, i, i, vp, vp]
         lib.kvc_decode_attend_static.restype = i
@@ -218,6 +224,42 @@ def kvc_read_compress_status(layer: Layer) -> int:
     out = C.c_int(-99)
     _check(_lib().kvc_read_compress_status(layer.handle, C.byref(out)), "kvc_read_compress_status")
     return out.value
+
+
+def kvc_fit_value_pca(V_vis: torch.Tensor, n: int, m: int, want_eig: bool = False, stream=None):
+    """FitValuePCA on the device.  V_vis [B, H_kv, R*n, d] -> (U [H_kv, m, n], mu [H_kv, d], eig [H_kv, n] fp64 or None,
+    sweeps of the eigen-solver)."""
+    B, H_kv, N_v, d = V_vis.shape
+    if N_v % n:
+        raise ValueError("N_v must be a whole number of n-token blocks")
+    dev, dt = V_vis.device, V_vis.dtype
+    U = torch.empty((H_kv, m, n), dtype=dt, device=dev)
+    mu = torch.empty((H_kv, d), dtype=dt, device=dev)
+    eig = torch.empty((H_kv, n), dtype=torch.float64, device=dev) if want_eig else None
+    ws = torch.empty(_lib().kvc_fit_workspace_bytes(H_kv, n), dtype=torch.uint8, device=dev)
+    sweeps = C.c_int(-1)
+    _check(_lib().kvc_fit_value_pca(_ptr(V_vis.contiguous()), B, N_v // n, H_kv, n, m, _DTYPES[dt], _ptr(U), _ptr(mu), _ptr(eig),
+                                    _ptr(ws), _stream(stream), C.byref(sweeps)), "kvc_fit_value_pca")
+    return U, mu, eig, sweeps.value
+
+
+def kvc_fit_key_reconstructor(K_vis: torch.Tensor, idx: torch.Tensor, n: int, rcond: float = 1e-10, stream=None):
+    """Least-squares key reconstructor for the retained index set idx ([m] or [H_kv, m], host).  -> (theta [H_kv, m, n],
+    sweeps of the eigen-solver)."""
+    B, H_kv, N_v, d = K_vis.shape
+    if N_v % n:
+        raise ValueError("N_v must be a whole number of n-token blocks")
+    dev, dt = K_vis.device, K_vis.dtype
+    idx_host = idx.detach().to("cpu", torch.int32).contiguous()
+    m = idx_host.shape[-1]
+    theta = torch.empty((H_kv, m, n), dtype=dt, device=dev)
+    ws = torch.empty(_lib().kvc_fit_workspace_bytes(H_kv, n), dtype=torch.uint8, device=dev)
+    sweeps = C.c_int(-1)
+    _check(_lib().kvc_fit_key_reconstructor(_ptr(K_vis.contiguous()), B, N_v // n, H_kv, n, m,
+                                            C.cast(idx_host.data_ptr(), C.POINTER(C.c_int32)), 1 if idx_host.dim() == 2 else 0,
+                                            float(rcond), _DTYPES[dt], _ptr(theta), _ptr(ws), _stream(stream), C.byref(sweeps)),
+           "kvc_fit_key_reconstructor")
+    return theta, sweeps.value
 
 
 def kvc_collapse_theta(W1: torch.Tensor, W2: torch.Tensor, stream=None) -> torch.Tensor:
