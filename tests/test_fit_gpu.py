@@ -30,7 +30,7 @@ SHAPES = [  # B, H_kv, R, grid, m
     (2, 3, 3, 5, 10),        # n = 25: odd, the solver pads one index
     (4, 2, 2, 12, 58),       # n = 144
     (2, 1, 1, 4, 16),        # m = n
-    (1, 2, 1, 3, 1),         # fewer observations (128) than ... n = 9, m = 1
+    (1, 2, 1, 3, 1),         # n = 9, m = 1: a single component
 ]
 
 
