@@ -573,7 +573,7 @@ def measure(shape, config_index, dev, rank, world, local, steps, warmup, profile
     peak, peak_src = peaks["hbm"], peaks["hbm_src"]
 
     roofline, kernels = None, {}
-    decode_kernels = ("scores", "output", "fused", "fused_tc", "fused_pair", "split_scores", "split_expand", "split_output")
+    decode_kernels = ("scores", "output", "fused", "fused_tc", "fused_pair", "resident", "split_scores", "split_expand", "split_output")
     if prof:
         tot = sum(v[0] for v in prof.values()) or 1.0
         for k, (t, n) in prof.items():
@@ -582,7 +582,7 @@ def measure(shape, config_index, dev, rank, world, local, steps, warmup, profile
                               "share": round(t / tot, 4)}
         dom = max(decode_kernels, key=lambda k: prof.get(k, (0.0, 0))[0])
         t_dom, n_dom = prof[dom]
-        if dom in ("fused", "fused_tc", "fused_pair"):
+        if dom in ("fused", "fused_tc", "fused_pair", "resident"):
             # one kernel per layer call: its launch duration is the decode part of the timed region over its launches
             # (events recorded inside the timed region, on the launching stream; consecutive launches overlap their
             # prologues, which the per-launch brackets of the second pass forbid)

@@ -94,7 +94,7 @@ KVC_API int kvc_retained_len(int n, int ratio_permille);
  * bf16 decode calls run Alg. 1 either as one kernel (steps 2-3 on mma.sync with the logits in registers, or on tcgen05
  * with the logits in tensor memory) or, for block lengths above 640, as three kernels (streaming scores, tcgen05
  * expansion per 128 rows and range of the n axis, streaming output); the library picks per shape (same results within
- * the bf16 tolerance).  The environment variable KVC_EXPANSION = "tcgen05" | "mma" | "pair" | "split", read when the
+ * the bf16 tolerance).  The environment variable KVC_EXPANSION = "tcgen05" | "mma" | "pair" | "split" | "resident", read when the
  * handle is created, forces one of them where it applies ("pair": the tcgen05 one-kernel path run by clusters of two
  * CTAs per (sequence, KV head)); "phases" forces the generic three-phase kernels that also serve fp32 storage. */
 KVC_API int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out);
@@ -284,7 +284,8 @@ typedef enum {
   KVC_KERNEL_SPLIT_SCORES = 10,   /* three-kernel bf16 path: Alg. 1 step 1, one pass over K_tilde */
   KVC_KERNEL_SPLIT_EXPAND = 11,   /* its steps 2-3 on tcgen05, per 128 expansion rows and range of the n axis; the text rows on idle SMs */
   KVC_KERNEL_SPLIT_OUTPUT = 12,   /* its step 4 and the normalisation, one pass over V_tilde, merged with the text partials */
-  KVC_KERNEL_COUNT = 13
+  KVC_KERNEL_RESIDENT = 13,       /* one-kernel bf16 path for short blocks whose theta and U stay in shared memory */
+  KVC_KERNEL_COUNT = 14
 } kvc_kernel_id;
 KVC_API int kvc_profile_start(int max_launches);
 KVC_API int kvc_profile_stop(void);

@@ -297,7 +297,7 @@ def capsule_views(layer: Layer, capsules, B: int, R: int):
             capsules[kb:total].view(layer.dtype).view(B, layer.H_kv, R, layer.m_v, layer.d))
 
 
-KVC_KERNEL_COUNT = 13
+KVC_KERNEL_COUNT = 14
 
 
 def kvc_profile_start(max_launches: int) -> None:

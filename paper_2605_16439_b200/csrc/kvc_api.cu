@@ -9,6 +9,7 @@
 
 #include "kvc_internal.cuh"
 #include "kvc_split.cuh"
+#include "kvc_resident.cuh"
 
 namespace kvc {
 
@@ -100,6 +101,7 @@ WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap) {
     }
     w.off_split = take(sb);
   }
+  w.off_resident = take(B > 0 && R > 0 && plan_resident(L, B, R, 0).ok ? resident_ws(L, B).bytes : 0);
   w.total = off;
   return w;
 }
@@ -198,7 +200,7 @@ int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out) {
   L->num_sms = 0;
   {
     const char* ex = std::getenv("KVC_EXPANSION");
-    L->use_tc = !ex ? 0 : (std::strcmp(ex, "tcgen05") == 0 ? 1 : (std::strcmp(ex, "pair") == 0 ? 2 : (std::strcmp(ex, "mma") == 0 ? -1 : (std::strcmp(ex, "phases") == 0 ? -2 : (std::strcmp(ex, "split") == 0 ? 3 : 0)))));
+    L->use_tc = !ex ? 0 : (std::strcmp(ex, "tcgen05") == 0 ? 1 : (std::strcmp(ex, "pair") == 0 ? 2 : (std::strcmp(ex, "mma") == 0 ? -1 : (std::strcmp(ex, "phases") == 0 ? -2 : (std::strcmp(ex, "split") == 0 ? 3 : (std::strcmp(ex, "resident") == 0 ? 4 : 0))))));
   }
   if (cudaGetDevice(&L->device) != cudaSuccess ||
       cudaDeviceGetAttribute(&L->num_sms, cudaDevAttrMultiProcessorCount, L->device) != cudaSuccess ||
@@ -338,6 +340,7 @@ int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B
   a.fpart_y = reinterpret_cast<float*>(ws + a.ws.off_fpy);
   a.fpart_ml = reinterpret_cast<float2*>(ws + a.ws.off_fpml);
   a.split_base = ws + a.ws.off_split;
+  a.resident_base = ws + a.ws.off_resident;
   a.R_b = R_b; a.T_b = T_b;
 
   // bf16 storage with TMA-compatible shapes and pointers: the whole of Algorithm 1 in one kernel
@@ -350,6 +353,14 @@ int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B
     const uintptr_t align = reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(capsules) |
                             reinterpret_cast<uintptr_t>(out) | (T > 0 ? reinterpret_cast<uintptr_t>(K_txt) |
                             reinterpret_cast<uintptr_t>(V_txt) : 0) | reinterpret_cast<uintptr_t>(L->desc.mu);
+    if (!plain && !one_sided && (align & 15) == 0 && L->use_tc == 4) {
+      const ResidentPlan rp = plan_resident(L, B, R, T);
+      if (rp.ok) {
+        bool encoded = false;
+        const cudaError_t re = launch_resident(L, a, rp, st, &encoded);
+        if (encoded) return cuda_status(re);
+      }
+    }
     if (!plain && !one_sided && (align & 15) == 0 && T <= 64 * SP_OUT_ROWS * SP_TEXT_CHUNK && use_split(L, B, R)) {
       const SplitPlan sp = plan_split(L, B, R);
       bool encoded = false;

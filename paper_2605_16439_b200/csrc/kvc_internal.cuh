@@ -72,6 +72,7 @@ struct WsLayout {
   size_t off_fpml; // float2 [B*H_kv][nrg][G]   their (max, sum)
   size_t off_fcnt; // u64 [B*H_kv]              arrival words of the one-kernel path: (call token, arrivals)
   size_t off_split;// the regions of the three-kernel bf16 path (kvc_split.cuh), 0 bytes when the shape does not take it
+  size_t off_resident; // the regions of the resident-parameter bf16 path (kvc_resident.cuh), likewise
   size_t total;
 };
 
@@ -164,6 +165,7 @@ struct DecodeArgs {
   float* fpart_y;      // partials of the one-kernel path
   float2* fpart_ml;
   void* split_base;    // regions of the three-kernel bf16 path
+  void* resident_base; // regions of the resident-parameter bf16 path
   WsLayout ws;
 };
 

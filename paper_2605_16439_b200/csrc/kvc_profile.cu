@@ -84,6 +84,7 @@ const char* kvc_kernel_name(int kernel_id) {
     case KVC_KERNEL_SPLIT_SCORES: return "split_scores";
     case KVC_KERNEL_SPLIT_EXPAND: return "split_expand";
     case KVC_KERNEL_SPLIT_OUTPUT: return "split_output";
+    case KVC_KERNEL_RESIDENT: return "resident";
     default: return "?";
   }
 }
