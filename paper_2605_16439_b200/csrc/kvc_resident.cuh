@@ -1,7 +1,9 @@
 // One-kernel bf16 decode path for short blocks whose parameters fit shared memory ("resident" path): theta[h] and U[h]
-// are loaded once per CTA and stay in shared memory, the capsule rows and the text rows stream through a ring of
-// 64-row tiles, and a CTA walks a contiguous run of work items (one vision block or one 64-row text chunk each) of its
-// KV head, carrying flash-style running (max, sum, y) per query head across the items of a (sequence, KV head).
+// are loaded once per CTA and stay in shared memory.  The work of a (sequence, KV head) is a list of items (one vision
+// block or one 64-row text chunk each); it is cut into `cpb` units, a CTA takes whole units of its KV head, and inside a
+// unit every WARP walks its own items from its own ring of 16-row pieces, carrying flash-style (max, sum, y) per query
+// head in registers: no barrier of the CTA until the unit ends, when the warps' results are merged through shared
+// memory (and the units of a pair through the workspace).
 #pragma once
 
 #include "kvc_tma.cuh"
@@ -9,30 +11,32 @@
 
 namespace kvc {
 
-constexpr int RS_TILE_ROWS = 64;                  // rows per ring tile (16 KB: two 64-channel halves, 128-byte swizzle)
-constexpr uint32_t RS_TILE_BYTES = RS_TILE_ROWS * 256u;
-constexpr int RS_WARPS = 8;                       // consumer warps (+ one producer warp)
-constexpr int RS_MAX_STAGES = 8;
+constexpr int RS_PIECE_ROWS = 16;                 // rows per ring piece (4 KB: two 64-channel halves, 128-byte swizzle)
+constexpr uint32_t RS_PIECE_BYTES = RS_PIECE_ROWS * 256u;
+constexpr int RS_TEXT_ROWS = 64;                  // text rows per item
+constexpr int RS_WARPS = 8;
+constexpr int RS_MAX_SLOTS = 6;                   // pieces in flight per warp
+constexpr int RS_MAX_CPB = 16;                    // units per (sequence, KV head)
+constexpr int RS_MAX_MP16 = 8;                    // m <= 128
 
 struct ResidentPlan {
   int ok;
-  int mp;            // m rounded up to 16: rows of the parameter panels, K extent of the first product
+  int mp;            // m rounded up to 16: rows of the parameter panels
   int ncg;           // n / 64 column panels of theta and U
-  int kt;            // 64-row tiles per block side
-  int ct;            // 64-row text chunks per (sequence, KV head) at this T
-  int items_b;       // work items per (sequence, KV head): R + ct
+  int ct;            // text items per (sequence, KV head) at this T
+  int items_b;       // items per (sequence, KV head): R + ct
+  int cpb;           // units per (sequence, KV head)
   int cph;           // CTAs per KV head
   int grid;
-  int stages;
-  int pitchS, pitchP, pitchW;                        // row pitches in elements
-  uint32_t par_bytes;                                // bytes of one parameter matrix in shared memory
-  uint32_t off_theta, off_U, off_ring, off_S, off_P, off_W, off_T, off_stat;
+  int slots;         // ring pieces per warp
+  uint32_t par_bytes;
+  uint32_t off_theta, off_U, off_ring;
   size_t smem;
 };
 
 struct ResidentWs {
-  size_t off_py;     // fp32 [B*H_kv][slots][16][D]
-  size_t off_pml;    // float2 [B*H_kv][slots][16]
+  size_t off_py;     // fp32 [B*H_kv][RS_MAX_CPB][8][D]
+  size_t off_pml;    // float2 [B*H_kv][RS_MAX_CPB][8]
   size_t off_cnt;    // u64 [B*H_kv] arrival words (token, count)
   size_t bytes;
 };
@@ -51,11 +55,9 @@ struct ResidentArgs {
   unsigned int token;
   int* status;
   int B, H_kv, G, R, m, mp, n, T;
-  int ncg, kt, ct, items_b, cph, stages;
-  int slots;         // partial slots per (sequence, KV head) in py / pml
-  int pitchS, pitchP, pitchW;
+  int ncg, ct, items_b, cpb, cph, slots;
   uint32_t par_bytes;
-  uint32_t off_theta, off_U, off_ring, off_S, off_P, off_W, off_T, off_stat;
+  uint32_t off_theta, off_U, off_ring;
 };
 
 }  // namespace kvc

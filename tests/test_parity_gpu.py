@@ -469,13 +469,14 @@ def _random_shapes(count, seed):
 
 @pytest.mark.parametrize("recipe", ["flat", "peaked", "structured"])
 @pytest.mark.parametrize("B,H_q,H_kv,grid,R,T,ratio", [
-    (1, 7, 1, 16, 6, 517, 600),        # the video shape: n = 256, m = 103, G = 7
-    (4, 28, 4, 16, 9, 130, 600),       # several CTAs per (sequence, KV head) and CTAs that cross sequences
+    (1, 7, 1, 16, 6, 517, 600),        # the video shape: n = 256, m = 103, G = 7; 16 units of one pair
+    (4, 28, 4, 16, 9, 130, 600),       # several units per (sequence, KV head), warps with and without items
     (2, 2, 2, 16, 3, 0, 700),          # MHA, no text
-    (3, 32, 2, 8, 5, 64, 250),         # n = 64, m = 48, G = 16
-    (2, 12, 1, 8, 40, 1, 900),         # m = 7: a single padded row tile, many blocks
+    (3, 16, 2, 8, 5, 64, 250),         # n = 64, m = 48, G = 8
+    (2, 6, 1, 8, 40, 1, 900),          # m = 7: a single padded piece, many blocks, one text row
     (5, 8, 2, 16, 1, 3000, 520),       # m = 123: the longest retained length the path holds at n = 256
-    (40, 8, 8, 16, 2, 20, 600),        # more work than one resident wave
+    (40, 8, 8, 16, 2, 20, 600),        # more pairs than SMs: one unit per pair, CTAs that walk several units
+    (3, 9, 3, 12, 4, 77, 400),         # n = 144 is not a multiple of 64: the plan declines, another kernel serves it
 ])
 def test_resident_parameter_path(B, H_q, H_kv, grid, R, T, ratio, recipe, monkeypatch):
     """The one-kernel path that keeps theta and U in shared memory (short blocks), forced where its plan applies."""
@@ -483,7 +484,10 @@ def test_resident_parameter_path(B, H_q, H_kv, grid, R, T, ratio, recipe, monkey
     shape = wl.Shape("resident", 1, B, H_q, H_kv, 128, grid, R, T, 1, "bf16", ratio_permille=ratio)
     p = tl.make_problem(shape, 4100 + B + R, T=T, T_cap=T + 7, recipe=recipe)
     counts = _fused_launches(lambda: _check(shape, p))
-    assert counts["resident"] == 1 and counts["fused"] + counts["scores"] == 0
+    if shape.n % 64 == 0:
+        assert counts["resident"] == 1 and counts["fused"] + counts["scores"] == 0
+    else:
+        assert counts["resident"] == 0
 
 
 @pytest.mark.parametrize("variant", ["mma", "tcgen05", "pair", "split"])
