@@ -99,6 +99,9 @@ KVC_API int kvc_retained_len(int n, int ratio_permille);
  * CTAs per (sequence, KV head)); "phases" forces the generic three-phase kernels that also serve fp32 storage. */
 KVC_API int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out);
 KVC_API int kvc_layer_destroy(kvc_layer* layer);
+/* Tells the handle that a capsule store it is used with has been written by something other than kvc_compress*: the next
+ * decode call on the handle reads the store only after the stream's previous kernel has finished (see kvc_decode_attend). */
+KVC_API int kvc_layer_capsules_written(kvc_layer* layer);
 
 /* Bytes of the capsule store for B sequences of R blocks:  K_tilde [B][H_kv][R][m_k][d] followed
  * by V_tilde [B][H_kv][R][m_v][d] (the compressed-cache term of App. D, Eq. 2, vision part), with m_k = m_v = m
@@ -131,7 +134,14 @@ KVC_API int kvc_compress(const kvc_layer* layer, const void* K_vis, const void* 
  * workspace: kvc_workspace_bytes(layer, B, R, T_max) bytes for the same B and R and any
  * T_max >= T; calls sharing a workspace must be stream-ordered.  All per-call device state (partials, arrival
  * words, status word) lives in the workspace, none in the layer handle: calls on one handle with different
- * workspaces may run concurrently on different streams. */
+ * workspaces may run concurrently on different streams.
+ * Early reads: the capsule store and the layer's parameters are fixed once written (Sec. 3.2: masks, reconstructors,
+ * bases and centring vectors are fixed at inference; the compressed cache is written at prefill).  A decode call may
+ * therefore begin to read them while the kernel that precedes it in the stream is still running; q, K_txt, V_txt, out
+ * and the workspace are touched only after that kernel has finished.  The first decode call on a handle after a
+ * kvc_compress / kvc_compress_ragged call on that handle reads the store late as well.  If anything else writes into a
+ * capsule store (a kernel of the caller that swaps cache pages in, say), call kvc_layer_capsules_written(layer) before
+ * the next decode call on it (copies issued with cudaMemcpyAsync need nothing: a kernel never overtakes a copy). */
 KVC_API int kvc_decode_attend(const kvc_layer* layer, const void* q, const void* capsules, int B, int R,
                       const void* K_txt, const void* V_txt, int T, int T_cap, void* out,
                       void* workspace, void* stream);

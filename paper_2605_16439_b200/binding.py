@@ -51,6 +51,7 @@ def _lib() -> C.CDLL:
         lib.kvc_layer_create.argtypes = [C.POINTER(kvc_layer_desc), C.POINTER(vp)]; lib.kvc_layer_create.restype = i
         lib.kvc_layer_destroy.argtypes = [vp]; lib.kvc_layer_destroy.restype = i
         lib.kvc_layer_m.argtypes = [vp]; lib.kvc_layer_m.restype = i
+        lib.kvc_layer_capsules_written.argtypes = [vp]; lib.kvc_layer_capsules_written.restype = i
         lib.kvc_layer_rows.argtypes = [vp, C.POINTER(i), C.POINTER(i)]; lib.kvc_layer_rows.restype = i
         lib.kvc_capsule_bytes.argtypes = [vp, i, i]; lib.kvc_capsule_bytes.restype = C.c_size_t
         lib.kvc_workspace_bytes.argtypes = [vp, i, i, i]; lib.kvc_workspace_bytes.restype = C.c_size_t

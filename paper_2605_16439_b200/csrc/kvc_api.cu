@@ -190,6 +190,7 @@ int kvc_layer_create(const kvc_layer_desc* desc, kvc_layer** out) {
   L->ms = (m + 15) / 16 * 16;
   L->G = desc->H_q / desc->H_kv;
   L->passthrough = pass ? 1 : 0;
+  L->capsules_fresh = 1;
   L->mode = mode;
   L->mk = key_side ? m : desc->n;
   L->mv = value_side ? m : desc->n;
@@ -232,6 +233,12 @@ int kvc_layer_destroy(kvc_layer* L) {
   return KVC_OK;
 }
 
+int kvc_layer_capsules_written(kvc_layer* L) {
+  if (!L) return KVC_ERR_ARG;
+  L->capsules_fresh = 1;
+  return KVC_OK;
+}
+
 int kvc_layer_m(const kvc_layer* L) { return L ? L->m : -1; }
 
 int kvc_layer_rows(const kvc_layer* L, int* key_rows, int* value_rows) {
@@ -265,6 +272,7 @@ int kvc_compress(const kvc_layer* L, const void* K_vis, const void* V_vis, int B
   const size_t kbytes = key_part_bytes(L, B, R), vbytes = kvc_capsule_bytes(L, B, R) - kbytes;
   void* Kc = capsules;
   void* Vc = static_cast<char*>(capsules) + kbytes;
+  const_cast<kvc_layer*>(L)->capsules_fresh = 1;
   cudaError_t e = cudaMemsetAsync(L->d_cstatus, 0, sizeof(int), st);   // status word of this compress call
   if (e != cudaSuccess) return cuda_status(e);
   // a side kept verbatim (rho = 0, or the one-sided modes) is a plain copy of its n rows per block
@@ -342,6 +350,8 @@ int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B
   a.split_base = ws + a.ws.off_split;
   a.resident_base = ws + a.ws.off_resident;
   a.R_b = R_b; a.T_b = T_b;
+  a.early_capsules = L->capsules_fresh ? 0 : 1;
+  const_cast<kvc_layer*>(L)->capsules_fresh = 0;
 
   // bf16 storage with TMA-compatible shapes and pointers: the whole of Algorithm 1 in one kernel
   {
@@ -409,6 +419,7 @@ int kvc_compress_ragged(const kvc_layer* L, const void* K_vis, const void* V_vis
       (T_cap > 0 && (!K_tail || !V_tail)))
     return KVC_ERR_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const_cast<kvc_layer*>(L)->capsules_fresh = 1;
   cudaError_t e = cudaMemsetAsync(L->d_cstatus, 0, sizeof(int), st);
   if (e != cudaSuccess) return cuda_status(e);
   void* Vc = capsules ? static_cast<char*>(capsules) + key_part_bytes(L, B, R_max) : nullptr;

@@ -110,6 +110,7 @@ struct kvc_layer {
   int m;                 // retained length
   int ms;                // row stride of score buffers (m rounded up to 16)
   int mode;              // KVC_MODE_KV, or one side kept verbatim (App. G): KVC_MODE_K_ONLY, KVC_MODE_V_ONLY
+  int capsules_fresh;    // set by kvc_compress*, cleared by the next decode call on the handle (which then reads the store late)
   int mk, mv;            // stored rows per block on the key side (n in the V-only mode) and on the value side (n in the K-only mode)
   int G;
   int passthrough;       // ratio_permille == 0
@@ -166,6 +167,7 @@ struct DecodeArgs {
   float2* fpart_ml;
   void* split_base;    // regions of the three-kernel bf16 path
   void* resident_base; // regions of the resident-parameter bf16 path
+  int early_capsules;  // the capsule store has not been written since the handle's last decode call began: kernels may read it early
   WsLayout ws;
 };
 

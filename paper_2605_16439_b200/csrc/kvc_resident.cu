@@ -42,10 +42,10 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   const int g = lane >> 2, t = lane & 3;
   const int h = blockIdx.x / a.cph, c = blockIdx.x - h * a.cph;
   const int units_h = a.B * a.cpb;
-  const int nsl = a.slots, np = a.mp / 16, G = a.G;
+  const int np = a.mp / 16, G = a.G;
   if (tid == 0) {
     for (int w = 0; w < RS_WARPS; ++w)
-      for (int s = 0; s < nsl; ++s) mbar_init(&full_bar[w][s], 1);
+      for (int s = 0; s < RS_MAX_SLOTS; ++s) mbar_init(&full_bar[w][s], 1);
     mbar_init(&par_bar, 1);
     fence_mbar_init();
   }
@@ -58,27 +58,41 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     tma_load_4d(sm + a.off_theta, &tmTh, 0, 0, 0, h, &par_bar);
     tma_load_4d(sm + a.off_U, &tmU, 0, 0, 0, h, &par_bar);
   }
-  grid_dep_wait();
-  grid_dep_launch();
-  if (blockIdx.x == 0 && tid == 0) *a.status = 0;
+  // Everything the stream's previous kernel may have written (queries, text rows, workspace) is touched only after the
+  // dependency wait; the capsule rows are not among it when a.early is set, and their first pieces are asked for at once.
+  bool waited = false;
+  auto dep_wait = [&]() {
+    if (waited) return;
+    grid_dep_wait();
+    grid_dep_launch();
+    if (blockIdx.x == 0 && tid == 0) *a.status = 0;
+    waited = true;
+  };
+  if (!a.early) dep_wait();
 
   const uint32_t sm_u = smem_addr(sm);
   const uint32_t th_u = sm_u + a.off_theta, U_u = sm_u + a.off_U;
-  unsigned char* ring_p = sm + a.off_ring + (size_t)warp * nsl * RS_PIECE_BYTES;
-  const uint32_t ring_u = smem_addr(ring_p);
   const uint32_t panel = (uint32_t)a.mp * 128u;                  // bytes of one 64-column panel of theta / U
   // ldmatrix lane roles: the lane supplies the address of row (lane & 7) of 8 x 8 matrix (lane >> 3)
   const int r8 = lane & 7, mat = lane >> 3;
   const int rowA = r8 + (mat & 1) * 8, selA = mat >> 1;          // plain: matrices (rows 0-7 | 8-15) x (k 0-7 | 8-15)
   const int rowT = r8 + (mat >> 1) * 8, selT = mat & 1;          // transposed: stored rows are the k index
 
-  uint32_t use_cnt = 0, iss_cnt = 0;                             // pieces consumed / issued by this warp so far
+  uint32_t pbits = 0;                                            // parity of the next completion of each of this warp's slots
   bool dead = false, par_ready = false;
 
   for (int u = c; u < units_h; u += a.cph) {
     const int b = u / a.cpb, part = u - b * a.cpb, bh = b * a.H_kv + h;
     const int ulo = part * a.items_b / a.cpb, uhi = (part + 1) * a.items_b / a.cpb;
-    const int wlo = ulo + (uhi - ulo) * warp / RS_WARPS, whi = ulo + (uhi - ulo) * (warp + 1) / RS_WARPS;
+    const int ni = uhi - ulo;
+    const int wlo = ulo + ni * warp / RS_WARPS, whi = ulo + ni * (warp + 1) / RS_WARPS;
+    // the ring pieces of the CTA go to the warps that have items in this unit (with fewer than 8 items: one item each)
+    const int nact = ni < RS_WARPS ? ni : RS_WARPS;
+    const int nsl = a.slots / nact < RS_MAX_SLOTS ? a.slots / nact : RS_MAX_SLOTS;
+    auto region = [&](int w) { return (size_t)(ni < RS_WARPS ? ni * w / RS_WARPS : w) * nsl * RS_PIECE_BYTES; };
+    unsigned char* ring_p = sm + a.off_ring + region(warp);
+    const uint32_t ring_u = smem_addr(ring_p);
+    uint32_t use_cnt = 0, iss_cnt = 0;                           // pieces consumed / issued by this warp in this unit
 
     // ---- this warp's load stream: the pieces of its items in the order it consumes them
     int p_k = wlo, p_idx = 0;
@@ -86,6 +100,7 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       if (p_k >= whi) return;
       const bool vis = p_k < a.R;
       const int half = vis ? np : RS_TEXT_ROWS / RS_PIECE_ROWS;
+      if (!vis) dep_wait();
       if (lane == 0) {
         const uint32_t slot = iss_cnt % (uint32_t)nsl;
         unsigned char* dst = ring_p + slot * RS_PIECE_BYTES;
@@ -103,8 +118,9 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       if (++p_idx == 2 * half) { p_idx = 0; ++p_k; }
     };
     auto wait_piece = [&]() -> uint32_t {
-      const uint32_t slot = use_cnt % (uint32_t)nsl, parity = (use_cnt / (uint32_t)nsl) & 1u;
+      const uint32_t slot = use_cnt % (uint32_t)nsl, parity = (pbits >> slot) & 1u;
       if (!dead && !mbar_wait_bounded(&full_bar[warp][slot], parity)) dead = true;
+      pbits ^= 1u << slot;
       __syncwarp();
       return ring_u + slot * RS_PIECE_BYTES;
     };
@@ -115,6 +131,7 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       issue_next();
     };
     for (int s = 0; s < nsl; ++s) issue_next();
+    dep_wait();
 
     float yacc[8][4];
 #pragma unroll
@@ -237,32 +254,33 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         rV0 = rV0 * cr0 + s0; rV1 = rV1 * cr1 + s1;
         rM0 = Mn0; rM1 = Mn1;
         rescale(cr0, cr1);
-        // ---- step 3: W^T[m x G] = U P^T, kept as B fragments for step 4 (row tiles of U inner, as above)
-        float wacc[RS_MAX_MP16][4];
+        // ---- step 3: W^T[m x G] = U P^T, kept as B fragments for step 4 (two accumulators per row tile: the chain over
+        // the n axis is the long one here)
+        uint32_t Wb[RS_MAX_MP16][2];
 #pragma unroll
-        for (int jt = 0; jt < RS_MAX_MP16; ++jt)
+        for (int jt = 0; jt < RS_MAX_MP16; ++jt) {
+          Wb[jt][0] = 0u; Wb[jt][1] = 0u;
+          if (jt < np) {
+            float w0[4] = {0.f, 0.f, 0.f, 0.f}, w1[4] = {0.f, 0.f, 0.f, 0.f};
+            const int jrow = 16 * jt + rowA;
+            const uint32_t rbase = U_u + (uint32_t)jrow * 128u;
 #pragma unroll
-          for (int e = 0; e < 4; ++e) wacc[jt][e] = 0.f;
-#pragma unroll
-        for (int ks = 0; ks < NT16; ++ks) {
-          const int ic = 2 * ks + selA;
-          const uint32_t cbase = U_u + (uint32_t)(ic >> 3) * panel;
-#pragma unroll
-          for (int jt = 0; jt < RS_MAX_MP16; ++jt) {
-            if (jt < np) {
-              const int jrow = 16 * jt + rowA;
+            for (int ks = 0; ks < NT16; ++ks) {
+              const int ic = 2 * ks + selA;
               uint32_t af[4];
-              ldsm_x4(af, cbase + (uint32_t)jrow * 128u + (uint32_t)(((ic & 7) ^ (jrow & 7)) << 4));
-              mma_bf16_16816(wacc[jt], af, Pb[ks][0], Pb[ks][1]);
+              ldsm_x4(af, rbase + (uint32_t)(ic >> 3) * panel + (uint32_t)(((ic & 7) ^ (jrow & 7)) << 4));
+              if (ks & 1) mma_bf16_16816(w1, af, Pb[ks][0], Pb[ks][1]);
+              else mma_bf16_16816(w0, af, Pb[ks][0], Pb[ks][1]);
             }
+            Wb[jt][0] = movm_t(pack2_bf16(w0[0] + w1[0], w0[1] + w1[1]));
+            Wb[jt][1] = movm_t(pack2_bf16(w0[2] + w1[2], w0[3] + w1[3]));
           }
         }
         // ---- step 4: y^T += V_tilde^T W^T
 #pragma unroll
         for (int pc = 0; pc < RS_MAX_MP16; ++pc) {
           if (pc < np) {
-            const uint32_t b0 = movm_t(pack2_bf16(wacc[pc][0], wacc[pc][1])), b1 = movm_t(pack2_bf16(wacc[pc][2], wacc[pc][3]));
-            value_piece(wait_piece(), b0, b1);
+            value_piece(wait_piece(), Wb[pc][0], Wb[pc][1]);
             done_piece();
           }
         }
@@ -329,25 +347,23 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         segs[16 + 2 * t] = rV0; segs[16 + 2 * t + 1] = rV1;
       }
     }
-    if (lane == 0) segs[24] = wlo < whi ? 1.f : 0.f;
     __syncthreads();
     const int head = warp;                                      // merge: warp = query head, lane = 4 channels
-    const size_t wstride = (size_t)nsl * RS_PIECE_BYTES / sizeof(float);
-    const float* seg0 = reinterpret_cast<const float*>(sm + a.off_ring);
+    auto has_items = [&](int w) { return ni * (w + 1) / RS_WARPS > ni * w / RS_WARPS; };
     if (head < G) {
       float Mx = -INFINITY;
 #pragma unroll
       for (int w = 0; w < RS_WARPS; ++w) {
-        const float* ss = seg0 + w * wstride + 8 * D;
-        if (ss[24] != 0.f) Mx = fmaxf(Mx, ss[head]);
+        const float* ss = reinterpret_cast<const float*>(sm + a.off_ring + region(w)) + 8 * D;
+        if (has_items(w)) Mx = fmaxf(Mx, ss[head]);
       }
       float Ls = 0.f, Vs = 0.f;
       float4 y = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
       for (int w = 0; w < RS_WARPS; ++w) {
-        const float* sy = seg0 + w * wstride;
+        const float* sy = reinterpret_cast<const float*>(sm + a.off_ring + region(w));
         const float* ss = sy + 8 * D;
-        if (ss[24] != 0.f) {
+        if (has_items(w)) {
           const float f = fast_exp2(ss[head] - Mx);
           Ls = fmaf(f, ss[8 + head], Ls);
           Vs = fmaf(f, ss[16 + head], Vs);
@@ -407,6 +423,7 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     }
     __syncthreads();                    // the rings take the next unit's pieces
   }
+  dep_wait();
   if (dead && lane == 0) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
 }
 
@@ -435,13 +452,14 @@ ResidentPlan plan_resident(const kvc_layer* L, int B, int R, int T) {
   p.grid = p.cph * H_kv;
   p.par_bytes = (uint32_t)p.ncg * (uint32_t)p.mp * 128u;
   const uint32_t fixed = 2u * p.par_bytes + 1024u + 2048u;
-  if (fixed + 2u * RS_WARPS * RS_PIECE_BYTES > RS_SMEM_LIMIT) return p;
-  p.slots = (int)((RS_SMEM_LIMIT - fixed) / (RS_WARPS * RS_PIECE_BYTES));
-  if (p.slots > RS_MAX_SLOTS) p.slots = RS_MAX_SLOTS;
+  if (fixed + 3u * RS_WARPS * RS_PIECE_BYTES > RS_SMEM_LIMIT) return p;
+  p.slots = (int)((RS_SMEM_LIMIT - fixed) / RS_PIECE_BYTES);
+  if (p.slots > RS_MAX_SLOTS * RS_WARPS) p.slots = RS_MAX_SLOTS * RS_WARPS;
+  if (p.slots < 3 * RS_WARPS) return p;            // a warp's region also stages its result (4 KB + statistics) at the end of a unit
   p.off_theta = 0;
   p.off_U = p.par_bytes;
   p.off_ring = 2u * p.par_bytes;
-  p.smem = (size_t)p.off_ring + (size_t)p.slots * RS_WARPS * RS_PIECE_BYTES + 1024;
+  p.smem = (size_t)p.off_ring + (size_t)p.slots * RS_PIECE_BYTES + 1024;
   p.ok = 1;
   return p;
 }
@@ -505,6 +523,7 @@ cudaError_t launch_resident(const kvc_layer* L, const DecodeArgs& a, const Resid
   ra.status = a.status;
   ra.B = B; ra.H_kv = H_kv; ra.G = a.G; ra.R = R; ra.m = m; ra.mp = p.mp; ra.n = n; ra.T = a.T;
   ra.ncg = p.ncg; ra.ct = p.ct; ra.items_b = p.items_b; ra.cpb = p.cpb; ra.cph = p.cph; ra.slots = p.slots;
+  ra.early = a.early_capsules;
   ra.par_bytes = p.par_bytes;
   ra.off_theta = p.off_theta; ra.off_U = p.off_U; ra.off_ring = p.off_ring;
   void (*kernel)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, ResidentArgs) =

@@ -15,7 +15,7 @@ constexpr int RS_PIECE_ROWS = 16;                 // rows per ring piece (4 KB: 
 constexpr uint32_t RS_PIECE_BYTES = RS_PIECE_ROWS * 256u;
 constexpr int RS_TEXT_ROWS = 64;                  // text rows per item
 constexpr int RS_WARPS = 8;
-constexpr int RS_MAX_SLOTS = 6;                   // pieces in flight per warp
+constexpr int RS_MAX_SLOTS = 8;                   // pieces in flight per warp
 constexpr int RS_MAX_CPB = 16;                    // units per (sequence, KV head)
 constexpr int RS_MAX_MP16 = 8;                    // m <= 128
 
@@ -28,7 +28,7 @@ struct ResidentPlan {
   int cpb;           // units per (sequence, KV head)
   int cph;           // CTAs per KV head
   int grid;
-  int slots;         // ring pieces per warp
+  int slots;         // ring pieces of the CTA; a unit deals them to the warps that have items
   uint32_t par_bytes;
   uint32_t off_theta, off_U, off_ring;
   size_t smem;
@@ -56,6 +56,7 @@ struct ResidentArgs {
   int* status;
   int B, H_kv, G, R, m, mp, n, T;
   int ncg, ct, items_b, cpb, cph, slots;
+  int early;         // 1: vision pieces may be loaded before the stream's previous kernel has finished (see kvc.h)
   uint32_t par_bytes;
   uint32_t off_theta, off_U, off_ring;
 };
