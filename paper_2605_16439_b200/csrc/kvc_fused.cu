@@ -105,7 +105,7 @@ fused_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             const int j0 = c * 16 * a.JC;
             mbar_expect_tx(bar, a.par_bytes + 2 * a.k_half_bytes);
             tma_load_4d(dst, tp, 0, j0, 0, h, bar);                  // parameters: never written by this library
-            if (first) { grid_dep_wait(); first = false; }            // everything else may come from the stream's previous kernel
+            if (first && !a.early) { grid_dep_wait(); first = false; }   // the capsule rows: late unless known to be settled
             tma_load_5d(dst + a.par_bytes, tk, 0, j0, r0, h, b0, bar);
             tma_load_5d(dst + a.par_bytes + a.k_half_bytes, tk, 64, j0, r0, h, b0, bar);
           }
@@ -1116,6 +1116,7 @@ cudaError_t launch_fused(const kvc_layer* L, const DecodeArgs& a, const FusedPla
   fa.cnt = a.fcnt;
   fa.token = a.token;
   fa.status = a.status;
+  fa.early = a.early_capsules;
 
   ProfScope prof(p.tc == 2 ? KVC_KERNEL_FUSED_PAIR : (p.tc ? KVC_KERNEL_FUSED_TC : KVC_KERNEL_FUSED), st);
   if (p.tc) return launch_fused_tc_kernel(tm, fa, p, st);

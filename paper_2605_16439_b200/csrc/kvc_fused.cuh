@@ -35,6 +35,7 @@ struct FusedArgs {
   unsigned long long* cnt;   // [B*H_kv] arrival words in the caller's workspace (see arrive_is_last)
   unsigned int token;        // this call's token, never 0
   int* status;        // device status word
+  int early;          // 1: capsule rows may be loaded before the stream's previous kernel has finished (see kvc.h)
 };
 
 // shared-memory barriers of one CTA

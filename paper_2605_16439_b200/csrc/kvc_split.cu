@@ -182,6 +182,7 @@ cudaError_t launch_split(const kvc_layer* L, const DecodeArgs& a, const SplitPla
   sa.tpy = reinterpret_cast<float*>(ws + w.off_tpy);
   sa.tpml = reinterpret_cast<float2*>(ws + w.off_tpml);
   sa.status = a.status;
+  sa.early = a.early_capsules;
   sa.B = B; sa.H_kv = H_kv; sa.G = G; sa.R = R; sa.m = m; sa.n = n; sa.T = a.T;
   sa.rows_h = p.rows_h; sa.ntile = p.ntile; sa.NS = p.NS; sa.NW = p.NW; sa.ms = p.ms; sa.nk1 = p.nk1;
   sa.npass = p.npass; sa.prow = p.prow; sa.nbox = p.nbox; sa.brow = p.brow; sa.tmem_cols = p.tmem_cols;

@@ -69,6 +69,7 @@ struct SplitArgs {
   float2* tpml;      // [B*H_kv][chunks][G]
   int* cnt;
   int* status;
+  int early;         // 1: capsule rows may be loaded before the stream's previous kernel has finished (see kvc.h)
   int B, H_kv, G, R, m, n, T;
   int rows_h, ntile, NS, NW, ms, nk1, npass, prow, nbox, brow, tmem_cols;
   int e_stages; uint32_t e_stage_bytes;

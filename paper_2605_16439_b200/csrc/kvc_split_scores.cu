@@ -46,7 +46,7 @@ split_scores_kernel(const __grid_constant__ CUtensorMap tmK, const SplitArgs a) 
         if (++pt == a.s_tiles_bh) { pt = 0; ++pbh; }
       }
     }
-    grid_dep_wait();                              // the capsules and the queries may come from the stream's previous kernel
+    if (!a.early) grid_dep_wait();                // the capsule rows: late unless known to be settled (the queries are read by the consumers, after their wait)
     uint32_t slot = 0, phase = 1;
     int bh = (int)(lo / a.s_tiles_bh), t = (int)(lo - (long long)bh * a.s_tiles_bh) - 1;
     for (int it = (int)(hi - lo); it > 0; --it) {
