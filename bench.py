@@ -43,6 +43,9 @@ KERNEL_SOURCES = {
     "fused": ("kvc_fused.cu", "kvc_fused.cuh", "kvc_tma.cuh", "kvc_async.cuh"),
     "fused_tc": ("kvc_fused_tc.cu", "kvc_fused.cuh", "kvc_tcgen05.cuh", "kvc_tma.cuh", "kvc_async.cuh"),
     "fused_pair": ("kvc_fused_tc.cu", "kvc_fused.cuh", "kvc_tcgen05.cuh", "kvc_tma.cuh", "kvc_async.cuh"),
+    "resident": ("kvc_resident.cu", "kvc_resident.cuh", "kvc_tma.cuh", "kvc_async.cuh"),
+    "split_scores+split_expand+split_output": ("kvc_split_scores.cu", "kvc_split_expand.cu", "kvc_split_output.cu", "kvc_split.cuh",
+                                               "kvc_tcgen05.cuh", "kvc_tma.cuh", "kvc_async.cuh"),
 }
 NCU_TRAFFIC_BYTES = {
     ("fused", "config1-llava-next-7b"): (209.4e6, "stale"),
