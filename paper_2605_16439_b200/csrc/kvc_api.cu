@@ -358,15 +358,17 @@ int decode_common(const kvc_layer* L, const void* q, const void* capsules, int B
     // R == 0 (text rows only, the uncompressed comparator): the same kernel with text stages only
     // rho = 0 stores K and V verbatim: vision rows and text rows are attended as plain rows by the text-only mode
     const bool plain = R == 0 || L->passthrough;
-    // one-sided modes and per-sequence lengths are served by the three-phase kernels below
-    const bool one_sided = (R > 0 && L->mode != KVC_MODE_KV) || R_b || T_b;
+    // one-sided modes are served by the three-phase kernels below; so are per-sequence lengths, except on the shapes the
+    // resident-parameter kernel takes (it reads the lengths itself)
+    const bool ragged = R_b != nullptr || T_b != nullptr;
+    const bool one_sided = (R > 0 && L->mode != KVC_MODE_KV) || ragged;
     const uintptr_t align = reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(capsules) |
                             reinterpret_cast<uintptr_t>(out) | (T > 0 ? reinterpret_cast<uintptr_t>(K_txt) |
                             reinterpret_cast<uintptr_t>(V_txt) : 0) | reinterpret_cast<uintptr_t>(L->desc.mu);
     // Short blocks whose theta and U fit shared memory (n <= 256, m <= 128, G <= 8) take the resident-parameter kernel: on
     // the n = 256, G = 7, m = 103 shape it ran ahead of the other one-kernel variants at every batch measured (1, 4, 16:
     // 19.2 / 19.5 / 42.4 us against 22.4 / 23.5 / 83.7 us).  KVC_EXPANSION=resident forces it, any other value keeps it off.
-    if (!plain && !one_sided && (align & 15) == 0 && (L->use_tc == 4 || L->use_tc == 0)) {
+    if (!plain && L->mode == KVC_MODE_KV && (align & 15) == 0 && (L->use_tc == 4 || L->use_tc == 0)) {
       const ResidentPlan rp = plan_resident(L, B, R, T);
       if (rp.ok) {
         bool encoded = false;

@@ -68,7 +68,14 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     if (blockIdx.x == 0 && tid == 0) *a.status = 0;
     waited = true;
   };
-  if (!a.early) dep_wait();
+  const bool ragged = a.R_b != nullptr || a.T_b != nullptr;     // the lengths are inputs like the queries: read after the wait
+  if (!a.early || ragged) dep_wait();
+  if (ragged) __syncthreads();                                  // the status word is cleared before a length is reported
+  if (ragged && blockIdx.x == 0)
+    for (int bb = tid; bb < a.B; bb += RS_THREADS) {
+      const bool bad = (a.R_b && (a.R_b[bb] < 0 || a.R_b[bb] > a.R)) || (a.T_b && (a.T_b[bb] < 0 || a.T_b[bb] > a.T));
+      if (bad) atomicExch(a.status, (int)KVC_ERR_BOUNDS);
+    }
 
   const uint32_t sm_u = smem_addr(sm);
   const uint32_t th_u = sm_u + a.off_theta, U_u = sm_u + a.off_U;
@@ -85,6 +92,11 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     const int b = u / a.cpb, part = u - b * a.cpb, bh = b * a.H_kv + h;
     const int ulo = part * a.items_b / a.cpb, uhi = (part + 1) * a.items_b / a.cpb;
     const int ni = uhi - ulo;
+    // blocks and text rows this sequence takes part with; an item beyond them is skipped (no loads, no arithmetic)
+    int Rb = a.R, Tb = a.T;
+    if (a.R_b) { Rb = a.R_b[b]; Rb = Rb < 0 ? 0 : (Rb > a.R ? a.R : Rb); }
+    if (a.T_b) { Tb = a.T_b[b]; Tb = Tb < 0 ? 0 : (Tb > a.T ? a.T : Tb); }
+    auto valid = [&](int k) { return k < a.R ? k < Rb : (k - a.R) * RS_TEXT_ROWS < Tb; };
     const int wlo = ulo + ni * warp / RS_WARPS, whi = ulo + ni * (warp + 1) / RS_WARPS;
     // the ring pieces of the CTA go to the warps that have items in this unit (with fewer than 8 items: one item each)
     const int nact = ni < RS_WARPS ? ni : RS_WARPS;
@@ -97,6 +109,7 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     // ---- this warp's load stream: the pieces of its items in the order it consumes them
     int p_k = wlo, p_idx = 0;
     auto issue_next = [&]() {
+      if (p_idx == 0) while (p_k < whi && !valid(p_k)) ++p_k;
       if (p_k >= whi) return;
       const bool vis = p_k < a.R;
       const int half = vis ? np : RS_TEXT_ROWS / RS_PIECE_ROWS;
@@ -189,6 +202,7 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     };
 
     for (int k = wlo; k < whi; ++k) {
+      if (!valid(k)) continue;
       if (k < a.R) {
         // ---- step 1: S^T, kept as B fragments (k = key rows, n = heads)
         uint32_t Sb[RS_MAX_MP16][2];
@@ -292,8 +306,8 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         for (int pc = 0; pc < 4; ++pc) {
           score_piece(wait_piece(), sc[pc]);
           const int row = base + pc * RS_PIECE_ROWS + g;
-          if (row >= a.T) { sc[pc][0] = -INFINITY; sc[pc][1] = -INFINITY; }
-          if (row + 8 >= a.T) { sc[pc][2] = -INFINITY; sc[pc][3] = -INFINITY; }
+          if (row >= Tb) { sc[pc][0] = -INFINITY; sc[pc][1] = -INFINITY; }
+          if (row + 8 >= Tb) { sc[pc][2] = -INFINITY; sc[pc][3] = -INFINITY; }
           done_piece();
         }
         float m0 = -INFINITY, m1 = -INFINITY;
@@ -306,15 +320,15 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         const float Mn0 = fmaxf(rM0, m0), Mn1 = fmaxf(rM1, m1);
         const float cr0 = rM0 == -INFINITY ? 0.f : fast_exp2(rM0 - Mn0), cr1 = rM1 == -INFINITY ? 0.f : fast_exp2(rM1 - Mn1);
         float s0 = 0.f, s1 = 0.f;
-        uint32_t Tb[4][2];
+        uint32_t Tb_frag[4][2];
 #pragma unroll
         for (int pc = 0; pc < 4; ++pc) {
           const float p0 = fast_exp2(sc[pc][0] - Mn0), p1 = fast_exp2(sc[pc][1] - Mn1);
           const float p2 = fast_exp2(sc[pc][2] - Mn0), p3 = fast_exp2(sc[pc][3] - Mn1);
           s0 += p0 + p2;
           s1 += p1 + p3;
-          Tb[pc][0] = movm_t(pack2_bf16(p0, p1));
-          Tb[pc][1] = movm_t(pack2_bf16(p2, p3));
+          Tb_frag[pc][0] = movm_t(pack2_bf16(p0, p1));
+          Tb_frag[pc][1] = movm_t(pack2_bf16(p2, p3));
         }
         over_rows(s0, s1, false);
         rL0 = rL0 * cr0 + s0; rL1 = rL1 * cr1 + s1;
@@ -323,7 +337,17 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         rescale(cr0, cr1);
 #pragma unroll
         for (int pc = 0; pc < 4; ++pc) {
-          value_piece(wait_piece(), Tb[pc][0], Tb[pc][1]);
+          const uint32_t st = wait_piece();
+          if (a.T_b) {
+            // rows past the sequence's text length hold whatever the caller's buffer holds (a zero probability does not
+            // silence a NaN): cleared in shared memory before the product
+            const int nv = Tb - (base + pc * RS_PIECE_ROWS);
+            if (nv < RS_PIECE_ROWS && lane < 16)
+              for (int r = nv < 0 ? 0 : nv; r < RS_PIECE_ROWS; ++r)
+                asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};\n" ::"r"(st + (uint32_t)(lane >> 3) * RS_HALF + (uint32_t)r * 128u + (uint32_t)(lane & 7) * 16u), "r"(0u) : "memory");
+            __syncwarp();
+          }
+          value_piece(st, Tb_frag[pc][0], Tb_frag[pc][1]);
           done_piece();
         }
       }
@@ -363,7 +387,7 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       for (int w = 0; w < RS_WARPS; ++w) {
         const float* sy = reinterpret_cast<const float*>(sm + a.off_ring + region(w));
         const float* ss = sy + 8 * D;
-        if (has_items(w)) {
+        if (has_items(w) && ss[head] != -INFINITY) {
           const float f = fast_exp2(ss[head] - Mx);
           Ls = fmaf(f, ss[8 + head], Ls);
           Vs = fmaf(f, ss[16 + head], Vs);
@@ -377,7 +401,7 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       y.z = fmaf(Vs, __uint_as_float(mraw.y << 16), y.z);
       y.w = fmaf(Vs, __uint_as_float(mraw.y & 0xffff0000u), y.w);
       if (a.cpb == 1) {
-        const float inv = 1.f / Ls;
+        const float inv = Ls > 0.f ? 1.f / Ls : 0.f;          // a sequence without any row: a zero output row
         *reinterpret_cast<uint2*>(a.out + ((size_t)bh * G + head) * D + lane * 4) =
             make_uint2(pack2_bf16(y.x * inv, y.y * inv), pack2_bf16(y.z * inv, y.w * inv));
       } else {
@@ -412,11 +436,11 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         float4 y = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int s = 0; s < RS_MAX_CPB; ++s) {
-          const float f = fast_exp2(st[s].x - Ms);
+          const float f = st[s].x == -INFINITY ? 0.f : fast_exp2(st[s].x - Ms);
           den = fmaf(f, st[s].y, den);
           y.x = fmaf(f, ys[s].x, y.x); y.y = fmaf(f, ys[s].y, y.y); y.z = fmaf(f, ys[s].z, y.z); y.w = fmaf(f, ys[s].w, y.w);
         }
-        const float inv = 1.f / den;
+        const float inv = den > 0.f ? 1.f / den : 0.f;
         *reinterpret_cast<uint2*>(a.out + ((size_t)bh * G + head) * D + lane * 4) =
             make_uint2(pack2_bf16(y.x * inv, y.y * inv), pack2_bf16(y.z * inv, y.w * inv));
       }
@@ -524,6 +548,7 @@ cudaError_t launch_resident(const kvc_layer* L, const DecodeArgs& a, const Resid
   ra.B = B; ra.H_kv = H_kv; ra.G = a.G; ra.R = R; ra.m = m; ra.mp = p.mp; ra.n = n; ra.T = a.T;
   ra.ncg = p.ncg; ra.ct = p.ct; ra.items_b = p.items_b; ra.cpb = p.cpb; ra.cph = p.cph; ra.slots = p.slots;
   ra.early = a.early_capsules;
+  ra.R_b = a.R_b; ra.T_b = a.T_b;
   ra.par_bytes = p.par_bytes;
   ra.off_theta = p.off_theta; ra.off_U = p.off_U; ra.off_ring = p.off_ring;
   void (*kernel)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, ResidentArgs) =

@@ -56,6 +56,8 @@ struct ResidentArgs {
   int* status;
   int B, H_kv, G, R, m, mp, n, T;
   int ncg, ct, items_b, cpb, cph, slots;
+  const int* R_b;    // per-sequence block counts (<= R) and text lengths (<= T), device arrays; nullptr: R and T for all
+  const int* T_b;
   int early;         // 1: vision pieces may be loaded before the stream's previous kernel has finished (see kvc.h)
   uint32_t par_bytes;
   uint32_t off_theta, off_U, off_ring;

@@ -31,13 +31,14 @@ def _status(layer, B, R, T, ws):
     return kvc.kvc_read_device_status(layer, B, R, T, ws)
 
 
+@pytest.mark.parametrize("grid", [12, 8, 16])          # n = 144: three-phase kernels; n = 64, 256 in bf16: the resident-parameter kernel
 @pytest.mark.parametrize("mode", ["kv", "k", "v"])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_mixed_block_counts_and_text_lengths_in_one_call(dtype, mode):
+def test_mixed_block_counts_and_text_lengths_in_one_call(dtype, mode, grid):
     R_b = [0, 1, 5, 5, 1, 0, 0, 3]
     T_b = [1, 0, 257, 0, 257, 257, 0, 64]
     B, R_max, T_cap = len(R_b), 5, 300
-    shape = wl.Shape("ragged", 1, B, 6, 2, 128, 12, R_max, T_cap, 1, dtype, 600)      # n = 144, G = 3
+    shape = wl.Shape("ragged", 1, B, 6, 2, 128, grid, R_max, T_cap, 1, dtype, 600)      # G = 3
     p = tl.make_problem(shape, 811, T=T_cap, T_cap=T_cap, recipe="peaked")
     layer = tl.gpu_layer(shape, p, DEV, mode)
     caps = kvc.alloc_capsules(layer, B, R_max, DEV)
@@ -52,9 +53,17 @@ def test_mixed_block_counts_and_text_lengths_in_one_call(dtype, mode):
     ws = kvc.alloc_workspace(layer, B, R_max, T_cap, DEV)
     ws.fill_(0xFF)                                       # NaN patterns: stale scratch must not matter either
     out = torch.full((B, shape.H_q, 128), float("nan"), dtype=wl.torch_dtype(dtype), device=DEV)
+    kvc.kvc_profile_start(16)
     kvc.kvc_decode_attend_ragged(layer, p["q"].to(DEV), caps, B, R_max, _i32(R_b), K_txt, V_txt, max(T_b), _i32(T_b),
                                  T_cap, out, ws)
     torch.cuda.synchronize()
+    kvc.kvc_profile_stop()
+    launches = {k: v[1] for k, v in kvc.kvc_profile_read().items()}
+    kvc.kvc_profile_start(0)
+    kvc.kvc_profile_stop()
+    # short blocks in bf16 take the resident-parameter kernel, which reads the lengths itself; everything else the three-phase kernels
+    assert launches["resident"] == (1 if (dtype == "bf16" and mode == "kv" and grid in (8, 16)) else 0)
+    assert launches["scores"] == 1 - launches["resident"]
     assert _status(layer, B, R_max, max(T_b), ws) == 0
     K_o, V_o = orc.compress(tl.np64(p["K_vis"]), tl.np64(p["V_vis"]), p["idx"].numpy(), tl.np64(p["U"]), tl.np64(p["mu"]),
                             shape.n, False, mode)
@@ -90,17 +99,18 @@ def caps_full(layer, p, B, R):
     return caps
 
 
+@pytest.mark.parametrize("grid", [12, 16])
 @pytest.mark.parametrize("mode", ["kv", "k", "v"])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_ragged_compress_with_left_over_rows_then_decode(dtype, mode):
+def test_ragged_compress_with_left_over_rows_then_decode(dtype, mode, grid):
     """Vision runs of 0, 1, 5 whole blocks and runs that are not a whole number of blocks: the left-over rows land in
     front of the text rows, bit-exact; the capsules of the whole blocks match the oracle; the decode on top matches."""
-    n, R_max, T_cap = 144, 5, 400
+    n, R_max, T_cap = grid * grid, 5, grid * grid + 300
     N_v = [0, n, 5 * n, 2 * n + 7, 3, 2 * n + (n - 1), 4 * n + 64]
     T_own = [9, 0, 130, 1, 0, 257, 0]
     B = len(N_v)
     N_cap = 6 * n
-    shape = wl.Shape("ragged", 1, B, 8, 2, 128, 12, 6, T_cap, 1, dtype, 600)
+    shape = wl.Shape("ragged", 1, B, 8, 2, 128, grid, 6, T_cap, 1, dtype, 600)
     p = tl.make_problem(shape, 907, T=T_cap, T_cap=T_cap, recipe="structured")
     dt = wl.torch_dtype(dtype)
     layer = tl.gpu_layer(shape, p, DEV, mode)
@@ -147,14 +157,15 @@ def test_ragged_compress_with_left_over_rows_then_decode(dtype, mode):
     tl.assert_close(tl.np64(out), want, dtype, "ragged compress + decode")
 
 
-def test_lengths_out_of_range_are_clamped_and_reported():
-    shape = wl.Shape("ragged", 1, 3, 4, 2, 128, 8, 2, 40, 1, "f32", 500)            # n = 64
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])          # three-phase kernels / the resident-parameter kernel
+def test_lengths_out_of_range_are_clamped_and_reported(dtype):
+    shape = wl.Shape("ragged", 1, 3, 4, 2, 128, 8, 2, 40, 1, dtype, 500)            # n = 64
     p = tl.make_problem(shape, 33, T=40, T_cap=40)
     layer = tl.gpu_layer(shape, p, DEV)
     B, R, n = 3, 2, 64
     caps = caps_full(layer, p, B, R)
     ws = kvc.alloc_workspace(layer, B, R, 40, DEV)
-    out = torch.empty((B, 4, 128), dtype=torch.float32, device=DEV)
+    out = torch.empty((B, 4, 128), dtype=wl.torch_dtype(dtype), device=DEV)
     args = (p["q"].to(DEV), caps, B, R)
     kvc.kvc_decode_attend_ragged(layer, *args, _i32([2, 3, -1]), p["K_txt"].to(DEV), p["V_txt"].to(DEV), 40, _i32([40, 41, 40]),
                                  40, out, ws)
@@ -163,14 +174,14 @@ def test_lengths_out_of_range_are_clamped_and_reported():
     K_o, V_o, _ = tl.oracle_run(shape, p)
     want = orc.decode_attend_ragged(tl.np64(p["q"]), K_o, V_o, tl.np64(p["theta"]), tl.np64(p["U"]), tl.np64(p["mu"]),
                                     tl.np64(p["K_txt"]), tl.np64(p["V_txt"]), [2, 2, 0], [40, 40, 40])
-    tl.assert_close(tl.np64(out), want, "f32", "clamped lengths")
+    tl.assert_close(tl.np64(out), want, dtype, "clamped lengths")
     kvc.kvc_decode_attend_ragged(layer, *args, _i32([2, 1, 0]), p["K_txt"].to(DEV), p["V_txt"].to(DEV), 40, _i32([40, 0, 7]),
                                  40, out, ws)
     torch.cuda.synchronize()
     assert _status(layer, B, R, 40, ws) == 0             # the next call clears it
     # compress: a run longer than the buffer, more blocks than R_max, more left-over rows than T_cap
     R_b, T_b = _i32([0, 0, 0]), _i32([0, 0, 0])
-    tail = torch.empty((B, 2, 5, 128), dtype=torch.float32, device=DEV)
+    tail = torch.empty((B, 2, 5, 128), dtype=wl.torch_dtype(dtype), device=DEV)
     Kv, Vv = p["K_vis"].to(DEV), p["V_vis"].to(DEV)
     for N_v, want_R, want_T in (([129, 64, 0], [2, 1, 0], [0, 0, 0]), ([128, 70, 5], [2, 1, 0], [0, 5, 5])):
         kvc.kvc_compress_ragged(layer, Kv, Vv, B, 2 * n, _i32(N_v), R, caps, tail, tail.clone(), 5, R_b, T_b)
