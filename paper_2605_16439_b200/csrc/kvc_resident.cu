@@ -28,7 +28,8 @@ __device__ __forceinline__ uint32_t movm_t(uint32_t x) {
   return y;
 }
 
-template <int NT16>
+// RAGGED: per-sequence block counts and text lengths are read from device arrays (the uniform instance carries none of that code)
+template <int NT16, bool RAGGED>
 __global__ void __launch_bounds__(RS_THREADS, 1)
 resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                        const __grid_constant__ CUtensorMap tmKt, const __grid_constant__ CUtensorMap tmVt,
@@ -68,7 +69,7 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     if (blockIdx.x == 0 && tid == 0) *a.status = 0;
     waited = true;
   };
-  const bool ragged = a.R_b != nullptr || a.T_b != nullptr;     // the lengths are inputs like the queries: read after the wait
+  constexpr bool ragged = RAGGED;                               // the lengths are inputs like the queries: read after the wait
   if (!a.early || ragged) dep_wait();
   if (ragged) __syncthreads();                                  // the status word is cleared before a length is reported
   if (ragged && blockIdx.x == 0)
@@ -94,9 +95,9 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     const int ni = uhi - ulo;
     // blocks and text rows this sequence takes part with; an item beyond them is skipped (no loads, no arithmetic)
     int Rb = a.R, Tb = a.T;
-    if (a.R_b) { Rb = a.R_b[b]; Rb = Rb < 0 ? 0 : (Rb > a.R ? a.R : Rb); }
-    if (a.T_b) { Tb = a.T_b[b]; Tb = Tb < 0 ? 0 : (Tb > a.T ? a.T : Tb); }
-    auto valid = [&](int k) { return k < a.R ? k < Rb : (k - a.R) * RS_TEXT_ROWS < Tb; };
+    if (RAGGED && a.R_b) { Rb = a.R_b[b]; Rb = Rb < 0 ? 0 : (Rb > a.R ? a.R : Rb); }
+    if (RAGGED && a.T_b) { Tb = a.T_b[b]; Tb = Tb < 0 ? 0 : (Tb > a.T ? a.T : Tb); }
+    auto valid = [&](int k) { return !RAGGED || (k < a.R ? k < Rb : (k - a.R) * RS_TEXT_ROWS < Tb); };
     const int wlo = ulo + ni * warp / RS_WARPS, whi = ulo + ni * (warp + 1) / RS_WARPS;
     // the ring pieces of the CTA go to the warps that have items in this unit (with fewer than 8 items: one item each)
     const int nact = ni < RS_WARPS ? ni : RS_WARPS;
@@ -338,7 +339,7 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
 #pragma unroll
         for (int pc = 0; pc < 4; ++pc) {
           const uint32_t st = wait_piece();
-          if (a.T_b) {
+          if (RAGGED && a.T_b) {
             // rows past the sequence's text length hold whatever the caller's buffer holds (a zero probability does not
             // silence a NaN): cleared in shared memory before the product
             const int nv = Tb - (base + pc * RS_PIECE_ROWS);
@@ -551,9 +552,12 @@ cudaError_t launch_resident(const kvc_layer* L, const DecodeArgs& a, const Resid
   ra.R_b = a.R_b; ra.T_b = a.T_b;
   ra.par_bytes = p.par_bytes;
   ra.off_theta = p.off_theta; ra.off_U = p.off_U; ra.off_ring = p.off_ring;
+  const bool rg = a.R_b != nullptr || a.T_b != nullptr;
   void (*kernel)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, ResidentArgs) =
-      n == 64 ? resident_decode_kernel<4> : n == 128 ? resident_decode_kernel<8> : n == 192 ? resident_decode_kernel<12>
-                                                                                            : resident_decode_kernel<16>;
+      n == 64    ? (rg ? resident_decode_kernel<4, true> : resident_decode_kernel<4, false>)
+      : n == 128 ? (rg ? resident_decode_kernel<8, true> : resident_decode_kernel<8, false>)
+      : n == 192 ? (rg ? resident_decode_kernel<12, true> : resident_decode_kernel<12, false>)
+                 : (rg ? resident_decode_kernel<16, true> : resident_decode_kernel<16, false>);
   cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), p.smem);
   if (e != cudaSuccess) return e;
   ProfScope prof(KVC_KERNEL_RESIDENT, st);
