@@ -36,8 +36,9 @@ NOMINAL_HBM_GBS = 8000.0        # nominal HBM3e bandwidth: the roofline fraction
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from one ncu capture,
 # keyed by (kernel, workload name): (bytes, digest of the kernel's source files when the counters were taken).  The
-# captures ran at 4 decode steps (text length 130 / 258); a text row adds exactly 2 * B * H_kv * d * 2 bytes, and the
-# figure here is scaled by that amount to the mid-run text length.  When the sources no longer match the digest the
+# captures ran at 4 decode steps (text length 130 / 258 / 514; profiles/*.md give the commands); a text row adds exactly
+# 2 * B * H_kv * d * 2 bytes, and the figure here is scaled by that amount to the mid-run text length.  For the three-kernel
+# path the figure is the sum over its three kernels (one layer call).  When the sources no longer match the digest the
 # bench reports traffic = null: the counters belong to another kernel.
 KERNEL_SOURCES = {
     "fused": ("kvc_fused.cu", "kvc_fused.cuh", "kvc_tma.cuh", "kvc_async.cuh"),
@@ -48,8 +49,9 @@ KERNEL_SOURCES = {
                                                "kvc_tcgen05.cuh", "kvc_tma.cuh", "kvc_async.cuh"),
 }
 NCU_TRAFFIC_BYTES = {
-    ("fused", "config1-llava-next-7b"): (209.4e6, "stale"),
-    ("fused_pair", "config2-qwen2-vl-7b"): (135.7e6, "stale"),
+    ("fused", "config1-llava-next-7b"): (208.4e6, "5e7f612f8ac6"),
+    ("split_scores+split_expand+split_output", "config2-qwen2-vl-7b"): (147.9e6, "0ca50a288632"),
+    ("resident", "config3-internvl3-8b-video"): (36.0e6, "7d4a0953cecd"),
 }
 
 
