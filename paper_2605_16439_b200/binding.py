@@ -170,6 +170,11 @@ def alloc_workspace(layer: Layer, B: int, R: int, T_cap: int, device="cuda") -> 
     return torch.empty(kvc_workspace_bytes(layer, B, R, T_cap), dtype=torch.uint8, device=device)
 
 
+def kvc_layer_capsules_written(layer: Layer) -> None:
+    """Call after anything but kvc_compress* has written into a capsule store used with this layer (see kvc.h)."""
+    _check(_lib().kvc_layer_capsules_written(layer.handle), "kvc_layer_capsules_written")
+
+
 def kvc_compress(layer: Layer, K_vis, V_vis, B: int, R: int, capsules, stream=None) -> None:
     _check(_lib().kvc_compress(layer.handle, _ptr(K_vis), _ptr(V_vis), B, R, _ptr(capsules), _stream(stream)),
            "kvc_compress")

@@ -24,6 +24,9 @@ InternVL3-shaped models, which are not available offline):
     position copies the score of its nearest retained key; theta[:, idx] = I), U with orthonormal
     rows (QR of a Gaussian matrix), the query scaled by 8 (logit standard deviation about 3) and the
     text keys ~ N(0, 0.45^2) (the scale of the smoothed vision keys, so text logits are alike).
+    Both sharp recipes scale the vision and text values (by 0.4 and 0.75) so that the outputs, which
+    are close to single value rows there, stay below about 2.6 in magnitude: one bf16 step is 2^-7
+    of the magnitude, and the absolute parity bound of the bf16 path is stated for outputs of order 1.
   * retained indices: evenly spaced, idx[j] = floor(j n / m); or a sorted seeded
     random subset (irregular gathers).
 bf16 workloads are rounded to bf16 once, here, and both sides start from the
@@ -188,27 +191,33 @@ def decode_inputs(shape: Shape, m: int, seed: int, device="cpu", T: int | None =
     T_cap = T if T_cap is None else T_cap
     s = seed * 16
     idx = evenly_spaced_idx(shape.n, m) if idx is None else idx
-    q_gain, kt_gain = 1.0, 1.0
+    q_gain, kt_gain, v_gain = 1.0, 1.0, 1.0      # v_gain keeps the sharp recipes' outputs within |y| < 2.6 (one bf16 step there: 2^-7)
     if recipe == "flat":
         theta, U, mu = params(shape.H_kv, m, shape.n, shape.d, s + 5, device, dt)
     elif recipe == "peaked":
         theta, U, mu = peaked_params(shape.H_kv, m, shape.n, shape.d, s + 5, device, dt)
-        kt_gain = 3.5
+        kt_gain, v_gain = 3.5, 0.4
     elif recipe == "structured":
         theta, U, mu = structured_params(shape.H_kv, m, shape.n, shape.d, idx, s + 5, device, dt)
-        q_gain, kt_gain = 8.0, 0.45
+        q_gain, kt_gain, v_gain = 8.0, 0.45, 0.75
     else:
         raise ValueError(f"unknown recipe {recipe!r}")
+    if v_gain != 1.0:
+        mu = _scaled(mu.float(), v_gain, dt)           # the centring vector lives on the values' scale
     return dict(
         K_vis=vision_kv(shape.B, shape.H_kv, shape.R, shape.grid, shape.d, s + 0, device, dt, shape.ar1),
-        V_vis=vision_kv(shape.B, shape.H_kv, shape.R, shape.grid, shape.d, s + 1, device, dt, shape.ar1),
+        V_vis=_scaled(vision_kv(shape.B, shape.H_kv, shape.R, shape.grid, shape.d, s + 1, device, torch.float32, shape.ar1), v_gain, dt),
         K_txt=gaussian((shape.B, shape.H_kv, T_cap, shape.d), s + 2, device, dt, kt_gain),
-        V_txt=gaussian((shape.B, shape.H_kv, T_cap, shape.d), s + 3, device, dt),
+        V_txt=gaussian((shape.B, shape.H_kv, T_cap, shape.d), s + 3, device, dt, v_gain),
         q=gaussian((shape.B, shape.H_q, shape.d), s + 4, device, dt, q_gain),
         theta=theta, U=U, mu=mu,
         idx=idx,
         T=T, T_cap=T_cap,
     )
+
+
+def _scaled(x: torch.Tensor, gain: float, dtype) -> torch.Tensor:
+    return (x if gain == 1.0 else x * gain).to(dtype).contiguous()
 
 
 def shard_batch(B_total: int, rank: int, world: int) -> tuple[int, int]:

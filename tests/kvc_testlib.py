@@ -15,7 +15,8 @@ TOL = {"f32": 1e-4, "bf16": 2e-2}       # max-abs bounds per storage type (fp32 
 # Regression bounds, asserted beside the contract: the kernels sit well inside it, and a test that only checked the
 # contract could not tell a wrong block order from rounding.  bf16: the output carries one rounding (2^-9 relative) on
 # top of the roundings of the stored scores, probabilities and weights; the absolute floor covers outputs near zero.
-REG_REL = {"f32": 5e-6, "bf16": 1.0e-2}      # observed on B200: at most 3.7e-7 (fp32) and 4.7e-3 (bf16) of max|out|
+REG_REL = {"f32": 5e-6, "bf16": 1.5e-2}      # observed on B200: at most 1.5e-6 (fp32) and 9.3e-3 (bf16) of max|out|; the bf16 maximum is
+                                             # the same to four digits for two unrelated kernels: the rounding of the stored capsules sets it
 REG_ABS = {"f32": 5e-6, "bf16": 3.0e-3}
 
 

@@ -316,6 +316,37 @@ def test_two_streams_on_one_handle_with_separate_workspaces():
         tl.assert_close(tl.np64(r["out"]), want, "bf16")
 
 
+@pytest.mark.parametrize("ci,kw", tl.REDUCED_7B)
+def test_capsule_store_rewritten_by_another_kernel_between_decode_calls(ci, kw):
+    """Once a handle has decoded, later calls may read the capsule store before the stream's previous kernel has finished.
+    A store that a kernel of the caller rewrites (here: a device copy by torch, as a cache swap-in would do) must be
+    announced with kvc_layer_capsules_written; the next call then reads it late and sees the new contents."""
+    shape = tl.small(wl.CONFIGS[ci], **kw)
+    pa = tl.make_problem(shape, wl.layer_seed(ci, 3), T=50, T_cap=64, recipe="peaked")
+    pb = tl.make_problem(shape, wl.layer_seed(ci, 4), T=50, T_cap=64, recipe="peaked")
+    pb["theta"], pb["U"], pb["mu"], pb["idx"] = pa["theta"], pa["U"], pa["mu"], pa["idx"]
+    layer = tl.gpu_layer(shape, pa)
+    B, R = shape.B, shape.R
+    caps, other = kvc.alloc_capsules(layer, B, R), kvc.alloc_capsules(layer, B, R)
+    kvc.kvc_compress(layer, pb["K_vis"].cuda(), pb["V_vis"].cuda(), B, R, other)
+    kvc.kvc_compress(layer, pa["K_vis"].cuda(), pa["V_vis"].cuda(), B, R, caps)
+    ws = kvc.alloc_workspace(layer, B, R, 64)
+    out = torch.empty((B, shape.H_q, 128), dtype=torch.bfloat16, device="cuda")
+    q, Kt, Vt = pa["q"].cuda(), pa["K_txt"].cuda(), pa["V_txt"].cuda()
+    for _ in range(3):                                    # the handle has decoded: early reads are on
+        kvc.kvc_decode_attend(layer, q, caps, B, R, Kt, Vt, 50, 64, out, ws)
+    torch.cuda.synchronize()
+    tl.assert_close(tl.np64(out), tl.oracle_run(shape, pa)[2], "bf16", "before the rewrite")
+    for _ in range(5):
+        caps.copy_(other)                                 # a kernel that is not the library's writes the store ...
+        kvc.kvc_layer_capsules_written(layer)             # ... and says so
+        kvc.kvc_decode_attend(layer, q, caps, B, R, Kt, Vt, 50, 64, out, ws)
+    torch.cuda.synchronize()
+    pm = dict(pa)
+    pm["K_vis"], pm["V_vis"] = pb["K_vis"], pb["V_vis"]
+    tl.assert_close(tl.np64(out), tl.oracle_run(shape, pm)[2], "bf16", "after the rewrite")
+
+
 def test_decode_steps_with_growing_text_tail():
     """A few decode steps: the text tail grows by one row per step inside a fixed-capacity buffer."""
     shape = tl.small(wl.CONFIGS[1], B=1, H_q=2, H_kv=2, R=2, grid=8)
