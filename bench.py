@@ -633,6 +633,11 @@ def measure(shape, config_index, dev, rank, world, local, steps, warmup, profile
             "decode_contract_gbs": round(decode_gbs, 1),
             "decode_frac_of_8tbs": round(decode_gbs / NOMINAL_HBM_GBS, 4),
             "decode_frac_of_measured_peak": round(decode_gbs / peak, 4),
+            # the same with the parameter bytes (theta, U, mu of the layer: read at least once per layer call, since the
+            # parameters of all layers exceed L2) added to the contract bytes
+            "decode_full_bytes_frac_of_measured_peak": round(
+                (contract + (2 * shape.H_kv * m * shape.n + shape.H_kv * shape.d) * elem_bytes(shape)) * calls
+                / (ms_decode * 1e-3) / 1e9 / peak, 4),
             "kernels": kernels, "ms_per_step_bracketed": ms_bracketed, "roofline": roofline, "compress": compress}
 
 
@@ -711,7 +716,9 @@ def main():
                     "workload": oshape.name, "steps": 2, "warmup": 1, "value": r["value"], "unit": "tokens/s",
                     "ms_per_step": r["ms_per_step"], "us_per_layer_call": round(r["ms_per_layer_call"] * 1e3, 2),
                     "decode_frac_of_measured_peak": r["decode_frac_of_measured_peak"],
-                    "decode_frac_of_8tbs": r["decode_frac_of_8tbs"], "roofline": r["roofline"], "compress": r["compress"],
+                    "decode_frac_of_8tbs": r["decode_frac_of_8tbs"],
+                    "decode_full_bytes_frac_of_measured_peak": r["decode_full_bytes_frac_of_measured_peak"],
+                    "roofline": r["roofline"], "compress": r["compress"],
                     "kernels": r["kernels"], "config": r["config"], "clocks": r["clocks"],
                     "comparator_us": round(comp["ms_per_layer_call"] * 1e3, 2) if comp else None})
                 torch.cuda.empty_cache()
