@@ -382,9 +382,10 @@ split_expand_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_consta
         if (lane == 0) {
           const uint32_t u_u = ring_u + slot * a.e_stage_bytes;
           const uint32_t p_u = sm_u + (uint32_t)kc * 16384u;
-#pragma unroll
+#pragma unroll 1                 // rolled: this code runs once per CTA, and its first pass is paced by instruction fetch
           for (int ks = 0; ks < 4; ++ks) {
             const uint64_t adesc = umma_smem_desc(p_u + (uint32_t)(ks * 32), 16u, 1024u, UMMA_LAYOUT_SW128);
+#pragma unroll 1
             for (int bx = 0; bx < a.nbox; ++bx) {
               const uint64_t bdesc = umma_smem_desc(u_u + bx * u_box + (uint32_t)(ks * 32), 16u, 1024u, UMMA_LAYOUT_SW128);
               umma_bf16(tb + (uint32_t)(bx * a.brow), adesc, bdesc, idesc_W, (kc | ks) ? 1u : 0u);
