@@ -50,7 +50,7 @@ KERNEL_SOURCES = {
 }
 NCU_TRAFFIC_BYTES = {
     ("fused", "config1-llava-next-7b"): (208.4e6, "5e7f612f8ac6"),
-    ("split_scores+split_expand+split_output", "config2-qwen2-vl-7b"): (147.9e6, "0ca50a288632"),
+    ("split_scores+split_expand+split_output", "config2-qwen2-vl-7b"): (147.7e6, "418d58b580f9"),
     ("resident", "config3-internvl3-8b-video"): (36.0e6, "7d4a0953cecd"),
 }
 
