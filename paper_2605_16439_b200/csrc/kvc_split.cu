@@ -98,7 +98,7 @@ SplitWs split_ws(const kvc_layer* L, const SplitPlan& p, int B, int R, int T) {
   w.off_S = take(sizeof(__nv_bfloat16) * (size_t)H_kv * p.rows_h * p.ms);
   w.off_Wp = take(sizeof(__nv_bfloat16) * (size_t)H_kv * p.NS * p.rows_h * p.ms);
   w.off_stat = take(sizeof(float2) * (size_t)H_kv * p.NS * p.rows_h);
-  const size_t nslot = p.o_cpb > 1 ? (size_t)p.o_cpb : 0;
+  const size_t nslot = (size_t)p.o_cpb;          // one slot per CTA of a pair; a pair served by one CTA still parks its part there
   w.off_py = take(sizeof(float) * (size_t)B * H_kv * nslot * G * D);
   w.off_pml = take(sizeof(float2) * (size_t)B * H_kv * nslot * G);
   w.off_cnt = take(sizeof(int) * (size_t)B * H_kv);

@@ -35,7 +35,7 @@ struct SplitPlan {
   int s_stages, s_grid; size_t s_smem;
   int vt;              // 64-row tiles per block of V_tilde
   int o_stages, o_grid; uint32_t o_stage_bytes, o_w_bytes; size_t o_smem;
-  int o_cpb;              // CTAs of the output kernel per (sequence, KV head) = its partial slots (1: no partials)
+  int o_cpb;              // CTAs of the output kernel per (sequence, KV head) = its partial slots
   uint32_t o_off_q, o_off_fac, o_off_red, o_off_stat;   // behind the ring
 };
 

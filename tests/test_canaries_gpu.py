@@ -46,6 +46,8 @@ CASES = [  # B, H_q, H_kv, grid, R, T, dtype, mode
     (2, 6, 2, 8, 3, 9, "bf16", "k"),
     (2, 6, 2, 8, 3, 9, "f32", "v"),
     (2, 4, 2, 8, 2, 0, "bf16", "kv"),        # no text
+    (38, 2, 2, 32, 1, 0, "bf16", "kv"),      # three-kernel path, one CTA of the output kernel per pair, no text
+    (40, 8, 8, 16, 2, 20, "bf16", "kv"),     # resident path, more pairs than SMs
 ]
 
 

@@ -541,6 +541,22 @@ def test_a_wait_that_nothing_completes_gives_up_and_the_context_stays_usable():
     _check(shape, p)
 
 
+@pytest.mark.parametrize("B,H_q,H_kv,grid,R,T", [
+    (38, 2, 2, 32, 2, 70),        # n = 1024, 76 pairs: more than half the SMs, one CTA of the output kernel per pair
+    (80, 7, 1, 32, 1, 0),         # no text, G = 7
+    (10, 16, 8, 8, 2, 37),        # the same through the forced path on a short block (80 pairs)
+    (40, 8, 8, 8, 2, 37),         # more pairs than SMs: CTAs that walk several pairs
+])
+def test_three_kernel_path_with_one_output_cta_per_pair(B, H_q, H_kv, grid, R, T, monkeypatch):
+    """Batches with more (sequence, KV head) pairs than half the SMs: every pair is served by one CTA of the output kernel,
+    which parks its part in the workspace like the CTAs of a shared pair do."""
+    monkeypatch.setenv("KVC_EXPANSION", "split")
+    shape = wl.Shape("one-cta-per-pair", 1, B, H_q, H_kv, 128, grid, R, T, 1, "bf16")
+    p = tl.make_problem(shape, 170 + B, T=T, T_cap=T + 3, recipe="peaked")
+    counts = _fused_launches(lambda: _check(shape, p))
+    assert counts["split_output"] == 1
+
+
 def test_more_units_than_sms_and_status_word_clean():
     """Persistent CTAs walk several work units each (ring parity carried across units)."""
     shape = wl.Shape("many-units", 1, 40, 8, 8, 128, 8, 2, 37, 1, "bf16")      # 8 * 40 = 320 units of one sequence
