@@ -105,7 +105,7 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     auto region = [&](int w) { return (size_t)(ni < RS_WARPS ? ni * w / RS_WARPS : w) * nsl * RS_PIECE_BYTES; };
     unsigned char* ring_p = sm + a.off_ring + region(warp);
     const uint32_t ring_u = smem_addr(ring_p);
-    uint32_t use_cnt = 0, iss_cnt = 0;                           // pieces consumed / issued by this warp in this unit
+    uint32_t use_slot = 0, iss_slot = 0;                         // slots of the next piece consumed / issued by this warp
 
     // ---- this warp's load stream: the pieces of its items in the order it consumes them
     int p_k = wlo, p_idx = 0;
@@ -116,32 +116,30 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       const int half = vis ? np : RS_TEXT_ROWS / RS_PIECE_ROWS;
       if (!vis) dep_wait();
       if (lane == 0) {
-        const uint32_t slot = iss_cnt % (uint32_t)nsl;
-        unsigned char* dst = ring_p + slot * RS_PIECE_BYTES;
-        uint64_t* bar = &full_bar[warp][slot];
+        unsigned char* dst = ring_p + iss_slot * RS_PIECE_BYTES;
+        uint64_t* bar = &full_bar[warp][iss_slot];
         const bool second = p_idx >= half;
         const int piece = second ? p_idx - half : p_idx;
         const CUtensorMap* tm = vis ? (second ? &tmV : &tmK) : (second ? &tmVt : &tmKt);
         const int row0 = vis ? piece * RS_PIECE_ROWS : (p_k - a.R) * RS_TEXT_ROWS + piece * RS_PIECE_ROWS;
         const int idx3 = vis ? bh * a.R + p_k : bh;
         mbar_expect_tx(bar, RS_PIECE_BYTES);
-        tma_load_3d(dst, tm, 0, row0, idx3, bar);
-        tma_load_3d(dst + RS_HALF, tm, 64, row0, idx3, bar);
+        tma_load_4d(dst, tm, 0, row0, 0, idx3, bar);               // both 64-channel halves of the 16 rows in one copy
       }
-      ++iss_cnt;
+      if (++iss_slot == (uint32_t)nsl) iss_slot = 0;
       if (++p_idx == 2 * half) { p_idx = 0; ++p_k; }
     };
     auto wait_piece = [&]() -> uint32_t {
-      const uint32_t slot = use_cnt % (uint32_t)nsl, parity = (pbits >> slot) & 1u;
+      const uint32_t slot = use_slot, parity = (pbits >> slot) & 1u;
       if (!dead && !mbar_wait_bounded(&full_bar[warp][slot], parity)) dead = true;
       pbits ^= 1u << slot;
       __syncwarp();
       return ring_u + slot * RS_PIECE_BYTES;
     };
-    auto done_piece = [&]() {          // every lane has read the piece: its slot takes the next load of the stream
+    // every lane has read the piece (ldmatrix has returned its data): its slot takes the next load of the stream
+    auto done_piece = [&]() {
       __syncwarp();
-      if (lane == 0) fence_proxy_async();
-      ++use_cnt;
+      if (++use_slot == (uint32_t)nsl) use_slot = 0;
       issue_next();
     };
     for (int s = 0; s < nsl; ++s) issue_next();
@@ -167,17 +165,20 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     }
     // scores of one 16-row piece against the queries: v[0..3] = (row g, heads 2t, 2t+1), (row g + 8, heads 2t, 2t+1)
     auto score_piece = [&](uint32_t st, float (&v)[4]) {
-      float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+      float c[4][4];                                // four chains of two products each
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) c[i][e] = 0.f;
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks) {
         const int cc = 2 * ks + selA;               // 16-byte piece of the 256-byte row
         uint32_t af[4];
         ldsm_x4(af, st + (uint32_t)(cc >> 3) * RS_HALF + (uint32_t)rowA * 128u + (uint32_t)(((cc & 7) ^ (rowA & 7)) << 4));
-        if (ks & 1) mma_bf16_16816(c1, af, qb[ks][0], qb[ks][1]);
-        else mma_bf16_16816(c0, af, qb[ks][0], qb[ks][1]);
+        mma_bf16_16816(c[ks & 3], af, qb[ks][0], qb[ks][1]);
       }
 #pragma unroll
-      for (int e = 0; e < 4; ++e) v[e] = (c0[e] + c1[e]) * RS_QSCALE;
+      for (int e = 0; e < 4; ++e) v[e] = ((c[0][e] + c[1][e]) + (c[2][e] + c[3][e])) * RS_QSCALE;
     };
     // y^T += (value rows of the piece)^T times the B fragment (k = the 16 rows, n = the heads)
     auto value_piece = [&](uint32_t st, uint32_t b0, uint32_t b1) {
@@ -446,6 +447,7 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
             make_uint2(pack2_bf16(y.x * inv, y.y * inv), pack2_bf16(y.z * inv, y.w * inv));
       }
     }
+    if (lane == 0) fence_proxy_async(); // the warp's result, written to its ring with ordinary stores, precedes the copies
     __syncthreads();                    // the rings take the next unit's pieces
   }
   dep_wait();
@@ -509,19 +511,20 @@ cudaError_t launch_resident(const kvc_layer* L, const DecodeArgs& a, const Resid
   *encoded = false;
   CUtensorMap tm[6];
   {
-    // K_tilde, V_tilde as (channels, m rows of a block, blocks): rows past a block's last are zero-filled
-    const uint64_t dims[3] = {(uint64_t)D, (uint64_t)m, (uint64_t)B * H_kv * R};
-    const uint64_t str[2] = {256ull, (uint64_t)m * 256};
-    const uint32_t box[3] = {64u, (uint32_t)RS_PIECE_ROWS, 1u};
-    if (!encode_tensor_map_bf16(&tm[0], a.Kc, 3, dims, str, box)) return cudaSuccess;
-    if (!encode_tensor_map_bf16(&tm[1], a.Vc, 3, dims, str, box)) return cudaSuccess;
+    // K_tilde, V_tilde as (64 channels, m rows of a block, channel half, blocks): a box lands as [half][16 rows][64];
+    // rows past a block's last are zero-filled
+    const uint64_t dims[4] = {64ull, (uint64_t)m, 2ull, (uint64_t)B * H_kv * R};
+    const uint64_t str[3] = {256ull, 128ull, (uint64_t)m * 256};
+    const uint32_t box[4] = {64u, (uint32_t)RS_PIECE_ROWS, 2u, 1u};
+    if (!encode_tensor_map_bf16(&tm[0], a.Kc, 4, dims, str, box)) return cudaSuccess;
+    if (!encode_tensor_map_bf16(&tm[1], a.Vc, 4, dims, str, box)) return cudaSuccess;
   }
   if (a.T > 0) {
-    const uint64_t dims[3] = {(uint64_t)D, (uint64_t)a.T, (uint64_t)B * H_kv};
-    const uint64_t str[2] = {256ull, (uint64_t)a.T_cap * 256};
-    const uint32_t box[3] = {64u, (uint32_t)RS_PIECE_ROWS, 1u};
-    if (!encode_tensor_map_bf16(&tm[2], a.K_txt, 3, dims, str, box)) return cudaSuccess;
-    if (!encode_tensor_map_bf16(&tm[3], a.V_txt, 3, dims, str, box)) return cudaSuccess;
+    const uint64_t dims[4] = {64ull, (uint64_t)a.T, 2ull, (uint64_t)B * H_kv};
+    const uint64_t str[3] = {256ull, 128ull, (uint64_t)a.T_cap * 256};
+    const uint32_t box[4] = {64u, (uint32_t)RS_PIECE_ROWS, 2u, 1u};
+    if (!encode_tensor_map_bf16(&tm[2], a.K_txt, 4, dims, str, box)) return cudaSuccess;
+    if (!encode_tensor_map_bf16(&tm[3], a.V_txt, 4, dims, str, box)) return cudaSuccess;
   } else {
     tm[2] = tm[0];
     tm[3] = tm[1];
