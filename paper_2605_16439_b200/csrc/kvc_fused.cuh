@@ -66,15 +66,28 @@ __device__ __forceinline__ RowRanges row_ranges(const FusedArgs& a, int rg) {
 // the caller's workspace, which is never initialised: it packs (token of the call that last touched it, arrivals of
 // that call), so whatever an earlier call or nobody left there reads as "no arrivals yet" for a new token.  The last
 // arriver clears the word, which also keeps a replayed launch (same token) correct.  Call after __threadfence().
+// One atomic add per arrival once the word carries the call's token; only the arrivals that still find another token
+// (the first of a call, and those racing with it) take the compare-and-swap path that installs it.
 __device__ __forceinline__ bool arrive_is_last(unsigned long long* word, unsigned int token, int expected) {
-  unsigned long long seen = *reinterpret_cast<volatile unsigned long long*>(word);
+  const unsigned long long mine = (unsigned long long)token << 32;
   for (;;) {
-    const unsigned int count = (unsigned int)(seen >> 32) == token ? (unsigned int)seen : 0u;
-    const bool last = (int)count + 1 == expected;
-    const unsigned long long want = last ? 0ull : (((unsigned long long)token << 32) | (count + 1u));
-    const unsigned long long prev = atomicCAS(word, seen, want);
-    if (prev == seen) return last;
-    seen = prev;
+    const unsigned long long old = atomicAdd(word, 1ull);
+    if ((unsigned int)(old >> 32) == token) {
+      const bool last = (int)(unsigned int)old + 1 == expected;
+      if (last) *reinterpret_cast<volatile unsigned long long*>(word) = 0ull;     // every arrival of the call has been counted
+      return last;
+    }
+    // a word of another call (or never written): this add counted nothing.  Install (token, 1) unless somebody else does first
+    unsigned long long seen = old + 1ull;
+    for (;;) {
+      if ((unsigned int)(seen >> 32) == token) break;                 // installed by another arrival: count this one above
+      const unsigned long long prev = atomicCAS(word, seen, mine | 1ull);
+      if (prev == seen) {
+        if (expected == 1) *reinterpret_cast<volatile unsigned long long*>(word) = 0ull;
+        return expected == 1;
+      }
+      seen = prev;
+    }
   }
 }
 

@@ -131,7 +131,8 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     };
     auto wait_piece = [&]() -> uint32_t {
       const uint32_t slot = use_slot, parity = (pbits >> slot) & 1u;
-      if (!dead && !mbar_wait_bounded(&full_bar[warp][slot], parity)) dead = true;
+      if (!mbar_test_wait(&full_bar[warp][slot], parity))          // usually complete already: one immediate look first
+        if (!dead && !mbar_wait_bounded(&full_bar[warp][slot], parity)) dead = true;
       pbits ^= 1u << slot;
       __syncwarp();
       return ring_u + slot * RS_PIECE_BYTES;
@@ -347,6 +348,7 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
             if (nv < RS_PIECE_ROWS && lane < 16)
               for (int r = nv < 0 ? 0 : nv; r < RS_PIECE_ROWS; ++r)
                 asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};\n" ::"r"(st + (uint32_t)(lane >> 3) * RS_HALF + (uint32_t)r * 128u + (uint32_t)(lane & 7) * 16u), "r"(0u) : "memory");
+            fence_proxy_async();                   // the cleared rows precede the copy that refills the slot
             __syncwarp();
           }
           value_piece(st, Tb_frag[pc][0], Tb_frag[pc][1]);
@@ -447,7 +449,7 @@ resident_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
             make_uint2(pack2_bf16(y.x * inv, y.y * inv), pack2_bf16(y.z * inv, y.w * inv));
       }
     }
-    if (lane == 0) fence_proxy_async(); // the warp's result, written to its ring with ordinary stores, precedes the copies
+    fence_proxy_async();                // the warps' results, written to their rings with ordinary stores, precede the copies
     __syncthreads();                    // the rings take the next unit's pieces
   }
   dep_wait();
