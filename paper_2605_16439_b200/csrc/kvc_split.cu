@@ -75,7 +75,7 @@ SplitPlan plan_split(const kvc_layer* L, int B, int R) {
     uint32_t off = 0;
     auto take = [&](uint32_t bytes) { uint32_t o = off; off = (off + bytes + 127u) & ~127u; return o; };
     p.o_off_q = take(16u * (uint32_t)D * 4u);                       // summed accumulators of a pair
-    p.o_off_fac = take((uint32_t)(R * p.NS) * 16u * 8u);
+    p.o_off_fac = take((uint32_t)(R * p.NS) * (uint32_t)SO_FAC_PITCH * 8u);
     p.o_off_red = take(8u * NH * 8u * (uint32_t)D * 4u);
     p.o_off_stat = take((uint32_t)(32 + 2 * (p.o_cpb + 64) * 16) * 4u);   // up to 64 text chunks (16384 text rows)
     if (off + 2048u + 2 * p.o_stage_bytes > SP_SMEM_LIMIT) return p;

@@ -16,6 +16,7 @@
 namespace kvc {
 
 constexpr int SP_TILE_ROWS = 128;      // retained key rows per stage of the score kernel; expansion rows per expansion CTA
+constexpr int SO_FAC_PITCH = 17;     // float2 entries per (block, range) row of the output kernel's factor table
 constexpr int SP_OUT_ROWS = 64;        // value rows (and text rows) per stage of the output kernel
 constexpr int SP_MAX_STAGES = 12;
 constexpr int SP_TEXT_CHUNK = 3;       // 64-row tiles of text per CTA of the text kernel (96 KB of stages: two CTAs per SM)

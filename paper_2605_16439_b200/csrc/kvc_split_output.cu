@@ -80,7 +80,7 @@ split_output_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
   const int l7 = lane & 7, lhi = lane >> 4, lmid = (lane >> 3) & 1;
   const int lrowB = l7 + lhi * 8;                   // ldmatrix address pattern: rows 0-7 | 0-7 | 8-15 | 8-15
   const uint32_t sm_u = smem_addr(sm);
-  float2* fac = reinterpret_cast<float2*>(sm + a.o_off_fac);                     // [R*NS][16]: (factor, scaled row sum)
+  float2* fac = reinterpret_cast<float2*>(sm + a.o_off_fac);                     // [R*NS][17]: (factor, scaled row sum) per head; the odd pitch spreads a head's entries over the banks
   float* red = reinterpret_cast<float*>(sm + a.o_off_red);                       // [8 warps][NH*8][128]
   float* vbuf = reinterpret_cast<float*>(sm + a.o_off_q);                        // [16][128] value part of the pair
   float* hmax = reinterpret_cast<float*>(sm + a.o_off_stat);                     // [16] maximum over the vision logits
@@ -161,19 +161,19 @@ split_output_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
       const int e = idx >> 4, g = idx & 15, rr = e / NS, s = e - rr * NS;
       float2 v = make_float2(-INFINITY, 0.f);
       if (g < G) v = __ldcg(&a.stat[((size_t)h * NS + s) * a.rows_h + (size_t)(b * R + rr) * G + g]);
-      fac[idx] = v;
+      fac[e * SO_FAC_PITCH + g] = v;
     }
     named_barrier_sync(1, SO_CONS);
     for (int g = warp; g < 16; g += SO_WARPS) {
       float mx = -INFINITY;
-      for (int e = lane; e < ne; e += 32) mx = fmaxf(mx, fac[e * 16 + g].x);
+      for (int e = lane; e < ne; e += 32) mx = fmaxf(mx, fac[e * SO_FAC_PITCH + g].x);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
       float l = 0.f;
       for (int e = lane; e < ne; e += 32) {
-        const float2 v = fac[e * 16 + g];
+        const float2 v = fac[e * SO_FAC_PITCH + g];
         const float f = g < G ? fast_exp2(v.x - mx) : 0.f;
-        fac[e * 16 + g] = make_float2(f, f * v.y);
+        fac[e * SO_FAC_PITCH + g] = make_float2(f, f * v.y);
         l += f * v.y;
       }
 #pragma unroll
@@ -194,7 +194,7 @@ split_output_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
         wait_full();
         const uint32_t v_u = sm_u + slot * a.o_stage_bytes;
         const unsigned char* wp = sm + (size_t)slot * a.o_stage_bytes + 2 * SO_HALF;      // [NS][G][64] bf16
-        const float2* fr = fac + (size_t)r * NS * 16;
+        const float2* fr = fac + (size_t)r * NS * SO_FAC_PITCH;
         if (jt * SP_OUT_ROWS + rg * 16 < a.m) {
           // B fragments: the weights of heads gid (+8) for rows 2 t4, 2 t4 + 1 (+8) of this row group, ranges joined
           uint32_t bw[NH][2];
@@ -205,7 +205,7 @@ split_output_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
             if (g < G) {
               const unsigned char* row = wp + (size_t)g * 128 + (rg * 16 + 2 * t4) * 2;
               for (int s = 0; s < NS; ++s) {
-                const float f = fr[s * 16 + g].x;
+                const float f = fr[s * SO_FAC_PITCH + g].x;
                 const uint32_t lo = *reinterpret_cast<const uint32_t*>(row), hi = *reinterpret_cast<const uint32_t*>(row + 16);
                 row += (size_t)G * 128;
                 w0 = fmaf(f, __uint_as_float(lo << 16), w0); w1 = fmaf(f, __uint_as_float(lo & 0xffff0000u), w1);
