@@ -267,8 +267,9 @@ def test_device_side_argument_errors_and_noops():
     assert float(out.abs().sum()) == 0.0
 
 
-def test_repeat_calls_are_bitwise_deterministic_and_workspace_needs_no_init():
-    shape = tl.small(wl.CONFIGS[2], B=2, H_q=14, H_kv=2, R=2, grid=16)
+@pytest.mark.parametrize("grid,R", [(16, 2), (24, 5), (32, 3)])     # resident, one-kernel and three-kernel paths
+def test_repeat_calls_are_bitwise_deterministic_and_workspace_needs_no_init(grid, R):
+    shape = tl.small(wl.CONFIGS[2], B=2, H_q=14, H_kv=2, R=R, grid=grid)
     p = tl.make_problem(shape, 96, T=70)
     layer = tl.gpu_layer(shape, p)
     B, R = shape.B, shape.R
@@ -277,14 +278,28 @@ def test_repeat_calls_are_bitwise_deterministic_and_workspace_needs_no_init():
     ws = kvc.alloc_workspace(layer, B, R, 70)
     q, Kt, Vt = p["q"].cuda(), p["K_txt"].cuda(), p["V_txt"].cuda()
     outs = []
-    for fill in (0x00, 0xFF, 0x7F):
-        ws.fill_(fill)                               # poison: the call may not depend on old contents
-        out = torch.empty((B, shape.H_q, 128), dtype=torch.bfloat16, device="cuda")
-        kvc.kvc_decode_attend(layer, q, caps, B, R, Kt, Vt, 70, 70, out, ws)
-        outs.append(out.clone())
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    for fill in (0x00, 0xFF, 0x7F, 0x01, "bytes", "counts"):
+        # poison: the call may not depend on old contents (the arrival words of split pairs live there: all-ones, small
+        # integers that look like counts of arrivals, random bytes)
+        if fill == "bytes":
+            ws.copy_(torch.randint(0, 256, ws.shape, dtype=torch.uint8, device="cuda", generator=gen))
+        elif fill == "counts":
+            ws.fill_(0)
+            w64 = ws[: ws.numel() // 8 * 8].view(torch.int64)
+            w64.copy_(torch.randint(0, 20, w64.shape, dtype=torch.int64, device="cuda", generator=gen))
+        else:
+            ws.fill_(fill)
+        for _ in range(2):                           # and not on what the call before left there
+            out = torch.empty((B, shape.H_q, 128), dtype=torch.bfloat16, device="cuda")
+            kvc.kvc_decode_attend(layer, q, caps, B, R, Kt, Vt, 70, 70, out, ws)
+            outs.append(out.clone())
     torch.cuda.synchronize()
-    assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16))
-    assert torch.equal(outs[0].view(torch.int16), outs[2].view(torch.int16))
+    assert kvc.kvc_read_device_status(layer, B, R, 70, ws) == 0
+    for o in outs[1:]:
+        assert torch.equal(outs[0].view(torch.int16), o.view(torch.int16))
+    _, _, out_o = tl.oracle_run(shape, p)
+    tl.assert_close(tl.np64(outs[0]), out_o, "bf16", "decode on a poisoned workspace")
 
 
 def test_two_streams_on_one_handle_with_separate_workspaces():
