@@ -27,68 +27,84 @@ struct ExpandBars {
 // Plain attention of the decode query over K_txt / V_txt (Sec. 3.2: the text K/V stay uncompressed and join the softmax
 // of the reconstructed vision positions), flash-style, as partials: the CTAs behind the expansion CTAs of the grid each
 // take a run of (sequence, KV head, chunk of up to 192 text rows) items and leave (max, sum, y) per head and item in
-// the workspace; the output kernel merges them with the vision part.  Warps 0-3 = 16 rows of every 64-row tile each,
-// warp 9 = producer (one stage per tile of a chunk, refilled for the next chunk as soon as its tile has been read).
+// the workspace; the output kernel merges them with the vision part.  An item is a chain of round trips (queries, three
+// tiles, the warps' states meeting in shared memory, the partial's store), so a CTA runs NG of them side by side: group g =
+// warps 4g..4g+3 (16 rows of every 64-row tile each) with its own stages, barriers and producer thread (lane 0 of warp
+// 9 - g; one stage per tile of a chunk, refilled for the next chunk as soon as its tile has been read), taking every NG-th
+// item of the CTA's run.
 constexpr uint32_t ST_HALF = SP_OUT_ROWS * 128;       // 64 rows x 64 channels
 constexpr uint32_t ST_STAGE = 4 * ST_HALF;            // K and V rows of a tile
 constexpr int ST_WARPS = 4;
 constexpr int ST_CONS = ST_WARPS * 32;
 
+constexpr uint32_t SP_SMEM_LIMIT_EXPAND = 232448;      // shared memory of a CTA, static part included
+constexpr int ST_STAT = 2 * ST_WARPS * 16 + 16;       // floats of a group's statistics: maxima [4][16], sums [4][16], maximum [16]
+// a group's shared memory: its stages and the four warps' parked accumulators [G heads][128]; two groups fit up to G = 7
+__host__ __device__ constexpr uint32_t st_group_bytes(int G) { return ((uint32_t)SP_TEXT_CHUNK * ST_STAGE + (uint32_t)ST_WARPS * G * D * 4 + 1023u) & ~1023u; }
+__host__ __device__ constexpr int st_groups(int G) { return 2u * st_group_bytes(G) + 1024u + 4096u <= SP_SMEM_LIMIT_EXPAND ? 2 : 1; }
+
 template <int NH>
-__device__ __forceinline__ void text_role(const CUtensorMap& tmKt, const CUtensorMap& tmVt, const SplitArgs& a, unsigned char* sm,
-                                          ExpandBars& bars, float* tmax /*[4*16]*/, float* tsum /*[4*16]*/, float* txm /*[16]*/) {
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+__device__ __forceinline__ void text_role(const CUtensorMap& tmKt, const CUtensorMap& tmVt, const SplitArgs& a, unsigned char* sm_cta,
+                                          ExpandBars& bars, float* stat_cta /*[NG][ST_STAT]*/) {
+  const int NG = st_groups(a.G);
+  const int tid_cta = threadIdx.x, warp_cta = tid_cta >> 5, lane = tid_cta & 31;
   const int G = a.G;
   const int tt = (a.T + SP_OUT_ROWS - 1) / SP_OUT_ROWS;
   const int nct = (tt + SP_TEXT_CHUNK - 1) / SP_TEXT_CHUNK;
   const long long items = (long long)a.B * a.H_kv * nct;
   const int j = (int)blockIdx.x - a.e_grid;
   const int i0 = (int)(items * j / a.tx_grid), i1 = (int)(items * (j + 1) / a.tx_grid);
-  if (tid == 0) {
-    for (int s = 0; s < SP_TEXT_CHUNK; ++s) { mbar_init(&bars.full[s], 1); mbar_init(&bars.empty[s], ST_WARPS); }
+  if (tid_cta == 0) {
+    for (int s = 0; s < NG * SP_TEXT_CHUNK; ++s) { mbar_init(&bars.full[s], 1); mbar_init(&bars.empty[s], ST_WARPS); }
     fence_mbar_init();
   }
   __syncthreads();
   grid_dep_launch();
-  if (warp == 9) {
+  // group of this warp: consumers 4g..4g+3, producer 9 - g
+  const int grp = warp_cta >= 10 - NG ? 9 - warp_cta : warp_cta / ST_WARPS;
+  if (grp >= NG) return;
+  unsigned char* sm = sm_cta + (size_t)grp * st_group_bytes(a.G);
+  uint64_t* full = bars.full + grp * SP_TEXT_CHUNK;
+  uint64_t* empty = bars.empty + grp * SP_TEXT_CHUNK;
+  float* tmax = stat_cta + grp * ST_STAT, *tsum = tmax + ST_WARPS * 16, *txm = tsum + ST_WARPS * 16;
+  if (warp_cta >= 10 - NG) {
     if (lane == 0) {
       tma_prefetch_desc(&tmKt); tma_prefetch_desc(&tmVt);
       uint32_t phase = 1;
-      for (int it = i0; it < i1; ++it, phase ^= 1u) {
+      for (int it = i0 + grp; it < i1; it += NG, phase ^= 1u) {
         const int bh = it / nct, ci = it - bh * nct;
         const int b = bh / a.H_kv, h = bh - b * a.H_kv;
         const int t0 = ci * SP_TEXT_CHUNK, t1 = min(tt, t0 + SP_TEXT_CHUNK);
         for (int tile = t0; tile < t1; ++tile) {
           const int s = tile - t0;
-          if (!mbar_wait_bounded(&bars.empty[s], phase)) { atomicExch(a.status, (int)KVC_ERR_TIMEOUT); return; }
+          if (!mbar_wait_bounded(&empty[s], phase)) { atomicExch(a.status, (int)KVC_ERR_TIMEOUT); return; }
           unsigned char* dst = sm + (uint32_t)s * ST_STAGE;
-          mbar_expect_tx(&bars.full[s], ST_STAGE);
+          mbar_expect_tx(&full[s], ST_STAGE);
           const int y = tile * SP_OUT_ROWS;
-          tma_load_4d(dst, &tmKt, 0, y, h, b, &bars.full[s]);
-          tma_load_4d(dst + ST_HALF, &tmKt, 64, y, h, b, &bars.full[s]);
-          tma_load_4d(dst + 2 * ST_HALF, &tmVt, 0, y, h, b, &bars.full[s]);
-          tma_load_4d(dst + 3 * ST_HALF, &tmVt, 64, y, h, b, &bars.full[s]);
+          tma_load_4d(dst, &tmKt, 0, y, h, b, &full[s]);
+          tma_load_4d(dst + ST_HALF, &tmKt, 64, y, h, b, &full[s]);
+          tma_load_4d(dst + 2 * ST_HALF, &tmVt, 0, y, h, b, &full[s]);
+          tma_load_4d(dst + 3 * ST_HALF, &tmVt, 64, y, h, b, &full[s]);
         }
         // a stage the chunk does not use still turns its barriers once, so that every stage is in the same round
         for (int s = t1 - t0; s < SP_TEXT_CHUNK; ++s) {
-          if (!mbar_wait_bounded(&bars.empty[s], phase)) { atomicExch(a.status, (int)KVC_ERR_TIMEOUT); return; }
-          mbar_expect_tx(&bars.full[s], 0);
+          if (!mbar_wait_bounded(&empty[s], phase)) { atomicExch(a.status, (int)KVC_ERR_TIMEOUT); return; }
+          mbar_expect_tx(&full[s], 0);
         }
       }
     }
     return;
   }
-  if (warp >= ST_WARPS) return;
-
+  const int warp = warp_cta - grp * ST_WARPS, tid = tid_cta - grp * ST_CONS;     // within the group
   const int rg = warp;                              // the 16-row group of a tile this warp takes
   const int gid = lane >> 2, t4 = lane & 3;
   const int l7 = lane & 7, lhi = lane >> 4, lmid = (lane >> 3) & 1;
   const int lrowB = l7 + lhi * 8;                   // ldmatrix address pattern: rows 0-7 | 0-7 | 8-15 | 8-15
   const uint32_t sm_u = smem_addr(sm);
-  float* red = reinterpret_cast<float*>(sm + SP_TEXT_CHUNK * ST_STAGE);          // [4 warps][NH*8][128]
+  float* red = reinterpret_cast<float*>(sm + SP_TEXT_CHUNK * ST_STAGE);          // [4 warps][G][128]
   bool dead = false;
   uint32_t phase = 0;
-  for (int it = i0; it < i1; ++it, phase ^= 1u) {
+  for (int it = i0 + grp; it < i1; it += NG, phase ^= 1u) {
     const int bh = it / nct, ci = it - bh * nct;
     const int b = bh / a.H_kv, h = bh - b * a.H_kv;
     const int t0 = ci * SP_TEXT_CHUNK, t1 = min(tt, t0 + SP_TEXT_CHUNK);
@@ -115,7 +131,7 @@ __device__ __forceinline__ void text_role(const CUtensorMap& tmKt, const CUtenso
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // heads gid and gid + 8
     for (int s = 0; s < SP_TEXT_CHUNK; ++s) {
       const int tile = t0 + s;
-      if (!dead && !mbar_wait_bounded(&bars.full[s], phase)) dead = true;
+      if (!dead && !mbar_wait_bounded(&full[s], phase)) dead = true;
       __syncwarp();
       if (tile < t1) {
         const uint32_t kt_u = sm_u + (uint32_t)s * ST_STAGE, vt_u = kt_u + 2 * ST_HALF;
@@ -199,11 +215,11 @@ __device__ __forceinline__ void text_role(const CUtensorMap& tmKt, const CUtenso
           }
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(&bars.empty[s]);
+      if (lane == 0) mbar_arrive(&empty[s]);
     }
     // the per-warp online-softmax states meet at one maximum per head
     if (t4 == 0) { tmax[warp * 16 + gid] = m_run[0]; tmax[warp * 16 + gid + 8] = m_run[1]; }
-    named_barrier_sync(1, ST_CONS);
+    named_barrier_sync(1 + grp, ST_CONS);
     {
       float scl[2];
 #pragma unroll
@@ -231,26 +247,29 @@ __device__ __forceinline__ void text_role(const CUtensorMap& tmKt, const CUtenso
       }
     }
     {
-      float* mine = red + (size_t)warp * (NH * 8 * D);
+      float* mine = red + (size_t)warp * (G * D);
 #pragma unroll
       for (int nh = 0; nh < NH; ++nh)
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
-          float* yp = mine + (nh * 8 + 2 * t4 + e) * D;
+          const int head = nh * 8 + 2 * t4 + e;
+          if (head < G) {
+            float* yp = mine + head * D;
 #pragma unroll
-          for (int mt = 0; mt < 8; ++mt) {
-            yp[mt * 16 + gid] = yacc[mt][nh][e];
-            yp[mt * 16 + gid + 8] = yacc[mt][nh][2 + e];
+            for (int mt = 0; mt < 8; ++mt) {
+              yp[mt * 16 + gid] = yacc[mt][nh][e];
+              yp[mt * 16 + gid + 8] = yacc[mt][nh][2 + e];
+            }
           }
         }
     }
-    named_barrier_sync(1, ST_CONS);
+    named_barrier_sync(1 + grp, ST_CONS);
     const size_t pbase = ((size_t)bh * nct + ci) * G;
     for (int idx = tid; idx < G * D; idx += ST_CONS) {
       const float* rp = red + idx;
       float y = 0.f;
 #pragma unroll
-      for (int w = 0; w < ST_WARPS; ++w) y += rp[(size_t)w * (NH * 8 * D)];
+      for (int w = 0; w < ST_WARPS; ++w) y += rp[(size_t)w * (G * D)];
       a.tpy[pbase * D + idx] = dead ? 0.f : y;
     }
     if (tid < G) {
@@ -259,7 +278,7 @@ __device__ __forceinline__ void text_role(const CUtensorMap& tmKt, const CUtenso
       for (int w = 0; w < ST_WARPS; ++w) l += tsum[w * 16 + tid];
       a.tpml[pbase + tid] = make_float2(txm[tid], l);
     }
-    named_barrier_sync(1, ST_CONS);                 // red and the statistics are free for the next item
+    named_barrier_sync(1 + grp, ST_CONS);                 // red and the statistics are free for the next item
   }
   if (dead && lane == 0) atomicExch(a.status, (int)KVC_ERR_TIMEOUT);
 }
@@ -273,11 +292,11 @@ split_expand_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_consta
   unsigned char* sm = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
   __shared__ __align__(8) ExpandBars bars;
   __shared__ uint32_t s_tmem;
-  __shared__ float s_tstat[2 * ST_WARPS * 16 + 16];
+  __shared__ float s_tstat[2 * ST_STAT];
   __shared__ float s_rstat[512];                  // row maxima and row sums of the two column halves
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if ((int)blockIdx.x >= a.e_grid) {             // a text CTA (it uses no tensor memory)
-    text_role<NH>(tmKt, tmVt, a, sm, bars, s_tstat, s_tstat + ST_WARPS * 16, s_tstat + 2 * ST_WARPS * 16);
+    text_role<NH>(tmKt, tmVt, a, sm, bars, s_tstat);
     return;
   }
 
@@ -548,7 +567,7 @@ static cudaError_t launch_expand_inst(const CUtensorMap* tm, const SplitArgs& a,
 // tm: S, theta, U, partial weights (store), K_txt, V_txt
 cudaError_t launch_split_expand(const CUtensorMap* tm, const SplitArgs& a, const SplitPlan& p, cudaStream_t st) {
   // a text CTA needs its stages and the reduction buffer of its four warps
-  const size_t text_smem = (size_t)SP_TEXT_CHUNK * ST_STAGE + (size_t)ST_WARPS * (a.G > 8 ? 2 : 1) * 8 * D * 4 + 1024;
+  const size_t text_smem = (size_t)st_groups(a.G) * st_group_bytes(a.G) + 1024;
   const size_t smem = a.tx_grid > 0 && text_smem > p.e_smem ? text_smem : p.e_smem;
   ProfScope prof(KVC_KERNEL_SPLIT_EXPAND, st);
   return a.G > 8 ? launch_expand_inst<2>(tm, a, smem, st) : launch_expand_inst<1>(tm, a, smem, st);
