@@ -116,11 +116,12 @@ cudaError_t launch_split(const kvc_layer* L, const DecodeArgs& a, const SplitPla
   const SplitWs w = split_ws(L, p, B, R, a.T);
   CUtensorMap tmK, tmS, tmTh, tmU, tmWs, tmO[4];
   {
-    // K_tilde as (channels, R m rows of a pair, pairs): rows past the pair's last are zero-filled, not read
-    const uint64_t dims[3] = {(uint64_t)D, (uint64_t)R * m, (uint64_t)B * H_kv};
-    const uint64_t str[2] = {256ull, (uint64_t)R * m * 256};
-    const uint32_t box[3] = {64u, (uint32_t)SP_TILE_ROWS, 1u};
-    if (!encode_tensor_map_bf16(&tmK, a.Kc, 3, dims, str, box)) return cudaSuccess;
+    // K_tilde as (64 channels, R m rows of a pair, channel half, pairs): a box lands as [half][128 rows][64]; rows past the
+    // pair's last are zero-filled, not read
+    const uint64_t dims[4] = {64ull, (uint64_t)R * m, 2ull, (uint64_t)B * H_kv};
+    const uint64_t str[3] = {256ull, 128ull, (uint64_t)R * m * 256};
+    const uint32_t box[4] = {64u, (uint32_t)SP_TILE_ROWS, 2u, 1u};
+    if (!encode_tensor_map_bf16(&tmK, a.Kc, 4, dims, str, box)) return cudaSuccess;
   }
   {
     const uint64_t dims[3] = {(uint64_t)m, (uint64_t)p.rows_h, (uint64_t)H_kv};
@@ -142,17 +143,19 @@ cudaError_t launch_split(const kvc_layer* L, const DecodeArgs& a, const SplitPla
     if (!encode_tensor_map_bf16(&tmU, a.U, 3, dims, str, box)) return cudaSuccess;
   }
   {
-    const uint64_t dims[5] = {(uint64_t)D, (uint64_t)m, (uint64_t)R, (uint64_t)H_kv, (uint64_t)B};
-    const uint64_t str[4] = {256ull, (uint64_t)m * 256, (uint64_t)R * m * 256, (uint64_t)H_kv * R * m * 256};
-    const uint32_t box[5] = {64u, (uint32_t)SP_OUT_ROWS, 1u, 1u, 1u};
-    if (!encode_tensor_map_bf16(&tmO[0], a.Vc, 5, dims, str, box)) return cudaSuccess;
+    // V_tilde as (64 channels, m rows of a block, channel half, blocks of all pairs): a box lands as [half][64 rows][64]
+    const uint64_t dims[4] = {64ull, (uint64_t)m, 2ull, (uint64_t)B * H_kv * R};
+    const uint64_t str[3] = {256ull, 128ull, (uint64_t)m * 256};
+    const uint32_t box[4] = {64u, (uint32_t)SP_OUT_ROWS, 2u, 1u};
+    if (!encode_tensor_map_bf16(&tmO[0], a.Vc, 4, dims, str, box)) return cudaSuccess;
   }
   if (a.T > 0) {
-    const uint64_t dims[4] = {(uint64_t)D, (uint64_t)a.T, (uint64_t)H_kv, (uint64_t)B};
-    const uint64_t str[3] = {256ull, (uint64_t)a.T_cap * 256, (uint64_t)H_kv * a.T_cap * 256};
-    const uint32_t box[4] = {64u, (uint32_t)SP_OUT_ROWS, 1u, 1u};
-    if (!encode_tensor_map_bf16(&tmO[1], a.K_txt, 4, dims, str, box)) return cudaSuccess;
-    if (!encode_tensor_map_bf16(&tmO[2], a.V_txt, 4, dims, str, box)) return cudaSuccess;
+    // the text rows as (64 channels, T rows, channel half, H_kv, B): a box lands as [half][64 rows][64]
+    const uint64_t dims[5] = {64ull, (uint64_t)a.T, 2ull, (uint64_t)H_kv, (uint64_t)B};
+    const uint64_t str[4] = {256ull, 128ull, (uint64_t)a.T_cap * 256, (uint64_t)H_kv * a.T_cap * 256};
+    const uint32_t box[5] = {64u, (uint32_t)SP_OUT_ROWS, 2u, 1u, 1u};
+    if (!encode_tensor_map_bf16(&tmO[1], a.K_txt, 5, dims, str, box)) return cudaSuccess;
+    if (!encode_tensor_map_bf16(&tmO[2], a.V_txt, 5, dims, str, box)) return cudaSuccess;
   } else {
     tmO[1] = tmO[0];
     tmO[2] = tmO[0];

@@ -81,10 +81,8 @@ __device__ __forceinline__ void text_role(const CUtensorMap& tmKt, const CUtenso
           unsigned char* dst = sm + (uint32_t)s * ST_STAGE;
           mbar_expect_tx(&full[s], ST_STAGE);
           const int y = tile * SP_OUT_ROWS;
-          tma_load_4d(dst, &tmKt, 0, y, h, b, &full[s]);
-          tma_load_4d(dst + ST_HALF, &tmKt, 64, y, h, b, &full[s]);
-          tma_load_4d(dst + 2 * ST_HALF, &tmVt, 0, y, h, b, &full[s]);
-          tma_load_4d(dst + 3 * ST_HALF, &tmVt, 64, y, h, b, &full[s]);
+          tma_load_5d(dst, &tmKt, 0, y, 0, h, b, &full[s]);                    // both 64-channel halves per copy
+          tma_load_5d(dst + 2 * ST_HALF, &tmVt, 0, y, 0, h, b, &full[s]);
         }
         // a stage the chunk does not use still turns its barriers once, so that every stage is in the same round
         for (int s = t1 - t0; s < SP_TEXT_CHUNK; ++s) {

@@ -59,15 +59,15 @@ split_output_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
     for (int bh = bh_first; bh < BH; bh += bh_step) {
       const int b = bh / a.H_kv, h = bh - b * a.H_kv;
       if (!waited) { grid_dep_wait(); waited = true; }     // the partial weights come from the expansion kernel
+      int r = v0 / vt, jt = v0 - r * vt;
       for (int rem = v0; rem < v1; ++rem) {
-        const int r = rem / vt, jt = rem - r * vt;
         if (!mbar_wait_bounded(&empty_bar[slot], phase)) { atomicExch(a.status, (int)KVC_ERR_TIMEOUT); return; }
         unsigned char* dst = sm + slot * a.o_stage_bytes;
         mbar_expect_tx(&full_bar[slot], 2 * SO_HALF + w_bytes);
-        tma_load_5d(dst, &tmV, 0, jt * SP_OUT_ROWS, r, h, b, &full_bar[slot]);
-        tma_load_5d(dst + SO_HALF, &tmV, 64, jt * SP_OUT_ROWS, r, h, b, &full_bar[slot]);
+        tma_load_4d(dst, &tmV, 0, jt * SP_OUT_ROWS, 0, bh * R + r, &full_bar[slot]);      // both 64-channel halves in one copy
         tma_load_4d(dst + 2 * SO_HALF, &tmW, jt * SP_OUT_ROWS, (b * R + r) * G, 0, h, &full_bar[slot]);
         if (++slot == (uint32_t)nst) { slot = 0; phase ^= 1u; }
+        if (++jt == vt) { jt = 0; ++r; }
       }
     }
     return;
@@ -283,22 +283,17 @@ split_output_kernel(const __grid_constant__ CUtensorMap tmV, const __grid_consta
           return reinterpret_cast<const float4*>(p < cpb ? a.py + (p0 + (size_t)p * G + g) * D + col
                                                          : a.tpy + (q0 + (size_t)(p - cpb) * G + g) * D + col);
         };
-        int p = 0;
-        for (; p + 8 <= np; p += 8) {
+        // eight partials' loads in flight at a time, the last group predicated (a pair has 2 + 3 partials at config 2: one
+        // round trip instead of three)
+        for (int p = 0; p < np; p += 8) {
           float4 y[8];
 #pragma unroll
-          for (int x = 0; x < 8; ++x) y[x] = __ldcg(src(p + x));
+          for (int x = 0; x < 8; ++x)
+            if (p + x < np) y[x] = __ldcg(src(p + x));
 #pragma unroll
-          for (int x = 0; x < 8; ++x) acc4(y[x], mlm[(p + x) * 16 + g]);
+          for (int x = 0; x < 8; ++x)
+            if (p + x < np) acc4(y[x], mlm[(p + x) * 16 + g]);
         }
-        for (; p + 2 <= np; p += 2) {
-          float4 y[2];
-#pragma unroll
-          for (int x = 0; x < 2; ++x) y[x] = __ldcg(src(p + x));
-#pragma unroll
-          for (int x = 0; x < 2; ++x) acc4(y[x], mlm[(p + x) * 16 + g]);
-        }
-        for (; p < np; ++p) acc4(__ldcg(src(p)), mlm[p * 16 + g]);
         uint2 o;
         o.x = pack2_bf16(num.x, num.y); o.y = pack2_bf16(num.z, num.w);
         *reinterpret_cast<uint2*>(a.out + ((size_t)b * a.H_kv * G + (size_t)h * G + g) * D + col) = o;

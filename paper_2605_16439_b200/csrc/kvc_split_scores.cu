@@ -41,8 +41,7 @@ split_scores_kernel(const __grid_constant__ CUtensorMap tmK, const SplitArgs a) 
       // data, so it need not wait for that kernel; the loads below do)
       int pbh = (int)(lo / a.s_tiles_bh), pt = (int)(lo - (long long)pbh * a.s_tiles_bh);
       for (int k = 0; k < nst && lo + k < hi; ++k) {
-        tma_prefetch_l2_3d(&tmK, 0, pt * SP_TILE_ROWS, pbh);
-        tma_prefetch_l2_3d(&tmK, 64, pt * SP_TILE_ROWS, pbh);
+        tma_prefetch_l2_4d(&tmK, 0, pt * SP_TILE_ROWS, 0, pbh);
         if (++pt == a.s_tiles_bh) { pt = 0; ++pbh; }
       }
     }
@@ -54,8 +53,7 @@ split_scores_kernel(const __grid_constant__ CUtensorMap tmK, const SplitArgs a) 
       if (!mbar_wait_bounded(&empty_bar[slot], phase)) { atomicExch(a.status, (int)KVC_ERR_TIMEOUT); return; }
       unsigned char* dst = sm + slot * SS_STAGE;
       mbar_expect_tx(&full_bar[slot], SS_STAGE);
-      tma_load_3d(dst, &tmK, 0, t * SP_TILE_ROWS, bh, &full_bar[slot]);
-      tma_load_3d(dst + SS_HALF, &tmK, 64, t * SP_TILE_ROWS, bh, &full_bar[slot]);
+      tma_load_4d(dst, &tmK, 0, t * SP_TILE_ROWS, 0, bh, &full_bar[slot]);      // both 64-channel halves in one copy
       if (++slot == (uint32_t)nst) { slot = 0; phase ^= 1u; }
     }
     return;
