@@ -49,9 +49,9 @@ KERNEL_SOURCES = {
                                                "kvc_tcgen05.cuh", "kvc_tma.cuh", "kvc_async.cuh"),
 }
 NCU_TRAFFIC_BYTES = {
-    ("fused", "config1-llava-next-7b"): (208.4e6, "b7cf5a7916bc"),
-    ("split_scores+split_expand+split_output", "config2-qwen2-vl-7b"): (147.7e6, "6c3d0d64f511"),
-    ("resident", "config3-internvl3-8b-video"): (36.0e6, "fdd07f544779"),
+    ("fused", "config1-llava-next-7b"): (208.4e6, "3788d05ac9fe"),
+    ("split_scores+split_expand+split_output", "config2-qwen2-vl-7b"): (147.7e6, "847534a6df3c"),
+    ("resident", "config3-internvl3-8b-video"): (36.0e6, "1e4ede360c43"),
 }
 
 
