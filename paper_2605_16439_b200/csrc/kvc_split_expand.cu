@@ -321,6 +321,10 @@ split_expand_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_consta
   tc_fence_after();
   const uint32_t tb = s_tmem;
   const uint32_t th_bytes = (uint32_t)ngrp * 8192u;    // theta rows of a chunk: [group][64 rows][128 B]
+  // The CTAs of a (KV head, range) walk the same theta and U chunks; each starts at another chunk (its row tile's number),
+  // so that they do not all ask the L2 slice that holds a line for it at the same moment.  The sums run over the same terms.
+  auto chunk1 = [&](int i) { const int k = i + tile % a.nk1; return k < a.nk1 ? k : k - a.nk1; };
+  auto chunk2 = [&](int i) { const int k = i + tile % ngrp; return k < ngrp ? k : k - ngrp; };
   const uint32_t u_box = (uint32_t)a.brow * 128u;
 
   if (warp == 9) {
@@ -332,17 +336,19 @@ split_expand_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_consta
       // the first ring of stages: theta rows (parameters, never written by the library) before the dependency wait,
       // the scores of the kernel before after it
       const int npre = a.nk1 < a.e_stages ? a.nk1 : a.e_stages;
-      for (int kc = 0; kc < npre; ++kc) {
-        unsigned char* dst = ring + kc * a.e_stage_bytes;
-        mbar_expect_tx(&bars.full[kc], 16384u + th_bytes);
-        tma_load_4d(dst + 16384, &tmTh, 0, kc * 64, n0 >> 6, h, &bars.full[kc]);
+      for (int i = 0; i < npre; ++i) {
+        const int kc = chunk1(i);
+        unsigned char* dst = ring + i * a.e_stage_bytes;
+        mbar_expect_tx(&bars.full[i], 16384u + th_bytes);
+        tma_load_4d(dst + 16384, &tmTh, 0, kc * 64, n0 >> 6, h, &bars.full[i]);
       }
       grid_dep_wait();
       grid_dep_launch();                      // only now: the output kernel relies on the score kernel being complete
-      for (int kc = 0; kc < npre; ++kc) tma_load_3d(ring + kc * a.e_stage_bytes, &tmS, kc * 64, tile * SP_TILE_ROWS, h, &bars.full[kc]);
+      for (int i = 0; i < npre; ++i) tma_load_3d(ring + i * a.e_stage_bytes, &tmS, chunk1(i) * 64, tile * SP_TILE_ROWS, h, &bars.full[i]);
       slot = (uint32_t)npre;
       if (slot == (uint32_t)a.e_stages) { slot = 0; phase ^= 1u; }
-      for (int kc = npre; kc < a.nk1 && ok; ++kc) {
+      for (int i = npre; i < a.nk1 && ok; ++i) {
+        const int kc = chunk1(i);
         if (!mbar_wait_bounded(&bars.empty[slot], phase)) { ok = false; break; }
         unsigned char* dst = ring + slot * a.e_stage_bytes;
         mbar_expect_tx(&bars.full[slot], 16384u + th_bytes);
@@ -351,7 +357,8 @@ split_expand_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_consta
         if (++slot == (uint32_t)a.e_stages) { slot = 0; phase ^= 1u; }
       }
       for (int wp = 0; wp < a.npass && ok; ++wp)
-        for (int kc = 0; kc < ngrp && ok; ++kc) {
+        for (int i = 0; i < ngrp && ok; ++i) {
+          const int kc = chunk2(i);
           if (!mbar_wait_bounded(&bars.empty[slot], phase)) { ok = false; break; }
           unsigned char* dst = ring + slot * a.e_stage_bytes;
           mbar_expect_tx(&bars.full[slot], (uint32_t)a.nbox * u_box);
@@ -372,7 +379,8 @@ split_expand_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_consta
       if (!dead && !mbar_wait_bounded(bar, parity)) dead = true;
       __syncwarp();
     };
-    for (int kc = 0; kc < a.nk1; ++kc) {
+    for (int i = 0; i < a.nk1; ++i) {
+      const int kc = chunk1(i);
       wait_on(&bars.full[slot], phase);
       tc_fence_after();
       if (lane == 0) {
@@ -381,10 +389,10 @@ split_expand_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_consta
         for (int ks = 0; ks < ksteps; ++ks) {
           const uint64_t adesc = umma_smem_desc(s_u + (uint32_t)(ks * 32), 16u, 1024u, UMMA_LAYOUT_SW128);
           const uint64_t bdesc = umma_smem_desc(th_u + (uint32_t)(ks * 2048), 8192u, 1024u, UMMA_LAYOUT_SW128);
-          umma_bf16(tb, adesc, bdesc, idesc_L, (kc | ks) ? 1u : 0u);
+          umma_bf16(tb, adesc, bdesc, idesc_L, (i | ks) ? 1u : 0u);
         }
         umma_commit(&bars.empty[slot]);
-        if (kc == a.nk1 - 1) umma_commit(&bars.l_done);
+        if (i == a.nk1 - 1) umma_commit(&bars.l_done);
       }
       __syncwarp();
       if (++slot == (uint32_t)a.e_stages) { slot = 0; phase ^= 1u; }
@@ -393,7 +401,8 @@ split_expand_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_consta
     for (int wp = 0; wp < a.npass; ++wp) {
       if (wp > 0) wait_on(&bars.w_free, (uint32_t)((wp - 1) & 1));
       tc_fence_after();
-      for (int kc = 0; kc < ngrp; ++kc) {
+      for (int i = 0; i < ngrp; ++i) {
+        const int kc = chunk2(i);
         wait_on(&bars.full[slot], phase);
         tc_fence_after();
         if (lane == 0) {
@@ -405,11 +414,11 @@ split_expand_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_consta
 #pragma unroll 1
             for (int bx = 0; bx < a.nbox; ++bx) {
               const uint64_t bdesc = umma_smem_desc(u_u + bx * u_box + (uint32_t)(ks * 32), 16u, 1024u, UMMA_LAYOUT_SW128);
-              umma_bf16(tb + (uint32_t)(bx * a.brow), adesc, bdesc, idesc_W, (kc | ks) ? 1u : 0u);
+              umma_bf16(tb + (uint32_t)(bx * a.brow), adesc, bdesc, idesc_W, (i | ks) ? 1u : 0u);
             }
           }
           umma_commit(&bars.empty[slot]);
-          if (kc == ngrp - 1) umma_commit(&bars.w_done);
+          if (i == ngrp - 1) umma_commit(&bars.w_done);
         }
         __syncwarp();
         if (++slot == (uint32_t)a.e_stages) { slot = 0; phase ^= 1u; }
