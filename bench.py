@@ -50,7 +50,7 @@ KERNEL_SOURCES = {
 }
 NCU_TRAFFIC_BYTES = {
     ("fused", "config1-llava-next-7b"): (208.4e6, "3788d05ac9fe"),
-    ("split_scores+split_expand+split_output", "config2-qwen2-vl-7b"): (147.7e6, "847534a6df3c"),
+    ("split_scores+split_expand+split_output", "config2-qwen2-vl-7b"): (147.7e6, "b9ec0383c83b"),
     ("resident", "config3-internvl3-8b-video"): (36.0e6, "1e4ede360c43"),
 }
 
