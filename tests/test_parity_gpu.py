@@ -572,6 +572,19 @@ def test_three_kernel_path_with_one_output_cta_per_pair(B, H_q, H_kv, grid, R, T
     assert counts["split_output"] == 1
 
 
+@pytest.mark.parametrize("T", [1, 63, 64, 65, 191, 192, 193, 385, 600])
+@pytest.mark.parametrize("H_q,H_kv", [(2, 2), (8, 2), (7, 1), (8, 1), (12, 1)])
+def test_three_kernel_path_text_lengths_and_group_sizes(H_q, H_kv, T, monkeypatch):
+    """The text rows of the three-kernel path: chunks of 192 rows dealt to text CTAs that run one or two of them side by side
+    (two up to seven query heads per KV head, one above), around the tile and chunk boundaries and with fewer chunks
+    than text CTAs."""
+    monkeypatch.setenv("KVC_EXPANSION", "split")
+    shape = wl.Shape("text-groups", 1, 3, H_q, H_kv, 128, 8, 2, T, 1, "bf16")
+    p = tl.make_problem(shape, 300 + T + H_q, T=T, T_cap=T + 5, recipe="peaked")
+    counts = _fused_launches(lambda: _check(shape, p))
+    assert counts["split_expand"] == 1
+
+
 def test_more_units_than_sms_and_status_word_clean():
     """Persistent CTAs walk several work units each (ring parity carried across units)."""
     shape = wl.Shape("many-units", 1, 40, 8, 8, 128, 8, 2, 37, 1, "bf16")      # 8 * 40 = 320 units of one sequence
