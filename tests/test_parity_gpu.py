@@ -585,6 +585,16 @@ def test_three_kernel_path_text_lengths_and_group_sizes(H_q, H_kv, T, monkeypatc
     assert counts["split_expand"] == 1
 
 
+def test_text_tail_longer_than_the_three_kernel_path_takes():
+    """n = 1024 with more than 12288 text rows: the three-kernel path does not apply (its output kernel keeps a weight per
+    text partial in shared memory) and the call falls back to a one-kernel variant."""
+    T = 12300
+    shape = wl.Shape("long-text", 1, 1, 2, 1, 128, 32, 1, T, 1, "bf16")
+    p = tl.make_problem(shape, 77, T=T, T_cap=T + 4)
+    counts = _fused_launches(lambda: _check(shape, p))
+    assert counts["split_expand"] == 0 and counts["fused"] + counts["fused_tc"] + counts["fused_pair"] >= 1
+
+
 def test_more_units_than_sms_and_status_word_clean():
     """Persistent CTAs walk several work units each (ring parity carried across units)."""
     shape = wl.Shape("many-units", 1, 40, 8, 8, 128, 8, 2, 37, 1, "bf16")      # 8 * 40 = 320 units of one sequence
