@@ -28,6 +28,11 @@ WsLayout ws_layout(const kvc_layer* L, int B, int R, int T_cap) {
   if (w.use_mma) {
     w.CG = ceil_div(ms, 256);
     w.cgw = (int)align_up((size_t)ceil_div(ms, w.CG), 16);
+    // the kernel keeps a 64-row score tile and a chunk of theta over all retained positions in shared memory: past about 720
+    // of them (n = 1024 at ratios below 0.3) that no longer fits, and the fp32 expansion takes over
+    if (expand_mma_smem_bytes(ms, w.cgw) > 227u * 1024u) { w.use_mma = 0; w.CG = 1; w.cgw = ms; }
+  }
+  if (w.use_mma) {
     row_tiles = ceil_div(rows_h, 64) * H_kv * w.CG;
   } else {
     row_tiles = ceil_div(rows_h, EXP_ROWS) * H_kv;

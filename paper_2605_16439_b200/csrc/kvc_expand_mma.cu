@@ -212,9 +212,13 @@ __global__ void __launch_bounds__(128) expand_mma_kernel(DecodeArgs a) {
   }
 }
 
+size_t expand_mma_smem_bytes(int ms, int cgw) {
+  return sizeof(__nv_bfloat16) * ((size_t)XM_ROWS * (ms + 8) + (size_t)ms * XM_LD + (size_t)cgw * XM_LD);
+}
+
 template <int NT_W>
 static cudaError_t launch_nt(const DecodeArgs& a, cudaStream_t st) {
-  const size_t smem = sizeof(__nv_bfloat16) * ((size_t)XM_ROWS * (a.ms + 8) + (size_t)a.ms * XM_LD + (size_t)a.ws.cgw * XM_LD);
+  const size_t smem = expand_mma_smem_bytes(a.ms, a.ws.cgw);
   {
     cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(expand_mma_kernel<NT_W>), smem);
     if (e != cudaSuccess) return e;

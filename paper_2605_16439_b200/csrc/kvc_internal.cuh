@@ -234,6 +234,8 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 // launchers (each returns a cudaError_t from the launch)
 cudaError_t launch_scores(const DecodeArgs& a, int dtype, cudaStream_t st);
 cudaError_t launch_expand(const DecodeArgs& a, int dtype, cudaStream_t st);
+// dynamic shared memory of the tensor-core expansion kernel for rows of `ms` retained positions cut into column groups of `cgw`
+size_t expand_mma_smem_bytes(int ms, int cgw);
 cudaError_t launch_expand_mma(const DecodeArgs& a, cudaStream_t st);
 cudaError_t launch_output(const DecodeArgs& a, int dtype, cudaStream_t st);
 // one-kernel path; *encoded == false (and nothing launched) if the tensor maps could not be built

@@ -595,6 +595,17 @@ def test_text_tail_longer_than_the_three_kernel_path_takes():
     assert counts["split_expand"] == 0 and counts["fused"] + counts["fused_tc"] + counts["fused_pair"] >= 1
 
 
+@pytest.mark.parametrize("ratio", [200, 290, 300])
+def test_three_phase_path_with_more_retained_rows_than_its_tensor_core_expansion_holds(ratio, monkeypatch):
+    """n = 1024 at low ratios (m = 820, 728, 717): the tensor-core expansion of the three-phase path keeps all retained positions of
+    a 64-row score tile in shared memory, which fits up to about 720; beyond that the fp32 expansion serves the call (ragged
+    calls and KVC_EXPANSION=phases reach this path on long blocks)."""
+    monkeypatch.setenv("KVC_EXPANSION", "phases")
+    shape = wl.Shape("long-m", 1, 2, 4, 2, 128, 32, 1, 20, 1, "bf16", ratio)
+    p = tl.make_problem(shape, 410 + ratio, T=20, T_cap=24, recipe="peaked")
+    _check(shape, p)
+
+
 def test_more_units_than_sms_and_status_word_clean():
     """Persistent CTAs walk several work units each (ring parity carried across units)."""
     shape = wl.Shape("many-units", 1, 40, 8, 8, 128, 8, 2, 37, 1, "bf16")      # 8 * 40 = 320 units of one sequence
